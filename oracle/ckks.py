@@ -1,0 +1,421 @@
+"""CPU oracle for the RNS-CKKS linear hot path (TEST INFRASTRUCTURE, fp64 / exact integers).
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this
+module; the product path never does, and this module imports nothing from the
+CUDA package.  It composes the C primitives of oracle/fesc_oracle.c into the
+operations the library exports, in the order the definitions state them:
+
+  * encode / decode / encrypt / decrypt (harness side; the paper's client holds
+    the secret key, Sec. 3 threat model),
+  * ct-pt multiply-accumulate  (Table "CKKS primitives": ptmul, add),
+  * rotation / conjugation = Galois automorphism then hybrid key switch
+    (Table "CKKS primitives": rot, conj; rho(v; r)_j = v_{(j+r) mod n}),
+  * rescale, ct x ct with relinearisation (ctmul),
+  * the BSGS plaintext-weight projection Y = XW (App. "Projection Kernel
+    Breakdown": packing idx(r,c) = c*T + r, accumulators c_p, giant-step fold).
+
+The paper uses its CKKS backend as a black box, so the internals follow the
+standard hybrid (dnum) key switching with the readings listed in the design
+notes: canonical residues, uncorrected fast basis conversion, ROUNDED division
+by P (key switch) and by the dropped prime (rescale).
+
+Layouts: a polynomial on k limbs is a uint64 array [k, N]; a ciphertext at
+level l is [2, l, N] (c0 then c1), evaluation form, bit-reversed order.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+
+import numpy as np
+
+from . import build as _build
+
+_lib = ctypes.CDLL(_build.build())
+_u64p = np.ctypeslib.ndpointer(dtype=np.uint64, flags="C_CONTIGUOUS")
+_i64p = np.ctypeslib.ndpointer(dtype=np.int64, flags="C_CONTIGUOUS")
+_c = ctypes
+_lib.orc_powmod.restype = _c.c_uint64
+_lib.orc_powmod.argtypes = [_c.c_uint64] * 3
+_lib.orc_min_psi.restype = _c.c_uint64
+_lib.orc_min_psi.argtypes = [_c.c_uint64, _c.c_uint32]
+_lib.orc_draw.restype = _c.c_uint64
+_lib.orc_draw.argtypes = [_c.c_uint64] * 3
+_lib.orc_ntt.argtypes = [_u64p, _u64p, _c.c_uint32, _c.c_uint32]
+_lib.orc_intt.argtypes = [_u64p, _u64p, _c.c_uint32, _c.c_uint32]
+_lib.orc_ntt_direct.argtypes = [_u64p, _u64p, _c.c_uint64, _c.c_uint32]
+for _n in ("orc_mul", "orc_muladd", "orc_add", "orc_sub", "orc_mul_scalar", "orc_add_scalar"):
+    getattr(_lib, _n).argtypes = [_u64p, _u64p, _u64p, _u64p, _c.c_uint32, _c.c_uint64]
+_lib.orc_autom_coeff.argtypes = [_u64p, _u64p, _u64p, _c.c_uint32, _c.c_uint32, _c.c_uint64]
+_lib.orc_autom_eval.argtypes = [_u64p, _u64p, _c.c_uint32, _c.c_uint32, _c.c_uint64]
+_lib.orc_fast_conv.argtypes = [_u64p, _u64p, _c.c_uint32, _u64p, _c.c_uint32, _u64p, _c.c_uint64, _c.c_int]
+_lib.orc_sample_uniform.argtypes = [_c.c_uint64, _c.c_uint64, _c.c_uint64, _u64p, _c.c_uint64]
+_lib.orc_sample_ternary.argtypes = [_c.c_uint64, _c.c_uint64, _i64p, _c.c_uint64]
+_lib.orc_sample_cbd.argtypes = [_c.c_uint64, _c.c_uint64, _i64p, _c.c_uint64]
+_lib.orc_signed_to_rns.argtypes = [_i64p, _u64p, _u64p, _c.c_uint32, _c.c_uint64]
+
+# domains of the counter-based generator
+DOM_SECRET, DOM_EVK_A, DOM_EVK_E, DOM_ENC_A, DOM_ENC_E = 1, 2, 3, 4, 5
+RELIN_KEY_ID = 0          # key id reserved for the relinearisation key
+CONJ = -(1 << 31)         # "rotation amount" that selects complex conjugation
+
+
+def make_tag(domain: int, key_id: int = 0, digit: int = 0, limb: int = 0) -> int:
+    return domain | (key_id << 8) | (digit << 40) | (limb << 48)
+
+
+def _arr(x) -> np.ndarray:
+    return np.ascontiguousarray(x, dtype=np.uint64)
+
+
+class Oracle:
+    """RNS-CKKS context: `n_q` data primes then `n_p` special primes (all = 1 mod 2N)."""
+
+    def __init__(self, log_n: int, primes, n_q: int, n_p: int, dnum: int, seed: int):
+        assert len(primes) == n_q + n_p and n_p >= 1 and dnum >= 1
+        self.log_n, self.N, self.n = log_n, 1 << log_n, 1 << (log_n - 1)
+        self.q = [int(p) for p in primes]
+        self.n_q, self.K = n_q, n_p
+        self.alpha = -(-n_q // dnum)
+        self.beta_max = -(-n_q // self.alpha)
+        self.seed = seed
+        self.special = list(range(n_q, n_q + n_p))
+        self.P = math.prod(self.q[i] for i in self.special)
+        for p in self.q:
+            assert _lib.orc_min_psi(p, log_n) != 0, "prime is not NTT friendly"
+        # secret key: ternary coefficients from the seed, kept in EVAL form on every limb
+        s = np.empty(self.N, dtype=np.int64)
+        _lib.orc_sample_ternary(seed, make_tag(DOM_SECRET), s, self.N)
+        self.s_coeff = s
+        allidx = list(range(n_q + n_p))
+        self.s_eval = self.ntt(self.signed_to_rns(s, allidx), allidx)
+        self.keys: dict[int, tuple[int, np.ndarray]] = {}
+        s2 = self.mul(self.s_eval, self.s_eval, allidx)
+        self.keys[RELIN_KEY_ID] = (0, self._gen_evk(RELIN_KEY_ID, s2))
+
+    # ---- limb-wise primitives ------------------------------------------------
+    def _q(self, idx) -> np.ndarray:
+        return np.array([self.q[i] for i in idx], dtype=np.uint64)
+
+    def ntt(self, a, idx):
+        a = _arr(a).copy().reshape(len(idx), self.N)
+        _lib.orc_ntt(a, self._q(idx), len(idx), self.log_n)
+        return a
+
+    def intt(self, a, idx):
+        a = _arr(a).copy().reshape(len(idx), self.N)
+        _lib.orc_intt(a, self._q(idx), len(idx), self.log_n)
+        return a
+
+    def _bin(self, fn, a, b, idx):
+        a, b = _arr(a), _arr(b)
+        out = np.empty_like(a)
+        fn(a, b, out, self._q(idx), len(idx), a.size // len(idx))
+        return out
+
+    def mul(self, a, b, idx):
+        return self._bin(_lib.orc_mul, a, b, idx)
+
+    def add(self, a, b, idx):
+        return self._bin(_lib.orc_add, a, b, idx)
+
+    def sub(self, a, b, idx):
+        return self._bin(_lib.orc_sub, a, b, idx)
+
+    def mul_scalar(self, a, scalars, idx):
+        c = np.array([int(s) % self.q[i] for s, i in zip(scalars, idx)], dtype=np.uint64)
+        return self._bin(_lib.orc_mul_scalar, a, c, idx)
+
+    def add_scalar(self, a, scalars, idx):
+        c = np.array([int(s) % self.q[i] for s, i in zip(scalars, idx)], dtype=np.uint64)
+        return self._bin(_lib.orc_add_scalar, a, c, idx)
+
+    def neg(self, a, idx):
+        return self.sub(np.zeros_like(_arr(a)), a, idx)
+
+    def signed_to_rns(self, v, idx):
+        v = np.ascontiguousarray(v, dtype=np.int64)
+        out = np.empty((len(idx), v.size), dtype=np.uint64)
+        _lib.orc_signed_to_rns(v, out, self._q(idx), len(idx), v.size)
+        return out
+
+    def fast_conv(self, a, src_idx, dst_idx, centred: bool = False):
+        a = _arr(a).reshape(len(src_idx), -1)
+        out = np.empty((len(dst_idx), a.shape[1]), dtype=np.uint64)
+        _lib.orc_fast_conv(a, self._q(src_idx), len(src_idx), self._q(dst_idx), len(dst_idx), out,
+                           a.shape[1], int(centred))
+        return out
+
+    # ---- Galois maps ---------------------------------------------------------
+    def galois_element(self, r: int) -> int:
+        """g with sigma_g = rho(.; r) (cyclic LEFT shift by r slots), or conjugation."""
+        if r == CONJ:
+            return 2 * self.N - 1
+        return pow(5, r % self.n, 2 * self.N)
+
+    def automorphism(self, a, g: int, k: int):
+        a = _arr(a).reshape(k, self.N)
+        out = np.empty_like(a)
+        _lib.orc_autom_eval(a, out, k, self.log_n, g)
+        return out
+
+    def automorphism_coeff(self, a, g: int, idx):
+        a = _arr(a).reshape(len(idx), self.N)
+        out = np.empty_like(a)
+        _lib.orc_autom_coeff(a, out, self._q(idx), len(idx), self.log_n, g)
+        return out
+
+    # ---- keys ------------------------------------------------------------------
+    def digit_limbs(self, j: int, level: int):
+        return list(range(j * self.alpha, min((j + 1) * self.alpha, level)))
+
+    def _gen_evk(self, key_id: int, s_prime_eval):
+        """Switching key from s' to s: for digit j and every modulus t (data and special),
+        a_j uniform (drawn in EVAL form), e_j centred binomial,
+        b_j = -a_j s + e_j + [t in digit j] (P mod q_t) s'.   Shape [beta, 2, n_q+K, N]."""
+        allidx = list(range(self.n_q + self.K))
+        evk = np.empty((self.beta_max, 2, len(allidx), self.N), dtype=np.uint64)
+        for j in range(self.beta_max):
+            a = np.empty((len(allidx), self.N), dtype=np.uint64)
+            for t in allidx:
+                _lib.orc_sample_uniform(self.seed, make_tag(DOM_EVK_A, key_id, j, t), self.q[t], a[t], self.N)
+            e = np.empty(self.N, dtype=np.int64)
+            _lib.orc_sample_cbd(self.seed, make_tag(DOM_EVK_E, key_id, j), e, self.N)
+            e_eval = self.ntt(self.signed_to_rns(e, allidx), allidx)
+            b = self.add(self.neg(self.mul(a, self.s_eval, allidx), allidx), e_eval, allidx)
+            dj = self.digit_limbs(j, self.n_q)
+            b[dj] = self.add(b[dj], self.mul_scalar(s_prime_eval[dj], [self.P] * len(dj), dj), dj)
+            evk[j, 0], evk[j, 1] = b, a
+        return evk
+
+    def add_galois_key(self, r: int, key_id: int):
+        assert key_id != RELIN_KEY_ID
+        g = self.galois_element(r)
+        allidx = list(range(self.n_q + self.K))
+        self.keys[key_id] = (g, self._gen_evk(key_id, self.automorphism(self.s_eval, g, len(allidx))))
+
+    # ---- hybrid key switch -----------------------------------------------------
+    def mod_up_digit(self, d_coeff, d_eval, j: int, level: int):
+        """Digit j of d extended to all level+K moduli, EVAL form."""
+        ext = list(range(level)) + self.special
+        D = self.digit_limbs(j, level)
+        others = [t for t in ext if t not in D]
+        conv = self.ntt(self.fast_conv(d_coeff[D], D, others), others)
+        out = np.empty((len(ext), self.N), dtype=np.uint64)
+        for pos, t in enumerate(ext):
+            out[pos] = d_eval[t] if t in D else conv[others.index(t)]
+        return out
+
+    def mod_down(self, c_ext, level: int):
+        """Division by P with centred remainder: [level+K, N] EVAL -> [level, N] EVAL.
+        c_i = (c'_i - Conv_i([c']_P)) * P^-1 mod q_i, Conv = centred fast conversion of the
+        special-limb residues (COEFF form) to q_i.  Equals round(c'/P) + e, |e| <= K/2,
+        e = 0 when K = 1."""
+        data = list(range(level))
+        r = self.intt(c_ext[level:], self.special)
+        u = self.ntt(self.fast_conv(r, self.special, data, centred=True), data)
+        pinv = [pow(self.P, -1, self.q[i]) for i in data]
+        return self.mul_scalar(self.sub(c_ext[:level], u, data), pinv, data)
+
+    def key_switch_raw(self, d_eval, key_id: int, level: int):
+        """Steps 1-4: returns the two accumulators on level+K moduli before division by P."""
+        evk = self.keys[key_id][1]
+        data = list(range(level))
+        ext = data + self.special
+        d_eval = _arr(d_eval).reshape(level, self.N)
+        d_coeff = self.intt(d_eval, data)
+        acc = np.zeros((2, len(ext), self.N), dtype=np.uint64)
+        for j in range(-(-level // self.alpha)):
+            dt = self.mod_up_digit(d_coeff, d_eval, j, level)
+            for p in range(2):
+                _lib.orc_muladd(dt, _arr(evk[j, p][ext]), acc[p], self._q(ext), len(ext), self.N)
+        return acc
+
+    def key_switch(self, d_eval, key_id: int, level: int):
+        acc = self.key_switch_raw(d_eval, key_id, level)
+        return np.stack([self.mod_down(acc[0], level), self.mod_down(acc[1], level)])
+
+    # ---- ciphertext operations ---------------------------------------------------
+    def ct_pt_mac(self, ct, pt, acc):
+        """acc_p += c_p (.) pt for p in {0,1}; returns the new accumulator."""
+        level = ct.shape[1]
+        data = list(range(level))
+        out = _arr(acc).copy()
+        for p in range(2):
+            _lib.orc_muladd(_arr(ct[p]), _arr(pt), out[p], self._q(data), level, self.N)
+        return out
+
+    def ct_add(self, a, b):
+        level = a.shape[1]
+        data = list(range(level))
+        return np.stack([self.add(a[p], b[p], data) for p in range(2)])
+
+    def rotate(self, ct, key_id: int):
+        """Automorphism FIRST, then key switch of the permuted c1:
+        (c0, c1) -> (sigma_g c0 + ks_0, ks_1)."""
+        level = ct.shape[1]
+        g = self.keys[key_id][0]
+        data = list(range(level))
+        c0 = self.automorphism(ct[0], g, level)
+        d = self.automorphism(ct[1], g, level)
+        ks = self.key_switch(d, key_id, level)
+        return np.stack([self.add(c0, ks[0], data), ks[1]])
+
+    def rescale(self, ct):
+        """Rounded division by the last prime, level l -> l-1:
+        c_i <- (c_i - [c_last]_centred) * q_last^-1 mod q_i  (= round(c / q_last) exactly)."""
+        level = ct.shape[1]
+        last = level - 1
+        rest = list(range(last))
+        ql = self.q[last]
+        out = np.empty((2, last, self.N), dtype=np.uint64)
+        qinv = [pow(ql, -1, self.q[i]) for i in rest]
+        for p in range(2):
+            r = self.intt(ct[p, last:last + 1], [last])            # COEFF, modulo q_last
+            u = self.ntt(self.fast_conv(r, [last], rest, centred=True), rest)
+            out[p] = self.mul_scalar(self.sub(ct[p, :last], u, rest), qinv, rest)
+        return out
+
+    def ct_ct_mul(self, a, b):
+        """(d0, d1, d2) = (a0 b0, a0 b1 + a1 b0, a1 b1); result (d0 + ks_0, d1 + ks_1) with
+        ks = KeySwitch(d2, relinearisation key).  No rescale."""
+        level = a.shape[1]
+        data = list(range(level))
+        d0 = self.mul(a[0], b[0], data)
+        d1 = self.add(self.mul(a[0], b[1], data), self.mul(a[1], b[0], data), data)
+        d2 = self.mul(a[1], b[1], data)
+        ks = self.key_switch(d2, RELIN_KEY_ID, level)
+        return np.stack([self.add(d0, ks[0], data), self.add(d1, ks[1], data)])
+
+    def mul_monomial_half(self, ct):
+        """Multiply both polynomials by X^(N/2) (every slot times i; exact)."""
+        level = ct.shape[1]
+        data = list(range(level))
+        mono = np.zeros(self.N, dtype=np.int64)
+        mono[self.N // 2] = 1
+        m_eval = self.ntt(self.signed_to_rns(mono, data), data)
+        return np.stack([self.mul(ct[p], m_eval, data) for p in range(2)])
+
+    # ---- BSGS projection -----------------------------------------------------------
+    def linear(self, ct_in, diags, desc, baby_key_ids, giant_key_ids):
+        """Y = XW on packed ciphertexts (App. "Projection Kernel Breakdown", real packing).
+
+        ct_in  [token_blocks, in_blocks, 2, l, N]
+        diags  [out_blocks, n2, in_blocks, n1, l, N]  plaintext diagonals D^(b)_{g,p,q}
+        returns [token_blocks, out_blocks, 2, l-1, N]:
+          acc_p = sum_g sum_q rot(x^(g), q*T) (.) D^(b)_{g,p,q};
+          y^(b) = sum_p rot(acc_p, p*n1*T);  then rescale.
+        baby_key_ids[q] rotates by q*T (q >= 1), giant_key_ids[p] by p*n1*T (p >= 1)."""
+        n1, n2 = desc["n1"], desc["n2"]
+        tbs, gin = ct_in.shape[0], ct_in.shape[1]
+        level = ct_in.shape[3]
+        nout = diags.shape[0]
+        out = np.empty((tbs, nout, 2, level - 1, self.N), dtype=np.uint64)
+        for tb in range(tbs):
+            rot = [[ct_in[tb, g] if q == 0 else self.rotate(ct_in[tb, g], baby_key_ids[q])
+                    for q in range(n1)] for g in range(gin)]
+            for b in range(nout):
+                y = None
+                for p in range(n2):
+                    acc = np.zeros((2, level, self.N), dtype=np.uint64)
+                    for g in range(gin):
+                        for q in range(n1):
+                            acc = self.ct_pt_mac(rot[g][q], diags[b, p, g, q], acc)
+                    if p > 0:
+                        acc = self.rotate(acc, giant_key_ids[p])
+                    y = acc if y is None else self.ct_add(y, acc)
+                out[tb, b] = self.rescale(y)
+        return out
+
+    # ---- harness: encode / decode / encrypt / decrypt ---------------------------------
+    def _slot_index(self):
+        idx = np.empty(self.n, dtype=np.int64)
+        g = 1
+        for j in range(self.n):
+            idx[j] = (g - 1) // 2
+            g = g * 5 % (2 * self.N)
+        return idx
+
+    def encode_coeffs(self, z, scale: float) -> np.ndarray:
+        """Integer coefficients round(scale * m_i) of the real polynomial m with
+        m(zeta^(5^j)) = z_j, zeta = exp(i pi / N); float64 with exact rint."""
+        z = np.asarray(z, dtype=np.complex128)
+        N = self.N
+        vals = np.zeros(N, dtype=np.complex128)
+        idx = self._slot_index()
+        vals[idx] = z
+        vals[N - 1 - idx] = np.conj(z)          # exponent 2N - 5^j  <->  index N-1-(5^j-1)/2
+        twist = np.exp(-1j * np.pi * np.arange(N) / N)
+        m = np.real(np.fft.fft(vals) * twist) / N
+        return np.rint(m * scale).astype(np.int64)
+
+    def encode(self, z, scale: float, level: int) -> np.ndarray:
+        data = list(range(level))
+        return self.ntt(self.signed_to_rns(self.encode_coeffs(z, scale), data), data)
+
+    def decode_coeffs(self, m) -> np.ndarray:
+        """Slots of a real-coefficient polynomial given as float64 coefficients."""
+        N = self.N
+        twist = np.exp(1j * np.pi * np.arange(N) / N)
+        vals = np.fft.ifft(np.asarray(m, dtype=np.float64) * twist) * N
+        return vals[self._slot_index()]
+
+    def encrypt(self, pt_eval, nonce: int) -> np.ndarray:
+        """Symmetric encryption: c1 = a uniform (EVAL), c0 = -a s + e + m."""
+        level = pt_eval.shape[0]
+        data = list(range(level))
+        a = np.empty((level, self.N), dtype=np.uint64)
+        for t in data:
+            _lib.orc_sample_uniform(self.seed, make_tag(DOM_ENC_A, nonce, 0, t), self.q[t], a[t], self.N)
+        e = np.empty(self.N, dtype=np.int64)
+        _lib.orc_sample_cbd(self.seed, make_tag(DOM_ENC_E, nonce), e, self.N)
+        e_eval = self.ntt(self.signed_to_rns(e, data), data)
+        c0 = self.add(self.add(self.neg(self.mul(a, self.s_eval[:level], data), data), e_eval, data), pt_eval, data)
+        return np.stack([c0, a])
+
+    def decrypt_coeffs(self, ct, use_limbs: int | None = None):
+        """Centred integer coefficients of c0 + c1 s, CRT-lifted from the first `use_limbs` limbs."""
+        level = ct.shape[1]
+        k = min(level, use_limbs or level)
+        data = list(range(k))
+        m = self.add(_arr(ct[0, :k]), self.mul(_arr(ct[1, :k]), self.s_eval[:k], data), data)
+        m = self.intt(m, data)
+        return crt_lift_centered(m, [self.q[i] for i in data])
+
+    def decrypt(self, ct, scale: float, use_limbs: int | None = None) -> np.ndarray:
+        coeffs = self.decrypt_coeffs(ct, use_limbs)
+        return self.decode_coeffs(np.array([float(c) for c in coeffs]) / scale)
+
+
+def crt_lift_centered(res, moduli):
+    """Residues [k, n] -> list of n Python ints in (-Q/2, Q/2]."""
+    Q = math.prod(moduli)
+    n = res.shape[1]
+    acc = np.zeros(n, dtype=object)
+    for i, q in enumerate(moduli):
+        Qi = Q // q
+        c = Qi * pow(Qi, -1, q)
+        acc = acc + res[i].astype(object) * c
+    acc = acc % Q
+    return [int(v) - Q if int(v) > Q // 2 else int(v) for v in acc]
+
+
+def pack_linear_input(x_block, T: int, C: int, n: int) -> np.ndarray:
+    """Slots idx(r,c) = c*T + r hold X[r, c] for one (token block, input block)."""
+    v = np.zeros(n)
+    rows, cols = x_block.shape
+    for c in range(cols):
+        v[c * T:c * T + rows] = x_block[:, c]
+    return v
+
+
+def linear_diagonal(W, b: int, g: int, p: int, q: int, T: int, C: int, n1: int) -> np.ndarray:
+    """D^(b)_{g,p,q}[idx(r,c)] = W[gC + (c+q) mod C, bC + (c - p*n1) mod C], zero outside W."""
+    d_in, d_out = W.shape
+    c = np.arange(C)
+    rows = g * C + (c + q) % C
+    cols = b * C + (c - p * n1) % C
+    ok = (rows < d_in) & (cols < d_out)
+    vals = np.zeros(C)
+    vals[ok] = W[rows[ok], cols[ok]]
+    return np.repeat(vals, T)
