@@ -1,0 +1,159 @@
+"""Thin Python binding of the sm_100a RNS-CKKS library (argument marshalling only).
+
+Every function below forwards to the C-ABI entry point of the same name in
+libfesc_b200.so (declared in include/fesc.h); all arithmetic runs in the CUDA kernels.
+Tensors are torch CUDA tensors of dtype int64 (bit pattern = the uint64 residue); the
+binding passes their data pointers and the current torch stream.  There is no CPU
+fallback: importing succeeds without the library, but the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfesc_b200.so")
+
+OK, EINVAL, ENOMEM, ECUDA, ELEVEL, ENOKEY, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
+CONJ = -(1 << 31)
+RELIN_KEY_ID = 0
+
+_lib = None
+
+
+class FescError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"fesc error {code}: {msg}")
+        self.code = code
+
+
+class BsgsDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint32) for n in
+                ("n1", "n2", "in_blocks", "out_blocks", "token_blocks", "n_limbs", "baby_key_base", "giant_key_base")]
+
+
+def lib():
+    """Load libfesc_b200.so (built by paper_2608_17442_b200.build); raise if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2608_17442_b200.build` "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        c = ctypes
+        vp, u32, u64, i32, sz = c.c_void_p, c.c_uint32, c.c_uint64, c.c_int32, c.c_size_t
+        sig = {
+            "fesc_ctx_create": [c.POINTER(vp), u32, c.POINTER(u64), u32, u32, u32, u64],
+            "fesc_ctx_destroy": [vp],
+            "fesc_sync": [vp, vp],
+            "fesc_ctx_add_galois_key": [vp, i32, u32],
+            "fesc_ctx_export_key": [vp, u32, vp, vp],
+            "fesc_ctx_export_secret": [vp, vp, vp],
+            "fesc_ctx_counters": [vp, c.POINTER(u64)],
+            "fesc_ntt": [vp, vp, u32, u32, u32, vp],
+            "fesc_intt": [vp, vp, u32, u32, u32, vp],
+            "fesc_ct_pt_mac": [vp, vp, vp, sz, vp, u32, u32, vp],
+            "fesc_rotate": [vp, vp, vp, u32, u32, u32, vp],
+            "fesc_rescale": [vp, vp, vp, u32, u32, vp],
+            "fesc_ct_ct_mul": [vp, vp, vp, vp, u32, u32, vp],
+            "fesc_linear": [vp, vp, vp, c.POINTER(BsgsDesc), vp, vp],
+        }
+        for name, args in sig.items():
+            f = getattr(L, name)
+            f.argtypes = args
+            f.restype = c.c_int
+        L.fesc_last_error.argtypes = [vp]
+        L.fesc_last_error.restype = c.c_char_p
+        L.fesc_ctx_num_digits.argtypes = [vp]
+        L.fesc_ctx_num_digits.restype = u32
+        _lib = L
+    return _lib
+
+
+def _stream():
+    import torch
+
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t):
+    assert t.is_cuda and t.is_contiguous() and t.element_size() == 8
+    return ctypes.c_void_p(t.data_ptr())
+
+
+class Context:
+    """Owner of a fesc_ctx handle; methods mirror the C entry points."""
+
+    def __init__(self, log_n: int, primes, n_q: int, n_p: int, dnum: int, seed: int):
+        self.log_n, self.N = log_n, 1 << log_n
+        self.n_q, self.n_p, self.dnum, self.seed = n_q, n_p, dnum, seed
+        self.primes = [int(p) for p in primes]
+        arr = (ctypes.c_uint64 * len(self.primes))(*self.primes)
+        h = ctypes.c_void_p()
+        rc = lib().fesc_ctx_create(ctypes.byref(h), log_n, arr, n_q, n_p, dnum, seed)
+        if rc != OK:
+            raise FescError(rc, "fesc_ctx_create failed")
+        self.h = h
+
+    def _chk(self, rc: int):
+        if rc != OK:
+            raise FescError(rc, lib().fesc_last_error(self.h).decode())
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib().fesc_ctx_destroy(self.h)
+            self.h = None
+
+    __del__ = close
+
+    def sync(self):
+        self._chk(lib().fesc_sync(self.h, _stream()))
+
+    @property
+    def num_digits(self) -> int:
+        return lib().fesc_ctx_num_digits(self.h)
+
+    def counters(self):
+        out = (ctypes.c_uint64 * 4)()
+        self._chk(lib().fesc_ctx_counters(self.h, out))
+        return list(out)
+
+    def add_galois_key(self, rot: int, key_id: int):
+        self._chk(lib().fesc_ctx_add_galois_key(self.h, rot, key_id))
+
+    def export_key(self, key_id: int):
+        import torch
+
+        out = torch.empty((self.num_digits, 2, self.n_q + self.n_p, self.N), dtype=torch.int64, device="cuda")
+        self._chk(lib().fesc_ctx_export_key(self.h, key_id, _ptr(out), _stream()))
+        return out
+
+    def export_secret(self):
+        import torch
+
+        out = torch.empty((self.n_q + self.n_p, self.N), dtype=torch.int64, device="cuda")
+        self._chk(lib().fesc_ctx_export_secret(self.h, _ptr(out), _stream()))
+        return out
+
+    def ntt(self, data, batch: int, first_limb: int, n_limbs: int):
+        self._chk(lib().fesc_ntt(self.h, _ptr(data), batch, first_limb, n_limbs, _stream()))
+
+    def intt(self, data, batch: int, first_limb: int, n_limbs: int):
+        self._chk(lib().fesc_intt(self.h, _ptr(data), batch, first_limb, n_limbs, _stream()))
+
+    def ct_pt_mac(self, ct, pt, acc, batch: int, n_limbs: int, pt_stride=None):
+        if pt_stride is None:
+            pt_stride = n_limbs * self.N
+        self._chk(lib().fesc_ct_pt_mac(self.h, _ptr(ct), _ptr(pt), pt_stride, _ptr(acc), batch, n_limbs, _stream()))
+
+    def rotate(self, ct_in, ct_out, batch: int, n_limbs: int, key_id: int):
+        self._chk(lib().fesc_rotate(self.h, _ptr(ct_in), _ptr(ct_out), batch, n_limbs, key_id, _stream()))
+
+    def rescale(self, ct_in, ct_out, batch: int, n_limbs: int):
+        self._chk(lib().fesc_rescale(self.h, _ptr(ct_in), _ptr(ct_out), batch, n_limbs, _stream()))
+
+    def ct_ct_mul(self, a, b, out, batch: int, n_limbs: int):
+        self._chk(lib().fesc_ct_ct_mul(self.h, _ptr(a), _ptr(b), _ptr(out), batch, n_limbs, _stream()))
+
+    def linear(self, ct_in, diags, desc: BsgsDesc, ct_out):
+        self._chk(lib().fesc_linear(self.h, _ptr(ct_in), _ptr(diags), ctypes.byref(desc), _ptr(ct_out), _stream()))

@@ -1,0 +1,164 @@
+// Internal declarations of the sm_100a RNS-CKKS library: device arithmetic, context layout.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <map>
+#include <string>
+#include <vector>
+
+#include "fesc.h"
+
+typedef unsigned long long u64;
+typedef unsigned __int128 u128;
+
+#define FESC_MAX_PRIMES 64
+#define FESC_MAX_SPECIAL 8
+#define FESC_MAX_ALPHA 8
+
+// ---------------------------------------------------------------------------------------
+// Per-prime constants (device copy lives in ctx->d_pc, indexed by prime index).
+// ---------------------------------------------------------------------------------------
+struct PrimeConst {
+    u64 q;
+    u64 mu;        // floor(2^64 / q)
+    u64 c64;       // 2^64 mod q
+    u64 c64s;      // floor(c64 * 2^64 / q)   (Shoup companion)
+    u64 ninv;      // N^-1 mod q
+    u64 ninvs;     // Shoup companion of ninv
+    u64 ninvw;     // N^-1 * psi^-brev(1) mod q  (last inverse stage, odd output)
+    u64 ninvws;
+};
+
+// ---------------------------------------------------------------------------------------
+// Device arithmetic.  All moduli are < 2^62, so 4q fits in 64 bits.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ u64 mulhi(u64 a, u64 b) { return __umul64hi(a, b); }
+
+// x*w mod q in [0, 2q) for any x < 2^64, w < q, ws = floor(w*2^64/q)
+__device__ __forceinline__ u64 shoup_lazy(u64 x, u64 w, u64 ws, u64 q) {
+    return x * w - mulhi(x, ws) * q;
+}
+__device__ __forceinline__ u64 csub(u64 x, u64 q) { return x >= q ? x - q : x; }
+__device__ __forceinline__ u64 shoup(u64 x, u64 w, u64 ws, u64 q) { return csub(shoup_lazy(x, w, ws, q), q); }
+__device__ __forceinline__ u64 addmod(u64 a, u64 b, u64 q) { return csub(a + b, q); }
+__device__ __forceinline__ u64 submod(u64 a, u64 b, u64 q) { return a >= b ? a - b : a + q - b; }
+
+// 128-bit accumulator
+struct acc128 {
+    u64 lo, hi;
+};
+__device__ __forceinline__ void mac128(acc128& a, u64 x, u64 y) {
+    u64 l = x * y, h = mulhi(x, y);
+    a.lo += l;
+    a.hi += h + (a.lo < l);
+}
+// (hi*2^64 + lo) mod q, canonical.  hi may be any 64-bit value.
+__device__ __forceinline__ u64 reduce128(u64 hi, u64 lo, const PrimeConst& pc) {
+    u64 a = shoup_lazy(hi, pc.c64, pc.c64s, pc.q);     // hi*2^64 mod q, in [0,2q)
+    u64 b = lo - mulhi(lo, pc.mu) * pc.q;              // lo mod q, in [0,2q)
+    u64 s = a + b;                                     // < 4q < 2^64
+    s = csub(s, 2 * pc.q);
+    return csub(s, pc.q);
+}
+__device__ __forceinline__ u64 mulmod(u64 x, u64 y, const PrimeConst& pc) {
+    return reduce128(mulhi(x, y), x * y, pc);
+}
+
+// counter-based generator (same public recipe as the header documents)
+__host__ __device__ __forceinline__ u64 mix64(u64 z) {
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+__host__ __device__ __forceinline__ u64 make_tag(u64 domain, u64 key_id, u64 digit, u64 limb) {
+    return domain | (key_id << 8) | (digit << 40) | (limb << 48);
+}
+
+// ---------------------------------------------------------------------------------------
+// Row maps: which prime a row of a batched buffer uses.  Row r uses prime[r % period];
+// 0xFF = skip the row.
+// ---------------------------------------------------------------------------------------
+struct RowMap {
+    uint32_t period;
+    uint8_t prime[252];
+};
+
+// ---------------------------------------------------------------------------------------
+// Basis-conversion tables (device copies; built on the host in ctx.cu)
+// ---------------------------------------------------------------------------------------
+// One key-switch digit at one level: source limbs [first, first+n_src), Q_j = their product.
+struct ModUpDigit {
+    uint32_t n_src, first;
+    u64 inv[FESC_MAX_ALPHA], invs[FESC_MAX_ALPHA];   // (Q_j/q_i)^-1 mod q_i and its Shoup companion
+    u64 mat[FESC_MAX_ALPHA][FESC_MAX_PRIMES];        // (Q_j/q_i) mod q_t, t = prime index
+};
+// Division by P = product of the special primes p_k.
+struct ModDownTab {
+    u64 inv[FESC_MAX_SPECIAL], invs[FESC_MAX_SPECIAL];   // (P/p_k)^-1 mod p_k
+    u64 half[FESC_MAX_SPECIAL];                          // floor(p_k / 2)
+    u64 mat[FESC_MAX_SPECIAL][FESC_MAX_PRIMES];          // (P/p_k) mod q_i
+    u64 wrap[FESC_MAX_SPECIAL + 1][FESC_MAX_PRIMES];     // cnt * P mod q_i
+    u64 pinv[FESC_MAX_PRIMES], pinvs[FESC_MAX_PRIMES];   // P^-1 mod q_i
+};
+// Rescale from level l (drops limb l-1); entry index l.
+struct RescaleTab {
+    u64 qinv[FESC_MAX_PRIMES], qinvs[FESC_MAX_PRIMES];   // q_{l-1}^-1 mod q_i
+    u64 wrap[FESC_MAX_PRIMES];                           // q_{l-1} mod q_i
+    u64 half;                                            // floor(q_{l-1} / 2)
+};
+struct Tables {
+    ModUpDigit* d_modup;      // [(level-1) * beta_max + digit], level = 1..n_q
+    ModDownTab* d_moddown;
+    RescaleTab* d_rescale;    // [level], level = 2..n_q (index 0,1 unused)
+    u64* d_Pmod_all;          // P mod q_t for every prime index (0 on special primes)
+};
+
+// ---------------------------------------------------------------------------------------
+// Context
+// ---------------------------------------------------------------------------------------
+struct EvalKey {
+    u64 g;          // Galois element (0 for the relinearisation key)
+    u64* d_key;     // [beta_max][2][n_q+n_p][N]
+};
+
+struct fesc_ctx {
+    uint32_t log_n, N, n_q, n_p, n_primes, dnum, alpha, beta_max;
+    u64 seed;
+    std::vector<u64> q;           // host primes
+    std::vector<PrimeConst> pc;   // host copy
+    PrimeConst* d_pc;             // device [n_primes]
+    ulonglong2* d_tw;             // forward twiddles [n_primes][N] (w, shoup)
+    ulonglong2* d_itw;            // inverse twiddles [n_primes][N]
+    u64* d_s;                     // secret key, EVAL, [n_primes][N]
+    Tables tabs;
+    std::map<uint32_t, EvalKey> keys;
+    // scratch
+    u64* d_scratch;
+    size_t scratch_bytes;
+    uint64_t counters[4];
+    std::string err;
+};
+
+#define FESC_CHECK_CUDA(ctx, call)                                                          \
+    do {                                                                                    \
+        cudaError_t e_ = (call);                                                            \
+        if (e_ != cudaSuccess) {                                                            \
+            (ctx)->err = std::string(#call) + ": " + cudaGetErrorString(e_);                \
+            return FESC_ECUDA;                                                              \
+        }                                                                                   \
+    } while (0)
+
+static inline int fesc_fail(fesc_ctx* ctx, int code, const std::string& msg) {
+    if (ctx) ctx->err = msg;
+    return code;
+}
+
+// internal launchers (ntt.cu)
+// rows: number of N-word rows starting at d_data; map gives the prime per row.
+int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool inverse, cudaStream_t st);
+// scratch (ctx.cu)
+int ctx_scratch(fesc_ctx* ctx, size_t bytes, u64** out);

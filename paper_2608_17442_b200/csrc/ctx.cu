@@ -1,0 +1,447 @@
+// Context: parameter validation, twiddle / basis-conversion tables, seeded key generation.
+#include "common.cuh"
+
+// ---------------------------------------------------------------------------------------
+// host modular arithmetic (table construction only)
+// ---------------------------------------------------------------------------------------
+static u64 h_mul(u64 a, u64 b, u64 q) { return (u64)((u128)a * b % q); }
+static u64 h_pow(u64 a, u64 e, u64 q) {
+    u64 r = 1;
+    a %= q;
+    for (; e; e >>= 1) {
+        if (e & 1) r = h_mul(r, a, q);
+        a = h_mul(a, a, q);
+    }
+    return r;
+}
+static u64 h_inv(u64 a, u64 q) { return h_pow(a % q, q - 2, q); }
+static u64 h_shoup(u64 w, u64 q) { return (u64)(((u128)w << 64) / q); }
+static bool h_is_prime(u64 n) {
+    if (n < 2) return false;
+    static const u64 bases[] = {2, 3, 5, 7, 11, 13, 17, 19, 23, 29, 31, 37};
+    for (u64 p : bases) {
+        if (n % p == 0) return n == p;
+    }
+    u64 d = n - 1;
+    int r = 0;
+    while ((d & 1) == 0) d >>= 1, r++;
+    for (u64 a : bases) {
+        u64 x = h_pow(a, d, n);
+        if (x == 1 || x == n - 1) continue;
+        bool comp = true;
+        for (int i = 1; i < r; i++) {
+            x = h_mul(x, x, n);
+            if (x == n - 1) {
+                comp = false;
+                break;
+            }
+        }
+        if (comp) return false;
+    }
+    return true;
+}
+static uint32_t h_brev(uint32_t x, uint32_t bits) {
+    uint32_t r = 0;
+    for (uint32_t i = 0; i < bits; i++) r = (r << 1) | ((x >> i) & 1);
+    return r;
+}
+// smallest primitive 2N-th root of unity
+static u64 h_min_root(u64 q, uint32_t log_n) {
+    const u64 N = 1ull << log_n;
+    u64 root = 0;
+    for (u64 g = 2; g < 4096 && !root; g++) {
+        u64 c = h_pow(g, (q - 1) / (2 * N), q);
+        if (h_pow(c, N, q) == q - 1) root = c;
+    }
+    if (!root) return 0;
+    u64 sq = h_mul(root, root, q), cur = root, best = root;
+    for (u64 i = 1; i < N; i++) {
+        cur = h_mul(cur, sq, q);
+        if (cur < best) best = cur;
+    }
+    return best;
+}
+
+// ---------------------------------------------------------------------------------------
+// key-generation kernels
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ u64 draw(u64 seed, u64 tag, u64 idx) { return mix64(mix64(seed ^ mix64(tag)) + idx); }
+
+// out[limb][i] uniform below q_limb, tag carries (domain, key_id, digit), limb index added here
+__global__ void k_sample_uniform(u64* __restrict__ out, const PrimeConst* __restrict__ pcs, uint32_t N, u64 seed,
+                                 u64 tag_base) {
+    const uint32_t limb = blockIdx.y;
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    u64 w = draw(seed, tag_base | ((u64)limb << 48), i);
+    out[(size_t)limb * N + i] = mulhi(w, pcs[limb].q);
+}
+// kind 0: ternary, kind 1: centred binomial (eta 21); the same small integer reduced on every limb
+__global__ void k_sample_small(u64* __restrict__ out, const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t n_limbs,
+                               u64 seed, u64 tag, int kind) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    u64 w = draw(seed, tag, i);
+    long long v;
+    if (kind == 0) {
+        v = (long long)mulhi(w, 3) - 1;
+    } else {
+        const u64 m = (1ull << 21) - 1;
+        v = (long long)__popcll(w & m) - (long long)__popcll((w >> 21) & m);
+    }
+    for (uint32_t l = 0; l < n_limbs; l++) {
+        u64 q = pcs[l].q;
+        out[(size_t)l * N + i] = v >= 0 ? (u64)v : q - (u64)(-v);
+    }
+}
+// b = -a*s + e + [limb in digit] * Pmod[limb] * sp      (all EVAL, all limbs)
+__global__ void k_make_b(u64* __restrict__ b, const u64* __restrict__ a, const u64* __restrict__ s,
+                         const u64* __restrict__ e, const u64* __restrict__ sp, const PrimeConst* __restrict__ pcs,
+                         const u64* __restrict__ Pmod, uint32_t N, uint32_t dig_lo, uint32_t dig_hi) {
+    const uint32_t limb = blockIdx.y;
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    const PrimeConst pc = pcs[limb];
+    const size_t o = (size_t)limb * N + i;
+    u64 v = submod(e[o], mulmod(a[o], s[o], pc), pc.q);
+    if (limb >= dig_lo && limb < dig_hi) v = addmod(v, mulmod(Pmod[limb], sp[o], pc), pc.q);
+    b[o] = v;
+}
+__global__ void k_square(u64* __restrict__ out, const u64* __restrict__ s, const PrimeConst* __restrict__ pcs,
+                         uint32_t N) {
+    const uint32_t limb = blockIdx.y;
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    const size_t o = (size_t)limb * N + i;
+    out[o] = mulmod(s[o], s[o], pcs[limb]);
+}
+// out[t] = in[pi_g(t)]: the Galois map in bit-reversed evaluation order
+__global__ void k_autom_rows(u64* __restrict__ out, const u64* __restrict__ in, uint32_t log_n, u64 g) {
+    const uint32_t N = 1u << log_n;
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= N) return;
+    const size_t row = blockIdx.y;
+    uint32_t u = __brev(t) >> (32 - log_n);
+    uint32_t e = (uint32_t)(((2ull * u + 1) * g) & (2ull * N - 1));
+    uint32_t src = __brev((e - 1) >> 1) >> (32 - log_n);
+    out[row * N + t] = in[row * N + src];
+}
+
+// ---------------------------------------------------------------------------------------
+int ctx_scratch(fesc_ctx* ctx, size_t bytes, u64** out) {
+    if (bytes > ctx->scratch_bytes) {
+        if (ctx->d_scratch) {
+            FESC_CHECK_CUDA(ctx, cudaDeviceSynchronize());
+            cudaFree(ctx->d_scratch);
+            ctx->d_scratch = nullptr;
+            ctx->scratch_bytes = 0;
+        }
+        size_t want = (bytes + (1u << 20) - 1) & ~(size_t)((1u << 20) - 1);
+        if (cudaMalloc(&ctx->d_scratch, want) != cudaSuccess) {
+            cudaGetLastError();
+            return fesc_fail(ctx, FESC_ENOMEM, "scratch allocation of " + std::to_string(want) + " bytes failed");
+        }
+        ctx->scratch_bytes = want;
+        ctx->counters[3] = want;
+    }
+    *out = ctx->d_scratch;
+    return FESC_OK;
+}
+
+template <typename T>
+static int upload(fesc_ctx* ctx, T** d, const std::vector<T>& h) {
+    if (cudaMalloc(d, h.size() * sizeof(T)) != cudaSuccess) {
+        cudaGetLastError();
+        return fesc_fail(ctx, FESC_ENOMEM, "table allocation failed");
+    }
+    FESC_CHECK_CUDA(ctx, cudaMemcpy(*d, h.data(), h.size() * sizeof(T), cudaMemcpyHostToDevice));
+    return FESC_OK;
+}
+
+static RowMap all_limbs_map(const fesc_ctx* ctx) {
+    RowMap m;
+    m.period = ctx->n_primes;
+    for (uint32_t i = 0; i < ctx->n_primes; i++) m.prime[i] = (uint8_t)i;
+    return m;
+}
+
+// Basis-conversion tables, computed with 128-bit host arithmetic.
+static int build_tables(fesc_ctx* ctx) {
+    const uint32_t nq = ctx->n_q, np = ctx->n_primes, K = ctx->n_p, alpha = ctx->alpha;
+    const std::vector<u64>& q = ctx->q;
+    int rc;
+    // ModUp: for every level and digit
+    std::vector<ModUpDigit> mu((size_t)nq * ctx->beta_max);
+    memset(mu.data(), 0, mu.size() * sizeof(ModUpDigit));
+    for (uint32_t level = 1; level <= nq; level++) {
+        for (uint32_t j = 0; j * alpha < level; j++) {
+            ModUpDigit& d = mu[(size_t)(level - 1) * ctx->beta_max + j];
+            d.first = j * alpha;
+            uint32_t hi = d.first + alpha < level ? d.first + alpha : level;
+            d.n_src = hi - d.first;
+            for (uint32_t a = 0; a < d.n_src; a++) {
+                uint32_t i = d.first + a;
+                // (Q_j / q_i) modulo every prime
+                for (uint32_t t = 0; t < np; t++) {
+                    u64 m = 1;
+                    for (uint32_t b = 0; b < d.n_src; b++)
+                        if (b != a) m = h_mul(m, q[d.first + b] % q[t], q[t]);
+                    d.mat[a][t] = m;
+                }
+                d.inv[a] = h_inv(d.mat[a][i], q[i]);
+                d.invs[a] = h_shoup(d.inv[a], q[i]);
+            }
+        }
+    }
+    if ((rc = upload(ctx, &ctx->tabs.d_modup, mu)) != FESC_OK) return rc;
+    // ModDown
+    std::vector<ModDownTab> mdv(1);
+    ModDownTab& md = mdv[0];
+    memset(&md, 0, sizeof(md));
+    std::vector<u64> Pmod(np, 0);
+    for (uint32_t k = 0; k < K; k++) {
+        u64 pk = q[nq + k];
+        u64 hat = 1;
+        for (uint32_t b = 0; b < K; b++)
+            if (b != k) hat = h_mul(hat, q[nq + b] % pk, pk);
+        md.inv[k] = h_inv(hat, pk);
+        md.invs[k] = h_shoup(md.inv[k], pk);
+        md.half[k] = pk / 2;
+        for (uint32_t i = 0; i < nq; i++) {
+            u64 m = 1;
+            for (uint32_t b = 0; b < K; b++)
+                if (b != k) m = h_mul(m, q[nq + b] % q[i], q[i]);
+            md.mat[k][i] = m;
+        }
+    }
+    for (uint32_t i = 0; i < nq; i++) {
+        u64 P = 1;
+        for (uint32_t b = 0; b < K; b++) P = h_mul(P, q[nq + b] % q[i], q[i]);
+        Pmod[i] = P;
+        md.pinv[i] = h_inv(P, q[i]);
+        md.pinvs[i] = h_shoup(md.pinv[i], q[i]);
+        for (uint32_t c = 0; c <= K; c++) md.wrap[c][i] = h_mul(c, P, q[i]);
+    }
+    if ((rc = upload(ctx, &ctx->tabs.d_moddown, mdv)) != FESC_OK) return rc;
+    if ((rc = upload(ctx, &ctx->tabs.d_Pmod_all, Pmod)) != FESC_OK) return rc;
+    // Rescale
+    std::vector<RescaleTab> rs(nq + 1);
+    memset(rs.data(), 0, rs.size() * sizeof(RescaleTab));
+    for (uint32_t level = 2; level <= nq; level++) {
+        u64 ql = q[level - 1];
+        rs[level].half = ql / 2;
+        for (uint32_t i = 0; i + 1 < level; i++) {
+            rs[level].qinv[i] = h_inv(ql % q[i], q[i]);
+            rs[level].qinvs[i] = h_shoup(rs[level].qinv[i], q[i]);
+            rs[level].wrap[i] = ql % q[i];
+        }
+    }
+    return upload(ctx, &ctx->tabs.d_rescale, rs);
+}
+static void free_tables(fesc_ctx* ctx) {
+    cudaFree(ctx->tabs.d_modup);
+    cudaFree(ctx->tabs.d_moddown);
+    cudaFree(ctx->tabs.d_rescale);
+    cudaFree(ctx->tabs.d_Pmod_all);
+}
+
+// Generate the switching key from s' (EVAL on all limbs, device) to s.
+static int gen_key(fesc_ctx* ctx, uint32_t key_id, const u64* d_sp, u64 g) {
+    const uint32_t N = ctx->N, np = ctx->n_primes;
+    const size_t limb_words = (size_t)np * N;
+    u64* d_key = nullptr;
+    if (cudaMalloc(&d_key, (size_t)ctx->beta_max * 2 * limb_words * sizeof(u64)) != cudaSuccess) {
+        cudaGetLastError();
+        return fesc_fail(ctx, FESC_ENOMEM, "key allocation failed");
+    }
+    u64* d_e = nullptr;
+    if (cudaMalloc(&d_e, limb_words * sizeof(u64)) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(d_key);
+        return fesc_fail(ctx, FESC_ENOMEM, "key allocation failed");
+    }
+    dim3 grid((N + 255) / 256, np);
+    RowMap map = all_limbs_map(ctx);
+    int rc = FESC_OK;
+    for (uint32_t j = 0; j < ctx->beta_max && rc == FESC_OK; j++) {
+        u64* b = d_key + (size_t)(2 * j) * limb_words;
+        u64* a = b + limb_words;
+        k_sample_uniform<<<grid, 256>>>(a, ctx->d_pc, N, ctx->seed, make_tag(2, key_id, j, 0));
+        k_sample_small<<<(N + 255) / 256, 256>>>(d_e, ctx->d_pc, N, np, ctx->seed, make_tag(3, key_id, j, 0), 1);
+        rc = ntt_launch(ctx, d_e, np, map, false, 0);
+        uint32_t lo = j * ctx->alpha, hi = lo + ctx->alpha;
+        if (hi > ctx->n_q) hi = ctx->n_q;
+        k_make_b<<<grid, 256>>>(b, a, ctx->d_s, d_e, d_sp, ctx->d_pc, ctx->tabs.d_Pmod_all, N, lo, hi);
+    }
+    cudaError_t e = cudaDeviceSynchronize();
+    cudaFree(d_e);
+    if (rc == FESC_OK && e != cudaSuccess) {
+        ctx->err = std::string("key generation: ") + cudaGetErrorString(e);
+        rc = FESC_ECUDA;
+    }
+    if (rc != FESC_OK) {
+        cudaFree(d_key);
+        return rc;
+    }
+    auto it = ctx->keys.find(key_id);
+    if (it != ctx->keys.end()) cudaFree(it->second.d_key);
+    ctx->keys[key_id] = EvalKey{g, d_key};
+    return FESC_OK;
+}
+
+extern "C" int fesc_ctx_create(fesc_ctx** out, uint32_t log_n, const uint64_t* primes, uint32_t n_q, uint32_t n_p,
+                               uint32_t dnum, uint64_t seed) {
+    if (!out) return FESC_EINVAL;
+    *out = nullptr;
+    if (!primes || n_q == 0 || n_p == 0 || dnum == 0 || n_q + n_p > FESC_MAX_PRIMES || n_p > FESC_MAX_SPECIAL)
+        return FESC_EINVAL;
+    if (!((log_n >= 4 && log_n <= 12) || log_n == 16)) return FESC_EINVAL;
+    fesc_ctx* ctx = new (std::nothrow) fesc_ctx();
+    if (!ctx) return FESC_ENOMEM;
+    ctx->log_n = log_n;
+    ctx->N = 1u << log_n;
+    ctx->n_q = n_q;
+    ctx->n_p = n_p;
+    ctx->n_primes = n_q + n_p;
+    ctx->dnum = dnum;
+    ctx->alpha = (n_q + dnum - 1) / dnum;
+    ctx->beta_max = (n_q + ctx->alpha - 1) / ctx->alpha;
+    ctx->seed = seed;
+    ctx->d_pc = nullptr;
+    ctx->d_tw = ctx->d_itw = nullptr;
+    ctx->d_s = nullptr;
+    ctx->d_scratch = nullptr;
+    ctx->scratch_bytes = 0;
+    memset(ctx->counters, 0, sizeof(ctx->counters));
+    memset(&ctx->tabs, 0, sizeof(ctx->tabs));
+    const uint32_t N = ctx->N, np = ctx->n_primes;
+    int rc = FESC_OK;
+    auto bail = [&](int code) {
+        fesc_ctx_destroy(ctx);
+        return code;
+    };
+    if (ctx->alpha > FESC_MAX_ALPHA) return bail(FESC_EINVAL);
+    // ---- validate primes, per-prime constants, twiddles ----
+    std::vector<ulonglong2> tw((size_t)np * N), itw((size_t)np * N);
+    for (uint32_t i = 0; i < np; i++) {
+        u64 q = primes[i];
+        if (q >= (1ull << 62) || q < 3 || (q - 1) % (2ull * N) != 0 || !h_is_prime(q)) return bail(FESC_EINVAL);
+        for (uint32_t k = 0; k < i; k++)
+            if (primes[k] == q) return bail(FESC_EINVAL);
+        u64 psi = h_min_root(q, log_n);
+        if (!psi) return bail(FESC_EINVAL);
+        u64 ipsi = h_inv(psi, q);
+        ctx->q.push_back(q);
+        PrimeConst pc;
+        pc.q = q;
+        pc.mu = (u64)((((u128)1) << 64) / q);
+        pc.c64 = (u64)((((u128)1) << 64) % q);
+        pc.c64s = h_shoup(pc.c64, q);
+        pc.ninv = h_inv(N % q, q);
+        pc.ninvs = h_shoup(pc.ninv, q);
+        // powers in bit-reversed order: tw[k] = psi^brev(k), itw[k] = psi^-brev(k)
+        std::vector<u64> pw(N), ipw(N);
+        pw[0] = ipw[0] = 1;
+        for (uint32_t k = 1; k < N; k++) {
+            pw[k] = h_mul(pw[k - 1], psi, q);
+            ipw[k] = h_mul(ipw[k - 1], ipsi, q);
+        }
+        for (uint32_t k = 0; k < N; k++) {
+            uint32_t r = h_brev(k, log_n);
+            tw[(size_t)i * N + k] = make_ulonglong2(pw[r], h_shoup(pw[r], q));
+            itw[(size_t)i * N + k] = make_ulonglong2(ipw[r], h_shoup(ipw[r], q));
+        }
+        pc.ninvw = h_mul(pc.ninv, ipw[h_brev(1, log_n)], q);
+        pc.ninvws = h_shoup(pc.ninvw, q);
+        ctx->pc.push_back(pc);
+    }
+    if ((rc = upload(ctx, &ctx->d_pc, ctx->pc)) != FESC_OK) return bail(rc);
+    if ((rc = upload(ctx, &ctx->d_tw, tw)) != FESC_OK) return bail(rc);
+    if ((rc = upload(ctx, &ctx->d_itw, itw)) != FESC_OK) return bail(rc);
+    if ((rc = build_tables(ctx)) != FESC_OK) return bail(rc);
+    // ---- secret key and relinearisation key ----
+    if (cudaMalloc(&ctx->d_s, (size_t)np * N * sizeof(u64)) != cudaSuccess) return bail(FESC_ENOMEM);
+    k_sample_small<<<(N + 255) / 256, 256>>>(ctx->d_s, ctx->d_pc, N, np, seed, make_tag(1, 0, 0, 0), 0);
+    if ((rc = ntt_launch(ctx, ctx->d_s, np, all_limbs_map(ctx), false, 0)) != FESC_OK) return bail(rc);
+    u64* d_s2 = nullptr;
+    if (cudaMalloc(&d_s2, (size_t)np * N * sizeof(u64)) != cudaSuccess) return bail(FESC_ENOMEM);
+    k_square<<<dim3((N + 255) / 256, np), 256>>>(d_s2, ctx->d_s, ctx->d_pc, N);
+    rc = gen_key(ctx, FESC_RELIN_KEY_ID, d_s2, 0);
+    cudaFree(d_s2);
+    if (rc != FESC_OK) return bail(rc);
+    memset(ctx->counters, 0, sizeof(ctx->counters));
+    *out = ctx;
+    return FESC_OK;
+}
+
+extern "C" int fesc_ctx_destroy(fesc_ctx* ctx) {
+    if (!ctx) return FESC_OK;
+    cudaDeviceSynchronize();
+    for (auto& kv : ctx->keys) cudaFree(kv.second.d_key);
+    cudaFree(ctx->d_pc);
+    cudaFree(ctx->d_tw);
+    cudaFree(ctx->d_itw);
+    cudaFree(ctx->d_s);
+    cudaFree(ctx->d_scratch);
+    free_tables(ctx);
+    delete ctx;
+    return FESC_OK;
+}
+
+extern "C" const char* fesc_last_error(const fesc_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+extern "C" int fesc_sync(fesc_ctx* ctx, void* stream) {
+    if (!ctx) return FESC_EINVAL;
+    FESC_CHECK_CUDA(ctx, cudaStreamSynchronize((cudaStream_t)stream));
+    FESC_CHECK_CUDA(ctx, cudaGetLastError());
+    return FESC_OK;
+}
+
+extern "C" int fesc_ctx_add_galois_key(fesc_ctx* ctx, int32_t rot, uint32_t key_id) {
+    if (!ctx) return FESC_EINVAL;
+    if (key_id == FESC_RELIN_KEY_ID || key_id >= (1u << 24)) return fesc_fail(ctx, FESC_EINVAL, "key id out of range");
+    const u64 twoN = 2ull * ctx->N;
+    u64 g;
+    if (rot == FESC_CONJ) {
+        g = twoN - 1;
+    } else {
+        const int64_t n = ctx->N / 2;
+        u64 r = (u64)((((int64_t)rot % n) + n) % n);
+        g = 1;
+        u64 b = 5;
+        for (; r; r >>= 1) {
+            if (r & 1) g = g * b % twoN;
+            b = b * b % twoN;
+        }
+    }
+    u64* d_sp = nullptr;
+    if (cudaMalloc(&d_sp, (size_t)ctx->n_primes * ctx->N * sizeof(u64)) != cudaSuccess) {
+        cudaGetLastError();
+        return fesc_fail(ctx, FESC_ENOMEM, "key allocation failed");
+    }
+    k_autom_rows<<<dim3((ctx->N + 255) / 256, ctx->n_primes), 256>>>(d_sp, ctx->d_s, ctx->log_n, g);
+    int rc = gen_key(ctx, key_id, d_sp, g);
+    cudaFree(d_sp);
+    return rc;
+}
+
+extern "C" int fesc_ctx_export_key(fesc_ctx* ctx, uint32_t key_id, uint64_t* d_dst, void* stream) {
+    if (!ctx || !d_dst) return FESC_EINVAL;
+    auto it = ctx->keys.find(key_id);
+    if (it == ctx->keys.end()) return fesc_fail(ctx, FESC_ENOKEY, "no key " + std::to_string(key_id));
+    size_t bytes = (size_t)ctx->beta_max * 2 * ctx->n_primes * ctx->N * sizeof(u64);
+    FESC_CHECK_CUDA(ctx, cudaMemcpyAsync(d_dst, it->second.d_key, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    return FESC_OK;
+}
+extern "C" int fesc_ctx_export_secret(fesc_ctx* ctx, uint64_t* d_dst, void* stream) {
+    if (!ctx || !d_dst) return FESC_EINVAL;
+    size_t bytes = (size_t)ctx->n_primes * ctx->N * sizeof(u64);
+    FESC_CHECK_CUDA(ctx, cudaMemcpyAsync(d_dst, ctx->d_s, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    return FESC_OK;
+}
+extern "C" uint32_t fesc_ctx_num_digits(const fesc_ctx* ctx) { return ctx ? ctx->beta_max : 0; }
+extern "C" int fesc_ctx_counters(const fesc_ctx* ctx, uint64_t out[4]) {
+    if (!ctx || !out) return FESC_EINVAL;
+    memcpy(out, ctx->counters, sizeof(ctx->counters));
+    return FESC_OK;
+}

@@ -1,0 +1,149 @@
+// BSGS plaintext-weight projection Y = XW on packed ciphertexts.
+//
+// Per group of token blocks: (1) baby rotations of every input ciphertext, batched per rotation
+// amount so a key is streamed once per batch; (2) one fused accumulate kernel that forms every
+// giant-step accumulator acc[tb][b][p] = sum_{g,q} rot[tb][g][q] (.) D[b][p][g][q] with 128-bit
+// lazy sums in registers, tiled TT token blocks x PT (b,p) pairs per thread so a rotated
+// ciphertext word is reused PT times and a diagonal word TT times; (3) giant rotations that
+// accumulate straight into acc[tb][b][0]; (4) rescale into the output.
+#include "ops.cuh"
+
+template <int TT, int PT>
+__global__ void __launch_bounds__(256) k_bsgs_accumulate(
+    const u64* __restrict__ in,     // [tbs][gin][2][level][N]            (q = 0 terms)
+    const u64* __restrict__ rot,    // [tbs][gin][n1][2][level][N]        (slot q = 0 unused)
+    const u64* __restrict__ diags,  // [nout][n2][gin][n1][level][N]
+    u64* __restrict__ acc,          // [tbs][nout][n2][2][level][N]
+    const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level, uint32_t tbs, uint32_t gin, uint32_t n1,
+    uint32_t bp_count /* nout*n2 */, uint32_t reduce_every) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t l = blockIdx.y;
+    const uint32_t bp_tiles = (bp_count + PT - 1) / PT;
+    const uint32_t tb0 = (blockIdx.z / bp_tiles) * TT, bp0 = (blockIdx.z % bp_tiles) * PT;
+    if (c >= N) return;
+    const PrimeConst pc = pcs[l];
+    const size_t poly = (size_t)level * N, ctw = 2 * poly;
+    const size_t o = (size_t)l * N + c;
+    acc128 a[TT][PT][2];
+#pragma unroll
+    for (int i = 0; i < TT; i++)
+#pragma unroll
+        for (int j = 0; j < PT; j++) a[i][j][0] = a[i][j][1] = acc128{0, 0};
+    const uint32_t terms = gin * n1;
+    uint32_t since = 0;
+    for (uint32_t gq = 0; gq < terms; gq++) {
+        const uint32_t g = gq / n1, q = gq % n1;
+        u64 x0[TT], x1[TT];
+#pragma unroll
+        for (int i = 0; i < TT; i++) {
+            const uint32_t tb = tb0 + i;
+            x0[i] = x1[i] = 0;
+            if (tb < tbs) {
+                const u64* src = q == 0 ? in + ((size_t)tb * gin + g) * ctw
+                                        : rot + (((size_t)tb * gin + g) * n1 + q) * ctw;
+                x0[i] = src[o];
+                x1[i] = src[poly + o];
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < PT; j++) {
+            const uint32_t bp = bp0 + j;
+            if (bp < bp_count) {
+                const u64 w = __ldg(diags + (((size_t)bp * gin + g) * n1 + q) * poly + o);
+#pragma unroll
+                for (int i = 0; i < TT; i++) {
+                    mac128(a[i][j][0], x0[i], w);
+                    mac128(a[i][j][1], x1[i], w);
+                }
+            }
+        }
+        if (++since == reduce_every) {
+            since = 0;
+#pragma unroll
+            for (int i = 0; i < TT; i++)
+#pragma unroll
+                for (int j = 0; j < PT; j++)
+#pragma unroll
+                    for (int p = 0; p < 2; p++) a[i][j][p] = acc128{reduce128(a[i][j][p].hi, a[i][j][p].lo, pc), 0};
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < TT; i++)
+#pragma unroll
+        for (int j = 0; j < PT; j++) {
+            const uint32_t tb = tb0 + i, bp = bp0 + j;
+            if (tb < tbs && bp < bp_count) {
+                u64* dst = acc + ((size_t)tb * bp_count + bp) * ctw;
+                dst[o] = reduce128(a[i][j][0].hi, a[i][j][0].lo, pc);
+                dst[poly + o] = reduce128(a[i][j][1].hi, a[i][j][1].lo, pc);
+            }
+        }
+}
+
+extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_t* d_diags, const fesc_bsgs_desc* desc,
+                           uint64_t* d_ct_out, void* stream) {
+    if (!ctx || !d_ct_in || !d_diags || !desc || !d_ct_out) return FESC_EINVAL;
+    const uint32_t n1 = desc->n1, n2 = desc->n2, gin = desc->in_blocks, nout = desc->out_blocks;
+    const uint32_t tbs = desc->token_blocks, level = desc->n_limbs, N = ctx->N;
+    if (!n1 || !n2 || !gin || !nout || !tbs) return fesc_fail(ctx, FESC_EINVAL, "linear: empty dimension");
+    if (level < 2 || level > ctx->n_q) return fesc_fail(ctx, FESC_ELEVEL, "linear: level out of range");
+    for (uint32_t q = 1; q < n1; q++)
+        if (!ctx->keys.count(desc->baby_key_base + q))
+            return fesc_fail(ctx, FESC_ENOKEY, "linear: missing baby-step key " + std::to_string(desc->baby_key_base + q));
+    for (uint32_t p = 1; p < n2; p++)
+        if (!ctx->keys.count(desc->giant_key_base + p))
+            return fesc_fail(ctx, FESC_ENOKEY, "linear: missing giant-step key " + std::to_string(desc->giant_key_base + p));
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t ctw = (size_t)2 * level * N;
+    // token blocks per group: keep the group's buffers near 12 GiB
+    const size_t per_tb = ((size_t)gin * n1 + (size_t)nout * n2) * ctw * sizeof(u64);
+    uint32_t tbg = (uint32_t)(((size_t)12 << 30) / per_tb);
+    if (tbg < 1) tbg = 1;
+    if (tbg > tbs) tbg = tbs;
+    const uint32_t max_batch = tbg * (gin > nout ? gin : nout);
+    const size_t ks_words = ks_scratch_words(ctx, level, ks_chunk(ctx, max_batch));
+    const size_t rs_words = (size_t)(tbg * nout < 16384 ? tbg * nout : 16384) * 2 * N;
+    const size_t rot_words = (size_t)tbg * gin * n1 * ctw, acc_words = (size_t)tbg * nout * n2 * ctw;
+    u64* scratch;
+    int rc = ctx_scratch(ctx, (rot_words + acc_words + (ks_words > rs_words ? ks_words : rs_words)) * sizeof(u64), &scratch);
+    if (rc != FESC_OK) return rc;
+    u64* rot = scratch;
+    u64* acc = rot + rot_words;
+    u64* ks = acc + acc_words;
+    // lazy 128-bit sums: reduce before terms * q^2 could reach 2^128
+    uint32_t qbits = 0;
+    for (uint32_t i = 0; i < level; i++) {
+        uint32_t b = 64 - __builtin_clzll(ctx->q[i]);
+        if (b > qbits) qbits = b;
+    }
+    uint32_t reduce_every = 2 * qbits >= 127 ? 1 : (2 * qbits <= 96 ? 0x7fffffffu : (1u << (127 - 2 * qbits)));
+    const u64* in = (const u64*)d_ct_in;
+    const u64* diags = (const u64*)d_diags;
+    u64* out = (u64*)d_ct_out;
+    for (uint32_t tb0 = 0; tb0 < tbs; tb0 += tbg) {
+        const uint32_t nt = tbs - tb0 < tbg ? tbs - tb0 : tbg;
+        const u64* gin_base = in + (size_t)tb0 * gin * ctw;
+        for (uint32_t q = 1; q < n1; q++) {
+            rc = rotate_internal(ctx, gin_base, ctw, rot + (size_t)q * ctw, (size_t)n1 * ctw, nt * gin, level,
+                                 desc->baby_key_base + q, ks, st, 0);
+            if (rc != FESC_OK) return rc;
+        }
+        constexpr int TT = 2, PT = 2;
+        const uint32_t bp_count = nout * n2;
+        const uint32_t tiles = ((nt + TT - 1) / TT) * ((bp_count + PT - 1) / PT);
+        if (tiles > 65535) return fesc_fail(ctx, FESC_EINVAL, "linear: too many accumulator tiles");
+        k_bsgs_accumulate<TT, PT><<<dim3((N + 255) / 256, level, tiles), 256, 0, st>>>(
+            gin_base, rot, diags, acc, ctx->d_pc, N, level, nt, gin, n1, bp_count, reduce_every);
+        FESC_CHECK_CUDA(ctx, cudaGetLastError());
+        ctx->counters[2] += (uint64_t)nt * bp_count * gin * n1;
+        for (uint32_t p = 1; p < n2; p++) {
+            rc = rotate_internal(ctx, acc + (size_t)p * ctw, (size_t)n2 * ctw, acc, (size_t)n2 * ctw, nt * nout, level,
+                                 desc->giant_key_base + p, ks, st, 1);
+            if (rc != FESC_OK) return rc;
+        }
+        rc = rescale_internal(ctx, acc, (size_t)n2 * ctw, out + (size_t)tb0 * nout * 2 * (level - 1) * N, nt * nout, level,
+                              ks, st);
+        if (rc != FESC_OK) return rc;
+    }
+    return FESC_OK;
+}

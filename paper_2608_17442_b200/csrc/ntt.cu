@@ -1,0 +1,342 @@
+// Negacyclic NTT / inverse NTT over RNS limbs for sm_100a.
+//
+// Forward: Cooley-Tukey butterflies with psi merged into the twiddles (natural order in,
+// bit-reversed evaluation order out); inverse: Gentleman-Sande with the inverse twiddles and
+// N^-1 folded into the last stage.  Twiddles carry a Shoup companion so a butterfly costs one
+// mul.hi.u64 and two mul.lo.u64 on the integer pipe; values stay lazily reduced ([0,4q) forward,
+// [0,2q) inverse) until the last stage.
+//
+// N = 2^16 runs as two kernels of 8 stages each.  Every thread keeps 8 points in registers and
+// does three (3+3+2) register rounds per kernel, exchanging through shared memory in between:
+//   * "strided" kernel: stages whose butterfly distance is >= 256.  A CTA owns 16 adjacent
+//     columns (128 B segments) of the 256 x 256 view of the limb.
+//   * "contiguous" kernel: stages with distance < 256.  One WARP owns one 256-point block, so
+//     the exchanges need only __syncwarp.
+// N <= 2^12 runs as one shared-memory kernel per row (tests and the tiny workload).
+#include "common.cuh"
+
+// twiddle index of local stage ls (of S) for local element e with prefix pre:
+//   pre * 2^ls + (e >> (S - ls))
+// (pre = 1 for the strided kernel; pre = 256 + block index for the contiguous kernel).
+
+struct Tw {
+    u64 w, s;
+};
+__device__ __forceinline__ Tw ldtw(const ulonglong2* __restrict__ t, uint32_t i) {
+    ulonglong2 v = __ldg(t + i);
+    return Tw{v.x, v.y};
+}
+
+// forward butterfly, inputs in [0,4q), outputs in [0,4q)
+__device__ __forceinline__ void ct_bfly(u64& x, u64& y, const Tw& t, u64 q, u64 q2) {
+    u64 u = csub(x, q2);
+    u64 v = shoup_lazy(y, t.w, t.s, q);
+    x = u + v;
+    y = u - v + q2;
+}
+// inverse butterfly, inputs in [0,2q), outputs in [0,2q)
+__device__ __forceinline__ void gs_bfly(u64& x, u64& y, const Tw& t, u64 q, u64 q2) {
+    u64 u = x, v = y;
+    x = csub(u + v, q2);
+    y = shoup_lazy(u - v + q2, t.w, t.s, q);
+}
+
+// Three forward stages on 8 registers holding elements e0 + k*d (k = 0..7); the twiddle
+// indices are base indices for the first pair of each stage.
+//   stage A: pairs (k,k+4), one twiddle         idxA
+//   stage B: pairs (k,k+2), twiddles            idxB + (k>>2)
+//   stage C: pairs (k,k+1), twiddles            idxC + (k>>1)
+__device__ __forceinline__ void fwd_round3(u64 (&x)[8], const ulonglong2* __restrict__ tw, uint32_t idxA,
+                                           uint32_t idxB, uint32_t idxC, u64 q, u64 q2) {
+    Tw a = ldtw(tw, idxA);
+#pragma unroll
+    for (int k = 0; k < 4; k++) ct_bfly(x[k], x[k + 4], a, q, q2);
+    Tw b0 = ldtw(tw, idxB), b1 = ldtw(tw, idxB + 1);
+    ct_bfly(x[0], x[2], b0, q, q2);
+    ct_bfly(x[1], x[3], b0, q, q2);
+    ct_bfly(x[4], x[6], b1, q, q2);
+    ct_bfly(x[5], x[7], b1, q, q2);
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+        Tw c = ldtw(tw, idxC + k);
+        ct_bfly(x[2 * k], x[2 * k + 1], c, q, q2);
+    }
+}
+// Two forward stages (pairs (k,k+2) then (k,k+1)) on two groups of 4.
+__device__ __forceinline__ void fwd_round2(u64 (&x)[8], const ulonglong2* __restrict__ tw, uint32_t idxB,
+                                           uint32_t idxC, u64 q, u64 q2) {
+    Tw b0 = ldtw(tw, idxB), b1 = ldtw(tw, idxB + 1);
+    ct_bfly(x[0], x[2], b0, q, q2);
+    ct_bfly(x[1], x[3], b0, q, q2);
+    ct_bfly(x[4], x[6], b1, q, q2);
+    ct_bfly(x[5], x[7], b1, q, q2);
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+        Tw c = ldtw(tw, idxC + k);
+        ct_bfly(x[2 * k], x[2 * k + 1], c, q, q2);
+    }
+}
+__device__ __forceinline__ void inv_round2(u64 (&x)[8], const ulonglong2* __restrict__ tw, uint32_t idxB,
+                                           uint32_t idxC, u64 q, u64 q2) {
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+        Tw c = ldtw(tw, idxC + k);
+        gs_bfly(x[2 * k], x[2 * k + 1], c, q, q2);
+    }
+    Tw b0 = ldtw(tw, idxB), b1 = ldtw(tw, idxB + 1);
+    gs_bfly(x[0], x[2], b0, q, q2);
+    gs_bfly(x[1], x[3], b0, q, q2);
+    gs_bfly(x[4], x[6], b1, q, q2);
+    gs_bfly(x[5], x[7], b1, q, q2);
+}
+__device__ __forceinline__ void inv_round3(u64 (&x)[8], const ulonglong2* __restrict__ tw, uint32_t idxA,
+                                           uint32_t idxB, uint32_t idxC, u64 q, u64 q2) {
+    inv_round2(x, tw, idxB, idxC, q, q2);
+    Tw a = ldtw(tw, idxA);
+#pragma unroll
+    for (int k = 0; k < 4; k++) gs_bfly(x[k], x[k + 4], a, q, q2);
+}
+
+// ---------------------------------------------------------------------------------------
+// N = 2^16, strided kernel (stages 0..7 forward / the last 8 stages inverse).
+// grid = (16 column tiles, rows); block = 512 threads = 16 columns x 32 sub-threads.
+// ---------------------------------------------------------------------------------------
+#define N16 65536u
+
+template <bool INV>
+__global__ void __launch_bounds__(512) ntt16_strided(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
+                                                     const PrimeConst* __restrict__ pcs, RowMap map) {
+    const uint32_t row = blockIdx.y;
+    const uint32_t pi = map.prime[row % map.period];
+    if (pi == 0xFF) return;
+    __shared__ u64 sm[256 * 16];
+    const PrimeConst pc = pcs[pi];
+    const u64 q = pc.q, q2 = 2 * pc.q;
+    const ulonglong2* tw = tw_all + (size_t)pi * N16;
+    u64* p = data + (size_t)row * N16 + blockIdx.x * 16;
+    const uint32_t col = threadIdx.x & 15, sub = threadIdx.x >> 4;
+    const uint32_t h2 = sub >> 2, l2 = sub & 3;
+    u64 x[8];
+    if (!INV) {
+        // round 1: hi = k*32 + sub, local stages 0,1,2
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = p[(size_t)(k * 32 + sub) * 256 + col];
+        fwd_round3(x, tw, 1, 2, 4, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[(k * 32 + sub) * 16 + col] = x[k];
+        __syncthreads();
+        // round 2: hi = h2*32 + k*4 + l2, local stages 3,4,5
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * 16 + col];
+        fwd_round3(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * 16 + col] = x[k];
+        __syncthreads();
+        // round 3: hi = sub*8 + k, local stages 6,7
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[(sub * 8 + k) * 16 + col];
+        fwd_round2(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) p[(size_t)(sub * 8 + k) * 256 + col] = x[k];  // lazily reduced, < 4q
+    } else {
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = p[(size_t)(sub * 8 + k) * 256 + col];  // < 2q from the contiguous kernel
+        inv_round2(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[(sub * 8 + k) * 16 + col] = x[k];
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * 16 + col];
+        inv_round3(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * 16 + col] = x[k];
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[(k * 32 + sub) * 16 + col];
+        // stages 2,1 then the last stage with N^-1 folded in
+        {
+#pragma unroll
+            for (int k = 0; k < 4; k++) {
+                Tw c = ldtw(tw, 4 + k);
+                gs_bfly(x[2 * k], x[2 * k + 1], c, q, q2);
+            }
+            Tw b0 = ldtw(tw, 2), b1 = ldtw(tw, 3);
+            gs_bfly(x[0], x[2], b0, q, q2);
+            gs_bfly(x[1], x[3], b0, q, q2);
+            gs_bfly(x[4], x[6], b1, q, q2);
+            gs_bfly(x[5], x[7], b1, q, q2);
+#pragma unroll
+            for (int k = 0; k < 4; k++) {
+                u64 u = x[k], v = x[k + 4];
+                x[k] = shoup(u + v, pc.ninv, pc.ninvs, q);
+                x[k + 4] = shoup(u - v + q2, pc.ninvw, pc.ninvws, q);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 8; k++) p[(size_t)(k * 32 + sub) * 256 + col] = x[k];
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// N = 2^16, contiguous kernel (stages 8..15 forward / the first 8 stages inverse).
+// grid = (16 tiles of 4096 points, rows); block = 512 threads = 16 warps, one 256-point block each.
+// Shared exchange buffer per warp: 256 points padded to e + (e >> 3) to avoid bank conflicts.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t pad8(uint32_t e) { return e + (e >> 3); }
+
+template <bool INV>
+__global__ void __launch_bounds__(512) ntt16_contig(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
+                                                    const PrimeConst* __restrict__ pcs, RowMap map) {
+    const uint32_t row = blockIdx.y;
+    const uint32_t pi = map.prime[row % map.period];
+    if (pi == 0xFF) return;
+    __shared__ u64 sm_all[16 * 288];
+    const PrimeConst pc = pcs[pi];
+    const u64 q = pc.q, q2 = 2 * pc.q;
+    const ulonglong2* tw = tw_all + (size_t)pi * N16;
+    const uint32_t warp = threadIdx.x >> 5, sub = threadIdx.x & 31;
+    const uint32_t blk = blockIdx.x * 16 + warp;   // 256-point block index within the limb
+    const uint32_t pre = 256 + blk;
+    u64* p = data + (size_t)row * N16 + (size_t)blk * 256;
+    u64* sm = sm_all + warp * 288;
+    const uint32_t h2 = sub >> 2, l2 = sub & 3;
+    u64 x[8];
+    if (!INV) {
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = p[k * 32 + sub];   // < 4q from the strided kernel
+        fwd_round3(x, tw, pre, 2 * pre, 4 * pre, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[pad8(k * 32 + sub)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[pad8(h2 * 32 + k * 4 + l2)];
+        fwd_round3(x, tw, 8 * pre + h2, 16 * pre + 2 * h2, 32 * pre + 4 * h2, q, q2);
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[pad8(h2 * 32 + k * 4 + l2)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[pad8(sub * 8 + k)];
+        fwd_round2(x, tw, 64 * pre + 2 * sub, 128 * pre + 4 * sub, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = csub(csub(x[k], q2), q);
+        ulonglong2* o = reinterpret_cast<ulonglong2*>(p + sub * 8);
+#pragma unroll
+        for (int k = 0; k < 4; k++) o[k] = make_ulonglong2(x[2 * k], x[2 * k + 1]);
+    } else {
+        const ulonglong2* in = reinterpret_cast<const ulonglong2*>(p + sub * 8);
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+            ulonglong2 v = in[k];
+            x[2 * k] = v.x;
+            x[2 * k + 1] = v.y;
+        }
+        inv_round2(x, tw, 64 * pre + 2 * sub, 128 * pre + 4 * sub, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[pad8(sub * 8 + k)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[pad8(h2 * 32 + k * 4 + l2)];
+        inv_round3(x, tw, 8 * pre + h2, 16 * pre + 2 * h2, 32 * pre + 4 * h2, q, q2);
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[pad8(h2 * 32 + k * 4 + l2)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[pad8(k * 32 + sub)];
+        inv_round3(x, tw, pre, 2 * pre, 4 * pre, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) p[k * 32 + sub] = x[k];   // < 2q, finished by the strided kernel
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// N <= 2^12: one CTA per row, radix-2 stages in shared memory.
+// ---------------------------------------------------------------------------------------
+template <bool INV>
+__global__ void __launch_bounds__(256) ntt_small(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
+                                                 const PrimeConst* __restrict__ pcs, RowMap map, uint32_t log_n) {
+    const uint32_t row = blockIdx.x;
+    const uint32_t pi = map.prime[row % map.period];
+    if (pi == 0xFF) return;
+    extern __shared__ u64 smx[];
+    const uint32_t N = 1u << log_n;
+    const PrimeConst pc = pcs[pi];
+    const u64 q = pc.q, q2 = 2 * pc.q;
+    const ulonglong2* tw = tw_all + (size_t)pi * N;
+    u64* p = data + (size_t)row * N;
+    for (uint32_t i = threadIdx.x; i < N; i += blockDim.x) smx[i] = p[i];
+    __syncthreads();
+    if (!INV) {
+        for (uint32_t s = 0; s < log_n; s++) {
+            const uint32_t t = N >> (s + 1);
+            for (uint32_t b = threadIdx.x; b < N / 2; b += blockDim.x) {
+                uint32_t i = b / t, k = b % t;
+                uint32_t j = i * 2 * t + k;
+                Tw w = ldtw(tw, (1u << s) + i);
+                u64 x = smx[j], y = smx[j + t];
+                ct_bfly(x, y, w, q, q2);
+                smx[j] = x;
+                smx[j + t] = y;
+            }
+            __syncthreads();
+        }
+        for (uint32_t i = threadIdx.x; i < N; i += blockDim.x) p[i] = csub(csub(smx[i], q2), q);
+    } else {
+        for (int s = (int)log_n - 1; s >= 1; s--) {
+            const uint32_t t = N >> (s + 1);
+            for (uint32_t b = threadIdx.x; b < N / 2; b += blockDim.x) {
+                uint32_t i = b / t, k = b % t;
+                uint32_t j = i * 2 * t + k;
+                Tw w = ldtw(tw, (1u << s) + i);
+                u64 x = smx[j], y = smx[j + t];
+                gs_bfly(x, y, w, q, q2);
+                smx[j] = x;
+                smx[j + t] = y;
+            }
+            __syncthreads();
+        }
+        const uint32_t t = N / 2;
+        for (uint32_t b = threadIdx.x; b < N / 2; b += blockDim.x) {
+            u64 u = smx[b], v = smx[b + t];
+            p[b] = shoup(u + v, pc.ninv, pc.ninvs, q);
+            p[b + t] = shoup(u - v + q2, pc.ninvw, pc.ninvws, q);
+        }
+    }
+}
+
+int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool inverse, cudaStream_t st) {
+    if (rows == 0) return FESC_OK;
+    if (rows > 0x7fffffffu) return fesc_fail(ctx, FESC_EINVAL, "ntt: too many rows");
+    const ulonglong2* tw = inverse ? ctx->d_itw : ctx->d_tw;
+    size_t live = 0;
+    for (uint32_t i = 0; i < map.period; i++) live += map.prime[i] != 0xFF;
+    ctx->counters[0] += rows / map.period * live;
+    if (ctx->log_n == 16) {
+        // gridDim.y is limited to 65535 rows per launch
+        for (size_t r0 = 0; r0 < rows;) {
+            size_t chunk = rows - r0;
+            size_t lim = 65535 / map.period * map.period;
+            if (lim == 0) return fesc_fail(ctx, FESC_EINVAL, "ntt: row map period too large");
+            if (chunk > lim) chunk = lim;
+            dim3 grid(16, (unsigned)chunk);
+            u64* base = d_data + r0 * (size_t)N16;
+            if (!inverse) {
+                ntt16_strided<false><<<grid, 512, 0, st>>>(base, tw, ctx->d_pc, map);
+                ntt16_contig<false><<<grid, 512, 0, st>>>(base, tw, ctx->d_pc, map);
+            } else {
+                ntt16_contig<true><<<grid, 512, 0, st>>>(base, tw, ctx->d_pc, map);
+                ntt16_strided<true><<<grid, 512, 0, st>>>(base, tw, ctx->d_pc, map);
+            }
+            r0 += chunk;
+        }
+    } else {
+        size_t smem = sizeof(u64) << ctx->log_n;
+        if (!inverse)
+            ntt_small<false><<<(unsigned)rows, 256, smem, st>>>(d_data, tw, ctx->d_pc, map, ctx->log_n);
+        else
+            ntt_small<true><<<(unsigned)rows, 256, smem, st>>>(d_data, tw, ctx->d_pc, map, ctx->log_n);
+    }
+    FESC_CHECK_CUDA(ctx, cudaGetLastError());
+    return FESC_OK;
+}

@@ -1,0 +1,477 @@
+// Ciphertext operations: ct-pt MAC, Galois automorphism, hybrid key switch, rotation,
+// rescale, ct x ct.  Every kernel streams limb rows of N words with coalesced accesses;
+// products of two data words are accumulated lazily in 128 bits and reduced once.
+#include "ops.cuh"
+
+// ---------------------------------------------------------------------------------------
+// ct-pt multiply-accumulate:  acc[b][p][l][c] += ct[b][p][l][c] * pt[b][l][c]
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_ct_pt_mac(const u64* __restrict__ ct, const u64* __restrict__ pt, size_t pt_stride,
+                                                   u64* __restrict__ acc, const PrimeConst* __restrict__ pcs,
+                                                   uint32_t N, uint32_t n_limbs) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t l = blockIdx.y, b = blockIdx.z;
+    if (c >= N) return;
+    const PrimeConst pc = pcs[l];
+    const size_t poly = (size_t)n_limbs * N;
+    const size_t o = (size_t)b * 2 * poly + (size_t)l * N + c;
+    const u64 w = pt[(size_t)b * pt_stride + (size_t)l * N + c];
+#pragma unroll
+    for (int p = 0; p < 2; p++) {
+        acc128 a{acc[o + p * poly], 0};
+        mac128(a, ct[o + p * poly], w);
+        acc[o + p * poly] = reduce128(a.hi, a.lo, pc);
+    }
+}
+
+extern "C" int fesc_ct_pt_mac(fesc_ctx* ctx, const uint64_t* d_ct, const uint64_t* d_pt, size_t pt_stride,
+                              uint64_t* d_acc, uint32_t batch, uint32_t n_limbs, void* stream) {
+    if (!ctx || !d_ct || !d_pt || !d_acc) return FESC_EINVAL;
+    if (n_limbs == 0 || n_limbs > ctx->n_q) return fesc_fail(ctx, FESC_ELEVEL, "ct_pt_mac: level out of range");
+    if (batch == 0) return FESC_OK;
+    if (batch > 65535) return fesc_fail(ctx, FESC_EINVAL, "ct_pt_mac: batch too large");
+    dim3 grid((ctx->N + 255) / 256, n_limbs, batch);
+    k_ct_pt_mac<<<grid, 256, 0, (cudaStream_t)stream>>>((const u64*)d_ct, (const u64*)d_pt, pt_stride, (u64*)d_acc,
+                                                        ctx->d_pc, ctx->N, n_limbs);
+    FESC_CHECK_CUDA(ctx, cudaGetLastError());
+    ctx->counters[2] += batch;
+    return FESC_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// NTT entry points
+// ---------------------------------------------------------------------------------------
+static int ntt_api(fesc_ctx* ctx, uint64_t* d_data, uint32_t batch, uint32_t first_limb, uint32_t n_limbs,
+                   void* stream, bool inv) {
+    if (!ctx || !d_data) return FESC_EINVAL;
+    if (n_limbs == 0 || first_limb + n_limbs > ctx->n_primes || n_limbs > sizeof(RowMap::prime))
+        return fesc_fail(ctx, FESC_EINVAL, "ntt: limb range out of bounds");
+    RowMap map;
+    map.period = n_limbs;
+    for (uint32_t i = 0; i < n_limbs; i++) map.prime[i] = (uint8_t)(first_limb + i);
+    return ntt_launch(ctx, (u64*)d_data, (size_t)batch * n_limbs, map, inv, (cudaStream_t)stream);
+}
+extern "C" int fesc_ntt(fesc_ctx* ctx, uint64_t* d_data, uint32_t batch, uint32_t first_limb, uint32_t n_limbs,
+                        void* stream) {
+    return ntt_api(ctx, d_data, batch, first_limb, n_limbs, stream, false);
+}
+extern "C" int fesc_intt(fesc_ctx* ctx, uint64_t* d_data, uint32_t batch, uint32_t first_limb, uint32_t n_limbs,
+                         void* stream) {
+    return ntt_api(ctx, d_data, batch, first_limb, n_limbs, stream, true);
+}
+
+// ---------------------------------------------------------------------------------------
+// Galois automorphism in evaluation order: out[t] = in[pi_g(t)],
+// pi_g(t) = brev(((2 brev(t) + 1) g mod 2N - 1) / 2).  Aligned blocks map to aligned blocks,
+// so a warp reading 32 consecutive t touches one 256-byte block of the source.
+// c0 goes to out0 (the result's first polynomial), c1 goes to BOTH d (kept in EVAL form for
+// the digit's own limbs) and dcoef (transformed in place afterwards).
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t galois_src(uint32_t t, uint32_t log_n, u64 g) {
+    uint32_t u = __brev(t) >> (32 - log_n);
+    uint32_t e = (uint32_t)(((2ull * u + 1) * g) & ((2ull << log_n) - 1));
+    return __brev((e - 1) >> 1) >> (32 - log_n);
+}
+__global__ void __launch_bounds__(256) k_autom_ct(const u64* __restrict__ in, size_t in_stride, u64* __restrict__ out0,
+                                                  size_t out_stride, u64* __restrict__ d, u64* __restrict__ dcoef,
+                                                  uint32_t log_n, uint32_t level, u64 g,
+                                                  const PrimeConst* __restrict__ pcs, int accumulate) {
+    const uint32_t N = 1u << log_n;
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t l = blockIdx.y, b = blockIdx.z;
+    if (t >= N) return;
+    const uint32_t src = galois_src(t, log_n, g);
+    const u64* ib = in + (size_t)b * in_stride;
+    const size_t poly = (size_t)level * N;
+    u64* o0 = out0 + (size_t)b * out_stride + (size_t)l * N + t;
+    u64 v0 = ib[(size_t)l * N + src];
+    if (accumulate) v0 = addmod(v0, *o0, pcs[l].q);
+    *o0 = v0;
+    u64 v = ib[poly + (size_t)l * N + src];
+    const size_t o = ((size_t)b * level + l) * N + t;
+    d[o] = v;
+    dcoef[o] = v;
+}
+
+// ---------------------------------------------------------------------------------------
+// ModUp: per digit j, uncorrected fast basis conversion of the digit's COEFF residues to every
+// other active modulus and to the special moduli.
+//   y_a = d_a * (Q_j/q_a)^-1 mod q_a   (canonical)
+//   ext[b][j][t] = sum_a y_a * ((Q_j/q_a) mod q_t) mod q_t
+// ext row order: data limbs 0..level-1 then the K special limbs; rows of the digit's own limbs
+// are left untouched (the inner product reads those from the EVAL-form input).
+// ---------------------------------------------------------------------------------------
+template <int ALPHA>
+__global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u64* __restrict__ ext,
+                                               const ModUpDigit* __restrict__ tab, const PrimeConst* __restrict__ pcs,
+                                               uint32_t N, uint32_t level, uint32_t n_q, uint32_t K, uint32_t beta) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t j = blockIdx.y, b = blockIdx.z;
+    if (c >= N) return;
+    const ModUpDigit* dg = tab + j;
+    const uint32_t first = dg->first, n_src = dg->n_src;
+    u64 y[ALPHA];
+#pragma unroll
+    for (int a = 0; a < ALPHA; a++) {
+        y[a] = 0;
+        if (a < n_src) {
+            u64 v = dcoef[((size_t)b * level + first + a) * N + c];
+            y[a] = shoup(v, dg->inv[a], dg->invs[a], pcs[first + a].q);
+        }
+    }
+    const uint32_t rows = level + K;
+    u64* out = ext + ((size_t)b * beta + j) * rows * N + c;
+    for (uint32_t t = 0; t < rows; t++) {
+        if (t >= first && t < first + n_src) continue;
+        const uint32_t pt = t < level ? t : n_q + (t - level);
+        acc128 acc{0, 0};
+#pragma unroll
+        for (int a = 0; a < ALPHA; a++)
+            if (a < n_src) mac128(acc, y[a], dg->mat[a][pt]);
+        out[(size_t)t * N] = reduce128(acc.hi, acc.lo, pcs[pt]);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Inner product with the switching key over all level+K moduli:
+//   acc[b][p][t] = sum_j dt_j[b][t] * key[j][p][t],   dt_j[t] = d[b][t] if t is in digit j, else ext[b][j][t].
+// One thread owns one (coefficient, modulus) and BT ciphertexts, so a key word is loaded once
+// for BT products.
+// ---------------------------------------------------------------------------------------
+template <int BT>
+__global__ void __launch_bounds__(256) k_inner(const u64* __restrict__ d, const u64* __restrict__ ext,
+                                               const u64* __restrict__ key, u64* __restrict__ acc,
+                                               const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
+                                               uint32_t n_q, uint32_t K, uint32_t alpha, uint32_t beta,
+                                               uint32_t batch) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t t = blockIdx.y, b0 = blockIdx.z * BT;
+    if (c >= N) return;
+    const uint32_t rows = level + K, np = n_q + K;
+    const uint32_t pt = t < level ? t : n_q + (t - level);
+    const uint32_t own = t < level ? t / alpha : 0xFFFFFFFFu;
+    acc128 a0[BT], a1[BT];
+#pragma unroll
+    for (int i = 0; i < BT; i++) a0[i] = a1[i] = acc128{0, 0};
+    for (uint32_t j = 0; j < beta; j++) {
+        const u64 kb = __ldg(key + ((size_t)(2 * j) * np + pt) * N + c);
+        const u64 ka = __ldg(key + ((size_t)(2 * j + 1) * np + pt) * N + c);
+#pragma unroll
+        for (int i = 0; i < BT; i++) {
+            const uint32_t b = b0 + i;
+            if (b < batch) {
+                u64 x = (j == own) ? d[((size_t)b * level + t) * N + c] : ext[(((size_t)b * beta + j) * rows + t) * N + c];
+                mac128(a0[i], x, kb);
+                mac128(a1[i], x, ka);
+            }
+        }
+    }
+    const PrimeConst pc = pcs[pt];
+#pragma unroll
+    for (int i = 0; i < BT; i++) {
+        const uint32_t b = b0 + i;
+        if (b < batch) {
+            acc[(((size_t)b * 2 + 0) * rows + t) * N + c] = reduce128(a0[i].hi, a0[i].lo, pc);
+            acc[(((size_t)b * 2 + 1) * rows + t) * N + c] = reduce128(a1[i].hi, a1[i].lo, pc);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Division by P, conversion step: special-limb residues (COEFF) -> u[b][p][i] (COEFF, data limbs)
+//   y_k = r_k * (P/p_k)^-1 mod p_k, taken in [-(p_k-1)/2, (p_k-1)/2];
+//   u_i = sum_k y_k (P/p_k) mod q_i = sum_k [y_k]_canonical (P/p_k) - #{y_k > p_k/2} * P  (mod q_i).
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_moddown_conv(const u64* __restrict__ acc, u64* __restrict__ u,
+                                                      const ModDownTab* __restrict__ tab,
+                                                      const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
+                                                      uint32_t n_q, uint32_t K) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t bp = blockIdx.y;   // b*2 + p
+    if (c >= N) return;
+    const uint32_t rows = level + K;
+    u64 y[FESC_MAX_SPECIAL];
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int k = 0; k < FESC_MAX_SPECIAL; k++) {
+        y[k] = 0;
+        if (k < K) {
+            u64 r = acc[((size_t)bp * rows + level + k) * N + c];
+            y[k] = shoup(r, tab->inv[k], tab->invs[k], pcs[n_q + k].q);
+            cnt += y[k] > tab->half[k];
+        }
+    }
+    for (uint32_t i = 0; i < level; i++) {
+        acc128 a{0, 0};
+#pragma unroll
+        for (int k = 0; k < FESC_MAX_SPECIAL; k++)
+            if (k < K) mac128(a, y[k], tab->mat[k][i]);
+        u64 v = reduce128(a.hi, a.lo, pcs[i]);
+        u[((size_t)bp * level + i) * N + c] = submod(v, tab->wrap[cnt][i], pcs[i].q);
+    }
+}
+
+// out[b][p][i] = (acc[b][p][i] - u[b][p][i]) * P^-1 + add[b][p][i]   (all EVAL)
+__global__ void __launch_bounds__(256) k_moddown_finish(const u64* __restrict__ acc, const u64* __restrict__ u,
+                                                        u64* __restrict__ out, size_t out_stride,
+                                                        const ModDownTab* __restrict__ tab,
+                                                        const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
+                                                        uint32_t K, int add_mask) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t i = blockIdx.y, bp = blockIdx.z;
+    if (c >= N) return;
+    const uint32_t b = bp >> 1, p = bp & 1;
+    const u64 q = pcs[i].q;
+    u64 v = submod(acc[((size_t)bp * (level + K) + i) * N + c], u[((size_t)bp * level + i) * N + c], q);
+    v = shoup(v, tab->pinv[i], tab->pinvs[i], q);
+    u64* o = out + (size_t)b * out_stride + ((size_t)p * level + i) * N + c;
+    if ((add_mask >> p) & 1) v = addmod(v, *o, q);
+    *o = v;
+}
+
+// Hybrid key switch of `batch` polynomials d[b] ([level][N], EVAL, contiguous) with scratch
+// dcoef (a copy of d, consumed), ext, acc, u.  Result is ADDED to out[b][p] when bit p of
+// add_mask is set, else stored.
+static int key_switch_chunk(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint32_t level, uint32_t batch,
+                            u64* out, size_t out_stride, int add_mask, cudaStream_t st) {
+    const uint32_t N = ctx->N, K = ctx->n_p, nq = ctx->n_q, alpha = ctx->alpha;
+    const uint32_t beta = (level + alpha - 1) / alpha, rows = level + K;
+    const uint32_t gx = (N + 255) / 256;
+    int rc;
+    RowMap m;
+    // 1. d -> COEFF
+    m.period = level;
+    for (uint32_t i = 0; i < level; i++) m.prime[i] = (uint8_t)i;
+    if ((rc = ntt_launch(ctx, ws.dcoef, (size_t)batch * level, m, true, st)) != FESC_OK) return rc;
+    // 2. ModUp
+    const ModUpDigit* tab = ctx->tabs.d_modup + (size_t)(level - 1) * ctx->beta_max;
+    dim3 gmu(gx, beta, batch);
+#define MODUP(A) k_modup<A><<<gmu, 256, 0, st>>>(ws.dcoef, ws.ext, tab, ctx->d_pc, N, level, nq, K, beta)
+    if (alpha <= 1) MODUP(1);
+    else if (alpha <= 2) MODUP(2);
+    else if (alpha <= 4) MODUP(4);
+    else if (alpha <= 6) MODUP(6);
+    else MODUP(8);
+#undef MODUP
+    // 3. NTT of the converted rows
+    if (beta * rows > sizeof(RowMap::prime)) return fesc_fail(ctx, FESC_EINVAL, "key switch: too many digit rows");
+    m.period = beta * rows;
+    for (uint32_t j = 0; j < beta; j++)
+        for (uint32_t t = 0; t < rows; t++) {
+            bool own = t < level && t / alpha == j;
+            m.prime[j * rows + t] = own ? 0xFF : (uint8_t)(t < level ? t : nq + (t - level));
+        }
+    if ((rc = ntt_launch(ctx, ws.ext, (size_t)batch * beta * rows, m, false, st)) != FESC_OK) return rc;
+    // 4. inner product with the key
+    if (batch >= 4) {
+        dim3 g(gx, rows, (batch + 3) / 4);
+        k_inner<4><<<g, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch);
+    } else if (batch >= 2) {
+        dim3 g(gx, rows, (batch + 1) / 2);
+        k_inner<2><<<g, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch);
+    } else {
+        dim3 g(gx, rows, 1);
+        k_inner<1><<<g, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch);
+    }
+    // 5. division by P
+    m.period = rows;
+    for (uint32_t t = 0; t < rows; t++) m.prime[t] = t < level ? 0xFF : (uint8_t)(nq + (t - level));
+    if ((rc = ntt_launch(ctx, ws.acc, (size_t)batch * 2 * rows, m, true, st)) != FESC_OK) return rc;
+    k_moddown_conv<<<dim3(gx, batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K);
+    m.period = level;
+    for (uint32_t i = 0; i < level; i++) m.prime[i] = (uint8_t)i;
+    if ((rc = ntt_launch(ctx, ws.u, (size_t)batch * 2 * level, m, false, st)) != FESC_OK) return rc;
+    k_moddown_finish<<<dim3(gx, level, batch * 2), 256, 0, st>>>(ws.acc, ws.u, out, out_stride, ctx->tabs.d_moddown,
+                                                                 ctx->d_pc, N, level, K, add_mask);
+    FESC_CHECK_CUDA(ctx, cudaGetLastError());
+    ctx->counters[1] += batch;
+    return FESC_OK;
+}
+
+size_t ks_scratch_words(const fesc_ctx* ctx, uint32_t level, uint32_t chunk) {
+    const uint32_t beta = (level + ctx->alpha - 1) / ctx->alpha, rows = level + ctx->n_p;
+    return (size_t)chunk * ctx->N * ((size_t)2 * level + (size_t)beta * rows + 2 * rows + 2 * level);
+}
+KsScratch ks_scratch_carve(const fesc_ctx* ctx, u64* base, uint32_t level, uint32_t chunk) {
+    const uint32_t beta = (level + ctx->alpha - 1) / ctx->alpha, rows = level + ctx->n_p;
+    const size_t N = ctx->N;
+    KsScratch ws;
+    ws.d = base;
+    ws.dcoef = ws.d + (size_t)chunk * level * N;
+    ws.ext = ws.dcoef + (size_t)chunk * level * N;
+    ws.acc = ws.ext + (size_t)chunk * beta * rows * N;
+    ws.u = ws.acc + (size_t)chunk * 2 * rows * N;
+    return ws;
+}
+
+uint32_t ks_chunk(const fesc_ctx* ctx, uint32_t batch) {
+    uint32_t c = ctx->log_n == 16 ? 8 : 64;
+    return batch < c ? batch : c;
+}
+
+// Rotation of `batch` ciphertexts with strides (words) between consecutive inputs / outputs.
+// accumulate != 0: the rotated ciphertext is ADDED to what `out` holds.
+int rotate_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, size_t out_stride, uint32_t batch,
+                    uint32_t level, uint32_t key_id, u64* scratch, cudaStream_t st, int accumulate) {
+    auto it = ctx->keys.find(key_id);
+    if (it == ctx->keys.end() || key_id == FESC_RELIN_KEY_ID)
+        return fesc_fail(ctx, FESC_ENOKEY, "rotate: no Galois key " + std::to_string(key_id));
+    const uint32_t chunk = ks_chunk(ctx, batch);
+    KsScratch ws = ks_scratch_carve(ctx, scratch, level, chunk);
+    for (uint32_t b0 = 0; b0 < batch; b0 += chunk) {
+        uint32_t nb = batch - b0 < chunk ? batch - b0 : chunk;
+        dim3 g((ctx->N + 255) / 256, level, nb);
+        k_autom_ct<<<g, 256, 0, st>>>(in + (size_t)b0 * in_stride, in_stride, out + (size_t)b0 * out_stride, out_stride,
+                                      ws.d, ws.dcoef, ctx->log_n, level, it->second.g, ctx->d_pc, accumulate);
+        int rc = key_switch_chunk(ctx, ws, it->second, level, nb, out + (size_t)b0 * out_stride, out_stride,
+                                  accumulate ? 3 : 1, st);
+        if (rc != FESC_OK) return rc;
+    }
+    return FESC_OK;
+}
+
+extern "C" int fesc_rotate(fesc_ctx* ctx, const uint64_t* d_in, uint64_t* d_out, uint32_t batch, uint32_t n_limbs,
+                           uint32_t key_id, void* stream) {
+    if (!ctx || !d_in || !d_out) return FESC_EINVAL;
+    if (n_limbs == 0 || n_limbs > ctx->n_q) return fesc_fail(ctx, FESC_ELEVEL, "rotate: level out of range");
+    if (batch == 0) return FESC_OK;
+    u64* scratch;
+    int rc = ctx_scratch(ctx, ks_scratch_words(ctx, n_limbs, ks_chunk(ctx, batch)) * sizeof(u64), &scratch);
+    if (rc != FESC_OK) return rc;
+    const size_t stride = (size_t)2 * n_limbs * ctx->N;
+    return rotate_internal(ctx, (const u64*)d_in, stride, (u64*)d_out, stride, batch, n_limbs, key_id, scratch,
+                           (cudaStream_t)stream, 0);
+}
+
+// ---------------------------------------------------------------------------------------
+// Rescale
+// ---------------------------------------------------------------------------------------
+// gather the last limb of every polynomial into r[b*2+p][N]
+__global__ void __launch_bounds__(256) k_take_last(const u64* __restrict__ in, size_t in_stride, u64* __restrict__ r,
+                                                   uint32_t N, uint32_t level) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t bp = blockIdx.y;
+    if (c >= N) return;
+    r[(size_t)bp * N + c] = in[(size_t)(bp >> 1) * in_stride + ((size_t)(bp & 1) * level + level - 1) * N + c];
+}
+// out[b][p][i] = centred(r) mod q_i  (COEFF)
+__global__ void __launch_bounds__(256) k_rescale_conv(const u64* __restrict__ r, u64* __restrict__ out, size_t out_stride,
+                                                      const RescaleTab* __restrict__ tab,
+                                                      const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t i = blockIdx.y, bp = blockIdx.z;
+    if (c >= N) return;
+    const u64 v = r[(size_t)bp * N + c];
+    const PrimeConst pc = pcs[i];
+    u64 w = v - mulhi(v, pc.mu) * pc.q;   // v mod q_i in [0, 2q)
+    w = csub(w, pc.q);
+    if (v > tab->half) w = submod(w, tab->wrap[i], pc.q);
+    out[(size_t)(bp >> 1) * out_stride + ((size_t)(bp & 1) * (level - 1) + i) * N + c] = w;
+}
+// out = (in - out) * q_last^-1
+__global__ void __launch_bounds__(256) k_rescale_finish(const u64* __restrict__ in, size_t in_stride,
+                                                        u64* __restrict__ out, size_t out_stride,
+                                                        const RescaleTab* __restrict__ tab,
+                                                        const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t i = blockIdx.y, bp = blockIdx.z;
+    if (c >= N) return;
+    const u64 q = pcs[i].q;
+    u64* o = out + (size_t)(bp >> 1) * out_stride + ((size_t)(bp & 1) * (level - 1) + i) * N + c;
+    u64 x = in[(size_t)(bp >> 1) * in_stride + ((size_t)(bp & 1) * level + i) * N + c];
+    *o = shoup(submod(x, *o, q), tab->qinv[i], tab->qinvs[i], q);
+}
+
+// out must be a contiguous batch [batch][2][level-1][N]; scratch holds batch*2*N words.
+int rescale_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, uint32_t batch, uint32_t level,
+                     u64* scratch, cudaStream_t st) {
+    const uint32_t N = ctx->N, gx = (N + 255) / 256;
+    const size_t out_stride = (size_t)2 * (level - 1) * N;
+    const RescaleTab* tab = ctx->tabs.d_rescale + level;
+    int rc;
+    for (uint32_t b0 = 0; b0 < batch; b0 += 16384) {
+        uint32_t nb = batch - b0 < 16384 ? batch - b0 : 16384;
+        const u64* ib = in + (size_t)b0 * in_stride;
+        u64* ob = out + (size_t)b0 * out_stride;
+        k_take_last<<<dim3(gx, nb * 2), 256, 0, st>>>(ib, in_stride, scratch, N, level);
+        RowMap m;
+        m.period = 1;
+        m.prime[0] = (uint8_t)(level - 1);
+        if ((rc = ntt_launch(ctx, scratch, (size_t)nb * 2, m, true, st)) != FESC_OK) return rc;
+        k_rescale_conv<<<dim3(gx, level - 1, nb * 2), 256, 0, st>>>(scratch, ob, out_stride, tab, ctx->d_pc, N, level);
+        m.period = level - 1;
+        for (uint32_t i = 0; i + 1 < level; i++) m.prime[i] = (uint8_t)i;
+        if ((rc = ntt_launch(ctx, ob, (size_t)nb * 2 * (level - 1), m, false, st)) != FESC_OK) return rc;
+        k_rescale_finish<<<dim3(gx, level - 1, nb * 2), 256, 0, st>>>(ib, in_stride, ob, out_stride, tab, ctx->d_pc, N,
+                                                                    level);
+    }
+    FESC_CHECK_CUDA(ctx, cudaGetLastError());
+    return FESC_OK;
+}
+
+extern "C" int fesc_rescale(fesc_ctx* ctx, const uint64_t* d_in, uint64_t* d_out, uint32_t batch, uint32_t n_limbs,
+                            void* stream) {
+    if (!ctx || !d_in || !d_out) return FESC_EINVAL;
+    if (n_limbs < 2 || n_limbs > ctx->n_q) return fesc_fail(ctx, FESC_ELEVEL, "rescale: level out of range");
+    if (batch == 0) return FESC_OK;
+    u64* scratch;
+    uint32_t nb = batch < 16384 ? batch : 16384;
+    int rc = ctx_scratch(ctx, (size_t)nb * 2 * ctx->N * sizeof(u64), &scratch);
+    if (rc != FESC_OK) return rc;
+    return rescale_internal(ctx, (const u64*)d_in, (size_t)2 * n_limbs * ctx->N, (u64*)d_out, batch, n_limbs, scratch,
+                            (cudaStream_t)stream);
+}
+
+// ---------------------------------------------------------------------------------------
+// ct x ct: tensor product, then relinearisation of d2
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_tensor(const u64* __restrict__ a, size_t a_stride, const u64* __restrict__ bb,
+                                                size_t b_stride, u64* __restrict__ out, size_t out_stride,
+                                                u64* __restrict__ d, u64* __restrict__ dcoef,
+                                                const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t l = blockIdx.y, b = blockIdx.z;
+    if (c >= N) return;
+    const PrimeConst pc = pcs[l];
+    const size_t poly = (size_t)level * N, o = (size_t)l * N + c;
+    const u64 a0 = a[b * a_stride + o], a1 = a[b * a_stride + poly + o];
+    const u64 b0 = bb[b * b_stride + o], b1 = bb[b * b_stride + poly + o];
+    out[b * out_stride + o] = mulmod(a0, b0, pc);
+    acc128 s{0, 0};
+    mac128(s, a0, b1);
+    mac128(s, a1, b0);
+    out[b * out_stride + poly + o] = reduce128(s.hi, s.lo, pc);
+    const u64 d2 = mulmod(a1, b1, pc);
+    const size_t od = ((size_t)b * level + l) * N + c;
+    d[od] = d2;
+    dcoef[od] = d2;
+}
+
+int ctmul_internal(fesc_ctx* ctx, const u64* a, size_t a_stride, const u64* b, size_t b_stride, u64* out,
+                   size_t out_stride, uint32_t batch, uint32_t level, u64* scratch, cudaStream_t st) {
+    const EvalKey& key = ctx->keys[FESC_RELIN_KEY_ID];
+    const uint32_t chunk = ks_chunk(ctx, batch);
+    KsScratch ws = ks_scratch_carve(ctx, scratch, level, chunk);
+    for (uint32_t b0 = 0; b0 < batch; b0 += chunk) {
+        uint32_t nb = batch - b0 < chunk ? batch - b0 : chunk;
+        dim3 g((ctx->N + 255) / 256, level, nb);
+        k_tensor<<<g, 256, 0, st>>>(a + (size_t)b0 * a_stride, a_stride, b + (size_t)b0 * b_stride, b_stride,
+                                    out + (size_t)b0 * out_stride, out_stride, ws.d, ws.dcoef, ctx->d_pc, ctx->N, level);
+        int rc = key_switch_chunk(ctx, ws, key, level, nb, out + (size_t)b0 * out_stride, out_stride, 3, st);
+        if (rc != FESC_OK) return rc;
+    }
+    return FESC_OK;
+}
+
+extern "C" int fesc_ct_ct_mul(fesc_ctx* ctx, const uint64_t* d_a, const uint64_t* d_b, uint64_t* d_out, uint32_t batch,
+                              uint32_t n_limbs, void* stream) {
+    if (!ctx || !d_a || !d_b || !d_out) return FESC_EINVAL;
+    if (n_limbs == 0 || n_limbs > ctx->n_q) return fesc_fail(ctx, FESC_ELEVEL, "ct_ct_mul: level out of range");
+    if (batch == 0) return FESC_OK;
+    u64* scratch;
+    int rc = ctx_scratch(ctx, ks_scratch_words(ctx, n_limbs, ks_chunk(ctx, batch)) * sizeof(u64), &scratch);
+    if (rc != FESC_OK) return rc;
+    const size_t stride = (size_t)2 * n_limbs * ctx->N;
+    return ctmul_internal(ctx, (const u64*)d_a, stride, (const u64*)d_b, stride, (u64*)d_out, stride, batch, n_limbs,
+                          scratch, (cudaStream_t)stream);
+}

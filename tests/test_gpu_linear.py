@@ -1,0 +1,85 @@
+"""GPU parity for the BSGS projection: residues equal the oracle's bit for bit, and the decrypted
+result equals X @ W in float64."""
+import numpy as np
+import pytest
+
+import fesc_synth as S
+from oracle.ckks import linear_diagonal, pack_linear_input
+from tests.gpu_util import add_key, ctx_pair, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+def _setup(pair, T, C, n1, n2, tokens, d_in, d_out, level, scale, wscale=1.0, key_base=1000):
+    ctx, orc, p = pair
+    n = orc.n
+    assert C * T == n and n1 * n2 == C
+    X, W = S.linear_inputs(p["seed"] + 4, tokens, d_in, d_out)
+    W = W * wscale
+    gin, nout, tbs = -(-d_in // C), -(-d_out // C), -(-tokens // T)
+    for q in range(1, n1):
+        add_key(pair, q * T, key_base + q)
+    for g in range(1, n2):
+        add_key(pair, g * n1 * T, key_base + 500 + g)
+    cts = np.empty((tbs, gin, 2, level, orc.N), dtype=np.uint64)
+    for tb in range(tbs):
+        for g in range(gin):
+            v = pack_linear_input(X[tb * T:(tb + 1) * T, g * C:(g + 1) * C], T, C, n)
+            cts[tb, g] = orc.encrypt(orc.encode(v, scale, level), 7000 + tb * gin + g)
+    diags = np.empty((nout, n2, gin, n1, level, orc.N), dtype=np.uint64)
+    for b in range(nout):
+        for pp in range(n2):
+            for g in range(gin):
+                for q in range(n1):
+                    diags[b, pp, g, q] = orc.encode(linear_diagonal(W, b, g, pp, q, T, C, n1), float(orc.q[level - 1]), level)
+    return X, W, cts, diags, (gin, nout, tbs)
+
+
+def _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=1000):
+    import torch
+    import paper_2608_17442_b200 as fesc
+
+    gin, nout, tbs = dims
+    desc = fesc.BsgsDesc(n1, n2, gin, nout, tbs, level, key_base, key_base + 500)
+    out = torch.empty((tbs, nout, 2, level - 1, cts.shape[-1]), dtype=torch.int64, device="cuda")
+    ctx.linear(to_dev(cts), to_dev(diags), desc, out)
+    return to_host(out)
+
+
+@pytest.mark.parametrize("shape", [(32, 16, 4, 4, 70, 40, 50, 5), (64, 8, 8, 1, 64, 8, 8, 3), (16, 32, 2, 16, 20, 33, 30, 24)])
+def test_linear_small_ring(shape):
+    T, C, n1, n2, tokens, d_in, d_out, level = shape
+    pair = ctx_pair("small")
+    ctx, orc, _ = pair
+    scale = 2.0**40
+    X, W, cts, diags, dims = _setup(pair, T, C, n1, n2, tokens, d_in, d_out, level, scale, wscale=10.0,
+                                    key_base=1000 + 37 * T)
+    got = _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=1000 + 37 * T)
+    kb = 1000 + 37 * T
+    want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)},
+                      {g: kb + 500 + g for g in range(1, n2)})
+    assert np.array_equal(got, want)
+    gin, nout, tbs = dims
+    Y = np.zeros((tbs * T, nout * C))
+    for tb in range(tbs):
+        for b in range(nout):
+            Y[tb * T:(tb + 1) * T, b * C:(b + 1) * C] = orc.decrypt(got[tb, b], scale, 2).real.reshape(C, T).T
+    assert np.abs(Y[:tokens, :d_out] - X @ W).max() < 2.0**-18
+
+
+def test_linear_full_ring_one_block():
+    """N = 2^16, 24 limbs, scale 2^40: one token block x one output block of the in_proj shape
+    (768 inputs = 3 input blocks, C=256, T=128, n1=32, n2=8); bit-exact and within 2^-18 of X @ W."""
+    pair = ctx_pair("full")
+    ctx, orc, _ = pair
+    T, C, n1, n2, level = 128, 256, 32, 8, 24
+    scale = 2.0**40
+    X, W, cts, diags, dims = _setup(pair, T, C, n1, n2, 128, 768, 256, level, scale, key_base=2000)
+    got = _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=2000)
+    want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: 2000 + q for q in range(1, n1)},
+                      {g: 2500 + g for g in range(1, n2)})
+    assert np.array_equal(got, want)
+    Y = orc.decrypt(got[0, 0], scale, 2).real.reshape(C, T).T
+    err = np.abs(Y - X @ W).max()
+    print("max |decrypt - X@W| = 2^%.2f" % np.log2(err))
+    assert err < 2.0**-18

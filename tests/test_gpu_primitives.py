@@ -1,0 +1,215 @@
+"""GPU parity: key generation, NTT, ct-pt MAC, rotation, rescale and ct x ct must equal the
+oracle's residues bit for bit on the same seeded inputs."""
+import numpy as np
+import pytest
+
+import fesc_synth as S
+from tests.gpu_util import add_key, ctx_pair, random_ct, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name", ["toy", "tiny", "small"])
+def test_keygen_matches_oracle(name):
+    pair = ctx_pair(name)
+    ctx, orc, _ = pair
+    assert np.array_equal(to_host(ctx.export_secret()), orc.s_eval)
+    assert np.array_equal(to_host(ctx.export_key(0)), orc.keys[0][1])
+    add_key(pair, 3, 7)
+    add_key(pair, -(1 << 31), 8)
+    assert np.array_equal(to_host(ctx.export_key(7)), orc.keys[7][1])
+    assert np.array_equal(to_host(ctx.export_key(8)), orc.keys[8][1])
+
+
+@pytest.mark.parametrize("name", ["toy", "tiny", "small"])
+def test_ntt_small_rings(name):
+    ctx, orc, p = ctx_pair(name)
+    idx = list(range(p["n_q"] + p["n_p"]))
+    batch = 3
+    a = np.stack([S.uniform_residues_np(1, b, orc.q, orc.N) for b in range(batch)])
+    d = to_dev(a)
+    ctx.ntt(d, batch, 0, len(idx))
+    want = np.stack([orc.ntt(a[b], idx) for b in range(batch)])
+    assert np.array_equal(to_host(d), want)
+    ctx.intt(d, batch, 0, len(idx))
+    assert np.array_equal(to_host(d), a)
+    # a sub-range of limbs starting at 1, inverse direction against the oracle
+    sub = idx[1:4]
+    b2 = np.ascontiguousarray(a[:, 1:4])
+    d2 = to_dev(b2)
+    ctx.intt(d2, batch, 1, 3)
+    assert np.array_equal(to_host(d2), np.stack([orc.intt(b2[b], sub) for b in range(batch)]))
+
+
+def test_ntt_full_ring_matches_oracle():
+    ctx, orc, p = ctx_pair("full")
+    idx = [0, 7, 23, 24, 27]   # 50-bit and 60-bit primes
+    a = np.stack([S.uniform_residues_np(2, 0, [orc.q[i]], orc.N)[0] for i in idx])
+    for i, pi in enumerate(idx):
+        d = to_dev(a[i:i + 1])
+        ctx.ntt(d, 1, pi, 1)
+        assert np.array_equal(to_host(d)[0], orc.ntt(a[i:i + 1], [pi])[0]), pi
+        ctx.intt(d, 1, pi, 1)
+        assert np.array_equal(to_host(d)[0], a[i])
+        d = to_dev(a[i:i + 1])
+        ctx.intt(d, 1, pi, 1)
+        assert np.array_equal(to_host(d)[0], orc.intt(a[i:i + 1], [pi])[0]), pi
+
+
+def test_ntt_sweep_workload_round_trip():
+    """Workload 2: 64 polynomials x 24 limbs of 50-bit primes at N = 2^16; forward then inverse is the
+    identity bit for bit, and sampled limbs of the forward transform equal the oracle's."""
+    import torch
+
+    ctx, orc, p = ctx_pair("full")
+    x = S.hashed_residues(S.config_seed(2), 0, orc.q[:24], 64 * orc.N, device="cuda")  # [24, 64*N]
+    x = x.view(24, 64, orc.N).permute(1, 0, 2).contiguous()
+    y = x.clone()
+    ctx.ntt(y, 64, 0, 24)
+    for (b, l) in ((0, 0), (17, 5), (63, 23)):
+        assert np.array_equal(to_host(y[b, l]), orc.ntt(to_host(x[b, l])[None], [l])[0])
+    ctx.intt(y, 64, 0, 24)
+    assert torch.equal(x, y)
+
+
+@pytest.mark.parametrize("name,level", [("toy", 6), ("toy", 3), ("tiny", 3), ("small", 24)])
+def test_ct_pt_mac(name, level):
+    ctx, orc, _ = ctx_pair(name)
+    batch = 4
+    ct = random_ct(orc, 3, 0, level, batch)
+    acc = random_ct(orc, 3, 1, level, batch)
+    pt = np.stack([S.uniform_residues_np(3, 9000 + b, orc.q[:level], orc.N) for b in range(batch)])
+    d_acc = to_dev(acc)
+    ctx.ct_pt_mac(to_dev(ct), to_dev(pt), d_acc, batch, level)
+    want = np.stack([orc.ct_pt_mac(ct[b], pt[b], acc[b]) for b in range(batch)])
+    assert np.array_equal(to_host(d_acc), want)
+    # one plaintext shared by the batch
+    d_acc = to_dev(acc)
+    ctx.ct_pt_mac(to_dev(ct), to_dev(pt[0]), d_acc, batch, level, pt_stride=0)
+    want = np.stack([orc.ct_pt_mac(ct[b], pt[0], acc[b]) for b in range(batch)])
+    assert np.array_equal(to_host(d_acc), want)
+
+
+def _check_rotate(name, level, batch, rot, key_id):
+    import torch
+
+    pair = ctx_pair(name)
+    ctx, orc, _ = pair
+    add_key(pair, rot, key_id)
+    ct = random_ct(orc, 4, level * 100 + key_id, level, batch)
+    out = torch.empty_like(to_dev(ct))
+    ctx.rotate(to_dev(ct), out, batch, level, key_id)
+    got = to_host(out)
+    for b in range(batch):
+        assert np.array_equal(got[b], orc.rotate(ct[b], key_id)), (name, level, b)
+
+
+@pytest.mark.parametrize("level", [6, 5, 4, 3, 2, 1])
+def test_rotate_toy_all_levels(level):
+    _check_rotate("toy", level, 3, 1, 11)
+    _check_rotate("toy", level, 2, -(1 << 31), 12)
+
+
+def test_rotate_tiny():
+    _check_rotate("tiny", 3, 4, 1, 21)
+    _check_rotate("tiny", 3, 4, 5, 22)
+    _check_rotate("tiny", 2, 1, 5, 22)
+
+
+@pytest.mark.parametrize("level", [24, 23, 21, 9, 1])
+def test_rotate_small_ring_full_limb_structure(level):
+    _check_rotate("small", level, 5, 8, 31)
+
+
+@pytest.mark.parametrize("name,level,batch", [("full", 24, 2), ("full", 22, 1), ("full_literal", 24, 1)])
+def test_rotate_full_ring(name, level, batch):
+    _check_rotate(name, level, batch, 8, 41)
+
+
+@pytest.mark.parametrize("name,level", [("toy", 6), ("toy", 2), ("tiny", 3), ("small", 24), ("small", 10)])
+def test_rescale(name, level):
+    import torch
+
+    ctx, orc, _ = ctx_pair(name)
+    batch = 3
+    ct = random_ct(orc, 5, level, level, batch)
+    out = torch.empty((batch, 2, level - 1, orc.N), dtype=torch.int64, device="cuda")
+    ctx.rescale(to_dev(ct), out, batch, level)
+    got = to_host(out)
+    for b in range(batch):
+        assert np.array_equal(got[b], orc.rescale(ct[b]))
+
+
+@pytest.mark.parametrize("name,level", [("toy", 6), ("toy", 3), ("small", 24), ("small", 6)])
+def test_ct_ct_mul(name, level):
+    import torch
+
+    ctx, orc, _ = ctx_pair(name)
+    batch = 3
+    a = random_ct(orc, 6, level, level, batch)
+    b_ = random_ct(orc, 6, level + 50, level, batch)
+    out = torch.empty_like(to_dev(a))
+    ctx.ct_ct_mul(to_dev(a), to_dev(b_), out, batch, level)
+    got = to_host(out)
+    for b in range(batch):
+        assert np.array_equal(got[b], orc.ct_ct_mul(a[b], b_[b]))
+
+
+def test_full_ring_rescale_and_ctmul():
+    import torch
+
+    ctx, orc, _ = ctx_pair("full")
+    a = random_ct(orc, 7, 0, 24, 1)
+    b_ = random_ct(orc, 7, 1, 24, 1)
+    out = torch.empty_like(to_dev(a))
+    ctx.ct_ct_mul(to_dev(a), to_dev(b_), out, 1, 24)
+    want = orc.ct_ct_mul(a[0], b_[0])
+    assert np.array_equal(to_host(out)[0], want)
+    res = torch.empty((1, 2, 23, orc.N), dtype=torch.int64, device="cuda")
+    ctx.rescale(out, res, 1, 24)
+    assert np.array_equal(to_host(res)[0], orc.rescale(want))
+
+
+def test_error_codes():
+    import torch
+    import paper_2608_17442_b200 as fesc
+
+    ctx, orc, p = ctx_pair("toy")
+    ct = to_dev(random_ct(orc, 8, 0, 6, 1))
+    out = torch.empty_like(ct)
+    with pytest.raises(fesc.FescError) as e:
+        ctx.rotate(ct, out, 1, 6, 999)
+    assert e.value.code == fesc.ENOKEY
+    with pytest.raises(fesc.FescError) as e:
+        ctx.rescale(ct, out, 1, 1)
+    assert e.value.code == fesc.ELEVEL
+    with pytest.raises(fesc.FescError) as e:
+        fesc.Context(6, [97, 193, 257], 2, 1, 2, 1)   # not = 1 mod 2N
+    assert e.value.code == fesc.EINVAL
+
+
+def test_workload_1_end_to_end():
+    """Tiny CKKS: 4 ciphertexts x random plaintext vector, rotate by +1 and +5, decrypt; residues
+    bit-exact and slots within 2^-16 of the float64 result."""
+    import torch
+
+    pair = ctx_pair("tiny")
+    ctx, orc, p = pair
+    add_key(pair, 1, 101)
+    add_key(pair, 5, 105)
+    scale = 2.0**30
+    z = S.uniform_slots(p["seed"], 0, 4, orc.n)
+    w = S.uniform_slots(p["seed"], 1, 4, orc.n)
+    cts = np.stack([orc.encrypt(orc.encode(z[i], scale, 3), i) for i in range(4)])
+    pts = np.stack([orc.encode(w[i], scale, 3) for i in range(4)])
+    prod = torch.zeros((4, 2, 3, orc.N), dtype=torch.int64, device="cuda")
+    ctx.ct_pt_mac(to_dev(cts), to_dev(pts), prod, 4, 3)
+    for key_id, r in ((101, 1), (105, 5)):
+        out = torch.empty_like(prod)
+        ctx.rotate(prod, out, 4, 3, key_id)
+        got = to_host(out)
+        for i in range(4):
+            want = orc.rotate(orc.ct_pt_mac(cts[i], pts[i], np.zeros_like(cts[i])), key_id)
+            assert np.array_equal(got[i], want)
+            slots = orc.decrypt(got[i], scale * scale)
+            assert np.abs(slots - np.roll(z[i] * w[i], -r)).max() < 2.0**-16
