@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the encrypted Mamba-2-base in_proj projection (768 -> 3352 at L = 2048 tokens)
+on B200, through the C-ABI library.
+
+One "step" = one fesc_linear call on the full workload: 48 input ciphertexts (16 token blocks x
+3 input blocks, N = 2^16, 24 limbs), 10 752 pre-encoded plaintext diagonals (126 GiB, resident),
+1 488 baby + 1 568 giant rotations (hybrid key switch, 6 digits), 172 032 ct-pt MACs, 224
+rescales.  Inputs are seeded synthetic residues (uniform below each prime) of exactly those
+shapes; arithmetic is data-independent, so timing equals that of real encodings.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` = key switches per second over the whole step, summed
+over ranks (each rank runs its own 2048-token batch: weak scaling, no data-path collective);
+`latency_ms` is the projection latency the metric names.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "encrypted 768->3352 projection latency at L=2048; key-switches/s; HBM GB/s vs peak"
+T_SEG, C_SEG, N1, N2 = 128, 256, 32, 8
+D_IN, D_OUT, TOKENS = 768, 3352, 2048
+LEVEL = 24
+BABY_BASE, GIANT_BASE = 1000, 1500
+
+
+def workload_dims(scale_down: int = 1):
+    gin = -(-D_IN // C_SEG)
+    nout = -(-D_OUT // C_SEG)
+    tbs = -(-TOKENS // T_SEG)
+    if scale_down > 1:   # debugging aid only; never used for a reported number
+        nout = max(1, nout // scale_down)
+        tbs = max(1, tbs // scale_down)
+    return gin, nout, tbs
+
+
+def key_switches_per_step(gin, nout, tbs):
+    return tbs * (gin * (N1 - 1) + nout * (N2 - 1))
+
+
+# ---------------------------------------------------------------------------------------------
+# distributed plumbing (one process per GPU; only a barrier and a max over ranks)
+# ---------------------------------------------------------------------------------------------
+def dist_setup(backend: str):
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1 and not dist.is_initialized():
+        dist.init_process_group(backend=backend)
+    return int(os.environ.get("RANK", "0")), world
+
+
+def max_over_ranks(value: float, device="cpu") -> float:
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()):
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier():
+    import torch.distributed as dist
+
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.QUERY}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self) -> dict:
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+                power.append(float(parts[3]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        os.unlink(self.f.name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "power_w_max": max(power),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------
+# synthetic inputs
+# ---------------------------------------------------------------------------------------------
+def make_inputs(primes, n, gin, nout, tbs, seed, device):
+    """ct_in [tbs][gin][2][LEVEL][N] and diags [nout][N2][gin][N1][LEVEL][N] filled with hashed
+    residues; stream ids: ciphertext (tb,g) -> tb*gin+g, diagonal chunk (b,p) -> 100000 + b*N2+p."""
+    import torch
+    import fesc_synth as S
+
+    q = primes[:LEVEL]
+    ct = torch.empty((tbs, gin, 2, LEVEL, n), dtype=torch.int64, device=device)
+    for tb in range(tbs):
+        for g in range(gin):
+            r = S.hashed_residues(seed, tb * gin + g, q, 2 * n, device=device)      # [LEVEL, 2n]
+            ct[tb, g] = r.view(LEVEL, 2, n).permute(1, 0, 2)
+    diags = torch.empty((nout, N2, gin, N1, LEVEL, n), dtype=torch.int64, device=device)
+    for b in range(nout):
+        for p in range(N2):
+            r = S.hashed_residues(seed, 100000 + b * N2 + p, q, gin * N1 * n, device=device)
+            diags[b, p] = r.view(LEVEL, gin, N1, n).permute(1, 2, 0, 3)
+            del r
+    return ct, diags
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# Integer-pipe ceiling for the 128-bit multiply-accumulate kernels: see DESIGN.md ("ALU roofline").
+SM_COUNT = 148
+IMAD_PER_CLK_PER_SM = 64          # 32-bit integer multiply-add issue rate assumed per SM per clock
+MAC128_IMAD = 4                   # one 64x64->128 product = 4 32x32->64 multiply-adds at minimum
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm and CPU baseline: the oracle, timed as it stands on a bounded sample
+# ---------------------------------------------------------------------------------------------
+def oracle_sample(steps: int, warmup: int):
+    """One token block x one output block x ONE input block of the projection through the
+    oracle: 31 baby + 7 giant rotations, 256 MACs, 1 rescale.  Returns (key-switches/s, ms/step, cores)."""
+    import numpy as np
+    import fesc_synth as S
+    from oracle.ckks import Oracle
+
+    p = S.params("full")
+    orc = Oracle(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+    for q in range(1, N1):
+        orc.add_galois_key(q * T_SEG, BABY_BASE + q)
+    for g in range(1, N2):
+        orc.add_galois_key(g * N1 * T_SEG, GIANT_BASE + g)
+    seed = S.config_seed(4)
+    ct = np.empty((1, 1, 2, LEVEL, orc.N), dtype=np.uint64)
+    for pp in range(2):
+        ct[0, 0, pp] = S.uniform_residues_np(seed, pp, orc.q[:LEVEL], orc.N)
+    diags = np.empty((1, N2, 1, N1, LEVEL, orc.N), dtype=np.uint64)
+    for pp in range(N2):
+        for q in range(N1):
+            diags[0, pp, 0, q] = S.uniform_residues_np(seed, 10 + pp * N1 + q, orc.q[:LEVEL], orc.N)
+    desc = dict(n1=N1, n2=N2)
+    bk = {q: BABY_BASE + q for q in range(1, N1)}
+    gk = {g: GIANT_BASE + g for g in range(1, N2)}
+    for _ in range(warmup):
+        orc.linear(ct, diags, desc, bk, gk)
+    t0 = time.perf_counter()
+    for _ in range(max(1, steps)):
+        orc.linear(ct, diags, desc, bk, gk)
+    dt = (time.perf_counter() - t0) / max(1, steps)
+    ks = (N1 - 1) + (N2 - 1)
+    cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    return ks / dt, dt * 1e3, cores
+
+
+SAMPLE_TEXT = ("1 token block x 1 output block x 1 input block of the projection "
+               "(31 baby + 7 giant rotations, 256 ct-pt MACs, 1 rescale; 1/672 of the step's MACs)")
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    value, ms, cores = oracle_sample(args.steps, min(args.warmup, 1))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "key-switches/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+        "config": {"workload": "in_proj 768->3352, L=2048, N=2^16, 24x50-bit limbs + 4x60-bit special, 6 digits "
+                               "(bounded sample per step: " + SAMPLE_TEXT + ")"},
+        "cpu_baseline": {"value": value, "unit": "key-switches/s", "cores": cores, "kind": "oracle",
+                         "sample": SAMPLE_TEXT},
+        "e2e": {"value": value, "unit": "key-switches/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import fesc_synth as S
+    import paper_2608_17442_b200 as fesc
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    rank, world = dist_setup("nccl")
+    dev = torch.device("cuda", local)
+
+    p = S.params("full")
+    ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+    n = ctx.N
+    for q in range(1, N1):
+        ctx.add_galois_key(q * T_SEG, BABY_BASE + q)
+    for g in range(1, N2):
+        ctx.add_galois_key(g * N1 * T_SEG, GIANT_BASE + g)
+    gin, nout, tbs = workload_dims(args.scale_down)
+    ks_per_step = key_switches_per_step(gin, nout, tbs)
+    ct, diags = make_inputs(p["primes"], n, gin, nout, tbs, S.config_seed(4) + rank, dev)
+    out = torch.empty((tbs, nout, 2, LEVEL - 1, n), dtype=torch.int64, device=dev)
+    torch.cuda.empty_cache()
+    desc = fesc.BsgsDesc(N1, N2, gin, nout, tbs, LEVEL, BABY_BASE, GIANT_BASE)
+
+    def step():
+        ctx.linear(ct, diags, desc, out)
+
+    # warm-up (also sizes the scratch arena) and a family breakdown on one untimed step
+    for _ in range(max(3, args.warmup) - 1):
+        step()
+    ctx.profile_enable(fesc.Context.PROFILE_FAMILIES, 120000)
+    step()
+    fam = ctx.profile_read()
+    ctx.profile_enable([])
+    total_fam = sum(v[0] for v in fam.values()) or 1.0
+    breakdown = {k: {"ms": round(v[0], 3), "records": v[1], "share": round(v[0] / total_fam, 4)} for k, v in fam.items()}
+    dominant = max(fam, key=lambda k: fam[k][0])
+
+    # timed region
+    ctx.profile_enable([dominant], 120000)
+    launches0 = ctx.counters()[4]
+    sampler = ClockSampler(local)
+    torch.cuda.synchronize()
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = max_over_ranks(e0.elapsed_time(e1), dev)
+    launches = ctx.counters()[4] - launches0
+    dom_ms, dom_records = ctx.profile_read()[dominant]
+    ctx.profile_enable([])
+    ms_per_step = ms_total / args.steps
+    value = world * ks_per_step / (ms_per_step * 1e-3)
+
+    # roofline of the dominant kernel family
+    hbm_peak, peak_kind = peaks()
+    word = 8
+    ctw = 2 * LEVEL * n * word
+    roof = {"kernel": dominant, "peak_source": peak_kind}
+    if dominant == "bsgs":
+        # one launch = one group of token blocks: every distinct input word read once, every output written once
+        groups = max(1, dom_records // args.steps)
+        tb_per_launch = tbs / groups
+        alg = tb_per_launch * gin * N1 * ctw + nout * N2 * gin * N1 * (ctw // 2) + tb_per_launch * nout * N2 * ctw
+        macs = tb_per_launch * nout * N2 * gin * N1 * 2 * LEVEL * n          # 64x64->128 multiply-adds
+        t = dom_ms * 1e-3 / max(1, dom_records)
+        sm_mhz = clocks.get("sm_mhz") or 1350.0
+        alu_peak = SM_COUNT * IMAD_PER_CLK_PER_SM * sm_mhz * 1e6 / MAC128_IMAD / 1e12   # T mul-adds / s
+        roof.update({"bound": "alu", "achieved": macs / t / 1e12, "peak": alu_peak, "unit": "T mac128/s",
+                     "frac": macs / t / 1e12 / alu_peak, "traffic": None,
+                     "hbm": {"achieved": alg / t / 1e9, "peak": hbm_peak, "unit": "GB/s", "frac": alg / t / 1e9 / hbm_peak,
+                             "algorithmic_bytes_per_launch": alg}})
+    else:
+        t = dom_ms * 1e-3 / max(1, dom_records)
+        roof.update({"bound": "alu", "achieved": None, "peak": None, "unit": "ms/launch", "frac": None,
+                     "traffic": None, "avg_launch_ms": t * 1e3})
+
+    # end to end: pinned host inputs -> device, projection, result -> pinned host, every step
+    h_in = torch.empty(ct.shape, dtype=torch.int64, pin_memory=True)
+    h_in.copy_(ct)
+    h_out = torch.empty(out.shape, dtype=torch.int64, pin_memory=True)
+    e2e_steps = max(1, min(args.steps, 3))
+    torch.cuda.synchronize()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        ct.copy_(h_in, non_blocking=True)
+        step()
+        h_out.copy_(out, non_blocking=True)
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dev) / e2e_steps
+    e2e = {"value": world * ks_per_step / (e2e_ms * 1e-3), "unit": "key-switches/s", "latency_ms": e2e_ms,
+           "h2d_bytes_per_step": ct.numel() * 8, "d2h_bytes_per_step": out.numel() * 8}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "key-switches/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "latency_ms": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+        "config": {"workload": "in_proj 768->3352, L=2048 tokens, N=2^16, 24x50-bit limbs + 4x60-bit special primes, "
+                               "6 key-switch digits, C=256 T=128 n1=32 n2=8",
+                   "input_cts": tbs * gin, "diagonals": nout * N2 * gin * N1, "output_cts": tbs * nout,
+                   "key_switches_per_step": ks_per_step, "macs_per_step": tbs * nout * N2 * gin * N1,
+                   "l2": "inputs larger than L2 (diagonals %.1f GiB stream every step)" % (diags.numel() * 8 / 2**30),
+                   "parallelism": "replicas x%d (independent 2048-token batches)" % world},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roof, "kernel_breakdown": breakdown,
+    }
+    if args.scale_down > 1:
+        line["config"]["workload"] += " [DEBUG scale_down=%d: not a reportable number]" % args.scale_down
+    if rank == 0 and world == 1 and not args.no_cpu:
+        v, ms, cores = oracle_sample(1, 0)
+        line["cpu_baseline"] = {"value": v, "unit": "key-switches/s", "cores": cores, "kind": "oracle",
+                                "sample": SAMPLE_TEXT, "ms": ms}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    del ctx
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--scale-down", dest="scale_down", type=int, default=1, help=argparse.SUPPRESS)
+    ap.add_argument("--no-cpu", dest="no_cpu", action="store_true", help="skip the CPU baseline leg")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

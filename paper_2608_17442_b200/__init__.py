@@ -50,6 +50,8 @@ def lib():
             "fesc_ctx_export_key": [vp, u32, vp, vp],
             "fesc_ctx_export_secret": [vp, vp, vp],
             "fesc_ctx_counters": [vp, c.POINTER(u64)],
+            "fesc_profile_enable": [vp, c.c_int, u32],
+            "fesc_profile_read": [vp, c.POINTER(c.c_float), c.POINTER(u64)],
             "fesc_ntt": [vp, vp, u32, u32, u32, vp],
             "fesc_intt": [vp, vp, u32, u32, u32, vp],
             "fesc_ct_pt_mac": [vp, vp, vp, sz, vp, u32, u32, vp],
@@ -114,9 +116,25 @@ class Context:
         return lib().fesc_ctx_num_digits(self.h)
 
     def counters(self):
-        out = (ctypes.c_uint64 * 4)()
+        out = (ctypes.c_uint64 * 8)()
         self._chk(lib().fesc_ctx_counters(self.h, out))
         return list(out)
+
+    PROFILE_FAMILIES = ("ntt", "modup", "inner", "moddown", "autom", "bsgs", "rescale", "pointwise")
+
+    def profile_enable(self, families, max_records: int = 65536):
+        """Time the named kernel families (iterable of PROFILE_FAMILIES names; empty = off)."""
+        mask = 0
+        for f in families:
+            mask |= 1 << self.PROFILE_FAMILIES.index(f)
+        self._chk(lib().fesc_profile_enable(self.h, mask, max_records))
+
+    def profile_read(self):
+        """{family: (milliseconds, records)} since the last read."""
+        ms = (ctypes.c_float * 8)()
+        rec = (ctypes.c_uint64 * 8)()
+        self._chk(lib().fesc_profile_read(self.h, ms, rec))
+        return {n: (float(ms[i]), int(rec[i])) for i, n in enumerate(self.PROFILE_FAMILIES)}
 
     def add_galois_key(self, rot: int, key_id: int):
         self._chk(lib().fesc_ctx_add_galois_key(self.h, rot, key_id))

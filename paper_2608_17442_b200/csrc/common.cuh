@@ -51,9 +51,10 @@ struct acc128 {
     u64 lo, hi;
 };
 __device__ __forceinline__ void mac128(acc128& a, u64 x, u64 y) {
-    u64 l = x * y, h = mulhi(x, y);
-    a.lo += l;
-    a.hi += h + (a.lo < l);
+    u128 v = ((u128)a.hi << 64) | a.lo;
+    v += (u128)x * y;
+    a.lo = (u64)v;
+    a.hi = (u64)(v >> 64);
 }
 // (hi*2^64 + lo) mod q, canonical.  hi may be any 64-bit value.
 __device__ __forceinline__ u64 reduce128(u64 hi, u64 lo, const PrimeConst& pc) {
@@ -125,6 +126,15 @@ struct EvalKey {
     u64* d_key;     // [beta_max][2][n_q+n_p][N]
 };
 
+// Optional per-kernel-family timing with CUDA events on the launching stream.
+enum { PF_NTT = 0, PF_MODUP, PF_INNER, PF_MODDOWN, PF_AUTOM, PF_BSGS, PF_RESCALE, PF_POINTWISE, PF_COUNT };
+struct Profiler {
+    uint32_t on = 0;               // bit f set: family f is timed
+    std::vector<cudaEvent_t> ev;   // pairs (start, stop)
+    std::vector<int> fam;
+    size_t used = 0;
+};
+
 struct fesc_ctx {
     uint32_t log_n, N, n_q, n_p, n_primes, dnum, alpha, beta_max;
     u64 seed;
@@ -139,9 +149,24 @@ struct fesc_ctx {
     // scratch
     u64* d_scratch;
     size_t scratch_bytes;
-    uint64_t counters[4];
+    uint64_t counters[8];
+    Profiler prof;
     std::string err;
 };
+
+static inline void prof_begin(fesc_ctx* ctx, int family, cudaStream_t st) {
+    Profiler& p = ctx->prof;
+    if (((p.on >> family) & 1) && p.used + 2 <= p.ev.size()) cudaEventRecord(p.ev[p.used], st);
+}
+static inline void prof_end(fesc_ctx* ctx, int family, cudaStream_t st, uint64_t launches = 1) {
+    ctx->counters[4] += launches;
+    Profiler& p = ctx->prof;
+    if (((p.on >> family) & 1) && p.used + 2 <= p.ev.size()) {
+        cudaEventRecord(p.ev[p.used + 1], st);
+        p.fam.push_back(family);
+        p.used += 2;
+    }
+}
 
 #define FESC_CHECK_CUDA(ctx, call)                                                          \
     do {                                                                                    \

@@ -378,6 +378,7 @@ extern "C" int fesc_ctx_destroy(fesc_ctx* ctx) {
     if (!ctx) return FESC_OK;
     cudaDeviceSynchronize();
     for (auto& kv : ctx->keys) cudaFree(kv.second.d_key);
+    for (cudaEvent_t e : ctx->prof.ev) cudaEventDestroy(e);
     cudaFree(ctx->d_pc);
     cudaFree(ctx->d_tw);
     cudaFree(ctx->d_itw);
@@ -439,8 +440,39 @@ extern "C" int fesc_ctx_export_secret(fesc_ctx* ctx, uint64_t* d_dst, void* stre
     FESC_CHECK_CUDA(ctx, cudaMemcpyAsync(d_dst, ctx->d_s, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
     return FESC_OK;
 }
+extern "C" int fesc_profile_enable(fesc_ctx* ctx, int on, uint32_t max_records) {
+    if (!ctx) return FESC_EINVAL;
+    Profiler& p = ctx->prof;
+    FESC_CHECK_CUDA(ctx, cudaDeviceSynchronize());
+    p.used = 0;
+    p.fam.clear();
+    if (on) {
+        while (p.ev.size() < 2 * (size_t)max_records) {
+            cudaEvent_t e;
+            FESC_CHECK_CUDA(ctx, cudaEventCreate(&e));
+            p.ev.push_back(e);
+        }
+    }
+    p.on = (uint32_t)on;
+    return FESC_OK;
+}
+extern "C" int fesc_profile_read(fesc_ctx* ctx, float ms[8], uint64_t records[8]) {
+    if (!ctx || !ms || !records) return FESC_EINVAL;
+    Profiler& p = ctx->prof;
+    FESC_CHECK_CUDA(ctx, cudaDeviceSynchronize());
+    for (int i = 0; i < 8; i++) ms[i] = 0.f, records[i] = 0;
+    for (size_t r = 0; r < p.fam.size(); r++) {
+        float t = 0.f;
+        FESC_CHECK_CUDA(ctx, cudaEventElapsedTime(&t, p.ev[2 * r], p.ev[2 * r + 1]));
+        ms[p.fam[r]] += t;
+        records[p.fam[r]]++;
+    }
+    p.used = 0;
+    p.fam.clear();
+    return FESC_OK;
+}
 extern "C" uint32_t fesc_ctx_num_digits(const fesc_ctx* ctx) { return ctx ? ctx->beta_max : 0; }
-extern "C" int fesc_ctx_counters(const fesc_ctx* ctx, uint64_t out[4]) {
+extern "C" int fesc_ctx_counters(const fesc_ctx* ctx, uint64_t out[8]) {
     if (!ctx || !out) return FESC_EINVAL;
     memcpy(out, ctx->counters, sizeof(ctx->counters));
     return FESC_OK;

@@ -6,57 +6,73 @@
 // lazy sums in registers, tiled TT token blocks x PT (b,p) pairs per thread so a rotated
 // ciphertext word is reused PT times and a diagonal word TT times; (3) giant rotations that
 // accumulate straight into acc[tb][b][0]; (4) rescale into the output.
+#include <stdlib.h>
+
 #include "ops.cuh"
 
 template <int TT, int PT>
-__global__ void __launch_bounds__(256) k_bsgs_accumulate(
-    const u64* __restrict__ in,     // [tbs][gin][2][level][N]            (q = 0 terms)
-    const u64* __restrict__ rot,    // [tbs][gin][n1][2][level][N]        (slot q = 0 unused)
-    const u64* __restrict__ diags,  // [nout][n2][gin][n1][level][N]
-    u64* __restrict__ acc,          // [tbs][nout][n2][2][level][N]
-    const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level, uint32_t tbs, uint32_t gin, uint32_t n1,
-    uint32_t bp_count /* nout*n2 */, uint32_t reduce_every) {
-    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
-    const uint32_t l = blockIdx.y;
-    const uint32_t bp_tiles = (bp_count + PT - 1) / PT;
-    const uint32_t tb0 = (blockIdx.z / bp_tiles) * TT, bp0 = (blockIdx.z % bp_tiles) * PT;
+__global__ void __launch_bounds__(256, (TT * PT >= 16 ? 1 : (TT * PT >= 4 ? 2 : 3))) k_bsgs_accumulate(
+    const u64* __restrict__ rot,    // [tbs][terms][2][level][N]   rotated inputs, term = g*n1 + q
+    const u64* __restrict__ diags,  // [bp_count][terms][level][N]
+    u64* __restrict__ acc,          // [tbs][bp_count][2][level][N]
+    const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level, uint32_t tbs, uint32_t terms,
+    uint32_t bp_count, uint32_t reduce_every) {
+    // blockIdx.x walks the (b,p) tiles of one (coefficient tile, limb, token-block tile), so CTAs
+    // that run together read the same ciphertext words: those come from HBM once and from L2 after.
+    const uint32_t c = blockIdx.y * blockDim.x + threadIdx.x;
+    const uint32_t l = blockIdx.z % level;
+    const uint32_t tb0 = (blockIdx.z / level) * TT, bp0 = blockIdx.x * PT;
     if (c >= N) return;
     const PrimeConst pc = pcs[l];
     const size_t poly = (size_t)level * N, ctw = 2 * poly;
     const size_t o = (size_t)l * N + c;
+    // out-of-range tile members recompute the last valid one and are not stored
+    const u64* xp[TT];
+    const u64* dp[PT];
+#pragma unroll
+    for (int i = 0; i < TT; i++) {
+        uint32_t tb = tb0 + i < tbs ? tb0 + i : tbs - 1;
+        xp[i] = rot + (size_t)tb * terms * ctw + o;
+    }
+#pragma unroll
+    for (int j = 0; j < PT; j++) {
+        uint32_t bp = bp0 + j < bp_count ? bp0 + j : bp_count - 1;
+        dp[j] = diags + (size_t)bp * terms * poly + o;
+    }
     acc128 a[TT][PT][2];
 #pragma unroll
     for (int i = 0; i < TT; i++)
 #pragma unroll
         for (int j = 0; j < PT; j++) a[i][j][0] = a[i][j][1] = acc128{0, 0};
-    const uint32_t terms = gin * n1;
+    // software pipeline: operands of term t+1 are in flight while term t is multiplied
+    u64 x0[TT], x1[TT], w[PT], nx0[TT], nx1[TT], nw[PT];
+#pragma unroll
+    for (int i = 0; i < TT; i++) {
+        x0[i] = xp[i][0];
+        x1[i] = xp[i][poly];
+    }
+#pragma unroll
+    for (int j = 0; j < PT; j++) w[j] = __ldg(dp[j]);
     uint32_t since = 0;
-    for (uint32_t gq = 0; gq < terms; gq++) {
-        const uint32_t g = gq / n1, q = gq % n1;
-        u64 x0[TT], x1[TT];
+#pragma unroll 1
+    for (uint32_t t = 0; t < terms; t++) {
+        const bool more = t + 1 < terms;
+        const size_t xo = more ? (size_t)(t + 1) * ctw : (size_t)t * ctw;
+        const size_t wo = more ? (size_t)(t + 1) * poly : (size_t)t * poly;
 #pragma unroll
         for (int i = 0; i < TT; i++) {
-            const uint32_t tb = tb0 + i;
-            x0[i] = x1[i] = 0;
-            if (tb < tbs) {
-                const u64* src = q == 0 ? in + ((size_t)tb * gin + g) * ctw
-                                        : rot + (((size_t)tb * gin + g) * n1 + q) * ctw;
-                x0[i] = src[o];
-                x1[i] = src[poly + o];
-            }
+            nx0[i] = xp[i][xo];
+            nx1[i] = xp[i][xo + poly];
         }
 #pragma unroll
-        for (int j = 0; j < PT; j++) {
-            const uint32_t bp = bp0 + j;
-            if (bp < bp_count) {
-                const u64 w = __ldg(diags + (((size_t)bp * gin + g) * n1 + q) * poly + o);
+        for (int j = 0; j < PT; j++) nw[j] = __ldg(dp[j] + wo);
 #pragma unroll
-                for (int i = 0; i < TT; i++) {
-                    mac128(a[i][j][0], x0[i], w);
-                    mac128(a[i][j][1], x1[i], w);
-                }
+        for (int j = 0; j < PT; j++)
+#pragma unroll
+            for (int i = 0; i < TT; i++) {
+                mac128(a[i][j][0], x0[i], w[j]);
+                mac128(a[i][j][1], x1[i], w[j]);
             }
-        }
         if (++since == reduce_every) {
             since = 0;
 #pragma unroll
@@ -66,6 +82,13 @@ __global__ void __launch_bounds__(256) k_bsgs_accumulate(
 #pragma unroll
                     for (int p = 0; p < 2; p++) a[i][j][p] = acc128{reduce128(a[i][j][p].hi, a[i][j][p].lo, pc), 0};
         }
+#pragma unroll
+        for (int i = 0; i < TT; i++) {
+            x0[i] = nx0[i];
+            x1[i] = nx1[i];
+        }
+#pragma unroll
+        for (int j = 0; j < PT; j++) w[j] = nw[j];
     }
 #pragma unroll
     for (int i = 0; i < TT; i++)
@@ -78,6 +101,20 @@ __global__ void __launch_bounds__(256) k_bsgs_accumulate(
                 dst[poly + o] = reduce128(a[i][j][1].hi, a[i][j][1].lo, pc);
             }
         }
+}
+
+// Tuning knob for experiments: FESC_BSGS_TILE=<TT><PT> (e.g. 24) picks the register tile.
+static int bsgs_tile() {
+    static int v = -1;
+    if (v < 0) {
+        const char* e = getenv("FESC_BSGS_TILE");
+        v = e ? atoi(e) : 0;
+    }
+    return v;
+}
+static size_t bsgs_group_bytes() {
+    const char* e = getenv("FESC_BSGS_GROUP_GIB");
+    return (size_t)(e ? atoi(e) : 12) << 30;
 }
 
 extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_t* d_diags, const fesc_bsgs_desc* desc,
@@ -97,7 +134,7 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
     const size_t ctw = (size_t)2 * level * N;
     // token blocks per group: keep the group's buffers near 12 GiB
     const size_t per_tb = ((size_t)gin * n1 + (size_t)nout * n2) * ctw * sizeof(u64);
-    uint32_t tbg = (uint32_t)(((size_t)12 << 30) / per_tb);
+    uint32_t tbg = (uint32_t)(bsgs_group_bytes() / per_tb);
     if (tbg < 1) tbg = 1;
     if (tbg > tbs) tbg = tbs;
     const uint32_t max_batch = tbg * (gin > nout ? gin : nout);
@@ -123,17 +160,35 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
     for (uint32_t tb0 = 0; tb0 < tbs; tb0 += tbg) {
         const uint32_t nt = tbs - tb0 < tbg ? tbs - tb0 : tbg;
         const u64* gin_base = in + (size_t)tb0 * gin * ctw;
+        // slot q = 0 of the rotated set is the input itself
+        FESC_CHECK_CUDA(ctx, cudaMemcpy2DAsync(rot, (size_t)n1 * ctw * sizeof(u64), gin_base, ctw * sizeof(u64),
+                                               ctw * sizeof(u64), (size_t)nt * gin, cudaMemcpyDeviceToDevice, st));
         for (uint32_t q = 1; q < n1; q++) {
             rc = rotate_internal(ctx, gin_base, ctw, rot + (size_t)q * ctw, (size_t)n1 * ctw, nt * gin, level,
                                  desc->baby_key_base + q, ks, st, 0);
             if (rc != FESC_OK) return rc;
         }
-        constexpr int TT = 2, PT = 2;
         const uint32_t bp_count = nout * n2;
-        const uint32_t tiles = ((nt + TT - 1) / TT) * ((bp_count + PT - 1) / PT);
-        if (tiles > 65535) return fesc_fail(ctx, FESC_EINVAL, "linear: too many accumulator tiles");
-        k_bsgs_accumulate<TT, PT><<<dim3((N + 255) / 256, level, tiles), 256, 0, st>>>(
-            gin_base, rot, diags, acc, ctx->d_pc, N, level, nt, gin, n1, bp_count, reduce_every);
+        prof_begin(ctx, PF_BSGS, st);
+#define BSGS(TT, PT)                                                                                          \
+    do {                                                                                                      \
+        dim3 grid((bp_count + PT - 1) / PT, (N + 255) / 256, level * ((nt + TT - 1) / TT));                   \
+        if (grid.z > 65535) return fesc_fail(ctx, FESC_EINVAL, "linear: too many accumulator tiles");         \
+        k_bsgs_accumulate<TT, PT><<<grid, 256, 0, st>>>(rot, diags, acc, ctx->d_pc, N, level, nt, gin * n1,  \
+                                                        bp_count, reduce_every);                              \
+    } while (0)
+        switch (bsgs_tile()) {
+            case 12: BSGS(1, 2); break;
+            case 14: BSGS(1, 4); break;
+            case 18: BSGS(1, 8); break;
+            case 22: BSGS(2, 2); break;
+            case 24: BSGS(2, 4); break;
+            case 28: BSGS(2, 8); break;
+            case 44: BSGS(4, 4); break;
+            default: if (nt >= 2) BSGS(2, 8); else BSGS(1, 8); break;
+        }
+#undef BSGS
+        prof_end(ctx, PF_BSGS, st);
         FESC_CHECK_CUDA(ctx, cudaGetLastError());
         ctx->counters[2] += (uint64_t)nt * bp_count * gin * n1;
         for (uint32_t p = 1; p < n2; p++) {

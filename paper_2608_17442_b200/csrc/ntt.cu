@@ -312,6 +312,8 @@ int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool 
     size_t live = 0;
     for (uint32_t i = 0; i < map.period; i++) live += map.prime[i] != 0xFF;
     ctx->counters[0] += rows / map.period * live;
+    prof_begin(ctx, PF_NTT, st);
+    uint64_t launches = 0;
     if (ctx->log_n == 16) {
         // gridDim.y is limited to 65535 rows per launch
         for (size_t r0 = 0; r0 < rows;) {
@@ -329,6 +331,7 @@ int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool 
                 ntt16_strided<true><<<grid, 512, 0, st>>>(base, tw, ctx->d_pc, map);
             }
             r0 += chunk;
+            launches += 2;
         }
     } else {
         size_t smem = sizeof(u64) << ctx->log_n;
@@ -336,7 +339,9 @@ int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool 
             ntt_small<false><<<(unsigned)rows, 256, smem, st>>>(d_data, tw, ctx->d_pc, map, ctx->log_n);
         else
             ntt_small<true><<<(unsigned)rows, 256, smem, st>>>(d_data, tw, ctx->d_pc, map, ctx->log_n);
+        launches = 1;
     }
+    prof_end(ctx, PF_NTT, st, launches);
     FESC_CHECK_CUDA(ctx, cudaGetLastError());
     return FESC_OK;
 }

@@ -31,8 +31,10 @@ extern "C" int fesc_ct_pt_mac(fesc_ctx* ctx, const uint64_t* d_ct, const uint64_
     if (batch == 0) return FESC_OK;
     if (batch > 65535) return fesc_fail(ctx, FESC_EINVAL, "ct_pt_mac: batch too large");
     dim3 grid((ctx->N + 255) / 256, n_limbs, batch);
+    prof_begin(ctx, PF_POINTWISE, (cudaStream_t)stream);
     k_ct_pt_mac<<<grid, 256, 0, (cudaStream_t)stream>>>((const u64*)d_ct, (const u64*)d_pt, pt_stride, (u64*)d_acc,
                                                         ctx->d_pc, ctx->N, n_limbs);
+    prof_end(ctx, PF_POINTWISE, (cudaStream_t)stream);
     FESC_CHECK_CUDA(ctx, cudaGetLastError());
     ctx->counters[2] += batch;
     return FESC_OK;
@@ -247,12 +249,14 @@ static int key_switch_chunk(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& k
     const ModUpDigit* tab = ctx->tabs.d_modup + (size_t)(level - 1) * ctx->beta_max;
     dim3 gmu(gx, beta, batch);
 #define MODUP(A) k_modup<A><<<gmu, 256, 0, st>>>(ws.dcoef, ws.ext, tab, ctx->d_pc, N, level, nq, K, beta)
+    prof_begin(ctx, PF_MODUP, st);
     if (alpha <= 1) MODUP(1);
     else if (alpha <= 2) MODUP(2);
     else if (alpha <= 4) MODUP(4);
     else if (alpha <= 6) MODUP(6);
     else MODUP(8);
 #undef MODUP
+    prof_end(ctx, PF_MODUP, st);
     // 3. NTT of the converted rows
     if (beta * rows > sizeof(RowMap::prime)) return fesc_fail(ctx, FESC_EINVAL, "key switch: too many digit rows");
     m.period = beta * rows;
@@ -263,6 +267,7 @@ static int key_switch_chunk(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& k
         }
     if ((rc = ntt_launch(ctx, ws.ext, (size_t)batch * beta * rows, m, false, st)) != FESC_OK) return rc;
     // 4. inner product with the key
+    prof_begin(ctx, PF_INNER, st);
     if (batch >= 4) {
         dim3 g(gx, rows, (batch + 3) / 4);
         k_inner<4><<<g, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch);
@@ -273,16 +278,21 @@ static int key_switch_chunk(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& k
         dim3 g(gx, rows, 1);
         k_inner<1><<<g, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch);
     }
+    prof_end(ctx, PF_INNER, st);
     // 5. division by P
     m.period = rows;
     for (uint32_t t = 0; t < rows; t++) m.prime[t] = t < level ? 0xFF : (uint8_t)(nq + (t - level));
     if ((rc = ntt_launch(ctx, ws.acc, (size_t)batch * 2 * rows, m, true, st)) != FESC_OK) return rc;
+    prof_begin(ctx, PF_MODDOWN, st);
     k_moddown_conv<<<dim3(gx, batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K);
+    prof_end(ctx, PF_MODDOWN, st);
     m.period = level;
     for (uint32_t i = 0; i < level; i++) m.prime[i] = (uint8_t)i;
     if ((rc = ntt_launch(ctx, ws.u, (size_t)batch * 2 * level, m, false, st)) != FESC_OK) return rc;
+    prof_begin(ctx, PF_MODDOWN, st);
     k_moddown_finish<<<dim3(gx, level, batch * 2), 256, 0, st>>>(ws.acc, ws.u, out, out_stride, ctx->tabs.d_moddown,
                                                                  ctx->d_pc, N, level, K, add_mask);
+    prof_end(ctx, PF_MODDOWN, st);
     FESC_CHECK_CUDA(ctx, cudaGetLastError());
     ctx->counters[1] += batch;
     return FESC_OK;
@@ -321,8 +331,10 @@ int rotate_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, si
     for (uint32_t b0 = 0; b0 < batch; b0 += chunk) {
         uint32_t nb = batch - b0 < chunk ? batch - b0 : chunk;
         dim3 g((ctx->N + 255) / 256, level, nb);
+        prof_begin(ctx, PF_AUTOM, st);
         k_autom_ct<<<g, 256, 0, st>>>(in + (size_t)b0 * in_stride, in_stride, out + (size_t)b0 * out_stride, out_stride,
                                       ws.d, ws.dcoef, ctx->log_n, level, it->second.g, ctx->d_pc, accumulate);
+        prof_end(ctx, PF_AUTOM, st);
         int rc = key_switch_chunk(ctx, ws, it->second, level, nb, out + (size_t)b0 * out_stride, out_stride,
                                   accumulate ? 3 : 1, st);
         if (rc != FESC_OK) return rc;
@@ -393,17 +405,23 @@ int rescale_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, u
         uint32_t nb = batch - b0 < 16384 ? batch - b0 : 16384;
         const u64* ib = in + (size_t)b0 * in_stride;
         u64* ob = out + (size_t)b0 * out_stride;
+        prof_begin(ctx, PF_RESCALE, st);
         k_take_last<<<dim3(gx, nb * 2), 256, 0, st>>>(ib, in_stride, scratch, N, level);
+        prof_end(ctx, PF_RESCALE, st);
         RowMap m;
         m.period = 1;
         m.prime[0] = (uint8_t)(level - 1);
         if ((rc = ntt_launch(ctx, scratch, (size_t)nb * 2, m, true, st)) != FESC_OK) return rc;
+        prof_begin(ctx, PF_RESCALE, st);
         k_rescale_conv<<<dim3(gx, level - 1, nb * 2), 256, 0, st>>>(scratch, ob, out_stride, tab, ctx->d_pc, N, level);
+        prof_end(ctx, PF_RESCALE, st);
         m.period = level - 1;
         for (uint32_t i = 0; i + 1 < level; i++) m.prime[i] = (uint8_t)i;
         if ((rc = ntt_launch(ctx, ob, (size_t)nb * 2 * (level - 1), m, false, st)) != FESC_OK) return rc;
+        prof_begin(ctx, PF_RESCALE, st);
         k_rescale_finish<<<dim3(gx, level - 1, nb * 2), 256, 0, st>>>(ib, in_stride, ob, out_stride, tab, ctx->d_pc, N,
                                                                     level);
+        prof_end(ctx, PF_RESCALE, st);
     }
     FESC_CHECK_CUDA(ctx, cudaGetLastError());
     return FESC_OK;
@@ -455,8 +473,10 @@ int ctmul_internal(fesc_ctx* ctx, const u64* a, size_t a_stride, const u64* b, s
     for (uint32_t b0 = 0; b0 < batch; b0 += chunk) {
         uint32_t nb = batch - b0 < chunk ? batch - b0 : chunk;
         dim3 g((ctx->N + 255) / 256, level, nb);
+        prof_begin(ctx, PF_POINTWISE, st);
         k_tensor<<<g, 256, 0, st>>>(a + (size_t)b0 * a_stride, a_stride, b + (size_t)b0 * b_stride, b_stride,
                                     out + (size_t)b0 * out_stride, out_stride, ws.d, ws.dcoef, ctx->d_pc, ctx->N, level);
+        prof_end(ctx, PF_POINTWISE, st);
         int rc = key_switch_chunk(ctx, ws, key, level, nb, out + (size_t)b0 * out_stride, out_stride, 3, st);
         if (rc != FESC_OK) return rc;
     }
