@@ -252,6 +252,8 @@ def run_ours(args):
     for g in range(1, N2):
         ctx.add_galois_key(g * N1 * T_SEG, GIANT_BASE + g)
     gin, nout, tbs = workload_dims(args.scale_down)
+    if args.profile_case:       # small case for profiler captures: a few GB on the device
+        gin, nout, tbs = 1, 1, 2
     ks_per_step = key_switches_per_step(gin, nout, tbs)
     ct, diags = make_inputs(p["primes"], n, gin, nout, tbs, S.config_seed(4) + rank, dev)
     out = torch.empty((tbs, nout, 2, LEVEL - 1, n), dtype=torch.int64, device=dev)
@@ -260,6 +262,14 @@ def run_ours(args):
 
     def step():
         ctx.linear(ct, diags, desc, out)
+
+    if args.profile_case or args.profile_step:
+        # one bare step for a profiler capture (no warm-up, no timing claims)
+        step()
+        torch.cuda.synchronize()
+        print(json.dumps({"profile_run": True, "gpu_launches": ctx.counters()[4],
+                          "dims": {"in_blocks": gin, "out_blocks": nout, "token_blocks": tbs}}), flush=True)
+        return
 
     # warm-up (also sizes the scratch arena) and a family breakdown on one untimed step
     for _ in range(max(3, args.warmup) - 1):
@@ -368,6 +378,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale-down", dest="scale_down", type=int, default=1, help=argparse.SUPPRESS)
     ap.add_argument("--no-cpu", dest="no_cpu", action="store_true", help="skip the CPU baseline leg")
+    ap.add_argument("--profile-case", dest="profile_case", action="store_true",
+                    help="run ONE step of a small case (1 input block, 1 output block, 2 token blocks) and exit; for ncu")
+    ap.add_argument("--profile-step", dest="profile_step", action="store_true",
+                    help="run ONE step of the full workload without warm-up and exit; for the ncu launch list")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
