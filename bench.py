@@ -166,8 +166,9 @@ def peaks():
 
 # Integer-pipe ceiling for the 128-bit multiply-accumulate kernels: see DESIGN.md ("ALU roofline").
 SM_COUNT = 148
-IMAD_PER_CLK_PER_SM = 64          # 32-bit integer multiply-add issue rate assumed per SM per clock
-MAC128_IMAD = 4                   # one 64x64->128 product = 4 32x32->64 multiply-adds at minimum
+IMAD_PER_CLK_PER_SM = 64          # 32-bit multiply-adds per SM per clock (measured 63.6 with a register chain)
+MAC128_IMAD = 8                   # 64x64->128 multiply-accumulate = 4 products of 32x32->64 = 8 multiply-adds
+BFLY_IMAD = 20                    # Shoup butterfly = one high + two low 64-bit products = 10 products
 
 
 # ---------------------------------------------------------------------------------------------
@@ -285,6 +286,7 @@ def run_ours(args):
     # timed region
     ctx.profile_enable([dominant], 120000)
     launches0 = ctx.counters()[4]
+    limb_ntts0 = ctx.counters()[0]
     sampler = ClockSampler(local)
     torch.cuda.synchronize()
     barrier()
@@ -299,6 +301,7 @@ def run_ours(args):
     clocks = sampler.stop()
     ms_total = max_over_ranks(e0.elapsed_time(e1), dev)
     launches = ctx.counters()[4] - launches0
+    limb_ntts = ctx.counters()[0] - limb_ntts0
     dom_ms, dom_records = ctx.profile_read()[dominant]
     ctx.profile_enable([])
     ms_per_step = ms_total / args.steps
@@ -322,6 +325,18 @@ def run_ours(args):
                      "frac": macs / t / 1e12 / alu_peak, "traffic": None,
                      "hbm": {"achieved": alg / t / 1e9, "peak": hbm_peak, "unit": "GB/s", "frac": alg / t / 1e9 / hbm_peak,
                              "algorithmic_bytes_per_launch": alg}})
+    elif dominant == "ntt":
+        # all transform launches of the timed steps: butterflies per second against the multiply-add ceiling
+        bfly = limb_ntts * (n // 2) * p["log_n"]
+        sm_mhz = clocks.get("sm_mhz") or 1350.0
+        alu_peak = SM_COUNT * IMAD_PER_CLK_PER_SM * sm_mhz * 1e6 / BFLY_IMAD / 1e12
+        ach = bfly / (dom_ms * 1e-3) / 1e12
+        roof.update({"bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "T butterflies/s",
+                     "frac": ach / alu_peak, "traffic": None, "limb_transforms_per_step": limb_ntts // args.steps,
+                     "family_ms_per_step": dom_ms / args.steps,
+                     "hbm": {"achieved": limb_ntts * 2 * n * 8 / (dom_ms * 1e-3) / 1e9, "peak": hbm_peak, "unit": "GB/s",
+                             "frac": limb_ntts * 2 * n * 8 / (dom_ms * 1e-3) / 1e9 / hbm_peak,
+                             "algorithmic_bytes_per_limb_transform": 2 * n * 8}})
     else:
         t = dom_ms * 1e-3 / max(1, dom_records)
         roof.update({"bound": "alu", "achieved": None, "peak": None, "unit": "ms/launch", "frac": None,

@@ -100,6 +100,15 @@ def params(name: str) -> dict:
         special = ntt_primes(60, 10, 4, seed)
         return dict(name=name, log_n=10, primes=data + special, n_q=24, n_p=4, dnum=6,
                     seed=seed, log_scale=40)
+    if name in ("scan_toy", "scan_small"):
+        # rings for the scan-contract tests: the paper's toy shape (16 slots) and a 128-slot analogue of
+        # the Mamba-2-base geometry; 50-bit chain, two 60-bit special primes, two limbs per digit
+        log_n, n_q = (5, 10) if name == "scan_toy" else (8, 16)
+        seed = config_seed(5)
+        data = ntt_primes(50, log_n, n_q, seed)
+        special = ntt_primes(60, log_n, 2, seed)
+        return dict(name=name, log_n=log_n, primes=data + special, n_q=n_q, n_p=2, dnum=n_q // 2,
+                    seed=seed, log_scale=40)
     raise KeyError(name)
 
 

@@ -1,0 +1,105 @@
+"""Pins for the scan-contract oracle: the float64 recurrence against its closed form, the paper's
+composition / reduction counts, and decrypt(scan(Enc factors)) against the recurrence on the paper's
+toy shape (L=4, H=2, P=4, d_s=2, K_s=2) and on a 128-slot analogue of the Mamba-2-base geometry."""
+import math
+
+import numpy as np
+import pytest
+
+import fesc_synth as S
+from oracle.ckks import Oracle
+from oracle.scan import (ScanConsts, ScanEvaluator, ScanShape, add_scan_keys, closed_form_counts, encrypt_inputs,
+                         float_recurrence, levels, unpack_output)
+
+
+def test_recurrence_matches_unrolled_closed_form():
+    x, a, B, C = S.scan_inputs(3, 9, 2, 3, 1, 4)
+    m = float_recurrence(x, a, B, C)
+    for k in (0, 4, 8):
+        want = np.zeros((2, 3))
+        for kp in range(k + 1):
+            decay = np.prod(a[kp + 1:k + 1], axis=0)          # per head
+            want += decay[:, None] * x[kp] * float(B[kp, 0] @ C[k, 0])
+        assert np.allclose(m[k], want, rtol=1e-12, atol=1e-12)
+    # one hand-checked step: h_0 = 0 so m_0 = x_0 (B_0 . C_0)
+    assert np.allclose(m[0], x[0] * float(B[0, 0] @ C[0, 0]))
+
+
+def _bk_nodes(B):
+    """(stage kind, left, right) of every composition of the network, 1-based positions."""
+    logB = int(math.log2(B))
+    nodes = []
+    for s in range(1, logB + 1):
+        nodes += [("up", k - (1 << (s - 1)), k) for k in range(1 << s, B + 1, 1 << s)]
+    for s in range(logB - 1, 0, -1):
+        nodes += [("down", k, k + (1 << (s - 1))) for k in range(1 << s, B, 1 << s) if k + (1 << (s - 1)) < B]
+    return nodes
+
+
+@pytest.mark.parametrize("B", [4, 8, 16, 256])
+def test_brent_kung_network_counts_and_prefixes(B):
+    nodes = _bk_nodes(B)
+    logB = int(math.log2(B))
+    assert sum(1 for n in nodes if n[0] == "up") == B - 1                    # App. "Prefix-Network Selection"
+    assert sum(1 for n in nodes if n[0] == "down") == B - 1 - logB
+    assert len(nodes) == 2 * B - logB - 2                                    # C_BK(n) = 2n - log2 n - 2
+    # the network computes every inclusive prefix: track covered intervals
+    cover = {k: (k, k) for k in range(1, B + 1)}
+    for _, l, r in nodes:
+        assert cover[l][1] + 1 == cover[r][0]
+        cover[r] = (cover[l][0], cover[r][1])
+    assert all(cover[k] == (1, k) for k in range(1, B + 1))
+
+
+def test_paper_ledger_values():
+    # Table "real-phantom-scan", Brent-Kung column: 2 * K_s * (2(L'-1) - log2 L') key switches, K_s = 12
+    for Lp, printed in ((128, 5.9e3), (256, 12.0e3), (512, 24.3e3), (1024, 48.9e3), (2048, 98.0e3)):
+        ks = 2 * 12 * (2 * (Lp - 1) - int(math.log2(Lp)))
+        assert abs(ks - printed) / printed < 0.01
+    assert 2 * 12 * (2 * 127 - 7) == 5928                                     # Table "cross_ssm_family", Mamba-2
+    # depth 2 ceil(log2 L') - 1
+    assert [2 * int(math.log2(Lp)) - 1 for Lp in (128, 256, 512, 1024, 2048)] == [13, 15, 17, 19, 21]
+    # K_s and reduction counts of the deployed shape (App. "Complex-Packed Reduction Accounting")
+    assert math.ceil(1536 * 128 / 16384) == 12
+    sh = ScanShape(32768, L=2048, H=24, P=64, d_s=128, B_blk=256)
+    assert (sh.K_s, sh.K_blk, sh.c_state, sh.hpc, sh.stride) == (12, 8, 128, 2, 256)
+    cf = closed_form_counts(sh)
+    assert cf["reduce_rot"] == 86016 and cf["reduce_conj"] == 12288
+    assert cf["compose"] == 96 * 502
+    lv = levels(24, sh.logB, sh.K_blk)
+    assert lv == dict(l0=24, l1=22, lS=14, linj=7, lout=4)
+    assert 2 * 768 // 768 and 2 * 24 * 64 + 2 * 128 + 24 == 3352              # d_out of in_proj
+
+
+def _run(name, **shape_kw):
+    p = S.params(name)
+    orc = Oracle(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+    sh = ScanShape(orc.n, **shape_kw)
+    x, a, B, C = S.scan_inputs(p["seed"], sh.L, sh.H, sh.P, 1, sh.d_s)
+    c = ScanConsts(orc, sh, p["n_q"], p["log_scale"])
+    add_scan_keys(orc, sh)
+    ev = ScanEvaluator(orc, sh, c)
+    out = ev.run(*encrypt_inputs(orc, sh, c, x, a, B, C))
+    return sh, ev, unpack_output(orc, sh, c, out), float_recurrence(x, a, B, C)
+
+
+def test_paper_toy_shape():
+    sh, ev, m, ref = _run("scan_toy", L=4, H=2, P=4, d_s=2, B_blk=4)
+    assert sh.K_s == 2 and ev.count["compose"] == closed_form_counts(sh)["compose"] == 8
+    assert ev.count["conj"] == closed_form_counts(sh)["reduce_conj"]
+    assert np.abs(m - ref).max() < 2.0**-24
+
+
+def test_analogue_with_carries_and_partial_block():
+    sh, ev, m, ref = _run("scan_small", L=40, H=8, P=4, d_s=8, B_blk=16)
+    cf = closed_form_counts(sh)
+    assert (sh.K_s, sh.K_blk, sh.hpc) == (4, 3, 2)
+    assert ev.count["compose"] == cf["compose"] == 312 and ev.count["conj"] == cf["reduce_conj"] == 96
+    assert np.abs(m - ref).max() < 2.0**-22
+
+
+def test_two_digit_offsets_and_odd_chunk_count():
+    sh, ev, m, ref = _run("scan_small", L=64, H=3, P=4, d_s=4, B_blk=32)
+    assert (sh.K_s, sh.K_blk, sh.dg, sh.hpc) == (3, 2, 16, 1)
+    assert ev.count["conj"] == closed_form_counts(sh)["reduce_conj"] == 64
+    assert np.abs(m - ref).max() < 2.0**-22
