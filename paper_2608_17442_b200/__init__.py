@@ -32,6 +32,14 @@ class BsgsDesc(ctypes.Structure):
                 ("n1", "n2", "in_blocks", "out_blocks", "token_blocks", "n_limbs", "baby_key_base", "giant_key_base")]
 
 
+class ScanDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint32) for n in ("L", "H", "P", "d_s", "B_blk", "stride", "n_limbs", "key_base")]
+
+
+class ScanConsts(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("d_mask_x", "d_mask_b", "d_mask_a", "d_mask_out", "adj_s", "adj_p")]
+
+
 def lib():
     """Load libfesc_b200.so (built by paper_2608_17442_b200.build); raise if it is missing."""
     global _lib
@@ -59,6 +67,7 @@ def lib():
             "fesc_rescale": [vp, vp, vp, u32, u32, vp],
             "fesc_ct_ct_mul": [vp, vp, vp, vp, u32, u32, vp],
             "fesc_linear": [vp, vp, vp, c.POINTER(BsgsDesc), vp, vp],
+            "fesc_scan_contract": [vp, vp, vp, vp, vp, c.POINTER(ScanDesc), c.POINTER(ScanConsts), vp, vp],
         }
         for name, args in sig.items():
             f = getattr(L, name)
@@ -175,3 +184,13 @@ class Context:
 
     def linear(self, ct_in, diags, desc: BsgsDesc, ct_out):
         self._chk(lib().fesc_linear(self.h, _ptr(ct_in), _ptr(diags), ctypes.byref(desc), _ptr(ct_out), _stream()))
+
+    def scan_contract(self, x, a, B, C, desc: ScanDesc, mask_x, mask_b, mask_a, mask_out, adj_s, adj_p, m_out):
+        """adj_s / adj_p: sequences of (n_limbs+1)^2 Python ints (host tables); masks: CUDA tensors."""
+        n = (desc.n_limbs + 1) ** 2
+        hs = (ctypes.c_uint64 * n)(*[int(v) for v in adj_s])
+        hp = (ctypes.c_uint64 * n)(*[int(v) for v in adj_p])
+        cs = ScanConsts(mask_x.data_ptr(), mask_b.data_ptr(), mask_a.data_ptr(), mask_out.data_ptr(),
+                        ctypes.cast(hs, ctypes.c_void_p).value, ctypes.cast(hp, ctypes.c_void_p).value)
+        self._chk(lib().fesc_scan_contract(self.h, _ptr(x), _ptr(a), _ptr(B), _ptr(C), ctypes.byref(desc),
+                                           ctypes.byref(cs), _ptr(m_out), _stream()))

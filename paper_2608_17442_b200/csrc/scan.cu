@@ -1,0 +1,510 @@
+// Factorized scan-contract on packed ciphertexts:
+//   h_k = br(a_k) (.) h_{k-1} + x_k (x) B_k,  h_0 = 0,   m_k = Sigma_{d_s}(h_k (.) br(C_k))
+// evaluated as: per token block, broadcast of the compact factors to the state packing (rotations,
+// masks, rotate-and-add fills), leaves (p, s) = (br a, br x (.) br B), a Brent-Kung network of affine
+// compositions (p_R p_L, p_R s_L + s_R), serialized block carries, carry injection, contraction with
+// br(C), a complex-paired rotate-add reduction over the state axis with one conjugation per chunk
+// pair, output mask and placement.  The host code below only sequences batched kernels (rotations
+// share a key per batch); every arithmetic step runs in the kernels of ops.cu / ntt.cu and the
+// pointwise kernels here.  Levels follow a fixed schedule (see fesc.h).
+#include <math.h>
+
+#include "ops.cuh"
+
+// ---------------------------------------------------------------------------------------
+// pointwise kernels on batches of compact ciphertexts [2][level][N]
+// ---------------------------------------------------------------------------------------
+// out = a + b (sub = 0) or a - b (sub = 1); b_stride may be 0
+__global__ void __launch_bounds__(256) k_ct_addsub(const u64* __restrict__ a, size_t a_stride, const u64* __restrict__ b,
+                                                   size_t b_stride, u64* __restrict__ out, size_t out_stride,
+                                                   const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
+                                                   int sub) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t pl = blockIdx.y, bi = blockIdx.z;   // pl = poly*level + limb
+    if (c >= N) return;
+    const u64 q = pcs[pl % level].q;
+    const size_t o = (size_t)pl * N + c;
+    const u64 x = a[bi * a_stride + o], y = b[bi * b_stride + o];
+    out[bi * out_stride + o] = sub ? submod(x, y, q) : addmod(x, y, q);
+}
+// out = ct (.) pt  (pt shared by the batch, [level][N])
+__global__ void __launch_bounds__(256) k_ct_ptmul(const u64* __restrict__ a, size_t a_stride, const u64* __restrict__ pt,
+                                                  u64* __restrict__ out, size_t out_stride,
+                                                  const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t l = blockIdx.y, bi = blockIdx.z;
+    if (c >= N) return;
+    const PrimeConst pc = pcs[l];
+    const size_t o = (size_t)l * N + c, poly = (size_t)level * N;
+    const u64 w = pt[o];
+    out[bi * out_stride + o] = mulmod(a[bi * a_stride + o], w, pc);
+    out[bi * out_stride + poly + o] = mulmod(a[bi * a_stride + poly + o], w, pc);
+}
+// keep the first `keep` limbs of a level-`src` ciphertext and multiply them by the integer k
+__global__ void __launch_bounds__(256) k_ct_scale_drop(const u64* __restrict__ a, size_t a_stride, u64* __restrict__ out,
+                                                       size_t out_stride, const PrimeConst* __restrict__ pcs, uint32_t N,
+                                                       uint32_t src, uint32_t keep, u64 k) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t l = blockIdx.y % keep, p = blockIdx.y / keep, bi = blockIdx.z;
+    if (c >= N) return;
+    const PrimeConst pc = pcs[l];
+    const u64 kk = k - mulhi(k, pc.mu) * pc.q;   // k mod q in [0, 2q)
+    out[bi * out_stride + ((size_t)p * keep + l) * N + c] =
+        mulmod(a[bi * a_stride + ((size_t)p * src + l) * N + c], csub(kk, pc.q), pc);
+}
+// multiply by the monomial X^(N/2) `times` times (times = 1: slots * i; times = 3: slots * -i).
+// In evaluation order X^(N/2) is I = psi^(N/2) on the first half of the indices and -I on the second.
+__global__ void __launch_bounds__(256) k_ct_mul_i(const u64* __restrict__ a, size_t a_stride, u64* __restrict__ out,
+                                                  size_t out_stride, const PrimeConst* __restrict__ pcs,
+                                                  const ulonglong2* __restrict__ tw, uint32_t N, uint32_t level,
+                                                  int times) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t pl = blockIdx.y, bi = blockIdx.z;
+    if (c >= N) return;
+    const uint32_t l = pl % level;
+    const u64 q = pcs[l].q;
+    const ulonglong2 I = tw[(size_t)l * N + 1];
+    const size_t o = (size_t)pl * N + c;
+    u64 v = shoup(a[bi * a_stride + o], I.x, I.y, q);
+    const bool neg = (c >= N / 2) != (times == 3);
+    out[bi * out_stride + o] = (neg && v) ? q - v : v;
+}
+// acc += sum over the batch
+__global__ void __launch_bounds__(256) k_ct_sum_into(const u64* __restrict__ a, size_t a_stride, uint32_t count,
+                                                     u64* __restrict__ acc, const PrimeConst* __restrict__ pcs,
+                                                     uint32_t N, uint32_t level) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t pl = blockIdx.y;
+    if (c >= N) return;
+    const u64 q = pcs[pl % level].q;
+    const size_t o = (size_t)pl * N + c;
+    u64 s = acc[o];
+    for (uint32_t i = 0; i < count; i++) s = addmod(s, a[i * a_stride + o], q);
+    acc[o] = s;
+}
+
+// ---------------------------------------------------------------------------------------
+// host-side sequencing
+// ---------------------------------------------------------------------------------------
+namespace {
+
+struct Arr {          // `count` compact ciphertexts [2][level][N], `stride` words apart
+    u64* p;
+    uint32_t count, level;
+    size_t stride;
+};
+
+struct Geometry {
+    uint32_t n, L, H, P, d_s, B, stride, c_state, E, hpc, R, K_s, K_blk, logB, dg;
+    uint32_t l0, l1, lS, linj, lout;
+};
+
+static uint32_t ilog2(uint32_t x) {
+    uint32_t r = 0;
+    while ((1u << (r + 1)) <= x) r++;
+    return r;
+}
+
+struct Exec {
+    fesc_ctx* ctx;
+    cudaStream_t st;
+    Geometry g;
+    const fesc_scan_desc* desc;
+    const fesc_scan_consts* cs;
+    bool dry;               // planning pass: no launches, only arena accounting
+    u64* arena;
+    size_t top, high;
+    u64* ks;                // key-switch scratch
+    u64* rs;                // rescale scratch
+    int rc;
+    uint32_t N;
+
+    size_t ctw(uint32_t level) const { return (size_t)2 * level * N; }
+    Arr alloc(uint32_t count, uint32_t level) {
+        Arr a{arena + top, count, level, ctw(level)};
+        top += (size_t)count * ctw(level);
+        if (top > high) high = top;
+        return a;
+    }
+    Arr at(const Arr& a, uint32_t i, uint32_t count = 1) const { return Arr{a.p + (size_t)i * a.stride, count, a.level, a.stride}; }
+    Arr strided(const Arr& a, uint32_t first, uint32_t step, uint32_t count) const {
+        return Arr{a.p + (size_t)first * a.stride, count, a.level, a.stride * step};
+    }
+    bool ok() const { return rc == FESC_OK; }
+    dim3 grid(uint32_t rows, uint32_t batch) const { return dim3((N + 255) / 256, rows, batch); }
+
+    uint32_t key_for(int64_t amount) const {
+        int64_t n = g.n;
+        return desc->key_base + (uint32_t)(((amount % n) + n) % n);
+    }
+    // out = rot(in, amount)   (amount = slot LEFT shift; in and out must not overlap)
+    void rot(const Arr& in, int64_t amount, const Arr& out) {
+        if (!ok()) return;
+        if (((amount % (int64_t)g.n) + g.n) % g.n == 0) return copy(in, out);
+        uint32_t kid = key_for(amount);
+        if (!ctx->keys.count(kid)) {
+            rc = fesc_fail(ctx, FESC_ENOKEY, "scan_contract: missing Galois key " + std::to_string(kid));
+            return;
+        }
+        if (dry) return;
+        rc = rotate_internal(ctx, in.p, in.stride, out.p, out.stride, in.count, in.level, kid, ks, st, 0);
+    }
+    void conj(const Arr& in, const Arr& out) {
+        if (!ok()) return;
+        uint32_t kid = desc->key_base + g.n;
+        if (!ctx->keys.count(kid)) {
+            rc = fesc_fail(ctx, FESC_ENOKEY, "scan_contract: missing conjugation key");
+            return;
+        }
+        if (dry) return;
+        rc = rotate_internal(ctx, in.p, in.stride, out.p, out.stride, in.count, in.level, kid, ks, st, 0);
+    }
+    void copy(const Arr& in, const Arr& out) {
+        if (!ok() || dry || in.p == out.p) return;
+        size_t w = ctw(in.level) * sizeof(u64);
+        cudaError_t e = cudaMemcpy2DAsync(out.p, out.stride * sizeof(u64), in.p, in.stride * sizeof(u64), w, in.count,
+                                          cudaMemcpyDeviceToDevice, st);
+        if (e != cudaSuccess) rc = fesc_fail(ctx, FESC_ECUDA, cudaGetErrorString(e));
+    }
+    void addsub(const Arr& a, const Arr& b, const Arr& out, int sub) {
+        if (!ok() || dry) return;
+        prof_begin(ctx, PF_POINTWISE, st);
+        k_ct_addsub<<<grid(2 * a.level, a.count), 256, 0, st>>>(a.p, a.stride, b.p, b.count == 1 && a.count > 1 ? 0 : b.stride,
+                                                                out.p, out.stride, ctx->d_pc, N, a.level, sub);
+        prof_end(ctx, PF_POINTWISE, st);
+    }
+    void add(const Arr& a, const Arr& b, const Arr& out) { addsub(a, b, out, 0); }
+    void sub(const Arr& a, const Arr& b, const Arr& out) { addsub(a, b, out, 1); }
+    void mul_i(const Arr& a, const Arr& out, int times) {
+        if (!ok() || dry) return;
+        prof_begin(ctx, PF_POINTWISE, st);
+        k_ct_mul_i<<<grid(2 * a.level, a.count), 256, 0, st>>>(a.p, a.stride, out.p, out.stride, ctx->d_pc, ctx->d_tw, N,
+                                                               a.level, times);
+        prof_end(ctx, PF_POINTWISE, st);
+    }
+    // contiguous `in` at level l -> contiguous `out` at level l-1
+    void rescale(const Arr& in, const Arr& out) {
+        if (!ok() || dry) return;
+        rc = rescale_internal(ctx, in.p, in.stride, out.p, in.count, in.level, rs, st);
+    }
+    // out (level-1, contiguous) = rescale(in (.) pt)
+    void ptmul_rescale(const Arr& in, const u64* pt, const Arr& out) {
+        size_t mark = top;
+        Arr t = alloc(in.count, in.level);
+        if (ok() && !dry) {
+            prof_begin(ctx, PF_POINTWISE, st);
+            k_ct_ptmul<<<grid(in.level, in.count), 256, 0, st>>>(in.p, in.stride, pt, t.p, t.stride, ctx->d_pc, N, in.level);
+            prof_end(ctx, PF_POINTWISE, st);
+            ctx->counters[2] += in.count;
+        }
+        rescale(t, out);
+        top = mark;
+    }
+    // out (level-1, contiguous) = rescale(a * b); b may be a single ciphertext shared by the batch
+    void mul_rescale(const Arr& a, const Arr& b, const Arr& out) {
+        size_t mark = top;
+        Arr t = alloc(a.count, a.level);
+        if (ok() && !dry)
+            rc = ctmul_internal(ctx, a.p, a.stride, b.p, (b.count == 1 && a.count > 1) ? 0 : b.stride, t.p, t.stride, a.count,
+                                a.level, ks, st);
+        rescale(t, out);
+        top = mark;
+    }
+    // out (level dst, contiguous) = in brought from its level to dst; kind 0: state-like, 1: multiplicand
+    void adjust(const Arr& in, uint32_t dst, int kind, const Arr& out) {
+        if (!ok()) return;
+        if (in.level == dst) return copy(in, out);
+        if (in.level < dst) {
+            rc = fesc_fail(ctx, FESC_ELEVEL, "scan_contract: level schedule violated");
+            return;
+        }
+        size_t mark = top;
+        Arr t = alloc(in.count, dst + 1);
+        if (!dry) {
+            const uint64_t* tab = kind ? cs->adj_p : cs->adj_s;
+            u64 k = tab[(size_t)in.level * (g.l0 + 1) + dst];
+            prof_begin(ctx, PF_POINTWISE, st);
+            k_ct_scale_drop<<<grid(2 * (dst + 1), in.count), 256, 0, st>>>(in.p, in.stride, t.p, t.stride, ctx->d_pc, N,
+                                                                           in.level, dst + 1, k);
+            prof_end(ctx, PF_POINTWISE, st);
+        }
+        rescale(t, out);
+        top = mark;
+    }
+    // a += rot(a, -unit * 2^b) for b = 0..steps-1
+    void fill_right(const Arr& a, uint32_t unit, uint32_t steps) {
+        size_t mark = top;
+        Arr t = alloc(a.count, a.level);
+        for (uint32_t b = 0; b < steps; b++) {
+            rot(a, -(int64_t)(unit << b), t);
+            add(a, t, a);
+        }
+        top = mark;
+    }
+    // out[t] = rot(src, unit * t) for t = 0..B-1, via t = t_lo + dg * t_hi
+    void extract_all(const Arr& src, int64_t unit, const Arr& out) {
+        size_t mark = top;
+        const uint32_t nh = g.B / g.dg;
+        Arr gi = alloc(nh, src.level);
+        for (uint32_t th = 0; th < nh; th++) rot(src, unit * (int64_t)(g.dg * th), at(gi, th));
+        for (uint32_t tl = 0; tl < g.dg; tl++) rot(gi, unit * (int64_t)tl, strided(out, tl, g.dg, nh));
+        top = mark;
+    }
+};
+
+}  // namespace
+
+static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, const u64* d_C, u64* d_out) {
+    const Geometry& g = X.g;
+    const uint32_t B = g.B, l0 = g.l0, l1 = g.l1, lS = g.lS, linj = g.linj, lout = g.lout;
+    const uint32_t N = X.N;
+    const size_t in_ctw = X.ctw(l0), out_ctw = X.ctw(lout);
+    if (!X.dry) {
+        cudaError_t e = cudaMemsetAsync(d_out, 0, (size_t)g.K_blk * g.K_s * out_ctw * sizeof(u64), X.st);
+        if (e != cudaSuccess) return fesc_fail(X.ctx, FESC_ECUDA, cudaGetErrorString(e));
+    }
+    // carries g_j per chunk (level lS - (j-1)), stored at capacity lS
+    Arr carry = X.alloc(g.K_s, lS);
+    std::vector<uint32_t> carry_level(g.K_s, 0);
+    for (uint32_t j = 0; j < g.K_blk && X.ok(); j++) {
+        const size_t block_mark = X.top;
+        // ---- br(B_t) at l0-1 and br(C_t) at linj-1, shared by every chunk ----
+        Arr brB = X.alloc(B, l0 - 1), brC = X.alloc(B, linj - 1);
+        for (int which = 0; which < 2; which++) {
+            size_t m = X.top;
+            Arr src{const_cast<u64*>((which ? d_C : d_B) + (size_t)j * in_ctw), 1, l0, in_ctw};
+            Arr ex = X.alloc(B, l0);
+            X.extract_all(src, g.d_s, ex);
+            if (which == 0) {
+                X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_b, brB);
+                X.fill_right(brB, g.stride, ilog2(g.c_state));
+            } else {
+                Arr full = X.alloc(B, l0 - 1);
+                X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_b, full);
+                X.fill_right(full, g.stride, ilog2(g.c_state));
+                X.adjust(full, linj - 1, 1, brC);
+            }
+            X.top = m;
+        }
+        // contracted products of the block, [chunk parity][token], level linj-2
+        Arr V = X.alloc(2 * B, linj - 2);
+        for (uint32_t kap = 0; kap < g.K_s && X.ok(); kap++) {
+            const size_t chunk_mark = X.top;
+            // position slots of the prefix network: capacity l1, current level tracked on the host
+            Arr Ps = X.alloc(B, l1), Ss = X.alloc(B, l1);
+            std::vector<uint32_t> lp(B, l1), ls(B, l1);
+            {   // ---- leaves ----
+                size_t m = X.top;
+                Arr srcx{const_cast<u64*>(d_x + ((size_t)j * g.K_s + kap) * in_ctw), 1, l0, in_ctw};
+                Arr apre = X.alloc(1, l0);
+                X.copy(Arr{const_cast<u64*>(d_a + ((size_t)j * g.K_s + kap) * in_ctw), 1, l0, in_ctw}, apre);
+                X.fill_right(apre, 1, ilog2(g.P));
+                Arr ex = X.alloc(B, l0), xr = X.alloc(B, l0 - 1), ar = X.alloc(B, l0 - 1);
+                X.extract_all(srcx, 1, ex);
+                X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_x, xr);
+                X.fill_right(xr, 1, ilog2(g.d_s));
+                X.extract_all(apre, g.P, ex);
+                X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_a, ar);
+                X.fill_right(ar, g.P, ilog2(g.R / g.P));
+                X.mul_rescale(xr, brB, Ss);      // s_t = br(x_t) (.) br(B_t), level l1 (slots are compact at l1)
+                X.adjust(ar, l1, 1, Ps);         // p_t = br(a_t)
+                X.top = m;
+            }
+            // ---- Brent-Kung network ----
+            // one stage: nodes (left position, right position), operands brought to `lvl`, results at lvl-1
+            auto stage = [&](const std::vector<uint32_t>& left, const std::vector<uint32_t>& right, uint32_t lvl, bool need_p) {
+                const uint32_t cnt = (uint32_t)left.size();
+                if (!cnt || !X.ok()) return;
+                size_t m = X.top;
+                Arr pL = X.alloc(cnt, lvl), sL = X.alloc(cnt, lvl), pR = X.alloc(cnt, lvl), sR = X.alloc(cnt, lvl - 1);
+                Arr np_ = X.alloc(cnt, lvl - 1), ns = X.alloc(cnt, lvl - 1);
+                for (uint32_t i = 0; i < cnt; i++) {
+                    const uint32_t a = left[i], b = right[i];
+                    if (need_p) X.adjust(Arr{Ps.p + (size_t)a * Ps.stride, 1, lp[a], X.ctw(lp[a])}, lvl, 1, X.at(pL, i));
+                    X.adjust(Arr{Ss.p + (size_t)a * Ss.stride, 1, ls[a], X.ctw(ls[a])}, lvl, 0, X.at(sL, i));
+                    X.adjust(Arr{Ps.p + (size_t)b * Ps.stride, 1, lp[b], X.ctw(lp[b])}, lvl, 1, X.at(pR, i));
+                    X.adjust(Arr{Ss.p + (size_t)b * Ss.stride, 1, ls[b], X.ctw(ls[b])}, lvl - 1, 0, X.at(sR, i));
+                }
+                if (need_p) X.mul_rescale(pR, pL, np_);
+                X.mul_rescale(pR, sL, ns);
+                X.add(ns, sR, ns);
+                for (uint32_t i = 0; i < cnt; i++) {
+                    const uint32_t b = right[i];
+                    if (need_p) {
+                        X.copy(X.at(np_, i), Arr{Ps.p + (size_t)b * Ps.stride, 1, lvl - 1, X.ctw(lvl - 1)});
+                        lp[b] = lvl - 1;
+                    }
+                    X.copy(X.at(ns, i), Arr{Ss.p + (size_t)b * Ss.stride, 1, lvl - 1, X.ctw(lvl - 1)});
+                    ls[b] = lvl - 1;
+                }
+                X.top = m;
+            };
+            for (uint32_t s = 1; s <= g.logB; s++) {
+                std::vector<uint32_t> left, right;
+                for (uint32_t k = 1u << s; k <= B; k += 1u << s) {
+                    left.push_back(k - (1u << (s - 1)) - 1);
+                    right.push_back(k - 1);
+                }
+                stage(left, right, l1 - (s - 1), true);
+            }
+            // summary of the block = last position after the up-sweep; keep a copy for the carry
+            Arr sumP = X.alloc(1, lS), sumS = X.alloc(1, lS);
+            X.copy(Arr{Ps.p + (size_t)(B - 1) * Ps.stride, 1, lS, X.ctw(lS)}, sumP);
+            X.copy(Arr{Ss.p + (size_t)(B - 1) * Ss.stride, 1, lS, X.ctw(lS)}, sumS);
+            uint32_t d = 0;
+            for (uint32_t s = g.logB - 1; s >= 1; s--) {
+                d++;
+                std::vector<uint32_t> left, right;
+                for (uint32_t k = 1u << s; k < B; k += 1u << s) {
+                    uint32_t r = k + (1u << (s - 1));
+                    if (r < B) {
+                        left.push_back(k - 1);
+                        right.push_back(r - 1);
+                    }
+                }
+                stage(left, right, lS - (d - 1), j > 0);
+            }
+            // ---- carry injection and contraction with br(C_t) ----
+            {
+                size_t m = X.top;
+                Arr h = X.alloc(B, linj - 1);
+                for (uint32_t t = 0; t < B; t++)
+                    X.adjust(Arr{Ss.p + (size_t)t * Ss.stride, 1, ls[t], X.ctw(ls[t])}, linj - 1, 0, X.at(h, t));
+                if (j > 0) {
+                    Arr pp = X.alloc(B, linj), gg = X.alloc(1, linj), pg = X.alloc(B, linj - 1);
+                    for (uint32_t t = 0; t < B; t++)
+                        X.adjust(Arr{Ps.p + (size_t)t * Ps.stride, 1, lp[t], X.ctw(lp[t])}, linj, 1, X.at(pp, t));
+                    X.adjust(Arr{carry.p + (size_t)kap * carry.stride, 1, carry_level[kap], X.ctw(carry_level[kap])}, linj, 0, gg);
+                    X.mul_rescale(pp, gg, pg);
+                    X.add(h, pg, h);
+                }
+                X.mul_rescale(h, brC, X.at(V, (kap & 1) * B, B));
+                X.top = m;
+            }
+            // ---- serialized carry g_{j+1} = S_j(g_j) ----
+            if (j + 1 < g.K_blk) {
+                Arr slot{carry.p + (size_t)kap * carry.stride, 1, 0, 0};
+                if (j == 0) {
+                    slot.level = lS;
+                    slot.stride = X.ctw(lS);
+                    X.copy(sumS, slot);
+                    carry_level[kap] = lS;
+                } else {
+                    const uint32_t lg = carry_level[kap];
+                    size_t m = X.top;
+                    Arr gcur{slot.p, 1, lg, X.ctw(lg)};
+                    Arr pa = X.alloc(1, lg), sa = X.alloc(1, lg - 1), ng = X.alloc(1, lg - 1);
+                    X.adjust(sumP, lg, 1, pa);
+                    X.adjust(sumS, lg - 1, 0, sa);
+                    X.mul_rescale(pa, gcur, ng);
+                    X.add(ng, sa, ng);
+                    X.copy(ng, Arr{slot.p, 1, lg - 1, X.ctw(lg - 1)});
+                    carry_level[kap] = lg - 1;
+                    X.top = m;
+                }
+            }
+            X.top = chunk_mark;
+            // ---- state-axis reduction of a chunk pair (or of the unpaired last chunk) ----
+            const bool second = (kap & 1) != 0, last = kap + 1 == g.K_s;
+            if (second || last) {
+                const bool paired = second;
+                const uint32_t k0 = paired ? kap - 1 : kap;
+                const uint32_t lred = linj - 2;
+                size_t m = X.top;
+                Arr chi = X.alloc(B, lred), tmp = X.alloc(B, lred);
+                Arr v0 = X.at(V, (k0 & 1) * B, B), v1 = X.at(V, ((k0 + 1) & 1) * B, B);
+                if (paired) {
+                    X.mul_i(v1, tmp, 1);
+                    X.add(v0, tmp, chi);
+                } else {
+                    X.copy(v0, chi);
+                }
+                for (uint32_t b = 0; b < ilog2(g.d_s); b++) {
+                    X.rot(chi, (int64_t)(1u << b), tmp);
+                    X.add(chi, tmp, chi);
+                }
+                Arr part = X.alloc(B, lred), y = X.alloc(B, lout), y2 = X.alloc(B, lout);
+                const uint32_t nparts = paired ? 2 : 1;
+                if (paired) X.conj(chi, tmp);
+                for (uint32_t which = 0; which < nparts; which++) {
+                    if (!paired) {
+                        X.add(chi, chi, part);
+                    } else if (which == 0) {
+                        X.add(chi, tmp, part);                 // 2 Re
+                    } else {
+                        X.sub(chi, tmp, part);
+                        X.mul_i(part, part, 3);                // -i (Xi - conj Xi) = 2 Im
+                    }
+                    X.ptmul_rescale(part, (const u64*)X.cs->d_mask_out, y);
+                    // placement: rotate right by t = t_lo + dg * t_hi
+                    const uint32_t nh = B / g.dg;
+                    for (uint32_t tl = 0; tl < g.dg; tl++)
+                        X.rot(X.strided(y, tl, g.dg, nh), -(int64_t)tl, X.strided(y2, tl, g.dg, nh));
+                    for (uint32_t th = 0; th < nh; th++)
+                        X.rot(X.at(y2, th * g.dg, g.dg), -(int64_t)(g.dg * th), X.at(y, th * g.dg, g.dg));
+                    if (X.ok() && !X.dry) {
+                        u64* dst = d_out + ((size_t)j * g.K_s + k0 + which) * out_ctw;
+                        prof_begin(X.ctx, PF_POINTWISE, X.st);
+                        k_ct_sum_into<<<dim3((N + 255) / 256, 2 * lout), 256, 0, X.st>>>(y.p, y.stride, B, dst, X.ctx->d_pc, N, lout);
+                        prof_end(X.ctx, PF_POINTWISE, X.st);
+                    }
+                }
+                X.top = m;
+            }
+        }
+        X.top = block_mark;
+    }
+    return X.rc;
+}
+
+extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint64_t* d_a, const uint64_t* d_B,
+                                  const uint64_t* d_C, const fesc_scan_desc* desc, const fesc_scan_consts* consts,
+                                  uint64_t* d_m_out, void* stream) {
+    if (!ctx || !d_x || !d_a || !d_B || !d_C || !desc || !consts || !d_m_out) return FESC_EINVAL;
+    if (!consts->d_mask_x || !consts->d_mask_a || !consts->d_mask_b || !consts->d_mask_out || !consts->adj_s || !consts->adj_p)
+        return fesc_fail(ctx, FESC_EINVAL, "scan_contract: missing constants");
+    Geometry g;
+    g.n = ctx->N / 2;
+    g.L = desc->L, g.H = desc->H, g.P = desc->P, g.d_s = desc->d_s, g.B = desc->B_blk;
+    auto pow2 = [](uint32_t v) { return v && !(v & (v - 1)); };
+    if (!g.L || !g.H || !pow2(g.P) || !pow2(g.d_s) || !pow2(g.B) || g.B < 2)
+        return fesc_fail(ctx, FESC_EINVAL, "scan_contract: P, d_s, B_blk must be powers of two, B_blk >= 2");
+    g.stride = desc->stride ? desc->stride : (g.d_s > g.B ? g.d_s : g.B);
+    if (!pow2(g.stride) || g.stride < g.d_s || g.stride < g.B || g.stride > g.n)
+        return fesc_fail(ctx, FESC_EINVAL, "scan_contract: bad stride");
+    g.c_state = g.n / g.stride;
+    g.E = g.H * g.P;
+    if (g.c_state % g.P || g.E % g.c_state) return fesc_fail(ctx, FESC_EINVAL, "scan_contract: channels do not tile the chunks");
+    g.hpc = g.c_state / g.P;
+    g.R = g.n / g.hpc;
+    g.K_s = g.E / g.c_state;
+    g.K_blk = (g.L + g.B - 1) / g.B;
+    g.logB = ilog2(g.B);
+    g.dg = g.B < 16 ? g.B : 16;
+    if ((uint64_t)g.B * g.d_s > g.n || (uint64_t)g.B * g.P > g.R)
+        return fesc_fail(ctx, FESC_EINVAL, "scan_contract: block does not fit the compact packings");
+    g.l0 = desc->n_limbs;
+    if (g.l0 > ctx->n_q || g.l0 < 2 * g.logB + 5) return fesc_fail(ctx, FESC_ELEVEL, "scan_contract: not enough levels");
+    g.l1 = g.l0 - 2;
+    g.lS = g.l1 - g.logB;
+    g.linj = g.l1 - 2 * g.logB + 1;
+    g.lout = g.linj - 3;
+    if (g.K_blk > 1 && g.lS < g.linj + (g.K_blk - 2))
+        return fesc_fail(ctx, FESC_ELEVEL, "scan_contract: carry chain runs below the injection level");
+    Exec X;
+    X.ctx = ctx, X.st = (cudaStream_t)stream, X.g = g, X.desc = desc, X.cs = consts;
+    X.N = ctx->N, X.rc = FESC_OK;
+    // planning pass for the arena size
+    X.dry = true, X.arena = reinterpret_cast<u64*>((uintptr_t)1 << 40), X.top = 0, X.high = 0, X.ks = X.rs = nullptr;
+    int rc = scan_run(X, (const u64*)d_x, (const u64*)d_a, (const u64*)d_B, (const u64*)d_C, (u64*)d_m_out);
+    if (rc != FESC_OK) return rc;
+    const size_t ks_words = ks_scratch_words(ctx, g.l0, ks_chunk(ctx, 2 * g.B));
+    const size_t rs_words = (size_t)2 * g.B * 2 * ctx->N;
+    u64* scratch;
+    rc = ctx_scratch(ctx, (X.high + ks_words + rs_words) * sizeof(u64), &scratch);
+    if (rc != FESC_OK) return rc;
+    X.dry = false, X.arena = scratch, X.top = 0;
+    X.ks = scratch + X.high;
+    X.rs = X.ks + ks_words;
+    return scan_run(X, (const u64*)d_x, (const u64*)d_a, (const u64*)d_B, (const u64*)d_C, (u64*)d_m_out);
+}

@@ -1,0 +1,64 @@
+"""GPU parity for the scan-contract: every output residue equals the oracle's, and the decrypted result
+equals the float64 recurrence, on the paper's toy shape and on 128-slot analogues of the deployed geometry
+(carries over three blocks with a partial last block; two-digit token offsets with an odd chunk count)."""
+import numpy as np
+import pytest
+
+import fesc_synth as S
+from oracle.ckks import CONJ
+from oracle.scan import (ScanConsts, ScanEvaluator, ScanShape, add_scan_keys, encrypt_inputs, float_recurrence,
+                         key_id_for, unpack_output)
+from tests.gpu_util import ctx_pair, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(name, **kw):
+    import torch
+    import paper_2608_17442_b200 as fesc
+
+    ctx, orc, p = ctx_pair(name)
+    sh = ScanShape(orc.n, **kw)
+    l0 = p["n_q"]
+    x, a, B, C = S.scan_inputs(p["seed"] + sh.L, sh.L, sh.H, sh.P, 1, sh.d_s)
+    c = ScanConsts(orc, sh, l0, p["log_scale"])
+    add_scan_keys(orc, sh)
+    for r in sh.rotation_amounts() + [CONJ]:
+        ctx.add_galois_key(r, key_id_for(sh, r))
+    ctX, ctA, ctB, ctC = encrypt_inputs(orc, sh, c, x, a, B, C)
+    want = ScanEvaluator(orc, sh, c).run(ctX, ctA, ctB, ctC)
+    adj_s = [c.adj_s.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
+    adj_p = [c.adj_p.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
+    out = torch.empty((sh.K_blk, sh.K_s, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
+    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000)
+    ctx.scan_contract(to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
+                      to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out)
+    ctx.sync()
+    got = to_host(out)
+    assert np.array_equal(got, want)
+    m = unpack_output(orc, sh, c, got)
+    return np.abs(m - float_recurrence(x, a, B, C)).max()
+
+
+def test_scan_paper_toy_shape():
+    assert _run("scan_toy", L=4, H=2, P=4, d_s=2, B_blk=4) < 2.0**-24
+
+
+def test_scan_analogue_with_carries_and_partial_block():
+    assert _run("scan_small", L=40, H=8, P=4, d_s=8, B_blk=16) < 2.0**-22
+
+
+def test_scan_two_digit_offsets_and_odd_chunk_count():
+    assert _run("scan_small", L=64, H=3, P=4, d_s=4, B_blk=32) < 2.0**-22
+
+
+def test_scan_missing_key_is_reported():
+    import torch
+    import paper_2608_17442_b200 as fesc
+
+    ctx, orc, p = ctx_pair("scan_toy")
+    z = torch.zeros((1, 2, 2, 10, orc.N), dtype=torch.int64, device="cuda")
+    desc = fesc.ScanDesc(4, 2, 4, 2, 4, 0, 10, 7000000)     # no keys under this base
+    with pytest.raises(fesc.FescError) as e:
+        ctx.scan_contract(z, z, z[0], z[0], desc, z, z, z, z, [0] * 121, [0] * 121, z)
+    assert e.value.code == fesc.ENOKEY
