@@ -62,3 +62,43 @@ def test_scan_missing_key_is_reported():
     with pytest.raises(fesc.FescError) as e:
         ctx.scan_contract(z, z, z[0], z[0], desc, z, z, z, z, [0] * 121, [0] * 121, z)
     assert e.value.code == fesc.ENOKEY
+
+
+def test_scan_deployed_geometry_decrypts_to_recurrence():
+    """N = 2^16, 24 limbs, stride 256, B_blk = 256, d_s = 128, P = 64 (the Mamba-2-base geometry) on a slice of
+    the model: 4 heads (one chunk pair) and 512 tokens (two blocks, so the carry and its injection run).
+    The oracle cannot follow ~36 000 key switches at this ring size, so the check here is the property that
+    holds at any size: the decrypted output equals the float64 recurrence."""
+    import time
+    import torch
+    import paper_2608_17442_b200 as fesc
+
+    ctx, orc, p = ctx_pair("full")
+    sh = ScanShape(orc.n, L=512, H=4, P=64, d_s=128, B_blk=256)
+    assert (sh.stride, sh.c_state, sh.hpc, sh.K_s, sh.K_blk) == (256, 128, 2, 2, 2)
+    l0 = 24
+    x, a, B, C = S.scan_inputs(S.config_seed(5), sh.L, sh.H, sh.P, 1, sh.d_s)
+    c = ScanConsts(orc, sh, l0, 40)
+    assert c.lv == dict(l0=24, l1=22, lS=14, linj=7, lout=4)
+    for r in sh.rotation_amounts() + [CONJ]:
+        ctx.add_galois_key(r, key_id_for(sh, r))
+    ctX, ctA, ctB, ctC = encrypt_inputs(orc, sh, c, x, a, B, C)
+    adj_s = [c.adj_s.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
+    adj_p = [c.adj_p.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
+    out = torch.empty((sh.K_blk, sh.K_s, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
+    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000)
+    args = (to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
+            to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out)
+    ks0 = ctx.counters()[1]
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    ctx.scan_contract(*args)
+    ctx.sync()
+    dt = time.perf_counter() - t0
+    ks = ctx.counters()[1] - ks0
+    m = unpack_output(orc, sh, c, to_host(out))
+    ref = float_recurrence(x, a, B, C)
+    err = np.abs(m - ref).max()
+    print("scan slice: %d key switches in %.2f s (%.0f /s), scratch %.1f GiB, max err 2^%.2f, max|m| %.2f"
+          % (ks, dt, ks / dt, ctx.counters()[3] / 2**30, np.log2(err), np.abs(ref).max()))
+    assert err < 2.0**-16
