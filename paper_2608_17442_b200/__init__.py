@@ -65,6 +65,7 @@ def lib():
             "fesc_ct_pt_mac": [vp, vp, vp, sz, vp, u32, u32, vp],
             "fesc_rotate": [vp, vp, vp, u32, u32, u32, vp],
             "fesc_rescale": [vp, vp, vp, u32, u32, vp],
+            "fesc_rescale_static": [vp, vp, vp, u32, u32, vp],
             "fesc_ct_ct_mul": [vp, vp, vp, vp, u32, u32, vp],
             "fesc_linear": [vp, vp, vp, c.POINTER(BsgsDesc), vp, vp],
             "fesc_scan_contract": [vp, vp, vp, vp, vp, c.POINTER(ScanDesc), c.POINTER(ScanConsts), vp, vp],
@@ -178,6 +179,14 @@ class Context:
 
     def rescale(self, ct_in, ct_out, batch: int, n_limbs: int):
         self._chk(lib().fesc_rescale(self.h, _ptr(ct_in), _ptr(ct_out), batch, n_limbs, _stream()))
+
+    def rescale_static(self, ct_in, ct_out, batch: int, n_limbs: int):
+        """fesc_rescale without any device allocation: scratch lives in a fixed 4 MiB array of the library
+        (batch * 2 * N <= 524 288 words).  For callers that cannot reach cudaMalloc (fixed memory budgets
+        owned by another allocator, latency-critical loops, hosts that forbid allocator calls).  The first
+        call on a device looks up the array's address; make it before any stream capture.  Calls share the
+        array: do not overlap them on the GPU."""
+        self._chk(lib().fesc_rescale_static(self.h, _ptr(ct_in), _ptr(ct_out), batch, n_limbs, _stream()))
 
     def ct_ct_mul(self, a, b, out, batch: int, n_limbs: int):
         self._chk(lib().fesc_ct_ct_mul(self.h, _ptr(a), _ptr(b), _ptr(out), batch, n_limbs, _stream()))
