@@ -27,74 +27,103 @@ __device__ __forceinline__ Tw ldtw(const ulonglong2* __restrict__ t, uint32_t i)
     return Tw{v.x, v.y};
 }
 
-// forward butterfly, inputs in [0,4q), outputs in [0,4q)
+// ---- classic lazy butterflies (any q < 2^62): forward values in [0,4q), inverse in [0,2q) ----
 __device__ __forceinline__ void ct_bfly(u64& x, u64& y, const Tw& t, u64 q, u64 q2) {
     u64 u = csub(x, q2);
     u64 v = shoup_lazy(y, t.w, t.s, q);
     x = u + v;
     y = u - v + q2;
 }
-// inverse butterfly, inputs in [0,2q), outputs in [0,2q)
 __device__ __forceinline__ void gs_bfly(u64& x, u64& y, const Tw& t, u64 q, u64 q2) {
     u64 u = x, v = y;
     x = csub(u + v, q2);
     y = shoup_lazy(u - v + q2, t.w, t.s, q);
 }
 
+// ---- wide lazy butterflies (q < 2^54): no conditional subtraction inside the transform ----
+// The high half of x*ws is taken from three of the four 32x32 partial products; it is at most 2
+// below the true value, so the lazy product lands in [0,4q) instead of [0,2q).
+__device__ __forceinline__ u64 mulhi_approx(u64 x, u64 y) {
+    const uint32_t x0 = (uint32_t)x, x1 = (uint32_t)(x >> 32), y0 = (uint32_t)y, y1 = (uint32_t)(y >> 32);
+    return (u64)x1 * y1 + __umulhi(x1, y0) + __umulhi(x0, y1);
+}
+__device__ __forceinline__ u64 shoup_lazy4(u64 x, u64 w, u64 ws, u64 q) { return x * w - mulhi_approx(x, ws) * q; }
+
+// Butterfly policy.  WIDE forward: inputs below a bound Bd give outputs below Bd + 4q (16 stages from
+// canonical input stay below 65q).  WIDE inverse: inputs below `off` give x below 2*off and y below 4q, so
+// the offset doubles per stage (8 stages from 4q stay below 2^10 q).
+template <bool WIDE>
+struct Bf {
+    static __device__ __forceinline__ void ct(u64& x, u64& y, const Tw& t, u64 q, u64 q2) {
+        if (WIDE) {
+            u64 u = x, v = shoup_lazy4(y, t.w, t.s, q);
+            x = u + v;
+            y = u - v + 2 * q2;
+        } else {
+            ct_bfly(x, y, t, q, q2);
+        }
+    }
+    static __device__ __forceinline__ void gs(u64& x, u64& y, const Tw& t, u64 q, u64 q2, u64 off) {
+        if (WIDE) {
+            u64 u = x, v = y;
+            x = u + v;
+            y = shoup_lazy4(u - v + off, t.w, t.s, q);
+        } else {
+            gs_bfly(x, y, t, q, q2);
+        }
+    }
+};
+
 // Three forward stages on 8 registers holding elements e0 + k*d (k = 0..7); the twiddle
 // indices are base indices for the first pair of each stage.
 //   stage A: pairs (k,k+4), one twiddle         idxA
 //   stage B: pairs (k,k+2), twiddles            idxB + (k>>2)
 //   stage C: pairs (k,k+1), twiddles            idxC + (k>>1)
+template <bool W>
+__device__ __forceinline__ void fwd_round2(u64 (&x)[8], const ulonglong2* __restrict__ tw, uint32_t idxB,
+                                           uint32_t idxC, u64 q, u64 q2) {
+    Tw b0 = ldtw(tw, idxB), b1 = ldtw(tw, idxB + 1);
+    Bf<W>::ct(x[0], x[2], b0, q, q2);
+    Bf<W>::ct(x[1], x[3], b0, q, q2);
+    Bf<W>::ct(x[4], x[6], b1, q, q2);
+    Bf<W>::ct(x[5], x[7], b1, q, q2);
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+        Tw c = ldtw(tw, idxC + k);
+        Bf<W>::ct(x[2 * k], x[2 * k + 1], c, q, q2);
+    }
+}
+template <bool W>
 __device__ __forceinline__ void fwd_round3(u64 (&x)[8], const ulonglong2* __restrict__ tw, uint32_t idxA,
                                            uint32_t idxB, uint32_t idxC, u64 q, u64 q2) {
     Tw a = ldtw(tw, idxA);
 #pragma unroll
-    for (int k = 0; k < 4; k++) ct_bfly(x[k], x[k + 4], a, q, q2);
-    Tw b0 = ldtw(tw, idxB), b1 = ldtw(tw, idxB + 1);
-    ct_bfly(x[0], x[2], b0, q, q2);
-    ct_bfly(x[1], x[3], b0, q, q2);
-    ct_bfly(x[4], x[6], b1, q, q2);
-    ct_bfly(x[5], x[7], b1, q, q2);
-#pragma unroll
-    for (int k = 0; k < 4; k++) {
-        Tw c = ldtw(tw, idxC + k);
-        ct_bfly(x[2 * k], x[2 * k + 1], c, q, q2);
-    }
+    for (int k = 0; k < 4; k++) Bf<W>::ct(x[k], x[k + 4], a, q, q2);
+    fwd_round2<W>(x, tw, idxB, idxC, q, q2);
 }
-// Two forward stages (pairs (k,k+2) then (k,k+1)) on two groups of 4.
-__device__ __forceinline__ void fwd_round2(u64 (&x)[8], const ulonglong2* __restrict__ tw, uint32_t idxB,
-                                           uint32_t idxC, u64 q, u64 q2) {
-    Tw b0 = ldtw(tw, idxB), b1 = ldtw(tw, idxB + 1);
-    ct_bfly(x[0], x[2], b0, q, q2);
-    ct_bfly(x[1], x[3], b0, q, q2);
-    ct_bfly(x[4], x[6], b1, q, q2);
-    ct_bfly(x[5], x[7], b1, q, q2);
-#pragma unroll
-    for (int k = 0; k < 4; k++) {
-        Tw c = ldtw(tw, idxC + k);
-        ct_bfly(x[2 * k], x[2 * k + 1], c, q, q2);
-    }
-}
+// Inverse rounds: stages in the opposite order (C, B, then A); `off` is the wide-mode offset of the
+// first stage of the round and doubles with every stage.
+template <bool W>
 __device__ __forceinline__ void inv_round2(u64 (&x)[8], const ulonglong2* __restrict__ tw, uint32_t idxB,
-                                           uint32_t idxC, u64 q, u64 q2) {
+                                           uint32_t idxC, u64 q, u64 q2, u64 off) {
 #pragma unroll
     for (int k = 0; k < 4; k++) {
         Tw c = ldtw(tw, idxC + k);
-        gs_bfly(x[2 * k], x[2 * k + 1], c, q, q2);
+        Bf<W>::gs(x[2 * k], x[2 * k + 1], c, q, q2, off);
     }
     Tw b0 = ldtw(tw, idxB), b1 = ldtw(tw, idxB + 1);
-    gs_bfly(x[0], x[2], b0, q, q2);
-    gs_bfly(x[1], x[3], b0, q, q2);
-    gs_bfly(x[4], x[6], b1, q, q2);
-    gs_bfly(x[5], x[7], b1, q, q2);
+    Bf<W>::gs(x[0], x[2], b0, q, q2, 2 * off);
+    Bf<W>::gs(x[1], x[3], b0, q, q2, 2 * off);
+    Bf<W>::gs(x[4], x[6], b1, q, q2, 2 * off);
+    Bf<W>::gs(x[5], x[7], b1, q, q2, 2 * off);
 }
+template <bool W>
 __device__ __forceinline__ void inv_round3(u64 (&x)[8], const ulonglong2* __restrict__ tw, uint32_t idxA,
-                                           uint32_t idxB, uint32_t idxC, u64 q, u64 q2) {
-    inv_round2(x, tw, idxB, idxC, q, q2);
+                                           uint32_t idxB, uint32_t idxC, u64 q, u64 q2, u64 off) {
+    inv_round2<W>(x, tw, idxB, idxC, q, q2, off);
     Tw a = ldtw(tw, idxA);
 #pragma unroll
-    for (int k = 0; k < 4; k++) gs_bfly(x[k], x[k + 4], a, q, q2);
+    for (int k = 0; k < 4; k++) Bf<W>::gs(x[k], x[k + 4], a, q, q2, 4 * off);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -102,6 +131,76 @@ __device__ __forceinline__ void inv_round3(u64 (&x)[8], const ulonglong2* __rest
 // grid = (16 column tiles, rows); block = 512 threads = 16 columns x 32 sub-threads.
 // ---------------------------------------------------------------------------------------
 #define N16 65536u
+#define WIDE_LIMIT (1ull << 54)
+
+template <bool INV, bool W>
+__device__ __forceinline__ void strided_body(u64* __restrict__ p, u64* __restrict__ sm, const ulonglong2* __restrict__ tw,
+                                             const PrimeConst& pc) {
+    const u64 q = pc.q, q2 = 2 * pc.q;
+    const uint32_t col = threadIdx.x & 15, sub = threadIdx.x >> 4;
+    const uint32_t h2 = sub >> 2, l2 = sub & 3;
+    u64 x[8];
+    if (!INV) {
+        // round 1: hi = k*32 + sub, local stages 0,1,2
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = p[(size_t)(k * 32 + sub) * 256 + col];
+        fwd_round3<W>(x, tw, 1, 2, 4, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[(k * 32 + sub) * 16 + col] = x[k];
+        __syncthreads();
+        // round 2: hi = h2*32 + k*4 + l2, local stages 3,4,5
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * 16 + col];
+        fwd_round3<W>(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * 16 + col] = x[k];
+        __syncthreads();
+        // round 3: hi = sub*8 + k, local stages 6,7
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[(sub * 8 + k) * 16 + col];
+        fwd_round2<W>(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) p[(size_t)(sub * 8 + k) * 256 + col] = x[k];  // lazily reduced
+    } else {
+        const u64 off = 2 * q2;   // inputs below 4q (wide) / 2q (classic) from the contiguous kernel
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = p[(size_t)(sub * 8 + k) * 256 + col];
+        inv_round2<W>(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, q2, off);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[(sub * 8 + k) * 16 + col] = x[k];
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * 16 + col];
+        inv_round3<W>(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, q2, 4 * off);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * 16 + col] = x[k];
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[(k * 32 + sub) * 16 + col];
+        // stages 2,1 then the last stage with N^-1 folded in (exact products, canonical output)
+        {
+#pragma unroll
+            for (int k = 0; k < 4; k++) {
+                Tw c = ldtw(tw, 4 + k);
+                Bf<W>::gs(x[2 * k], x[2 * k + 1], c, q, q2, 32 * off);
+            }
+            Tw b0 = ldtw(tw, 2), b1 = ldtw(tw, 3);
+            Bf<W>::gs(x[0], x[2], b0, q, q2, 64 * off);
+            Bf<W>::gs(x[1], x[3], b0, q, q2, 64 * off);
+            Bf<W>::gs(x[4], x[6], b1, q, q2, 64 * off);
+            Bf<W>::gs(x[5], x[7], b1, q, q2, 64 * off);
+            const u64 last = W ? 128 * off : q2;
+#pragma unroll
+            for (int k = 0; k < 4; k++) {
+                u64 u = x[k], v = x[k + 4];
+                x[k] = shoup(u + v, pc.ninv, pc.ninvs, q);
+                x[k + 4] = shoup(u - v + last, pc.ninvw, pc.ninvws, q);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 8; k++) p[(size_t)(k * 32 + sub) * 256 + col] = x[k];
+    }
+}
 
 template <bool INV>
 __global__ void __launch_bounds__(512) ntt16_strided(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
@@ -111,70 +210,12 @@ __global__ void __launch_bounds__(512) ntt16_strided(u64* __restrict__ data, con
     if (pi == 0xFF) return;
     __shared__ u64 sm[256 * 16];
     const PrimeConst pc = pcs[pi];
-    const u64 q = pc.q, q2 = 2 * pc.q;
     const ulonglong2* tw = tw_all + (size_t)pi * N16;
     u64* p = data + (size_t)row * N16 + blockIdx.x * 16;
-    const uint32_t col = threadIdx.x & 15, sub = threadIdx.x >> 4;
-    const uint32_t h2 = sub >> 2, l2 = sub & 3;
-    u64 x[8];
-    if (!INV) {
-        // round 1: hi = k*32 + sub, local stages 0,1,2
-#pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = p[(size_t)(k * 32 + sub) * 256 + col];
-        fwd_round3(x, tw, 1, 2, 4, q, q2);
-#pragma unroll
-        for (int k = 0; k < 8; k++) sm[(k * 32 + sub) * 16 + col] = x[k];
-        __syncthreads();
-        // round 2: hi = h2*32 + k*4 + l2, local stages 3,4,5
-#pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * 16 + col];
-        fwd_round3(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, q2);
-#pragma unroll
-        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * 16 + col] = x[k];
-        __syncthreads();
-        // round 3: hi = sub*8 + k, local stages 6,7
-#pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[(sub * 8 + k) * 16 + col];
-        fwd_round2(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, q2);
-#pragma unroll
-        for (int k = 0; k < 8; k++) p[(size_t)(sub * 8 + k) * 256 + col] = x[k];  // lazily reduced, < 4q
-    } else {
-#pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = p[(size_t)(sub * 8 + k) * 256 + col];  // < 2q from the contiguous kernel
-        inv_round2(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, q2);
-#pragma unroll
-        for (int k = 0; k < 8; k++) sm[(sub * 8 + k) * 16 + col] = x[k];
-        __syncthreads();
-#pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * 16 + col];
-        inv_round3(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, q2);
-#pragma unroll
-        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * 16 + col] = x[k];
-        __syncthreads();
-#pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[(k * 32 + sub) * 16 + col];
-        // stages 2,1 then the last stage with N^-1 folded in
-        {
-#pragma unroll
-            for (int k = 0; k < 4; k++) {
-                Tw c = ldtw(tw, 4 + k);
-                gs_bfly(x[2 * k], x[2 * k + 1], c, q, q2);
-            }
-            Tw b0 = ldtw(tw, 2), b1 = ldtw(tw, 3);
-            gs_bfly(x[0], x[2], b0, q, q2);
-            gs_bfly(x[1], x[3], b0, q, q2);
-            gs_bfly(x[4], x[6], b1, q, q2);
-            gs_bfly(x[5], x[7], b1, q, q2);
-#pragma unroll
-            for (int k = 0; k < 4; k++) {
-                u64 u = x[k], v = x[k + 4];
-                x[k] = shoup(u + v, pc.ninv, pc.ninvs, q);
-                x[k + 4] = shoup(u - v + q2, pc.ninvw, pc.ninvws, q);
-            }
-        }
-#pragma unroll
-        for (int k = 0; k < 8; k++) p[(size_t)(k * 32 + sub) * 256 + col] = x[k];
-    }
+    if (pc.q < WIDE_LIMIT)
+        strided_body<INV, true>(p, sm, tw, pc);
+    else
+        strided_body<INV, false>(p, sm, tw, pc);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -184,6 +225,69 @@ __global__ void __launch_bounds__(512) ntt16_strided(u64* __restrict__ data, con
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t pad8(uint32_t e) { return e + (e >> 3); }
 
+template <bool INV, bool W>
+__device__ __forceinline__ void contig_body(u64* __restrict__ p, u64* __restrict__ sm, const ulonglong2* __restrict__ tw,
+                                            const PrimeConst& pc, uint32_t pre) {
+    const u64 q = pc.q, q2 = 2 * pc.q;
+    const uint32_t sub = threadIdx.x & 31;
+    const uint32_t h2 = sub >> 2, l2 = sub & 3;
+    u64 x[8];
+    if (!INV) {
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = p[k * 32 + sub];   // lazily reduced by the strided kernel
+        fwd_round3<W>(x, tw, pre, 2 * pre, 4 * pre, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[pad8(k * 32 + sub)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[pad8(h2 * 32 + k * 4 + l2)];
+        fwd_round3<W>(x, tw, 8 * pre + h2, 16 * pre + 2 * h2, 32 * pre + 4 * h2, q, q2);
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[pad8(h2 * 32 + k * 4 + l2)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[pad8(sub * 8 + k)];
+        fwd_round2<W>(x, tw, 64 * pre + 2 * sub, 128 * pre + 4 * sub, q, q2);
+#pragma unroll
+        for (int k = 0; k < 8; k++) {
+            if (W) x[k] = x[k] - mulhi_approx(x[k], pc.mu) * q;   // below 65q -> below 4q
+            x[k] = csub(csub(x[k], q2), q);
+        }
+        ulonglong2* o = reinterpret_cast<ulonglong2*>(p + sub * 8);
+#pragma unroll
+        for (int k = 0; k < 4; k++) o[k] = make_ulonglong2(x[2 * k], x[2 * k + 1]);
+    } else {
+        const u64 off = 2 * q2;   // canonical input is below 4q
+        const ulonglong2* in = reinterpret_cast<const ulonglong2*>(p + sub * 8);
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+            ulonglong2 v = in[k];
+            x[2 * k] = v.x;
+            x[2 * k + 1] = v.y;
+        }
+        inv_round2<W>(x, tw, 64 * pre + 2 * sub, 128 * pre + 4 * sub, q, q2, off);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[pad8(sub * 8 + k)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[pad8(h2 * 32 + k * 4 + l2)];
+        inv_round3<W>(x, tw, 8 * pre + h2, 16 * pre + 2 * h2, 32 * pre + 4 * h2, q, q2, 4 * off);
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[pad8(h2 * 32 + k * 4 + l2)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[pad8(k * 32 + sub)];
+        inv_round3<W>(x, tw, pre, 2 * pre, 4 * pre, q, q2, 32 * off);
+#pragma unroll
+        for (int k = 0; k < 8; k++) {
+            if (W) x[k] = x[k] - mulhi_approx(x[k], pc.mu) * q;   // below 2^10 q -> below 4q
+            p[k * 32 + sub] = x[k];                               // finished by the strided kernel
+        }
+    }
+}
+
 template <bool INV>
 __global__ void __launch_bounds__(512) ntt16_contig(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
                                                     const PrimeConst* __restrict__ pcs, RowMap map) {
@@ -192,62 +296,15 @@ __global__ void __launch_bounds__(512) ntt16_contig(u64* __restrict__ data, cons
     if (pi == 0xFF) return;
     __shared__ u64 sm_all[16 * 288];
     const PrimeConst pc = pcs[pi];
-    const u64 q = pc.q, q2 = 2 * pc.q;
     const ulonglong2* tw = tw_all + (size_t)pi * N16;
-    const uint32_t warp = threadIdx.x >> 5, sub = threadIdx.x & 31;
+    const uint32_t warp = threadIdx.x >> 5;
     const uint32_t blk = blockIdx.x * 16 + warp;   // 256-point block index within the limb
-    const uint32_t pre = 256 + blk;
     u64* p = data + (size_t)row * N16 + (size_t)blk * 256;
     u64* sm = sm_all + warp * 288;
-    const uint32_t h2 = sub >> 2, l2 = sub & 3;
-    u64 x[8];
-    if (!INV) {
-#pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = p[k * 32 + sub];   // < 4q from the strided kernel
-        fwd_round3(x, tw, pre, 2 * pre, 4 * pre, q, q2);
-#pragma unroll
-        for (int k = 0; k < 8; k++) sm[pad8(k * 32 + sub)] = x[k];
-        __syncwarp();
-#pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[pad8(h2 * 32 + k * 4 + l2)];
-        fwd_round3(x, tw, 8 * pre + h2, 16 * pre + 2 * h2, 32 * pre + 4 * h2, q, q2);
-        __syncwarp();
-#pragma unroll
-        for (int k = 0; k < 8; k++) sm[pad8(h2 * 32 + k * 4 + l2)] = x[k];
-        __syncwarp();
-#pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[pad8(sub * 8 + k)];
-        fwd_round2(x, tw, 64 * pre + 2 * sub, 128 * pre + 4 * sub, q, q2);
-#pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = csub(csub(x[k], q2), q);
-        ulonglong2* o = reinterpret_cast<ulonglong2*>(p + sub * 8);
-#pragma unroll
-        for (int k = 0; k < 4; k++) o[k] = make_ulonglong2(x[2 * k], x[2 * k + 1]);
-    } else {
-        const ulonglong2* in = reinterpret_cast<const ulonglong2*>(p + sub * 8);
-#pragma unroll
-        for (int k = 0; k < 4; k++) {
-            ulonglong2 v = in[k];
-            x[2 * k] = v.x;
-            x[2 * k + 1] = v.y;
-        }
-        inv_round2(x, tw, 64 * pre + 2 * sub, 128 * pre + 4 * sub, q, q2);
-#pragma unroll
-        for (int k = 0; k < 8; k++) sm[pad8(sub * 8 + k)] = x[k];
-        __syncwarp();
-#pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[pad8(h2 * 32 + k * 4 + l2)];
-        inv_round3(x, tw, 8 * pre + h2, 16 * pre + 2 * h2, 32 * pre + 4 * h2, q, q2);
-        __syncwarp();
-#pragma unroll
-        for (int k = 0; k < 8; k++) sm[pad8(h2 * 32 + k * 4 + l2)] = x[k];
-        __syncwarp();
-#pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[pad8(k * 32 + sub)];
-        inv_round3(x, tw, pre, 2 * pre, 4 * pre, q, q2);
-#pragma unroll
-        for (int k = 0; k < 8; k++) p[k * 32 + sub] = x[k];   // < 2q, finished by the strided kernel
-    }
+    if (pc.q < WIDE_LIMIT)
+        contig_body<INV, true>(p, sm, tw, pc, 256 + blk);
+    else
+        contig_body<INV, false>(p, sm, tw, pc, 256 + blk);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -213,3 +213,35 @@ def test_workload_1_end_to_end():
             assert np.array_equal(got[i], want)
             slots = orc.decrypt(got[i], scale * scale)
             assert np.abs(slots - np.roll(z[i] * w[i], -r)).max() < 2.0**-16
+
+
+def test_workload_3_rotations_full_ring():
+    """Key-switch / rotation workload: N = 2^16, 24 x 50-bit limbs + 4 x 60-bit special primes, 6 digits;
+    32 ciphertexts of U[-1,1] slots at scale 2^40; 16 key slots (baby steps 1..8, giant steps 8*{1..8}).
+    Every rotation of the batch is decrypted and compared with the float64 shift (2^-18); four sampled
+    (ciphertext, key) pairs are compared with the oracle bit for bit."""
+    import torch
+
+    pair = ctx_pair("full")
+    ctx, orc, p = pair
+    amounts = list(range(1, 9)) + [8 * g for g in range(1, 9)]
+    scale = 2.0**40
+    z = S.uniform_slots(S.config_seed(3), 0, 32, orc.n)
+    cts = np.stack([orc.encrypt(orc.encode(z[i], scale, 24), 3000 + i) for i in range(32)])
+    d_in = to_dev(cts)
+    out = torch.empty_like(d_in)
+    sampled = {(0, 0), (7, 5), (19, 8), (31, 15)}
+    worst = 0.0
+    for k, r in enumerate(amounts):
+        key_id = 300 + k
+        ctx.add_galois_key(r, key_id)
+        ctx.rotate(d_in, out, 32, 24, key_id)
+        got = to_host(out)
+        for i in range(32):
+            worst = max(worst, np.abs(orc.decrypt(got[i], scale, 2).real - np.roll(z[i], -r)).max())
+            if (i, k) in sampled:
+                if key_id not in orc.keys:
+                    orc.add_galois_key(r, key_id)
+                assert np.array_equal(got[i], orc.rotate(cts[i], key_id)), (i, k)
+    print("workload 3: max |decrypt - shift| = 2^%.2f over 512 rotations" % np.log2(worst))
+    assert worst < 2.0**-18
