@@ -30,6 +30,10 @@ struct PrimeConst {
     u64 ninvs;     // Shoup companion of ninv
     u64 ninvw;     // N^-1 * psi^-brev(1) mod q  (last inverse stage, odd output)
     u64 ninvws;
+    double qd;     // q, 1/q, ninv, ninvw as doubles (exact for q < 2^50; used by the FP64 butterflies)
+    double qinvd;
+    double ninvd;
+    double ninvwd;
 };
 
 // ---------------------------------------------------------------------------------------
@@ -143,6 +147,8 @@ struct fesc_ctx {
     PrimeConst* d_pc;             // device [n_primes]
     ulonglong2* d_tw;             // forward twiddles [n_primes][N] (w, shoup)
     ulonglong2* d_itw;            // inverse twiddles [n_primes][N]
+    double* d_twf;                // the same twiddles as doubles, rows of primes >= 2^50 unused
+    double* d_itwf;
     u64* d_s;                     // secret key, EVAL, [n_primes][N]
     Tables tabs;
     std::map<uint32_t, EvalKey> keys;

@@ -309,6 +309,7 @@ extern "C" int fesc_ctx_create(fesc_ctx** out, uint32_t log_n, const uint64_t* p
     ctx->seed = seed;
     ctx->d_pc = nullptr;
     ctx->d_tw = ctx->d_itw = nullptr;
+    ctx->d_twf = ctx->d_itwf = nullptr;
     ctx->d_s = nullptr;
     ctx->d_scratch = nullptr;
     ctx->scratch_bytes = 0;
@@ -323,6 +324,7 @@ extern "C" int fesc_ctx_create(fesc_ctx** out, uint32_t log_n, const uint64_t* p
     if (ctx->alpha > FESC_MAX_ALPHA) return bail(FESC_EINVAL);
     // ---- validate primes, per-prime constants, twiddles ----
     std::vector<ulonglong2> tw((size_t)np * N), itw((size_t)np * N);
+    std::vector<double> twf((size_t)np * N, 0.0), itwf((size_t)np * N, 0.0);
     for (uint32_t i = 0; i < np; i++) {
         u64 q = primes[i];
         if (q >= (1ull << 62) || q < 3 || (q - 1) % (2ull * N) != 0 || !h_is_prime(q)) return bail(FESC_EINVAL);
@@ -350,14 +352,24 @@ extern "C" int fesc_ctx_create(fesc_ctx** out, uint32_t log_n, const uint64_t* p
             uint32_t r = h_brev(k, log_n);
             tw[(size_t)i * N + k] = make_ulonglong2(pw[r], h_shoup(pw[r], q));
             itw[(size_t)i * N + k] = make_ulonglong2(ipw[r], h_shoup(ipw[r], q));
+            if (q < (1ull << 50)) {
+                twf[(size_t)i * N + k] = (double)pw[r];
+                itwf[(size_t)i * N + k] = (double)ipw[r];
+            }
         }
         pc.ninvw = h_mul(pc.ninv, ipw[h_brev(1, log_n)], q);
         pc.ninvws = h_shoup(pc.ninvw, q);
+        pc.qd = (double)q;
+        pc.qinvd = 1.0 / (double)q;
+        pc.ninvd = (double)pc.ninv;
+        pc.ninvwd = (double)pc.ninvw;
         ctx->pc.push_back(pc);
     }
     if ((rc = upload(ctx, &ctx->d_pc, ctx->pc)) != FESC_OK) return bail(rc);
     if ((rc = upload(ctx, &ctx->d_tw, tw)) != FESC_OK) return bail(rc);
     if ((rc = upload(ctx, &ctx->d_itw, itw)) != FESC_OK) return bail(rc);
+    if ((rc = upload(ctx, &ctx->d_twf, twf)) != FESC_OK) return bail(rc);
+    if ((rc = upload(ctx, &ctx->d_itwf, itwf)) != FESC_OK) return bail(rc);
     if ((rc = build_tables(ctx)) != FESC_OK) return bail(rc);
     // ---- secret key and relinearisation key ----
     if (cudaMalloc(&ctx->d_s, (size_t)np * N * sizeof(u64)) != cudaSuccess) return bail(FESC_ENOMEM);
@@ -382,6 +394,8 @@ extern "C" int fesc_ctx_destroy(fesc_ctx* ctx) {
     cudaFree(ctx->d_pc);
     cudaFree(ctx->d_tw);
     cudaFree(ctx->d_itw);
+    cudaFree(ctx->d_twf);
+    cudaFree(ctx->d_itwf);
     cudaFree(ctx->d_s);
     cudaFree(ctx->d_scratch);
     free_tables(ctx);

@@ -202,8 +202,222 @@ __device__ __forceinline__ void strided_body(u64* __restrict__ p, u64* __restric
     }
 }
 
+__device__ __forceinline__ uint32_t pad8(uint32_t e) { return e + (e >> 3); }
+
+// ---------------------------------------------------------------------------------------
+// FP64 butterflies for primes below 2^50.
+// B200 issues 64 FP64 FMAs per clock per SM on a pipe of its own, while a 64-bit modular product on
+// the integer side costs about 40 cycles of the 32-bit multiplier pipe per warp.  For q < 2^50 every
+// residue and every lazily reduced value below 2^53 is an exact double, and
+//     h = fl(y*w),  l = fma(y, w, -h)           (h + l = y*w exactly)
+//     c = rint(h * (1/q)),  v = fma(-c, q, h) + l (= y*w - c*q exactly, an integer below 2^53)
+// is an exact signed lazy product: |v| <= (1/2 + 3|y| 2^-53) q.  Sums and differences of such values are
+// exact while they stay below 2^53, so a butterfly is 8 FP64 operations.  With |inputs| <= q/2 three
+// forward stages stay below 3.5q and three inverse stages below 4q (< 8q <= 2^53); x - rint(x/q) q brings a
+// value back to |x| <= q/2 between register rounds.  The result equals the integer transform bit for bit.
+// The two kernels of one transform hand the data over as doubles in the caller's buffer.
+// ---------------------------------------------------------------------------------------
+#define FP_LIMIT (1ull << 50)
+__device__ __forceinline__ double fp_modmul(double y, double w, double q, double qinv) {
+    const double h = __dmul_rn(y, w);
+    const double l = __fma_rn(y, w, -h);
+    const double c = rint(__dmul_rn(h, qinv));
+    return __dadd_rn(__fma_rn(-c, q, h), l);
+}
+__device__ __forceinline__ double fp_reduce(double x, double q, double qinv) {
+    return __fma_rn(-rint(__dmul_rn(x, qinv)), q, x);
+}
+// canonical residue -> double in [-q/2, q/2)
+__device__ __forceinline__ double fp_load(u64 a, double q) {
+    double d = __longlong_as_double((long long)(a | 0x4330000000000000ull)) - 4503599627370496.0;
+    return d + d >= q ? d - q : d;
+}
+// integer-valued double with |x| <= q -> canonical residue
+__device__ __forceinline__ u64 fp_store(double x, double q, double qinv) {
+    x = fp_reduce(x, q, qinv);
+    x = x < 0.0 ? x + q : x;
+    return (u64)__double_as_longlong(x + 4503599627370496.0) & 0x000FFFFFFFFFFFFFull;
+}
+__device__ __forceinline__ double ldf(const double* __restrict__ t, uint32_t i) { return __ldg(t + i); }
+__device__ __forceinline__ void fp_ct(double& x, double& y, double w, double q, double qinv) {
+    const double v = fp_modmul(y, w, q, qinv), u = x;
+    x = u + v;
+    y = u - v;
+}
+__device__ __forceinline__ void fp_gs(double& x, double& y, double w, double q, double qinv) {
+    const double u = x, v = y;
+    x = u + v;
+    y = fp_modmul(u - v, w, q, qinv);
+}
+__device__ __forceinline__ void fp_fwd_round2(double (&x)[8], const double* __restrict__ tw, uint32_t idxB, uint32_t idxC,
+                                              double q, double qinv) {
+    const double b0 = ldf(tw, idxB), b1 = ldf(tw, idxB + 1);
+    fp_ct(x[0], x[2], b0, q, qinv);
+    fp_ct(x[1], x[3], b0, q, qinv);
+    fp_ct(x[4], x[6], b1, q, qinv);
+    fp_ct(x[5], x[7], b1, q, qinv);
+#pragma unroll
+    for (int k = 0; k < 4; k++) fp_ct(x[2 * k], x[2 * k + 1], ldf(tw, idxC + k), q, qinv);
+}
+__device__ __forceinline__ void fp_fwd_round3(double (&x)[8], const double* __restrict__ tw, uint32_t idxA, uint32_t idxB,
+                                              uint32_t idxC, double q, double qinv) {
+    const double a = ldf(tw, idxA);
+#pragma unroll
+    for (int k = 0; k < 4; k++) fp_ct(x[k], x[k + 4], a, q, qinv);
+    fp_fwd_round2(x, tw, idxB, idxC, q, qinv);
+}
+__device__ __forceinline__ void fp_inv_round2(double (&x)[8], const double* __restrict__ tw, uint32_t idxB, uint32_t idxC,
+                                              double q, double qinv) {
+#pragma unroll
+    for (int k = 0; k < 4; k++) fp_gs(x[2 * k], x[2 * k + 1], ldf(tw, idxC + k), q, qinv);
+    const double b0 = ldf(tw, idxB), b1 = ldf(tw, idxB + 1);
+    fp_gs(x[0], x[2], b0, q, qinv);
+    fp_gs(x[1], x[3], b0, q, qinv);
+    fp_gs(x[4], x[6], b1, q, qinv);
+    fp_gs(x[5], x[7], b1, q, qinv);
+}
+__device__ __forceinline__ void fp_inv_round3(double (&x)[8], const double* __restrict__ tw, uint32_t idxA, uint32_t idxB,
+                                              uint32_t idxC, double q, double qinv) {
+    fp_inv_round2(x, tw, idxB, idxC, q, qinv);
+    const double a = ldf(tw, idxA);
+#pragma unroll
+    for (int k = 0; k < 4; k++) fp_gs(x[k], x[k + 4], a, q, qinv);
+}
+__device__ __forceinline__ void fp_reduce8(double (&x)[8], double q, double qinv) {
+#pragma unroll
+    for (int k = 0; k < 8; k++) x[k] = fp_reduce(x[k], q, qinv);
+}
+
+template <bool INV>
+__device__ __forceinline__ void strided_body_fp(u64* __restrict__ p, double* __restrict__ sm, const double* __restrict__ tw,
+                                                const PrimeConst& pc) {
+    const double q = pc.qd, qinv = pc.qinvd;
+    const uint32_t col = threadIdx.x & 15, sub = threadIdx.x >> 4;
+    const uint32_t h2 = sub >> 2, l2 = sub & 3;
+    double x[8];
+    if (!INV) {
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = fp_load(p[(size_t)(k * 32 + sub) * 256 + col], q);
+        fp_fwd_round3(x, tw, 1, 2, 4, q, qinv);
+        fp_reduce8(x, q, qinv);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[(k * 32 + sub) * 16 + col] = x[k];
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * 16 + col];
+        fp_fwd_round3(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, qinv);
+        fp_reduce8(x, q, qinv);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * 16 + col] = x[k];
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[(sub * 8 + k) * 16 + col];
+        fp_fwd_round2(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, qinv);
+        fp_reduce8(x, q, qinv);
+        // handed to the contiguous kernel as doubles, |x| <= q/2
+#pragma unroll
+        for (int k = 0; k < 8; k++) p[(size_t)(sub * 8 + k) * 256 + col] = (u64)__double_as_longlong(x[k]);
+    } else {
+        // doubles with |x| <= q/2 from the contiguous kernel
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = __longlong_as_double((long long)p[(size_t)(sub * 8 + k) * 256 + col]);
+        fp_inv_round2(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, qinv);
+        fp_reduce8(x, q, qinv);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[(sub * 8 + k) * 16 + col] = x[k];
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * 16 + col];
+        fp_inv_round3(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, qinv);
+        fp_reduce8(x, q, qinv);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * 16 + col] = x[k];
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[(k * 32 + sub) * 16 + col];
+        // stages 2, 1, then the last stage with N^-1 folded in
+#pragma unroll
+        for (int k = 0; k < 4; k++) fp_gs(x[2 * k], x[2 * k + 1], ldf(tw, 4 + k), q, qinv);
+        {
+            const double b0 = ldf(tw, 2), b1 = ldf(tw, 3);
+            fp_gs(x[0], x[2], b0, q, qinv);
+            fp_gs(x[1], x[3], b0, q, qinv);
+            fp_gs(x[4], x[6], b1, q, qinv);
+            fp_gs(x[5], x[7], b1, q, qinv);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+            const double u = x[k], v = x[k + 4];
+            x[k] = fp_modmul(u + v, pc.ninvd, q, qinv);
+            x[k + 4] = fp_modmul(u - v, pc.ninvwd, q, qinv);
+        }
+#pragma unroll
+        for (int k = 0; k < 8; k++) p[(size_t)(k * 32 + sub) * 256 + col] = fp_store(x[k], q, qinv);
+    }
+}
+
+template <bool INV>
+__device__ __forceinline__ void contig_body_fp(u64* __restrict__ p, double* __restrict__ sm, const double* __restrict__ tw,
+                                               const PrimeConst& pc, uint32_t pre) {
+    const double q = pc.qd, qinv = pc.qinvd;
+    const uint32_t sub = threadIdx.x & 31;
+    const uint32_t h2 = sub >> 2, l2 = sub & 3;
+    double x[8];
+    if (!INV) {
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = __longlong_as_double((long long)p[k * 32 + sub]);   // |x| <= q/2
+        fp_fwd_round3(x, tw, pre, 2 * pre, 4 * pre, q, qinv);
+        fp_reduce8(x, q, qinv);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[pad8(k * 32 + sub)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[pad8(h2 * 32 + k * 4 + l2)];
+        fp_fwd_round3(x, tw, 8 * pre + h2, 16 * pre + 2 * h2, 32 * pre + 4 * h2, q, qinv);
+        fp_reduce8(x, q, qinv);
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[pad8(h2 * 32 + k * 4 + l2)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[pad8(sub * 8 + k)];
+        fp_fwd_round2(x, tw, 64 * pre + 2 * sub, 128 * pre + 4 * sub, q, qinv);
+        ulonglong2* o = reinterpret_cast<ulonglong2*>(p + sub * 8);
+#pragma unroll
+        for (int k = 0; k < 4; k++) o[k] = make_ulonglong2(fp_store(x[2 * k], q, qinv), fp_store(x[2 * k + 1], q, qinv));
+    } else {
+        const ulonglong2* in = reinterpret_cast<const ulonglong2*>(p + sub * 8);
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+            ulonglong2 v = in[k];
+            x[2 * k] = fp_load(v.x, q);
+            x[2 * k + 1] = fp_load(v.y, q);
+        }
+        fp_inv_round2(x, tw, 64 * pre + 2 * sub, 128 * pre + 4 * sub, q, qinv);
+        fp_reduce8(x, q, qinv);
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[pad8(sub * 8 + k)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[pad8(h2 * 32 + k * 4 + l2)];
+        fp_inv_round3(x, tw, 8 * pre + h2, 16 * pre + 2 * h2, 32 * pre + 4 * h2, q, qinv);
+        fp_reduce8(x, q, qinv);
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) sm[pad8(h2 * 32 + k * 4 + l2)] = x[k];
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; k++) x[k] = sm[pad8(k * 32 + sub)];
+        fp_inv_round3(x, tw, pre, 2 * pre, 4 * pre, q, qinv);
+        fp_reduce8(x, q, qinv);
+#pragma unroll
+        for (int k = 0; k < 8; k++) p[k * 32 + sub] = (u64)__double_as_longlong(x[k]);   // doubles, |x| <= q/2
+    }
+}
+
 template <bool INV>
 __global__ void __launch_bounds__(512) ntt16_strided(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
+                                                     const double* __restrict__ twf_all,
                                                      const PrimeConst* __restrict__ pcs, RowMap map) {
     const uint32_t row = blockIdx.y;
     const uint32_t pi = map.prime[row % map.period];
@@ -212,7 +426,9 @@ __global__ void __launch_bounds__(512) ntt16_strided(u64* __restrict__ data, con
     const PrimeConst pc = pcs[pi];
     const ulonglong2* tw = tw_all + (size_t)pi * N16;
     u64* p = data + (size_t)row * N16 + blockIdx.x * 16;
-    if (pc.q < WIDE_LIMIT)
+    if (pc.q < FP_LIMIT)
+        strided_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc);
+    else if (pc.q < WIDE_LIMIT)
         strided_body<INV, true>(p, sm, tw, pc);
     else
         strided_body<INV, false>(p, sm, tw, pc);
@@ -223,7 +439,6 @@ __global__ void __launch_bounds__(512) ntt16_strided(u64* __restrict__ data, con
 // grid = (16 tiles of 4096 points, rows); block = 512 threads = 16 warps, one 256-point block each.
 // Shared exchange buffer per warp: 256 points padded to e + (e >> 3) to avoid bank conflicts.
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t pad8(uint32_t e) { return e + (e >> 3); }
 
 template <bool INV, bool W>
 __device__ __forceinline__ void contig_body(u64* __restrict__ p, u64* __restrict__ sm, const ulonglong2* __restrict__ tw,
@@ -290,6 +505,7 @@ __device__ __forceinline__ void contig_body(u64* __restrict__ p, u64* __restrict
 
 template <bool INV>
 __global__ void __launch_bounds__(512) ntt16_contig(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
+                                                    const double* __restrict__ twf_all,
                                                     const PrimeConst* __restrict__ pcs, RowMap map) {
     const uint32_t row = blockIdx.y;
     const uint32_t pi = map.prime[row % map.period];
@@ -301,7 +517,9 @@ __global__ void __launch_bounds__(512) ntt16_contig(u64* __restrict__ data, cons
     const uint32_t blk = blockIdx.x * 16 + warp;   // 256-point block index within the limb
     u64* p = data + (size_t)row * N16 + (size_t)blk * 256;
     u64* sm = sm_all + warp * 288;
-    if (pc.q < WIDE_LIMIT)
+    if (pc.q < FP_LIMIT)
+        contig_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, 256 + blk);
+    else if (pc.q < WIDE_LIMIT)
         contig_body<INV, true>(p, sm, tw, pc, 256 + blk);
     else
         contig_body<INV, false>(p, sm, tw, pc, 256 + blk);
@@ -366,6 +584,7 @@ int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool 
     if (rows == 0) return FESC_OK;
     if (rows > 0x7fffffffu) return fesc_fail(ctx, FESC_EINVAL, "ntt: too many rows");
     const ulonglong2* tw = inverse ? ctx->d_itw : ctx->d_tw;
+    const double* twf = inverse ? ctx->d_itwf : ctx->d_twf;
     size_t live = 0;
     for (uint32_t i = 0; i < map.period; i++) live += map.prime[i] != 0xFF;
     ctx->counters[0] += rows / map.period * live;
@@ -381,11 +600,11 @@ int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool 
             dim3 grid(16, (unsigned)chunk);
             u64* base = d_data + r0 * (size_t)N16;
             if (!inverse) {
-                ntt16_strided<false><<<grid, 512, 0, st>>>(base, tw, ctx->d_pc, map);
-                ntt16_contig<false><<<grid, 512, 0, st>>>(base, tw, ctx->d_pc, map);
+                ntt16_strided<false><<<grid, 512, 0, st>>>(base, tw, twf, ctx->d_pc, map);
+                ntt16_contig<false><<<grid, 512, 0, st>>>(base, tw, twf, ctx->d_pc, map);
             } else {
-                ntt16_contig<true><<<grid, 512, 0, st>>>(base, tw, ctx->d_pc, map);
-                ntt16_strided<true><<<grid, 512, 0, st>>>(base, tw, ctx->d_pc, map);
+                ntt16_contig<true><<<grid, 512, 0, st>>>(base, tw, twf, ctx->d_pc, map);
+                ntt16_strided<true><<<grid, 512, 0, st>>>(base, tw, twf, ctx->d_pc, map);
             }
             r0 += chunk;
             launches += 2;
