@@ -72,6 +72,42 @@ __device__ __forceinline__ u64 mulmod(u64 x, u64 y, const PrimeConst& pc) {
     return reduce128(mulhi(x, y), x * y, pc);
 }
 
+// ---------------------------------------------------------------------------------------
+// Exact modular arithmetic on the FP64 pipe for moduli below 2^50.
+// B200 issues 64 FP64 FMAs per clock per SM on a pipe of its own, while a 64x64 product costs about 26
+// cycles of the 32-bit multiplier pipe per warp.  For q < 2^50 every residue is an exact double and
+//     h = fl(y*w),  l = fma(y, w, -h)              (h + l = y*w exactly)
+//     c = rint(h * (1/q)),  v = fma(-c, q, h) + l    (= y*w - c*q exactly, an integer below 2^53)
+// is an exact signed lazy product with |v| <= (1/2 + 3 |y| 2^-53) q for |y| < 2^53, 0 <= w < q.
+// Sums of such values are exact while they stay below 2^53 (8q); x - rint(x/q) q brings them back to
+// |x| <= q/2.  Results equal the integer arithmetic bit for bit.
+// ---------------------------------------------------------------------------------------
+#define FESC_FP_LIMIT (1ull << 50)
+__device__ __forceinline__ double fp_modmul(double y, double w, double q, double qinv) {
+    const double h = __dmul_rn(y, w);
+    const double l = __fma_rn(y, w, -h);
+    const double c = rint(__dmul_rn(h, qinv));
+    return __dadd_rn(__fma_rn(-c, q, h), l);
+}
+__device__ __forceinline__ double fp_reduce(double x, double q, double qinv) {
+    return __fma_rn(-rint(__dmul_rn(x, qinv)), q, x);
+}
+// integer below 2^52 -> double (exact)
+__device__ __forceinline__ double fp_from_u64(u64 a) {
+    return __longlong_as_double((long long)(a | 0x4330000000000000ull)) - 4503599627370496.0;
+}
+// canonical residue -> double in [-q/2, q/2)
+__device__ __forceinline__ double fp_load(u64 a, double q) {
+    const double d = fp_from_u64(a);
+    return d + d >= q ? d - q : d;
+}
+// integer-valued double below 2^53 -> canonical residue
+__device__ __forceinline__ u64 fp_store(double x, double q, double qinv) {
+    x = fp_reduce(x, q, qinv);
+    x = x < 0.0 ? x + q : x;
+    return (u64)__double_as_longlong(x + 4503599627370496.0) & 0x000FFFFFFFFFFFFFull;
+}
+
 // counter-based generator (same public recipe as the header documents)
 __host__ __device__ __forceinline__ u64 mix64(u64 z) {
     z += 0x9E3779B97F4A7C15ull;

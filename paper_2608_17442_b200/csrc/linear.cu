@@ -103,6 +103,195 @@ __global__ void __launch_bounds__(256, (TT * PT >= 16 ? 1 : (TT * PT >= 4 ? 2 : 
         }
 }
 
+// The same accumulation on the FP64 pipe, for limbs whose primes are all below 2^50: every term is an
+// exact signed lazy product (fp_modmul), partial sums stay below 2^53 because they are folded back to
+// |acc| <= q/2 every 8 terms.  Accumulators are single doubles, so the 2 x 8 tile needs half the
+// registers of the 128-bit version and two CTAs fit per SM.
+template <int TT, int PT>
+__global__ void __launch_bounds__(256, 2) k_bsgs_accumulate_fp(
+    const u64* __restrict__ rot, const u64* __restrict__ diags, u64* __restrict__ acc,
+    const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level, uint32_t tbs, uint32_t terms, uint32_t bp_count) {
+    const uint32_t c = blockIdx.y * blockDim.x + threadIdx.x;
+    const uint32_t l = blockIdx.z % level;
+    const uint32_t tb0 = (blockIdx.z / level) * TT, bp0 = blockIdx.x * PT;
+    if (c >= N) return;
+    const double q = pcs[l].qd, qinv = pcs[l].qinvd;
+    const size_t poly = (size_t)level * N, ctw = 2 * poly;
+    const size_t o = (size_t)l * N + c;
+    const u64* xp[TT];
+    const u64* dp[PT];
+#pragma unroll
+    for (int i = 0; i < TT; i++) {
+        uint32_t tb = tb0 + i < tbs ? tb0 + i : tbs - 1;
+        xp[i] = rot + (size_t)tb * terms * ctw + o;
+    }
+#pragma unroll
+    for (int j = 0; j < PT; j++) {
+        uint32_t bp = bp0 + j < bp_count ? bp0 + j : bp_count - 1;
+        dp[j] = diags + (size_t)bp * terms * poly + o;
+    }
+    double a[TT][PT][2];
+#pragma unroll
+    for (int i = 0; i < TT; i++)
+#pragma unroll
+        for (int j = 0; j < PT; j++) a[i][j][0] = a[i][j][1] = 0.0;
+    u64 nx0[TT], nx1[TT], nw[PT];
+#pragma unroll
+    for (int i = 0; i < TT; i++) {
+        nx0[i] = xp[i][0];
+        nx1[i] = xp[i][poly];
+    }
+#pragma unroll
+    for (int j = 0; j < PT; j++) nw[j] = __ldg(dp[j]);
+#pragma unroll 1
+    for (uint32_t t = 0; t < terms; t++) {
+        double x0[TT], x1[TT], w[PT];
+#pragma unroll
+        for (int i = 0; i < TT; i++) {
+            x0[i] = fp_load(nx0[i], q);
+            x1[i] = fp_load(nx1[i], q);
+        }
+#pragma unroll
+        for (int j = 0; j < PT; j++) w[j] = fp_from_u64(nw[j]);
+        const uint32_t tn = t + 1 < terms ? t + 1 : t;
+#pragma unroll
+        for (int i = 0; i < TT; i++) {
+            nx0[i] = xp[i][(size_t)tn * ctw];
+            nx1[i] = xp[i][(size_t)tn * ctw + poly];
+        }
+#pragma unroll
+        for (int j = 0; j < PT; j++) nw[j] = __ldg(dp[j] + (size_t)tn * poly);
+#pragma unroll
+        for (int j = 0; j < PT; j++)
+#pragma unroll
+            for (int i = 0; i < TT; i++) {
+                a[i][j][0] += fp_modmul(x0[i], w[j], q, qinv);
+                a[i][j][1] += fp_modmul(x1[i], w[j], q, qinv);
+            }
+        if ((t & 7) == 7) {
+#pragma unroll
+            for (int i = 0; i < TT; i++)
+#pragma unroll
+                for (int j = 0; j < PT; j++) {
+                    a[i][j][0] = fp_reduce(a[i][j][0], q, qinv);
+                    a[i][j][1] = fp_reduce(a[i][j][1], q, qinv);
+                }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < TT; i++)
+#pragma unroll
+        for (int j = 0; j < PT; j++) {
+            const uint32_t tb = tb0 + i, bp = bp0 + j;
+            if (tb < tbs && bp < bp_count) {
+                u64* dst = acc + ((size_t)tb * bp_count + bp) * ctw;
+                dst[o] = fp_store(a[i][j][0], q, qinv);
+                dst[poly + o] = fp_store(a[i][j][1], q, qinv);
+            }
+        }
+}
+
+// FP64 accumulate with asynchronous staging: every thread copies its own operand words of the next
+// STAGES-1 terms into shared memory with cp.async (8 bytes each, no barrier: a thread only reads back what
+// it copied), so several terms of operands are in flight per thread without holding them in registers.
+__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N_>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N_) : "memory");
+}
+
+template <int TT, int PT, int STAGES>
+__global__ void __launch_bounds__(256, 2) k_bsgs_accumulate_fp_staged(
+    const u64* __restrict__ rot, const u64* __restrict__ diags, u64* __restrict__ acc,
+    const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level, uint32_t tbs, uint32_t terms, uint32_t bp_count) {
+    constexpr int ROWS = 2 * TT + PT;
+    extern __shared__ __align__(16) u64 stage[];          // [STAGES][ROWS][256]
+    const uint32_t tid = threadIdx.x;
+    const uint32_t c = blockIdx.y * 256 + tid;            // N is a multiple of 256
+    const uint32_t l = blockIdx.z % level;
+    const uint32_t tb0 = (blockIdx.z / level) * TT, bp0 = blockIdx.x * PT;
+    const double q = pcs[l].qd, qinv = pcs[l].qinvd;
+    const size_t poly = (size_t)level * N, ctw = 2 * poly;
+    const size_t o = (size_t)l * N + c;
+    const u64* xp[TT];
+    const u64* dp[PT];
+#pragma unroll
+    for (int i = 0; i < TT; i++) {
+        uint32_t tb = tb0 + i < tbs ? tb0 + i : tbs - 1;
+        xp[i] = rot + (size_t)tb * terms * ctw + o;
+    }
+#pragma unroll
+    for (int j = 0; j < PT; j++) {
+        uint32_t bp = bp0 + j < bp_count ? bp0 + j : bp_count - 1;
+        dp[j] = diags + (size_t)bp * terms * poly + o;
+    }
+    auto issue = [&](uint32_t t) {
+        u64* dst = stage + (size_t)(t % STAGES) * ROWS * 256 + tid;
+#pragma unroll
+        for (int i = 0; i < TT; i++) {
+            cp_async8(dst + (2 * i) * 256, xp[i] + (size_t)t * ctw);
+            cp_async8(dst + (2 * i + 1) * 256, xp[i] + (size_t)t * ctw + poly);
+        }
+#pragma unroll
+        for (int j = 0; j < PT; j++) cp_async8(dst + (2 * TT + j) * 256, dp[j] + (size_t)t * poly);
+    };
+    for (uint32_t t = 0; t < STAGES - 1; t++) {
+        if (t < terms) issue(t);
+        cp_async_commit();
+    }
+    double a[TT][PT][2];
+#pragma unroll
+    for (int i = 0; i < TT; i++)
+#pragma unroll
+        for (int j = 0; j < PT; j++) a[i][j][0] = a[i][j][1] = 0.0;
+#pragma unroll 1
+    for (uint32_t t = 0; t < terms; t++) {
+        if (t + STAGES - 1 < terms) issue(t + STAGES - 1);
+        cp_async_commit();
+        cp_async_wait<STAGES - 1>();                       // the group of term t has landed
+        const u64* sm = stage + (size_t)(t % STAGES) * ROWS * 256 + tid;
+        double x0[TT], x1[TT];
+#pragma unroll
+        for (int i = 0; i < TT; i++) {
+            x0[i] = fp_load(sm[(2 * i) * 256], q);
+            x1[i] = fp_load(sm[(2 * i + 1) * 256], q);
+        }
+#pragma unroll
+        for (int j = 0; j < PT; j++) {
+            const double w = fp_from_u64(sm[(2 * TT + j) * 256]);
+#pragma unroll
+            for (int i = 0; i < TT; i++) {
+                a[i][j][0] += fp_modmul(x0[i], w, q, qinv);
+                a[i][j][1] += fp_modmul(x1[i], w, q, qinv);
+            }
+        }
+        if ((t & 7) == 7) {
+#pragma unroll
+            for (int i = 0; i < TT; i++)
+#pragma unroll
+                for (int j = 0; j < PT; j++) {
+                    a[i][j][0] = fp_reduce(a[i][j][0], q, qinv);
+                    a[i][j][1] = fp_reduce(a[i][j][1], q, qinv);
+                }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < TT; i++)
+#pragma unroll
+        for (int j = 0; j < PT; j++) {
+            const uint32_t tb = tb0 + i, bp = bp0 + j;
+            if (tb < tbs && bp < bp_count) {
+                u64* dst = acc + ((size_t)tb * bp_count + bp) * ctw;
+                dst[o] = fp_store(a[i][j][0], q, qinv);
+                dst[poly + o] = fp_store(a[i][j][1], q, qinv);
+            }
+        }
+}
+
 // Tuning knob for experiments: FESC_BSGS_TILE=<TT><PT> (e.g. 24) picks the register tile.
 static int bsgs_tile() {
     static int v = -1;
@@ -177,7 +366,42 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
         k_bsgs_accumulate<TT, PT><<<grid, 256, 0, st>>>(rot, diags, acc, ctx->d_pc, N, level, nt, gin * n1,  \
                                                         bp_count, reduce_every);                              \
     } while (0)
-        switch (bsgs_tile()) {
+#define BSGS_FP(TT, PT)                                                                                       \
+    do {                                                                                                      \
+        dim3 grid((bp_count + PT - 1) / PT, (N + 255) / 256, level * ((nt + TT - 1) / TT));                   \
+        if (grid.z > 65535) return fesc_fail(ctx, FESC_EINVAL, "linear: too many accumulator tiles");         \
+        k_bsgs_accumulate_fp<TT, PT><<<grid, 256, 0, st>>>(rot, diags, acc, ctx->d_pc, N, level, nt, gin * n1, \
+                                                           bp_count);                                         \
+    } while (0)
+#define BSGS_FPS(TT, PT, ST)                                                                                  \
+    do {                                                                                                      \
+        dim3 grid((bp_count + PT - 1) / PT, N / 256, level * ((nt + TT - 1) / TT));                           \
+        if (grid.z > 65535) return fesc_fail(ctx, FESC_EINVAL, "linear: too many accumulator tiles");         \
+        const size_t smem = (size_t)ST * (2 * TT + PT) * 2048;                                                \
+        auto kern = k_bsgs_accumulate_fp_staged<TT, PT, ST>;                                                  \
+        FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        kern<<<grid, 256, smem, st>>>(rot, diags, acc, ctx->d_pc, N, level, nt, gin * n1, bp_count);          \
+    } while (0)
+        const bool fp_ok = qbits <= 50;   // every active prime below 2^50: exact FP64 products
+        const int tile = bsgs_tile();
+        if (fp_ok && tile == 0) {
+            if (N % 256 == 0 && nt >= 2) BSGS_FPS(2, 8, 3);
+            else if (nt >= 2) BSGS_FP(2, 8);
+            else BSGS_FP(1, 8);
+        } else if (fp_ok && tile == 2028 && N % 256 == 0) {
+            BSGS_FPS(2, 8, 3);
+        } else if (fp_ok && tile == 2128 && N % 256 == 0) {
+            BSGS_FPS(2, 8, 4);
+        } else if (fp_ok && tile == 2044 && N % 256 == 0) {
+            BSGS_FPS(4, 4, 4);
+        } else if (fp_ok && tile == 1024) {
+            BSGS_FP(2, 4);
+        } else if (fp_ok && tile == 1044) {
+            BSGS_FP(4, 4);
+        } else if (fp_ok && tile == 1018) {
+            BSGS_FP(1, 8);
+        } else
+        switch (tile) {
             case 12: BSGS(1, 2); break;
             case 14: BSGS(1, 4); break;
             case 18: BSGS(1, 8); break;

@@ -217,27 +217,7 @@ __device__ __forceinline__ uint32_t pad8(uint32_t e) { return e + (e >> 3); }
 // value back to |x| <= q/2 between register rounds.  The result equals the integer transform bit for bit.
 // The two kernels of one transform hand the data over as doubles in the caller's buffer.
 // ---------------------------------------------------------------------------------------
-#define FP_LIMIT (1ull << 50)
-__device__ __forceinline__ double fp_modmul(double y, double w, double q, double qinv) {
-    const double h = __dmul_rn(y, w);
-    const double l = __fma_rn(y, w, -h);
-    const double c = rint(__dmul_rn(h, qinv));
-    return __dadd_rn(__fma_rn(-c, q, h), l);
-}
-__device__ __forceinline__ double fp_reduce(double x, double q, double qinv) {
-    return __fma_rn(-rint(__dmul_rn(x, qinv)), q, x);
-}
-// canonical residue -> double in [-q/2, q/2)
-__device__ __forceinline__ double fp_load(u64 a, double q) {
-    double d = __longlong_as_double((long long)(a | 0x4330000000000000ull)) - 4503599627370496.0;
-    return d + d >= q ? d - q : d;
-}
-// integer-valued double with |x| <= q -> canonical residue
-__device__ __forceinline__ u64 fp_store(double x, double q, double qinv) {
-    x = fp_reduce(x, q, qinv);
-    x = x < 0.0 ? x + q : x;
-    return (u64)__double_as_longlong(x + 4503599627370496.0) & 0x000FFFFFFFFFFFFFull;
-}
+#define FP_LIMIT FESC_FP_LIMIT
 __device__ __forceinline__ double ldf(const double* __restrict__ t, uint32_t i) { return __ldg(t + i); }
 __device__ __forceinline__ void fp_ct(double& x, double& y, double w, double q, double qinv) {
     const double v = fp_modmul(y, w, q, qinv), u = x;

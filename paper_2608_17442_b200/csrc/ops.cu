@@ -123,14 +123,34 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
     }
     const uint32_t rows = level + K;
     u64* out = ext + ((size_t)b * beta + j) * rows * N + c;
+    // every y_a is below 2^50 when its source prime is: exact FP64 products for targets below 2^50
+    bool src_small = true;
+    double yd[ALPHA];
+#pragma unroll
+    for (int a = 0; a < ALPHA; a++) {
+        yd[a] = 0.0;
+        if (a < n_src) {
+            src_small = src_small && pcs[first + a].q < FESC_FP_LIMIT;
+            yd[a] = fp_from_u64(y[a] & 0x000FFFFFFFFFFFFFull);
+        }
+    }
     for (uint32_t t = 0; t < rows; t++) {
         if (t >= first && t < first + n_src) continue;
         const uint32_t pt = t < level ? t : n_q + (t - level);
-        acc128 acc{0, 0};
+        if (src_small && pcs[pt].q < FESC_FP_LIMIT) {
+            const double q = pcs[pt].qd, qinv = pcs[pt].qinvd;
+            double s = 0.0;
 #pragma unroll
-        for (int a = 0; a < ALPHA; a++)
-            if (a < n_src) mac128(acc, y[a], dg->mat[a][pt]);
-        out[(size_t)t * N] = reduce128(acc.hi, acc.lo, pcs[pt]);
+            for (int a = 0; a < ALPHA; a++)
+                if (a < n_src) s += fp_modmul(yd[a], fp_from_u64(dg->mat[a][pt]), q, qinv);
+            out[(size_t)t * N] = fp_store(s, q, qinv);
+        } else {
+            acc128 acc{0, 0};
+#pragma unroll
+            for (int a = 0; a < ALPHA; a++)
+                if (a < n_src) mac128(acc, y[a], dg->mat[a][pt]);
+            out[(size_t)t * N] = reduce128(acc.hi, acc.lo, pcs[pt]);
+        }
     }
 }
 
@@ -152,6 +172,45 @@ __global__ void __launch_bounds__(256) k_inner(const u64* __restrict__ d, const 
     const uint32_t rows = level + K, np = n_q + K;
     const uint32_t pt = t < level ? t : n_q + (t - level);
     const uint32_t own = t < level ? t / alpha : 0xFFFFFFFFu;
+    if (pcs[pt].q < FESC_FP_LIMIT) {
+        // exact FP64 products: |x| <= q/2, key words in [0,q); beta terms of at most 0.7q each stay below
+        // 2^53 for beta <= 8, and are folded back every 8 digits otherwise
+        const double q = pcs[pt].qd, qinv = pcs[pt].qinvd;
+        double f0[BT], f1[BT];
+#pragma unroll
+        for (int i = 0; i < BT; i++) f0[i] = f1[i] = 0.0;
+        for (uint32_t j = 0; j < beta; j++) {
+            const double kb = fp_from_u64(__ldg(key + ((size_t)(2 * j) * np + pt) * N + c));
+            const double ka = fp_from_u64(__ldg(key + ((size_t)(2 * j + 1) * np + pt) * N + c));
+#pragma unroll
+            for (int i = 0; i < BT; i++) {
+                const uint32_t b = b0 + i;
+                if (b < batch) {
+                    const u64 xi = (j == own) ? d[((size_t)b * level + t) * N + c]
+                                              : ext[(((size_t)b * beta + j) * rows + t) * N + c];
+                    const double x = fp_load(xi, q);
+                    f0[i] += fp_modmul(x, kb, q, qinv);
+                    f1[i] += fp_modmul(x, ka, q, qinv);
+                }
+            }
+            if ((j & 7) == 7) {
+#pragma unroll
+                for (int i = 0; i < BT; i++) {
+                    f0[i] = fp_reduce(f0[i], q, qinv);
+                    f1[i] = fp_reduce(f1[i], q, qinv);
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < BT; i++) {
+            const uint32_t b = b0 + i;
+            if (b < batch) {
+                acc[(((size_t)b * 2 + 0) * rows + t) * N + c] = fp_store(f0[i], q, qinv);
+                acc[(((size_t)b * 2 + 1) * rows + t) * N + c] = fp_store(f1[i], q, qinv);
+            }
+        }
+        return;
+    }
     acc128 a0[BT], a1[BT];
 #pragma unroll
     for (int i = 0; i < BT; i++) a0[i] = a1[i] = acc128{0, 0};
