@@ -142,6 +142,7 @@ struct ModDownTab {
     u64 inv[FESC_MAX_SPECIAL], invs[FESC_MAX_SPECIAL];   // (P/p_k)^-1 mod p_k
     u64 half[FESC_MAX_SPECIAL];                          // floor(p_k / 2)
     u64 mat[FESC_MAX_SPECIAL][FESC_MAX_PRIMES];          // (P/p_k) mod q_i
+    u64 mat30[FESC_MAX_SPECIAL][FESC_MAX_PRIMES];        // (P/p_k) * 2^30 mod q_i
     u64 wrap[FESC_MAX_SPECIAL + 1][FESC_MAX_PRIMES];     // cnt * P mod q_i
     u64 pinv[FESC_MAX_PRIMES], pinvs[FESC_MAX_PRIMES];   // P^-1 mod q_i
 };

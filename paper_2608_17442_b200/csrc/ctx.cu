@@ -212,6 +212,7 @@ static int build_tables(fesc_ctx* ctx) {
             for (uint32_t b = 0; b < K; b++)
                 if (b != k) m = h_mul(m, q[nq + b] % q[i], q[i]);
             md.mat[k][i] = m;
+            md.mat30[k][i] = h_mul(m, (1ull << 30) % q[i], q[i]);
         }
     }
     for (uint32_t i = 0; i < nq; i++) {

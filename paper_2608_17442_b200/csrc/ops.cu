@@ -172,33 +172,63 @@ __global__ void __launch_bounds__(256) k_inner(const u64* __restrict__ d, const 
     const uint32_t rows = level + K, np = n_q + K;
     const uint32_t pt = t < level ? t : n_q + (t - level);
     const uint32_t own = t < level ? t / alpha : 0xFFFFFFFFu;
+    // operand words of one digit: key (b, a) and the BT ciphertext words; clamped indices keep loads valid
+    auto load_digit = [&](uint32_t j, u64& kb, u64& ka, u64 (&x)[BT]) {
+        kb = __ldg(key + ((size_t)(2 * j) * np + pt) * N + c);
+        ka = __ldg(key + ((size_t)(2 * j + 1) * np + pt) * N + c);
+#pragma unroll
+        for (int i = 0; i < BT; i++) {
+            const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
+            x[i] = (j == own) ? d[((size_t)b * level + t) * N + c] : ext[(((size_t)b * beta + j) * rows + t) * N + c];
+        }
+    };
     if (pcs[pt].q < FESC_FP_LIMIT) {
-        // exact FP64 products: |x| <= q/2, key words in [0,q); beta terms of at most 0.7q each stay below
-        // 2^53 for beta <= 8, and are folded back every 8 digits otherwise
+        // exact FP64 products: |x| <= q/2, key words in [0,q); up to 8 terms of at most 0.7q stay below 2^53,
+        // longer sums are folded back every 8 digits.  The next digit's words are loaded while this one is used.
         const double q = pcs[pt].qd, qinv = pcs[pt].qinvd;
         double f0[BT], f1[BT];
 #pragma unroll
         for (int i = 0; i < BT; i++) f0[i] = f1[i] = 0.0;
-        for (uint32_t j = 0; j < beta; j++) {
-            const double kb = fp_from_u64(__ldg(key + ((size_t)(2 * j) * np + pt) * N + c));
-            const double ka = fp_from_u64(__ldg(key + ((size_t)(2 * j + 1) * np + pt) * N + c));
+        if (beta <= 8) {
+            // all digits' words are requested before the first product, so a thread has up to
+            // 8 * (2 + BT) loads in flight
+            u64 kb[8], ka[8], x[8][BT];
 #pragma unroll
-            for (int i = 0; i < BT; i++) {
-                const uint32_t b = b0 + i;
-                if (b < batch) {
-                    const u64 xi = (j == own) ? d[((size_t)b * level + t) * N + c]
-                                              : ext[(((size_t)b * beta + j) * rows + t) * N + c];
-                    const double x = fp_load(xi, q);
-                    f0[i] += fp_modmul(x, kb, q, qinv);
-                    f1[i] += fp_modmul(x, ka, q, qinv);
+            for (int j = 0; j < 8; j++)
+                if ((uint32_t)j < beta) load_digit(j, kb[j], ka[j], x[j]);
+#pragma unroll
+            for (int j = 0; j < 8; j++)
+                if ((uint32_t)j < beta) {
+                    const double dkb = fp_from_u64(kb[j]), dka = fp_from_u64(ka[j]);
+#pragma unroll
+                    for (int i = 0; i < BT; i++) {
+                        const double xd = fp_load(x[j][i], q);
+                        f0[i] += fp_modmul(xd, dkb, q, qinv);
+                        f1[i] += fp_modmul(xd, dka, q, qinv);
+                    }
                 }
-            }
-            if ((j & 7) == 7) {
+        } else {
+            u64 kb, ka, x[BT], nkb, nka, nx[BT];
+            load_digit(0, kb, ka, x);
+            for (uint32_t j = 0; j < beta; j++) {
+                load_digit(j + 1 < beta ? j + 1 : j, nkb, nka, nx);
+                const double dkb = fp_from_u64(kb), dka = fp_from_u64(ka);
 #pragma unroll
                 for (int i = 0; i < BT; i++) {
-                    f0[i] = fp_reduce(f0[i], q, qinv);
-                    f1[i] = fp_reduce(f1[i], q, qinv);
+                    const double xd = fp_load(x[i], q);
+                    f0[i] += fp_modmul(xd, dkb, q, qinv);
+                    f1[i] += fp_modmul(xd, dka, q, qinv);
                 }
+                if ((j & 7) == 7) {
+#pragma unroll
+                    for (int i = 0; i < BT; i++) {
+                        f0[i] = fp_reduce(f0[i], q, qinv);
+                        f1[i] = fp_reduce(f1[i], q, qinv);
+                    }
+                }
+                kb = nkb, ka = nka;
+#pragma unroll
+                for (int i = 0; i < BT; i++) x[i] = nx[i];
             }
         }
 #pragma unroll
@@ -214,17 +244,19 @@ __global__ void __launch_bounds__(256) k_inner(const u64* __restrict__ d, const 
     acc128 a0[BT], a1[BT];
 #pragma unroll
     for (int i = 0; i < BT; i++) a0[i] = a1[i] = acc128{0, 0};
-    for (uint32_t j = 0; j < beta; j++) {
-        const u64 kb = __ldg(key + ((size_t)(2 * j) * np + pt) * N + c);
-        const u64 ka = __ldg(key + ((size_t)(2 * j + 1) * np + pt) * N + c);
+    {
+        u64 kb, ka, x[BT], nkb, nka, nx[BT];
+        load_digit(0, kb, ka, x);
+        for (uint32_t j = 0; j < beta; j++) {
+            load_digit(j + 1 < beta ? j + 1 : j, nkb, nka, nx);
 #pragma unroll
-        for (int i = 0; i < BT; i++) {
-            const uint32_t b = b0 + i;
-            if (b < batch) {
-                u64 x = (j == own) ? d[((size_t)b * level + t) * N + c] : ext[(((size_t)b * beta + j) * rows + t) * N + c];
-                mac128(a0[i], x, kb);
-                mac128(a1[i], x, ka);
+            for (int i = 0; i < BT; i++) {
+                mac128(a0[i], x[i], kb);
+                mac128(a1[i], x[i], ka);
             }
+            kb = nkb, ka = nka;
+#pragma unroll
+            for (int i = 0; i < BT; i++) x[i] = nx[i];
         }
     }
     const PrimeConst pc = pcs[pt];
@@ -262,13 +294,33 @@ __global__ void __launch_bounds__(256) k_moddown_conv(const u64* __restrict__ ac
             cnt += y[k] > tab->half[k];
         }
     }
-    for (uint32_t i = 0; i < level; i++) {
-        acc128 a{0, 0};
+    // 30-bit halves of every y_k as doubles, for targets below 2^50 (exact FP64 products)
+    double yh[FESC_MAX_SPECIAL], yl[FESC_MAX_SPECIAL];
 #pragma unroll
-        for (int k = 0; k < FESC_MAX_SPECIAL; k++)
-            if (k < K) mac128(a, y[k], tab->mat[k][i]);
-        u64 v = reduce128(a.hi, a.lo, pcs[i]);
-        u[((size_t)bp * level + i) * N + c] = submod(v, tab->wrap[cnt][i], pcs[i].q);
+    for (int k = 0; k < FESC_MAX_SPECIAL; k++) {
+        yh[k] = fp_from_u64(y[k] >> 30);
+        yl[k] = fp_from_u64(y[k] & ((1ull << 30) - 1));
+    }
+    for (uint32_t i = 0; i < level; i++) {
+        if (pcs[i].q < FESC_FP_LIMIT) {
+            const double q = pcs[i].qd, qinv = pcs[i].qinvd;
+            double s = -fp_from_u64(tab->wrap[cnt][i]);
+#pragma unroll
+            for (int k = 0; k < FESC_MAX_SPECIAL; k++)
+                if (k < K) {
+                    s += fp_modmul(yh[k], fp_from_u64(tab->mat30[k][i]), q, qinv);
+                    s += fp_modmul(yl[k], fp_from_u64(tab->mat[k][i]), q, qinv);
+                    if (k == 3) s = fp_reduce(s, q, qinv);
+                }
+            u[((size_t)bp * level + i) * N + c] = fp_store(s, q, qinv);
+        } else {
+            acc128 a{0, 0};
+#pragma unroll
+            for (int k = 0; k < FESC_MAX_SPECIAL; k++)
+                if (k < K) mac128(a, y[k], tab->mat[k][i]);
+            u64 v = reduce128(a.hi, a.lo, pcs[i]);
+            u[((size_t)bp * level + i) * N + c] = submod(v, tab->wrap[cnt][i], pcs[i].q);
+        }
     }
 }
 
@@ -283,9 +335,17 @@ __global__ void __launch_bounds__(256) k_moddown_finish(const u64* __restrict__ 
     if (c >= N) return;
     const uint32_t b = bp >> 1, p = bp & 1;
     const u64 q = pcs[i].q;
-    u64 v = submod(acc[((size_t)bp * (level + K) + i) * N + c], u[((size_t)bp * level + i) * N + c], q);
-    v = shoup(v, tab->pinv[i], tab->pinvs[i], q);
     u64* o = out + (size_t)b * out_stride + ((size_t)p * level + i) * N + c;
+    const u64 av = acc[((size_t)bp * (level + K) + i) * N + c], uv = u[((size_t)bp * level + i) * N + c];
+    if (q < FESC_FP_LIMIT) {
+        const double qd = pcs[i].qd, qinv = pcs[i].qinvd;
+        double s = fp_modmul(fp_load(av, qd) - fp_load(uv, qd), fp_from_u64(tab->pinv[i]), qd, qinv);
+        if ((add_mask >> p) & 1) s += fp_load(*o, qd);
+        *o = fp_store(s, qd, qinv);
+        return;
+    }
+    u64 v = submod(av, uv, q);
+    v = shoup(v, tab->pinv[i], tab->pinvs[i], q);
     if ((add_mask >> p) & 1) v = addmod(v, *o, q);
     *o = v;
 }
