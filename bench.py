@@ -166,9 +166,12 @@ def peaks():
 
 # Integer-pipe ceiling for the 128-bit multiply-accumulate kernels: see DESIGN.md ("ALU roofline").
 SM_COUNT = 148
-IMAD_PER_CLK_PER_SM = 64          # 32-bit multiply-adds per SM per clock (measured 63.6 with a register chain)
-MAC128_IMAD = 8                   # 64x64->128 multiply-accumulate = 4 products of 32x32->64 = 8 multiply-adds
-BFLY_IMAD = 20                    # Shoup butterfly = one high + two low 64-bit products = 10 products
+IMAD_PER_CLK_PER_SM = 64          # 32-bit multiply-adds per SM per clock (measured 63 with a register chain)
+FP64_PER_CLK_PER_SM = 64          # FP64 FMAs per SM per clock (measured 63 with a register chain)
+BFLY_IMAD = 20                    # integer Shoup butterfly (primes >= 2^50): 10 products of 32x32->64
+BFLY_FP64 = 8.5                   # FP64 butterfly (primes < 2^50): 5 ops product + 2 adds + 1.5 fold-back share
+MAC_FP64 = 6                      # FP64 multiply-accumulate: 5 ops exact product + 1 add
+INT_LIMB_SHARE = 32.0 / 224.0     # transforms on the 60-bit special primes per key switch (integer path)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -320,8 +323,8 @@ def run_ours(args):
         macs = tb_per_launch * nout * N2 * gin * N1 * 2 * LEVEL * n          # 64x64->128 multiply-adds
         t = dom_ms * 1e-3 / max(1, dom_records)
         sm_mhz = clocks.get("sm_mhz") or 1350.0
-        alu_peak = SM_COUNT * IMAD_PER_CLK_PER_SM * sm_mhz * 1e6 / MAC128_IMAD / 1e12   # T mul-adds / s
-        roof.update({"bound": "alu", "achieved": macs / t / 1e12, "peak": alu_peak, "unit": "T mac128/s",
+        alu_peak = SM_COUNT * FP64_PER_CLK_PER_SM * sm_mhz * 1e6 / MAC_FP64 / 1e12   # T modular mul-adds / s
+        roof.update({"bound": "alu", "achieved": macs / t / 1e12, "peak": alu_peak, "unit": "T modular mac/s (FP64 pipe)",
                      "frac": macs / t / 1e12 / alu_peak, "traffic": None,
                      "hbm": {"achieved": alg / t / 1e9, "peak": hbm_peak, "unit": "GB/s", "frac": alg / t / 1e9 / hbm_peak,
                              "algorithmic_bytes_per_launch": alg}})
@@ -329,9 +332,13 @@ def run_ours(args):
         # all transform launches of the timed steps: butterflies per second against the multiply-add ceiling
         bfly = limb_ntts * (n // 2) * p["log_n"]
         sm_mhz = clocks.get("sm_mhz") or 1350.0
-        alu_peak = SM_COUNT * IMAD_PER_CLK_PER_SM * sm_mhz * 1e6 / BFLY_IMAD / 1e12
+        peak_fp = SM_COUNT * FP64_PER_CLK_PER_SM * sm_mhz * 1e6 / BFLY_FP64 / 1e12
+        peak_int = SM_COUNT * IMAD_PER_CLK_PER_SM * sm_mhz * 1e6 / BFLY_IMAD / 1e12
+        alu_peak = 1.0 / ((1.0 - INT_LIMB_SHARE) / peak_fp + INT_LIMB_SHARE / peak_int)
         ach = bfly / (dom_ms * 1e-3) / 1e12
-        roof.update({"bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "T butterflies/s",
+        roof.update({"bound": "alu", "achieved": ach, "peak": alu_peak,
+                     "unit": "T butterflies/s (FP64 pipe for 50-bit primes, integer pipe for 60-bit)",
+                     "peak_fp64_path": peak_fp, "peak_integer_path": peak_int,
                      "frac": ach / alu_peak, "traffic": None, "limb_transforms_per_step": limb_ntts // args.steps,
                      "family_ms_per_step": dom_ms / args.steps,
                      "hbm": {"achieved": limb_ntts * 2 * n * 8 / (dom_ms * 1e-3) / 1e9, "peak": hbm_peak, "unit": "GB/s",

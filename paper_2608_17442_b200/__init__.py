@@ -12,7 +12,7 @@ import ctypes
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libfesc_b200.so")
+LIB_PATH = os.environ.get("FESC_LIB", os.path.join(_HERE, "libfesc_b200.so"))
 
 OK, EINVAL, ENOMEM, ECUDA, ELEVEL, ENOKEY, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 CONJ = -(1 << 31)

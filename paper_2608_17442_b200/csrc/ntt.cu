@@ -15,6 +15,15 @@
 // N <= 2^12 runs as one shared-memory kernel per row (tests and the tiny workload).
 #include "common.cuh"
 
+// CTA shapes of the N = 2^16 kernels: columns per CTA of the strided kernel (x 32 sub-threads) and
+// 256-point blocks (= warps) per CTA of the contiguous kernel.
+#ifndef NTT_COLS
+#define NTT_COLS 8
+#endif
+#ifndef NTT_WARPS
+#define NTT_WARPS 8
+#endif
+
 // twiddle index of local stage ls (of S) for local element e with prefix pre:
 //   pre * 2^ls + (e >> (S - ls))
 // (pre = 1 for the strided kernel; pre = 256 + block index for the contiguous kernel).
@@ -137,7 +146,7 @@ template <bool INV, bool W>
 __device__ __forceinline__ void strided_body(u64* __restrict__ p, u64* __restrict__ sm, const ulonglong2* __restrict__ tw,
                                              const PrimeConst& pc) {
     const u64 q = pc.q, q2 = 2 * pc.q;
-    const uint32_t col = threadIdx.x & 15, sub = threadIdx.x >> 4;
+    const uint32_t col = threadIdx.x & (NTT_COLS - 1), sub = threadIdx.x / NTT_COLS;
     const uint32_t h2 = sub >> 2, l2 = sub & 3;
     u64 x[8];
     if (!INV) {
@@ -146,18 +155,18 @@ __device__ __forceinline__ void strided_body(u64* __restrict__ p, u64* __restric
         for (int k = 0; k < 8; k++) x[k] = p[(size_t)(k * 32 + sub) * 256 + col];
         fwd_round3<W>(x, tw, 1, 2, 4, q, q2);
 #pragma unroll
-        for (int k = 0; k < 8; k++) sm[(k * 32 + sub) * 16 + col] = x[k];
+        for (int k = 0; k < 8; k++) sm[(k * 32 + sub) * NTT_COLS + col] = x[k];
         __syncthreads();
         // round 2: hi = h2*32 + k*4 + l2, local stages 3,4,5
 #pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * 16 + col];
+        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * NTT_COLS + col];
         fwd_round3<W>(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, q2);
 #pragma unroll
-        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * 16 + col] = x[k];
+        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * NTT_COLS + col] = x[k];
         __syncthreads();
         // round 3: hi = sub*8 + k, local stages 6,7
 #pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[(sub * 8 + k) * 16 + col];
+        for (int k = 0; k < 8; k++) x[k] = sm[(sub * 8 + k) * NTT_COLS + col];
         fwd_round2<W>(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, q2);
 #pragma unroll
         for (int k = 0; k < 8; k++) p[(size_t)(sub * 8 + k) * 256 + col] = x[k];  // lazily reduced
@@ -167,16 +176,16 @@ __device__ __forceinline__ void strided_body(u64* __restrict__ p, u64* __restric
         for (int k = 0; k < 8; k++) x[k] = p[(size_t)(sub * 8 + k) * 256 + col];
         inv_round2<W>(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, q2, off);
 #pragma unroll
-        for (int k = 0; k < 8; k++) sm[(sub * 8 + k) * 16 + col] = x[k];
+        for (int k = 0; k < 8; k++) sm[(sub * 8 + k) * NTT_COLS + col] = x[k];
         __syncthreads();
 #pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * 16 + col];
+        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * NTT_COLS + col];
         inv_round3<W>(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, q2, 4 * off);
 #pragma unroll
-        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * 16 + col] = x[k];
+        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * NTT_COLS + col] = x[k];
         __syncthreads();
 #pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[(k * 32 + sub) * 16 + col];
+        for (int k = 0; k < 8; k++) x[k] = sm[(k * 32 + sub) * NTT_COLS + col];
         // stages 2,1 then the last stage with N^-1 folded in (exact products, canonical output)
         {
 #pragma unroll
@@ -272,7 +281,7 @@ template <bool INV>
 __device__ __forceinline__ void strided_body_fp(u64* __restrict__ p, double* __restrict__ sm, const double* __restrict__ tw,
                                                 const PrimeConst& pc) {
     const double q = pc.qd, qinv = pc.qinvd;
-    const uint32_t col = threadIdx.x & 15, sub = threadIdx.x >> 4;
+    const uint32_t col = threadIdx.x & (NTT_COLS - 1), sub = threadIdx.x / NTT_COLS;
     const uint32_t h2 = sub >> 2, l2 = sub & 3;
     double x[8];
     if (!INV) {
@@ -281,17 +290,17 @@ __device__ __forceinline__ void strided_body_fp(u64* __restrict__ p, double* __r
         fp_fwd_round3(x, tw, 1, 2, 4, q, qinv);
         fp_reduce8(x, q, qinv);
 #pragma unroll
-        for (int k = 0; k < 8; k++) sm[(k * 32 + sub) * 16 + col] = x[k];
+        for (int k = 0; k < 8; k++) sm[(k * 32 + sub) * NTT_COLS + col] = x[k];
         __syncthreads();
 #pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * 16 + col];
+        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * NTT_COLS + col];
         fp_fwd_round3(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, qinv);
         fp_reduce8(x, q, qinv);
 #pragma unroll
-        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * 16 + col] = x[k];
+        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * NTT_COLS + col] = x[k];
         __syncthreads();
 #pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[(sub * 8 + k) * 16 + col];
+        for (int k = 0; k < 8; k++) x[k] = sm[(sub * 8 + k) * NTT_COLS + col];
         fp_fwd_round2(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, qinv);
         fp_reduce8(x, q, qinv);
         // handed to the contiguous kernel as doubles, |x| <= q/2
@@ -304,17 +313,17 @@ __device__ __forceinline__ void strided_body_fp(u64* __restrict__ p, double* __r
         fp_inv_round2(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, qinv);
         fp_reduce8(x, q, qinv);
 #pragma unroll
-        for (int k = 0; k < 8; k++) sm[(sub * 8 + k) * 16 + col] = x[k];
+        for (int k = 0; k < 8; k++) sm[(sub * 8 + k) * NTT_COLS + col] = x[k];
         __syncthreads();
 #pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * 16 + col];
+        for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * NTT_COLS + col];
         fp_inv_round3(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, qinv);
         fp_reduce8(x, q, qinv);
 #pragma unroll
-        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * 16 + col] = x[k];
+        for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * NTT_COLS + col] = x[k];
         __syncthreads();
 #pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = sm[(k * 32 + sub) * 16 + col];
+        for (int k = 0; k < 8; k++) x[k] = sm[(k * 32 + sub) * NTT_COLS + col];
         // stages 2, 1, then the last stage with N^-1 folded in
 #pragma unroll
         for (int k = 0; k < 4; k++) fp_gs(x[2 * k], x[2 * k + 1], ldf(tw, 4 + k), q, qinv);
@@ -396,16 +405,17 @@ __device__ __forceinline__ void contig_body_fp(u64* __restrict__ p, double* __re
 }
 
 template <bool INV>
-__global__ void __launch_bounds__(512) ntt16_strided(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
+__global__ void __launch_bounds__(NTT_COLS * 32) ntt16_strided(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
                                                      const double* __restrict__ twf_all,
-                                                     const PrimeConst* __restrict__ pcs, RowMap map) {
+                                                     const PrimeConst* __restrict__ pcs, RowMap map,
+                                                     uint32_t row_base) {
     const uint32_t row = blockIdx.y;
-    const uint32_t pi = map.prime[row % map.period];
+    const uint32_t pi = map.prime[(row_base + row) % map.period];
     if (pi == 0xFF) return;
-    __shared__ u64 sm[256 * 16];
+    __shared__ u64 sm[256 * NTT_COLS];
     const PrimeConst pc = pcs[pi];
     const ulonglong2* tw = tw_all + (size_t)pi * N16;
-    u64* p = data + (size_t)row * N16 + blockIdx.x * 16;
+    u64* p = data + (size_t)row * N16 + blockIdx.x * NTT_COLS;
     if (pc.q < FP_LIMIT)
         strided_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc);
     else if (pc.q < WIDE_LIMIT)
@@ -484,17 +494,18 @@ __device__ __forceinline__ void contig_body(u64* __restrict__ p, u64* __restrict
 }
 
 template <bool INV>
-__global__ void __launch_bounds__(512) ntt16_contig(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
+__global__ void __launch_bounds__(NTT_WARPS * 32) ntt16_contig(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
                                                     const double* __restrict__ twf_all,
-                                                    const PrimeConst* __restrict__ pcs, RowMap map) {
+                                                    const PrimeConst* __restrict__ pcs, RowMap map,
+                                                    uint32_t row_base) {
     const uint32_t row = blockIdx.y;
-    const uint32_t pi = map.prime[row % map.period];
+    const uint32_t pi = map.prime[(row_base + row) % map.period];
     if (pi == 0xFF) return;
-    __shared__ u64 sm_all[16 * 288];
+    __shared__ u64 sm_all[NTT_WARPS * 288];
     const PrimeConst pc = pcs[pi];
     const ulonglong2* tw = tw_all + (size_t)pi * N16;
     const uint32_t warp = threadIdx.x >> 5;
-    const uint32_t blk = blockIdx.x * 16 + warp;   // 256-point block index within the limb
+    const uint32_t blk = blockIdx.x * NTT_WARPS + warp;   // 256-point block index within the limb
     u64* p = data + (size_t)row * N16 + (size_t)blk * 256;
     u64* sm = sm_all + warp * 288;
     if (pc.q < FP_LIMIT)
@@ -571,22 +582,21 @@ int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool 
     prof_begin(ctx, PF_NTT, st);
     uint64_t launches = 0;
     if (ctx->log_n == 16) {
-        // gridDim.y is limited to 65535 rows per launch
-        for (size_t r0 = 0; r0 < rows;) {
-            size_t chunk = rows - r0;
-            size_t lim = 65535 / map.period * map.period;
-            if (lim == 0) return fesc_fail(ctx, FESC_EINVAL, "ntt: row map period too large");
-            if (chunk > lim) chunk = lim;
-            dim3 grid(16, (unsigned)chunk);
+        // gridDim.y is limited to 65535 rows per launch.  (Splitting into L2-sized chunks was measured:
+        // slower, the extra launch tails cost more than the L2 hits save.)
+        const size_t chunk_rows = 65535;
+        for (size_t r0 = 0; r0 < rows; r0 += chunk_rows) {
+            const size_t chunk = rows - r0 < chunk_rows ? rows - r0 : chunk_rows;
+            const uint32_t rb = (uint32_t)(r0 % map.period);
+            dim3 gs(256 / NTT_COLS, (unsigned)chunk), gc(256 / NTT_WARPS, (unsigned)chunk);
             u64* base = d_data + r0 * (size_t)N16;
             if (!inverse) {
-                ntt16_strided<false><<<grid, 512, 0, st>>>(base, tw, twf, ctx->d_pc, map);
-                ntt16_contig<false><<<grid, 512, 0, st>>>(base, tw, twf, ctx->d_pc, map);
+                ntt16_strided<false><<<gs, NTT_COLS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb);
+                ntt16_contig<false><<<gc, NTT_WARPS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb);
             } else {
-                ntt16_contig<true><<<grid, 512, 0, st>>>(base, tw, twf, ctx->d_pc, map);
-                ntt16_strided<true><<<grid, 512, 0, st>>>(base, tw, twf, ctx->d_pc, map);
+                ntt16_contig<true><<<gc, NTT_WARPS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb);
+                ntt16_strided<true><<<gs, NTT_COLS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb);
             }
-            r0 += chunk;
             launches += 2;
         }
     } else {
