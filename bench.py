@@ -392,6 +392,86 @@ def run_ours(args):
     del ctx
 
 
+# ---------------------------------------------------------------------------------------------
+# optional second workload: the scan-contract of one Mamba-2-base layer (or a slice of it)
+# ---------------------------------------------------------------------------------------------
+def scan_rotation_amounts(n, P, d_s, B, stride):
+    """Slot rotations the scan-contract uses (see include/fesc.h), as left shifts modulo n."""
+    import math
+
+    dg = min(16, B)
+    c_state = n // stride
+    R = P * stride
+    am = set()
+    for unit in (1, P, d_s):
+        am |= {unit * t % n for t in range(1, dg)} | {unit * dg * t % n for t in range(1, B // dg)}
+    am |= {(-t) % n for t in range(1, dg)} | {(-dg * t) % n for t in range(1, B // dg)}
+    am |= {(-(1 << b)) % n for b in range(int(math.log2(max(d_s, P))))}
+    am |= {(-P * (1 << b)) % n for b in range(int(math.log2(R // P)))}
+    am |= {(-stride * (1 << b)) % n for b in range(int(math.log2(c_state)))}
+    am |= {(1 << b) for b in range(int(math.log2(d_s)))}
+    am.discard(0)
+    return sorted(am)
+
+
+def run_scan(args):
+    """Times fesc_scan_contract on synthetic residues of the deployed geometry (N=2^16, 24 limbs, stride 256,
+    B_blk=256, d_s=128, P=64).  --workload scan_slice: 4 heads x 512 tokens; scan_layer: 24 heads x 2048 tokens."""
+    import torch
+    import fesc_synth as S
+    import paper_2608_17442_b200 as fesc
+
+    torch.cuda.set_device(0)
+    p = S.params("full")
+    ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+    n, N = ctx.N // 2, ctx.N
+    H, L = (4, 512) if args.workload == "scan_slice" else (24, 2048)
+    P, d_s, B, stride, l0 = 64, 128, 256, 256, 24
+    K_s, K_blk = H * P // (n // stride), L // B
+    base = 100000
+    for r in scan_rotation_amounts(n, P, d_s, B, stride):
+        ctx.add_galois_key(r, base + r)
+    ctx.add_galois_key(fesc.CONJ, base + n)
+    seed = S.config_seed(5)
+    q = p["primes"][:l0]
+
+    def cts(count, stream):
+        r = S.hashed_residues(seed, stream, q, count * 2 * N, device="cuda")
+        return r.view(l0, count, 2, N).permute(1, 2, 0, 3).contiguous()
+
+    x, a = cts(K_blk * K_s, 1), cts(K_blk * K_s, 2)
+    Bc, Cc = cts(K_blk, 3), cts(K_blk, 4)
+    masks = [S.hashed_residues(seed, 10 + i, q, N, device="cuda").contiguous() for i in range(4)]
+    linj = l0 - 2 - 2 * 8 + 1
+    out = torch.empty((K_blk, K_s, 2, linj - 3, N), dtype=torch.int64, device="cuda")
+    adj = [(1 << 49) + 12345 * i for i in range((l0 + 1) ** 2)]
+    desc = fesc.ScanDesc(L, H, P, d_s, B, 0, l0, base)
+    torch.cuda.empty_cache()
+
+    def step():
+        ctx.scan_contract(x, a, Bc, Cc, desc, masks[0], masks[1], masks[2], masks[3][:linj - 2], adj, adj, out)
+
+    if args.workload == "scan_slice":
+        step()                      # warm-up (sizes the scratch arena)
+    ctx.sync()
+    c0 = ctx.counters()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    step()
+    e1.record()
+    ctx.sync()
+    c1 = ctx.counters()
+    ms = e0.elapsed_time(e1)
+    ks = c1[1] - c0[1]
+    print(json.dumps({"metric": "scan-contract key-switches/s", "value": ks / (ms * 1e-3), "unit": "key-switches/s",
+                      "n_gpus": 1, "steps": 1, "warmup": 1 if args.workload == "scan_slice" else 0, "ms_per_step": ms,
+                      "higher_is_better": True, "dtype": "u64", "data": "synthetic",
+                      "config": {"workload": "%s: L=%d, H=%d, P=64, d_s=128, B_blk=256, K_s=%d, N=2^16, 24 limbs"
+                                             % (args.workload, L, H, K_s)},
+                      "key_switches": ks, "limb_transforms": c1[0] - c0[0], "gpu_launches": c1[4] - c0[4],
+                      "scratch_gib": c1[3] / 2**30}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -404,7 +484,11 @@ def main():
                     help="run ONE step of a small case (1 input block, 1 output block, 2 token blocks) and exit; for ncu")
     ap.add_argument("--profile-step", dest="profile_step", action="store_true",
                     help="run ONE step of the full workload without warm-up and exit; for the ncu launch list")
+    ap.add_argument("--workload", default="in_proj", choices=["in_proj", "scan_slice", "scan_layer"],
+                    help="in_proj (default, the benchmark metric) or a scan-contract run")
     args = ap.parse_args()
+    if args.workload != "in_proj":
+        return run_scan(args)
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -112,11 +112,15 @@ class Context:
             raise FescError(rc, lib().fesc_last_error(self.h).decode())
 
     def close(self):
-        if getattr(self, "h", None):
-            lib().fesc_ctx_destroy(self.h)
+        if getattr(self, "h", None) and _lib is not None:
+            _lib.fesc_ctx_destroy(self.h)
             self.h = None
 
-    __del__ = close
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:      # interpreter shutdown: module globals may already be gone
+            pass
 
     def sync(self):
         self._chk(lib().fesc_sync(self.h, _stream()))
