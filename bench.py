@@ -262,7 +262,7 @@ def run_ours(args):
     ct, diags = make_inputs(p["primes"], n, gin, nout, tbs, S.config_seed(4) + rank, dev)
     out = torch.empty((tbs, nout, 2, LEVEL - 1, n), dtype=torch.int64, device=dev)
     torch.cuda.empty_cache()
-    desc = fesc.BsgsDesc(N1, N2, gin, nout, tbs, LEVEL, BABY_BASE, GIANT_BASE)
+    desc = fesc.BsgsDesc(N1, N2, gin, nout, tbs, LEVEL, BABY_BASE, GIANT_BASE, int(args.hoist))
 
     def step():
         ctx.linear(ct, diags, desc, out)
@@ -373,7 +373,8 @@ def run_ours(args):
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "latency_ms": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
         "config": {"workload": "in_proj 768->3352, L=2048 tokens, N=2^16, 24x50-bit limbs + 4x60-bit special primes, "
-                               "6 key-switch digits, C=256 T=128 n1=32 n2=8",
+                               "6 key-switch digits, C=256 T=128 n1=32 n2=8, baby rotations %s"
+                               % ("hoisted (one decomposition per input ciphertext)" if args.hoist else "by plain rotations"),
                    "input_cts": tbs * gin, "diagonals": nout * N2 * gin * N1, "output_cts": tbs * nout,
                    "key_switches_per_step": ks_per_step, "macs_per_step": tbs * nout * N2 * gin * N1,
                    "l2": "inputs larger than L2 (diagonals %.1f GiB stream every step)" % (diags.numel() * 8 / 2**30),
@@ -484,6 +485,8 @@ def main():
                     help="run ONE step of a small case (1 input block, 1 output block, 2 token blocks) and exit; for ncu")
     ap.add_argument("--profile-step", dest="profile_step", action="store_true",
                     help="run ONE step of the full workload without warm-up and exit; for the ncu launch list")
+    ap.add_argument("--hoist", type=int, default=1, choices=[0, 1],
+                    help="1: baby rotations share one decomposition per input ciphertext (fesc_rotate_hoisted)")
     ap.add_argument("--workload", default="in_proj", choices=["in_proj", "scan_slice", "scan_layer"],
                     help="in_proj (default, the benchmark metric) or a scan-contract run")
     args = ap.parse_args()

@@ -261,6 +261,32 @@ class Oracle:
         ks = self.key_switch(d, key_id, level)
         return np.stack([self.add(c0, ks[0], data), ks[1]])
 
+    def rotate_hoisted(self, ct, key_ids):
+        """Several rotations of ONE ciphertext that share the decomposition of c1 ("hoisting"; a second,
+        separately defined mode).  c1 is brought to COEFF form, extended digit by digit (ModUp) and
+        transformed back ONCE; for every key the automorphism is applied to the extended digits (in EVAL
+        form a permutation), then inner product with the key and division by P as in `key_switch`:
+            out_g = (sigma_g c0 + ks0, ks1),  ks = ModDown( sum_j sigma_g(d~_j) (.) evk_{g,j} ).
+        The residues differ from `rotate` (the conversion overshoot is permuted instead of recomputed);
+        the decrypted value is the same rotation."""
+        level = ct.shape[1]
+        data = list(range(level))
+        ext = data + self.special
+        d_eval = _arr(ct[1])
+        d_coeff = self.intt(d_eval, data)
+        digits = [self.mod_up_digit(d_coeff, d_eval, j, level) for j in range(-(-level // self.alpha))]
+        outs = []
+        for kid in key_ids:
+            g, evk = self.keys[kid]
+            acc = np.zeros((2, len(ext), self.N), dtype=np.uint64)
+            for j, dj in enumerate(digits):
+                dt = self.automorphism(dj, g, len(ext))
+                for p in range(2):
+                    _lib.orc_muladd(dt, _arr(evk[j, p][ext]), acc[p], self._q(ext), len(ext), self.N)
+            c0 = self.automorphism(ct[0], g, level)
+            outs.append(np.stack([self.add(c0, self.mod_down(acc[0], level), data), self.mod_down(acc[1], level)]))
+        return outs
+
     def rescale(self, ct):
         """Rounded division by the last prime, level l -> l-1:
         c_i <- (c_i - [c_last]_centred) * q_last^-1 mod q_i  (= round(c / q_last) exactly)."""
@@ -297,7 +323,7 @@ class Oracle:
         return np.stack([self.mul(ct[p], m_eval, data) for p in range(2)])
 
     # ---- BSGS projection -----------------------------------------------------------
-    def linear(self, ct_in, diags, desc, baby_key_ids, giant_key_ids):
+    def linear(self, ct_in, diags, desc, baby_key_ids, giant_key_ids, hoist: bool = False):
         """Y = XW on packed ciphertexts (App. "Projection Kernel Breakdown", real packing).
 
         ct_in  [token_blocks, in_blocks, 2, l, N]
@@ -305,15 +331,20 @@ class Oracle:
         returns [token_blocks, out_blocks, 2, l-1, N]:
           acc_p = sum_g sum_q rot(x^(g), q*T) (.) D^(b)_{g,p,q};
           y^(b) = sum_p rot(acc_p, p*n1*T);  then rescale.
-        baby_key_ids[q] rotates by q*T (q >= 1), giant_key_ids[p] by p*n1*T (p >= 1)."""
+        baby_key_ids[q] rotates by q*T (q >= 1), giant_key_ids[p] by p*n1*T (p >= 1).
+        hoist=True: the baby rotations use `rotate_hoisted` (different residues, same values)."""
         n1, n2 = desc["n1"], desc["n2"]
         tbs, gin = ct_in.shape[0], ct_in.shape[1]
         level = ct_in.shape[3]
         nout = diags.shape[0]
         out = np.empty((tbs, nout, 2, level - 1, self.N), dtype=np.uint64)
         for tb in range(tbs):
-            rot = [[ct_in[tb, g] if q == 0 else self.rotate(ct_in[tb, g], baby_key_ids[q])
-                    for q in range(n1)] for g in range(gin)]
+            if hoist:   # baby rotations of one input share its decomposition
+                rot = [[ct_in[tb, g]] + self.rotate_hoisted(ct_in[tb, g], [baby_key_ids[q] for q in range(1, n1)])
+                       for g in range(gin)]
+            else:
+                rot = [[ct_in[tb, g] if q == 0 else self.rotate(ct_in[tb, g], baby_key_ids[q])
+                        for q in range(n1)] for g in range(gin)]
             for b in range(nout):
                 y = None
                 for p in range(n2):

@@ -29,7 +29,8 @@ class FescError(RuntimeError):
 
 class BsgsDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint32) for n in
-                ("n1", "n2", "in_blocks", "out_blocks", "token_blocks", "n_limbs", "baby_key_base", "giant_key_base")]
+                ("n1", "n2", "in_blocks", "out_blocks", "token_blocks", "n_limbs", "baby_key_base", "giant_key_base",
+                 "hoist")]
 
 
 class ScanDesc(ctypes.Structure):
@@ -64,6 +65,7 @@ def lib():
             "fesc_intt": [vp, vp, u32, u32, u32, vp],
             "fesc_ct_pt_mac": [vp, vp, vp, sz, vp, u32, u32, vp],
             "fesc_rotate": [vp, vp, vp, u32, u32, u32, vp],
+            "fesc_rotate_hoisted": [vp, vp, vp, u32, u32, c.POINTER(u32), u32, vp],
             "fesc_rescale": [vp, vp, vp, u32, u32, vp],
             "fesc_rescale_static": [vp, vp, vp, u32, u32, vp],
             "fesc_ct_ct_mul": [vp, vp, vp, vp, u32, u32, vp],
@@ -180,6 +182,10 @@ class Context:
 
     def rotate(self, ct_in, ct_out, batch: int, n_limbs: int, key_id: int):
         self._chk(lib().fesc_rotate(self.h, _ptr(ct_in), _ptr(ct_out), batch, n_limbs, key_id, _stream()))
+
+    def rotate_hoisted(self, ct_in, ct_out, batch: int, n_limbs: int, key_ids):
+        ids = (ctypes.c_uint32 * len(key_ids))(*key_ids)
+        self._chk(lib().fesc_rotate_hoisted(self.h, _ptr(ct_in), _ptr(ct_out), batch, n_limbs, ids, len(key_ids), _stream()))
 
     def rescale(self, ct_in, ct_out, batch: int, n_limbs: int):
         self._chk(lib().fesc_rescale(self.h, _ptr(ct_in), _ptr(ct_out), batch, n_limbs, _stream()))

@@ -352,10 +352,18 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
         // slot q = 0 of the rotated set is the input itself
         FESC_CHECK_CUDA(ctx, cudaMemcpy2DAsync(rot, (size_t)n1 * ctw * sizeof(u64), gin_base, ctw * sizeof(u64),
                                                ctw * sizeof(u64), (size_t)nt * gin, cudaMemcpyDeviceToDevice, st));
-        for (uint32_t q = 1; q < n1; q++) {
-            rc = rotate_internal(ctx, gin_base, ctw, rot + (size_t)q * ctw, (size_t)n1 * ctw, nt * gin, level,
-                                 desc->baby_key_base + q, ks, st, 0);
+        if (desc->hoist && n1 > 1) {
+            std::vector<uint32_t> ids;
+            for (uint32_t q = 1; q < n1; q++) ids.push_back(desc->baby_key_base + q);
+            rc = rotate_hoisted_internal(ctx, gin_base, ctw, rot + ctw, (size_t)n1 * ctw, ctw, nt * gin, level, ids.data(),
+                                         n1 - 1, ks, st);
             if (rc != FESC_OK) return rc;
+        } else {
+            for (uint32_t q = 1; q < n1; q++) {
+                rc = rotate_internal(ctx, gin_base, ctw, rot + (size_t)q * ctw, (size_t)n1 * ctw, nt * gin, level,
+                                     desc->baby_key_base + q, ks, st, 0);
+                if (rc != FESC_OK) return rc;
+            }
         }
         const uint32_t bp_count = nout * n2;
         prof_begin(ctx, PF_BSGS, st);

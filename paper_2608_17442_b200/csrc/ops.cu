@@ -161,14 +161,16 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
 // for BT products.
 // ---------------------------------------------------------------------------------------
 template <int BT>
-__global__ void __launch_bounds__(256) k_inner(const u64* __restrict__ d, const u64* __restrict__ ext,
+__global__ void __launch_bounds__(256, 2) k_inner(const u64* __restrict__ d, const u64* __restrict__ ext,
                                                const u64* __restrict__ key, u64* __restrict__ acc,
                                                const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
                                                uint32_t n_q, uint32_t K, uint32_t alpha, uint32_t beta,
-                                               uint32_t batch) {
+                                               uint32_t batch, uint32_t log_n, u64 g) {
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t t = blockIdx.y, b0 = blockIdx.z * BT;
     if (c >= N) return;
+    // hoisted rotations: the automorphism acts on the extended digits, i.e. they are read at pi_g(c)
+    const uint32_t cs = g ? galois_src(c, log_n, g) : c;
     const uint32_t rows = level + K, np = n_q + K;
     const uint32_t pt = t < level ? t : n_q + (t - level);
     const uint32_t own = t < level ? t / alpha : 0xFFFFFFFFu;
@@ -179,7 +181,7 @@ __global__ void __launch_bounds__(256) k_inner(const u64* __restrict__ d, const 
 #pragma unroll
         for (int i = 0; i < BT; i++) {
             const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
-            x[i] = (j == own) ? d[((size_t)b * level + t) * N + c] : ext[(((size_t)b * beta + j) * rows + t) * N + c];
+            x[i] = (j == own) ? d[((size_t)b * level + t) * N + cs] : ext[(((size_t)b * beta + j) * rows + t) * N + cs];
         }
     };
     if (pcs[pt].q < FESC_FP_LIMIT) {
@@ -350,11 +352,9 @@ __global__ void __launch_bounds__(256) k_moddown_finish(const u64* __restrict__ 
     *o = v;
 }
 
-// Hybrid key switch of `batch` polynomials d[b] ([level][N], EVAL, contiguous) with scratch
-// dcoef (a copy of d, consumed), ext, acc, u.  Result is ADDED to out[b][p] when bit p of
-// add_mask is set, else stored.
-static int key_switch_chunk(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint32_t level, uint32_t batch,
-                            u64* out, size_t out_stride, int add_mask, cudaStream_t st) {
+// Steps 1-3 of the key switch: ws.dcoef -> COEFF, digit-wise basis extension into ws.ext, NTT of the
+// converted rows.  The result (ws.d, ws.ext) can serve several keys (hoisted rotations).
+static int ks_decompose(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint32_t batch, cudaStream_t st) {
     const uint32_t N = ctx->N, K = ctx->n_p, nq = ctx->n_q, alpha = ctx->alpha;
     const uint32_t beta = (level + alpha - 1) / alpha, rows = level + K;
     const uint32_t gx = (N + 255) / 256;
@@ -385,17 +385,33 @@ static int key_switch_chunk(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& k
             m.prime[j * rows + t] = own ? 0xFF : (uint8_t)(t < level ? t : nq + (t - level));
         }
     if ((rc = ntt_launch(ctx, ws.ext, (size_t)batch * beta * rows, m, false, st)) != FESC_OK) return rc;
+    FESC_CHECK_CUDA(ctx, cudaGetLastError());
+    return FESC_OK;
+}
+
+// Steps 4-5: inner product with `key` (digits read through the Galois permutation of g when g != 0) and
+// division by P; the result is ADDED to out[b][p] when bit p of add_mask is set, else stored.
+static int ks_apply(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint32_t level, uint32_t batch, u64* out,
+                    size_t out_stride, int add_mask, cudaStream_t st, u64 g) {
+    const uint32_t N = ctx->N, K = ctx->n_p, nq = ctx->n_q, alpha = ctx->alpha;
+    const uint32_t beta = (level + alpha - 1) / alpha, rows = level + K;
+    const uint32_t gx = (N + 255) / 256;
+    int rc;
+    RowMap m;
     // 4. inner product with the key
     prof_begin(ctx, PF_INNER, st);
     if (batch >= 4) {
-        dim3 g(gx, rows, (batch + 3) / 4);
-        k_inner<4><<<g, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch);
+        dim3 gd(gx, rows, (batch + 3) / 4);
+        k_inner<4><<<gd, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch,
+                                       ctx->log_n, g);
     } else if (batch >= 2) {
-        dim3 g(gx, rows, (batch + 1) / 2);
-        k_inner<2><<<g, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch);
+        dim3 gd(gx, rows, (batch + 1) / 2);
+        k_inner<2><<<gd, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch,
+                                       ctx->log_n, g);
     } else {
-        dim3 g(gx, rows, 1);
-        k_inner<1><<<g, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch);
+        dim3 gd(gx, rows, 1);
+        k_inner<1><<<gd, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch,
+                                       ctx->log_n, g);
     }
     prof_end(ctx, PF_INNER, st);
     // 5. division by P
@@ -415,6 +431,15 @@ static int key_switch_chunk(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& k
     FESC_CHECK_CUDA(ctx, cudaGetLastError());
     ctx->counters[1] += batch;
     return FESC_OK;
+}
+
+// Hybrid key switch of `batch` polynomials d[b] ([level][N], EVAL, contiguous) with scratch
+// dcoef (a copy of d, consumed), ext, acc, u.
+static int key_switch_chunk(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint32_t level, uint32_t batch,
+                            u64* out, size_t out_stride, int add_mask, cudaStream_t st) {
+    int rc = ks_decompose(ctx, ws, level, batch, st);
+    if (rc != FESC_OK) return rc;
+    return ks_apply(ctx, ws, key, level, batch, out, out_stride, add_mask, st, 0);
 }
 
 size_t ks_scratch_words(const fesc_ctx* ctx, uint32_t level, uint32_t chunk) {
@@ -459,6 +484,70 @@ int rotate_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, si
         if (rc != FESC_OK) return rc;
     }
     return FESC_OK;
+}
+
+// c0 of every ciphertext through the Galois permutation into out[b][0]; with g == 0, c1 copied to d and dcoef
+__global__ void __launch_bounds__(256) k_hoist_prepare(const u64* __restrict__ in, size_t in_stride, u64* __restrict__ out0,
+                                                       size_t out_stride, u64* __restrict__ d, u64* __restrict__ dcoef,
+                                                       uint32_t log_n, uint32_t level, u64 g) {
+    const uint32_t N = 1u << log_n;
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t l = blockIdx.y, b = blockIdx.z;
+    if (t >= N) return;
+    const u64* ib = in + (size_t)b * in_stride;
+    if (g) {
+        out0[(size_t)b * out_stride + (size_t)l * N + t] = ib[(size_t)l * N + galois_src(t, log_n, g)];
+    } else {
+        const u64 v = ib[((size_t)level + l) * N + t];
+        const size_t o = ((size_t)b * level + l) * N + t;
+        d[o] = v;
+        dcoef[o] = v;
+    }
+}
+
+// Hoisted rotations: every ciphertext of the batch is decomposed once and rotated by each of the n_keys
+// keys.  Output k of ciphertext b goes to out + k*key_stride + b*out_stride.
+int rotate_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, size_t out_stride,
+                            size_t key_stride, uint32_t batch, uint32_t level, const uint32_t* key_ids, uint32_t n_keys,
+                            u64* scratch, cudaStream_t st) {
+    for (uint32_t k = 0; k < n_keys; k++)
+        if (!ctx->keys.count(key_ids[k]) || key_ids[k] == FESC_RELIN_KEY_ID)
+            return fesc_fail(ctx, FESC_ENOKEY, "rotate_hoisted: no Galois key " + std::to_string(key_ids[k]));
+    const uint32_t chunk = ks_chunk(ctx, batch);
+    KsScratch ws = ks_scratch_carve(ctx, scratch, level, chunk);
+    for (uint32_t b0 = 0; b0 < batch; b0 += chunk) {
+        const uint32_t nb = batch - b0 < chunk ? batch - b0 : chunk;
+        dim3 g((ctx->N + 255) / 256, level, nb);
+        const u64* ib = in + (size_t)b0 * in_stride;
+        prof_begin(ctx, PF_AUTOM, st);
+        k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, nullptr, 0, ws.d, ws.dcoef, ctx->log_n, level, 0);
+        prof_end(ctx, PF_AUTOM, st);
+        int rc = ks_decompose(ctx, ws, level, nb, st);
+        if (rc != FESC_OK) return rc;
+        for (uint32_t k = 0; k < n_keys; k++) {
+            const EvalKey& key = ctx->keys[key_ids[k]];
+            u64* ob = out + (size_t)k * key_stride + (size_t)b0 * out_stride;
+            prof_begin(ctx, PF_AUTOM, st);
+            k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, ob, out_stride, nullptr, nullptr, ctx->log_n, level, key.g);
+            prof_end(ctx, PF_AUTOM, st);
+            rc = ks_apply(ctx, ws, key, level, nb, ob, out_stride, 1, st, key.g);
+            if (rc != FESC_OK) return rc;
+        }
+    }
+    return FESC_OK;
+}
+
+extern "C" int fesc_rotate_hoisted(fesc_ctx* ctx, const uint64_t* d_in, uint64_t* d_out, uint32_t batch,
+                                   uint32_t n_limbs, const uint32_t* key_ids, uint32_t n_keys, void* stream) {
+    if (!ctx || !d_in || !d_out || (!key_ids && n_keys)) return FESC_EINVAL;
+    if (n_limbs == 0 || n_limbs > ctx->n_q) return fesc_fail(ctx, FESC_ELEVEL, "rotate_hoisted: level out of range");
+    if (batch == 0 || n_keys == 0) return FESC_OK;
+    u64* scratch;
+    int rc = ctx_scratch(ctx, ks_scratch_words(ctx, n_limbs, ks_chunk(ctx, batch)) * sizeof(u64), &scratch);
+    if (rc != FESC_OK) return rc;
+    const size_t stride = (size_t)2 * n_limbs * ctx->N;
+    return rotate_hoisted_internal(ctx, (const u64*)d_in, stride, (u64*)d_out, stride, (size_t)batch * stride, batch,
+                                   n_limbs, key_ids, n_keys, scratch, (cudaStream_t)stream);
 }
 
 extern "C" int fesc_rotate(fesc_ctx* ctx, const uint64_t* d_in, uint64_t* d_out, uint32_t batch, uint32_t n_limbs,

@@ -17,6 +17,9 @@ uint32_t ks_chunk(const fesc_ctx* ctx, uint32_t batch);
 
 int rotate_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, size_t out_stride, uint32_t batch,
                     uint32_t level, uint32_t key_id, u64* scratch, cudaStream_t st, int accumulate);
+int rotate_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, size_t out_stride,
+                            size_t key_stride, uint32_t batch, uint32_t level, const uint32_t* key_ids, uint32_t n_keys,
+                            u64* scratch, cudaStream_t st);
 int rescale_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, uint32_t batch, uint32_t level,
                      u64* scratch, cudaStream_t st);
 int ctmul_internal(fesc_ctx* ctx, const u64* a, size_t a_stride, const u64* b, size_t b_stride, u64* out,

@@ -35,12 +35,12 @@ def _setup(pair, T, C, n1, n2, tokens, d_in, d_out, level, scale, wscale=1.0, ke
     return X, W, cts, diags, (gin, nout, tbs)
 
 
-def _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=1000):
+def _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=1000, hoist=0):
     import torch
     import paper_2608_17442_b200 as fesc
 
     gin, nout, tbs = dims
-    desc = fesc.BsgsDesc(n1, n2, gin, nout, tbs, level, key_base, key_base + 500)
+    desc = fesc.BsgsDesc(n1, n2, gin, nout, tbs, level, key_base, key_base + 500, hoist)
     out = torch.empty((tbs, nout, 2, level - 1, cts.shape[-1]), dtype=torch.int64, device="cuda")
     ctx.linear(to_dev(cts), to_dev(diags), desc, out)
     return to_host(out)
@@ -59,7 +59,18 @@ def test_linear_small_ring(shape):
     want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)},
                       {g: kb + 500 + g for g in range(1, n2)})
     assert np.array_equal(got, want)
+    # hoisted baby rotations: other residues (own oracle mode), same values
+    got_h = _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=kb, hoist=1)
+    want_h = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)},
+                        {g: kb + 500 + g for g in range(1, n2)}, hoist=True)
+    assert np.array_equal(got_h, want_h)
+    assert n1 == 1 or not np.array_equal(got_h, got)
     gin, nout, tbs = dims
+    for tb in range(tbs):
+        for b in range(nout):
+            yh = orc.decrypt(got_h[tb, b], scale, 2).real.reshape(C, T).T
+            assert np.abs(yh[:min(T, tokens - tb * T), :min(C, d_out - b * C)]
+                          - (X @ W)[tb * T:(tb + 1) * T, b * C:(b + 1) * C]).max() < 2.0**-18
     Y = np.zeros((tbs * T, nout * C))
     for tb in range(tbs):
         for b in range(nout):

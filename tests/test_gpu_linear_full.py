@@ -14,7 +14,8 @@ from tests.gpu_util import ctx_pair, to_host
 pytestmark = pytest.mark.gpu
 
 
-def test_in_proj_full_size_sampled_against_oracle():
+@pytest.mark.parametrize("hoist", [0, 1])
+def test_in_proj_full_size_sampled_against_oracle(hoist):
     import torch
     import bench
     import paper_2608_17442_b200 as fesc
@@ -36,7 +37,7 @@ def test_in_proj_full_size_sampled_against_oracle():
     ct, diags = bench.make_inputs(p["primes"], orc.N, gin, nout, tbs, seed, torch.device("cuda"))
     out = torch.empty((tbs, nout, 2, level - 1, orc.N), dtype=torch.int64, device="cuda")
     torch.cuda.empty_cache()
-    desc = fesc.BsgsDesc(n1, n2, gin, nout, tbs, level, bench.BABY_BASE, bench.GIANT_BASE)
+    desc = fesc.BsgsDesc(n1, n2, gin, nout, tbs, level, bench.BABY_BASE, bench.GIANT_BASE, hoist)
     ctx.linear(ct, diags, desc, out)
     ctx.sync()
     # properties on every output: residues are canonical
@@ -61,5 +62,5 @@ def test_in_proj_full_size_sampled_against_oracle():
     gc.collect()
     torch.cuda.empty_cache()
     want = orc.linear(ct_s, dg_s, dict(n1=n1, n2=n2), {q: bench.BABY_BASE + q for q in range(1, n1)},
-                      {g: bench.GIANT_BASE + g for g in range(1, n2)})
+                      {g: bench.GIANT_BASE + g for g in range(1, n2)}, hoist=bool(hoist))
     assert np.array_equal(got, want[0, 0])

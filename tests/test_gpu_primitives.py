@@ -245,3 +245,23 @@ def test_workload_3_rotations_full_ring():
                 assert np.array_equal(got[i], orc.rotate(cts[i], key_id)), (i, k)
     print("workload 3: max |decrypt - shift| = 2^%.2f over 512 rotations" % np.log2(worst))
     assert worst < 2.0**-18
+
+
+@pytest.mark.parametrize("name,level,batch", [("toy", 6, 3), ("toy", 5, 2), ("small", 24, 5), ("small", 9, 2), ("full", 24, 2)])
+def test_rotate_hoisted(name, level, batch):
+    """Hoisted mode: one decomposition per ciphertext, several keys; residues equal the oracle's hoisted mode."""
+    import torch
+
+    pair = ctx_pair(name)
+    ctx, orc, _ = pair
+    rots = [(1, 51), (7, 52), (-(1 << 31), 53)]
+    for r, kid in rots:
+        add_key(pair, r, kid)
+    ct = random_ct(orc, 11, level, level, batch)
+    out = torch.empty((len(rots), batch, 2, level, orc.N), dtype=torch.int64, device="cuda")
+    ctx.rotate_hoisted(to_dev(ct), out, batch, level, [k for _, k in rots])
+    got = to_host(out)
+    for b in range(batch):
+        want = orc.rotate_hoisted(ct[b], [k for _, k in rots])
+        for k in range(len(rots)):
+            assert np.array_equal(got[k, b], want[k]), (name, level, b, k)

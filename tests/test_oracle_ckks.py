@@ -247,3 +247,26 @@ def test_tiny_workload_through_oracle():
         for kid, r in ((1, 1), (2, 5)):
             got = o.decrypt(o.rotate(pr, kid), scale * scale)
             assert np.abs(got - np.roll(z[i] * w[i], -r)).max() < 2.0**-16
+
+
+def test_hoisted_rotations_are_rotations_and_share_noise_bound(toy_oracle):
+    """The hoisted mode gives the same slot shift as `rotate`; its residues differ only by the permuted ModUp
+    overshoot, so both decrypt to the shift within the same tolerance."""
+    o = toy_oracle
+    scale = 2.0**20
+    z = S.uniform_slots(14, 0, 1, o.n)[0]
+    ct = o.encrypt(o.encode(z, scale, 6), 5)
+    for r, kid in ((1, 31), (4, 32), (-3, 33)):
+        o.add_galois_key(r, kid)
+    outs = o.rotate_hoisted(ct, [31, 32, 33])
+    for (r, kid), got in zip(((1, 31), (4, 32), (-3, 33)), outs):
+        assert np.abs(o.decrypt(got, scale) - np.roll(z, -r)).max() < 2e-4
+        plain = o.rotate(ct, kid)
+        assert got.shape == plain.shape
+        # same c1-independent part: the difference of the two results decrypts to (almost) zero
+        diff = np.stack([o.sub(got[p], plain[p], list(range(6))) for p in range(2)])
+        assert np.abs(o.decrypt(diff, scale)).max() < 2e-4
+    # at a level where the last digit is partial
+    ct5 = np.ascontiguousarray(ct[:, :5])
+    got = o.rotate_hoisted(ct5, [32])[0]
+    assert np.abs(o.decrypt(got, scale) - np.roll(z, -4)).max() < 2e-4

@@ -13,7 +13,7 @@ def _ctx(log_n):
     return Oracle(log_n, data + special, 3, 1, 3, 4242)
 
 
-def _run(o, X, W, T, C, n1, n2):
+def _run(o, X, W, T, C, n1, n2, hoist=False):
     n = o.n
     assert C * T == n and n1 * n2 == C
     tokens, d_in = X.shape
@@ -35,7 +35,8 @@ def _run(o, X, W, T, C, n1, n2):
             for g in range(gin):
                 for q in range(n1):
                     diags[b, p, g, q] = o.encode(linear_diagonal(W, b, g, p, q, T, C, n1), float(o.q[level - 1]), level)
-    out = o.linear(cts, diags, dict(n1=n1, n2=n2), {q: 100 + q for q in range(1, n1)}, {p: 200 + p for p in range(1, n2)})
+    out = o.linear(cts, diags, dict(n1=n1, n2=n2), {q: 100 + q for q in range(1, n1)}, {p: 200 + p for p in range(1, n2)},
+                   hoist=hoist)
     Y = np.zeros((tbs * T, nout * C))
     for tb in range(tbs):
         for b in range(nout):
@@ -57,6 +58,13 @@ def test_multi_block_projection(shape):
     o = _ctx(int(np.log2(T * C)) + 1)
     X, W = S.linear_inputs(12, tokens, d_in, d_out)
     Y = _run(o, X, W * 50, T, C, n1, n2)
+    assert np.abs(Y - X @ (W * 50)).max() < 1e-4
+
+
+def test_projection_with_hoisted_baby_rotations():
+    o = _ctx(7)
+    X, W = S.linear_inputs(14, 9, 19, 13)
+    Y = _run(o, X, W * 50, 8, 8, 4, 2, hoist=True)
     assert np.abs(Y - X @ (W * 50)).max() < 1e-4
 
 
