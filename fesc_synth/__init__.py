@@ -109,6 +109,18 @@ def params(name: str) -> dict:
         special = ntt_primes(60, log_n, 2, seed)
         return dict(name=name, log_n=log_n, primes=data + special, n_q=n_q, n_p=2, dnum=n_q // 2,
                     seed=seed, log_scale=40)
+    if name == "wide":
+        # 55-bit data primes: exercises the integer (non-FP64) kernels of the library
+        seed = config_seed(0)
+        data = ntt_primes(55, 10, 6, seed)
+        special = ntt_primes(60, 10, 2, seed)
+        return dict(name=name, log_n=10, primes=data + special, n_q=6, n_p=2, dnum=3, seed=seed, log_scale=40)
+    if name == "full52":
+        # N=2^16 with 52-bit data primes: the integer wide-lazy transform path
+        seed = config_seed(0)
+        data = ntt_primes(52, 16, 2, seed)
+        special = ntt_primes(60, 16, 1, seed)
+        return dict(name=name, log_n=16, primes=data + special, n_q=2, n_p=1, dnum=2, seed=seed, log_scale=40)
     raise KeyError(name)
 
 

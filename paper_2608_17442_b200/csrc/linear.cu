@@ -292,14 +292,15 @@ __global__ void __launch_bounds__(256, 2) k_bsgs_accumulate_fp_staged(
         }
 }
 
-// Tuning knob for experiments: FESC_BSGS_TILE=<TT><PT> (e.g. 24) picks the register tile.
-static int bsgs_tile() {
+// Knobs for experiments: FESC_BSGS_INT=1 selects the 128-bit integer accumulate kernel,
+// FESC_BSGS_GROUP_GIB the scratch budget that decides how many token blocks are processed per group.
+static bool bsgs_force_int() {
     static int v = -1;
     if (v < 0) {
-        const char* e = getenv("FESC_BSGS_TILE");
-        v = e ? atoi(e) : 0;
+        const char* e = getenv("FESC_BSGS_INT");
+        v = e && atoi(e) ? 1 : 0;
     }
-    return v;
+    return v == 1;
 }
 static size_t bsgs_group_bytes() {
     const char* e = getenv("FESC_BSGS_GROUP_GIB");
@@ -390,35 +391,14 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
         FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
         kern<<<grid, 256, smem, st>>>(rot, diags, acc, ctx->d_pc, N, level, nt, gin * n1, bp_count);          \
     } while (0)
-        const bool fp_ok = qbits <= 50;   // every active prime below 2^50: exact FP64 products
-        const int tile = bsgs_tile();
-        if (fp_ok && tile == 0) {
-            if (N % 256 == 0 && nt >= 2) BSGS_FPS(2, 8, 3);
-            else if (nt >= 2) BSGS_FP(2, 8);
-            else BSGS_FP(1, 8);
-        } else if (fp_ok && tile == 2028 && N % 256 == 0) {
-            BSGS_FPS(2, 8, 3);
-        } else if (fp_ok && tile == 2128 && N % 256 == 0) {
-            BSGS_FPS(2, 8, 4);
-        } else if (fp_ok && tile == 2044 && N % 256 == 0) {
-            BSGS_FPS(4, 4, 4);
-        } else if (fp_ok && tile == 1024) {
-            BSGS_FP(2, 4);
-        } else if (fp_ok && tile == 1044) {
-            BSGS_FP(4, 4);
-        } else if (fp_ok && tile == 1018) {
-            BSGS_FP(1, 8);
-        } else
-        switch (tile) {
-            case 12: BSGS(1, 2); break;
-            case 14: BSGS(1, 4); break;
-            case 18: BSGS(1, 8); break;
-            case 22: BSGS(2, 2); break;
-            case 24: BSGS(2, 4); break;
-            case 28: BSGS(2, 8); break;
-            case 44: BSGS(4, 4); break;
-            default: if (nt >= 2) BSGS(2, 8); else BSGS(1, 8); break;
-        }
+        // all active primes below 2^50: exact FP64 products (staged variant when rows split into 256-word tiles);
+        // otherwise 128-bit integer accumulation.  FESC_BSGS_INT=1 forces the integer kernel (for comparisons).
+        const bool fp_ok = qbits <= 50 && !bsgs_force_int();
+        if (fp_ok && N % 256 == 0 && nt >= 2) BSGS_FPS(2, 8, 3);
+        else if (fp_ok && nt >= 2) BSGS_FP(2, 8);
+        else if (fp_ok) BSGS_FP(1, 8);
+        else if (nt >= 2) BSGS(2, 8);
+        else BSGS(1, 8);
 #undef BSGS
         prof_end(ctx, PF_BSGS, st);
         FESC_CHECK_CUDA(ctx, cudaGetLastError());

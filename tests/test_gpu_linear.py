@@ -78,6 +78,19 @@ def test_linear_small_ring(shape):
     assert np.abs(Y[:tokens, :d_out] - X @ W).max() < 2.0**-18
 
 
+def test_linear_integer_kernels_with_55_bit_primes():
+    """The 128-bit integer accumulate kernel (primes above 50 bits) against the oracle."""
+    pair = ctx_pair("wide")
+    ctx, orc, _ = pair
+    T, C, n1, n2, level = 32, 16, 4, 4, 6
+    X, W, cts, diags, dims = _setup(pair, T, C, n1, n2, 50, 30, 20, level, 2.0**40, wscale=10.0, key_base=3000)
+    for hoist in (0, 1):
+        got = _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=3000, hoist=hoist)
+        want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: 3000 + q for q in range(1, n1)},
+                          {g: 3500 + g for g in range(1, n2)}, hoist=bool(hoist))
+        assert np.array_equal(got, want)
+
+
 def test_linear_full_ring_one_block():
     """N = 2^16, 24 limbs, scale 2^40: one token block x one output block of the in_proj shape
     (768 inputs = 3 input blocks, C=256, T=128, n1=32, n2=8); bit-exact and within 2^-18 of X @ W."""

@@ -265,3 +265,46 @@ def test_rotate_hoisted(name, level, batch):
         want = orc.rotate_hoisted(ct[b], [k for _, k in rots])
         for k in range(len(rots)):
             assert np.array_equal(got[k, b], want[k]), (name, level, b, k)
+
+
+def test_integer_paths_with_primes_above_50_bits():
+    """Primes of 52 and 55 bits take the integer kernels (wide-lazy transform at N = 2^16, 128-bit lazy
+    accumulation in ModUp / inner product / ModDown); same bit-exact bar."""
+    import torch
+
+    ctx, orc, p = ctx_pair("full52")
+    a = np.stack([S.uniform_residues_np(21, i, [orc.q[i]], orc.N)[0] for i in range(3)])[None]
+    d = to_dev(a)
+    ctx.ntt(d, 1, 0, 3)
+    assert np.array_equal(to_host(d)[0], orc.ntt(a[0], [0, 1, 2]))
+    ctx.intt(d, 1, 0, 3)
+    assert np.array_equal(to_host(d), a)
+    d = to_dev(a)
+    ctx.intt(d, 1, 0, 3)
+    assert np.array_equal(to_host(d)[0], orc.intt(a[0], [0, 1, 2]))
+    pair = ctx_pair("wide")
+    ctx, orc, p = pair
+    add_key(pair, 3, 61)
+    add_key(pair, 9, 62)
+    for level in (6, 5, 2):
+        ct = random_ct(orc, 22, level, level, 3)
+        out = torch.empty_like(to_dev(ct))
+        ctx.rotate(to_dev(ct), out, 3, level, 61)
+        got = to_host(out)
+        for b in range(3):
+            assert np.array_equal(got[b], orc.rotate(ct[b], 61))
+        hout = torch.empty((2, 3, 2, level, orc.N), dtype=torch.int64, device="cuda")
+        ctx.rotate_hoisted(to_dev(ct), hout, 3, level, [61, 62])
+        for b in range(3):
+            want = orc.rotate_hoisted(ct[b], [61, 62])
+            assert np.array_equal(to_host(hout)[0, b], want[0]) and np.array_equal(to_host(hout)[1, b], want[1])
+        ct2 = random_ct(orc, 23, level, level, 3)
+        ctx.ct_ct_mul(to_dev(ct), to_dev(ct2), out, 3, level)
+        got = to_host(out)
+        for b in range(3):
+            assert np.array_equal(got[b], orc.ct_ct_mul(ct[b], ct2[b]))
+        if level >= 2:
+            res = torch.empty((3, 2, level - 1, orc.N), dtype=torch.int64, device="cuda")
+            ctx.rescale(to_dev(ct), res, 3, level)
+            for b in range(3):
+                assert np.array_equal(to_host(res)[b], orc.rescale(ct[b]))
