@@ -257,7 +257,7 @@ def run_ours(args):
         ctx.add_galois_key(g * N1 * T_SEG, GIANT_BASE + g)
     gin, nout, tbs = workload_dims(args.scale_down)
     if args.profile_case:       # small case for profiler captures: a few GB on the device
-        gin, nout, tbs = 1, 1, 2
+        gin, nout, tbs = 1, 1, 4
     ks_per_step = key_switches_per_step(gin, nout, tbs)
     ct, diags = make_inputs(p["primes"], n, gin, nout, tbs, S.config_seed(4) + rank, dev)
     out = torch.empty((tbs, nout, 2, LEVEL - 1, n), dtype=torch.int64, device=dev)

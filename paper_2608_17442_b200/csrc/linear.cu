@@ -2,11 +2,13 @@
 //
 // Per group of token blocks: (1) baby rotations of every input ciphertext, batched per rotation
 // amount so a key is streamed once per batch; (2) one fused accumulate kernel that forms every
-// giant-step accumulator acc[tb][b][p] = sum_{g,q} rot[tb][g][q] (.) D[b][p][g][q] with 128-bit
-// lazy sums in registers, tiled TT token blocks x PT (b,p) pairs per thread so a rotated
+// giant-step accumulator acc[tb][b][p] = sum_{g,q} rot[tb][g][q] (.) D[b][p][g][q] exactly in
+// registers (mixed integer/FP64 sums for primes below 2^50, exact FP64 products, or 128-bit lazy
+// integer sums), tiled TT token blocks x PT (b,p) pairs per thread so a rotated
 // ciphertext word is reused PT times and a diagonal word TT times; (3) giant rotations that
 // accumulate straight into acc[tb][b][0]; (4) rescale into the output.
 #include <stdlib.h>
+#include <string.h>
 
 #include "ops.cuh"
 
@@ -198,6 +200,9 @@ __device__ __forceinline__ void cp_async8(void* smem_dst, const void* gmem_src) 
     asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
                  : "memory");
 }
+__device__ __forceinline__ void cp_async8s(uint32_t smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N_>
 __device__ __forceinline__ void cp_async_wait() {
@@ -205,7 +210,7 @@ __device__ __forceinline__ void cp_async_wait() {
 }
 
 template <int TT, int PT, int STAGES>
-__global__ void __launch_bounds__(256, 2) k_bsgs_accumulate_fp_staged(
+__global__ void __launch_bounds__(256, (TT * PT > 16 ? 1 : 2)) k_bsgs_accumulate_fp_staged(
     const u64* __restrict__ rot, const u64* __restrict__ diags, u64* __restrict__ acc,
     const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level, uint32_t tbs, uint32_t terms, uint32_t bp_count) {
     constexpr int ROWS = 2 * TT + PT;
@@ -292,19 +297,137 @@ __global__ void __launch_bounds__(256, 2) k_bsgs_accumulate_fp_staged(
         }
 }
 
-// Knobs for experiments: FESC_BSGS_INT=1 selects the 128-bit integer accumulate kernel,
-// FESC_BSGS_GROUP_GIB the scratch budget that decides how many token blocks are processed per group.
-static bool bsgs_force_int() {
+// Mixed-pipe exact accumulation for primes below 2^50 (at most 256 terms).  The sum S = sum_t x_t w_t
+// (below 2^108) is tracked twice: its low 64 bits exactly on the integer multiplier pipe (one 32x32+64 and two
+// 32-bit multiply-adds per term), and its magnitude approximately on the FP64 pipe (ONE fused multiply-add per
+// term; every rounding is below 2^53, so 256 terms stay within 2^61 of S).  S is then the unique integer that is
+// congruent to the low part modulo 2^64 and within 2^63 of the approximation; one 128-bit reduction follows.
+// Per term that is 8 multiplier-pipe cycles and 2 FP64-pipe cycles per warp, on pipes that run concurrently,
+// instead of 6 FP64 operations and a rounding.
+template <int TT, int PT, int STAGES>
+__global__ void __launch_bounds__(256, (TT * PT >= 12 ? 1 : 2)) k_bsgs_accumulate_mixed(
+    const u64* __restrict__ rot, const u64* __restrict__ diags, u64* __restrict__ acc,
+    const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level, uint32_t tbs, uint32_t terms, uint32_t bp_count) {
+    constexpr int ROWS = 2 * TT + PT;
+    extern __shared__ __align__(16) u64 stage[];          // [STAGES][ROWS][256]
+    const uint32_t tid = threadIdx.x;
+    const uint32_t c = blockIdx.y * 256 + tid;
+    const uint32_t l = blockIdx.z % level;
+    const uint32_t tb0 = (blockIdx.z / level) * TT, bp0 = blockIdx.x * PT;
+    const PrimeConst pc = pcs[l];
+    const size_t poly = (size_t)level * N, ctw = 2 * poly;
+    const size_t o = (size_t)l * N + c;
+    // one running pointer per operand; the rows of a stage sit at block-uniform offsets from it
+    size_t xoff[TT], doff[PT];
+#pragma unroll
+    for (int i = 0; i < TT; i++) xoff[i] = (size_t)(tb0 + i < tbs ? tb0 + i : tbs - 1) * terms * ctw;
+#pragma unroll
+    for (int j = 0; j < PT; j++) doff[j] = (size_t)(bp0 + j < bp_count ? bp0 + j : bp_count - 1) * terms * poly;
+    const u64* xrun = rot + o;
+    const u64* drun = diags + o;
+    uint32_t slot = 0;                                     // stage that the next issue fills
+    const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(stage) + tid * 8;
+    auto issue = [&]() {
+        const uint32_t dst = sbase + slot * (ROWS * 2048);
+#pragma unroll
+        for (int i = 0; i < TT; i++) {
+            cp_async8s(dst + (2 * i) * 2048, xrun + xoff[i]);
+            cp_async8s(dst + (2 * i + 1) * 2048, xrun + xoff[i] + poly);
+        }
+#pragma unroll
+        for (int j = 0; j < PT; j++) cp_async8s(dst + (2 * TT + j) * 2048, drun + doff[j]);
+        xrun += ctw;
+        drun += poly;
+        slot = slot + 1 == STAGES ? 0 : slot + 1;
+    };
+    for (uint32_t t = 0; t < STAGES - 1; t++) {
+        if (t < terms) issue();
+        cp_async_commit();
+    }
+    u64 lo[TT][PT][2];        // S mod 2^64 (low product word accumulated with wrap-around)
+    uint32_t hi[TT][PT][2];   // cross terms, weight 2^32, modulo 2^32
+    double ap[TT][PT][2];     // S approximately
+#pragma unroll
+    for (int i = 0; i < TT; i++)
+#pragma unroll
+        for (int j = 0; j < PT; j++)
+#pragma unroll
+            for (int p = 0; p < 2; p++) lo[i][j][p] = 0, hi[i][j][p] = 0, ap[i][j][p] = 0.0;
+    uint32_t rslot = 0;                                    // stage that the next term reads
+#pragma unroll 1
+    for (uint32_t t = 0; t < terms; t++) {
+        if (t + STAGES - 1 < terms) issue();
+        cp_async_commit();
+        cp_async_wait<STAGES - 1>();
+        const u64* sm = stage + (size_t)rslot * ROWS * 256 + tid;
+        rslot = rslot + 1 == STAGES ? 0 : rslot + 1;
+        uint32_t x0[TT][2], x1[TT][2];
+        double xd[TT][2];
+#pragma unroll
+        for (int i = 0; i < TT; i++)
+#pragma unroll
+            for (int p = 0; p < 2; p++) {
+                const u64 v = sm[(2 * i + p) * 256];
+                x0[i][p] = (uint32_t)v;
+                x1[i][p] = (uint32_t)(v >> 32);
+                xd[i][p] = __ull2double_rn(v);       // exact: v < 2^50
+            }
+#pragma unroll
+        for (int j = 0; j < PT; j++) {
+            const u64 v = sm[(2 * TT + j) * 256];
+            const uint32_t w0 = (uint32_t)v, w1 = (uint32_t)(v >> 32);
+            const double wd = __ull2double_rn(v);
+#pragma unroll
+            for (int i = 0; i < TT; i++)
+#pragma unroll
+                for (int p = 0; p < 2; p++) {
+                    asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(lo[i][j][p]) : "r"(x0[i][p]), "r"(w0));
+                    asm("mad.lo.u32 %0, %1, %2, %0;" : "+r"(hi[i][j][p]) : "r"(x1[i][p]), "r"(w0));
+                    asm("mad.lo.u32 %0, %1, %2, %0;" : "+r"(hi[i][j][p]) : "r"(x0[i][p]), "r"(w1));
+                    ap[i][j][p] = __fma_rn(xd[i][p], wd, ap[i][j][p]);
+                }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < TT; i++)
+#pragma unroll
+        for (int j = 0; j < PT; j++) {
+            const uint32_t tb = tb0 + i, bp = bp0 + j;
+            if (tb < tbs && bp < bp_count) {
+                u64* dst = acc + ((size_t)tb * bp_count + bp) * ctw;
+#pragma unroll
+                for (int p = 0; p < 2; p++) {
+                    const u64 low = lo[i][j][p] + ((u64)hi[i][j][p] << 32);
+                    // the high word of S: round((approximation - low) / 2^64)
+                    const double k = rint((ap[i][j][p] - __ull2double_rn(low)) * 5.421010862427522e-20);
+                    dst[p * poly + o] = reduce128((u64)__double2ll_rn(k), low, pc);
+                }
+            }
+        }
+}
+
+// Knobs for experiments.  FESC_BSGS_KERNEL picks the accumulate kernel: "int" the 128-bit integer one, "fp" the
+// exact-FP64 one, anything else the default (mixed-pipe where it applies).  FESC_BSGS_GROUP_GIB fixes the scratch
+// budget that decides how many token blocks are processed per group (default: from the free device memory).
+static int bsgs_kernel() {
     static int v = -1;
     if (v < 0) {
-        const char* e = getenv("FESC_BSGS_INT");
-        v = e && atoi(e) ? 1 : 0;
+        const char* e = getenv("FESC_BSGS_KERNEL");
+        v = !e ? 0 : (!strcmp(e, "int") ? 2 : (!strcmp(e, "fp") ? 1 : 0));
     }
-    return v == 1;
+    return v;
 }
-static size_t bsgs_group_bytes() {
+// Larger groups re-read the diagonals less often and give the key-switch kernels larger batches; every token block
+// of a group needs its rotated inputs and its partial sums resident.  Budget: 60% of what is free (counting the
+// scratch arena the context already holds), between 2 and 24 GiB.
+static size_t bsgs_group_bytes(fesc_ctx* ctx) {
     const char* e = getenv("FESC_BSGS_GROUP_GIB");
-    return (size_t)(e ? atoi(e) : 12) << 30;
+    if (e && atoi(e) > 0) return (size_t)atoi(e) << 30;
+    size_t free_b = 0, total_b = 0;
+    if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) return (size_t)12 << 30;
+    size_t budget = (free_b + ctx->scratch_bytes) / 10 * 6;
+    const size_t lo = (size_t)2 << 30, hi = (size_t)24 << 30;
+    return budget < lo ? lo : (budget > hi ? hi : budget);
 }
 
 extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_t* d_diags, const fesc_bsgs_desc* desc,
@@ -322,9 +445,9 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
             return fesc_fail(ctx, FESC_ENOKEY, "linear: missing giant-step key " + std::to_string(desc->giant_key_base + p));
     cudaStream_t st = (cudaStream_t)stream;
     const size_t ctw = (size_t)2 * level * N;
-    // token blocks per group: keep the group's buffers near 12 GiB
+    // token blocks per group, from the scratch budget
     const size_t per_tb = ((size_t)gin * n1 + (size_t)nout * n2) * ctw * sizeof(u64);
-    uint32_t tbg = (uint32_t)(bsgs_group_bytes() / per_tb);
+    uint32_t tbg = (uint32_t)(bsgs_group_bytes(ctx) / per_tb);
     if (tbg < 1) tbg = 1;
     if (tbg > tbs) tbg = tbs;
     const uint32_t max_batch = tbg * (gin > nout ? gin : nout);
@@ -393,8 +516,18 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
     } while (0)
         // all active primes below 2^50: exact FP64 products (staged variant when rows split into 256-word tiles);
         // otherwise 128-bit integer accumulation.  FESC_BSGS_INT=1 forces the integer kernel (for comparisons).
-        const bool fp_ok = qbits <= 50 && !bsgs_force_int();
-        if (fp_ok && N % 256 == 0 && nt >= 2) BSGS_FPS(2, 8, 3);
+#define BSGS_MIX(TT, PT, ST)                                                                                  \
+    do {                                                                                                      \
+        dim3 grid((bp_count + PT - 1) / PT, N / 256, level * ((nt + TT - 1) / TT));                           \
+        if (grid.z > 65535) return fesc_fail(ctx, FESC_EINVAL, "linear: too many accumulator tiles");         \
+        const size_t smem = (size_t)ST * (2 * TT + PT) * 2048;                                                \
+        auto kern = k_bsgs_accumulate_mixed<TT, PT, ST>;                                                      \
+        FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        kern<<<grid, 256, smem, st>>>(rot, diags, acc, ctx->d_pc, N, level, nt, gin * n1, bp_count);          \
+    } while (0)
+        const bool fp_ok = qbits <= 50 && bsgs_kernel() != 2;
+        if (fp_ok && bsgs_kernel() == 0 && N % 256 == 0 && nt >= 2 && gin * n1 <= 256) BSGS_MIX(2, 8, 3);
+        else if (fp_ok && N % 256 == 0 && nt >= 2) BSGS_FPS(2, 8, 3);
         else if (fp_ok && nt >= 2) BSGS_FP(2, 8);
         else if (fp_ok) BSGS_FP(1, 8);
         else if (nt >= 2) BSGS(2, 8);
