@@ -78,6 +78,30 @@ def test_linear_small_ring(shape):
     assert np.abs(Y[:tokens, :d_out] - X @ W).max() < 2.0**-18
 
 
+def test_linear_accumulate_extreme_residues_256_terms():
+    """Worst case for the mixed integer/FP64 sums: 256 terms per accumulator, every residue q-1 (largest products,
+    largest rounding of the FP64 magnitude) in one half of the data and uniform residues in the other."""
+    pair = ctx_pair("small")
+    ctx, orc, p = pair
+    T, C, n1, n2, level = 32, 16, 16, 1, 4
+    gin, nout, tbs = 16, 2, 3
+    kb = 5000
+    for q in range(1, n1):
+        add_key(pair, q * T, kb + q)
+    qs = np.array(orc.q[:level], dtype=np.uint64)
+    primes = [int(x) for x in qs]
+    cts = np.stack([S.uniform_residues_np(p["seed"] + 91, i, primes, orc.N)
+                    for i in range(tbs * gin * 2)]).reshape(tbs, gin, 2, level, orc.N)
+    diags = np.stack([S.uniform_residues_np(p["seed"] + 92, i, primes, orc.N)
+                      for i in range(nout * n2 * gin * n1)]).reshape(nout, n2, gin, n1, level, orc.N)
+    cts[:, :, :, :, : orc.N // 2] = (qs - 1)[None, None, None, :, None]
+    diags[:, :, :, :, :, : orc.N // 2] = (qs - 1)[None, None, None, None, :, None]
+    for hoist in (0, 1):
+        got = _run_gpu(ctx, cts, diags, n1, n2, (gin, nout, tbs), level, key_base=kb, hoist=hoist)
+        want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)}, {}, hoist=bool(hoist))
+        assert np.array_equal(got, want)
+
+
 def test_linear_integer_kernels_with_55_bit_primes():
     """The 128-bit integer accumulate kernel (primes above 50 bits) against the oracle."""
     pair = ctx_pair("wide")
