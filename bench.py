@@ -177,7 +177,7 @@ INT_LIMB_SHARE = 32.0 / 224.0     # transforms on the 60-bit special primes per 
 # ---------------------------------------------------------------------------------------------
 # reference arm and CPU baseline: the oracle, timed as it stands on a bounded sample
 # ---------------------------------------------------------------------------------------------
-def oracle_sample(steps: int, warmup: int):
+def oracle_sample(steps: int, warmup: int, hoist: bool = True, defer: bool = True):
     """One token block x one output block x ONE input block of the projection through the
     oracle: 31 baby + 7 giant rotations, 256 MACs, 1 rescale.  Returns (key-switches/s, ms/step, cores)."""
     import numpy as np
@@ -202,10 +202,10 @@ def oracle_sample(steps: int, warmup: int):
     bk = {q: BABY_BASE + q for q in range(1, N1)}
     gk = {g: GIANT_BASE + g for g in range(1, N2)}
     for _ in range(warmup):
-        orc.linear(ct, diags, desc, bk, gk)
+        orc.linear(ct, diags, desc, bk, gk, hoist=hoist, defer=defer)
     t0 = time.perf_counter()
     for _ in range(max(1, steps)):
-        orc.linear(ct, diags, desc, bk, gk)
+        orc.linear(ct, diags, desc, bk, gk, hoist=hoist, defer=defer)
     dt = (time.perf_counter() - t0) / max(1, steps)
     ks = (N1 - 1) + (N2 - 1)
     cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
@@ -220,7 +220,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    value, ms, cores = oracle_sample(args.steps, min(args.warmup, 1))
+    value, ms, cores = oracle_sample(args.steps, min(args.warmup, 1), bool(args.hoist), bool(args.defer))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "key-switches/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": ms,
@@ -262,7 +262,7 @@ def run_ours(args):
     ct, diags = make_inputs(p["primes"], n, gin, nout, tbs, S.config_seed(4) + rank, dev)
     out = torch.empty((tbs, nout, 2, LEVEL - 1, n), dtype=torch.int64, device=dev)
     torch.cuda.empty_cache()
-    desc = fesc.BsgsDesc(N1, N2, gin, nout, tbs, LEVEL, BABY_BASE, GIANT_BASE, int(args.hoist))
+    desc = fesc.BsgsDesc(N1, N2, gin, nout, tbs, LEVEL, BABY_BASE, GIANT_BASE, int(args.hoist), int(args.defer))
 
     def step():
         ctx.linear(ct, diags, desc, out)
@@ -374,7 +374,8 @@ def run_ours(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
         "config": {"workload": "in_proj 768->3352, L=2048 tokens, N=2^16, 24x50-bit limbs + 4x60-bit special primes, "
                                "6 key-switch digits, C=256 T=128 n1=32 n2=8, baby rotations %s"
-                               % ("hoisted (one decomposition per input ciphertext)" if args.hoist else "by plain rotations"),
+                               % ("hoisted (one decomposition per input ciphertext)" if args.hoist else "by plain rotations")
+                               + (", one division by P per output for the giant-step sum" if args.defer else ""),
                    "input_cts": tbs * gin, "diagonals": nout * N2 * gin * N1, "output_cts": tbs * nout,
                    "key_switches_per_step": ks_per_step, "macs_per_step": tbs * nout * N2 * gin * N1,
                    "l2": "inputs larger than L2 (diagonals %.1f GiB stream every step)" % (diags.numel() * 8 / 2**30),
@@ -385,7 +386,7 @@ def run_ours(args):
     if args.scale_down > 1:
         line["config"]["workload"] += " [DEBUG scale_down=%d: not a reportable number]" % args.scale_down
     if rank == 0 and world == 1 and not args.no_cpu:
-        v, ms, cores = oracle_sample(1, 0)
+        v, ms, cores = oracle_sample(1, 0, bool(args.hoist), bool(args.defer))
         line["cpu_baseline"] = {"value": v, "unit": "key-switches/s", "cores": cores, "kind": "oracle",
                                 "sample": SAMPLE_TEXT, "ms": ms}
     if rank == 0:
@@ -485,6 +486,8 @@ def main():
                     help="run ONE step of a small case (1 input block, 1 output block, 2 token blocks) and exit; for ncu")
     ap.add_argument("--profile-step", dest="profile_step", action="store_true",
                     help="run ONE step of the full workload without warm-up and exit; for the ncu launch list")
+    ap.add_argument("--defer", type=int, default=1, choices=[0, 1],
+                    help="1: one division by P per output for the whole giant-step sum")
     ap.add_argument("--hoist", type=int, default=1, choices=[0, 1],
                     help="1: baby rotations share one decomposition per input ciphertext (fesc_rotate_hoisted)")
     ap.add_argument("--workload", default="in_proj", choices=["in_proj", "scan_slice", "scan_layer"],

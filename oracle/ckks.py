@@ -323,7 +323,30 @@ class Oracle:
         return np.stack([self.mul(ct[p], m_eval, data) for p in range(2)])
 
     # ---- BSGS projection -----------------------------------------------------------
-    def linear(self, ct_in, diags, desc, baby_key_ids, giant_key_ids, hoist: bool = False):
+    def giant_sum_deferred(self, accs, giant_key_ids):
+        """sum_p rot(acc_p, giant step p) with ONE division by P for the whole sum (a separately defined mode):
+            y0 = acc_0[0] + sum_{p>=1} sigma_p(acc_p[0]) + ModDown( sum_{p>=1} raw_p[0] ),
+            y1 = acc_0[1]                                 + ModDown( sum_{p>=1} raw_p[1] ),
+        raw_p = the key-switch accumulators of sigma_p(acc_p[1]) on the extended basis, added limb-wise.
+        Division by P is additive up to its rounding, so the value equals the sum of the separate rotations;
+        the residues differ (one rounding instead of n2 - 1) unless there is a single giant step."""
+        level = accs[0].shape[1]
+        data = list(range(level))
+        ext = data + self.special
+        y0, y1 = _arr(accs[0][0]).copy(), _arr(accs[0][1]).copy()
+        raw = np.zeros((2, len(ext), self.N), dtype=np.uint64)
+        for p in range(1, len(accs)):
+            kid = giant_key_ids[p]
+            g = self.keys[kid][0]
+            y0 = self.add(y0, self.automorphism(accs[p][0], g, level), data)
+            r = self.key_switch_raw(self.automorphism(accs[p][1], g, level), kid, level)
+            raw = np.stack([self.add(raw[c], r[c], ext) for c in range(2)])
+        if len(accs) > 1:
+            y0 = self.add(y0, self.mod_down(raw[0], level), data)
+            y1 = self.add(y1, self.mod_down(raw[1], level), data)
+        return np.stack([y0, y1])
+
+    def linear(self, ct_in, diags, desc, baby_key_ids, giant_key_ids, hoist: bool = False, defer: bool = False):
         """Y = XW on packed ciphertexts (App. "Projection Kernel Breakdown", real packing).
 
         ct_in  [token_blocks, in_blocks, 2, l, N]
@@ -332,7 +355,8 @@ class Oracle:
           acc_p = sum_g sum_q rot(x^(g), q*T) (.) D^(b)_{g,p,q};
           y^(b) = sum_p rot(acc_p, p*n1*T);  then rescale.
         baby_key_ids[q] rotates by q*T (q >= 1), giant_key_ids[p] by p*n1*T (p >= 1).
-        hoist=True: the baby rotations use `rotate_hoisted` (different residues, same values)."""
+        hoist=True: the baby rotations use `rotate_hoisted` (different residues, same values).
+        defer=True: the giant-step sum uses `giant_sum_deferred` (one division by P per output)."""
         n1, n2 = desc["n1"], desc["n2"]
         tbs, gin = ct_in.shape[0], ct_in.shape[1]
         level = ct_in.shape[3]
@@ -347,14 +371,20 @@ class Oracle:
                         for q in range(n1)] for g in range(gin)]
             for b in range(nout):
                 y = None
+                accs = []
                 for p in range(n2):
                     acc = np.zeros((2, level, self.N), dtype=np.uint64)
                     for g in range(gin):
                         for q in range(n1):
                             acc = self.ct_pt_mac(rot[g][q], diags[b, p, g, q], acc)
+                    if defer:
+                        accs.append(acc)
+                        continue
                     if p > 0:
                         acc = self.rotate(acc, giant_key_ids[p])
                     y = acc if y is None else self.ct_add(y, acc)
+                if defer:
+                    y = self.giant_sum_deferred(accs, giant_key_ids)
                 out[tb, b] = self.rescale(y)
         return out
 

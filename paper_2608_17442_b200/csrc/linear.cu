@@ -6,7 +6,8 @@
 // registers (mixed integer/FP64 sums for primes below 2^50, exact FP64 products, or 128-bit lazy
 // integer sums), tiled TT token blocks x PT (b,p) pairs per thread so a rotated
 // ciphertext word is reused PT times and a diagonal word TT times; (3) giant rotations that
-// accumulate straight into acc[tb][b][0]; (4) rescale into the output.
+// accumulate straight into acc[tb][b][0] (optionally with one division by P for the whole sum);
+// (4) rescale into the output.
 #include <stdlib.h>
 #include <string.h>
 
@@ -536,10 +537,15 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
         prof_end(ctx, PF_BSGS, st);
         FESC_CHECK_CUDA(ctx, cudaGetLastError());
         ctx->counters[2] += (uint64_t)nt * bp_count * gin * n1;
-        for (uint32_t p = 1; p < n2; p++) {
-            rc = rotate_internal(ctx, acc + (size_t)p * ctw, (size_t)n2 * ctw, acc, (size_t)n2 * ctw, nt * nout, level,
-                                 desc->giant_key_base + p, ks, st, 1);
+        if (desc->defer) {
+            rc = giant_sum_deferred_internal(ctx, acc, n2, ctw, nt * nout, level, desc->giant_key_base, ks, st);
             if (rc != FESC_OK) return rc;
+        } else {
+            for (uint32_t p = 1; p < n2; p++) {
+                rc = rotate_internal(ctx, acc + (size_t)p * ctw, (size_t)n2 * ctw, acc, (size_t)n2 * ctw, nt * nout,
+                                     level, desc->giant_key_base + p, ks, st, 1);
+                if (rc != FESC_OK) return rc;
+            }
         }
         rc = rescale_internal(ctx, acc, (size_t)n2 * ctw, out + (size_t)tb0 * nout * 2 * (level - 1) * N, nt * nout, level,
                               ks, st);

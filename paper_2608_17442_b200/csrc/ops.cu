@@ -165,7 +165,7 @@ __global__ void __launch_bounds__(256, 2) k_inner(const u64* __restrict__ d, con
                                                const u64* __restrict__ key, u64* __restrict__ acc,
                                                const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
                                                uint32_t n_q, uint32_t K, uint32_t alpha, uint32_t beta,
-                                               uint32_t batch, uint32_t log_n, u64 g) {
+                                               uint32_t batch, uint32_t log_n, u64 g, int accumulate) {
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t t = blockIdx.y, b0 = blockIdx.z * BT;
     if (c >= N) return;
@@ -190,7 +190,14 @@ __global__ void __launch_bounds__(256, 2) k_inner(const u64* __restrict__ d, con
         const double q = pcs[pt].qd, qinv = pcs[pt].qinvd;
         double f0[BT], f1[BT];
 #pragma unroll
-        for (int i = 0; i < BT; i++) f0[i] = f1[i] = 0.0;
+        for (int i = 0; i < BT; i++) {
+            f0[i] = f1[i] = 0.0;
+            if (accumulate) {   // running sum over several keys (division by P deferred)
+                const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
+                f0[i] = fp_load(acc[(((size_t)b * 2 + 0) * rows + t) * N + c], q);
+                f1[i] = fp_load(acc[(((size_t)b * 2 + 1) * rows + t) * N + c], q);
+            }
+        }
         if (beta <= 8) {
             // all digits' words are requested before the first product, so a thread has up to
             // 8 * (2 + BT) loads in flight
@@ -266,8 +273,12 @@ __global__ void __launch_bounds__(256, 2) k_inner(const u64* __restrict__ d, con
     for (int i = 0; i < BT; i++) {
         const uint32_t b = b0 + i;
         if (b < batch) {
-            acc[(((size_t)b * 2 + 0) * rows + t) * N + c] = reduce128(a0[i].hi, a0[i].lo, pc);
-            acc[(((size_t)b * 2 + 1) * rows + t) * N + c] = reduce128(a1[i].hi, a1[i].lo, pc);
+            u64* o0 = acc + (((size_t)b * 2 + 0) * rows + t) * N + c;
+            u64* o1 = acc + (((size_t)b * 2 + 1) * rows + t) * N + c;
+            u64 r0 = reduce128(a0[i].hi, a0[i].lo, pc), r1 = reduce128(a1[i].hi, a1[i].lo, pc);
+            if (accumulate) r0 = addmod(r0, *o0, pc.q), r1 = addmod(r1, *o1, pc.q);
+            *o0 = r0;
+            *o1 = r1;
         }
     }
 }
@@ -389,32 +400,41 @@ static int ks_decompose(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint
     return FESC_OK;
 }
 
-// Steps 4-5: inner product with `key` (digits read through the Galois permutation of g when g != 0) and
-// division by P; the result is ADDED to out[b][p] when bit p of add_mask is set, else stored.
-static int ks_apply(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint32_t level, uint32_t batch, u64* out,
-                    size_t out_stride, int add_mask, cudaStream_t st, u64 g) {
+// Step 4: inner product with `key` (digits read through the Galois permutation of g when g != 0) into ws.acc;
+// accumulate != 0 adds to what ws.acc holds (sums over several keys before one division by P).
+static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint32_t level, uint32_t batch,
+                    cudaStream_t st, u64 g, int accumulate) {
     const uint32_t N = ctx->N, K = ctx->n_p, nq = ctx->n_q, alpha = ctx->alpha;
     const uint32_t beta = (level + alpha - 1) / alpha, rows = level + K;
     const uint32_t gx = (N + 255) / 256;
-    int rc;
-    RowMap m;
-    // 4. inner product with the key
     prof_begin(ctx, PF_INNER, st);
     if (batch >= 4) {
         dim3 gd(gx, rows, (batch + 3) / 4);
         k_inner<4><<<gd, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch,
-                                       ctx->log_n, g);
+                                       ctx->log_n, g, accumulate);
     } else if (batch >= 2) {
         dim3 gd(gx, rows, (batch + 1) / 2);
         k_inner<2><<<gd, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch,
-                                       ctx->log_n, g);
+                                       ctx->log_n, g, accumulate);
     } else {
         dim3 gd(gx, rows, 1);
         k_inner<1><<<gd, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch,
-                                       ctx->log_n, g);
+                                       ctx->log_n, g, accumulate);
     }
     prof_end(ctx, PF_INNER, st);
-    // 5. division by P
+    FESC_CHECK_CUDA(ctx, cudaGetLastError());
+    ctx->counters[1] += batch;
+    return FESC_OK;
+}
+
+// Step 5: division of ws.acc by P; the result is ADDED to out[b][p] when bit p of add_mask is set, else stored.
+static int ks_moddown(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint32_t batch, u64* out, size_t out_stride,
+                      int add_mask, cudaStream_t st) {
+    const uint32_t N = ctx->N, K = ctx->n_p, nq = ctx->n_q;
+    const uint32_t rows = level + K;
+    const uint32_t gx = (N + 255) / 256;
+    int rc;
+    RowMap m;
     m.period = rows;
     for (uint32_t t = 0; t < rows; t++) m.prime[t] = t < level ? 0xFF : (uint8_t)(nq + (t - level));
     if ((rc = ntt_launch(ctx, ws.acc, (size_t)batch * 2 * rows, m, true, st)) != FESC_OK) return rc;
@@ -429,8 +449,15 @@ static int ks_apply(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint
                                                                  ctx->d_pc, N, level, K, add_mask);
     prof_end(ctx, PF_MODDOWN, st);
     FESC_CHECK_CUDA(ctx, cudaGetLastError());
-    ctx->counters[1] += batch;
     return FESC_OK;
+}
+
+// Steps 4-5 for one key.
+static int ks_apply(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint32_t level, uint32_t batch, u64* out,
+                    size_t out_stride, int add_mask, cudaStream_t st, u64 g) {
+    int rc = ks_inner(ctx, ws, key, level, batch, st, g, 0);
+    if (rc != FESC_OK) return rc;
+    return ks_moddown(ctx, ws, level, batch, out, out_stride, add_mask, st);
 }
 
 // Hybrid key switch of `batch` polynomials d[b] ([level][N], EVAL, contiguous) with scratch
@@ -460,6 +487,8 @@ KsScratch ks_scratch_carve(const fesc_ctx* ctx, u64* base, uint32_t level, uint3
 
 uint32_t ks_chunk(const fesc_ctx* ctx, uint32_t batch) {
     uint32_t c = ctx->log_n == 16 ? 8 : 64;
+    static const int e = getenv("FESC_KS_CHUNK") ? atoi(getenv("FESC_KS_CHUNK")) : 0;
+    if (e > 0) c = (uint32_t)e;
     return batch < c ? batch : c;
 }
 
@@ -503,6 +532,38 @@ __global__ void __launch_bounds__(256) k_hoist_prepare(const u64* __restrict__ i
         d[o] = v;
         dcoef[o] = v;
     }
+}
+
+// sum_p rot(acc[b][p], key n = key_base + p) for p = 1..n_terms-1 ADDED into acc[b][0], with one division by P
+// per ciphertext: the inner products of all p are summed on the extended basis first.  acc holds `batch` groups of
+// n_terms ciphertexts (ct_words each, group stride n_terms * ct_words).
+int giant_sum_deferred_internal(fesc_ctx* ctx, u64* acc, uint32_t n_terms, size_t ct_words, uint32_t batch,
+                                uint32_t level, uint32_t key_base, u64* scratch, cudaStream_t st) {
+    if (n_terms < 2) return FESC_OK;
+    for (uint32_t p = 1; p < n_terms; p++)
+        if (!ctx->keys.count(key_base + p) || key_base + p == FESC_RELIN_KEY_ID)
+            return fesc_fail(ctx, FESC_ENOKEY, "giant steps: no Galois key " + std::to_string(key_base + p));
+    const uint32_t chunk = ks_chunk(ctx, batch);
+    KsScratch ws = ks_scratch_carve(ctx, scratch, level, chunk);
+    const size_t stride = (size_t)n_terms * ct_words;
+    for (uint32_t b0 = 0; b0 < batch; b0 += chunk) {
+        const uint32_t nb = batch - b0 < chunk ? batch - b0 : chunk;
+        dim3 g((ctx->N + 255) / 256, level, nb);
+        u64* base = acc + (size_t)b0 * stride;
+        for (uint32_t p = 1; p < n_terms; p++) {
+            const EvalKey& key = ctx->keys[key_base + p];
+            prof_begin(ctx, PF_AUTOM, st);
+            k_autom_ct<<<g, 256, 0, st>>>(base + (size_t)p * ct_words, stride, base, stride, ws.d, ws.dcoef, ctx->log_n,
+                                          level, key.g, ctx->d_pc, 1);
+            prof_end(ctx, PF_AUTOM, st);
+            int rc = ks_decompose(ctx, ws, level, nb, st);
+            if (rc != FESC_OK) return rc;
+            if ((rc = ks_inner(ctx, ws, key, level, nb, st, 0, p > 1)) != FESC_OK) return rc;
+        }
+        int rc = ks_moddown(ctx, ws, level, nb, base, stride, 3, st);
+        if (rc != FESC_OK) return rc;
+    }
+    return FESC_OK;
 }
 
 // Hoisted rotations: every ciphertext of the batch is decomposed once and rotated by each of the n_keys

@@ -35,12 +35,12 @@ def _setup(pair, T, C, n1, n2, tokens, d_in, d_out, level, scale, wscale=1.0, ke
     return X, W, cts, diags, (gin, nout, tbs)
 
 
-def _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=1000, hoist=0):
+def _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=1000, hoist=0, defer=0):
     import torch
     import paper_2608_17442_b200 as fesc
 
     gin, nout, tbs = dims
-    desc = fesc.BsgsDesc(n1, n2, gin, nout, tbs, level, key_base, key_base + 500, hoist)
+    desc = fesc.BsgsDesc(n1, n2, gin, nout, tbs, level, key_base, key_base + 500, hoist, defer)
     out = torch.empty((tbs, nout, 2, level - 1, cts.shape[-1]), dtype=torch.int64, device="cuda")
     ctx.linear(to_dev(cts), to_dev(diags), desc, out)
     return to_host(out)
@@ -65,6 +65,12 @@ def test_linear_small_ring(shape):
                         {g: kb + 500 + g for g in range(1, n2)}, hoist=True)
     assert np.array_equal(got_h, want_h)
     assert n1 == 1 or not np.array_equal(got_h, got)
+    # one division by P for the whole giant-step sum (own oracle mode), alone and with hoisting
+    for hoist in (0, 1):
+        got_d = _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=kb, hoist=hoist, defer=1)
+        want_d = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)},
+                            {g: kb + 500 + g for g in range(1, n2)}, hoist=bool(hoist), defer=True)
+        assert np.array_equal(got_d, want_d)
     gin, nout, tbs = dims
     for tb in range(tbs):
         for b in range(nout):
@@ -108,10 +114,10 @@ def test_linear_integer_kernels_with_55_bit_primes():
     ctx, orc, _ = pair
     T, C, n1, n2, level = 32, 16, 4, 4, 6
     X, W, cts, diags, dims = _setup(pair, T, C, n1, n2, 50, 30, 20, level, 2.0**40, wscale=10.0, key_base=3000)
-    for hoist in (0, 1):
-        got = _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=3000, hoist=hoist)
+    for hoist, defer in ((0, 0), (1, 0), (1, 1)):
+        got = _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=3000, hoist=hoist, defer=defer)
         want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: 3000 + q for q in range(1, n1)},
-                          {g: 3500 + g for g in range(1, n2)}, hoist=bool(hoist))
+                          {g: 3500 + g for g in range(1, n2)}, hoist=bool(hoist), defer=bool(defer))
         assert np.array_equal(got, want)
 
 

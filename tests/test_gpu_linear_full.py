@@ -14,8 +14,8 @@ from tests.gpu_util import ctx_pair, to_host
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("hoist", [0, 1])
-def test_in_proj_full_size_sampled_against_oracle(hoist):
+@pytest.mark.parametrize("hoist,defer", [(0, 0), (1, 1)])
+def test_in_proj_full_size_sampled_against_oracle(hoist, defer):
     import torch
     import bench
     import paper_2608_17442_b200 as fesc
@@ -37,7 +37,7 @@ def test_in_proj_full_size_sampled_against_oracle(hoist):
     ct, diags = bench.make_inputs(p["primes"], orc.N, gin, nout, tbs, seed, torch.device("cuda"))
     out = torch.empty((tbs, nout, 2, level - 1, orc.N), dtype=torch.int64, device="cuda")
     torch.cuda.empty_cache()
-    desc = fesc.BsgsDesc(n1, n2, gin, nout, tbs, level, bench.BABY_BASE, bench.GIANT_BASE, hoist)
+    desc = fesc.BsgsDesc(n1, n2, gin, nout, tbs, level, bench.BABY_BASE, bench.GIANT_BASE, hoist, defer)
     ctx.linear(ct, diags, desc, out)
     ctx.sync()
     # properties on every output: residues are canonical
@@ -62,5 +62,5 @@ def test_in_proj_full_size_sampled_against_oracle(hoist):
     gc.collect()
     torch.cuda.empty_cache()
     want = orc.linear(ct_s, dg_s, dict(n1=n1, n2=n2), {q: bench.BABY_BASE + q for q in range(1, n1)},
-                      {g: bench.GIANT_BASE + g for g in range(1, n2)}, hoist=bool(hoist))
+                      {g: bench.GIANT_BASE + g for g in range(1, n2)}, hoist=bool(hoist), defer=bool(defer))
     assert np.array_equal(got, want[0, 0])

@@ -13,7 +13,7 @@ def _ctx(log_n):
     return Oracle(log_n, data + special, 3, 1, 3, 4242)
 
 
-def _run(o, X, W, T, C, n1, n2, hoist=False):
+def _run(o, X, W, T, C, n1, n2, hoist=False, defer=False, raw=False):
     n = o.n
     assert C * T == n and n1 * n2 == C
     tokens, d_in = X.shape
@@ -36,7 +36,9 @@ def _run(o, X, W, T, C, n1, n2, hoist=False):
                 for q in range(n1):
                     diags[b, p, g, q] = o.encode(linear_diagonal(W, b, g, p, q, T, C, n1), float(o.q[level - 1]), level)
     out = o.linear(cts, diags, dict(n1=n1, n2=n2), {q: 100 + q for q in range(1, n1)}, {p: 200 + p for p in range(1, n2)},
-                   hoist=hoist)
+                   hoist=hoist, defer=defer)
+    if raw:
+        return out
     Y = np.zeros((tbs * T, nout * C))
     for tb in range(tbs):
         for b in range(nout):
@@ -66,6 +68,49 @@ def test_projection_with_hoisted_baby_rotations():
     X, W = S.linear_inputs(14, 9, 19, 13)
     Y = _run(o, X, W * 50, 8, 8, 4, 2, hoist=True)
     assert np.abs(Y - X @ (W * 50)).max() < 1e-4
+
+
+def test_projection_with_deferred_division_in_giant_steps():
+    """One division by P per output: same values; with a single giant step the residues are those of the
+    separate rotation (the sum has one term).  (With several the sums differ by a few units before the
+    rescale, see the next test; the rescale then hides almost all of it.)"""
+    o = _ctx(7)
+    X, W = S.linear_inputs(15, 6, 20, 10)
+    for hoist in (False, True):
+        Y = _run(o, X, W * 50, 4, 16, 4, 4, hoist=hoist, defer=True)
+        assert np.abs(Y - X @ (W * 50)).max() < 1e-4
+    a = _run(o, X, W * 50, 4, 16, 8, 2, raw=True)
+    b = _run(o, X, W * 50, 4, 16, 8, 2, defer=True, raw=True)
+    assert np.array_equal(a, b)
+
+
+def test_deferred_division_is_additive_up_to_rounding():
+    """ModDown(sum raw_p) and sum ModDown(raw_p) differ by at most n2 - 1 in every coefficient (big-integer check
+    of the claim that the deferred mode computes the same ciphertext up to rounding)."""
+    from oracle.ckks import crt_lift_centered
+    o = _ctx(5)
+    level = 3
+    data = list(range(level))
+    for p in range(1, 4):
+        o.add_galois_key(p, 300 + p)
+    rng = np.random.default_rng(5)
+    accs = [np.stack([np.stack([rng.integers(0, o.q[i], o.N, dtype=np.uint64) for i in data]) for _ in range(2)])
+            for _ in range(4)]
+    keys = {p: 300 + p for p in range(1, 4)}
+    lazy = o.giant_sum_deferred(accs, keys)
+    eager = accs[0]
+    for p in range(1, 4):
+        eager = o.ct_add(eager, o.rotate(accs[p], keys[p]))
+    Q = 1
+    for i in data:
+        Q *= o.q[i]
+    seen = 0
+    for c in range(2):
+        d = o.sub(lazy[c], eager[c], data)
+        diff = crt_lift_centered(o.intt(d, data), [o.q[i] for i in data])
+        assert max(abs(int(v)) for v in diff) <= 3
+        seen += sum(1 for v in diff if int(v) != 0)
+    assert seen > 0
 
 
 def test_diagonal_formula_on_plain_slots():
