@@ -171,6 +171,11 @@ FP64_PER_CLK_PER_SM = 64          # FP64 FMAs per SM per clock (measured 63 with
 BFLY_IMAD = 20                    # integer Shoup butterfly (primes >= 2^50): 10 products of 32x32->64
 BFLY_FP64 = 8.5                   # FP64 butterfly (primes < 2^50): 5 ops product + 2 adds + 1.5 fold-back share
 MAC_FP64 = 6                      # FP64 multiply-accumulate: 5 ops exact product + 1 add
+MAC_MIXED_CYCLES = 8              # mixed-pipe multiply-accumulate: multiplier-pipe cycles per warp (one 32x32+64 = 4,
+                                  # two 32-bit multiply-adds = 2 each) on each of the 4 sub-partitions of an SM
+# DRAM bytes of ONE accumulate launch of the default workload (4 token blocks x 112 accumulators x 96 terms),
+# read + written, from the ncu capture summarised in profiles/bsgs_accumulate_mixed.md
+BSGS_TRAFFIC_4TB = 145058871040 + 11272472832
 INT_LIMB_SHARE = 32.0 / 224.0     # transforms on the 60-bit special primes per key switch (integer path)
 
 
@@ -323,9 +328,14 @@ def run_ours(args):
         macs = tb_per_launch * nout * N2 * gin * N1 * 2 * LEVEL * n          # 64x64->128 multiply-adds
         t = dom_ms * 1e-3 / max(1, dom_records)
         sm_mhz = clocks.get("sm_mhz") or 1350.0
-        alu_peak = SM_COUNT * FP64_PER_CLK_PER_SM * sm_mhz * 1e6 / MAC_FP64 / 1e12   # T modular mul-adds / s
-        roof.update({"bound": "alu", "achieved": macs / t / 1e12, "peak": alu_peak, "unit": "T modular mac/s (FP64 pipe)",
-                     "frac": macs / t / 1e12 / alu_peak, "traffic": None,
+        # the default kernel keeps the low 64 bits of every sum on the integer multiplier pipe
+        alu_peak = SM_COUNT * 4 * 32 * sm_mhz * 1e6 / MAC_MIXED_CYCLES / 1e12        # T modular mul-adds / s
+        fp64_peak = SM_COUNT * FP64_PER_CLK_PER_SM * sm_mhz * 1e6 / MAC_FP64 / 1e12
+        traffic = BSGS_TRAFFIC_4TB if (args.scale_down == 1 and abs(tb_per_launch - 4) < 1e-9) else None
+        roof.update({"bound": "alu", "achieved": macs / t / 1e12, "peak": alu_peak,
+                     "unit": "T modular mac/s (integer multiplier pipe, 8 cycles per warp-mac)",
+                     "peak_fp64_only_scheme": fp64_peak,
+                     "frac": macs / t / 1e12 / alu_peak, "traffic": traffic,
                      "hbm": {"achieved": alg / t / 1e9, "peak": hbm_peak, "unit": "GB/s", "frac": alg / t / 1e9 / hbm_peak,
                              "algorithmic_bytes_per_launch": alg}})
     elif dominant == "ntt":

@@ -313,8 +313,11 @@ __global__ void __launch_bounds__(256, (TT * PT >= 12 ? 1 : 2)) k_bsgs_accumulat
     extern __shared__ __align__(16) u64 stage[];          // [STAGES][ROWS][256]
     const uint32_t tid = threadIdx.x;
     const uint32_t c = blockIdx.y * 256 + tid;
-    const uint32_t l = blockIdx.z % level;
-    const uint32_t tb0 = (blockIdx.z / level) * TT, bp0 = blockIdx.x * PT;
+    // blockIdx.x = (b,p) tile * token-block tiles + token-block tile: CTAs that read the same diagonal rows are
+    // scheduled next to each other (the second read hits L2), and so are the (b,p) tiles that share ciphertext rows
+    const uint32_t tb_tiles = (tbs + TT - 1) / TT;
+    const uint32_t l = blockIdx.z;
+    const uint32_t tb0 = (blockIdx.x % tb_tiles) * TT, bp0 = (blockIdx.x / tb_tiles) * PT;
     const PrimeConst pc = pcs[l];
     const size_t poly = (size_t)level * N, ctw = 2 * poly;
     const size_t o = (size_t)l * N + c;
@@ -519,8 +522,7 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
         // otherwise 128-bit integer accumulation.  FESC_BSGS_INT=1 forces the integer kernel (for comparisons).
 #define BSGS_MIX(TT, PT, ST)                                                                                  \
     do {                                                                                                      \
-        dim3 grid((bp_count + PT - 1) / PT, N / 256, level * ((nt + TT - 1) / TT));                           \
-        if (grid.z > 65535) return fesc_fail(ctx, FESC_EINVAL, "linear: too many accumulator tiles");         \
+        dim3 grid(((bp_count + PT - 1) / PT) * ((nt + TT - 1) / TT), N / 256, level);                         \
         const size_t smem = (size_t)ST * (2 * TT + PT) * 2048;                                                \
         auto kern = k_bsgs_accumulate_mixed<TT, PT, ST>;                                                      \
         FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
