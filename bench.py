@@ -179,6 +179,60 @@ BSGS_TRAFFIC_4TB = 145058871040 + 11272472832
 INT_LIMB_SHARE = 32.0 / 224.0     # transforms on the 60-bit special primes per key switch (integer path)
 
 
+def isolated_kernels(ctx, fesc, torch, ct, out, hbm_peak, n):
+    """The memory-bound kernels timed alone (CUDA events / the library's family timers), untimed part of the run:
+    the plain ct-pt multiply-accumulate and one batch of 32 plain rotations by one key (key-switch inner product,
+    limb transforms)."""
+    res = {}
+    word = 8
+    batch = 32
+    x = ct.reshape(-1, 2, LEVEL, n)[:batch]                          # 32 input ciphertexts of the step
+    acc = out.reshape(-1)[: batch * 2 * LEVEL * n].view(batch, 2, LEVEL, n)
+    pt = torch.empty((batch, LEVEL, n), dtype=torch.int64, device=ct.device)
+    pt.copy_(x[:, 0])
+    acc.zero_()
+    for _ in range(3):
+        ctx.ct_pt_mac(x, pt, acc, batch, LEVEL)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 10
+    e0.record()
+    for _ in range(reps):
+        ctx.ct_pt_mac(x, pt, acc, batch, LEVEL)
+    e1.record()
+    torch.cuda.synchronize()
+    t = e0.elapsed_time(e1) * 1e-3 / reps
+    by = batch * (2 + 1 + 2 + 2) * LEVEL * n * word                  # ct, pt, acc read, acc written
+    res["ct_pt_mac"] = {"achieved": by / t / 1e9, "peak": hbm_peak, "unit": "GB/s", "frac": by / t / 1e9 / hbm_peak,
+                        "bytes_per_launch": by, "macs_per_s": batch / t,
+                        "l2": "operands of one launch 2.8 GB, larger than L2"}
+    del pt
+    # 32 rotations by one key (batches of 8 inside the library)
+    ctx.rotate(x, acc, batch, LEVEL, BABY_BASE + 1)
+    ctx.profile_enable(["ntt", "inner", "modup", "moddown", "autom"], 4096)
+    c0 = ctx.counters()
+    e0.record()
+    ctx.rotate(x, acc, batch, LEVEL, BABY_BASE + 1)
+    e1.record()
+    torch.cuda.synchronize()
+    fam = ctx.profile_read()
+    ctx.profile_enable([])
+    c1 = ctx.counters()
+    t = e0.elapsed_time(e1) * 1e-3
+    beta = ctx.num_digits
+    rows = LEVEL + ctx.n_p
+    launches = max(1, fam["inner"][1])
+    by = batch * (beta + 2) * rows * n * word + launches * beta * 2 * rows * n * word   # digits in, sums out, key per launch
+    ti = fam["inner"][0] * 1e-3
+    res["evk_inner_product"] = {"achieved": by / ti / 1e9, "peak": hbm_peak, "unit": "GB/s", "frac": by / ti / 1e9 / hbm_peak,
+                                "bytes": by, "launches": launches, "ms": fam["inner"][0]}
+    res["rotation_batch32"] = {"key_switches_per_s": batch / t, "ms": t * 1e3,
+                               "limb_transforms": c1[0] - c0[0],
+                               "limb_transforms_per_s": (c1[0] - c0[0]) / (fam["ntt"][0] * 1e-3),
+                               "family_ms": {k: round(v[0], 3) for k, v in fam.items() if v[1]}}
+    return res
+
+
 # ---------------------------------------------------------------------------------------------
 # reference arm and CPU baseline: the oracle, timed as it stands on a bounded sample
 # ---------------------------------------------------------------------------------------------
@@ -378,6 +432,8 @@ def run_ours(args):
     e2e = {"value": world * ks_per_step / (e2e_ms * 1e-3), "unit": "key-switches/s", "latency_ms": e2e_ms,
            "h2d_bytes_per_step": ct.numel() * 8, "d2h_bytes_per_step": out.numel() * 8}
 
+    isolated = isolated_kernels(ctx, fesc, torch, ct, out, hbm_peak, n) if (rank == 0 and args.scale_down == 1) else None
+
     line = {
         "metric": METRIC, "value": value, "unit": "key-switches/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "latency_ms": ms_per_step,
@@ -393,6 +449,8 @@ def run_ours(args):
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roof, "kernel_breakdown": breakdown,
     }
+    if isolated:
+        line["isolated"] = isolated
     if args.scale_down > 1:
         line["config"]["workload"] += " [DEBUG scale_down=%d: not a reportable number]" % args.scale_down
     if rank == 0 and world == 1 and not args.no_cpu:

@@ -192,6 +192,7 @@ struct fesc_ctx {
     // scratch
     u64* d_scratch;
     size_t scratch_bytes;
+    uint32_t* d_status;           // device word: non-zero after a bounded device-side wait gave up
     uint64_t counters[8];
     Profiler prof;
     std::string err;

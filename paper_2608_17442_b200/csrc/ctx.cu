@@ -313,6 +313,7 @@ extern "C" int fesc_ctx_create(fesc_ctx** out, uint32_t log_n, const uint64_t* p
     ctx->d_twf = ctx->d_itwf = nullptr;
     ctx->d_s = nullptr;
     ctx->d_scratch = nullptr;
+    ctx->d_status = nullptr;
     ctx->scratch_bytes = 0;
     memset(ctx->counters, 0, sizeof(ctx->counters));
     memset(&ctx->tabs, 0, sizeof(ctx->tabs));
@@ -374,6 +375,8 @@ extern "C" int fesc_ctx_create(fesc_ctx** out, uint32_t log_n, const uint64_t* p
     if ((rc = build_tables(ctx)) != FESC_OK) return bail(rc);
     // ---- secret key and relinearisation key ----
     if (cudaMalloc(&ctx->d_s, (size_t)np * N * sizeof(u64)) != cudaSuccess) return bail(FESC_ENOMEM);
+    if (cudaMalloc(&ctx->d_status, sizeof(uint32_t)) != cudaSuccess) return bail(FESC_ENOMEM);
+    if (cudaMemset(ctx->d_status, 0, sizeof(uint32_t)) != cudaSuccess) return bail(FESC_ECUDA);
     k_sample_small<<<(N + 255) / 256, 256>>>(ctx->d_s, ctx->d_pc, N, np, seed, make_tag(1, 0, 0, 0), 0);
     if ((rc = ntt_launch(ctx, ctx->d_s, np, all_limbs_map(ctx), false, 0)) != FESC_OK) return bail(rc);
     u64* d_s2 = nullptr;
@@ -399,6 +402,7 @@ extern "C" int fesc_ctx_destroy(fesc_ctx* ctx) {
     cudaFree(ctx->d_itwf);
     cudaFree(ctx->d_s);
     cudaFree(ctx->d_scratch);
+    cudaFree(ctx->d_status);
     free_tables(ctx);
     delete ctx;
     return FESC_OK;
@@ -410,6 +414,14 @@ extern "C" int fesc_sync(fesc_ctx* ctx, void* stream) {
     if (!ctx) return FESC_EINVAL;
     FESC_CHECK_CUDA(ctx, cudaStreamSynchronize((cudaStream_t)stream));
     FESC_CHECK_CUDA(ctx, cudaGetLastError());
+    // a kernel whose bounded wait on an asynchronous copy ran out records it here
+    uint32_t status = 0;
+    FESC_CHECK_CUDA(ctx, cudaMemcpy(&status, ctx->d_status, sizeof(status), cudaMemcpyDeviceToHost));
+    if (status) {
+        cudaMemset(ctx->d_status, 0, sizeof(uint32_t));
+        return fesc_fail(ctx, FESC_ETIMEOUT, "a device-side wait on an asynchronous copy gave up (code " +
+                                                 std::to_string(status) + "); results of that call are invalid");
+    }
     return FESC_OK;
 }
 

@@ -160,33 +160,49 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
 // One thread owns one (coefficient, modulus) and BT ciphertexts, so a key word is loaded once
 // for BT products.
 // ---------------------------------------------------------------------------------------
-template <int BT>
-__global__ void __launch_bounds__(256, 2) k_inner(const u64* __restrict__ d, const u64* __restrict__ ext,
+#ifndef INNER_MINB
+#define INNER_MINB 3
+#endif
+// PATH 0: the row's prime decides at run time; 1: the caller guarantees primes below 2^50 on rows
+// [row0, row0 + gridDim.y) (exact FP64 products only); 2: the caller sends those rows to the 128-bit integer sums.
+template <int BT, int PATH>
+__global__ void __launch_bounds__(256, (BT >= 8 ? 2 : INNER_MINB)) k_inner(const u64* __restrict__ d, const u64* __restrict__ ext,
                                                const u64* __restrict__ key, u64* __restrict__ acc,
                                                const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
                                                uint32_t n_q, uint32_t K, uint32_t alpha, uint32_t beta,
-                                               uint32_t batch, uint32_t log_n, u64 g, int accumulate) {
+                                               uint32_t batch, uint32_t log_n, u64 g, int accumulate, uint32_t row0) {
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
-    const uint32_t t = blockIdx.y, b0 = blockIdx.z * BT;
+    const uint32_t t = row0 + blockIdx.y, b0 = blockIdx.z * BT;
     if (c >= N) return;
     // hoisted rotations: the automorphism acts on the extended digits, i.e. they are read at pi_g(c)
     const uint32_t cs = g ? galois_src(c, log_n, g) : c;
     const uint32_t rows = level + K, np = n_q + K;
     const uint32_t pt = t < level ? t : n_q + (t - level);
     const uint32_t own = t < level ? t / alpha : 0xFFFFFFFFu;
-    // operand words of one digit: key (b, a) and the BT ciphertext words; clamped indices keep loads valid
-    auto load_digit = [&](uint32_t j, u64& kb, u64& ka, u64 (&x)[BT]) {
-        kb = __ldg(key + ((size_t)(2 * j) * np + pt) * N + c);
-        ka = __ldg(key + ((size_t)(2 * j + 1) * np + pt) * N + c);
+    // operand words of one digit: key (b, a) and the BT ciphertext words; clamped indices keep loads valid.
+    // All addresses are a per-thread base plus a multiple of one stride (no per-load index products).
+    const size_t kstride = (size_t)np * N, xstride = (size_t)rows * N;
+    const u64* kp = key + (size_t)pt * N + c;
+    const u64* xp[BT];
+    const u64* op[BT];
 #pragma unroll
-        for (int i = 0; i < BT; i++) {
-            const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
-            x[i] = (j == own) ? d[((size_t)b * level + t) * N + cs] : ext[(((size_t)b * beta + j) * rows + t) * N + cs];
-        }
+    for (int i = 0; i < BT; i++) {
+        const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
+        xp[i] = ext + ((size_t)b * beta * rows + t) * N + cs;
+        op[i] = d + ((size_t)b * level + (t < level ? t : 0)) * N + cs;
+    }
+    auto load_digit = [&](uint32_t j, u64& kb, u64& ka, u64 (&x)[BT]) {
+        kb = __ldg(kp + (size_t)(2 * j) * kstride);
+        ka = __ldg(kp + (size_t)(2 * j + 1) * kstride);
+#pragma unroll
+        for (int i = 0; i < BT; i++) x[i] = (j == own) ? *op[i] : xp[i][(size_t)j * xstride];
     };
-    if (pcs[pt].q < FESC_FP_LIMIT) {
-        // exact FP64 products: |x| <= q/2, key words in [0,q); up to 8 terms of at most 0.7q stay below 2^53,
-        // longer sums are folded back every 8 digits.  The next digit's words are loaded while this one is used.
+    if (PATH == 1 || (PATH == 0 && pcs[pt].q < FESC_FP_LIMIT)) {
+        // exact FP64 products: |x| <= q/2, key words in [0,q); up to 8 terms of at most 0.7q (plus a running sum
+        // of at most q/2) stay below 2^53, longer sums are folded back every 8 digits.  The next digit's words
+        // are requested before this digit's products start: 2 + BT loads in flight per thread, few registers,
+        // so that three or four CTAs per SM overlap their loads and products (measured: one digit ahead with
+        // 4 CTAs per SM moves 1.5x the bytes per second of all-digits-up-front with 2).
         const double q = pcs[pt].qd, qinv = pcs[pt].qinvd;
         double f0[BT], f1[BT];
 #pragma unroll
@@ -198,47 +214,28 @@ __global__ void __launch_bounds__(256, 2) k_inner(const u64* __restrict__ d, con
                 f1[i] = fp_load(acc[(((size_t)b * 2 + 1) * rows + t) * N + c], q);
             }
         }
-        if (beta <= 8) {
-            // all digits' words are requested before the first product, so a thread has up to
-            // 8 * (2 + BT) loads in flight
-            u64 kb[8], ka[8], x[8][BT];
+        u64 kb, ka, x[BT], nkb, nka, nx[BT];
+        load_digit(0, kb, ka, x);
+#pragma unroll 1
+        for (uint32_t j = 0; j < beta; j++) {
+            load_digit(j + 1 < beta ? j + 1 : j, nkb, nka, nx);
+            const double dkb = fp_from_u64(kb), dka = fp_from_u64(ka);
 #pragma unroll
-            for (int j = 0; j < 8; j++)
-                if ((uint32_t)j < beta) load_digit(j, kb[j], ka[j], x[j]);
-#pragma unroll
-            for (int j = 0; j < 8; j++)
-                if ((uint32_t)j < beta) {
-                    const double dkb = fp_from_u64(kb[j]), dka = fp_from_u64(ka[j]);
-#pragma unroll
-                    for (int i = 0; i < BT; i++) {
-                        const double xd = fp_load(x[j][i], q);
-                        f0[i] += fp_modmul(xd, dkb, q, qinv);
-                        f1[i] += fp_modmul(xd, dka, q, qinv);
-                    }
-                }
-        } else {
-            u64 kb, ka, x[BT], nkb, nka, nx[BT];
-            load_digit(0, kb, ka, x);
-            for (uint32_t j = 0; j < beta; j++) {
-                load_digit(j + 1 < beta ? j + 1 : j, nkb, nka, nx);
-                const double dkb = fp_from_u64(kb), dka = fp_from_u64(ka);
+            for (int i = 0; i < BT; i++) {
+                const double xd = fp_load(x[i], q);
+                f0[i] += fp_modmul(xd, dkb, q, qinv);
+                f1[i] += fp_modmul(xd, dka, q, qinv);
+            }
+            if ((j & 7) == 6) {   // before the 8th term since the last fold (a running sum may be included)
 #pragma unroll
                 for (int i = 0; i < BT; i++) {
-                    const double xd = fp_load(x[i], q);
-                    f0[i] += fp_modmul(xd, dkb, q, qinv);
-                    f1[i] += fp_modmul(xd, dka, q, qinv);
+                    f0[i] = fp_reduce(f0[i], q, qinv);
+                    f1[i] = fp_reduce(f1[i], q, qinv);
                 }
-                if ((j & 7) == 7) {
-#pragma unroll
-                    for (int i = 0; i < BT; i++) {
-                        f0[i] = fp_reduce(f0[i], q, qinv);
-                        f1[i] = fp_reduce(f1[i], q, qinv);
-                    }
-                }
-                kb = nkb, ka = nka;
-#pragma unroll
-                for (int i = 0; i < BT; i++) x[i] = nx[i];
             }
+            kb = nkb, ka = nka;
+#pragma unroll
+            for (int i = 0; i < BT; i++) x[i] = nx[i];
         }
 #pragma unroll
         for (int i = 0; i < BT; i++) {
@@ -250,36 +247,212 @@ __global__ void __launch_bounds__(256, 2) k_inner(const u64* __restrict__ d, con
         }
         return;
     }
-    acc128 a0[BT], a1[BT];
-#pragma unroll
-    for (int i = 0; i < BT; i++) a0[i] = a1[i] = acc128{0, 0};
-    {
-        u64 kb, ka, x[BT], nkb, nka, nx[BT];
-        load_digit(0, kb, ka, x);
-        for (uint32_t j = 0; j < beta; j++) {
-            load_digit(j + 1 < beta ? j + 1 : j, nkb, nka, nx);
-#pragma unroll
-            for (int i = 0; i < BT; i++) {
-                mac128(a0[i], x[i], kb);
-                mac128(a1[i], x[i], ka);
+    if (PATH != 1) {
+        acc128 a0[BT], a1[BT];
+    #pragma unroll
+        for (int i = 0; i < BT; i++) a0[i] = a1[i] = acc128{0, 0};
+        {
+            u64 kb, ka, x[BT], nkb, nka, nx[BT];
+            load_digit(0, kb, ka, x);
+            for (uint32_t j = 0; j < beta; j++) {
+                load_digit(j + 1 < beta ? j + 1 : j, nkb, nka, nx);
+    #pragma unroll
+                for (int i = 0; i < BT; i++) {
+                    mac128(a0[i], x[i], kb);
+                    mac128(a1[i], x[i], ka);
+                }
+                kb = nkb, ka = nka;
+    #pragma unroll
+                for (int i = 0; i < BT; i++) x[i] = nx[i];
             }
-            kb = nkb, ka = nka;
-#pragma unroll
-            for (int i = 0; i < BT; i++) x[i] = nx[i];
+        }
+        const PrimeConst pc = pcs[pt];
+    #pragma unroll
+        for (int i = 0; i < BT; i++) {
+            const uint32_t b = b0 + i;
+            if (b < batch) {
+                u64* o0 = acc + (((size_t)b * 2 + 0) * rows + t) * N + c;
+                u64* o1 = acc + (((size_t)b * 2 + 1) * rows + t) * N + c;
+                u64 r0 = reduce128(a0[i].hi, a0[i].lo, pc), r1 = reduce128(a1[i].hi, a1[i].lo, pc);
+                if (accumulate) r0 = addmod(r0, *o0, pc.q), r1 = addmod(r1, *o1, pc.q);
+                *o0 = r0;
+                *o1 = r1;
+            }
         }
     }
-    const PrimeConst pc = pcs[pt];
+}
+
+// ---------------------------------------------------------------------------------------
+// The same inner product with operands staged by bulk asynchronous copies (TMA, no multicast).
+// A persistent CTA walks over tiles (limb row t, 256 coefficients, BT ciphertexts).  One thread requests, per
+// digit, the two key rows and the BT digit rows of the NEXT tile (2 KB each) into the other half of shared memory,
+// completion counted in bytes on an mbarrier, while all threads multiply out the current tile from shared memory;
+// nothing is staged through registers, so one CTA keeps 2 x beta x (2 + BT) x 2 KB in flight.  Tiles that share key
+// rows (same row and coefficient block, other ciphertext group) are adjacent in the tile order, i.e. run at the
+// same time on neighbouring SMs and share the key through L2.  For hoisted rotations the source block of the
+// digit rows is the image of the coefficient block under the Galois permutation (aligned blocks map to aligned
+// blocks) and a thread picks its word inside the block.  Every wait is bounded: a wait that runs out sets the
+// status word and the CTA returns.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// returns 0 when the phase completed, 1 when the poll budget ran out
+__device__ __forceinline__ uint32_t mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < (1u << 20); it++) {
+        if (mbar_try_wait(bar, parity)) return 0;
+        if (it > 64) __nanosleep(64);
+    }
+    return 1;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+template <int BT>
+__global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ d, const u64* __restrict__ ext,
+                                                      const u64* __restrict__ key, u64* __restrict__ acc,
+                                                      const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
+                                                      uint32_t n_q, uint32_t K, uint32_t alpha, uint32_t beta,
+                                                      uint32_t batch, uint32_t log_n, u64 g, int accumulate,
+                                                      uint32_t n_tiles, uint32_t* __restrict__ status) {
+    constexpr int R = 2 + BT;                                // rows per digit: key b, key a, BT ciphertexts
+    extern __shared__ __align__(128) u64 smem[];             // [2 stages][beta][R][256] then two barriers
+    const uint32_t tid = threadIdx.x;
+    const uint32_t rows = level + K, np = n_q + K, nblk = N >> 8, ngrp = (batch + BT - 1) / BT;
+    const uint32_t stage_words = beta * R * 256;
+    const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem);
+    const uint32_t bar0 = sbase + 2 * stage_words * 8;
+    if (tid == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    auto decode = [&](uint32_t tile, uint32_t& t, uint32_t& cblk, uint32_t& b0) {
+        const uint32_t grp = tile % ngrp, rest = tile / ngrp;
+        cblk = rest % nblk;
+        t = rest / nblk;
+        b0 = grp * BT;
+    };
+    auto issue = [&](uint32_t tile, uint32_t stage) {        // thread 0 only
+        uint32_t t, cblk, b0;
+        decode(tile, t, cblk, b0);
+        const uint32_t pt = t < level ? t : n_q + (t - level);
+        const uint32_t own = t < level ? t / alpha : 0xFFFFFFFFu;
+        const uint32_t sblk = g ? (galois_src(cblk << 8, log_n, g) >> 8) : cblk;
+        const uint32_t bar = bar0 + stage * 8;
+        uint32_t dst = sbase + stage * stage_words * 8;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier reads of this half precede the refill
+        mbar_expect_tx(bar, stage_words * 8);
+        for (uint32_t j = 0; j < beta; j++) {
+            bulk_g2s(dst, key + ((size_t)(2 * j) * np + pt) * N + (cblk << 8), 2048, bar);
+            bulk_g2s(dst + 2048, key + ((size_t)(2 * j + 1) * np + pt) * N + (cblk << 8), 2048, bar);
+            dst += 4096;
 #pragma unroll
-    for (int i = 0; i < BT; i++) {
-        const uint32_t b = b0 + i;
-        if (b < batch) {
-            u64* o0 = acc + (((size_t)b * 2 + 0) * rows + t) * N + c;
-            u64* o1 = acc + (((size_t)b * 2 + 1) * rows + t) * N + c;
-            u64 r0 = reduce128(a0[i].hi, a0[i].lo, pc), r1 = reduce128(a1[i].hi, a1[i].lo, pc);
-            if (accumulate) r0 = addmod(r0, *o0, pc.q), r1 = addmod(r1, *o1, pc.q);
-            *o0 = r0;
-            *o1 = r1;
+            for (int i = 0; i < BT; i++) {
+                const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
+                const u64* src = (j == own) ? d + ((size_t)b * level + t) * N : ext + (((size_t)b * beta + j) * rows + t) * N;
+                bulk_g2s(dst, src + (sblk << 8), 2048, bar);
+                dst += 2048;
+            }
         }
+    };
+    uint32_t tile = blockIdx.x;
+    if (tid == 0 && tile < n_tiles) issue(tile, 0);
+    for (uint32_t k = 0; tile < n_tiles; k++, tile += gridDim.x) {
+        const uint32_t stage = k & 1;
+        if (tid == 0 && tile + gridDim.x < n_tiles) issue(tile + gridDim.x, stage ^ 1);
+        const uint32_t late = mbar_wait_bounded(bar0 + stage * 8, (k >> 1) & 1);
+        if (__syncthreads_or((int)late)) {                   // block-uniform: give up together
+            if (tid == 0) {
+                atomicExch(status, 1u);
+                if (tile + gridDim.x < n_tiles) mbar_wait_bounded(bar0 + (stage ^ 1) * 8, ((k + 1) >> 1) & 1);
+            }
+            return;
+        }
+        uint32_t t, cblk, b0;
+        decode(tile, t, cblk, b0);
+        const uint32_t c = (cblk << 8) + tid;
+        const uint32_t si = g ? (galois_src(c, log_n, g) & 255u) : tid;
+        const uint32_t pt = t < level ? t : n_q + (t - level);
+        const u64* sm = smem + (size_t)stage * stage_words;
+        if (pcs[pt].q < FESC_FP_LIMIT) {
+            const double q = pcs[pt].qd, qinv = pcs[pt].qinvd;
+            double f0[BT], f1[BT];
+#pragma unroll
+            for (int i = 0; i < BT; i++) {
+                f0[i] = f1[i] = 0.0;
+                if (accumulate) {
+                    const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
+                    f0[i] = fp_load(acc[(((size_t)b * 2 + 0) * rows + t) * N + c], q);
+                    f1[i] = fp_load(acc[(((size_t)b * 2 + 1) * rows + t) * N + c], q);
+                }
+            }
+            for (uint32_t j = 0; j < beta; j++) {
+                const u64* dj = sm + (size_t)j * R * 256;
+                const double dkb = fp_from_u64(dj[tid]), dka = fp_from_u64(dj[256 + tid]);
+#pragma unroll
+                for (int i = 0; i < BT; i++) {
+                    const double xd = fp_load(dj[(2 + i) * 256 + si], q);
+                    f0[i] += fp_modmul(xd, dkb, q, qinv);
+                    f1[i] += fp_modmul(xd, dka, q, qinv);
+                }
+                if ((j & 7) == 7) {
+#pragma unroll
+                    for (int i = 0; i < BT; i++) {
+                        f0[i] = fp_reduce(f0[i], q, qinv);
+                        f1[i] = fp_reduce(f1[i], q, qinv);
+                    }
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < BT; i++) {
+                const uint32_t b = b0 + i;
+                if (b < batch) {
+                    acc[(((size_t)b * 2 + 0) * rows + t) * N + c] = fp_store(f0[i], q, qinv);
+                    acc[(((size_t)b * 2 + 1) * rows + t) * N + c] = fp_store(f1[i], q, qinv);
+                }
+            }
+        } else {
+            const PrimeConst pc = pcs[pt];
+            acc128 a0[BT], a1[BT];
+#pragma unroll
+            for (int i = 0; i < BT; i++) a0[i] = a1[i] = acc128{0, 0};
+            for (uint32_t j = 0; j < beta; j++) {
+                const u64* dj = sm + (size_t)j * R * 256;
+                const u64 kb = dj[tid], ka = dj[256 + tid];
+#pragma unroll
+                for (int i = 0; i < BT; i++) {
+                    const u64 x = dj[(2 + i) * 256 + si];
+                    mac128(a0[i], x, kb);
+                    mac128(a1[i], x, ka);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < BT; i++) {
+                const uint32_t b = b0 + i;
+                if (b < batch) {
+                    u64* o0 = acc + (((size_t)b * 2 + 0) * rows + t) * N + c;
+                    u64* o1 = acc + (((size_t)b * 2 + 1) * rows + t) * N + c;
+                    u64 r0 = reduce128(a0[i].hi, a0[i].lo, pc), r1 = reduce128(a1[i].hi, a1[i].lo, pc);
+                    if (accumulate) r0 = addmod(r0, *o0, pc.q), r1 = addmod(r1, *o1, pc.q);
+                    *o0 = r0;
+                    *o1 = r1;
+                }
+            }
+        }
+        __syncthreads();                                     // this half may be refilled from now on
     }
 }
 
@@ -408,19 +581,39 @@ static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint
     const uint32_t beta = (level + alpha - 1) / alpha, rows = level + K;
     const uint32_t gx = (N + 255) / 256;
     prof_begin(ctx, PF_INNER, st);
-    if (batch >= 4) {
-        dim3 gd(gx, rows, (batch + 3) / 4);
-        k_inner<4><<<gd, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch,
-                                       ctx->log_n, g, accumulate);
-    } else if (batch >= 2) {
-        dim3 gd(gx, rows, (batch + 1) / 2);
-        k_inner<2><<<gd, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch,
-                                       ctx->log_n, g, accumulate);
-    } else {
-        dim3 gd(gx, rows, 1);
-        k_inner<1><<<gd, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch,
-                                       ctx->log_n, g, accumulate);
-    }
+    static const int use_tma = getenv("FESC_INNER_TMA") ? 1 : 0;
+#define INNER(BT_, PATH_, ROW0_, NROWS_)                                                                        \
+    do {                                                                                                        \
+        dim3 gd(gx, NROWS_, (batch + BT_ - 1) / BT_);                                                           \
+        k_inner<BT_, PATH_><<<gd, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, \
+                                                beta, batch, ctx->log_n, g, accumulate, ROW0_);                 \
+    } while (0)
+    // data rows on primes below 2^50 and special rows above: one launch per kind, each compiled for its arithmetic
+    bool split = true;
+    for (uint32_t i = 0; i < level; i++) split = split && ctx->q[i] < FESC_FP_LIMIT;
+    for (uint32_t k = 0; k < K; k++) split = split && ctx->q[nq + k] >= FESC_FP_LIMIT;
+    if (use_tma && N % 256 == 0 && beta <= 8 && batch >= 3) {   // 128-bit sums of <= 8 products below 2^124 cannot wrap
+        const uint32_t n_tiles = rows * (N >> 8) * ((batch + 3) / 4);
+        const size_t smem = (size_t)2 * beta * 6 * 2048 + 16;
+        int dev = 0, sms = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(k_inner_tma<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        const uint32_t grid = n_tiles < (uint32_t)sms ? n_tiles : (uint32_t)sms;
+        k_inner_tma<4><<<grid, 256, smem, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta,
+                                                 batch, ctx->log_n, g, accumulate, n_tiles, ctx->d_status);
+    } else if (split) {
+        if (batch >= 6) INNER(8, 1, 0, level);
+        else if (batch >= 3) INNER(4, 1, 0, level);
+        else if (batch == 2) INNER(2, 1, 0, level);
+        else INNER(1, 1, 0, level);
+        if (batch >= 3) INNER(4, 2, level, K);
+        else if (batch == 2) INNER(2, 2, level, K);
+        else INNER(1, 2, level, K);
+    } else if (batch >= 3) INNER(4, 0, 0, rows);
+    else if (batch == 2) INNER(2, 0, 0, rows);
+    else INNER(1, 0, 0, rows);
+#undef INNER
     prof_end(ctx, PF_INNER, st);
     FESC_CHECK_CUDA(ctx, cudaGetLastError());
     ctx->counters[1] += batch;
