@@ -136,6 +136,7 @@ struct ModUpDigit {
     uint32_t n_src, first;
     u64 inv[FESC_MAX_ALPHA], invs[FESC_MAX_ALPHA];   // (Q_j/q_i)^-1 mod q_i and its Shoup companion
     u64 mat[FESC_MAX_ALPHA][FESC_MAX_PRIMES];        // (Q_j/q_i) mod q_t, t = prime index
+    double matd[FESC_MAX_ALPHA][FESC_MAX_PRIMES];    // the same as doubles (exact for targets below 2^53)
 };
 // Division by P = product of the special primes p_k.
 struct ModDownTab {
@@ -145,6 +146,8 @@ struct ModDownTab {
     u64 mat30[FESC_MAX_SPECIAL][FESC_MAX_PRIMES];        // (P/p_k) * 2^30 mod q_i
     u64 wrap[FESC_MAX_SPECIAL + 1][FESC_MAX_PRIMES];     // cnt * P mod q_i
     u64 pinv[FESC_MAX_PRIMES], pinvs[FESC_MAX_PRIMES];   // P^-1 mod q_i
+    double matd[FESC_MAX_SPECIAL][FESC_MAX_PRIMES], mat30d[FESC_MAX_SPECIAL][FESC_MAX_PRIMES];   // as doubles
+    double wrapd[FESC_MAX_SPECIAL + 1][FESC_MAX_PRIMES], pinvd[FESC_MAX_PRIMES];
 };
 // Rescale from level l (drops limb l-1); entry index l.
 struct RescaleTab {

@@ -187,6 +187,7 @@ static int build_tables(fesc_ctx* ctx) {
                     for (uint32_t b = 0; b < d.n_src; b++)
                         if (b != a) m = h_mul(m, q[d.first + b] % q[t], q[t]);
                     d.mat[a][t] = m;
+                    d.matd[a][t] = (double)m;
                 }
                 d.inv[a] = h_inv(d.mat[a][i], q[i]);
                 d.invs[a] = h_shoup(d.inv[a], q[i]);
@@ -213,6 +214,8 @@ static int build_tables(fesc_ctx* ctx) {
                 if (b != k) m = h_mul(m, q[nq + b] % q[i], q[i]);
             md.mat[k][i] = m;
             md.mat30[k][i] = h_mul(m, (1ull << 30) % q[i], q[i]);
+            md.matd[k][i] = (double)md.mat[k][i];
+            md.mat30d[k][i] = (double)md.mat30[k][i];
         }
     }
     for (uint32_t i = 0; i < nq; i++) {
@@ -222,6 +225,8 @@ static int build_tables(fesc_ctx* ctx) {
         md.pinv[i] = h_inv(P, q[i]);
         md.pinvs[i] = h_shoup(md.pinv[i], q[i]);
         for (uint32_t c = 0; c <= K; c++) md.wrap[c][i] = h_mul(c, P, q[i]);
+        for (uint32_t c = 0; c <= K; c++) md.wrapd[c][i] = (double)md.wrap[c][i];
+        md.pinvd[i] = (double)md.pinv[i];
     }
     if ((rc = upload(ctx, &ctx->tabs.d_moddown, mdv)) != FESC_OK) return rc;
     if ((rc = upload(ctx, &ctx->tabs.d_Pmod_all, Pmod)) != FESC_OK) return rc;

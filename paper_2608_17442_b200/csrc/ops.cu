@@ -103,54 +103,78 @@ __global__ void __launch_bounds__(256) k_autom_ct(const u64* __restrict__ in, si
 // ext row order: data limbs 0..level-1 then the K special limbs; rows of the digit's own limbs
 // are left untouched (the inner product reads those from the EVAL-form input).
 // ---------------------------------------------------------------------------------------
-template <int ALPHA>
+template <int ALPHA, int VEC>
 __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u64* __restrict__ ext,
                                                const ModUpDigit* __restrict__ tab, const PrimeConst* __restrict__ pcs,
                                                uint32_t N, uint32_t level, uint32_t n_q, uint32_t K, uint32_t beta) {
-    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    // VEC adjacent coefficients per thread: every table word and every prime constant serves VEC products
+    const uint32_t c = (blockIdx.x * blockDim.x + threadIdx.x) * VEC;
     const uint32_t j = blockIdx.y, b = blockIdx.z;
     if (c >= N) return;
     const ModUpDigit* dg = tab + j;
     const uint32_t first = dg->first, n_src = dg->n_src;
-    u64 y[ALPHA];
+    u64 y[ALPHA][VEC];
+    bool src_small = true;
 #pragma unroll
     for (int a = 0; a < ALPHA; a++) {
-        y[a] = 0;
+#pragma unroll
+        for (int v = 0; v < VEC; v++) y[a][v] = 0;
         if (a < n_src) {
-            u64 v = dcoef[((size_t)b * level + first + a) * N + c];
-            y[a] = shoup(v, dg->inv[a], dg->invs[a], pcs[first + a].q);
+            const u64* src = dcoef + ((size_t)b * level + first + a) * N + c;
+            const u64 q = pcs[first + a].q, inv = dg->inv[a], invs = dg->invs[a];
+            src_small = src_small && q < FESC_FP_LIMIT;
+            u64 w[VEC];
+            if (VEC == 2) {
+                const ulonglong2 t2 = *reinterpret_cast<const ulonglong2*>(src);
+                w[0] = t2.x, w[VEC - 1] = t2.y;
+            } else {
+                w[0] = *src;
+            }
+#pragma unroll
+            for (int v = 0; v < VEC; v++) y[a][v] = shoup(w[v], inv, invs, q);
         }
     }
     const uint32_t rows = level + K;
     u64* out = ext + ((size_t)b * beta + j) * rows * N + c;
     // every y_a is below 2^50 when its source prime is: exact FP64 products for targets below 2^50
-    bool src_small = true;
-    double yd[ALPHA];
+    double yd[ALPHA][VEC];
 #pragma unroll
-    for (int a = 0; a < ALPHA; a++) {
-        yd[a] = 0.0;
-        if (a < n_src) {
-            src_small = src_small && pcs[first + a].q < FESC_FP_LIMIT;
-            yd[a] = fp_from_u64(y[a] & 0x000FFFFFFFFFFFFFull);
-        }
-    }
+    for (int a = 0; a < ALPHA; a++)
+#pragma unroll
+        for (int v = 0; v < VEC; v++) yd[a][v] = fp_from_u64(y[a][v] & 0x000FFFFFFFFFFFFFull);
     for (uint32_t t = 0; t < rows; t++) {
         if (t >= first && t < first + n_src) continue;
         const uint32_t pt = t < level ? t : n_q + (t - level);
+        u64 r[VEC];
         if (src_small && pcs[pt].q < FESC_FP_LIMIT) {
             const double q = pcs[pt].qd, qinv = pcs[pt].qinvd;
-            double s = 0.0;
+            double s[VEC];
+#pragma unroll
+            for (int v = 0; v < VEC; v++) s[v] = 0.0;
 #pragma unroll
             for (int a = 0; a < ALPHA; a++)
-                if (a < n_src) s += fp_modmul(yd[a], fp_from_u64(dg->mat[a][pt]), q, qinv);
-            out[(size_t)t * N] = fp_store(s, q, qinv);
+                if (a < n_src) {
+                    const double m = dg->matd[a][pt];
+#pragma unroll
+                    for (int v = 0; v < VEC; v++) s[v] += fp_modmul(yd[a][v], m, q, qinv);
+                }
+#pragma unroll
+            for (int v = 0; v < VEC; v++) r[v] = fp_store(s[v], q, qinv);
         } else {
-            acc128 acc{0, 0};
+            const PrimeConst pc = pcs[pt];
 #pragma unroll
-            for (int a = 0; a < ALPHA; a++)
-                if (a < n_src) mac128(acc, y[a], dg->mat[a][pt]);
-            out[(size_t)t * N] = reduce128(acc.hi, acc.lo, pcs[pt]);
+            for (int v = 0; v < VEC; v++) {
+                acc128 acc{0, 0};
+#pragma unroll
+                for (int a = 0; a < ALPHA; a++)
+                    if (a < n_src) mac128(acc, y[a][v], dg->mat[a][pt]);
+                r[v] = reduce128(acc.hi, acc.lo, pc);
+            }
         }
+        if (VEC == 2)
+            *reinterpret_cast<ulonglong2*>(out + (size_t)t * N) = make_ulonglong2(r[0], r[VEC - 1]);
+        else
+            out[(size_t)t * N] = r[0];
     }
 }
 
@@ -461,52 +485,86 @@ __global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ d,
 //   y_k = r_k * (P/p_k)^-1 mod p_k, taken in [-(p_k-1)/2, (p_k-1)/2];
 //   u_i = sum_k y_k (P/p_k) mod q_i = sum_k [y_k]_canonical (P/p_k) - #{y_k > p_k/2} * P  (mod q_i).
 // ---------------------------------------------------------------------------------------
+template <int VEC>
 __global__ void __launch_bounds__(256) k_moddown_conv(const u64* __restrict__ acc, u64* __restrict__ u,
                                                       const ModDownTab* __restrict__ tab,
                                                       const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
                                                       uint32_t n_q, uint32_t K) {
-    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    // VEC adjacent coefficients per thread: every table word and every prime constant serves VEC products
+    const uint32_t c = (blockIdx.x * blockDim.x + threadIdx.x) * VEC;
     const uint32_t bp = blockIdx.y;   // b*2 + p
     if (c >= N) return;
     const uint32_t rows = level + K;
-    u64 y[FESC_MAX_SPECIAL];
-    uint32_t cnt = 0;
+    u64 y[FESC_MAX_SPECIAL][VEC];
+    uint32_t cnt[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; v++) cnt[v] = 0;
 #pragma unroll
     for (int k = 0; k < FESC_MAX_SPECIAL; k++) {
-        y[k] = 0;
+#pragma unroll
+        for (int v = 0; v < VEC; v++) y[k][v] = 0;
         if (k < K) {
-            u64 r = acc[((size_t)bp * rows + level + k) * N + c];
-            y[k] = shoup(r, tab->inv[k], tab->invs[k], pcs[n_q + k].q);
-            cnt += y[k] > tab->half[k];
+            const u64* src = acc + ((size_t)bp * rows + level + k) * N + c;
+            u64 w[VEC];
+            if (VEC == 2) {
+                const ulonglong2 t2 = *reinterpret_cast<const ulonglong2*>(src);
+                w[0] = t2.x, w[VEC - 1] = t2.y;
+            } else {
+                w[0] = *src;
+            }
+            const u64 inv = tab->inv[k], invs = tab->invs[k], pk = pcs[n_q + k].q, half = tab->half[k];
+#pragma unroll
+            for (int v = 0; v < VEC; v++) {
+                y[k][v] = shoup(w[v], inv, invs, pk);
+                cnt[v] += y[k][v] > half;
+            }
         }
     }
     // 30-bit halves of every y_k as doubles, for targets below 2^50 (exact FP64 products)
-    double yh[FESC_MAX_SPECIAL], yl[FESC_MAX_SPECIAL];
+    double yh[FESC_MAX_SPECIAL][VEC], yl[FESC_MAX_SPECIAL][VEC];
 #pragma unroll
-    for (int k = 0; k < FESC_MAX_SPECIAL; k++) {
-        yh[k] = fp_from_u64(y[k] >> 30);
-        yl[k] = fp_from_u64(y[k] & ((1ull << 30) - 1));
-    }
+    for (int k = 0; k < FESC_MAX_SPECIAL; k++)
+#pragma unroll
+        for (int v = 0; v < VEC; v++) {
+            yh[k][v] = fp_from_u64(y[k][v] >> 30);
+            yl[k][v] = fp_from_u64(y[k][v] & ((1ull << 30) - 1));
+        }
     for (uint32_t i = 0; i < level; i++) {
+        u64 r[VEC];
         if (pcs[i].q < FESC_FP_LIMIT) {
             const double q = pcs[i].qd, qinv = pcs[i].qinvd;
-            double s = -fp_from_u64(tab->wrap[cnt][i]);
+            double s[VEC];
+#pragma unroll
+            for (int v = 0; v < VEC; v++) s[v] = -tab->wrapd[cnt[v]][i];
 #pragma unroll
             for (int k = 0; k < FESC_MAX_SPECIAL; k++)
                 if (k < K) {
-                    s += fp_modmul(yh[k], fp_from_u64(tab->mat30[k][i]), q, qinv);
-                    s += fp_modmul(yl[k], fp_from_u64(tab->mat[k][i]), q, qinv);
-                    if (k == 3) s = fp_reduce(s, q, qinv);
-                }
-            u[((size_t)bp * level + i) * N + c] = fp_store(s, q, qinv);
-        } else {
-            acc128 a{0, 0};
+                    const double m30 = tab->mat30d[k][i], m = tab->matd[k][i];
 #pragma unroll
-            for (int k = 0; k < FESC_MAX_SPECIAL; k++)
-                if (k < K) mac128(a, y[k], tab->mat[k][i]);
-            u64 v = reduce128(a.hi, a.lo, pcs[i]);
-            u[((size_t)bp * level + i) * N + c] = submod(v, tab->wrap[cnt][i], pcs[i].q);
+                    for (int v = 0; v < VEC; v++) {
+                        s[v] += fp_modmul(yh[k][v], m30, q, qinv);
+                        s[v] += fp_modmul(yl[k][v], m, q, qinv);
+                        if (k == 3) s[v] = fp_reduce(s[v], q, qinv);
+                    }
+                }
+#pragma unroll
+            for (int v = 0; v < VEC; v++) r[v] = fp_store(s[v], q, qinv);
+        } else {
+            const PrimeConst pc = pcs[i];
+#pragma unroll
+            for (int v = 0; v < VEC; v++) {
+                acc128 a{0, 0};
+#pragma unroll
+                for (int k = 0; k < FESC_MAX_SPECIAL; k++)
+                    if (k < K) mac128(a, y[k][v], tab->mat[k][i]);
+                r[v] = submod(reduce128(a.hi, a.lo, pc), tab->wrap[cnt[v]][i], pc.q);
+            }
         }
+        u64* dst = u + ((size_t)bp * level + i) * N + c;
+        if (VEC == 2)
+            *reinterpret_cast<ulonglong2*>(dst) = make_ulonglong2(r[0], r[VEC - 1]);
+        else
+            *dst = r[0];
     }
 }
 
@@ -550,8 +608,13 @@ static int ks_decompose(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint
     if ((rc = ntt_launch(ctx, ws.dcoef, (size_t)batch * level, m, true, st)) != FESC_OK) return rc;
     // 2. ModUp
     const ModUpDigit* tab = ctx->tabs.d_modup + (size_t)(level - 1) * ctx->beta_max;
-    dim3 gmu(gx, beta, batch);
-#define MODUP(A) k_modup<A><<<gmu, 256, 0, st>>>(ws.dcoef, ws.ext, tab, ctx->d_pc, N, level, nq, K, beta)
+    const bool vec2 = N % 512 == 0;
+    dim3 gmu(vec2 ? N / 512 : gx, beta, batch);
+#define MODUP(A)                                                                                           \
+    do {                                                                                                   \
+        if (vec2) k_modup<A, 2><<<gmu, 256, 0, st>>>(ws.dcoef, ws.ext, tab, ctx->d_pc, N, level, nq, K, beta); \
+        else k_modup<A, 1><<<gmu, 256, 0, st>>>(ws.dcoef, ws.ext, tab, ctx->d_pc, N, level, nq, K, beta);  \
+    } while (0)
     prof_begin(ctx, PF_MODUP, st);
     if (alpha <= 1) MODUP(1);
     else if (alpha <= 2) MODUP(2);
@@ -632,7 +695,10 @@ static int ks_moddown(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint32
     for (uint32_t t = 0; t < rows; t++) m.prime[t] = t < level ? 0xFF : (uint8_t)(nq + (t - level));
     if ((rc = ntt_launch(ctx, ws.acc, (size_t)batch * 2 * rows, m, true, st)) != FESC_OK) return rc;
     prof_begin(ctx, PF_MODDOWN, st);
-    k_moddown_conv<<<dim3(gx, batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K);
+    if (N % 512 == 0)
+        k_moddown_conv<2><<<dim3(N / 512, batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K);
+    else
+        k_moddown_conv<1><<<dim3(gx, batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K);
     prof_end(ctx, PF_MODDOWN, st);
     m.period = level;
     for (uint32_t i = 0; i < level; i++) m.prime[i] = (uint8_t)i;
