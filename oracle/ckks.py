@@ -287,6 +287,30 @@ class Oracle:
             outs.append(np.stack([self.add(c0, self.mod_down(acc[0], level), data), self.mod_down(acc[1], level)]))
         return outs
 
+    def rotate_sum_hoisted(self, ct, key_ids):
+        """ct + sum_k rot_k(ct): hoisted rotations (one decomposition of c1) whose key-switch accumulators are
+        summed on the extended basis and divided by P ONCE (a separately defined mode, used by the radix-4
+        rotate-and-add fills of the scan):
+            out0 = c0 + sum_k sigma_k(c0) + ModDown( sum_k sum_j sigma_k(d~_j) (.) evk_{k,j}[0] ),
+            out1 = c1                     + ModDown( sum_k sum_j sigma_k(d~_j) (.) evk_{k,j}[1] )."""
+        level = ct.shape[1]
+        data = list(range(level))
+        ext = data + self.special
+        d_eval = _arr(ct[1])
+        d_coeff = self.intt(d_eval, data)
+        digits = [self.mod_up_digit(d_coeff, d_eval, j, level) for j in range(-(-level // self.alpha))]
+        acc = np.zeros((2, len(ext), self.N), dtype=np.uint64)
+        y0 = _arr(ct[0]).copy()
+        for kid in key_ids:
+            g, evk = self.keys[kid]
+            for j, dj in enumerate(digits):
+                dt = self.automorphism(dj, g, len(ext))
+                for p in range(2):
+                    _lib.orc_muladd(dt, _arr(evk[j, p][ext]), acc[p], self._q(ext), len(ext), self.N)
+            y0 = self.add(y0, self.automorphism(ct[0], g, level), data)
+        return np.stack([self.add(y0, self.mod_down(acc[0], level), data),
+                         self.add(_arr(ct[1]), self.mod_down(acc[1], level), data)])
+
     def rescale(self, ct):
         """Rounded division by the last prime, level l -> l-1:
         c_i <- (c_i - [c_last]_centred) * q_last^-1 mod q_i  (= round(c / q_last) exactly)."""

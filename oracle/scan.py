@@ -77,7 +77,14 @@ class ScanShape:
         self.dg = min(16, B_blk)                      # base of the two-digit token offset t = t_lo + dg*t_hi
 
     # rotation amounts (slot LEFT shifts, modulo n) the dataflow uses
-    def rotation_amounts(self):
+    def chains(self):
+        """(signed unit, steps) of every rotate-and-add chain ct += rot(ct, unit * 2^b), b = 0..steps-1."""
+        lg = lambda v: int(math.log2(v))
+        return [(-1, lg(self.P)), (-1, lg(self.d_s)), (-self.P, lg(self.R // self.P)),
+                (-self.stride, lg(self.c_state)), (1, lg(self.d_s))]
+
+    def rotation_amounts(self, hoist: bool = False):
+        """hoist=True adds the amounts 3 * unit * 2^b of the radix-4 chains (b even, b + 1 < steps)."""
         n, dg, B = self.n, self.dg, self.B
         lo = range(1, dg)
         hi = range(1, B // dg)
@@ -89,6 +96,9 @@ class ScanShape:
         am |= {(-self.P * (1 << b)) % n for b in range(int(math.log2(self.R // self.P)))}        # a fill
         am |= {(-self.stride * (1 << b)) % n for b in range(int(math.log2(self.c_state)))}       # B, C fill
         am |= {(1 << b) for b in range(int(math.log2(self.d_s)))}                        # state reduction
+        if hoist:
+            for unit, steps in self.chains():
+                am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
         am.discard(0)
         return sorted(am)
 
@@ -141,8 +151,8 @@ def key_id_for(shape: ScanShape, amount: int, base: int = 100000) -> int:
     return base + shape.n if amount == CONJ else base + amount % shape.n
 
 
-def add_scan_keys(orc: Oracle, shape: ScanShape, base: int = 100000):
-    for r in shape.rotation_amounts():
+def add_scan_keys(orc: Oracle, shape: ScanShape, base: int = 100000, hoist: bool = False):
+    for r in shape.rotation_amounts(hoist):
         if key_id_for(shape, r, base) not in orc.keys:
             orc.add_galois_key(r, key_id_for(shape, r, base))
     if key_id_for(shape, CONJ, base) not in orc.keys:
@@ -200,8 +210,11 @@ def unpack_output(orc: Oracle, shape: ScanShape, consts: ScanConsts, out):
 # homomorphic evaluation
 # ---------------------------------------------------------------------------------------------
 class ScanEvaluator:
-    def __init__(self, orc: Oracle, shape: ScanShape, consts: ScanConsts, key_base: int = 100000):
-        self.o, self.sh, self.c, self.kb = orc, shape, consts, key_base
+    def __init__(self, orc: Oracle, shape: ScanShape, consts: ScanConsts, key_base: int = 100000, hoist: bool = False):
+        """hoist=True (a separately defined mode, other residues, same values): rotate-and-add chains take two
+        steps at once as ct + rot(ct, d) + rot(ct, 2d) + rot(ct, 3d) with one decomposition and one division by P
+        (`rotate_sum_hoisted`), and the low digit of the two-digit token offsets uses `rotate_hoisted`."""
+        self.o, self.sh, self.c, self.kb, self.hoist = orc, shape, consts, key_base, hoist
         self.count = dict(rot=0, conj=0, ctmul=0, adjust=0, ptmul=0, compose=0)
 
     # -- primitives ---------------------------------------------------------------------------
@@ -242,19 +255,41 @@ class ScanEvaluator:
         scaled = np.stack([self.o.mul_scalar(cut[p], [k] * (dst + 1), lv) for p in range(2)])
         return self.o.rescale(scaled)
 
-    def fill_right(self, ct, unit, steps):
-        """ct += rot(ct, -unit*2^b) for b = 0..steps-1 (copies a block to 2^steps consecutive blocks)."""
-        for b in range(steps):
-            ct = self.add(ct, self.rot(ct, -(unit << b)))
+    def chain(self, ct, unit, steps):
+        """ct += rot(ct, unit*2^b) for b = 0..steps-1 (unit signed).  Hoisted mode: steps (b, b+1) together."""
+        b = 0
+        while b < steps:
+            d = unit * (1 << b)
+            if self.hoist and b + 1 < steps:
+                self.count["rot"] += 3
+                ct = self.o.rotate_sum_hoisted(ct, [key_id_for(self.sh, k * d, self.kb) for k in (1, 2, 3)])
+                b += 2
+            else:
+                ct = self.add(ct, self.rot(ct, d))
+                b += 1
         return ct
 
-    def two_digit_rot(self, giants, t, unit):
-        """rot(src, unit*t) with t = t_lo + dg*t_hi; `giants[t_hi]` caches rot(src, unit*dg*t_hi)."""
-        return self.rot(giants[t // self.sh.dg], unit * (t % self.sh.dg))
+    def fill_right(self, ct, unit, steps):
+        """ct += rot(ct, -unit*2^b) for b = 0..steps-1 (copies a block to 2^steps consecutive blocks)."""
+        return self.chain(ct, -unit, steps)
 
-    def giants_of(self, ct, unit):
+    def extract_all(self, ct, unit):
+        """[rot(ct, unit*t) for t < B] with t = t_lo + dg*t_hi: rot(ct, unit*dg*t_hi) first, then the low digit
+        (in hoisted mode the dg-1 low-digit rotations of one ciphertext share its decomposition)."""
         sh = self.sh
-        return [ct if th == 0 else self.rot(ct, unit * sh.dg * th) for th in range(sh.B // sh.dg)]
+        out = [None] * sh.B
+        for th in range(sh.B // sh.dg):
+            g = ct if th == 0 else self.rot(ct, unit * sh.dg * th)
+            out[th * sh.dg] = g
+            if self.hoist and sh.dg > 1:
+                self.count["rot"] += sh.dg - 1
+                lows = self.o.rotate_hoisted(g, [key_id_for(sh, unit * tl, self.kb) for tl in range(1, sh.dg)])
+                for tl in range(1, sh.dg):
+                    out[th * sh.dg + tl] = lows[tl - 1]
+            else:
+                for tl in range(1, sh.dg):
+                    out[th * sh.dg + tl] = self.rot(g, unit * tl)
+        return out
 
     def compose(self, left, right, lvl, need_p=True):
         """(p_L, s_L) then (p_R, s_R), all brought to level lvl; result at lvl-1:
@@ -270,10 +305,10 @@ class ScanEvaluator:
     def broadcast_bc(self, ct):
         """brB_t (or brC_t) for every token of the block: level l0-1, value B_t[i] at every (e', i)."""
         sh, c = self.sh, self.c
-        g = self.giants_of(ct, sh.d_s)
+        ex = self.extract_all(ct, sh.d_s)
         out = []
         for t in range(sh.B):
-            u = self.ptmul_rescale(self.two_digit_rot(g, t, sh.d_s), c.mask_b)
+            u = self.ptmul_rescale(ex[t], c.mask_b)
             out.append(self.fill_right(u, sh.stride, int(math.log2(sh.c_state))))
         return out
 
@@ -281,12 +316,12 @@ class ScanEvaluator:
         sh, c = self.sh, self.c
         l1 = c.lv["l1"]
         apre = self.fill_right(ctA, 1, int(math.log2(sh.P)))
-        gx, ga = self.giants_of(ctX, 1), self.giants_of(apre, sh.P)
+        ex, ea = self.extract_all(ctX, 1), self.extract_all(apre, sh.P)
         T = []
         for t in range(sh.B):
-            xr = self.ptmul_rescale(self.two_digit_rot(gx, t, 1), c.mask_x)
+            xr = self.ptmul_rescale(ex[t], c.mask_x)
             xr = self.fill_right(xr, 1, int(math.log2(sh.d_s)))
-            ar = self.ptmul_rescale(self.two_digit_rot(ga, t, sh.P), c.mask_a)
+            ar = self.ptmul_rescale(ea[t], c.mask_a)
             ar = self.fill_right(ar, sh.P, int(math.log2(sh.R // sh.P)))
             s = self.mul_rescale(xr, brB[t])
             T.append((self.adjust(ar, l1, "p"), s))
@@ -350,8 +385,7 @@ class ScanEvaluator:
             for kap in range(0, sh.K_s, 2):
                 paired = kap + 1 < sh.K_s
                 chi = self.add(v[t][kap], o.mul_monomial_half(v[t][kap + 1])) if paired else v[t][kap]
-                for b in range(steps):
-                    chi = self.add(chi, self.rot(chi, 1 << b))
+                chi = self.chain(chi, 1, steps)
                 if paired:
                     bar = self.conj(chi)
                     parts = [self.add(chi, bar), self.neg_times_i(self.sub(chi, bar))]   # 2 Re, 2 Im

@@ -270,3 +270,35 @@ def test_hoisted_rotations_are_rotations_and_share_noise_bound(toy_oracle):
     ct5 = np.ascontiguousarray(ct[:, :5])
     got = o.rotate_hoisted(ct5, [32])[0]
     assert np.abs(o.decrypt(got, scale) - np.roll(z, -4)).max() < 2e-4
+
+
+def test_rotate_sum_hoisted_is_the_sum_of_rotations(toy_oracle):
+    """ct + sum_k rot_k(ct) with one decomposition and one division by P: decrypts to z + sum_k roll(z, -r_k), and
+    differs from the sum of separately hoisted rotations by at most one unit per rotation in every coefficient
+    (big-integer check of the additivity of the division by P up to rounding)."""
+    from oracle.ckks import crt_lift_centered
+    o = toy_oracle
+    scale = 2.0**20
+    z = S.uniform_slots(15, 0, 1, o.n)[0]
+    level = 5
+    data = list(range(level))
+    ct = np.ascontiguousarray(o.encrypt(o.encode(z, scale, 6), 9)[:, :level])
+    rots = ((-1, 41), (-2, 42), (-3, 43))
+    for r, kid in rots:
+        o.add_galois_key(r, kid)
+    got = o.rotate_sum_hoisted(ct, [k for _, k in rots])
+    want = z + sum(np.roll(z, -r) for r, _ in rots)
+    assert np.abs(o.decrypt(got, scale) - want).max() < 5e-4
+    ref = ct
+    for out in o.rotate_hoisted(ct, [k for _, k in rots]):
+        ref = o.ct_add(ref, out)
+    seen = 0
+    for c in range(2):
+        d = o.sub(got[c], ref[c], data)
+        diff = crt_lift_centered(o.intt(d, data), [o.q[i] for i in data])
+        assert max(abs(int(v)) for v in diff) <= len(rots)
+        seen += sum(1 for v in diff if int(v) != 0)
+    assert seen > 0
+    # a single rotation: exactly ct + rotate_hoisted
+    one = o.rotate_sum_hoisted(ct, [42])
+    assert np.array_equal(one, o.ct_add(ct, o.rotate_hoisted(ct, [42])[0]))

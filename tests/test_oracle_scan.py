@@ -71,14 +71,14 @@ def test_paper_ledger_values():
     assert 2 * 768 // 768 and 2 * 24 * 64 + 2 * 128 + 24 == 3352              # d_out of in_proj
 
 
-def _run(name, **shape_kw):
+def _run(name, hoist=False, **shape_kw):
     p = S.params(name)
     orc = Oracle(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
     sh = ScanShape(orc.n, **shape_kw)
     x, a, B, C = S.scan_inputs(p["seed"], sh.L, sh.H, sh.P, 1, sh.d_s)
     c = ScanConsts(orc, sh, p["n_q"], p["log_scale"])
-    add_scan_keys(orc, sh)
-    ev = ScanEvaluator(orc, sh, c)
+    add_scan_keys(orc, sh, hoist=hoist)
+    ev = ScanEvaluator(orc, sh, c, hoist=hoist)
     out = ev.run(*encrypt_inputs(orc, sh, c, x, a, B, C))
     return sh, ev, unpack_output(orc, sh, c, out), float_recurrence(x, a, B, C)
 
@@ -102,4 +102,18 @@ def test_two_digit_offsets_and_odd_chunk_count():
     sh, ev, m, ref = _run("scan_small", L=64, H=3, P=4, d_s=4, B_blk=32)
     assert (sh.K_s, sh.K_blk, sh.dg, sh.hpc) == (3, 2, 16, 1)
     assert ev.count["conj"] == closed_form_counts(sh)["reduce_conj"] == 64
+    assert np.abs(m - ref).max() < 2.0**-22
+
+
+def test_hoisted_mode_same_values():
+    """Radix-4 rotate-and-add chains (three rotations per two steps, one decomposition and one division by P) and
+    hoisted low-digit extraction: every other count is unchanged and the decrypted contract output stays within the
+    plain mode's bound."""
+    sh, ev, m, ref = _run("scan_toy", hoist=True, L=4, H=2, P=4, d_s=2, B_blk=4)
+    _, ev0, m0, _ = _run("scan_toy", L=4, H=2, P=4, d_s=2, B_blk=4)
+    assert {k: v for k, v in ev.count.items() if k != "rot"} == {k: v for k, v in ev0.count.items() if k != "rot"}
+    assert ev.count["rot"] > ev0.count["rot"]
+    assert np.abs(m - ref).max() < 2.0**-24 and np.abs(m - m0).max() < 2.0**-24
+    sh, ev, m, ref = _run("scan_small", hoist=True, L=64, H=3, P=4, d_s=4, B_blk=32)
+    assert (sh.K_s, sh.K_blk, sh.dg) == (3, 2, 16)
     assert np.abs(m - ref).max() < 2.0**-22
