@@ -465,7 +465,7 @@ def run_ours(args):
 # ---------------------------------------------------------------------------------------------
 # optional second workload: the scan-contract of one Mamba-2-base layer (or a slice of it)
 # ---------------------------------------------------------------------------------------------
-def scan_rotation_amounts(n, P, d_s, B, stride):
+def scan_rotation_amounts(n, P, d_s, B, stride, hoist=False):
     """Slot rotations the scan-contract uses (see include/fesc.h), as left shifts modulo n."""
     import math
 
@@ -480,6 +480,10 @@ def scan_rotation_amounts(n, P, d_s, B, stride):
     am |= {(-P * (1 << b)) % n for b in range(int(math.log2(R // P)))}
     am |= {(-stride * (1 << b)) % n for b in range(int(math.log2(c_state)))}
     am |= {(1 << b) for b in range(int(math.log2(d_s)))}
+    if hoist:    # radix-4 rotate-and-add chains also rotate by 3 * unit * 2^b (b even, b + 1 < steps)
+        lg = lambda v: int(math.log2(v))
+        for unit, steps in ((-1, lg(P)), (-1, lg(d_s)), (-P, lg(R // P)), (-stride, lg(c_state)), (1, lg(d_s))):
+            am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
     am.discard(0)
     return sorted(am)
 
@@ -499,7 +503,7 @@ def run_scan(args):
     P, d_s, B, stride, l0 = 64, 128, 256, 256, 24
     K_s, K_blk = H * P // (n // stride), L // B
     base = 100000
-    for r in scan_rotation_amounts(n, P, d_s, B, stride):
+    for r in scan_rotation_amounts(n, P, d_s, B, stride, bool(args.hoist)):
         ctx.add_galois_key(r, base + r)
     ctx.add_galois_key(fesc.CONJ, base + n)
     seed = S.config_seed(5)
@@ -515,7 +519,7 @@ def run_scan(args):
     linj = l0 - 2 - 2 * 8 + 1
     out = torch.empty((K_blk, K_s, 2, linj - 3, N), dtype=torch.int64, device="cuda")
     adj = [(1 << 49) + 12345 * i for i in range((l0 + 1) ** 2)]
-    desc = fesc.ScanDesc(L, H, P, d_s, B, 0, l0, base)
+    desc = fesc.ScanDesc(L, H, P, d_s, B, 0, l0, base, int(args.hoist))
     torch.cuda.empty_cache()
 
     def step():
@@ -536,8 +540,9 @@ def run_scan(args):
     print(json.dumps({"metric": "scan-contract key-switches/s", "value": ks / (ms * 1e-3), "unit": "key-switches/s",
                       "n_gpus": 1, "steps": 1, "warmup": 1 if args.workload == "scan_slice" else 0, "ms_per_step": ms,
                       "higher_is_better": True, "dtype": "u64", "data": "synthetic",
-                      "config": {"workload": "%s: L=%d, H=%d, P=64, d_s=128, B_blk=256, K_s=%d, N=2^16, 24 limbs"
-                                             % (args.workload, L, H, K_s)},
+                      "config": {"workload": "%s: L=%d, H=%d, P=64, d_s=128, B_blk=256, K_s=%d, N=2^16, 24 limbs, %s"
+                                             % (args.workload, L, H, K_s,
+                                                "radix-4 hoisted rotate-and-add chains" if args.hoist else "plain rotations")},
                       "key_switches": ks, "limb_transforms": c1[0] - c0[0], "gpu_launches": c1[4] - c0[4],
                       "scratch_gib": c1[3] / 2**30}), flush=True)
 

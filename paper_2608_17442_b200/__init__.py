@@ -34,7 +34,8 @@ class BsgsDesc(ctypes.Structure):
 
 
 class ScanDesc(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_uint32) for n in ("L", "H", "P", "d_s", "B_blk", "stride", "n_limbs", "key_base")]
+    _fields_ = [(n, ctypes.c_uint32) for n in ("L", "H", "P", "d_s", "B_blk", "stride", "n_limbs", "key_base",
+                                                       "hoist")]
 
 
 class ScanConsts(ctypes.Structure):
@@ -66,6 +67,7 @@ def lib():
             "fesc_ct_pt_mac": [vp, vp, vp, sz, vp, u32, u32, vp],
             "fesc_rotate": [vp, vp, vp, u32, u32, u32, vp],
             "fesc_rotate_hoisted": [vp, vp, vp, u32, u32, c.POINTER(u32), u32, vp],
+            "fesc_rotate_sum_hoisted": [vp, vp, vp, u32, u32, c.POINTER(u32), u32, vp],
             "fesc_rescale": [vp, vp, vp, u32, u32, vp],
             "fesc_rescale_static": [vp, vp, vp, u32, u32, vp],
             "fesc_ct_ct_mul": [vp, vp, vp, vp, u32, u32, vp],
@@ -182,6 +184,10 @@ class Context:
 
     def rotate(self, ct_in, ct_out, batch: int, n_limbs: int, key_id: int):
         self._chk(lib().fesc_rotate(self.h, _ptr(ct_in), _ptr(ct_out), batch, n_limbs, key_id, _stream()))
+
+    def rotate_sum_hoisted(self, ct_in, ct_out, batch: int, n_limbs: int, key_ids):
+        ids = (ctypes.c_uint32 * len(key_ids))(*key_ids)
+        self._chk(lib().fesc_rotate_sum_hoisted(self.h, _ptr(ct_in), _ptr(ct_out), batch, n_limbs, ids, len(key_ids), _stream()))
 
     def rotate_hoisted(self, ct_in, ct_out, batch: int, n_limbs: int, key_ids):
         ids = (ctypes.c_uint32 * len(key_ids))(*key_ids)

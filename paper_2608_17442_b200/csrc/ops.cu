@@ -857,6 +857,74 @@ int rotate_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64*
     return FESC_OK;
 }
 
+// out = in + sum_k rot_k(in): c0 and the Galois images of c0 are summed here, c1 is copied; the key-switch part
+// is added by the division step.
+struct GaloisSet {
+    u64 g[8];
+    uint32_t n;
+};
+__global__ void __launch_bounds__(256) k_rotsum_prepare(const u64* __restrict__ in, size_t in_stride, u64* __restrict__ out,
+                                                        size_t out_stride, uint32_t log_n, uint32_t level, GaloisSet gs,
+                                                        const PrimeConst* __restrict__ pcs) {
+    const uint32_t N = 1u << log_n;
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t l = blockIdx.y, b = blockIdx.z;
+    if (t >= N) return;
+    const u64* ib = in + (size_t)b * in_stride;
+    u64* ob = out + (size_t)b * out_stride;
+    const u64 q = pcs[l].q;
+    u64 v = ib[(size_t)l * N + t];
+    for (uint32_t k = 0; k < gs.n; k++) v = addmod(v, ib[(size_t)l * N + galois_src(t, log_n, gs.g[k])], q);
+    ob[(size_t)l * N + t] = v;
+    ob[((size_t)level + l) * N + t] = ib[((size_t)level + l) * N + t];
+}
+
+// out[b] = in[b] + sum_k rot(in[b], key k): one decomposition per ciphertext, the inner products of all keys summed
+// on the extended basis, one division by P (in and out must not overlap; at most 8 keys).
+int rotate_sum_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, size_t out_stride,
+                                uint32_t batch, uint32_t level, const uint32_t* key_ids, uint32_t n_keys, u64* scratch,
+                                cudaStream_t st) {
+    if (n_keys == 0 || n_keys > 8) return fesc_fail(ctx, FESC_EINVAL, "rotate_sum_hoisted: 1 to 8 keys");
+    GaloisSet gs;
+    gs.n = n_keys;
+    for (uint32_t k = 0; k < n_keys; k++) {
+        if (!ctx->keys.count(key_ids[k]) || key_ids[k] == FESC_RELIN_KEY_ID)
+            return fesc_fail(ctx, FESC_ENOKEY, "rotate_sum_hoisted: no Galois key " + std::to_string(key_ids[k]));
+        gs.g[k] = ctx->keys[key_ids[k]].g;
+    }
+    const uint32_t chunk = ks_chunk(ctx, batch);
+    KsScratch ws = ks_scratch_carve(ctx, scratch, level, chunk);
+    for (uint32_t b0 = 0; b0 < batch; b0 += chunk) {
+        const uint32_t nb = batch - b0 < chunk ? batch - b0 : chunk;
+        dim3 g((ctx->N + 255) / 256, level, nb);
+        const u64* ib = in + (size_t)b0 * in_stride;
+        u64* ob = out + (size_t)b0 * out_stride;
+        prof_begin(ctx, PF_AUTOM, st);
+        k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, nullptr, 0, ws.d, ws.dcoef, ctx->log_n, level, 0);
+        k_rotsum_prepare<<<g, 256, 0, st>>>(ib, in_stride, ob, out_stride, ctx->log_n, level, gs, ctx->d_pc);
+        prof_end(ctx, PF_AUTOM, st, 2);
+        int rc = ks_decompose(ctx, ws, level, nb, st);
+        if (rc != FESC_OK) return rc;
+        for (uint32_t k = 0; k < n_keys; k++)
+            if ((rc = ks_inner(ctx, ws, ctx->keys[key_ids[k]], level, nb, st, gs.g[k], k > 0)) != FESC_OK) return rc;
+        if ((rc = ks_moddown(ctx, ws, level, nb, ob, out_stride, 3, st)) != FESC_OK) return rc;
+    }
+    return FESC_OK;
+}
+
+extern "C" int fesc_rotate_sum_hoisted(fesc_ctx* ctx, const uint64_t* d_in, uint64_t* d_out, uint32_t batch,
+                                       uint32_t n_limbs, const uint32_t* key_ids, uint32_t n_keys, void* stream) {
+    if (!ctx || !d_in || !d_out || !key_ids || d_in == d_out) return FESC_EINVAL;
+    if (n_limbs == 0 || n_limbs > ctx->n_q) return fesc_fail(ctx, FESC_ELEVEL, "rotate_sum_hoisted: level out of range");
+    if (batch == 0) return FESC_OK;
+    u64* scratch;
+    int rc = ctx_scratch(ctx, ks_scratch_words(ctx, n_limbs, ks_chunk(ctx, batch)) * sizeof(u64), &scratch);
+    if (rc != FESC_OK) return rc;
+    const size_t stride = (size_t)2 * n_limbs * ctx->N;
+    return rotate_sum_hoisted_internal(ctx, (const u64*)d_in, stride, (u64*)d_out, stride, batch, n_limbs, key_ids,
+                                       n_keys, scratch, (cudaStream_t)stream);
+}
+
 extern "C" int fesc_rotate_hoisted(fesc_ctx* ctx, const uint64_t* d_in, uint64_t* d_out, uint32_t batch,
                                    uint32_t n_limbs, const uint32_t* key_ids, uint32_t n_keys, void* stream) {
     if (!ctx || !d_in || !d_out || (!key_ids && n_keys)) return FESC_EINVAL;

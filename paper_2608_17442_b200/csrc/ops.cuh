@@ -20,6 +20,9 @@ int rotate_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, si
 int rotate_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, size_t out_stride,
                             size_t key_stride, uint32_t batch, uint32_t level, const uint32_t* key_ids, uint32_t n_keys,
                             u64* scratch, cudaStream_t st);
+int rotate_sum_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, size_t out_stride,
+                                uint32_t batch, uint32_t level, const uint32_t* key_ids, uint32_t n_keys, u64* scratch,
+                                cudaStream_t st);
 int giant_sum_deferred_internal(fesc_ctx* ctx, u64* acc, uint32_t n_terms, size_t ct_words, uint32_t batch,
                                 uint32_t level, uint32_t key_base, u64* scratch, cudaStream_t st);
 int rescale_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, uint32_t batch, uint32_t level,

@@ -231,23 +231,55 @@ struct Exec {
         rescale(t, out);
         top = mark;
     }
-    // a += rot(a, -unit * 2^b) for b = 0..steps-1
-    void fill_right(const Arr& a, uint32_t unit, uint32_t steps) {
+    bool key_ok(int64_t amount) {
+        uint32_t kid = key_for(amount);
+        if (ctx->keys.count(kid)) return true;
+        rc = fesc_fail(ctx, FESC_ENOKEY, "scan_contract: missing Galois key " + std::to_string(kid));
+        return false;
+    }
+    // a += rot(a, unit * 2^b) for b = 0..steps-1 (unit signed).  Hoisted mode takes steps (b, b+1) together:
+    // a + rot(a, d) + rot(a, 2d) + rot(a, 3d), d = unit * 2^b, with one decomposition and one division by P.
+    void chain(const Arr& a, int64_t unit, uint32_t steps) {
         size_t mark = top;
         Arr t = alloc(a.count, a.level);
-        for (uint32_t b = 0; b < steps; b++) {
-            rot(a, -(int64_t)(unit << b), t);
-            add(a, t, a);
+        uint32_t b = 0;
+        while (b < steps && ok()) {
+            const int64_t d = unit * (int64_t)(1u << b);
+            if (desc->hoist && b + 1 < steps) {
+                if (!key_ok(d) || !key_ok(2 * d) || !key_ok(3 * d)) break;
+                if (!dry) {
+                    const uint32_t ids[3] = {key_for(d), key_for(2 * d), key_for(3 * d)};
+                    rc = rotate_sum_hoisted_internal(ctx, a.p, a.stride, t.p, t.stride, a.count, a.level, ids, 3, ks, st);
+                    copy(t, a);
+                }
+                b += 2;
+            } else {
+                rot(a, d, t);
+                add(a, t, a);
+                b += 1;
+            }
         }
         top = mark;
     }
-    // out[t] = rot(src, unit * t) for t = 0..B-1, via t = t_lo + dg * t_hi
+    void fill_right(const Arr& a, uint32_t unit, uint32_t steps) { chain(a, -(int64_t)unit, steps); }
+    // out[t] = rot(src, unit * t) for t = 0..B-1, via t = t_lo + dg * t_hi (hoisted mode: the dg-1 low-digit
+    // rotations of one ciphertext share its decomposition)
     void extract_all(const Arr& src, int64_t unit, const Arr& out) {
         size_t mark = top;
         const uint32_t nh = g.B / g.dg;
         Arr gi = alloc(nh, src.level);
         for (uint32_t th = 0; th < nh; th++) rot(src, unit * (int64_t)(g.dg * th), at(gi, th));
-        for (uint32_t tl = 0; tl < g.dg; tl++) rot(gi, unit * (int64_t)tl, strided(out, tl, g.dg, nh));
+        if (desc->hoist && g.dg > 1) {
+            copy(gi, strided(out, 0, g.dg, nh));
+            std::vector<uint32_t> ids;
+            for (uint32_t tl = 1; tl < g.dg && ok(); tl++)
+                if (key_ok(unit * (int64_t)tl)) ids.push_back(key_for(unit * (int64_t)tl));
+            if (ok() && !dry)
+                rc = rotate_hoisted_internal(ctx, gi.p, gi.stride, out.p + out.stride, out.stride * g.dg, out.stride, nh,
+                                             src.level, ids.data(), (uint32_t)ids.size(), ks, st);
+        } else {
+            for (uint32_t tl = 0; tl < g.dg; tl++) rot(gi, unit * (int64_t)tl, strided(out, tl, g.dg, nh));
+        }
         top = mark;
     }
 };
@@ -419,10 +451,7 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
                 } else {
                     X.copy(v0, chi);
                 }
-                for (uint32_t b = 0; b < ilog2(g.d_s); b++) {
-                    X.rot(chi, (int64_t)(1u << b), tmp);
-                    X.add(chi, tmp, chi);
-                }
+                X.chain(chi, 1, ilog2(g.d_s));
                 Arr part = X.alloc(B, lred), y = X.alloc(B, lout), y2 = X.alloc(B, lout);
                 const uint32_t nparts = paired ? 2 : 1;
                 if (paired) X.conj(chi, tmp);

@@ -267,6 +267,25 @@ def test_rotate_hoisted(name, level, batch):
             assert np.array_equal(got[k, b], want[k]), (name, level, b, k)
 
 
+@pytest.mark.parametrize("name,level,batch,n_keys", [("toy", 6, 3, 3), ("toy", 5, 2, 1), ("small", 24, 9, 3),
+                                                     ("small", 9, 2, 2), ("wide", 6, 3, 3), ("full", 24, 2, 3)])
+def test_rotate_sum_hoisted(name, level, batch, n_keys):
+    """ct + sum_k rot_k(ct) with one decomposition and one division by P: residues equal the oracle's definition."""
+    import torch
+
+    pair = ctx_pair(name)
+    ctx, orc, _ = pair
+    rots = [(-2, 71), (-4, 72), (-6, 73)][:n_keys]
+    for r, kid in rots:
+        add_key(pair, r, kid)
+    ct = random_ct(orc, 12, level, level, batch)
+    out = torch.empty((batch, 2, level, orc.N), dtype=torch.int64, device="cuda")
+    ctx.rotate_sum_hoisted(to_dev(ct), out, batch, level, [k for _, k in rots])
+    got = to_host(out)
+    for b in range(batch):
+        assert np.array_equal(got[b], orc.rotate_sum_hoisted(ct[b], [k for _, k in rots])), (name, level, b)
+
+
 def test_integer_paths_with_primes_above_50_bits():
     """Primes of 52 and 55 bits take the integer kernels (wide-lazy transform at N = 2^16, 128-bit lazy
     accumulation in ModUp / inner product / ModDown); same bit-exact bar."""

@@ -13,7 +13,7 @@ from tests.gpu_util import ctx_pair, to_dev, to_host
 pytestmark = pytest.mark.gpu
 
 
-def _run(name, **kw):
+def _run(name, hoist=0, **kw):
     import torch
     import paper_2608_17442_b200 as fesc
 
@@ -22,15 +22,15 @@ def _run(name, **kw):
     l0 = p["n_q"]
     x, a, B, C = S.scan_inputs(p["seed"] + sh.L, sh.L, sh.H, sh.P, 1, sh.d_s)
     c = ScanConsts(orc, sh, l0, p["log_scale"])
-    add_scan_keys(orc, sh)
-    for r in sh.rotation_amounts() + [CONJ]:
+    add_scan_keys(orc, sh, hoist=bool(hoist))
+    for r in sh.rotation_amounts(bool(hoist)) + [CONJ]:
         ctx.add_galois_key(r, key_id_for(sh, r))
     ctX, ctA, ctB, ctC = encrypt_inputs(orc, sh, c, x, a, B, C)
-    want = ScanEvaluator(orc, sh, c).run(ctX, ctA, ctB, ctC)
+    want = ScanEvaluator(orc, sh, c, hoist=bool(hoist)).run(ctX, ctA, ctB, ctC)
     adj_s = [c.adj_s.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
     adj_p = [c.adj_p.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
     out = torch.empty((sh.K_blk, sh.K_s, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
-    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000)
+    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000, hoist)
     ctx.scan_contract(to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
                       to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out)
     ctx.sync()
@@ -40,16 +40,19 @@ def _run(name, **kw):
     return np.abs(m - float_recurrence(x, a, B, C)).max()
 
 
-def test_scan_paper_toy_shape():
-    assert _run("scan_toy", L=4, H=2, P=4, d_s=2, B_blk=4) < 2.0**-24
+@pytest.mark.parametrize("hoist", [0, 1])
+def test_scan_paper_toy_shape(hoist):
+    assert _run("scan_toy", hoist, L=4, H=2, P=4, d_s=2, B_blk=4) < 2.0**-24
 
 
-def test_scan_analogue_with_carries_and_partial_block():
-    assert _run("scan_small", L=40, H=8, P=4, d_s=8, B_blk=16) < 2.0**-22
+@pytest.mark.parametrize("hoist", [0, 1])
+def test_scan_analogue_with_carries_and_partial_block(hoist):
+    assert _run("scan_small", hoist, L=40, H=8, P=4, d_s=8, B_blk=16) < 2.0**-22
 
 
-def test_scan_two_digit_offsets_and_odd_chunk_count():
-    assert _run("scan_small", L=64, H=3, P=4, d_s=4, B_blk=32) < 2.0**-22
+@pytest.mark.parametrize("hoist", [0, 1])
+def test_scan_two_digit_offsets_and_odd_chunk_count(hoist):
+    assert _run("scan_small", hoist, L=64, H=3, P=4, d_s=4, B_blk=32) < 2.0**-22
 
 
 def test_scan_missing_key_is_reported():
@@ -64,7 +67,8 @@ def test_scan_missing_key_is_reported():
     assert e.value.code == fesc.ENOKEY
 
 
-def test_scan_deployed_geometry_decrypts_to_recurrence():
+@pytest.mark.parametrize("hoist", [1])
+def test_scan_deployed_geometry_decrypts_to_recurrence(hoist):
     """N = 2^16, 24 limbs, stride 256, B_blk = 256, d_s = 128, P = 64 (the Mamba-2-base geometry) on a slice of
     the model: 4 heads (one chunk pair) and 512 tokens (two blocks, so the carry and its injection run).
     The oracle cannot follow ~36 000 key switches at this ring size, so the check here is the property that
@@ -80,13 +84,13 @@ def test_scan_deployed_geometry_decrypts_to_recurrence():
     x, a, B, C = S.scan_inputs(S.config_seed(5), sh.L, sh.H, sh.P, 1, sh.d_s)
     c = ScanConsts(orc, sh, l0, 40)
     assert c.lv == dict(l0=24, l1=22, lS=14, linj=7, lout=4)
-    for r in sh.rotation_amounts() + [CONJ]:
+    for r in sh.rotation_amounts(bool(hoist)) + [CONJ]:
         ctx.add_galois_key(r, key_id_for(sh, r))
     ctX, ctA, ctB, ctC = encrypt_inputs(orc, sh, c, x, a, B, C)
     adj_s = [c.adj_s.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
     adj_p = [c.adj_p.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
     out = torch.empty((sh.K_blk, sh.K_s, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
-    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000)
+    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000, hoist)
     args = (to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
             to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out)
     ks0 = ctx.counters()[1]
