@@ -525,8 +525,15 @@ def run_scan(args):
     def step():
         ctx.scan_contract(x, a, Bc, Cc, desc, masks[0], masks[1], masks[2], masks[3][:linj - 2], adj, adj, out)
 
+    breakdown = None
     if args.workload == "scan_slice":
         step()                      # warm-up (sizes the scratch arena)
+        ctx.sync()
+        ctx.profile_enable(fesc.Context.PROFILE_FAMILIES, 600000)
+        step()                      # family breakdown on an untimed step
+        fam = ctx.profile_read()
+        ctx.profile_enable([])
+        breakdown = {k: {"ms": round(v[0], 1), "records": v[1]} for k, v in fam.items() if v[1]}
     ctx.sync()
     c0 = ctx.counters()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -544,7 +551,7 @@ def run_scan(args):
                                              % (args.workload, L, H, K_s,
                                                 "radix-4 hoisted rotate-and-add chains" if args.hoist else "plain rotations")},
                       "key_switches": ks, "limb_transforms": c1[0] - c0[0], "gpu_launches": c1[4] - c0[4],
-                      "scratch_gib": c1[3] / 2**30}), flush=True)
+                      "scratch_gib": c1[3] / 2**30, "kernel_breakdown": breakdown}), flush=True)
 
 
 def main():

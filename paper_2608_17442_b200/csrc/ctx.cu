@@ -360,8 +360,9 @@ extern "C" int fesc_ctx_create(fesc_ctx** out, uint32_t log_n, const uint64_t* p
             tw[(size_t)i * N + k] = make_ulonglong2(pw[r], h_shoup(pw[r], q));
             itw[(size_t)i * N + k] = make_ulonglong2(ipw[r], h_shoup(ipw[r], q));
             if (q < (1ull << 50)) {
-                twf[(size_t)i * N + k] = (double)pw[r];
-                itwf[(size_t)i * N + k] = (double)ipw[r];
+                // centred representatives (|w| <= q/2) halve the rounding term of the exact FP64 product
+                twf[(size_t)i * N + k] = pw[r] > q / 2 ? -(double)(q - pw[r]) : (double)pw[r];
+                itwf[(size_t)i * N + k] = ipw[r] > q / 2 ? -(double)(q - ipw[r]) : (double)ipw[r];
             }
         }
         pc.ninvw = h_mul(pc.ninv, ipw[h_brev(1, log_n)], q);

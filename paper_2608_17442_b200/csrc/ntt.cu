@@ -220,10 +220,14 @@ __device__ __forceinline__ uint32_t pad8(uint32_t e) { return e + (e >> 3); }
 // residue and every lazily reduced value below 2^53 is an exact double, and
 //     h = fl(y*w),  l = fma(y, w, -h)           (h + l = y*w exactly)
 //     c = rint(h * (1/q)),  v = fma(-c, q, h) + l (= y*w - c*q exactly, an integer below 2^53)
-// is an exact signed lazy product: |v| <= (1/2 + 3|y| 2^-53) q.  Sums and differences of such values are
-// exact while they stay below 2^53, so a butterfly is 8 FP64 operations.  With |inputs| <= q/2 three
-// forward stages stay below 3.5q and three inverse stages below 4q (< 8q <= 2^53); x - rint(x/q) q brings a
-// value back to |x| <= q/2 between register rounds.  The result equals the integer transform bit for bit.
+// is an exact signed lazy product: |v| <= (1/2 + 3|y w| 2^-53 / q) q, i.e. (1/2 + 1.5 |y| 2^-53) q with the
+// twiddles stored as centred doubles (|w| <= q/2).  Sums and differences of such values are exact while they
+// stay below 2^53 = 8q.  Forward (Cooley-Tukey: x +- v, bound B -> 1.1875 B + q/2 per stage): from q/2 the bound
+// after 1..7 stages is 1.10, 1.80, 2.64, 3.63, 4.81, 6.21, 7.88 q, and from a canonical input (below q) three
+// stages reach 3.47q; so the strided kernel folds back once after its first round and once at the end, the
+// contiguous kernel once after its first round.  Inverse (Gentleman-Sande: x + v doubles the bound): three
+// stages from q/2 reach 4q, so every round ends with a fold-back x - rint(x/q) q to |x| <= q/2.
+// The result equals the integer transform bit for bit.
 // The two kernels of one transform hand the data over as doubles in the caller's buffer.
 // ---------------------------------------------------------------------------------------
 #define FP_LIMIT FESC_FP_LIMIT
@@ -238,15 +242,21 @@ __device__ __forceinline__ void fp_gs(double& x, double& y, double w, double q, 
     x = u + v;
     y = fp_modmul(u - v, w, q, qinv);
 }
+// idxB is even and idxC a multiple of 4 at every call site: 16-byte loads
+__device__ __forceinline__ double2 ldf2(const double* __restrict__ t, uint32_t i) {
+    return __ldg(reinterpret_cast<const double2*>(t + i));
+}
 __device__ __forceinline__ void fp_fwd_round2(double (&x)[8], const double* __restrict__ tw, uint32_t idxB, uint32_t idxC,
                                               double q, double qinv) {
-    const double b0 = ldf(tw, idxB), b1 = ldf(tw, idxB + 1);
-    fp_ct(x[0], x[2], b0, q, qinv);
-    fp_ct(x[1], x[3], b0, q, qinv);
-    fp_ct(x[4], x[6], b1, q, qinv);
-    fp_ct(x[5], x[7], b1, q, qinv);
-#pragma unroll
-    for (int k = 0; k < 4; k++) fp_ct(x[2 * k], x[2 * k + 1], ldf(tw, idxC + k), q, qinv);
+    const double2 b = ldf2(tw, idxB), c0 = ldf2(tw, idxC), c1 = ldf2(tw, idxC + 2);
+    fp_ct(x[0], x[2], b.x, q, qinv);
+    fp_ct(x[1], x[3], b.x, q, qinv);
+    fp_ct(x[4], x[6], b.y, q, qinv);
+    fp_ct(x[5], x[7], b.y, q, qinv);
+    fp_ct(x[0], x[1], c0.x, q, qinv);
+    fp_ct(x[2], x[3], c0.y, q, qinv);
+    fp_ct(x[4], x[5], c1.x, q, qinv);
+    fp_ct(x[6], x[7], c1.y, q, qinv);
 }
 __device__ __forceinline__ void fp_fwd_round3(double (&x)[8], const double* __restrict__ tw, uint32_t idxA, uint32_t idxB,
                                               uint32_t idxC, double q, double qinv) {
@@ -257,13 +267,15 @@ __device__ __forceinline__ void fp_fwd_round3(double (&x)[8], const double* __re
 }
 __device__ __forceinline__ void fp_inv_round2(double (&x)[8], const double* __restrict__ tw, uint32_t idxB, uint32_t idxC,
                                               double q, double qinv) {
-#pragma unroll
-    for (int k = 0; k < 4; k++) fp_gs(x[2 * k], x[2 * k + 1], ldf(tw, idxC + k), q, qinv);
-    const double b0 = ldf(tw, idxB), b1 = ldf(tw, idxB + 1);
-    fp_gs(x[0], x[2], b0, q, qinv);
-    fp_gs(x[1], x[3], b0, q, qinv);
-    fp_gs(x[4], x[6], b1, q, qinv);
-    fp_gs(x[5], x[7], b1, q, qinv);
+    const double2 b = ldf2(tw, idxB), c0 = ldf2(tw, idxC), c1 = ldf2(tw, idxC + 2);
+    fp_gs(x[0], x[1], c0.x, q, qinv);
+    fp_gs(x[2], x[3], c0.y, q, qinv);
+    fp_gs(x[4], x[5], c1.x, q, qinv);
+    fp_gs(x[6], x[7], c1.y, q, qinv);
+    fp_gs(x[0], x[2], b.x, q, qinv);
+    fp_gs(x[1], x[3], b.x, q, qinv);
+    fp_gs(x[4], x[6], b.y, q, qinv);
+    fp_gs(x[5], x[7], b.y, q, qinv);
 }
 __device__ __forceinline__ void fp_inv_round3(double (&x)[8], const double* __restrict__ tw, uint32_t idxA, uint32_t idxB,
                                               uint32_t idxC, double q, double qinv) {
@@ -286,16 +298,15 @@ __device__ __forceinline__ void strided_body_fp(u64* __restrict__ p, double* __r
     double x[8];
     if (!INV) {
 #pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = fp_load(p[(size_t)(k * 32 + sub) * 256 + col], q);
-        fp_fwd_round3(x, tw, 1, 2, 4, q, qinv);
+        for (int k = 0; k < 8; k++) x[k] = fp_from_u64(p[(size_t)(k * 32 + sub) * 256 + col]);   // canonical, below q
+        fp_fwd_round3(x, tw, 1, 2, 4, q, qinv);                                                  // below 3.47q
         fp_reduce8(x, q, qinv);
 #pragma unroll
         for (int k = 0; k < 8; k++) sm[(k * 32 + sub) * NTT_COLS + col] = x[k];
         __syncthreads();
 #pragma unroll
         for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * NTT_COLS + col];
-        fp_fwd_round3(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, qinv);
-        fp_reduce8(x, q, qinv);
+        fp_fwd_round3(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, qinv);                        // below 2.64q, 4.81q next
 #pragma unroll
         for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * NTT_COLS + col] = x[k];
         __syncthreads();
@@ -362,8 +373,7 @@ __device__ __forceinline__ void contig_body_fp(u64* __restrict__ p, double* __re
         __syncwarp();
 #pragma unroll
         for (int k = 0; k < 8; k++) x[k] = sm[pad8(h2 * 32 + k * 4 + l2)];
-        fp_fwd_round3(x, tw, 8 * pre + h2, 16 * pre + 2 * h2, 32 * pre + 4 * h2, q, qinv);
-        fp_reduce8(x, q, qinv);
+        fp_fwd_round3(x, tw, 8 * pre + h2, 16 * pre + 2 * h2, 32 * pre + 4 * h2, q, qinv);   // below 2.64q, 4.81q next
         __syncwarp();
 #pragma unroll
         for (int k = 0; k < 8; k++) sm[pad8(h2 * 32 + k * 4 + l2)] = x[k];
