@@ -412,6 +412,40 @@ class Oracle:
                 out[tb, b] = self.rescale(y)
         return out
 
+    # ---- causal depthwise convolution (Sec. "Causal Depthwise Convolution", Eq. conv1d_depthwise) ------------
+    def conv(self, ct_in, masks, bias, d_conv: int, T: int, key_base: int):
+        """eta = b + sum_r M_r (.) rho(q; delta_r) on the projection packing idx(token, channel) = channel*T + token.
+
+        ct_in  [token_blocks, blocks, 2, l, N]   q of every (token block, channel block)
+        masks  [blocks, 2*d_conv - 1, l, N]      M_0..M_{d-1}, then M'_1..M'_{d-1} (tap weight times causal mask)
+        bias   [blocks, l, N]                    encoded at the scale of the products
+        returns [token_blocks, blocks, 2, l-1, N].
+        Tap r >= 1 of token k reads token k-r: inside the block that is rho(q; -r) masked to tokens k >= r (M_r); the
+        first r tokens read the previous block's last tokens, rho(q_prev; T - r) masked to k < r (M'_r; absent for the
+        first block: q_t = 0 for t < 0).  The 2(d_conv-1) rotations of one ciphertext use `rotate_hoisted`; key ids:
+        key_base + r for -r, key_base + d_conv + r for T - r."""
+        tbs, blocks = ct_in.shape[0], ct_in.shape[1]
+        level = ct_in.shape[3]
+        data = list(range(level))
+        out = np.empty((tbs, blocks, 2, level - 1, self.N), dtype=np.uint64)
+        taps = list(range(1, d_conv))
+        prev = None
+        for tb in range(tbs):
+            ids = [key_base + r for r in taps] + ([key_base + d_conv + r for r in taps] if tb + 1 < tbs else [])
+            cur = []
+            for b in range(blocks):
+                rots = self.rotate_hoisted(ct_in[tb, b], ids) if ids else []
+                acc = self.ct_pt_mac(ct_in[tb, b], masks[b, 0], np.zeros((2, level, self.N), dtype=np.uint64))
+                for i, r in enumerate(taps):
+                    acc = self.ct_pt_mac(rots[i], masks[b, r], acc)
+                    if prev is not None:
+                        acc = self.ct_pt_mac(prev[b][i], masks[b, d_conv - 1 + r], acc)
+                acc[0] = self.add(acc[0], _arr(bias[b]), data)
+                out[tb, b] = self.rescale(acc)
+                cur.append(rots[len(taps):])
+            prev = cur if tb + 1 < tbs else None
+        return out
+
     # ---- harness: encode / decode / encrypt / decrypt ---------------------------------
     def _slot_index(self):
         idx = np.empty(self.n, dtype=np.int64)
@@ -504,3 +538,21 @@ def linear_diagonal(W, b: int, g: int, p: int, q: int, T: int, C: int, n1: int) 
     vals = np.zeros(C)
     vals[ok] = W[rows[ok], cols[ok]]
     return np.repeat(vals, T)
+
+
+def conv_masks(w, b_conv, blk: int, T: int, C: int, n: int):
+    """Slot vectors of one channel block for `Oracle.conv`: w [channels, d_conv] tap weights, b_conv [channels].
+    Returns (M [2*d_conv-1, n], bias [n]): M_r[c*T+k] = w[c,r] for k >= r, M'_r[c*T+k] = w[c,r] for k < r."""
+    channels, d_conv = w.shape
+    M = np.zeros((2 * d_conv - 1, n))
+    bias = np.zeros(n)
+    for c in range(C):
+        ch = blk * C + c
+        if ch >= channels:
+            break
+        bias[c * T:(c + 1) * T] = b_conv[ch]
+        for r in range(d_conv):
+            M[r, c * T + r:(c + 1) * T] = w[ch, r]
+            if r >= 1:
+                M[d_conv - 1 + r, c * T:c * T + r] = w[ch, r]
+    return M, bias
