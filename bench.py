@@ -554,6 +554,58 @@ def run_scan(args):
                       "scratch_gib": c1[3] / 2**30, "kernel_breakdown": breakdown}), flush=True)
 
 
+def run_conv(args):
+    """Times fesc_conv on synthetic residues of the Mamba-2-base shape: the xBC channels (1536 + 2*128 = 1792 = 7
+    channel blocks of 256) x 2048 tokens (16 token blocks of 128), d_conv = 4, 24 limbs."""
+    import torch
+    import fesc_synth as S
+    import paper_2608_17442_b200 as fesc
+
+    torch.cuda.set_device(0)
+    p = S.params("full")
+    ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+    N = ctx.N
+    d_conv, T, blocks, tbs, level, base = 4, T_SEG, 7, 16, LEVEL, 3000
+    for r in range(1, d_conv):
+        ctx.add_galois_key(-r, base + r)
+        ctx.add_galois_key(T - r, base + d_conv + r)
+    seed = S.config_seed(5)
+    q = p["primes"][:level]
+    r = S.hashed_residues(seed, 21, q, tbs * blocks * 2 * N, device="cuda")
+    ct = r.view(level, tbs, blocks, 2, N).permute(1, 2, 3, 0, 4).contiguous()
+    r = S.hashed_residues(seed, 22, q, blocks * (2 * d_conv - 1) * N, device="cuda")
+    masks = r.view(level, blocks, 2 * d_conv - 1, N).permute(1, 2, 0, 3).contiguous()
+    r = S.hashed_residues(seed, 23, q, blocks * N, device="cuda")
+    bias = r.view(level, blocks, N).permute(1, 0, 2).contiguous()
+    del r
+    out = torch.empty((tbs, blocks, 2, level - 1, N), dtype=torch.int64, device="cuda")
+    desc = fesc.ConvDesc(d_conv, T, blocks, tbs, level, base)
+    for _ in range(max(3, args.warmup)):
+        ctx.conv(ct, masks, bias, desc, out)
+    ctx.profile_enable(fesc.Context.PROFILE_FAMILIES, 60000)
+    ctx.conv(ct, masks, bias, desc, out)
+    fam = ctx.profile_read()
+    ctx.profile_enable([])
+    c0 = ctx.counters()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        ctx.conv(ct, masks, bias, desc, out)
+    e1.record()
+    ctx.sync()
+    c1 = ctx.counters()
+    ms = e0.elapsed_time(e1) / args.steps
+    ks = (c1[1] - c0[1]) // args.steps
+    print(json.dumps({"metric": "causal depthwise convolution latency; key-switches/s", "value": ks / (ms * 1e-3),
+                      "unit": "key-switches/s", "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup),
+                      "ms_per_step": ms, "higher_is_better": True, "dtype": "u64", "data": "synthetic",
+                      "config": {"workload": "conv: 1792 channels x 2048 tokens, d_conv=4, T=128, 7 channel blocks x 16 "
+                                             "token blocks, N=2^16, 24 limbs, hoisted rotations"},
+                      "key_switches_per_step": ks, "gpu_launches": (c1[4] - c0[4]) // args.steps,
+                      "kernel_breakdown": {k: {"ms": round(v[0], 2), "records": v[1]} for k, v in fam.items() if v[1]}}),
+          flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -570,9 +622,11 @@ def main():
                     help="1: one division by P per output for the whole giant-step sum")
     ap.add_argument("--hoist", type=int, default=1, choices=[0, 1],
                     help="1: baby rotations share one decomposition per input ciphertext (fesc_rotate_hoisted)")
-    ap.add_argument("--workload", default="in_proj", choices=["in_proj", "scan_slice", "scan_layer"],
-                    help="in_proj (default, the benchmark metric) or a scan-contract run")
+    ap.add_argument("--workload", default="in_proj", choices=["in_proj", "scan_slice", "scan_layer", "conv"],
+                    help="in_proj (default, the benchmark metric), a scan-contract run or the depthwise convolution")
     args = ap.parse_args()
+    if args.workload == "conv":
+        return run_conv(args)
     if args.workload != "in_proj":
         return run_scan(args)
     if args.impl == "reference":

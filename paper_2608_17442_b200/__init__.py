@@ -33,6 +33,10 @@ class BsgsDesc(ctypes.Structure):
                  "hoist", "defer")]
 
 
+class ConvDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint32) for n in ("d_conv", "T", "blocks", "token_blocks", "n_limbs", "key_base")]
+
+
 class ScanDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint32) for n in ("L", "H", "P", "d_s", "B_blk", "stride", "n_limbs", "key_base",
                                                        "hoist")]
@@ -68,6 +72,7 @@ def lib():
             "fesc_rotate": [vp, vp, vp, u32, u32, u32, vp],
             "fesc_rotate_hoisted": [vp, vp, vp, u32, u32, c.POINTER(u32), u32, vp],
             "fesc_rotate_sum_hoisted": [vp, vp, vp, u32, u32, c.POINTER(u32), u32, vp],
+            "fesc_conv": [vp, vp, vp, vp, c.POINTER(ConvDesc), vp, vp],
             "fesc_rescale": [vp, vp, vp, u32, u32, vp],
             "fesc_rescale_static": [vp, vp, vp, u32, u32, vp],
             "fesc_ct_ct_mul": [vp, vp, vp, vp, u32, u32, vp],
@@ -184,6 +189,9 @@ class Context:
 
     def rotate(self, ct_in, ct_out, batch: int, n_limbs: int, key_id: int):
         self._chk(lib().fesc_rotate(self.h, _ptr(ct_in), _ptr(ct_out), batch, n_limbs, key_id, _stream()))
+
+    def conv(self, ct_in, masks, bias, desc: "ConvDesc", ct_out):
+        self._chk(lib().fesc_conv(self.h, _ptr(ct_in), _ptr(masks), _ptr(bias), ctypes.byref(desc), _ptr(ct_out), _stream()))
 
     def rotate_sum_hoisted(self, ct_in, ct_out, batch: int, n_limbs: int, key_ids):
         ids = (ctypes.c_uint32 * len(key_ids))(*key_ids)
