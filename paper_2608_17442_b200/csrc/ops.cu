@@ -222,8 +222,8 @@ __global__ void __launch_bounds__(256, (BT >= 8 ? 2 : INNER_MINB)) k_inner(const
         for (int i = 0; i < BT; i++) x[i] = (j == own) ? *op[i] : xp[i][(size_t)j * xstride];
     };
     if (PATH == 1 || (PATH == 0 && pcs[pt].q < FESC_FP_LIMIT)) {
-        // exact FP64 products: |x| <= q/2, key words in [0,q); up to 8 terms of at most 0.7q (plus a running sum
-        // of at most q/2) stay below 2^53, longer sums are folded back every 8 digits.  The next digit's words
+        // exact FP64 products of canonical words (both below q): every product is below 0.875q, so a running sum of
+        // at most q/2 plus 7 terms stays below 2^53 = 8q; longer sums are folded back after every 7th digit.  The next digit's words
         // are requested before this digit's products start: 2 + BT loads in flight per thread, few registers,
         // so that three or four CTAs per SM overlap their loads and products (measured: one digit ahead with
         // 4 CTAs per SM moves 1.5x the bytes per second of all-digits-up-front with 2).
@@ -246,11 +246,11 @@ __global__ void __launch_bounds__(256, (BT >= 8 ? 2 : INNER_MINB)) k_inner(const
             const double dkb = fp_from_u64(kb), dka = fp_from_u64(ka);
 #pragma unroll
             for (int i = 0; i < BT; i++) {
-                const double xd = fp_load(x[i], q);
+                const double xd = fp_from_u64(x[i]);   // canonical operands: every product is below 0.875q
                 f0[i] += fp_modmul(xd, dkb, q, qinv);
                 f1[i] += fp_modmul(xd, dka, q, qinv);
             }
-            if ((j & 7) == 6) {   // before the 8th term since the last fold (a running sum may be included)
+            if ((j & 7) == 6) {   // q/2 (a running sum) + 7 terms stay below 6.7q; fold before the 8th
 #pragma unroll
                 for (int i = 0; i < BT; i++) {
                     f0[i] = fp_reduce(f0[i], q, qinv);
