@@ -346,6 +346,20 @@ class Oracle:
         m_eval = self.ntt(self.signed_to_rns(mono, data), data)
         return np.stack([self.mul(ct[p], m_eval, data) for p in range(2)])
 
+    def split_complex(self, ct, conj_key_id: int):
+        """Real and imaginary slot parts of a complex-packed ciphertext, each doubled (exact, no rescale):
+            re2 = ct + conj(ct)            (slots 2 Re z)
+            im2 = -i (ct - conj(ct))       (slots 2 Im z;  -i = X^(N/2) three times)
+        with conj = the rotation under the conjugation key.  Used to run a real-weight projection on two token
+        blocks at once (App. "Projection Kernel Breakdown": pairing in the real and imaginary channels)."""
+        level = ct.shape[1]
+        data = list(range(level))
+        bar = self.rotate(ct, conj_key_id)
+        re2 = self.ct_add(ct, bar)
+        diff = np.stack([self.sub(ct[p], bar[p], data) for p in range(2)])
+        im2 = self.mul_monomial_half(self.mul_monomial_half(self.mul_monomial_half(diff)))
+        return re2, im2
+
     # ---- BSGS projection -----------------------------------------------------------
     def giant_sum_deferred(self, accs, giant_key_ids):
         """sum_p rot(acc_p, giant step p) with ONE division by P for the whole sum (a separately defined mode):

@@ -302,3 +302,15 @@ def test_rotate_sum_hoisted_is_the_sum_of_rotations(toy_oracle):
     # a single rotation: exactly ct + rotate_hoisted
     one = o.rotate_sum_hoisted(ct, [42])
     assert np.array_equal(one, o.ct_add(ct, o.rotate_hoisted(ct, [42])[0]))
+
+
+def test_split_complex_returns_doubled_real_and_imaginary_parts(toy_oracle):
+    o = toy_oracle
+    scale = 2.0**20
+    z = S.uniform_slots(16, 0, 2, o.n)
+    o.add_galois_key(CONJ, 47)
+    ct = o.encrypt(o.encode(z[0] + 1j * z[1], scale, 4), 21)
+    re2, im2 = o.split_complex(ct, 47)
+    assert np.abs(o.decrypt(re2, scale) - 2 * z[0]).max() < 3e-4
+    assert np.abs(o.decrypt(im2, scale) - 2 * z[1]).max() < 3e-4
+    assert np.abs(o.decrypt(re2, scale).imag).max() < 3e-4 and np.abs(o.decrypt(im2, scale).imag).max() < 3e-4
