@@ -73,6 +73,7 @@ def lib():
             "fesc_rotate_hoisted": [vp, vp, vp, u32, u32, c.POINTER(u32), u32, vp],
             "fesc_rotate_sum_hoisted": [vp, vp, vp, u32, u32, c.POINTER(u32), u32, vp],
             "fesc_conv": [vp, vp, vp, vp, c.POINTER(ConvDesc), vp, vp],
+            "fesc_split_complex": [vp, vp, vp, vp, u32, u32, u32, vp],
             "fesc_rescale": [vp, vp, vp, u32, u32, vp],
             "fesc_rescale_static": [vp, vp, vp, u32, u32, vp],
             "fesc_ct_ct_mul": [vp, vp, vp, vp, u32, u32, vp],
@@ -189,6 +190,9 @@ class Context:
 
     def rotate(self, ct_in, ct_out, batch: int, n_limbs: int, key_id: int):
         self._chk(lib().fesc_rotate(self.h, _ptr(ct_in), _ptr(ct_out), batch, n_limbs, key_id, _stream()))
+
+    def split_complex(self, ct_in, re2, im2, batch: int, n_limbs: int, conj_key_id: int):
+        self._chk(lib().fesc_split_complex(self.h, _ptr(ct_in), _ptr(re2), _ptr(im2), batch, n_limbs, conj_key_id, _stream()))
 
     def conv(self, ct_in, masks, bias, desc: "ConvDesc", ct_out):
         self._chk(lib().fesc_conv(self.h, _ptr(ct_in), _ptr(masks), _ptr(bias), ctypes.byref(desc), _ptr(ct_out), _stream()))

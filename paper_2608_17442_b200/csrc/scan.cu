@@ -537,3 +537,33 @@ extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint
     X.rs = X.ks + ks_words;
     return scan_run(X, (const u64*)d_x, (const u64*)d_a, (const u64*)d_B, (const u64*)d_C, (u64*)d_m_out);
 }
+
+// ---------------------------------------------------------------------------------------
+// Real and imaginary slot parts of complex-packed ciphertexts, each doubled:
+//   re2 = ct + conj(ct),  im2 = -i (ct - conj(ct))   (-i = the monomial X^(N/2) applied three times, exact).
+// ---------------------------------------------------------------------------------------
+extern "C" int fesc_split_complex(fesc_ctx* ctx, const uint64_t* d_in, uint64_t* d_re2, uint64_t* d_im2, uint32_t batch,
+                                  uint32_t n_limbs, uint32_t conj_key_id, void* stream) {
+    if (!ctx || !d_in || !d_re2 || !d_im2 || d_in == d_re2 || d_in == d_im2 || d_re2 == d_im2) return FESC_EINVAL;
+    if (n_limbs == 0 || n_limbs > ctx->n_q) return fesc_fail(ctx, FESC_ELEVEL, "split_complex: level out of range");
+    if (batch == 0) return FESC_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    const uint32_t N = ctx->N;
+    const size_t ctw = (size_t)2 * n_limbs * N;
+    u64* scratch;
+    int rc = ctx_scratch(ctx, ks_scratch_words(ctx, n_limbs, ks_chunk(ctx, batch)) * sizeof(u64), &scratch);
+    if (rc != FESC_OK) return rc;
+    const u64* in = (const u64*)d_in;
+    u64 *re = (u64*)d_re2, *im = (u64*)d_im2;
+    // conj(ct) into re, then im = ct - conj, re = ct + conj, im *= -i
+    rc = rotate_internal(ctx, in, ctw, re, ctw, batch, n_limbs, conj_key_id, scratch, st, 0);
+    if (rc != FESC_OK) return rc;
+    const dim3 g((N + 255) / 256, 2 * n_limbs, batch);
+    prof_begin(ctx, PF_POINTWISE, st);
+    k_ct_addsub<<<g, 256, 0, st>>>(in, ctw, re, ctw, im, ctw, ctx->d_pc, N, n_limbs, 1);
+    k_ct_addsub<<<g, 256, 0, st>>>(in, ctw, re, ctw, re, ctw, ctx->d_pc, N, n_limbs, 0);
+    k_ct_mul_i<<<g, 256, 0, st>>>(im, ctw, im, ctw, ctx->d_pc, ctx->d_tw, N, n_limbs, 3);
+    prof_end(ctx, PF_POINTWISE, st, 3);
+    FESC_CHECK_CUDA(ctx, cudaGetLastError());
+    return FESC_OK;
+}

@@ -108,6 +108,57 @@ def test_linear_accumulate_extreme_residues_256_terms():
         assert np.array_equal(got, want)
 
 
+def test_linear_on_complex_paired_token_blocks():
+    """Two token blocks in the real and imaginary channels of one ciphertext, real diagonals: one projection and one
+    conjugation per output give both results (residues bit-exact against the oracle, values against X @ W)."""
+    import torch
+    from oracle.ckks import CONJ
+
+    pair = ctx_pair("small")
+    ctx, orc, p = pair
+    T, C, n1, n2, level, scale = 32, 16, 4, 4, 5, 2.0**40
+    tokens, d_in, d_out, kb = 4 * T, 40, 50, 8000
+    n = orc.n
+    X, W = S.linear_inputs(p["seed"] + 9, tokens, d_in, d_out)
+    W = W * 10.0
+    gin, nout, pairs = -(-d_in // C), -(-d_out // C), tokens // (2 * T)
+    for q in range(1, n1):
+        add_key(pair, q * T, kb + q)
+    for g in range(1, n2):
+        add_key(pair, g * n1 * T, kb + 500 + g)
+    add_key(pair, CONJ, kb + 999)
+    cts = np.empty((pairs, gin, 2, level, orc.N), dtype=np.uint64)
+    for u in range(pairs):
+        for g in range(gin):
+            v0 = pack_linear_input(X[(2 * u) * T:(2 * u + 1) * T, g * C:(g + 1) * C], T, C, n)
+            v1 = pack_linear_input(X[(2 * u + 1) * T:(2 * u + 2) * T, g * C:(g + 1) * C], T, C, n)
+            cts[u, g] = orc.encrypt(orc.encode(v0 + 1j * v1, scale, level), 7700 + u * gin + g)
+    diags = np.empty((nout, n2, gin, n1, level, orc.N), dtype=np.uint64)
+    for b in range(nout):
+        for pp in range(n2):
+            for g in range(gin):
+                for q in range(n1):
+                    diags[b, pp, g, q] = orc.encode(linear_diagonal(W, b, g, pp, q, T, C, n1), float(orc.q[level - 1]), level)
+    got = _run_gpu(ctx, cts, diags, n1, n2, (gin, nout, pairs), level, key_base=kb, hoist=1, defer=1)
+    want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)},
+                      {g: kb + 500 + g for g in range(1, n2)}, hoist=True, defer=True)
+    assert np.array_equal(got, want)
+    batch = pairs * nout
+    z = to_dev(got.reshape(batch, 2, level - 1, orc.N))
+    re2, im2 = torch.empty_like(z), torch.empty_like(z)
+    ctx.split_complex(z, re2, im2, batch, level - 1, kb + 999)
+    re2, im2 = to_host(re2), to_host(im2)
+    Y = X @ W
+    for u in range(pairs):
+        for b in range(nout):
+            wr, wi = orc.split_complex(want[u, b], kb + 999)
+            assert np.array_equal(re2[u * nout + b], wr) and np.array_equal(im2[u * nout + b], wi)
+            cols = slice(b * C, min((b + 1) * C, d_out))
+            for part, tb in ((wr, 2 * u), (wi, 2 * u + 1)):
+                y = orc.decrypt(part, 2 * scale, 2).real.reshape(C, T).T
+                assert np.abs(y[:, :cols.stop - cols.start] - Y[tb * T:(tb + 1) * T, cols]).max() < 2.0**-18
+
+
 def test_linear_integer_kernels_with_55_bit_primes():
     """The 128-bit integer accumulate kernel (primes above 50 bits) against the oracle."""
     pair = ctx_pair("wide")
