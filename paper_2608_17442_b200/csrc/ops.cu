@@ -74,8 +74,19 @@ __device__ __forceinline__ uint32_t galois_src(uint32_t t, uint32_t log_n, u64 g
     uint32_t e = (uint32_t)(((2ull * u + 1) * g) & ((2ull << log_n) - 1));
     return __brev((e - 1) >> 1) >> (32 - log_n);
 }
+// Where the EVAL-form polynomial being switched is kept: the rows of the extended-digit buffer that belong to a
+// digit's own limbs (row l of digit l / alpha), which the basis extension leaves untouched.  The inner product then
+// reads every (digit, row) from one array.
+struct OwnRows {
+    u64* ext;
+    uint32_t alpha, beta, rows;
+};
+__device__ __forceinline__ size_t own_index(const OwnRows& w, uint32_t b, uint32_t l, uint32_t N) {
+    return (((size_t)b * w.beta + l / w.alpha) * w.rows + l) * N;
+}
+struct KsScratch;
 __global__ void __launch_bounds__(256) k_autom_ct(const u64* __restrict__ in, size_t in_stride, u64* __restrict__ out0,
-                                                  size_t out_stride, u64* __restrict__ d, u64* __restrict__ dcoef,
+                                                  size_t out_stride, OwnRows d, u64* __restrict__ dcoef,
                                                   uint32_t log_n, uint32_t level, u64 g,
                                                   const PrimeConst* __restrict__ pcs, int accumulate) {
     const uint32_t N = 1u << log_n;
@@ -90,9 +101,8 @@ __global__ void __launch_bounds__(256) k_autom_ct(const u64* __restrict__ in, si
     if (accumulate) v0 = addmod(v0, *o0, pcs[l].q);
     *o0 = v0;
     u64 v = ib[poly + (size_t)l * N + src];
-    const size_t o = ((size_t)b * level + l) * N + t;
-    d[o] = v;
-    dcoef[o] = v;
+    d.ext[own_index(d, b, l, N) + t] = v;
+    dcoef[((size_t)b * level + l) * N + t] = v;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -190,7 +200,7 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
 // PATH 0: the row's prime decides at run time; 1: the caller guarantees primes below 2^50 on rows
 // [row0, row0 + gridDim.y) (exact FP64 products only); 2: the caller sends those rows to the 128-bit integer sums.
 template <int BT, int PATH>
-__global__ void __launch_bounds__(256, (BT >= 8 ? 2 : INNER_MINB)) k_inner(const u64* __restrict__ d, const u64* __restrict__ ext,
+__global__ void __launch_bounds__(256, (BT >= 8 ? 2 : INNER_MINB)) k_inner(const u64* __restrict__ ext,
                                                const u64* __restrict__ key, u64* __restrict__ acc,
                                                const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
                                                uint32_t n_q, uint32_t K, uint32_t alpha, uint32_t beta,
@@ -202,24 +212,21 @@ __global__ void __launch_bounds__(256, (BT >= 8 ? 2 : INNER_MINB)) k_inner(const
     const uint32_t cs = g ? galois_src(c, log_n, g) : c;
     const uint32_t rows = level + K, np = n_q + K;
     const uint32_t pt = t < level ? t : n_q + (t - level);
-    const uint32_t own = t < level ? t / alpha : 0xFFFFFFFFu;
     // operand words of one digit: key (b, a) and the BT ciphertext words; clamped indices keep loads valid.
     // All addresses are a per-thread base plus a multiple of one stride (no per-load index products).
     const size_t kstride = (size_t)np * N, xstride = (size_t)rows * N;
     const u64* kp = key + (size_t)pt * N + c;
     const u64* xp[BT];
-    const u64* op[BT];
 #pragma unroll
     for (int i = 0; i < BT; i++) {
         const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
         xp[i] = ext + ((size_t)b * beta * rows + t) * N + cs;
-        op[i] = d + ((size_t)b * level + (t < level ? t : 0)) * N + cs;
     }
     auto load_digit = [&](uint32_t j, u64& kb, u64& ka, u64 (&x)[BT]) {
         kb = __ldg(kp + (size_t)(2 * j) * kstride);
         ka = __ldg(kp + (size_t)(2 * j + 1) * kstride);
 #pragma unroll
-        for (int i = 0; i < BT; i++) x[i] = (j == own) ? *op[i] : xp[i][(size_t)j * xstride];
+        for (int i = 0; i < BT; i++) x[i] = xp[i][(size_t)j * xstride];
     };
     if (PATH == 1 || (PATH == 0 && pcs[pt].q < FESC_FP_LIMIT)) {
         // exact FP64 products of canonical words (both below q): every product is below 0.875q, so a running sum of
@@ -344,7 +351,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 }
 
 template <int BT>
-__global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ d, const u64* __restrict__ ext,
+__global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ ext,
                                                       const u64* __restrict__ key, u64* __restrict__ acc,
                                                       const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
                                                       uint32_t n_q, uint32_t K, uint32_t alpha, uint32_t beta,
@@ -373,7 +380,6 @@ __global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ d,
         uint32_t t, cblk, b0;
         decode(tile, t, cblk, b0);
         const uint32_t pt = t < level ? t : n_q + (t - level);
-        const uint32_t own = t < level ? t / alpha : 0xFFFFFFFFu;
         const uint32_t sblk = g ? (galois_src(cblk << 8, log_n, g) >> 8) : cblk;
         const uint32_t bar = bar0 + stage * 8;
         uint32_t dst = sbase + stage * stage_words * 8;
@@ -386,7 +392,7 @@ __global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ d,
 #pragma unroll
             for (int i = 0; i < BT; i++) {
                 const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
-                const u64* src = (j == own) ? d + ((size_t)b * level + t) * N : ext + (((size_t)b * beta + j) * rows + t) * N;
+                const u64* src = ext + (((size_t)b * beta + j) * rows + t) * N;
                 bulk_g2s(dst, src + (sblk << 8), 2048, bar);
                 dst += 2048;
             }
@@ -648,7 +654,7 @@ static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint
 #define INNER(BT_, PATH_, ROW0_, NROWS_)                                                                        \
     do {                                                                                                        \
         dim3 gd(gx, NROWS_, (batch + BT_ - 1) / BT_);                                                           \
-        k_inner<BT_, PATH_><<<gd, 256, 0, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, \
+        k_inner<BT_, PATH_><<<gd, 256, 0, st>>>(ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, \
                                                 beta, batch, ctx->log_n, g, accumulate, ROW0_);                 \
     } while (0)
     // data rows on primes below 2^50 and special rows above: one launch per kind, each compiled for its arithmetic
@@ -663,7 +669,7 @@ static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(k_inner_tma<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         const uint32_t grid = n_tiles < (uint32_t)sms ? n_tiles : (uint32_t)sms;
-        k_inner_tma<4><<<grid, 256, smem, st>>>(ws.d, ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta,
+        k_inner_tma<4><<<grid, 256, smem, st>>>(ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta,
                                                  batch, ctx->log_n, g, accumulate, n_tiles, ctx->d_status);
     } else if (split) {
         if (batch >= 6) INNER(8, 1, 0, level);
@@ -728,16 +734,19 @@ static int key_switch_chunk(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& k
     return ks_apply(ctx, ws, key, level, batch, out, out_stride, add_mask, st, 0);
 }
 
+static OwnRows own_rows(const fesc_ctx* ctx, const KsScratch& ws, uint32_t level) {
+    return OwnRows{ws.ext, ctx->alpha, (level + ctx->alpha - 1) / ctx->alpha, level + ctx->n_p};
+}
+
 size_t ks_scratch_words(const fesc_ctx* ctx, uint32_t level, uint32_t chunk) {
     const uint32_t beta = (level + ctx->alpha - 1) / ctx->alpha, rows = level + ctx->n_p;
-    return (size_t)chunk * ctx->N * ((size_t)2 * level + (size_t)beta * rows + 2 * rows + 2 * level);
+    return (size_t)chunk * ctx->N * ((size_t)level + (size_t)beta * rows + 2 * rows + 2 * level);
 }
 KsScratch ks_scratch_carve(const fesc_ctx* ctx, u64* base, uint32_t level, uint32_t chunk) {
     const uint32_t beta = (level + ctx->alpha - 1) / ctx->alpha, rows = level + ctx->n_p;
     const size_t N = ctx->N;
     KsScratch ws;
-    ws.d = base;
-    ws.dcoef = ws.d + (size_t)chunk * level * N;
+    ws.dcoef = base;
     ws.ext = ws.dcoef + (size_t)chunk * level * N;
     ws.acc = ws.ext + (size_t)chunk * beta * rows * N;
     ws.u = ws.acc + (size_t)chunk * 2 * rows * N;
@@ -765,7 +774,7 @@ int rotate_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, si
         dim3 g((ctx->N + 255) / 256, level, nb);
         prof_begin(ctx, PF_AUTOM, st);
         k_autom_ct<<<g, 256, 0, st>>>(in + (size_t)b0 * in_stride, in_stride, out + (size_t)b0 * out_stride, out_stride,
-                                      ws.d, ws.dcoef, ctx->log_n, level, it->second.g, ctx->d_pc, accumulate);
+                                      own_rows(ctx, ws, level), ws.dcoef, ctx->log_n, level, it->second.g, ctx->d_pc, accumulate);
         prof_end(ctx, PF_AUTOM, st);
         int rc = key_switch_chunk(ctx, ws, it->second, level, nb, out + (size_t)b0 * out_stride, out_stride,
                                   accumulate ? 3 : 1, st);
@@ -776,7 +785,7 @@ int rotate_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, si
 
 // c0 of every ciphertext through the Galois permutation into out[b][0]; with g == 0, c1 copied to d and dcoef
 __global__ void __launch_bounds__(256) k_hoist_prepare(const u64* __restrict__ in, size_t in_stride, u64* __restrict__ out0,
-                                                       size_t out_stride, u64* __restrict__ d, u64* __restrict__ dcoef,
+                                                       size_t out_stride, OwnRows d, u64* __restrict__ dcoef,
                                                        uint32_t log_n, uint32_t level, u64 g) {
     const uint32_t N = 1u << log_n;
     const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
@@ -787,9 +796,8 @@ __global__ void __launch_bounds__(256) k_hoist_prepare(const u64* __restrict__ i
         out0[(size_t)b * out_stride + (size_t)l * N + t] = ib[(size_t)l * N + galois_src(t, log_n, g)];
     } else {
         const u64 v = ib[((size_t)level + l) * N + t];
-        const size_t o = ((size_t)b * level + l) * N + t;
-        d[o] = v;
-        dcoef[o] = v;
+        d.ext[own_index(d, b, l, N) + t] = v;
+        dcoef[((size_t)b * level + l) * N + t] = v;
     }
 }
 
@@ -812,7 +820,7 @@ int giant_sum_deferred_internal(fesc_ctx* ctx, u64* acc, uint32_t n_terms, size_
         for (uint32_t p = 1; p < n_terms; p++) {
             const EvalKey& key = ctx->keys[key_base + p];
             prof_begin(ctx, PF_AUTOM, st);
-            k_autom_ct<<<g, 256, 0, st>>>(base + (size_t)p * ct_words, stride, base, stride, ws.d, ws.dcoef, ctx->log_n,
+            k_autom_ct<<<g, 256, 0, st>>>(base + (size_t)p * ct_words, stride, base, stride, own_rows(ctx, ws, level), ws.dcoef, ctx->log_n,
                                           level, key.g, ctx->d_pc, 1);
             prof_end(ctx, PF_AUTOM, st);
             int rc = ks_decompose(ctx, ws, level, nb, st);
@@ -840,7 +848,7 @@ int rotate_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64*
         dim3 g((ctx->N + 255) / 256, level, nb);
         const u64* ib = in + (size_t)b0 * in_stride;
         prof_begin(ctx, PF_AUTOM, st);
-        k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, nullptr, 0, ws.d, ws.dcoef, ctx->log_n, level, 0);
+        k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, nullptr, 0, own_rows(ctx, ws, level), ws.dcoef, ctx->log_n, level, 0);
         prof_end(ctx, PF_AUTOM, st);
         int rc = ks_decompose(ctx, ws, level, nb, st);
         if (rc != FESC_OK) return rc;
@@ -848,7 +856,7 @@ int rotate_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64*
             const EvalKey& key = ctx->keys[key_ids[k]];
             u64* ob = out + (size_t)k * key_stride + (size_t)b0 * out_stride;
             prof_begin(ctx, PF_AUTOM, st);
-            k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, ob, out_stride, nullptr, nullptr, ctx->log_n, level, key.g);
+            k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, ob, out_stride, OwnRows{nullptr, 1, 1, 1}, nullptr, ctx->log_n, level, key.g);
             prof_end(ctx, PF_AUTOM, st);
             rc = ks_apply(ctx, ws, key, level, nb, ob, out_stride, 1, st, key.g);
             if (rc != FESC_OK) return rc;
@@ -900,7 +908,7 @@ int rotate_sum_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, 
         const u64* ib = in + (size_t)b0 * in_stride;
         u64* ob = out + (size_t)b0 * out_stride;
         prof_begin(ctx, PF_AUTOM, st);
-        k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, nullptr, 0, ws.d, ws.dcoef, ctx->log_n, level, 0);
+        k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, nullptr, 0, own_rows(ctx, ws, level), ws.dcoef, ctx->log_n, level, 0);
         k_rotsum_prepare<<<g, 256, 0, st>>>(ib, in_stride, ob, out_stride, ctx->log_n, level, gs, ctx->d_pc);
         prof_end(ctx, PF_AUTOM, st, 2);
         int rc = ks_decompose(ctx, ws, level, nb, st);
@@ -1041,7 +1049,7 @@ extern "C" int fesc_rescale(fesc_ctx* ctx, const uint64_t* d_in, uint64_t* d_out
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) k_tensor(const u64* __restrict__ a, size_t a_stride, const u64* __restrict__ bb,
                                                 size_t b_stride, u64* __restrict__ out, size_t out_stride,
-                                                u64* __restrict__ d, u64* __restrict__ dcoef,
+                                                OwnRows d, u64* __restrict__ dcoef,
                                                 const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level) {
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t l = blockIdx.y, b = blockIdx.z;
@@ -1056,9 +1064,8 @@ __global__ void __launch_bounds__(256) k_tensor(const u64* __restrict__ a, size_
     mac128(s, a1, b0);
     out[b * out_stride + poly + o] = reduce128(s.hi, s.lo, pc);
     const u64 d2 = mulmod(a1, b1, pc);
-    const size_t od = ((size_t)b * level + l) * N + c;
-    d[od] = d2;
-    dcoef[od] = d2;
+    d.ext[own_index(d, b, l, N) + c] = d2;
+    dcoef[((size_t)b * level + l) * N + c] = d2;
 }
 
 int ctmul_internal(fesc_ctx* ctx, const u64* a, size_t a_stride, const u64* b, size_t b_stride, u64* out,
@@ -1071,7 +1078,7 @@ int ctmul_internal(fesc_ctx* ctx, const u64* a, size_t a_stride, const u64* b, s
         dim3 g((ctx->N + 255) / 256, level, nb);
         prof_begin(ctx, PF_POINTWISE, st);
         k_tensor<<<g, 256, 0, st>>>(a + (size_t)b0 * a_stride, a_stride, b + (size_t)b0 * b_stride, b_stride,
-                                    out + (size_t)b0 * out_stride, out_stride, ws.d, ws.dcoef, ctx->d_pc, ctx->N, level);
+                                    out + (size_t)b0 * out_stride, out_stride, own_rows(ctx, ws, level), ws.dcoef, ctx->d_pc, ctx->N, level);
         prof_end(ctx, PF_POINTWISE, st);
         int rc = key_switch_chunk(ctx, ws, key, level, nb, out + (size_t)b0 * out_stride, out_stride, 3, st);
         if (rc != FESC_OK) return rc;

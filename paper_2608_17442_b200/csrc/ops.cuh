@@ -3,13 +3,12 @@
 #include "common.cuh"
 
 // Scratch of one key-switch chunk (all [chunk][...][N] words):
-//   d     [level]            the polynomial being switched, EVAL
-//   dcoef [level]            copy of d, transformed to COEFF in place
-//   ext   [beta][level+K]    converted digits
+//   dcoef [level]            the polynomial being switched, transformed to COEFF in place
+//   ext   [beta][level+K]    converted digits; the rows of a digit's own limbs hold the polynomial itself (EVAL)
 //   acc   [2][level+K]       inner-product accumulators
 //   u     [2][level]         converted special-limb part
 struct KsScratch {
-    u64 *d, *dcoef, *ext, *acc, *u;
+    u64 *dcoef, *ext, *acc, *u;
 };
 size_t ks_scratch_words(const fesc_ctx* ctx, uint32_t level, uint32_t chunk);
 KsScratch ks_scratch_carve(const fesc_ctx* ctx, u64* base, uint32_t level, uint32_t chunk);
