@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
 // for BT products.
 // ---------------------------------------------------------------------------------------
 #ifndef INNER_MINB
-#define INNER_MINB 3
+#define INNER_MINB 4
 #endif
 // PATH 0: the row's prime decides at run time; 1: the caller guarantees primes below 2^50 on rows
 // [row0, row0 + gridDim.y) (exact FP64 products only); 2: the caller sends those rows to the 128-bit integer sums.
@@ -232,8 +232,9 @@ __global__ void __launch_bounds__(256, (BT >= 8 ? 2 : INNER_MINB)) k_inner(const
         // exact FP64 products of canonical words (both below q): every product is below 0.875q, so a running sum of
         // at most q/2 plus 7 terms stays below 2^53 = 8q; longer sums are folded back after every 7th digit.  The next digit's words
         // are requested before this digit's products start: 2 + BT loads in flight per thread, few registers,
-        // so that three or four CTAs per SM overlap their loads and products (measured: one digit ahead with
-        // 4 CTAs per SM moves 1.5x the bytes per second of all-digits-up-front with 2).
+        // so that four CTAs per SM overlap their loads and products (measured: one digit ahead with 4 CTAs of 4
+        // ciphertexts per thread moves 1.6x the bytes per second of all-digits-up-front with 2 CTAs; 8 ciphertexts
+        // per thread with 2 CTAs and 2 per thread with 6 CTAs are both slower).
         const double q = pcs[pt].qd, qinv = pcs[pt].qinvd;
         double f0[BT], f1[BT];
 #pragma unroll
@@ -672,8 +673,7 @@ static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint
         k_inner_tma<4><<<grid, 256, smem, st>>>(ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta,
                                                  batch, ctx->log_n, g, accumulate, n_tiles, ctx->d_status);
     } else if (split) {
-        if (batch >= 6) INNER(8, 1, 0, level);
-        else if (batch >= 3) INNER(4, 1, 0, level);
+        if (batch >= 3) INNER(4, 1, 0, level);
         else if (batch == 2) INNER(2, 1, 0, level);
         else INNER(1, 1, 0, level);
         if (batch >= 3) INNER(4, 2, level, K);
