@@ -113,6 +113,29 @@ __global__ void __launch_bounds__(256) k_autom_ct(const u64* __restrict__ in, si
 // ext row order: data limbs 0..level-1 then the K special limbs; rows of the digit's own limbs
 // are left untouched (the inner product reads those from the EVAL-form input).
 // ---------------------------------------------------------------------------------------
+// VEC (1, 2 or 4) adjacent words with 16-byte accesses where possible
+template <int VEC>
+__device__ __forceinline__ void ldv(const u64* __restrict__ src, u64 (&w)[VEC]) {
+    if (VEC == 1) {
+        w[0] = *src;
+    } else {
+#pragma unroll
+        for (int v = 0; v < VEC / 2; v++) {
+            const ulonglong2 t2 = reinterpret_cast<const ulonglong2*>(src)[v];
+            w[2 * v] = t2.x, w[(2 * v + 1) % VEC] = t2.y;
+        }
+    }
+}
+template <int VEC>
+__device__ __forceinline__ void stv(u64* __restrict__ dst, const u64 (&r)[VEC]) {
+    if (VEC == 1) {
+        *dst = r[0];
+    } else {
+#pragma unroll
+        for (int v = 0; v < VEC / 2; v++) reinterpret_cast<ulonglong2*>(dst)[v] = make_ulonglong2(r[2 * v], r[(2 * v + 1) % VEC]);
+    }
+}
+
 template <int ALPHA, int VEC>
 __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u64* __restrict__ ext,
                                                const ModUpDigit* __restrict__ tab, const PrimeConst* __restrict__ pcs,
@@ -134,12 +157,7 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
             const u64 q = pcs[first + a].q, inv = dg->inv[a], invs = dg->invs[a];
             src_small = src_small && q < FESC_FP_LIMIT;
             u64 w[VEC];
-            if (VEC == 2) {
-                const ulonglong2 t2 = *reinterpret_cast<const ulonglong2*>(src);
-                w[0] = t2.x, w[VEC - 1] = t2.y;
-            } else {
-                w[0] = *src;
-            }
+            ldv<VEC>(src, w);
 #pragma unroll
             for (int v = 0; v < VEC; v++) y[a][v] = shoup(w[v], inv, invs, q);
         }
@@ -181,10 +199,7 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
                 r[v] = reduce128(acc.hi, acc.lo, pc);
             }
         }
-        if (VEC == 2)
-            *reinterpret_cast<ulonglong2*>(out + (size_t)t * N) = make_ulonglong2(r[0], r[VEC - 1]);
-        else
-            out[(size_t)t * N] = r[0];
+        stv<VEC>(out + (size_t)t * N, r);
     }
 }
 
@@ -194,6 +209,10 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
 // One thread owns one (coefficient, modulus) and BT ciphertexts, so a key word is loaded once
 // for BT products.
 // ---------------------------------------------------------------------------------------
+// coefficients per thread of the basis-conversion kernels
+#ifndef KS_VEC
+#define KS_VEC 2
+#endif
 #ifndef INNER_MINB
 #define INNER_MINB 4
 #endif
@@ -513,12 +532,7 @@ __global__ void __launch_bounds__(256) k_moddown_conv(const u64* __restrict__ ac
         if (k < K) {
             const u64* src = acc + ((size_t)bp * rows + level + k) * N + c;
             u64 w[VEC];
-            if (VEC == 2) {
-                const ulonglong2 t2 = *reinterpret_cast<const ulonglong2*>(src);
-                w[0] = t2.x, w[VEC - 1] = t2.y;
-            } else {
-                w[0] = *src;
-            }
+            ldv<VEC>(src, w);
             const u64 inv = tab->inv[k], invs = tab->invs[k], pk = pcs[n_q + k].q, half = tab->half[k];
 #pragma unroll
             for (int v = 0; v < VEC; v++) {
@@ -567,11 +581,7 @@ __global__ void __launch_bounds__(256) k_moddown_conv(const u64* __restrict__ ac
                 r[v] = submod(reduce128(a.hi, a.lo, pc), tab->wrap[cnt[v]][i], pc.q);
             }
         }
-        u64* dst = u + ((size_t)bp * level + i) * N + c;
-        if (VEC == 2)
-            *reinterpret_cast<ulonglong2*>(dst) = make_ulonglong2(r[0], r[VEC - 1]);
-        else
-            *dst = r[0];
+        stv<VEC>(u + ((size_t)bp * level + i) * N + c, r);
     }
 }
 
@@ -615,11 +625,11 @@ static int ks_decompose(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint
     if ((rc = ntt_launch(ctx, ws.dcoef, (size_t)batch * level, m, true, st)) != FESC_OK) return rc;
     // 2. ModUp
     const ModUpDigit* tab = ctx->tabs.d_modup + (size_t)(level - 1) * ctx->beta_max;
-    const bool vec2 = N % 512 == 0;
-    dim3 gmu(vec2 ? N / 512 : gx, beta, batch);
+    const bool vec2 = N % (256 * KS_VEC) == 0;
+    dim3 gmu(vec2 ? N / (256 * KS_VEC) : gx, beta, batch);
 #define MODUP(A)                                                                                           \
     do {                                                                                                   \
-        if (vec2) k_modup<A, 2><<<gmu, 256, 0, st>>>(ws.dcoef, ws.ext, tab, ctx->d_pc, N, level, nq, K, beta); \
+        if (vec2) k_modup<A, KS_VEC><<<gmu, 256, 0, st>>>(ws.dcoef, ws.ext, tab, ctx->d_pc, N, level, nq, K, beta); \
         else k_modup<A, 1><<<gmu, 256, 0, st>>>(ws.dcoef, ws.ext, tab, ctx->d_pc, N, level, nq, K, beta);  \
     } while (0)
     prof_begin(ctx, PF_MODUP, st);
@@ -701,8 +711,8 @@ static int ks_moddown(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint32
     for (uint32_t t = 0; t < rows; t++) m.prime[t] = t < level ? 0xFF : (uint8_t)(nq + (t - level));
     if ((rc = ntt_launch(ctx, ws.acc, (size_t)batch * 2 * rows, m, true, st)) != FESC_OK) return rc;
     prof_begin(ctx, PF_MODDOWN, st);
-    if (N % 512 == 0)
-        k_moddown_conv<2><<<dim3(N / 512, batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K);
+    if (N % (256 * KS_VEC) == 0)
+        k_moddown_conv<KS_VEC><<<dim3(N / (256 * KS_VEC), batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K);
     else
         k_moddown_conv<1><<<dim3(gx, batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K);
     prof_end(ctx, PF_MODDOWN, st);
