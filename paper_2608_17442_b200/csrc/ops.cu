@@ -661,7 +661,7 @@ static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint
     const uint32_t beta = (level + alpha - 1) / alpha, rows = level + K;
     const uint32_t gx = (N + 255) / 256;
     prof_begin(ctx, PF_INNER, st);
-    static const int use_tma = getenv("FESC_INNER_TMA") ? 1 : 0;
+    const bool use_tma = getenv("FESC_INNER_TMA") != nullptr;   // read per call so a test can switch it
 #define INNER(BT_, PATH_, ROW0_, NROWS_)                                                                        \
     do {                                                                                                        \
         dim3 gd(gx, NROWS_, (batch + BT_ - 1) / BT_);                                                           \

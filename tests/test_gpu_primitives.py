@@ -286,6 +286,35 @@ def test_rotate_sum_hoisted(name, level, batch, n_keys):
         assert np.array_equal(got[b], orc.rotate_sum_hoisted(ct[b], [k for _, k in rots])), (name, level, b)
 
 
+def test_inner_product_staged_by_bulk_copies(monkeypatch):
+    """The persistent inner-product kernel whose operands arrive by bulk asynchronous copies with bounded mbarrier
+    waits (FESC_INNER_TMA=1): plain, hoisted and rotate-and-add key switches stay bit-exact and no wait gives up."""
+    import torch
+
+    monkeypatch.setenv("FESC_INNER_TMA", "1")
+    for name, level, batch in (("small", 24, 5), ("full", 24, 3)):
+        pair = ctx_pair(name)
+        ctx, orc, _ = pair
+        rots = [(3, 81), (-5, 82)]
+        for r, kid in rots:
+            add_key(pair, r, kid)
+        ct = random_ct(orc, 13, level, level, batch)
+        dev = to_dev(ct)
+        out = torch.empty_like(dev)
+        ctx.rotate(dev, out, batch, level, 81)
+        hout = torch.empty((2, batch, 2, level, orc.N), dtype=torch.int64, device="cuda")
+        ctx.rotate_hoisted(dev, hout, batch, level, [81, 82])
+        sout = torch.empty_like(dev)
+        ctx.rotate_sum_hoisted(dev, sout, batch, level, [81, 82])
+        ctx.sync()                                  # FESC_ETIMEOUT would be raised here
+        got, hgot, sgot = to_host(out), to_host(hout), to_host(sout)
+        for b in range(batch):
+            assert np.array_equal(got[b], orc.rotate(ct[b], 81))
+            want = orc.rotate_hoisted(ct[b], [81, 82])
+            assert np.array_equal(hgot[0, b], want[0]) and np.array_equal(hgot[1, b], want[1])
+            assert np.array_equal(sgot[b], orc.rotate_sum_hoisted(ct[b], [81, 82]))
+
+
 def test_integer_paths_with_primes_above_50_bits():
     """Primes of 52 and 55 bits take the integer kernels (wide-lazy transform at N = 2^16, 128-bit lazy
     accumulation in ModUp / inner product / ModDown); same bit-exact bar."""
