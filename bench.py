@@ -30,6 +30,7 @@ sys.path.insert(0, ROOT)
 METRIC = "encrypted 768->3352 projection latency at L=2048; key-switches/s; HBM GB/s vs peak"
 T_SEG, C_SEG, N1, N2 = 128, 256, 32, 8
 D_IN, D_OUT, TOKENS = 768, 3352, 2048
+PROJ = "in_proj"            # "out_proj" (1536 -> 768) is selected by --workload out_proj
 LEVEL = 24
 BABY_BASE, GIANT_BASE = 1000, 1500
 
@@ -385,7 +386,7 @@ def run_ours(args):
         # the default kernel keeps the low 64 bits of every sum on the integer multiplier pipe
         alu_peak = SM_COUNT * 4 * 32 * sm_mhz * 1e6 / MAC_MIXED_CYCLES / 1e12        # T modular mul-adds / s
         fp64_peak = SM_COUNT * FP64_PER_CLK_PER_SM * sm_mhz * 1e6 / MAC_FP64 / 1e12
-        traffic = BSGS_TRAFFIC_4TB if (args.scale_down == 1 and abs(tb_per_launch - 4) < 1e-9) else None
+        traffic = BSGS_TRAFFIC_4TB if (PROJ == "in_proj" and args.scale_down == 1 and abs(tb_per_launch - 4) < 1e-9) else None
         roof.update({"bound": "alu", "achieved": macs / t / 1e12, "peak": alu_peak,
                      "unit": "T modular mac/s (integer multiplier pipe, 8 cycles per warp-mac)",
                      "peak_fp64_only_scheme": fp64_peak,
@@ -496,9 +497,9 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": "key-switches/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "latency_ms": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
-        "config": {"workload": "in_proj 768->3352, L=2048 tokens, N=2^16, 24x50-bit limbs + 4x60-bit special primes, "
+        "config": {"workload": "%s %d->%d, L=2048 tokens, N=2^16, 24x50-bit limbs + 4x60-bit special primes, "
                                "6 key-switch digits, C=256 T=128 n1=32 n2=8, baby rotations %s"
-                               % ("hoisted (one decomposition per input ciphertext)" if args.hoist else "by plain rotations")
+                               % (PROJ, D_IN, D_OUT, "hoisted (one decomposition per input ciphertext)" if args.hoist else "by plain rotations")
                                + (", one division by P per output for the giant-step sum" if args.defer else ""),
                    "input_cts": tbs * gin, "diagonals": nout * N2 * gin * N1, "output_cts": tbs * nout,
                    "key_switches_per_step": ks_per_step, "macs_per_step": tbs * nout * N2 * gin * N1,
@@ -682,9 +683,15 @@ def main():
                     help="1: one division by P per output for the whole giant-step sum")
     ap.add_argument("--hoist", type=int, default=1, choices=[0, 1],
                     help="1: baby rotations share one decomposition per input ciphertext (fesc_rotate_hoisted)")
-    ap.add_argument("--workload", default="in_proj", choices=["in_proj", "scan_slice", "scan_layer", "conv"],
-                    help="in_proj (default, the benchmark metric), a scan-contract run or the depthwise convolution")
+    ap.add_argument("--workload", default="in_proj", choices=["in_proj", "out_proj", "scan_slice", "scan_layer", "conv"],
+                    help="in_proj (default, the benchmark metric), out_proj (1536 -> 768), a scan-contract run or the "
+                         "depthwise convolution")
     args = ap.parse_args()
+    if args.workload == "out_proj":
+        global D_IN, D_OUT, PROJ, METRIC
+        D_IN, D_OUT, PROJ = 1536, 768, "out_proj"
+        METRIC = "encrypted 1536->768 projection latency at L=2048; key-switches/s"
+        args.workload = "in_proj"
     if args.workload == "conv":
         return run_conv(args)
     if args.workload != "in_proj":
