@@ -498,8 +498,8 @@ def run_ours(args):
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "latency_ms": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
         "config": {"workload": "%s %d->%d, L=2048 tokens, N=2^16, 24x50-bit limbs + 4x60-bit special primes, "
-                               "6 key-switch digits, C=256 T=128 n1=32 n2=8, baby rotations %s"
-                               % (PROJ, D_IN, D_OUT, "hoisted (one decomposition per input ciphertext)" if args.hoist else "by plain rotations")
+                               "6 key-switch digits, C=256 T=128 n1=%d n2=%d, baby rotations %s"
+                               % (PROJ, D_IN, D_OUT, N1, N2, "hoisted (one decomposition per input ciphertext)" if args.hoist else "by plain rotations")
                                + (", one division by P per output for the giant-step sum" if args.defer else ""),
                    "input_cts": tbs * gin, "diagonals": nout * N2 * gin * N1, "output_cts": tbs * nout,
                    "key_switches_per_step": ks_per_step, "macs_per_step": tbs * nout * N2 * gin * N1,
@@ -688,8 +688,9 @@ def main():
                          "depthwise convolution")
     args = ap.parse_args()
     if args.workload == "out_proj":
-        global D_IN, D_OUT, PROJ, METRIC
+        global D_IN, D_OUT, PROJ, METRIC, N1, N2
         D_IN, D_OUT, PROJ = 1536, 768, "out_proj"
+        N1, N2 = 16, 16      # 6 input blocks, 3 output blocks: fewer, cheaper rotations than 32 x 8
         METRIC = "encrypted 1536->768 projection latency at L=2048; key-switches/s"
         args.workload = "in_proj"
     if args.workload == "conv":
