@@ -51,11 +51,23 @@ def test_brent_kung_network_counts_and_prefixes(B):
     assert all(cover[k] == (1, k) for k in range(1, B + 1))
 
 
+def _golden(name):
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", name)
+    return [[float(v) for v in line.split()] for line in open(path) if line.strip() and not line.startswith("#")]
+
+
 def test_paper_ledger_values():
-    # Table "real-phantom-scan", Brent-Kung column: 2 * K_s * (2(L'-1) - log2 L') key switches, K_s = 12
-    for Lp, printed in ((128, 5.9e3), (256, 12.0e3), (512, 24.3e3), (1024, 48.9e3), (2048, 98.0e3)):
-        ks = 2 * 12 * (2 * (Lp - 1) - int(math.log2(Lp)))
-        assert abs(ks - printed) / printed < 0.01
+    # Table "real-phantom-scan": compositions of each prefix network over L' positions, times 2 K_s key switches
+    for Lp, seq_k, seq_d, ks_k, ks_d, skl_k, skl_d, bk_k, bk_d in _golden("real_phantom_scan.txt"):
+        Lp, lg = int(Lp), int(math.log2(Lp))
+        counts = {"seq": Lp - 1, "ks": Lp * lg - (Lp - 1), "skl": Lp // 2 * lg, "bk": 2 * (Lp - 1) - lg}
+        for key, printed in (("seq", seq_k), ("ks", ks_k), ("skl", skl_k), ("bk", bk_k)):
+            assert abs(2 * 12 * counts[key] / 1e3 - printed) <= 0.0501, (Lp, key)
+        assert (seq_d, ks_d, skl_d, bk_d) == (Lp - 1, lg, lg, 2 * lg - 1)
+        assert counts["bk"] == len(_bk_nodes(Lp))                              # the network this build evaluates
+    (d_s, K_s, printed), = _golden("cross_ssm_family.txt")
+    assert (d_s, K_s) == (128, 12) and 2 * 12 * (2 * 127 - 7) == printed
     assert 2 * 12 * (2 * 127 - 7) == 5928                                     # Table "cross_ssm_family", Mamba-2
     # depth 2 ceil(log2 L') - 1
     assert [2 * int(math.log2(Lp)) - 1 for Lp in (128, 256, 512, 1024, 2048)] == [13, 15, 17, 19, 21]
