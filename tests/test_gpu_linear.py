@@ -188,3 +188,11 @@ def test_linear_full_ring_one_block():
     err = np.abs(Y - X @ W).max()
     print("max |decrypt - X@W| = 2^%.2f" % np.log2(err))
     assert err < 2.0**-18
+    # the benchmark's default modes (hoisted baby steps, one division by P per output): own residues, same values
+    got_m = _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=2000, hoist=1, defer=1)
+    want_m = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: 2000 + q for q in range(1, n1)},
+                        {g: 2500 + g for g in range(1, n2)}, hoist=True, defer=True)
+    assert np.array_equal(got_m, want_m)
+    err_m = np.abs(orc.decrypt(got_m[0, 0], scale, 2).real.reshape(C, T).T - X @ W).max()
+    print("hoisted + deferred: max |decrypt - X@W| = 2^%.2f" % np.log2(err_m))
+    assert err_m < 2.0**-18
