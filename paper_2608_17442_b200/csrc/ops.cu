@@ -334,7 +334,7 @@ __global__ void __launch_bounds__(256, (BT >= 8 ? 2 : INNER_MINB)) k_inner(const
 }
 
 // ---------------------------------------------------------------------------------------
-// The same inner product with operands staged by bulk asynchronous copies (TMA, no multicast).
+// The same inner product with operands staged by bulk asynchronous copies (TMA; every copy targets this CTA only).
 // A persistent CTA walks over tiles (limb row t, 256 coefficients, BT ciphertexts).  One thread requests, per
 // digit, the two key rows and the BT digit rows of the NEXT tile (2 KB each) into the other half of shared memory,
 // completion counted in bytes on an mbarrier, while all threads multiply out the current tile from shared memory;
