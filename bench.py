@@ -9,10 +9,15 @@ rescales.  Inputs are seeded synthetic residues (uniform below each prime) of ex
 shapes; arithmetic is data-independent, so timing equals that of real encodings.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python bench.py --workload out_proj | conv | scan_slice | scan_layer      (the other stages of a layer)
 
 Prints ONE JSON line (rank 0).  `value` = key switches per second over the whole step, summed
 over ranks (each rank runs its own 2048-token batch: weak scaling, no data-path collective);
-`latency_ms` is the projection latency the metric names.
+`latency_ms` is the projection latency the metric names.  The default step uses hoisted baby
+rotations and one division by P per output (--hoist 0 --defer 0: the plain definitions); beside
+the headline the line carries `roofline`, `kernel_breakdown`, `e2e`, `clocks`, `cpu_baseline`,
+`isolated` (ct-pt MAC and key-switch inner product alone) and `variants` (token blocks paired in
+the real and imaginary channels).
 """
 from __future__ import annotations
 
@@ -676,7 +681,7 @@ def main():
     ap.add_argument("--scale-down", dest="scale_down", type=int, default=1, help=argparse.SUPPRESS)
     ap.add_argument("--no-cpu", dest="no_cpu", action="store_true", help="skip the CPU baseline leg")
     ap.add_argument("--profile-case", dest="profile_case", action="store_true",
-                    help="run ONE step of a small case (1 input block, 1 output block, 2 token blocks) and exit; for ncu")
+                    help="run ONE step of a small case (1 input block, 1 output block, 4 token blocks) and exit; for ncu")
     ap.add_argument("--profile-step", dest="profile_step", action="store_true",
                     help="run ONE step of the full workload without warm-up and exit; for the ncu launch list")
     ap.add_argument("--defer", type=int, default=1, choices=[0, 1],
