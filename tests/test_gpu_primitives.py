@@ -188,6 +188,44 @@ def test_error_codes():
     assert e.value.code == fesc.EINVAL
 
 
+def test_empty_batches_and_rejected_arguments():
+    """Empty batches are no-ops that leave the outputs untouched; impossible shapes are refused before any launch."""
+    import torch
+    import paper_2608_17442_b200 as fesc
+
+    pair = ctx_pair("toy")
+    ctx, orc, p = pair
+    add_key(pair, 1, 91)
+    ct = to_dev(random_ct(orc, 9, 0, 6, 2))
+    out = torch.full_like(ct, 7)
+    ctx.ntt(ct, 0, 0, 6)
+    ctx.intt(ct, 0, 0, 6)
+    ctx.rotate(ct, out, 0, 6, 91)
+    ctx.rotate_hoisted(ct, out, 0, 6, [91])
+    ctx.rotate_sum_hoisted(ct, out, 0, 6, [91])
+    ctx.ct_pt_mac(ct, ct[:, 0].contiguous(), out, 0, 6)
+    ctx.rescale(ct, out, 0, 6)
+    ctx.ct_ct_mul(ct, ct, out, 0, 6)
+    ctx.sync()
+    assert bool((out == 7).all())
+    for bad in (lambda: ctx.ntt(ct, 1, 5, 9),                                   # limbs past the last prime
+                lambda: ctx.rotate(ct, out, 1, 99, 91),                         # level above n_q
+                lambda: ctx.rotate_sum_hoisted(ct, out, 1, 6, [91] * 9),        # more than 8 keys
+                lambda: ctx.linear(ct, ct, fesc.BsgsDesc(0, 1, 1, 1, 1, 6, 1, 1), out),
+                lambda: ctx.linear(ct, ct, fesc.BsgsDesc(2, 2, 1, 1, 1, 1, 1, 1), out),      # level 1 cannot rescale
+                lambda: ctx.conv(ct, ct, ct, fesc.ConvDesc(9, 8, 1, 1, 6, 1), out),          # more than 8 taps
+                lambda: ctx.conv(ct, ct, ct, fesc.ConvDesc(2, 5, 1, 1, 6, 1), out)):         # T does not divide the slots
+        with pytest.raises(fesc.FescError) as e:
+            bad()
+        assert e.value.code in (fesc.EINVAL, fesc.ELEVEL)
+    # one limb: transforms and multiply-accumulate still work
+    one = to_dev(random_ct(orc, 10, 0, 1, 1))
+    ref = to_host(one).copy()
+    ctx.intt(one, 2, 0, 1)
+    ctx.ntt(one, 2, 0, 1)
+    assert np.array_equal(to_host(one), ref)
+
+
 def test_workload_1_end_to_end():
     """Tiny CKKS: 4 ciphertexts x random plaintext vector, rotate by +1 and +5, decrypt; residues
     bit-exact and slots within 2^-16 of the float64 result."""
