@@ -219,7 +219,7 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
 // PATH 0: the row's prime decides at run time; 1: the caller guarantees primes below 2^50 on rows
 // [row0, row0 + gridDim.y) (exact FP64 products only); 2: the caller sends those rows to the 128-bit integer sums.
 template <int BT, int PATH>
-__global__ void __launch_bounds__(256, (BT >= 8 ? 2 : INNER_MINB)) k_inner(const u64* __restrict__ ext,
+__global__ void __launch_bounds__(256, INNER_MINB) k_inner(const u64* __restrict__ ext,
                                                const u64* __restrict__ key, u64* __restrict__ acc,
                                                const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
                                                uint32_t n_q, uint32_t K, uint32_t alpha, uint32_t beta,
@@ -612,7 +612,7 @@ __global__ void __launch_bounds__(256) k_moddown_finish(const u64* __restrict__ 
 }
 
 // Steps 1-3 of the key switch: ws.dcoef -> COEFF, digit-wise basis extension into ws.ext, NTT of the
-// converted rows.  The result (ws.d, ws.ext) can serve several keys (hoisted rotations).
+// converted rows.  The result (ws.ext, own-limb rows included) can serve several keys (hoisted rotations).
 static int ks_decompose(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint32_t batch, cudaStream_t st) {
     const uint32_t N = ctx->N, K = ctx->n_p, nq = ctx->n_q, alpha = ctx->alpha;
     const uint32_t beta = (level + alpha - 1) / alpha, rows = level + K;
