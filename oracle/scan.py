@@ -30,7 +30,8 @@ Every product is s x p or p x p of operands at the same level, followed by a res
 higher level is brought down by `adjust`: keep its first l_dst+1 limbs, multiply by the integer
 round(S[l_dst] q_{l_dst} / S[l_src]), rescale.  Masks are plaintexts at scale S_p of their level.
 
-Level schedule (logB = log2 B):  inputs l0;  masked / filled factors l0-1;  leaves (p, s) at l1 = l0-2;
+Level schedule (logB = log2 B):  inputs l0;  masked / filled factors l0-1 (br(C): masked at l0-1, brought to linj-1,
+filled there);  leaves (p, s) at l1 = l0-2;
 up-sweep stage s -> l1-s;  summaries at lS = l1-logB;  down-sweep stage number d (1..logB-1) works at
 lS-(d-1) -> lS-d;  carries g_j (j >= 1) at lS-(j-1);  injection at linj = l1-2logB+1 -> states at linj-1;
 contraction -> linj-2;  reduction, conjugation, unpacking there;  output mask -> l_out = linj-3.
@@ -302,13 +303,17 @@ class ScanEvaluator:
         return (p, s)
 
     # -- one token block ----------------------------------------------------------------------
-    def broadcast_bc(self, ct):
-        """brB_t (or brC_t) for every token of the block: level l0-1, value B_t[i] at every (e', i)."""
+    def broadcast_bc(self, ct, level=None):
+        """brB_t (or brC_t) for every token of the block, value B_t[i] at every (e', i): level l0-1, or brought down
+        to `level` BEFORE the rotate-and-add fill (br(C) is only needed at the injection level, where a rotation
+        costs a fraction of one at the top level)."""
         sh, c = self.sh, self.c
         ex = self.extract_all(ct, sh.d_s)
         out = []
         for t in range(sh.B):
             u = self.ptmul_rescale(ex[t], c.mask_b)
+            if level is not None:
+                u = self.adjust(u, level, "p")
             out.append(self.fill_right(u, sh.stride, int(math.log2(sh.c_state))))
         return out
 
@@ -354,7 +359,7 @@ class ScanEvaluator:
         carry = [None] * sh.K_s                       # g_j per chunk: the state before block j
         for j in range(sh.K_blk):
             brB = self.broadcast_bc(ctB[j])
-            brC = [self.adjust(u, linj - 1, "p") for u in self.broadcast_bc(ctC[j])]
+            brC = self.broadcast_bc(ctC[j], linj - 1)
             v = [[None] * sh.K_s for _ in range(sh.B)]
             for kap in range(sh.K_s):
                 T = self.leaves(ctX[j, kap], ctA[j, kap], brB)

@@ -311,10 +311,11 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
                 X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_b, brB);
                 X.fill_right(brB, g.stride, ilog2(g.c_state));
             } else {
+                // br(C) is only needed at the injection level: bring it down first, fill there (cheap rotations)
                 Arr full = X.alloc(B, l0 - 1);
                 X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_b, full);
-                X.fill_right(full, g.stride, ilog2(g.c_state));
                 X.adjust(full, linj - 1, 1, brC);
+                X.fill_right(brC, g.stride, ilog2(g.c_state));
             }
             X.top = m;
         }
