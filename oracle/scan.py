@@ -326,10 +326,10 @@ class ScanEvaluator:
         for t in range(sh.B):
             xr = self.ptmul_rescale(ex[t], c.mask_x)
             xr = self.fill_right(xr, 1, int(math.log2(sh.d_s)))
-            ar = self.ptmul_rescale(ea[t], c.mask_a)
+            ar = self.adjust(self.ptmul_rescale(ea[t], c.mask_a), l1, "p")        # to the leaf level, then fill
             ar = self.fill_right(ar, sh.P, int(math.log2(sh.R // sh.P)))
             s = self.mul_rescale(xr, brB[t])
-            T.append((self.adjust(ar, l1, "p"), s))
+            T.append((ar, s))
         return T
 
     def brent_kung(self, T, need_p_down):

@@ -338,9 +338,9 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
                 X.fill_right(xr, 1, ilog2(g.d_s));
                 X.extract_all(apre, g.P, ex);
                 X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_a, ar);
-                X.fill_right(ar, g.P, ilog2(g.R / g.P));
+                X.adjust(ar, l1, 1, Ps);         // p_t = br(a_t): to the leaf level first, then the fill
+                X.fill_right(Ps, g.P, ilog2(g.R / g.P));
                 X.mul_rescale(xr, brB, Ss);      // s_t = br(x_t) (.) br(B_t), level l1 (slots are compact at l1)
-                X.adjust(ar, l1, 1, Ps);         // p_t = br(a_t)
                 X.top = m;
             }
             // ---- Brent-Kung network ----
