@@ -10,6 +10,7 @@ shapes; arithmetic is data-independent, so timing equals that of real encodings.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
   python bench.py --workload out_proj | conv | scan_slice | scan_layer      (the other stages of a layer)
+  python bench.py --workload rotations                                      (512 plain rotations, both digit layouts)
 
 Prints ONE JSON line (rank 0).  `value` = key switches per second over the whole step, summed
 over ranks (each rank runs its own 2048-token batch: weak scaling, no data-path collective);
@@ -620,6 +621,69 @@ def run_scan(args):
                       "scratch_gib": c1[3] / 2**30, "kernel_breakdown": breakdown}), flush=True)
 
 
+def run_rotations(args):
+    """Key-switch / rotation workload: 32 ciphertexts (N = 2^16, 24 limbs), 16 key slots (rotations 1..8 and 8*{1..8}),
+    512 plain rotations per step, for the graded digit layout (6 digits of 4 limbs) and the literal dnum = 4 layout
+    (4 digits of 6 limbs): rotations/s, evaluation-key GB/s, limb transforms/s."""
+    import torch
+    import fesc_synth as S
+    import paper_2608_17442_b200 as fesc
+
+    torch.cuda.set_device(0)
+    hbm_peak, _ = peaks()
+    res = {}
+    amounts = list(range(1, 9)) + [8 * g for g in range(1, 9)]
+    for name in ("full", "full_literal"):
+        p = S.params(name)
+        ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+        N = ctx.N
+        for k, r in enumerate(amounts):
+            ctx.add_galois_key(r, 300 + k)
+        q = p["primes"][:LEVEL]
+        r = S.hashed_residues(S.config_seed(3), 1, q, 32 * 2 * N, device="cuda")
+        ct = r.view(LEVEL, 32, 2, N).permute(1, 2, 0, 3).contiguous()
+        out = torch.empty_like(ct)
+        del r
+
+        def step():
+            for k in range(16):
+                ctx.rotate(ct, out, 32, LEVEL, 300 + k)
+
+        for _ in range(max(3, args.warmup)):
+            step()
+        ctx.profile_enable(fesc.Context.PROFILE_FAMILIES, 60000)
+        step()
+        fam = ctx.profile_read()
+        ctx.profile_enable([])
+        c0 = ctx.counters()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        ctx.sync()
+        c1 = ctx.counters()
+        ms = e0.elapsed_time(e1) / args.steps
+        beta, rows = ctx.num_digits, LEVEL + ctx.n_p
+        launches = fam["inner"][1]
+        evk_bytes = launches * beta * 2 * rows * N * 8                      # key words streamed by the inner products
+        inner_bytes = 512 * (beta + 2) * rows * N * 8 + evk_bytes
+        res[name] = {"digits": beta, "ms_per_step": ms, "rotations_per_s": 512 / (ms * 1e-3),
+                     "limb_transforms_per_s": (c1[0] - c0[0]) / args.steps / (ms * 1e-3),
+                     "evk_gbs_in_inner_product": evk_bytes / (fam["inner"][0] * 1e-3) / 1e9,
+                     "inner_product_gbs": inner_bytes / (fam["inner"][0] * 1e-3) / 1e9,
+                     "inner_product_frac_of_hbm_peak": inner_bytes / (fam["inner"][0] * 1e-3) / 1e9 / hbm_peak,
+                     "family_ms": {k: round(v[0], 2) for k, v in fam.items() if v[1]}}
+        del ctx, ct, out
+        torch.cuda.empty_cache()
+    g = res["full"]
+    print(json.dumps({"metric": "plain rotations (automorphism + hybrid key switch) per second", "value": g["rotations_per_s"],
+                      "unit": "key-switches/s", "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup),
+                      "ms_per_step": g["ms_per_step"], "higher_is_better": True, "dtype": "u64", "data": "synthetic",
+                      "config": {"workload": "rotations: 32 ciphertexts x 16 keys = 512 rotations, N=2^16, 24 limbs + 4 special"},
+                      "layouts": res}), flush=True)
+
+
 def run_conv(args):
     """Times fesc_conv on synthetic residues of the Mamba-2-base shape: the xBC channels (1536 + 2*128 = 1792 = 7
     channel blocks of 256) x 2048 tokens (16 token blocks of 128), d_conv = 4, 24 limbs."""
@@ -688,7 +752,7 @@ def main():
                     help="1: one division by P per output for the whole giant-step sum")
     ap.add_argument("--hoist", type=int, default=1, choices=[0, 1],
                     help="1: baby rotations share one decomposition per input ciphertext (fesc_rotate_hoisted)")
-    ap.add_argument("--workload", default="in_proj", choices=["in_proj", "out_proj", "scan_slice", "scan_layer", "conv"],
+    ap.add_argument("--workload", default="in_proj", choices=["in_proj", "out_proj", "rotations", "scan_slice", "scan_layer", "conv"],
                     help="in_proj (default, the benchmark metric), out_proj (1536 -> 768), a scan-contract run or the "
                          "depthwise convolution")
     args = ap.parse_args()
@@ -700,6 +764,8 @@ def main():
         args.workload = "in_proj"
     if args.workload == "conv":
         return run_conv(args)
+    if args.workload == "rotations":
+        return run_rotations(args)
     if args.workload != "in_proj":
         return run_scan(args)
     if args.impl == "reference":
