@@ -498,6 +498,36 @@ def run_ours(args):
                                             "note": "token blocks 2u and 2u+1 in the real and imaginary channels; "
                                                     "fesc_linear on 8 complex token blocks + fesc_split_complex"}}
         del zc
+        # the paper's own pairing (App. "Projection Kernel Breakdown"): input blocks 2u and 2u+1 in the real and
+        # imaginary channels with complex diagonals, real part of every output by one conjugation.  Timed on the same
+        # buffers reinterpreted as ceil(gin/2) input blocks (residues are random either way).
+        gp = -(-gin // 2)
+        if gp < gin:
+            desc3 = fesc.BsgsDesc(N1, N2, gp, nout, tbs, LEVEL, BABY_BASE, GIANT_BASE, int(args.hoist), int(args.defer))
+            ct3 = ct.reshape(-1)[: tbs * gp * 2 * LEVEL * n].view(tbs, gp, 2, LEVEL, n)
+            dg3 = diags.reshape(-1)[: nout * N2 * gp * N1 * LEVEL * n].view(nout, N2, gp, N1, LEVEL, n)
+            z3 = torch.empty((tbs * nout, 2, LEVEL - 1, n), dtype=torch.int64, device=dev)
+            o3 = out.reshape(tbs * nout, 2, LEVEL - 1, n)
+
+            def paired_in():
+                ctx.linear(ct3, dg3, desc3, z3)
+                ctx.split_complex(z3, o3, None, tbs * nout, LEVEL - 1, conj_id)
+
+            paired_in()
+            c0 = ctx.counters()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(args.steps):
+                paired_in()
+            e1.record()
+            torch.cuda.synchronize()
+            c1 = ctx.counters()
+            variants["paired_input_blocks"] = {
+                "latency_ms": e0.elapsed_time(e1) / args.steps, "key_switches_per_step": (c1[1] - c0[1]) // args.steps,
+                "input_cts": tbs * gp, "output_cts": tbs * nout,
+                "note": "input blocks 2u and 2u+1 in the real and imaginary channels, complex diagonals; "
+                        "fesc_linear on %d input blocks + real part by fesc_split_complex" % gp}
+            del z3
 
     line = {
         "metric": METRIC, "value": value, "unit": "key-switches/s", "n_gpus": world, "steps": args.steps,

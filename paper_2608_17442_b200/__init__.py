@@ -192,7 +192,8 @@ class Context:
         self._chk(lib().fesc_rotate(self.h, _ptr(ct_in), _ptr(ct_out), batch, n_limbs, key_id, _stream()))
 
     def split_complex(self, ct_in, re2, im2, batch: int, n_limbs: int, conj_key_id: int):
-        self._chk(lib().fesc_split_complex(self.h, _ptr(ct_in), _ptr(re2), _ptr(im2), batch, n_limbs, conj_key_id, _stream()))
+        self._chk(lib().fesc_split_complex(self.h, _ptr(ct_in), _ptr(re2), _ptr(im2) if im2 is not None else None, batch,
+                                           n_limbs, conj_key_id, _stream()))
 
     def conv(self, ct_in, masks, bias, desc: "ConvDesc", ct_out):
         self._chk(lib().fesc_conv(self.h, _ptr(ct_in), _ptr(masks), _ptr(bias), ctypes.byref(desc), _ptr(ct_out), _stream()))

@@ -545,7 +545,7 @@ extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint
 // ---------------------------------------------------------------------------------------
 extern "C" int fesc_split_complex(fesc_ctx* ctx, const uint64_t* d_in, uint64_t* d_re2, uint64_t* d_im2, uint32_t batch,
                                   uint32_t n_limbs, uint32_t conj_key_id, void* stream) {
-    if (!ctx || !d_in || !d_re2 || !d_im2 || d_in == d_re2 || d_in == d_im2 || d_re2 == d_im2) return FESC_EINVAL;
+    if (!ctx || !d_in || !d_re2 || d_in == d_re2 || d_in == d_im2 || d_re2 == d_im2) return FESC_EINVAL;
     if (n_limbs == 0 || n_limbs > ctx->n_q) return fesc_fail(ctx, FESC_ELEVEL, "split_complex: level out of range");
     if (batch == 0) return FESC_OK;
     cudaStream_t st = (cudaStream_t)stream;
@@ -561,10 +561,10 @@ extern "C" int fesc_split_complex(fesc_ctx* ctx, const uint64_t* d_in, uint64_t*
     if (rc != FESC_OK) return rc;
     const dim3 g((N + 255) / 256, 2 * n_limbs, batch);
     prof_begin(ctx, PF_POINTWISE, st);
-    k_ct_addsub<<<g, 256, 0, st>>>(in, ctw, re, ctw, im, ctw, ctx->d_pc, N, n_limbs, 1);
+    if (im) k_ct_addsub<<<g, 256, 0, st>>>(in, ctw, re, ctw, im, ctw, ctx->d_pc, N, n_limbs, 1);
     k_ct_addsub<<<g, 256, 0, st>>>(in, ctw, re, ctw, re, ctw, ctx->d_pc, N, n_limbs, 0);
-    k_ct_mul_i<<<g, 256, 0, st>>>(im, ctw, im, ctw, ctx->d_pc, ctx->d_tw, N, n_limbs, 3);
-    prof_end(ctx, PF_POINTWISE, st, 3);
+    if (im) k_ct_mul_i<<<g, 256, 0, st>>>(im, ctw, im, ctw, ctx->d_pc, ctx->d_tw, N, n_limbs, 3);
+    prof_end(ctx, PF_POINTWISE, st, im ? 3 : 1);
     FESC_CHECK_CUDA(ctx, cudaGetLastError());
     return FESC_OK;
 }

@@ -159,6 +159,59 @@ def test_linear_on_complex_paired_token_blocks():
                 assert np.abs(y[:, :cols.stop - cols.start] - Y[tb * T:(tb + 1) * T, cols]).max() < 2.0**-18
 
 
+def test_linear_on_complex_paired_input_blocks():
+    """The paper's pairing (App. "Projection Kernel Breakdown"): input blocks 2u and 2u+1 in the real and imaginary
+    channels, complex diagonals D^(2u) - i D^(2u+1); the real part of the result is X @ W.  Three input blocks become
+    two ciphertexts per token block; residues bit-exact against the oracle, values against X @ W."""
+    import torch
+    from oracle.ckks import CONJ
+
+    pair = ctx_pair("small")
+    ctx, orc, p = pair
+    T, C, n1, n2, level, scale = 32, 16, 4, 4, 5, 2.0**40
+    tokens, d_in, d_out, kb = 2 * T, 40, 50, 8200
+    n = orc.n
+    X, W = S.linear_inputs(p["seed"] + 10, tokens, d_in, d_out)
+    W = W * 10.0
+    gin, nout, tbs = -(-d_in // C), -(-d_out // C), tokens // T
+    gpair = -(-gin // 2)
+    for q in range(1, n1):
+        add_key(pair, q * T, kb + q)
+    for g in range(1, n2):
+        add_key(pair, g * n1 * T, kb + 500 + g)
+    add_key(pair, CONJ, kb + 999)
+    blk = lambda tb, g: pack_linear_input(X[tb * T:(tb + 1) * T, g * C:(g + 1) * C], T, C, n) if g < gin else np.zeros(n)
+    cts = np.empty((tbs, gpair, 2, level, orc.N), dtype=np.uint64)
+    for tb in range(tbs):
+        for u in range(gpair):
+            cts[tb, u] = orc.encrypt(orc.encode(blk(tb, 2 * u) + 1j * blk(tb, 2 * u + 1), scale, level), 7800 + tb * gpair + u)
+    dg = lambda b, g, pp, q: linear_diagonal(W, b, g, pp, q, T, C, n1) if g < gin else np.zeros(n)
+    diags = np.empty((nout, n2, gpair, n1, level, orc.N), dtype=np.uint64)
+    for b in range(nout):
+        for pp in range(n2):
+            for u in range(gpair):
+                for q in range(n1):
+                    diags[b, pp, u, q] = orc.encode(dg(b, 2 * u, pp, q) - 1j * dg(b, 2 * u + 1, pp, q),
+                                                    float(orc.q[level - 1]), level)
+    got = _run_gpu(ctx, cts, diags, n1, n2, (gpair, nout, tbs), level, key_base=kb, hoist=1, defer=1)
+    want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)},
+                      {g: kb + 500 + g for g in range(1, n2)}, hoist=True, defer=True)
+    assert np.array_equal(got, want)
+    batch = tbs * nout
+    z = to_dev(got.reshape(batch, 2, level - 1, orc.N))
+    re2 = torch.empty_like(z)
+    ctx.split_complex(z, re2, None, batch, level - 1, kb + 999)
+    re2 = to_host(re2)
+    Y = X @ W
+    for tb in range(tbs):
+        for b in range(nout):
+            wr, _ = orc.split_complex(want[tb, b], kb + 999)
+            assert np.array_equal(re2[tb * nout + b], wr)
+            cols = slice(b * C, min((b + 1) * C, d_out))
+            y = orc.decrypt(wr, 2 * scale, 2).real.reshape(C, T).T
+            assert np.abs(y[:, :cols.stop - cols.start] - Y[tb * T:(tb + 1) * T, cols]).max() < 2.0**-18
+
+
 def test_linear_integer_kernels_with_55_bit_primes():
     """The 128-bit integer accumulate kernel (primes above 50 bits) against the oracle."""
     pair = ctx_pair("wide")
