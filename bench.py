@@ -176,8 +176,8 @@ SM_COUNT = 148
 IMAD_PER_CLK_PER_SM = 64          # 32-bit multiply-adds per SM per clock (measured 63 with a register chain)
 FP64_PER_CLK_PER_SM = 64          # FP64 FMAs per SM per clock (measured 63 with a register chain)
 BFLY_IMAD = 20                    # integer Shoup butterfly (primes >= 2^50): 10 products of 32x32->64
-BFLY_FP64 = 8.5                   # FP64 butterfly (primes < 2^50): 5 ops product + 2 adds + 1.5 fold-back share
-                                  # (kept at 8.5 after a fold-back was removed, so the bound only got stricter)
+BFLY_FP64 = 8.5                   # FP64 butterfly (primes < 2^50): 5 ops product + 2 adds + ~1.5 fold-back / conversion share
+                                  # (counted per pass: 8.25 forward strided, 8.75 forward contiguous, 8.5-9.5 inverse)
 MAC_FP64 = 6                      # FP64 multiply-accumulate: 5 ops exact product + 1 add
 MAC_MIXED_CYCLES = 8              # mixed-pipe multiply-accumulate: multiplier-pipe cycles per warp (one 32x32+64 = 4,
                                   # two 32-bit multiply-adds = 2 each) on each of the 4 sub-partitions of an SM
