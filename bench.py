@@ -586,20 +586,64 @@ def scan_rotation_amounts(n, P, d_s, B, stride, hoist=False):
     return sorted(am)
 
 
+def scan_partition(K_s: int, world: int):
+    """State chunks of every rank: chunk PAIRS (2l, 2l+1) stay together (they are reduced in the real and imaginary
+    lanes of one ciphertext); pairs are dealt out in contiguous, near-equal runs.  Returns [(first chunk, count)]."""
+    pairs = -(-K_s // 2)
+    out = []
+    for r in range(world):
+        lo, hi = pairs * r // world, pairs * (r + 1) // world
+        first, end = 2 * lo, min(2 * hi, K_s)
+        out.append((first, max(0, end - first)))
+    return out
+
+
+def gather_chunk_outputs(local, parts, rank, world, K_blk, K_s):
+    """The one exchange of the sharded scan: every rank contributes the output ciphertexts of its chunks
+    ([K_blk, chunks, ...]); all ranks end with the full [K_blk, K_s, ...] tensor.  One all_gather of equal-sized
+    buffers (ranks with fewer chunks pad), NCCL on GPUs, gloo in the CPU test."""
+    import torch
+    import torch.distributed as dist
+
+    width = max(c for _, c in parts)
+    tail = tuple(local.shape[2:])
+    buf = torch.zeros((K_blk, width) + tail, dtype=local.dtype, device=local.device)
+    buf[:, : local.shape[1]] = local
+    if world > 1:
+        bufs = [torch.empty_like(buf) for _ in range(world)]
+        dist.all_gather(bufs, buf)
+    else:
+        bufs = [buf]
+    full = torch.empty((K_blk, K_s) + tail, dtype=local.dtype, device=local.device)
+    for r, (first, count) in enumerate(parts):
+        if count:
+            full[:, first:first + count] = bufs[r][:, :count]
+    return full
+
+
 def run_scan(args):
     """Times fesc_scan_contract on synthetic residues of the deployed geometry (N=2^16, 24 limbs, stride 256,
-    B_blk=256, d_s=128, P=64).  --workload scan_slice: 4 heads x 512 tokens; scan_layer: 24 heads x 2048 tokens."""
+    B_blk=256, d_s=128, P=64).  --workload scan_slice: 4 heads x 512 tokens; scan_layer: 24 heads x 2048 tokens.
+    With --gpus N (one process per GPU) the state chunks are dealt out to the ranks in pairs (Alg. 7: chunks are
+    independent; the compact factors B, C are replicated) and the outputs are exchanged ONCE at the end by an
+    all-gather, inside the timed region: strong scaling, time = max over ranks."""
     import torch
     import fesc_synth as S
     import paper_2608_17442_b200 as fesc
 
-    torch.cuda.set_device(0)
+    rank, world = dist_setup("nccl")
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
     p = S.params("full")
     ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
     n, N = ctx.N // 2, ctx.N
     H, L = (4, 512) if args.workload == "scan_slice" else (24, 2048)
     P, d_s, B, stride, l0 = 64, 128, 256, 256, 24
     K_s, K_blk = H * P // (n // stride), L // B
+    hpc = (n // stride) // P                                   # heads per chunk
+    parts = scan_partition(K_s, world)
+    first, mine = parts[rank]
     base = 100000
     for r in scan_rotation_amounts(n, P, d_s, B, stride, bool(args.hoist)):
         ctx.add_galois_key(r, base + r)
@@ -608,20 +652,26 @@ def run_scan(args):
     q = p["primes"][:l0]
 
     def cts(count, stream):
-        r = S.hashed_residues(seed, stream, q, count * 2 * N, device="cuda")
+        r = S.hashed_residues(seed, stream, q, count * 2 * N, device=dev)
         return r.view(l0, count, 2, N).permute(1, 2, 0, 3).contiguous()
 
-    x, a = cts(K_blk * K_s, 1), cts(K_blk * K_s, 2)
+    def chunk_cts(stream):                                     # [K_blk][mine] ciphertexts of this rank's chunks
+        full = cts(K_blk * K_s, stream).view(K_blk, K_s, 2, l0, N)
+        return full[:, first:first + mine].contiguous()
+
+    x, a = chunk_cts(1), chunk_cts(2)
     Bc, Cc = cts(K_blk, 3), cts(K_blk, 4)
-    masks = [S.hashed_residues(seed, 10 + i, q, N, device="cuda").contiguous() for i in range(4)]
+    masks = [S.hashed_residues(seed, 10 + i, q, N, device=dev).contiguous() for i in range(4)]
     linj = l0 - 2 - 2 * 8 + 1
-    out = torch.empty((K_blk, K_s, 2, linj - 3, N), dtype=torch.int64, device="cuda")
+    out = torch.empty((K_blk, max(mine, 1), 2, linj - 3, N), dtype=torch.int64, device=dev)
     adj = [(1 << 49) + 12345 * i for i in range((l0 + 1) ** 2)]
-    desc = fesc.ScanDesc(L, H, P, d_s, B, 0, l0, base, int(args.hoist))
+    desc = fesc.ScanDesc(L, mine * hpc, P, d_s, B, 0, l0, base, int(args.hoist))
     torch.cuda.empty_cache()
 
     def step():
-        ctx.scan_contract(x, a, Bc, Cc, desc, masks[0], masks[1], masks[2], masks[3][:linj - 2], adj, adj, out)
+        if mine:
+            ctx.scan_contract(x, a, Bc, Cc, desc, masks[0], masks[1], masks[2], masks[3][:linj - 2], adj, adj, out)
+        return gather_chunk_outputs(out[:, :mine], parts, rank, world, K_blk, K_s) if world > 1 else out
 
     breakdown = None
     if args.workload == "scan_slice":
@@ -633,23 +683,33 @@ def run_scan(args):
         ctx.profile_enable([])
         breakdown = {k: {"ms": round(v[0], 1), "records": v[1]} for k, v in fam.items() if v[1]}
     ctx.sync()
+    barrier()
     c0 = ctx.counters()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     step()
     e1.record()
     ctx.sync()
+    barrier()
     c1 = ctx.counters()
-    ms = e0.elapsed_time(e1)
-    ks = c1[1] - c0[1]
-    print(json.dumps({"metric": "scan-contract key-switches/s", "value": ks / (ms * 1e-3), "unit": "key-switches/s",
-                      "n_gpus": 1, "steps": 1, "warmup": 1 if args.workload == "scan_slice" else 0, "ms_per_step": ms,
-                      "higher_is_better": True, "dtype": "u64", "data": "synthetic",
-                      "config": {"workload": "%s: L=%d, H=%d, P=64, d_s=128, B_blk=256, K_s=%d, N=2^16, 24 limbs, %s"
-                                             % (args.workload, L, H, K_s,
-                                                "radix-4 hoisted rotate-and-add chains" if args.hoist else "plain rotations")},
-                      "key_switches": ks, "limb_transforms": c1[0] - c0[0], "gpu_launches": c1[4] - c0[4],
-                      "scratch_gib": c1[3] / 2**30, "kernel_breakdown": breakdown}), flush=True)
+    ms = max_over_ranks(e0.elapsed_time(e1), dev)
+    ks_local = torch.tensor([float(c1[1] - c0[1])], dtype=torch.float64, device=dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(ks_local)
+    ks = int(ks_local.item())
+    if rank == 0:
+        print(json.dumps({"metric": "scan-contract key-switches/s", "value": ks / (ms * 1e-3), "unit": "key-switches/s",
+                          "n_gpus": world, "steps": 1, "warmup": 1 if args.workload == "scan_slice" else 0,
+                          "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "dtype": "u64",
+                          "data": "synthetic",
+                          "config": {"workload": "%s: L=%d, H=%d, P=64, d_s=128, B_blk=256, K_s=%d, N=2^16, 24 limbs, %s"
+                                                 % (args.workload, L, H, K_s,
+                                                    "radix-4 hoisted rotate-and-add chains" if args.hoist else "plain rotations"),
+                                     "parallelism": "state chunks in pairs over %d rank(s): %s; one all-gather of the outputs"
+                                                    % (world, [c for _, c in parts])},
+                          "key_switches": ks, "limb_transforms": c1[0] - c0[0], "gpu_launches": c1[4] - c0[4],
+                          "scratch_gib": c1[3] / 2**30, "kernel_breakdown": breakdown}), flush=True)
 
 
 def run_rotations(args):

@@ -62,3 +62,55 @@ def test_workload_counts():
     assert tbs * gin == 48 and nout * bench.N2 * gin * bench.N1 == 10752 and tbs * nout == 224
     assert tbs * nout * bench.N2 * gin * bench.N1 == 172032
     assert tbs * gin * (bench.N1 - 1) == 1488 and tbs * nout * (bench.N2 - 1) == 1568
+
+
+def test_scan_partition_keeps_chunk_pairs_together():
+    sys.path.insert(0, ROOT)
+    import bench
+
+    for K_s in (12, 11, 2, 1):
+        for world in (1, 2, 3, 4, 6, 8):
+            parts = bench.scan_partition(K_s, world)
+            assert len(parts) == world
+            covered = []
+            for first, count in parts:
+                assert first % 2 == 0                              # a rank starts on a pair boundary
+                covered += list(range(first, first + count))
+            assert covered == list(range(K_s))                     # every chunk exactly once, in order
+            sizes = [-(-c // 2) for _, c in parts]
+            assert max(sizes) - min(sizes) <= 1                    # pairs are balanced to within one
+    assert [c for _, c in bench.scan_partition(12, 4)] == [2, 4, 2, 4]
+    assert [c for _, c in bench.scan_partition(12, 3)] == [4, 4, 4]
+
+
+GATHER_WORKER = r"""
+import os, sys, json
+sys.path.insert(0, %r)
+import torch, bench
+rank, world = bench.dist_setup("gloo")
+K_blk, K_s = 2, 5
+parts = bench.scan_partition(K_s, world)
+first, mine = parts[rank]
+local = torch.empty((K_blk, mine, 3), dtype=torch.int64)
+for j in range(K_blk):
+    for c in range(mine):
+        local[j, c] = 100 * j + (first + c)
+full = bench.gather_chunk_outputs(local, parts, rank, world, K_blk, K_s)
+want = torch.tensor([[[100 * j + c] * 3 for c in range(K_s)] for j in range(K_blk)])
+print(json.dumps({"rank": rank, "ok": bool((full == want).all()), "parts": parts}))
+"""
+
+
+def test_two_gloo_ranks_gather_their_chunk_outputs_once():
+    port = _free_port()
+    procs = []
+    for r in range(2):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, "-c", GATHER_WORKER % ROOT], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.PIPE, text=True))
+    for p in procs:
+        o, e = p.communicate(timeout=120)
+        assert p.returncode == 0, e
+        res = json.loads(o.strip().splitlines()[-1])
+        assert res["ok"] and res["parts"] == [[0, 2], [2, 3]]      # 5 chunks: pair (0,1) | pair (2,3) and the odd chunk 4
