@@ -370,6 +370,30 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                  "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier phase that nothing completes, with a small poll budget;
+// the wait runs out, the status word is set and the kernel returns (no copy is in flight, nothing faults).
+__global__ void k_wait_limit_selftest(uint32_t* __restrict__ status) {
+    __shared__ __align__(8) unsigned long long bar;
+    const uint32_t b = (uint32_t)__cvta_generic_to_shared(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    uint32_t late = 1;
+    for (uint32_t it = 0; it < 4096 && late; it++) {
+        late = !mbar_try_wait(b, 0);
+        if (late) __nanosleep(32);
+    }
+    if (__any_sync(0xffffffffu, late) && threadIdx.x == 0) atomicExch(status, 2u);
+}
+extern "C" int fesc_selftest_wait_limit(fesc_ctx* ctx, void* stream) {
+    if (!ctx) return FESC_EINVAL;
+    k_wait_limit_selftest<<<1, 32, 0, (cudaStream_t)stream>>>(ctx->d_status);
+    FESC_CHECK_CUDA(ctx, cudaGetLastError());
+    return FESC_OK;
+}
+
 template <int BT>
 __global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ ext,
                                                       const u64* __restrict__ key, u64* __restrict__ acc,

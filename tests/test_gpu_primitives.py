@@ -226,6 +226,27 @@ def test_empty_batches_and_rejected_arguments():
     assert np.array_equal(to_host(one), ref)
 
 
+def test_bounded_wait_runs_out_and_is_reported():
+    """A device-side wait that nothing completes gives up after its poll budget: the next sync reports
+    FESC_ETIMEOUT once, and the context keeps working (no fault, no hang)."""
+    import torch
+    import paper_2608_17442_b200 as fesc
+
+    ctx, orc, p = ctx_pair("toy")
+    ctx.sync()
+    ctx.selftest_wait_limit()
+    with pytest.raises(fesc.FescError) as e:
+        ctx.sync()
+    assert e.value.code == fesc.ETIMEOUT
+    ctx.sync()                                          # the status word was cleared
+    data = to_dev(random_ct(orc, 14, 0, 6, 1))
+    ref = to_host(data).copy()
+    ctx.intt(data, 2, 0, 6)
+    ctx.ntt(data, 2, 0, 6)
+    ctx.sync()
+    assert np.array_equal(to_host(data), ref)
+
+
 def test_workload_1_end_to_end():
     """Tiny CKKS: 4 ciphertexts x random plaintext vector, rotate by +1 and +5, decrypt; residues
     bit-exact and slots within 2^-16 of the float64 result."""
