@@ -247,6 +247,45 @@ def test_bounded_wait_runs_out_and_is_reported():
     assert np.array_equal(to_host(data), ref)
 
 
+@pytest.mark.parametrize("level", [1, 2, 3, 4, 5, 7, 8, 13, 21, 23])
+def test_key_switch_paths_at_every_digit_shape(level):
+    """Levels that leave a partial last digit, a single digit or a single limb, with batches of 1 to 6 ciphertexts
+    (every per-thread batch tile of the inner product): plain, hoisted and rotate-and-add rotations, ct x ct and
+    rescale against the oracle."""
+    import torch
+
+    pair = ctx_pair("small")
+    ctx, orc, _ = pair
+    for r, kid in ((2, 95), (-7, 96)):
+        add_key(pair, r, kid)
+    batch = 1 + level % 6
+    ct = random_ct(orc, 15, level, level, batch)
+    other = random_ct(orc, 16, level, level, batch)
+    dev = to_dev(ct)
+    out = torch.empty_like(dev)
+    ctx.rotate(dev, out, batch, level, 95)
+    rot = to_host(out)
+    hout = torch.empty((2, batch, 2, level, orc.N), dtype=torch.int64, device="cuda")
+    ctx.rotate_hoisted(dev, hout, batch, level, [95, 96])
+    hrot = to_host(hout)
+    ctx.rotate_sum_hoisted(dev, out, batch, level, [95, 96])
+    srot = to_host(out)
+    ctx.ct_ct_mul(dev, to_dev(other), out, batch, level)
+    prod = to_host(out)
+    for b in range(batch):
+        assert np.array_equal(rot[b], orc.rotate(ct[b], 95)), (level, b)
+        want = orc.rotate_hoisted(ct[b], [95, 96])
+        assert np.array_equal(hrot[0, b], want[0]) and np.array_equal(hrot[1, b], want[1]), (level, b)
+        assert np.array_equal(srot[b], orc.rotate_sum_hoisted(ct[b], [95, 96])), (level, b)
+        assert np.array_equal(prod[b], orc.ct_ct_mul(ct[b], other[b])), (level, b)
+    if level >= 2:
+        res = torch.empty((batch, 2, level - 1, orc.N), dtype=torch.int64, device="cuda")
+        ctx.rescale(dev, res, batch, level)
+        got = to_host(res)
+        for b in range(batch):
+            assert np.array_equal(got[b], orc.rescale(ct[b])), (level, b)
+
+
 def test_workload_1_end_to_end():
     """Tiny CKKS: 4 ciphertexts x random plaintext vector, rotate by +1 and +5, decrypt; residues
     bit-exact and slots within 2^-16 of the float64 result."""
