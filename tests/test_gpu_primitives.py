@@ -286,6 +286,36 @@ def test_key_switch_paths_at_every_digit_shape(level):
             assert np.array_equal(got[b], orc.rescale(ct[b])), (level, b)
 
 
+@pytest.mark.parametrize("level,batch", [(4, 5), (7, 3), (14, 2)])
+def test_full_ring_low_levels(level, batch):
+    """N = 2^16 at the low levels the scan-contract works at (injection, reduction, output): rotations in all three
+    modes, ct x ct and rescale against the oracle."""
+    import torch
+
+    pair = ctx_pair("full")
+    ctx, orc, _ = pair
+    for r, kid in ((1, 97), (-16, 98)):
+        add_key(pair, r, kid)
+    ct = random_ct(orc, 17, level, level, batch)
+    other = random_ct(orc, 18, level, level, batch)
+    dev = to_dev(ct)
+    out = torch.empty_like(dev)
+    ctx.rotate(dev, out, batch, level, 97)
+    rot = to_host(out)
+    ctx.rotate_sum_hoisted(dev, out, batch, level, [97, 98])
+    srot = to_host(out)
+    ctx.ct_ct_mul(dev, to_dev(other), out, batch, level)
+    prod = to_host(out)
+    res = torch.empty((batch, 2, level - 1, orc.N), dtype=torch.int64, device="cuda")
+    ctx.rescale(dev, res, batch, level)
+    resc = to_host(res)
+    for b in range(batch):
+        assert np.array_equal(rot[b], orc.rotate(ct[b], 97)), (level, b)
+        assert np.array_equal(srot[b], orc.rotate_sum_hoisted(ct[b], [97, 98])), (level, b)
+        assert np.array_equal(prod[b], orc.ct_ct_mul(ct[b], other[b])), (level, b)
+        assert np.array_equal(resc[b], orc.rescale(ct[b])), (level, b)
+
+
 def test_workload_1_end_to_end():
     """Tiny CKKS: 4 ciphertexts x random plaintext vector, rotate by +1 and +5, decrypt; residues
     bit-exact and slots within 2^-16 of the float64 result."""
