@@ -291,14 +291,17 @@ __device__ __forceinline__ void fp_reduce8(double (&x)[8], double q, double qinv
 
 template <bool INV>
 __device__ __forceinline__ void strided_body_fp(u64* __restrict__ p, double* __restrict__ sm, const double* __restrict__ tw,
-                                                const PrimeConst& pc) {
+                                                const PrimeConst& pc, int in_double) {
     const double q = pc.qd, qinv = pc.qinvd;
     const uint32_t col = threadIdx.x & (NTT_COLS - 1), sub = threadIdx.x / NTT_COLS;
     const uint32_t h2 = sub >> 2, l2 = sub & 3;
     double x[8];
     if (!INV) {
 #pragma unroll
-        for (int k = 0; k < 8; k++) x[k] = fp_from_u64(p[(size_t)(k * 32 + sub) * 256 + col]);   // canonical, below q
+        for (int k = 0; k < 8; k++) {   // canonical words (below q), or doubles with |x| <= q/2 from a conversion kernel
+            const u64 v = p[(size_t)(k * 32 + sub) * 256 + col];
+            x[k] = in_double ? __longlong_as_double((long long)v) : fp_from_u64(v);
+        }
         fp_fwd_round3(x, tw, 1, 2, 4, q, qinv);                                                  // below 3.47q
         fp_reduce8(x, q, qinv);
 #pragma unroll
@@ -418,7 +421,7 @@ template <bool INV>
 __global__ void __launch_bounds__(NTT_COLS * 32) ntt16_strided(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
                                                      const double* __restrict__ twf_all,
                                                      const PrimeConst* __restrict__ pcs, RowMap map,
-                                                     uint32_t row_base) {
+                                                     uint32_t row_base, int in_double) {
     const uint32_t row = blockIdx.y;
     const uint32_t pi = map.prime[(row_base + row) % map.period];
     if (pi == 0xFF) return;
@@ -427,7 +430,7 @@ __global__ void __launch_bounds__(NTT_COLS * 32) ntt16_strided(u64* __restrict__
     const ulonglong2* tw = tw_all + (size_t)pi * N16;
     u64* p = data + (size_t)row * N16 + blockIdx.x * NTT_COLS;
     if (pc.q < FP_LIMIT)
-        strided_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc);
+        strided_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, in_double);
     else if (pc.q < WIDE_LIMIT)
         strided_body<INV, true>(p, sm, tw, pc);
     else
@@ -581,7 +584,7 @@ __global__ void __launch_bounds__(256) ntt_small(u64* __restrict__ data, const u
     }
 }
 
-int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool inverse, cudaStream_t st) {
+int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool inverse, cudaStream_t st, bool in_double) {
     if (rows == 0) return FESC_OK;
     if (rows > 0x7fffffffu) return fesc_fail(ctx, FESC_EINVAL, "ntt: too many rows");
     const ulonglong2* tw = inverse ? ctx->d_itw : ctx->d_tw;
@@ -601,11 +604,11 @@ int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool 
             dim3 gs(256 / NTT_COLS, (unsigned)chunk), gc(256 / NTT_WARPS, (unsigned)chunk);
             u64* base = d_data + r0 * (size_t)N16;
             if (!inverse) {
-                ntt16_strided<false><<<gs, NTT_COLS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb);
+                ntt16_strided<false><<<gs, NTT_COLS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb, in_double ? 1 : 0);
                 ntt16_contig<false><<<gc, NTT_WARPS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb);
             } else {
                 ntt16_contig<true><<<gc, NTT_WARPS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb);
-                ntt16_strided<true><<<gs, NTT_COLS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb);
+                ntt16_strided<true><<<gs, NTT_COLS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb, 0);
             }
             launches += 2;
         }

@@ -139,7 +139,8 @@ __device__ __forceinline__ void stv(u64* __restrict__ dst, const u64 (&r)[VEC]) 
 template <int ALPHA, int VEC>
 __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u64* __restrict__ ext,
                                                const ModUpDigit* __restrict__ tab, const PrimeConst* __restrict__ pcs,
-                                               uint32_t N, uint32_t level, uint32_t n_q, uint32_t K, uint32_t beta) {
+                                               uint32_t N, uint32_t level, uint32_t n_q, uint32_t K, uint32_t beta,
+                                               int out_double) {
     // VEC adjacent coefficients per thread: every table word and every prime constant serves VEC products
     const uint32_t c = (blockIdx.x * blockDim.x + threadIdx.x) * VEC;
     const uint32_t j = blockIdx.y, b = blockIdx.z;
@@ -187,7 +188,7 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
                     for (int v = 0; v < VEC; v++) s[v] += fp_modmul(yd[a][v], m, q, qinv);
                 }
 #pragma unroll
-            for (int v = 0; v < VEC; v++) r[v] = fp_store(s[v], q, qinv);
+            for (int v = 0; v < VEC; v++) r[v] = out_double ? fp_handoff(s[v], q, qinv) : fp_store(s[v], q, qinv);
         } else {
             const PrimeConst pc = pcs[pt];
 #pragma unroll
@@ -197,6 +198,8 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
                 for (int a = 0; a < ALPHA; a++)
                     if (a < n_src) mac128(acc, y[a][v], dg->mat[a][pt]);
                 r[v] = reduce128(acc.hi, acc.lo, pc);
+                // the hand-over format follows the TARGET prime (the transform picks its arithmetic by that prime)
+                if (out_double && pc.q < FESC_FP_LIMIT) r[v] = (u64)__double_as_longlong(fp_load(r[v], pc.qd));
             }
         }
         stv<VEC>(out + (size_t)t * N, r);
@@ -539,7 +542,7 @@ template <int VEC>
 __global__ void __launch_bounds__(256) k_moddown_conv(const u64* __restrict__ acc, u64* __restrict__ u,
                                                       const ModDownTab* __restrict__ tab,
                                                       const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
-                                                      uint32_t n_q, uint32_t K) {
+                                                      uint32_t n_q, uint32_t K, int out_double) {
     // VEC adjacent coefficients per thread: every table word and every prime constant serves VEC products
     const uint32_t c = (blockIdx.x * blockDim.x + threadIdx.x) * VEC;
     const uint32_t bp = blockIdx.y;   // b*2 + p
@@ -593,7 +596,7 @@ __global__ void __launch_bounds__(256) k_moddown_conv(const u64* __restrict__ ac
                     }
                 }
 #pragma unroll
-            for (int v = 0; v < VEC; v++) r[v] = fp_store(s[v], q, qinv);
+            for (int v = 0; v < VEC; v++) r[v] = out_double ? fp_handoff(s[v], q, qinv) : fp_store(s[v], q, qinv);
         } else {
             const PrimeConst pc = pcs[i];
 #pragma unroll
@@ -649,12 +652,13 @@ static int ks_decompose(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint
     if ((rc = ntt_launch(ctx, ws.dcoef, (size_t)batch * level, m, true, st)) != FESC_OK) return rc;
     // 2. ModUp
     const ModUpDigit* tab = ctx->tabs.d_modup + (size_t)(level - 1) * ctx->beta_max;
+    const int dbl = ctx->log_n == 16;   // the N = 2^16 forward transform takes doubles straight from the conversion
     const bool vec2 = N % (256 * KS_VEC) == 0;
     dim3 gmu(vec2 ? N / (256 * KS_VEC) : gx, beta, batch);
 #define MODUP(A)                                                                                           \
     do {                                                                                                   \
-        if (vec2) k_modup<A, KS_VEC><<<gmu, 256, 0, st>>>(ws.dcoef, ws.ext, tab, ctx->d_pc, N, level, nq, K, beta); \
-        else k_modup<A, 1><<<gmu, 256, 0, st>>>(ws.dcoef, ws.ext, tab, ctx->d_pc, N, level, nq, K, beta);  \
+        if (vec2) k_modup<A, KS_VEC><<<gmu, 256, 0, st>>>(ws.dcoef, ws.ext, tab, ctx->d_pc, N, level, nq, K, beta, dbl); \
+        else k_modup<A, 1><<<gmu, 256, 0, st>>>(ws.dcoef, ws.ext, tab, ctx->d_pc, N, level, nq, K, beta, dbl);  \
     } while (0)
     prof_begin(ctx, PF_MODUP, st);
     if (alpha <= 1) MODUP(1);
@@ -672,7 +676,7 @@ static int ks_decompose(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint
             bool own = t < level && t / alpha == j;
             m.prime[j * rows + t] = own ? 0xFF : (uint8_t)(t < level ? t : nq + (t - level));
         }
-    if ((rc = ntt_launch(ctx, ws.ext, (size_t)batch * beta * rows, m, false, st)) != FESC_OK) return rc;
+    if ((rc = ntt_launch(ctx, ws.ext, (size_t)batch * beta * rows, m, false, st, dbl != 0)) != FESC_OK) return rc;
     FESC_CHECK_CUDA(ctx, cudaGetLastError());
     return FESC_OK;
 }
@@ -736,13 +740,13 @@ static int ks_moddown(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint32
     if ((rc = ntt_launch(ctx, ws.acc, (size_t)batch * 2 * rows, m, true, st)) != FESC_OK) return rc;
     prof_begin(ctx, PF_MODDOWN, st);
     if (N % (256 * KS_VEC) == 0)
-        k_moddown_conv<KS_VEC><<<dim3(N / (256 * KS_VEC), batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K);
+        k_moddown_conv<KS_VEC><<<dim3(N / (256 * KS_VEC), batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K, ctx->log_n == 16);
     else
-        k_moddown_conv<1><<<dim3(gx, batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K);
+        k_moddown_conv<1><<<dim3(gx, batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K, ctx->log_n == 16);
     prof_end(ctx, PF_MODDOWN, st);
     m.period = level;
     for (uint32_t i = 0; i < level; i++) m.prime[i] = (uint8_t)i;
-    if ((rc = ntt_launch(ctx, ws.u, (size_t)batch * 2 * level, m, false, st)) != FESC_OK) return rc;
+    if ((rc = ntt_launch(ctx, ws.u, (size_t)batch * 2 * level, m, false, st, ctx->log_n == 16)) != FESC_OK) return rc;
     prof_begin(ctx, PF_MODDOWN, st);
     k_moddown_finish<<<dim3(gx, level, batch * 2), 256, 0, st>>>(ws.acc, ws.u, out, out_stride, ctx->tabs.d_moddown,
                                                                  ctx->d_pc, N, level, K, add_mask);
