@@ -60,6 +60,7 @@ def lib():
             "fesc_ctx_create": [c.POINTER(vp), u32, c.POINTER(u64), u32, u32, u32, u64],
             "fesc_ctx_destroy": [vp],
             "fesc_sync": [vp, vp],
+            "fesc_ctx_trim": [vp],
             "fesc_selftest_wait_limit": [vp, vp],
             "fesc_ctx_add_galois_key": [vp, i32, u32],
             "fesc_ctx_export_key": [vp, u32, vp, vp],
@@ -132,6 +133,10 @@ class Context:
             self.close()
         except Exception:      # interpreter shutdown: module globals may already be gone
             pass
+
+    def trim(self):
+        """Release the scratch arena (it is reserved again on demand)."""
+        self._chk(lib().fesc_ctx_trim(self.h))
 
     def selftest_wait_limit(self):
         self._chk(lib().fesc_selftest_wait_limit(self.h, _stream()))

@@ -414,6 +414,18 @@ extern "C" int fesc_ctx_destroy(fesc_ctx* ctx) {
     return FESC_OK;
 }
 
+extern "C" int fesc_ctx_trim(fesc_ctx* ctx) {
+    if (!ctx) return FESC_EINVAL;
+    if (ctx->d_scratch) {
+        FESC_CHECK_CUDA(ctx, cudaDeviceSynchronize());
+        cudaFree(ctx->d_scratch);
+        ctx->d_scratch = nullptr;
+        ctx->scratch_bytes = 0;
+        ctx->counters[3] = 0;
+    }
+    return FESC_OK;
+}
+
 extern "C" const char* fesc_last_error(const fesc_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
 
 extern "C" int fesc_sync(fesc_ctx* ctx, void* stream) {

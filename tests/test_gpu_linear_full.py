@@ -22,6 +22,7 @@ def test_in_proj_full_size_sampled_against_oracle(hoist, defer):
 
     pair = ctx_pair("full")
     ctx, orc, p = pair
+    ctx.trim()                     # an earlier test may have left a large scratch arena on this cached context
     gin, nout, tbs = bench.workload_dims()
     assert (gin, nout, tbs) == (3, 14, 16)
     n1, n2, T, level = bench.N1, bench.N2, bench.T_SEG, bench.LEVEL
