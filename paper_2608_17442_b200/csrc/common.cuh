@@ -233,8 +233,9 @@ static inline int fesc_fail(fesc_ctx* ctx, int code, const std::string& msg) {
 // rows: number of N-word rows starting at d_data; map gives the prime per row.
 // in_double (forward, N = 2^16 only): rows on primes below 2^50 hold doubles with |x| <= q/2 (bit patterns) written by a
 // basis-conversion kernel instead of canonical words.
+// out_double (forward, N = 2^16 only): such rows are left as doubles with |x| <= q/2 for a consumer that computes in FP64.
 int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool inverse, cudaStream_t st,
-               bool in_double = false);
+               bool in_double = false, bool out_double = false);
 // double with |x| <= q/2 as handed to the forward transform
 __device__ __forceinline__ u64 fp_handoff(double s, double q, double qinv) {
     return (u64)__double_as_longlong(fp_reduce(s, q, qinv));

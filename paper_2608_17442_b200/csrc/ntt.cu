@@ -361,7 +361,7 @@ __device__ __forceinline__ void strided_body_fp(u64* __restrict__ p, double* __r
 
 template <bool INV>
 __device__ __forceinline__ void contig_body_fp(u64* __restrict__ p, double* __restrict__ sm, const double* __restrict__ tw,
-                                               const PrimeConst& pc, uint32_t pre) {
+                                               const PrimeConst& pc, uint32_t pre, int out_double) {
     const double q = pc.qd, qinv = pc.qinvd;
     const uint32_t sub = threadIdx.x & 31;
     const uint32_t h2 = sub >> 2, l2 = sub & 3;
@@ -386,7 +386,9 @@ __device__ __forceinline__ void contig_body_fp(u64* __restrict__ p, double* __re
         fp_fwd_round2(x, tw, 64 * pre + 2 * sub, 128 * pre + 4 * sub, q, qinv);
         ulonglong2* o = reinterpret_cast<ulonglong2*>(p + sub * 8);
 #pragma unroll
-        for (int k = 0; k < 4; k++) o[k] = make_ulonglong2(fp_store(x[2 * k], q, qinv), fp_store(x[2 * k + 1], q, qinv));
+        for (int k = 0; k < 4; k++)   // canonical words, or doubles with |x| <= q/2 for a consumer that computes in FP64
+            o[k] = out_double ? make_ulonglong2(fp_handoff(x[2 * k], q, qinv), fp_handoff(x[2 * k + 1], q, qinv))
+                              : make_ulonglong2(fp_store(x[2 * k], q, qinv), fp_store(x[2 * k + 1], q, qinv));
     } else {
         const ulonglong2* in = reinterpret_cast<const ulonglong2*>(p + sub * 8);
 #pragma unroll
@@ -510,7 +512,7 @@ template <bool INV>
 __global__ void __launch_bounds__(NTT_WARPS * 32) ntt16_contig(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
                                                     const double* __restrict__ twf_all,
                                                     const PrimeConst* __restrict__ pcs, RowMap map,
-                                                    uint32_t row_base) {
+                                                    uint32_t row_base, int out_double) {
     const uint32_t row = blockIdx.y;
     const uint32_t pi = map.prime[(row_base + row) % map.period];
     if (pi == 0xFF) return;
@@ -522,7 +524,7 @@ __global__ void __launch_bounds__(NTT_WARPS * 32) ntt16_contig(u64* __restrict__
     u64* p = data + (size_t)row * N16 + (size_t)blk * 256;
     u64* sm = sm_all + warp * 288;
     if (pc.q < FP_LIMIT)
-        contig_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, 256 + blk);
+        contig_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, 256 + blk, out_double);
     else if (pc.q < WIDE_LIMIT)
         contig_body<INV, true>(p, sm, tw, pc, 256 + blk);
     else
@@ -584,7 +586,8 @@ __global__ void __launch_bounds__(256) ntt_small(u64* __restrict__ data, const u
     }
 }
 
-int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool inverse, cudaStream_t st, bool in_double) {
+int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool inverse, cudaStream_t st, bool in_double,
+               bool out_double) {
     if (rows == 0) return FESC_OK;
     if (rows > 0x7fffffffu) return fesc_fail(ctx, FESC_EINVAL, "ntt: too many rows");
     const ulonglong2* tw = inverse ? ctx->d_itw : ctx->d_tw;
@@ -605,9 +608,9 @@ int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool 
             u64* base = d_data + r0 * (size_t)N16;
             if (!inverse) {
                 ntt16_strided<false><<<gs, NTT_COLS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb, in_double ? 1 : 0);
-                ntt16_contig<false><<<gc, NTT_WARPS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb);
+                ntt16_contig<false><<<gc, NTT_WARPS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb, out_double ? 1 : 0);
             } else {
-                ntt16_contig<true><<<gc, NTT_WARPS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb);
+                ntt16_contig<true><<<gc, NTT_WARPS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb, 0);
                 ntt16_strided<true><<<gs, NTT_COLS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb, 0);
             }
             launches += 2;

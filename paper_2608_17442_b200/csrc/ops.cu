@@ -80,7 +80,11 @@ __device__ __forceinline__ uint32_t galois_src(uint32_t t, uint32_t log_n, u64 g
 struct OwnRows {
     u64* ext;
     uint32_t alpha, beta, rows;
+    int as_double;   // rows on primes below 2^50 are kept as doubles with |x| <= q/2 (the FP64 inner product's format)
 };
+__device__ __forceinline__ u64 own_word(const OwnRows& w, u64 v, const PrimeConst& pc) {
+    return (w.as_double && pc.q < FESC_FP_LIMIT) ? (u64)__double_as_longlong(fp_load(v, pc.qd)) : v;
+}
 __device__ __forceinline__ size_t own_index(const OwnRows& w, uint32_t b, uint32_t l, uint32_t N) {
     return (((size_t)b * w.beta + l / w.alpha) * w.rows + l) * N;
 }
@@ -101,7 +105,7 @@ __global__ void __launch_bounds__(256) k_autom_ct(const u64* __restrict__ in, si
     if (accumulate) v0 = addmod(v0, *o0, pcs[l].q);
     *o0 = v0;
     u64 v = ib[poly + (size_t)l * N + src];
-    d.ext[own_index(d, b, l, N) + t] = v;
+    d.ext[own_index(d, b, l, N) + t] = own_word(d, v, pcs[l]);
     dcoef[((size_t)b * level + l) * N + t] = v;
 }
 
@@ -226,7 +230,8 @@ __global__ void __launch_bounds__(256, INNER_MINB) k_inner(const u64* __restrict
                                                const u64* __restrict__ key, u64* __restrict__ acc,
                                                const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
                                                uint32_t n_q, uint32_t K, uint32_t alpha, uint32_t beta,
-                                               uint32_t batch, uint32_t log_n, u64 g, int accumulate, uint32_t row0) {
+                                               uint32_t batch, uint32_t log_n, u64 g, int accumulate, uint32_t row0,
+                                               int x_double) {
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t t = row0 + blockIdx.y, b0 = blockIdx.z * BT;
     if (c >= N) return;
@@ -276,7 +281,8 @@ __global__ void __launch_bounds__(256, INNER_MINB) k_inner(const u64* __restrict
             const double dkb = fp_from_u64(kb), dka = fp_from_u64(ka);
 #pragma unroll
             for (int i = 0; i < BT; i++) {
-                const double xd = fp_from_u64(x[i]);   // canonical operands: every product is below 0.875q
+                // canonical words (every product below 0.875q) or doubles with |x| <= q/2 left by the producers
+                const double xd = x_double ? __longlong_as_double((long long)x[i]) : fp_from_u64(x[i]);
                 f0[i] += fp_modmul(xd, dkb, q, qinv);
                 f1[i] += fp_modmul(xd, dka, q, qinv);
             }
@@ -403,7 +409,7 @@ __global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ ex
                                                       const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
                                                       uint32_t n_q, uint32_t K, uint32_t alpha, uint32_t beta,
                                                       uint32_t batch, uint32_t log_n, u64 g, int accumulate,
-                                                      uint32_t n_tiles, uint32_t* __restrict__ status) {
+                                                      uint32_t n_tiles, uint32_t* __restrict__ status, int x_double) {
     constexpr int R = 2 + BT;                                // rows per digit: key b, key a, BT ciphertexts
     extern __shared__ __align__(128) u64 smem[];             // [2 stages][beta][R][256] then two barriers
     const uint32_t tid = threadIdx.x;
@@ -481,7 +487,8 @@ __global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ ex
                 const double dkb = fp_from_u64(dj[tid]), dka = fp_from_u64(dj[256 + tid]);
 #pragma unroll
                 for (int i = 0; i < BT; i++) {
-                    const double xd = fp_load(dj[(2 + i) * 256 + si], q);
+                    const u64 xw = dj[(2 + i) * 256 + si];
+                    const double xd = x_double ? __longlong_as_double((long long)xw) : fp_load(xw, q);
                     f0[i] += fp_modmul(xd, dkb, q, qinv);
                     f1[i] += fp_modmul(xd, dka, q, qinv);
                 }
@@ -676,7 +683,7 @@ static int ks_decompose(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint
             bool own = t < level && t / alpha == j;
             m.prime[j * rows + t] = own ? 0xFF : (uint8_t)(t < level ? t : nq + (t - level));
         }
-    if ((rc = ntt_launch(ctx, ws.ext, (size_t)batch * beta * rows, m, false, st, dbl != 0)) != FESC_OK) return rc;
+    if ((rc = ntt_launch(ctx, ws.ext, (size_t)batch * beta * rows, m, false, st, dbl != 0, dbl != 0)) != FESC_OK) return rc;
     FESC_CHECK_CUDA(ctx, cudaGetLastError());
     return FESC_OK;
 }
@@ -694,7 +701,7 @@ static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint
     do {                                                                                                        \
         dim3 gd(gx, NROWS_, (batch + BT_ - 1) / BT_);                                                           \
         k_inner<BT_, PATH_><<<gd, 256, 0, st>>>(ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, \
-                                                beta, batch, ctx->log_n, g, accumulate, ROW0_);                 \
+                                                beta, batch, ctx->log_n, g, accumulate, ROW0_, ctx->log_n == 16); \
     } while (0)
     // data rows on primes below 2^50 and special rows above: one launch per kind, each compiled for its arithmetic
     bool split = true;
@@ -709,7 +716,7 @@ static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint
         FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(k_inner_tma<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         const uint32_t grid = n_tiles < (uint32_t)sms ? n_tiles : (uint32_t)sms;
         k_inner_tma<4><<<grid, 256, smem, st>>>(ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta,
-                                                 batch, ctx->log_n, g, accumulate, n_tiles, ctx->d_status);
+                                                 batch, ctx->log_n, g, accumulate, n_tiles, ctx->d_status, ctx->log_n == 16);
     } else if (split) {
         if (batch >= 3) INNER(4, 1, 0, level);
         else if (batch == 2) INNER(2, 1, 0, level);
@@ -773,7 +780,7 @@ static int key_switch_chunk(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& k
 }
 
 static OwnRows own_rows(const fesc_ctx* ctx, const KsScratch& ws, uint32_t level) {
-    return OwnRows{ws.ext, ctx->alpha, (level + ctx->alpha - 1) / ctx->alpha, level + ctx->n_p};
+    return OwnRows{ws.ext, ctx->alpha, (level + ctx->alpha - 1) / ctx->alpha, level + ctx->n_p, ctx->log_n == 16};
 }
 
 size_t ks_scratch_words(const fesc_ctx* ctx, uint32_t level, uint32_t chunk) {
@@ -824,7 +831,8 @@ int rotate_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, si
 // c0 of every ciphertext through the Galois permutation into out[b][0]; with g == 0, c1 copied to d and dcoef
 __global__ void __launch_bounds__(256) k_hoist_prepare(const u64* __restrict__ in, size_t in_stride, u64* __restrict__ out0,
                                                        size_t out_stride, OwnRows d, u64* __restrict__ dcoef,
-                                                       uint32_t log_n, uint32_t level, u64 g) {
+                                                       uint32_t log_n, uint32_t level, u64 g,
+                                                       const PrimeConst* __restrict__ pcs) {
     const uint32_t N = 1u << log_n;
     const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t l = blockIdx.y, b = blockIdx.z;
@@ -834,7 +842,7 @@ __global__ void __launch_bounds__(256) k_hoist_prepare(const u64* __restrict__ i
         out0[(size_t)b * out_stride + (size_t)l * N + t] = ib[(size_t)l * N + galois_src(t, log_n, g)];
     } else {
         const u64 v = ib[((size_t)level + l) * N + t];
-        d.ext[own_index(d, b, l, N) + t] = v;
+        d.ext[own_index(d, b, l, N) + t] = own_word(d, v, pcs[l]);
         dcoef[((size_t)b * level + l) * N + t] = v;
     }
 }
@@ -886,7 +894,7 @@ int rotate_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64*
         dim3 g((ctx->N + 255) / 256, level, nb);
         const u64* ib = in + (size_t)b0 * in_stride;
         prof_begin(ctx, PF_AUTOM, st);
-        k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, nullptr, 0, own_rows(ctx, ws, level), ws.dcoef, ctx->log_n, level, 0);
+        k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, nullptr, 0, own_rows(ctx, ws, level), ws.dcoef, ctx->log_n, level, 0, ctx->d_pc);
         prof_end(ctx, PF_AUTOM, st);
         int rc = ks_decompose(ctx, ws, level, nb, st);
         if (rc != FESC_OK) return rc;
@@ -894,7 +902,7 @@ int rotate_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64*
             const EvalKey& key = ctx->keys[key_ids[k]];
             u64* ob = out + (size_t)k * key_stride + (size_t)b0 * out_stride;
             prof_begin(ctx, PF_AUTOM, st);
-            k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, ob, out_stride, OwnRows{nullptr, 1, 1, 1}, nullptr, ctx->log_n, level, key.g);
+            k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, ob, out_stride, OwnRows{nullptr, 1, 1, 1, 0}, nullptr, ctx->log_n, level, key.g, ctx->d_pc);
             prof_end(ctx, PF_AUTOM, st);
             rc = ks_apply(ctx, ws, key, level, nb, ob, out_stride, 1, st, key.g);
             if (rc != FESC_OK) return rc;
@@ -946,7 +954,7 @@ int rotate_sum_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, 
         const u64* ib = in + (size_t)b0 * in_stride;
         u64* ob = out + (size_t)b0 * out_stride;
         prof_begin(ctx, PF_AUTOM, st);
-        k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, nullptr, 0, own_rows(ctx, ws, level), ws.dcoef, ctx->log_n, level, 0);
+        k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, nullptr, 0, own_rows(ctx, ws, level), ws.dcoef, ctx->log_n, level, 0, ctx->d_pc);
         k_rotsum_prepare<<<g, 256, 0, st>>>(ib, in_stride, ob, out_stride, ctx->log_n, level, gs, ctx->d_pc);
         prof_end(ctx, PF_AUTOM, st, 2);
         int rc = ks_decompose(ctx, ws, level, nb, st);
@@ -1102,7 +1110,7 @@ __global__ void __launch_bounds__(256) k_tensor(const u64* __restrict__ a, size_
     mac128(s, a1, b0);
     out[b * out_stride + poly + o] = reduce128(s.hi, s.lo, pc);
     const u64 d2 = mulmod(a1, b1, pc);
-    d.ext[own_index(d, b, l, N) + c] = d2;
+    d.ext[own_index(d, b, l, N) + c] = own_word(d, d2, pc);
     dcoef[((size_t)b * level + l) * N + c] = d2;
 }
 
