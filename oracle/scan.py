@@ -35,6 +35,10 @@ filled there);  leaves (p, s) at l1 = l0-2;
 up-sweep stage s -> l1-s;  summaries at lS = l1-logB;  down-sweep stage number d (1..logB-1) works at
 lS-(d-1) -> lS-d;  carries g_j (j >= 1) at lS-(j-1);  injection at linj = l1-2logB+1 -> states at linj-1;
 contraction -> linj-2;  reduction, conjugation, unpacking there;  output mask -> l_out = linj-3.
+
+Other prefix networks (App. "Prefix-Network Selection"; `network` = "ks" Kogge-Stone, "sk" Sklansky; "bk" above is the
+default): stage s = 1..logB combines operands at l1-(s-1) into results at l1-s, every prefix is complete at lS and there
+is no down-sweep, so linj = lS - max(K_blk-2, 0) (the carry before the last block still sits at or above linj).
 """
 from __future__ import annotations
 
@@ -104,10 +108,14 @@ class ScanShape:
         return sorted(am)
 
 
-def levels(l0: int, logB: int, K_blk: int):
+NETWORKS = ("bk", "ks", "sk")
+
+
+def levels(l0: int, logB: int, K_blk: int, network: str = "bk"):
+    assert network in NETWORKS
     l1 = l0 - 2
     lS = l1 - logB
-    linj = l1 - 2 * logB + 1
+    linj = l1 - 2 * logB + 1 if network == "bk" else lS - max(K_blk - 2, 0)
     lout = linj - 3
     assert lout >= 1, "not enough levels"
     assert K_blk <= 1 or lS - (K_blk - 2) >= linj, "carry chain runs below the injection level"
@@ -117,9 +125,10 @@ def levels(l0: int, logB: int, K_blk: int):
 class ScanConsts:
     """Harness-side constants: canonical scales, level-adjust integers, mask plaintexts."""
 
-    def __init__(self, orc: Oracle, shape: ScanShape, l0: int, log_scale: int):
+    def __init__(self, orc: Oracle, shape: ScanShape, l0: int, log_scale: int, network: str = "bk"):
         q = orc.q
-        self.lv = levels(l0, shape.logB, shape.K_blk)
+        self.network = network
+        self.lv = levels(l0, shape.logB, shape.K_blk, network)
         self.S_s = {l0: float(2**log_scale)}
         self.S_p = {l0: float(q[l0 - 1])}
         for l in range(l0, 1, -1):
@@ -216,6 +225,7 @@ class ScanEvaluator:
         steps at once as ct + rot(ct, d) + rot(ct, 2d) + rot(ct, 3d) with one decomposition and one division by P
         (`rotate_sum_hoisted`), and the low digit of the two-digit token offsets uses `rotate_hoisted`."""
         self.o, self.sh, self.c, self.kb, self.hoist = orc, shape, consts, key_base, hoist
+        self.network = consts.network       # the level schedule in `consts` belongs to one network
         self.count = dict(rot=0, conj=0, ctmul=0, adjust=0, ptmul=0, compose=0)
 
     # -- primitives ---------------------------------------------------------------------------
@@ -350,6 +360,37 @@ class ScanEvaluator:
                     T[r - 1] = self.compose(T[k - 1], T[r - 1], lS - (d - 1), need_p=need_p_down)
         return summary
 
+    def kogge_stone(self, T, last_p):
+        """Kogge-Stone network (App. "Prefix-Network Selection"): at stage s every position k > 2^(s-1) (1-based)
+        takes t_k <- t_{k - 2^(s-1)} o t_k with both operands from stage s-1.  B log2 B - (B-1) compositions."""
+        sh, l1 = self.sh, self.c.lv["l1"]
+        for s in range(1, sh.logB + 1):
+            d = 1 << (s - 1)
+            prev = list(T)
+            for k in range(d + 1, sh.B + 1):
+                T[k - 1] = self.compose(prev[k - d - 1], prev[k - 1], l1 - (s - 1), need_p=(s < sh.logB or last_p))
+        return T[sh.B - 1]
+
+    def sklansky(self, T, last_p):
+        """Sklansky network: at stage s the positions of the upper half of every aligned block of 2^s (0-based
+        k in [b 2^s + 2^(s-1), (b+1) 2^s)) take t_k <- t_{b 2^s + 2^(s-1) - 1} o t_k.  (B/2) log2 B compositions."""
+        sh, l1 = self.sh, self.c.lv["l1"]
+        for s in range(1, sh.logB + 1):
+            half = 1 << (s - 1)
+            prev = list(T)
+            for b in range(sh.B >> s):
+                src = (b << s) + half - 1
+                for k in range(src + 1, (b + 1) << s):
+                    T[k] = self.compose(prev[src], prev[k], l1 - (s - 1), need_p=(s < sh.logB or last_p))
+        return T[sh.B - 1]
+
+    def prefix_network(self, T, later_block):
+        """In-place inclusive prefixes of the block's tuples; returns the block summary (at level lS).  The decay
+        products that only an incoming state would use are not formed for the first block."""
+        if self.network == "bk":
+            return self.brent_kung(T, need_p_down=later_block)
+        return (self.kogge_stone if self.network == "ks" else self.sklansky)(T, later_block)
+
     def run(self, ctX, ctA, ctB, ctC):
         """ctX, ctA [K_blk, K_s, 2, l0, N]; ctB, ctC [K_blk, 2, l0, N] -> out [K_blk, K_s, 2, l_out, N]."""
         sh, c, o = self.sh, self.c, self.o
@@ -363,7 +404,7 @@ class ScanEvaluator:
             v = [[None] * sh.K_s for _ in range(sh.B)]
             for kap in range(sh.K_s):
                 T = self.leaves(ctX[j, kap], ctA[j, kap], brB)
-                summary = self.brent_kung(T, need_p_down=(j > 0))
+                summary = self.prefix_network(T, j > 0)
                 g = carry[kap]
                 for t in range(sh.B):
                     sP = self.adjust(T[t][1], linj - 1, "s")
@@ -407,12 +448,14 @@ class ScanEvaluator:
         return o.mul_monomial_half(o.mul_monomial_half(o.mul_monomial_half(ct)))
 
 
-def closed_form_counts(shape: ScanShape):
+def closed_form_counts(shape: ScanShape, network: str = "bk"):
     """Counts the dataflow must reproduce (pins against the paper's ledgers)."""
     sh = shape
-    bk = 2 * (sh.B - 1) - sh.logB                     # Brent-Kung compositions for B positions
+    per_block = dict(bk=2 * (sh.B - 1) - sh.logB,                 # compositions of each network over B positions
+                     ks=sh.B * sh.logB - (sh.B - 1),
+                     sk=(sh.B // 2) * sh.logB)[network]
     return dict(
-        compose=sh.K_blk * sh.K_s * bk,
+        compose=sh.K_blk * sh.K_s * per_block,
         reduce_rot=sh.K_blk * sh.B * (-(-sh.K_s // 2)) * int(math.log2(sh.d_s)),
         reduce_conj=sh.K_blk * sh.B * (sh.K_s // 2),
     )

@@ -51,6 +51,36 @@ def test_brent_kung_network_counts_and_prefixes(B):
     assert all(cover[k] == (1, k) for k in range(1, B + 1))
 
 
+def _ks_nodes(B):
+    """Kogge-Stone stages (1-based positions): stage s, every k > 2^(s-1) combines with k - 2^(s-1)."""
+    return [[(k - (1 << (s - 1)), k) for k in range((1 << (s - 1)) + 1, B + 1)] for s in range(1, int(math.log2(B)) + 1)]
+
+
+def _sk_nodes(B):
+    """Sklansky stages (1-based positions): the upper half of every aligned block of 2^s takes the lower half's last."""
+    stages = []
+    for s in range(1, int(math.log2(B)) + 1):
+        h = 1 << (s - 1)
+        stages.append([(b * 2 * h + h, k) for b in range(B >> s) for k in range(b * 2 * h + h + 1, (b + 1) * 2 * h + 1)])
+    return stages
+
+
+@pytest.mark.parametrize("B", [4, 8, 16, 256])
+def test_kogge_stone_and_sklansky_counts_and_prefixes(B):
+    logB = int(math.log2(B))
+    for stages, total in ((_ks_nodes(B), B * logB - (B - 1)), (_sk_nodes(B), B // 2 * logB)):
+        assert len(stages) == logB and sum(len(st) for st in stages) == total     # App. "Prefix-Network Selection"
+        cover = {k: (k, k) for k in range(1, B + 1)}
+        for st in stages:
+            prev = dict(cover)                                 # both operands come from the previous stage
+            for l, r in st:
+                assert prev[l][1] + 1 == prev[r][0]
+                cover[r] = (prev[l][0], prev[r][1])
+        assert all(cover[k] == (1, k) for k in range(1, B + 1))
+    assert [len(st) for st in _ks_nodes(B)] == [B - (1 << (s - 1)) for s in range(1, logB + 1)]
+    assert all(len(st) == B // 2 for st in _sk_nodes(B))
+
+
 def _golden(name):
     import os
     path = os.path.join(os.path.dirname(__file__), "golden", name)
@@ -83,12 +113,12 @@ def test_paper_ledger_values():
     assert 2 * 768 // 768 and 2 * 24 * 64 + 2 * 128 + 24 == 3352              # d_out of in_proj
 
 
-def _run(name, hoist=False, **shape_kw):
+def _run(name, hoist=False, network="bk", **shape_kw):
     p = S.params(name)
     orc = Oracle(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
     sh = ScanShape(orc.n, **shape_kw)
     x, a, B, C = S.scan_inputs(p["seed"], sh.L, sh.H, sh.P, 1, sh.d_s)
-    c = ScanConsts(orc, sh, p["n_q"], p["log_scale"])
+    c = ScanConsts(orc, sh, p["n_q"], p["log_scale"], network)
     add_scan_keys(orc, sh, hoist=hoist)
     ev = ScanEvaluator(orc, sh, c, hoist=hoist)
     out = ev.run(*encrypt_inputs(orc, sh, c, x, a, B, C))
@@ -129,3 +159,20 @@ def test_hoisted_mode_same_values():
     sh, ev, m, ref = _run("scan_small", hoist=True, L=64, H=3, P=4, d_s=4, B_blk=32)
     assert (sh.K_s, sh.K_blk, sh.dg) == (3, 2, 16)
     assert np.abs(m - ref).max() < 2.0**-22
+
+
+@pytest.mark.parametrize("network", ["ks", "sk"])
+def test_other_prefix_networks(network):
+    """Kogge-Stone and Sklansky networks (App. "Prefix-Network Selection"): composition counts of the closed forms,
+    the shallower level schedule, and the same contract output as the recurrence (toy shape; analogue with carries
+    over three blocks and a partial last block)."""
+    sh, ev, m, ref = _run("scan_toy", network=network, L=4, H=2, P=4, d_s=2, B_blk=4)
+    assert ev.count["compose"] == closed_form_counts(sh, network)["compose"] == {"ks": 10, "sk": 8}[network]
+    assert np.abs(m - ref).max() < 2.0**-24
+    sh, ev, m, ref = _run("scan_small", network=network, L=40, H=8, P=4, d_s=8, B_blk=16)
+    per_block = {"ks": 16 * 4 - 15, "sk": 8 * 4}[network]
+    assert ev.count["compose"] == closed_form_counts(sh, network)["compose"] == 12 * per_block
+    assert ev.c.lv["linj"] == ev.c.lv["lS"] - 1 and ev.c.lv["lout"] == ev.c.lv["linj"] - 3
+    assert np.abs(m - ref).max() < 2.0**-22
+    # deployed shape: depth log2 B instead of 2 log2 B - 1
+    assert levels(24, 8, 8, network) == dict(l0=24, l1=22, lS=14, linj=8, lout=5)
