@@ -662,10 +662,12 @@ def run_scan(args):
     x, a = chunk_cts(1), chunk_cts(2)
     Bc, Cc = cts(K_blk, 3), cts(K_blk, 4)
     masks = [S.hashed_residues(seed, 10 + i, q, N, device=dev).contiguous() for i in range(4)]
-    linj = l0 - 2 - 2 * 8 + 1
+    net = {"bk": fesc.NET_BRENT_KUNG, "ks": fesc.NET_KOGGE_STONE, "sk": fesc.NET_SKLANSKY}[args.network]
+    # injection level: 2 log2(B) - 1 network stages below the leaves (Brent-Kung), or log2(B) stages and the carries
+    linj = l0 - 2 - 2 * 8 + 1 if args.network == "bk" else l0 - 2 - 8 - max(K_blk - 2, 0)
     out = torch.empty((K_blk, max(mine, 1), 2, linj - 3, N), dtype=torch.int64, device=dev)
     adj = [(1 << 49) + 12345 * i for i in range((l0 + 1) ** 2)]
-    desc = fesc.ScanDesc(L, mine * hpc, P, d_s, B, 0, l0, base, int(args.hoist))
+    desc = fesc.ScanDesc(L, mine * hpc, P, d_s, B, 0, l0, base, int(args.hoist), net)
     torch.cuda.empty_cache()
 
     def step():
@@ -703,8 +705,9 @@ def run_scan(args):
                           "n_gpus": world, "steps": 1, "warmup": 1 if args.workload == "scan_slice" else 0,
                           "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "dtype": "u64",
                           "data": "synthetic",
-                          "config": {"workload": "%s: L=%d, H=%d, P=64, d_s=128, B_blk=256, K_s=%d, N=2^16, 24 limbs, %s"
+                          "config": {"workload": "%s: L=%d, H=%d, P=64, d_s=128, B_blk=256, K_s=%d, N=2^16, 24 limbs, %s network, %s"
                                                  % (args.workload, L, H, K_s,
+                                                    {"bk": "Brent-Kung", "ks": "Kogge-Stone", "sk": "Sklansky"}[args.network],
                                                     "radix-4 hoisted rotate-and-add chains" if args.hoist else "plain rotations"),
                                      "parallelism": "state chunks in pairs over %d rank(s): %s; one all-gather of the outputs"
                                                     % (world, [c for _, c in parts])},
@@ -843,6 +846,8 @@ def main():
                     help="1: one division by P per output for the whole giant-step sum")
     ap.add_argument("--hoist", type=int, default=1, choices=[0, 1],
                     help="1: baby rotations share one decomposition per input ciphertext (fesc_rotate_hoisted)")
+    ap.add_argument("--network", default="bk", choices=["bk", "ks", "sk"],
+                    help="scan workloads: prefix network (Brent-Kung, Kogge-Stone, Sklansky)")
     ap.add_argument("--workload", default="in_proj", choices=["in_proj", "out_proj", "rotations", "scan_slice", "scan_layer", "conv"],
                     help="in_proj (default, the benchmark metric), out_proj (1536 -> 768), a scan-contract run or the "
                          "depthwise convolution")

@@ -16,6 +16,7 @@ LIB_PATH = os.environ.get("FESC_LIB", os.path.join(_HERE, "libfesc_b200.so"))
 
 OK, EINVAL, ENOMEM, ECUDA, ELEVEL, ENOKEY, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 CONJ = -(1 << 31)
+NET_BRENT_KUNG, NET_KOGGE_STONE, NET_SKLANSKY = 0, 1, 2     # fesc_scan_desc.network
 RELIN_KEY_ID = 0
 
 _lib = None
@@ -39,7 +40,7 @@ class ConvDesc(ctypes.Structure):
 
 class ScanDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint32) for n in ("L", "H", "P", "d_s", "B_blk", "stride", "n_limbs", "key_base",
-                                                       "hoist")]
+                                                       "hoist", "network")]
 
 
 class ScanConsts(ctypes.Structure):

@@ -372,20 +372,37 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
                 }
                 X.top = m;
             };
+            const uint32_t network = X.desc->network;
             for (uint32_t s = 1; s <= g.logB; s++) {
                 std::vector<uint32_t> left, right;
-                for (uint32_t k = 1u << s; k <= B; k += 1u << s) {
-                    left.push_back(k - (1u << (s - 1)) - 1);
-                    right.push_back(k - 1);
+                const uint32_t half = 1u << (s - 1);
+                if (network == FESC_NET_KOGGE_STONE) {          // every k > 2^(s-1) with k - 2^(s-1) (1-based)
+                    for (uint32_t k = half + 1; k <= B; k++) {
+                        left.push_back(k - half - 1);
+                        right.push_back(k - 1);
+                    }
+                } else if (network == FESC_NET_SKLANSKY) {      // upper half of every block of 2^s with the lower half's last
+                    for (uint32_t b = 0; b < (B >> s); b++)
+                        for (uint32_t k = (b << s) + half; k < ((b + 1) << s); k++) {
+                            left.push_back((b << s) + half - 1);
+                            right.push_back(k);
+                        }
+                } else {
+                    for (uint32_t k = 1u << s; k <= B; k += 1u << s) {
+                        left.push_back(k - half - 1);
+                        right.push_back(k - 1);
+                    }
                 }
-                stage(left, right, l1 - (s - 1), true);
+                // the last stage of a one-pass network forms decay products only for an incoming state
+                stage(left, right, l1 - (s - 1), network == FESC_NET_BRENT_KUNG || s < g.logB || j > 0);
             }
-            // summary of the block = last position after the up-sweep; keep a copy for the carry
+            // summary of the block = last position after the up-sweep (after the last stage of a one-pass network);
+            // keep a copy for the carry (the first block's decay product is not used)
             Arr sumP = X.alloc(1, lS), sumS = X.alloc(1, lS);
-            X.copy(Arr{Ps.p + (size_t)(B - 1) * Ps.stride, 1, lS, X.ctw(lS)}, sumP);
+            if (network == FESC_NET_BRENT_KUNG || j > 0) X.copy(Arr{Ps.p + (size_t)(B - 1) * Ps.stride, 1, lS, X.ctw(lS)}, sumP);
             X.copy(Arr{Ss.p + (size_t)(B - 1) * Ss.stride, 1, lS, X.ctw(lS)}, sumS);
             uint32_t d = 0;
-            for (uint32_t s = g.logB - 1; s >= 1; s--) {
+            for (uint32_t s = g.logB - 1; s >= 1 && network == FESC_NET_BRENT_KUNG; s--) {
                 d++;
                 std::vector<uint32_t> left, right;
                 for (uint32_t k = 1u << s; k < B; k += 1u << s) {
@@ -514,10 +531,13 @@ extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint
     if ((uint64_t)g.B * g.d_s > g.n || (uint64_t)g.B * g.P > g.R)
         return fesc_fail(ctx, FESC_EINVAL, "scan_contract: block does not fit the compact packings");
     g.l0 = desc->n_limbs;
-    if (g.l0 > ctx->n_q || g.l0 < 2 * g.logB + 5) return fesc_fail(ctx, FESC_ELEVEL, "scan_contract: not enough levels");
+    if (desc->network > FESC_NET_SKLANSKY) return fesc_fail(ctx, FESC_EINVAL, "scan_contract: unknown prefix network");
+    const uint32_t below_summary =
+        desc->network == FESC_NET_BRENT_KUNG ? g.logB - 1 : (g.K_blk > 2 ? g.K_blk - 2 : 0);   // lS - linj
+    if (g.l0 > ctx->n_q || g.l0 < g.logB + below_summary + 6) return fesc_fail(ctx, FESC_ELEVEL, "scan_contract: not enough levels");
     g.l1 = g.l0 - 2;
     g.lS = g.l1 - g.logB;
-    g.linj = g.l1 - 2 * g.logB + 1;
+    g.linj = g.lS - below_summary;
     g.lout = g.linj - 3;
     if (g.K_blk > 1 && g.lS < g.linj + (g.K_blk - 2))
         return fesc_fail(ctx, FESC_ELEVEL, "scan_contract: carry chain runs below the injection level");

@@ -13,7 +13,7 @@ from tests.gpu_util import ctx_pair, to_dev, to_host
 pytestmark = pytest.mark.gpu
 
 
-def _run(name, hoist=0, **kw):
+def _run(name, hoist=0, network="bk", **kw):
     import torch
     import paper_2608_17442_b200 as fesc
 
@@ -21,7 +21,7 @@ def _run(name, hoist=0, **kw):
     sh = ScanShape(orc.n, **kw)
     l0 = p["n_q"]
     x, a, B, C = S.scan_inputs(p["seed"] + sh.L, sh.L, sh.H, sh.P, 1, sh.d_s)
-    c = ScanConsts(orc, sh, l0, p["log_scale"])
+    c = ScanConsts(orc, sh, l0, p["log_scale"], network)
     add_scan_keys(orc, sh, hoist=bool(hoist))
     for r in sh.rotation_amounts(bool(hoist)) + [CONJ]:
         ctx.add_galois_key(r, key_id_for(sh, r))
@@ -30,7 +30,8 @@ def _run(name, hoist=0, **kw):
     adj_s = [c.adj_s.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
     adj_p = [c.adj_p.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
     out = torch.empty((sh.K_blk, sh.K_s, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
-    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000, hoist)
+    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000, hoist,
+                         {"bk": fesc.NET_BRENT_KUNG, "ks": fesc.NET_KOGGE_STONE, "sk": fesc.NET_SKLANSKY}[network])
     ctx.scan_contract(to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
                       to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out)
     ctx.sync()
@@ -53,6 +54,26 @@ def test_scan_analogue_with_carries_and_partial_block(hoist):
 @pytest.mark.parametrize("hoist", [0, 1])
 def test_scan_two_digit_offsets_and_odd_chunk_count(hoist):
     assert _run("scan_small", hoist, L=64, H=3, P=4, d_s=4, B_blk=32) < 2.0**-22
+
+
+@pytest.mark.parametrize("network", ["ks", "sk"])
+def test_scan_other_prefix_networks(network):
+    """Kogge-Stone and Sklansky networks: bit-exact against the oracle's network of the same name (toy shape; carries
+    over three blocks with a partial last block, plain and hoisted rotations)."""
+    assert _run("scan_toy", 0, network, L=4, H=2, P=4, d_s=2, B_blk=4) < 2.0**-24
+    assert _run("scan_small", 0, network, L=40, H=8, P=4, d_s=8, B_blk=16) < 2.0**-22
+    assert _run("scan_small", 1, network, L=64, H=3, P=4, d_s=4, B_blk=32) < 2.0**-22
+
+
+def test_scan_unknown_network_is_refused():
+    import torch
+    import paper_2608_17442_b200 as fesc
+    ctx, orc, p = ctx_pair("scan_toy")
+    z = torch.zeros(8, dtype=torch.int64, device="cuda")
+    desc = fesc.ScanDesc(4, 2, 4, 2, 4, 0, p["n_q"], 100000, 0, 7)
+    with pytest.raises(fesc.FescError) as e:
+        ctx.scan_contract(z, z, z, z, desc, z, z, z, z, [0], [0], z)
+    assert e.value.code == fesc.EINVAL
 
 
 def test_scan_missing_key_is_reported():
