@@ -460,6 +460,36 @@ class Oracle:
             prev = cur if tb + 1 < tbs else None
         return out
 
+    def norm_square(self, y):
+        """u = y~ (.) y~ (Alg. "one Block", the squares that feed the NeRMS protocol): ciphertext product with
+        relinearisation, then rescale.  y [batch, 2, l, N] -> [batch, 2, l-1, N]."""
+        return np.stack([self.rescale(self.ct_ct_mul(c, c)) for c in y])
+
+    def norm_scale(self, y, s, gamma, T: int, key_base: int):
+        """y^ = gamma_RMS (.) (y~ (.) br(s_RMS)) (Alg. "one Block", the step before HEOutProj) on the projection
+        packing idx(token, channel) = channel*T + token.
+
+        y      [token_blocks, blocks, 2, l, N]   gated scan output of every (token block, channel block)
+        s      [token_blocks, 2, l, N]           slot k < T = the inverse RMS of token k, all other slots 0
+        gamma  [blocks, l-1, N]                  per-channel weights, slot c*T + k = gamma[channel c of the block]
+        returns [token_blocks, blocks, 2, l-2, N].
+        br(s): log2(n/T) rotate-right-and-add steps by T*2^b (the rotation by -(T << b) under key id key_base + b),
+        shared by the channel blocks of a token block; then a ciphertext product (relinearised, rescaled) and a
+        plaintext product (rescaled)."""
+        tbs, blocks, level = y.shape[0], y.shape[1], y.shape[3]
+        steps = (self.n // T).bit_length() - 1
+        assert (T << steps) == self.n and level >= 3
+        out = np.empty((tbs, blocks, 2, level - 2, self.N), dtype=np.uint64)
+        for tb in range(tbs):
+            f = _arr(s[tb])
+            for b in range(steps):
+                f = self.ct_add(f, self.rotate(f, key_base + b))
+            for blk in range(blocks):
+                prod = self.rescale(self.ct_ct_mul(y[tb, blk], f))
+                zero = np.zeros((2, level - 1, self.N), dtype=np.uint64)
+                out[tb, blk] = self.rescale(self.ct_pt_mac(prod, gamma[blk], zero))
+        return out
+
     # ---- harness: encode / decode / encrypt / decrypt ---------------------------------
     def _slot_index(self):
         idx = np.empty(self.n, dtype=np.int64)
