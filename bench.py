@@ -9,7 +9,7 @@ rescales.  Inputs are seeded synthetic residues (uniform below each prime) of ex
 shapes; arithmetic is data-independent, so timing equals that of real encodings.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-  python bench.py --workload out_proj | conv | scan_slice | scan_layer      (the other stages of a layer)
+  python bench.py --workload out_proj | conv | norm | scan_slice | scan_layer  (the other stages of a layer)
   python bench.py --workload rotations                                      (512 plain rotations, both digit layouts)
 
 Prints ONE JSON line (rank 0).  `value` = key switches per second over the whole step, summed
@@ -830,6 +830,66 @@ def run_conv(args):
           flush=True)
 
 
+def run_norm(args):
+    """Times the CKKS steps around the NeRMS protocol on synthetic residues of the Mamba-2-base shape: 1536 channels
+    (6 channel blocks of 256) x 2048 tokens (16 token blocks of 128), 24 limbs: fesc_norm_square on the 96
+    ciphertexts, then fesc_norm_scale (8 rotate-and-add steps per token block, 96 ciphertext products, 96 plaintext
+    products, two rescales)."""
+    import torch
+    import fesc_synth as S
+    import paper_2608_17442_b200 as fesc
+
+    torch.cuda.set_device(0)
+    p = S.params("full")
+    ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+    N = ctx.N
+    T, blocks, tbs, level, base = T_SEG, 6, 16, LEVEL, 3500
+    steps_fill = (N // 2 // T).bit_length() - 1
+    for b in range(steps_fill):
+        ctx.add_galois_key(-(T << b), base + b)
+    seed = S.config_seed(5)
+    q = p["primes"][:level]
+    r = S.hashed_residues(seed, 31, q, tbs * blocks * 2 * N, device="cuda")
+    y = r.view(level, tbs, blocks, 2, N).permute(1, 2, 3, 0, 4).contiguous()
+    r = S.hashed_residues(seed, 32, q, tbs * 2 * N, device="cuda")
+    sfac = r.view(level, tbs, 2, N).permute(1, 2, 0, 3).contiguous()
+    r = S.hashed_residues(seed, 33, q[:level - 1], blocks * N, device="cuda")
+    gamma = r.view(level - 1, blocks, N).permute(1, 0, 2).contiguous()
+    del r
+    u = torch.empty((tbs * blocks, 2, level - 1, N), dtype=torch.int64, device="cuda")
+    out = torch.empty((tbs, blocks, 2, level - 2, N), dtype=torch.int64, device="cuda")
+    desc = fesc.NormDesc(T, blocks, tbs, level, base)
+
+    def step():
+        ctx.norm_square(y, u, tbs * blocks, level)
+        ctx.norm_scale(y, sfac, gamma, desc, out)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    ctx.profile_enable(fesc.Context.PROFILE_FAMILIES, 60000)
+    step()
+    fam = ctx.profile_read()
+    ctx.profile_enable([])
+    c0 = ctx.counters()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    ctx.sync()
+    c1 = ctx.counters()
+    ms = e0.elapsed_time(e1) / args.steps
+    ks = (c1[1] - c0[1]) // args.steps
+    print(json.dumps({"metric": "NeRMS-side CKKS steps latency; key-switches/s", "value": ks / (ms * 1e-3),
+                      "unit": "key-switches/s", "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup),
+                      "ms_per_step": ms, "higher_is_better": True, "dtype": "u64", "data": "synthetic",
+                      "config": {"workload": "norm: squares and gamma (.) (y (.) br(s)) for 1536 channels x 2048 tokens, "
+                                             "T=128, 6 channel blocks x 16 token blocks, N=2^16, 24 limbs"},
+                      "key_switches_per_step": ks, "gpu_launches": (c1[4] - c0[4]) // args.steps,
+                      "kernel_breakdown": {k: {"ms": round(v[0], 2), "records": v[1]} for k, v in fam.items() if v[1]}}),
+          flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -848,9 +908,9 @@ def main():
                     help="1: baby rotations share one decomposition per input ciphertext (fesc_rotate_hoisted)")
     ap.add_argument("--network", default="bk", choices=["bk", "ks", "sk"],
                     help="scan workloads: prefix network (Brent-Kung, Kogge-Stone, Sklansky)")
-    ap.add_argument("--workload", default="in_proj", choices=["in_proj", "out_proj", "rotations", "scan_slice", "scan_layer", "conv"],
-                    help="in_proj (default, the benchmark metric), out_proj (1536 -> 768), a scan-contract run or the "
-                         "depthwise convolution")
+    ap.add_argument("--workload", default="in_proj", choices=["in_proj", "out_proj", "rotations", "scan_slice", "scan_layer", "conv", "norm"],
+                    help="in_proj (default, the benchmark metric), out_proj (1536 -> 768), a scan-contract run, the "
+                         "depthwise convolution or the CKKS steps around the normalisation")
     args = ap.parse_args()
     if args.workload == "out_proj":
         global D_IN, D_OUT, PROJ, METRIC, N1, N2
@@ -860,6 +920,8 @@ def main():
         args.workload = "in_proj"
     if args.workload == "conv":
         return run_conv(args)
+    if args.workload == "norm":
+        return run_norm(args)
     if args.workload == "rotations":
         return run_rotations(args)
     if args.workload != "in_proj":

@@ -38,6 +38,10 @@ class ConvDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint32) for n in ("d_conv", "T", "blocks", "token_blocks", "n_limbs", "key_base")]
 
 
+class NormDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint32) for n in ("T", "blocks", "token_blocks", "n_limbs", "key_base")]
+
+
 class ScanDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint32) for n in ("L", "H", "P", "d_s", "B_blk", "stride", "n_limbs", "key_base",
                                                        "hoist", "network")]
@@ -76,6 +80,8 @@ def lib():
             "fesc_rotate_hoisted": [vp, vp, vp, u32, u32, c.POINTER(u32), u32, vp],
             "fesc_rotate_sum_hoisted": [vp, vp, vp, u32, u32, c.POINTER(u32), u32, vp],
             "fesc_conv": [vp, vp, vp, vp, c.POINTER(ConvDesc), vp, vp],
+            "fesc_norm_square": [vp, vp, vp, c.c_uint32, c.c_uint32, vp],
+            "fesc_norm_scale": [vp, vp, vp, vp, c.POINTER(NormDesc), vp, vp],
             "fesc_split_complex": [vp, vp, vp, vp, u32, u32, u32, vp],
             "fesc_rescale": [vp, vp, vp, u32, u32, vp],
             "fesc_rescale_static": [vp, vp, vp, u32, u32, vp],
@@ -204,6 +210,12 @@ class Context:
     def split_complex(self, ct_in, re2, im2, batch: int, n_limbs: int, conj_key_id: int):
         self._chk(lib().fesc_split_complex(self.h, _ptr(ct_in), _ptr(re2), _ptr(im2) if im2 is not None else None, batch,
                                            n_limbs, conj_key_id, _stream()))
+
+    def norm_square(self, y, out, batch, n_limbs):
+        self._chk(lib().fesc_norm_square(self.h, _ptr(y), _ptr(out), batch, n_limbs, _stream()))
+
+    def norm_scale(self, y, s, gamma, desc: "NormDesc", out):
+        self._chk(lib().fesc_norm_scale(self.h, _ptr(y), _ptr(s), _ptr(gamma), ctypes.byref(desc), _ptr(out), _stream()))
 
     def conv(self, ct_in, masks, bias, desc: "ConvDesc", ct_out):
         self._chk(lib().fesc_conv(self.h, _ptr(ct_in), _ptr(masks), _ptr(bias), ctypes.byref(desc), _ptr(ct_out), _stream()))

@@ -12,14 +12,14 @@ def _ctx(log_n, n_q=4):
     return Oracle(log_n, data + special, n_q, 1, n_q, 5151)
 
 
-def run_norm(o, y, s, gamma, T, C, level, scale=2.0**40, key_base=700, nonce=300):
+def run_norm(o, y, s, gamma, T, C, level, scale=2.0**40, key_base=700, nonce=300, add_key=None):
     """y [tokens, channels], s [tokens], gamma [channels] -> (cts, s_cts, gamma_pts, out, Y^ [tokens, channels])."""
     tokens, channels = y.shape
     n = o.n
     blocks, tbs = -(-channels // C), -(-tokens // T)
     steps = (n // T).bit_length() - 1
     for b in range(steps):
-        o.add_galois_key(-(T << b), key_base + b)
+        (add_key or o.add_galois_key)(-(T << b), key_base + b)
     cts = np.empty((tbs, blocks, 2, level, o.N), dtype=np.uint64)
     s_cts = np.empty((tbs, 2, level, o.N), dtype=np.uint64)
     for tb in range(tbs):
