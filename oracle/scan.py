@@ -36,6 +36,14 @@ up-sweep stage s -> l1-s;  summaries at lS = l1-logB;  down-sweep stage number d
 lS-(d-1) -> lS-d;  carries g_j (j >= 1) at lS-(j-1);  injection at linj = l1-2logB+1 -> states at linj-1;
 contraction -> linj-2;  reduction, conjugation, unpacking there;  output mask -> l_out = linj-3.
 
+Grouped leaf build (`group` = G > 0, a separately defined mode: other residues, same values).  Building br(x_t) and
+br(a_t) token by token costs log2(d_s) and log2(R/P) rotate-and-add steps per token at the top levels.  With groups of
+G consecutive tokens the group is extracted, masked (slots [0,G) of every stride for x, [0,GP) of every head region for
+a) and filled ONCE for its G tokens (log2(d_s/G), log2(R/(GP)) steps: the pattern of G tokens repeats), a second mask
+keeps the copies of one token (slot class g modulo G, block class g modulo GP) one level lower, and log2 G signed steps
+(towards lower slots for the bits set in g, higher slots for the others) fill the classes in between.  The second mask
+costs one level: br(B_t) is brought to l0-2 before its fill and the leaves sit at l1 = l0-3.
+
 Other prefix networks (App. "Prefix-Network Selection"; `network` = "ks" Kogge-Stone, "sk" Sklansky; "bk" above is the
 default): stage s = 1..logB combines operands at l1-(s-1) into results at l1-s, every prefix is complete at lS and there
 is no down-sweep, so linj = lS - max(K_blk-2, 0) (the carry before the last block still sits at or above linj).
@@ -88,8 +96,15 @@ class ScanShape:
         return [(-1, lg(self.P)), (-1, lg(self.d_s)), (-self.P, lg(self.R // self.P)),
                 (-self.stride, lg(self.c_state)), (1, lg(self.d_s))]
 
-    def rotation_amounts(self, hoist: bool = False):
-        """hoist=True adds the amounts 3 * unit * 2^b of the radix-4 chains (b even, b + 1 < steps)."""
+    @staticmethod
+    def class_deltas(g: int, G: int, unit: int):
+        """Signed slot shifts (LEFT positive) of the steps that copy class g of a period of G blocks of `unit` slots to
+        every class: bit b of g set -> the copies move to lower slots (+unit 2^b), else to higher slots (-unit 2^b)."""
+        return [unit * (1 << b) if (g >> b) & 1 else -unit * (1 << b) for b in range(int(math.log2(G)))]
+
+    def rotation_amounts(self, hoist: bool = False, group: int = 0):
+        """hoist=True adds the amounts 3 * unit * 2^b of the radix-4 chains (b even, b + 1 < steps); group=G adds the
+        group extraction amounts and the signed class steps (in hoisted mode also the sums of their pairs)."""
         n, dg, B = self.n, self.dg, self.B
         lo = range(1, dg)
         hi = range(1, B // dg)
@@ -104,6 +119,18 @@ class ScanShape:
         if hoist:
             for unit, steps in self.chains():
                 am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
+        if group:
+            G = group
+            cnt = B // G
+            dgg = min(16, cnt)
+            for unit in (G, G * self.P):                                                   # extraction of the groups
+                am |= {unit * t % n for t in range(1, dgg)} | {unit * dgg * t % n for t in range(1, cnt // dgg)}
+            for unit in (1, self.P):
+                for g in range(G):
+                    d = self.class_deltas(g, G, unit)
+                    am |= {v % n for v in d}
+                    if hoist:
+                        am |= {(d[b] + d[b + 1]) % n for b in range(0, len(d) - 1, 2)}
         am.discard(0)
         return sorted(am)
 
@@ -111,9 +138,9 @@ class ScanShape:
 NETWORKS = ("bk", "ks", "sk")
 
 
-def levels(l0: int, logB: int, K_blk: int, network: str = "bk"):
+def levels(l0: int, logB: int, K_blk: int, network: str = "bk", group: int = 0):
     assert network in NETWORKS
-    l1 = l0 - 2
+    l1 = l0 - 3 if group else l0 - 2
     lS = l1 - logB
     linj = l1 - 2 * logB + 1 if network == "bk" else lS - max(K_blk - 2, 0)
     lout = linj - 3
@@ -125,10 +152,10 @@ def levels(l0: int, logB: int, K_blk: int, network: str = "bk"):
 class ScanConsts:
     """Harness-side constants: canonical scales, level-adjust integers, mask plaintexts."""
 
-    def __init__(self, orc: Oracle, shape: ScanShape, l0: int, log_scale: int, network: str = "bk"):
+    def __init__(self, orc: Oracle, shape: ScanShape, l0: int, log_scale: int, network: str = "bk", group: int = 0):
         q = orc.q
-        self.network = network
-        self.lv = levels(l0, shape.logB, shape.K_blk, network)
+        self.network, self.group = network, group
+        self.lv = levels(l0, shape.logB, shape.K_blk, network, group)
         self.S_s = {l0: float(2**log_scale)}
         self.S_p = {l0: float(q[l0 - 1])}
         for l in range(l0, 1, -1):
@@ -150,6 +177,17 @@ class ScanConsts:
         self.mask_x = orc.encode(mx, self.S_p[l0], l0)
         self.mask_b = orc.encode(mb, self.S_p[l0], l0)
         self.mask_a = orc.encode(ma, self.S_p[l0], l0)
+        if group:
+            G, P, R, d_s = group, shape.P, shape.R, shape.d_s
+            assert G >= 2 and G & (G - 1) == 0 and G <= min(shape.B, d_s) and G * P <= R
+            slot = np.arange(n)
+            in_stride, in_region = slot % st, slot % R
+            self.mask_xg = orc.encode((in_stride < G).astype(float), self.S_p[l0], l0)
+            self.mask_ag = orc.encode((in_region < G * P).astype(float), self.S_p[l0], l0)
+            self.mask_x2 = np.stack([orc.encode(((in_stride < d_s) & (in_stride % G == g)).astype(float),
+                                                self.S_p[l0 - 1], l0 - 1) for g in range(G)])
+            self.mask_a2 = np.stack([orc.encode(((in_region // P) % G == g).astype(float), self.S_p[l0 - 1], l0 - 1)
+                                     for g in range(G)])
         lred, lout = self.lv["linj"] - 2, self.lv["lout"]
         # the unpacked reduction carries a factor 2 (Re*2, Im*2); the output mask removes it and lands on S_s[lout]
         self.out_mask_scale = self.S_s[lout] * q[lout] / (2.0 * self.S_s[lred])
@@ -161,8 +199,8 @@ def key_id_for(shape: ScanShape, amount: int, base: int = 100000) -> int:
     return base + shape.n if amount == CONJ else base + amount % shape.n
 
 
-def add_scan_keys(orc: Oracle, shape: ScanShape, base: int = 100000, hoist: bool = False):
-    for r in shape.rotation_amounts(hoist):
+def add_scan_keys(orc: Oracle, shape: ScanShape, base: int = 100000, hoist: bool = False, group: int = 0):
+    for r in shape.rotation_amounts(hoist, group):
         if key_id_for(shape, r, base) not in orc.keys:
             orc.add_galois_key(r, key_id_for(shape, r, base))
     if key_id_for(shape, CONJ, base) not in orc.keys:
@@ -226,6 +264,7 @@ class ScanEvaluator:
         (`rotate_sum_hoisted`), and the low digit of the two-digit token offsets uses `rotate_hoisted`."""
         self.o, self.sh, self.c, self.kb, self.hoist = orc, shape, consts, key_base, hoist
         self.network = consts.network       # the level schedule in `consts` belongs to one network
+        self.group = consts.group           # ... and to one leaf build
         self.count = dict(rot=0, conj=0, ctmul=0, adjust=0, ptmul=0, compose=0)
 
     # -- primitives ---------------------------------------------------------------------------
@@ -280,26 +319,44 @@ class ScanEvaluator:
                 b += 1
         return ct
 
+    def signed_chain(self, ct, deltas):
+        """ct += rot(ct, delta) for every delta in turn (LEFT shifts, signed).  Hoisted mode: two steps together as
+        ct + rot(ct, d1) + rot(ct, d2) + rot(ct, d1 + d2), one decomposition and one division by P."""
+        b = 0
+        while b < len(deltas):
+            if self.hoist and b + 1 < len(deltas):
+                d1, d2 = deltas[b], deltas[b + 1]
+                self.count["rot"] += 3
+                ct = self.o.rotate_sum_hoisted(ct, [key_id_for(self.sh, d, self.kb) for d in (d1, d2, d1 + d2)])
+                b += 2
+            else:
+                ct = self.add(ct, self.rot(ct, deltas[b]))
+                b += 1
+        return ct
+
     def fill_right(self, ct, unit, steps):
         """ct += rot(ct, -unit*2^b) for b = 0..steps-1 (copies a block to 2^steps consecutive blocks)."""
         return self.chain(ct, -unit, steps)
 
-    def extract_all(self, ct, unit):
-        """[rot(ct, unit*t) for t < B] with t = t_lo + dg*t_hi: rot(ct, unit*dg*t_hi) first, then the low digit
-        (in hoisted mode the dg-1 low-digit rotations of one ciphertext share its decomposition)."""
+    def extract_all(self, ct, unit, count=None):
+        """[rot(ct, unit*t) for t < count (default B)] with t = t_lo + dg*t_hi, dg = min(16, count):
+        rot(ct, unit*dg*t_hi) first, then the low digit (in hoisted mode the dg-1 low-digit rotations of one
+        ciphertext share its decomposition)."""
         sh = self.sh
-        out = [None] * sh.B
-        for th in range(sh.B // sh.dg):
-            g = ct if th == 0 else self.rot(ct, unit * sh.dg * th)
-            out[th * sh.dg] = g
-            if self.hoist and sh.dg > 1:
-                self.count["rot"] += sh.dg - 1
-                lows = self.o.rotate_hoisted(g, [key_id_for(sh, unit * tl, self.kb) for tl in range(1, sh.dg)])
-                for tl in range(1, sh.dg):
-                    out[th * sh.dg + tl] = lows[tl - 1]
+        count = sh.B if count is None else count
+        dg = min(16, count)
+        out = [None] * count
+        for th in range(count // dg):
+            g = ct if th == 0 else self.rot(ct, unit * dg * th)
+            out[th * dg] = g
+            if self.hoist and dg > 1:
+                self.count["rot"] += dg - 1
+                lows = self.o.rotate_hoisted(g, [key_id_for(sh, unit * tl, self.kb) for tl in range(1, dg)])
+                for tl in range(1, dg):
+                    out[th * dg + tl] = lows[tl - 1]
             else:
-                for tl in range(1, sh.dg):
-                    out[th * sh.dg + tl] = self.rot(g, unit * tl)
+                for tl in range(1, dg):
+                    out[th * dg + tl] = self.rot(g, unit * tl)
         return out
 
     def compose(self, left, right, lvl, need_p=True):
@@ -340,6 +397,24 @@ class ScanEvaluator:
             ar = self.fill_right(ar, sh.P, int(math.log2(sh.R // sh.P)))
             s = self.mul_rescale(xr, brB[t])
             T.append((ar, s))
+        return T
+
+    def leaves_grouped(self, ctX, ctA, brB):
+        """Leaves (br a_t, br x_t (.) br B_t) at l1 = l0-3 with the grouped build (module header): groups of G tokens
+        are extracted, masked and filled once; a second mask and log2 G signed steps separate the tokens."""
+        sh, c, G = self.sh, self.c, self.group
+        l1, lg = c.lv["l1"], lambda v: int(math.log2(v))
+        apre = self.fill_right(ctA, 1, lg(sh.P))
+        gx, ga = self.extract_all(ctX, G, sh.B // G), self.extract_all(apre, G * sh.P, sh.B // G)
+        T = []
+        for u in range(sh.B // G):
+            xg = self.fill_right(self.ptmul_rescale(gx[u], c.mask_xg), G, lg(sh.d_s // G))
+            ag = self.fill_right(self.ptmul_rescale(ga[u], c.mask_ag), G * sh.P, lg(sh.R // (G * sh.P)))
+            for g in range(G):
+                xr = self.signed_chain(self.ptmul_rescale(xg, c.mask_x2[g]), sh.class_deltas(g, G, 1))
+                ar = self.adjust(self.ptmul_rescale(ag, c.mask_a2[g]), l1, "p")
+                ar = self.signed_chain(ar, sh.class_deltas(g, G, sh.P))
+                T.append((ar, self.mul_rescale(xr, brB[u * G + g])))
         return T
 
     def brent_kung(self, T, need_p_down):
@@ -399,11 +474,11 @@ class ScanEvaluator:
         out = np.zeros((sh.K_blk, sh.K_s, 2, lout, o.N), dtype=np.uint64)
         carry = [None] * sh.K_s                       # g_j per chunk: the state before block j
         for j in range(sh.K_blk):
-            brB = self.broadcast_bc(ctB[j])
+            brB = self.broadcast_bc(ctB[j], lv["l0"] - 2 if self.group else None)
             brC = self.broadcast_bc(ctC[j], linj - 1)
             v = [[None] * sh.K_s for _ in range(sh.B)]
             for kap in range(sh.K_s):
-                T = self.leaves(ctX[j, kap], ctA[j, kap], brB)
+                T = (self.leaves_grouped if self.group else self.leaves)(ctX[j, kap], ctA[j, kap], brB)
                 summary = self.prefix_network(T, j > 0)
                 g = carry[kap]
                 for t in range(sh.B):

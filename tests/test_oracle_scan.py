@@ -113,13 +113,13 @@ def test_paper_ledger_values():
     assert 2 * 768 // 768 and 2 * 24 * 64 + 2 * 128 + 24 == 3352              # d_out of in_proj
 
 
-def _run(name, hoist=False, network="bk", **shape_kw):
+def _run(name, hoist=False, network="bk", group=0, **shape_kw):
     p = S.params(name)
     orc = Oracle(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
     sh = ScanShape(orc.n, **shape_kw)
     x, a, B, C = S.scan_inputs(p["seed"], sh.L, sh.H, sh.P, 1, sh.d_s)
-    c = ScanConsts(orc, sh, p["n_q"], p["log_scale"], network)
-    add_scan_keys(orc, sh, hoist=hoist)
+    c = ScanConsts(orc, sh, p["n_q"], p["log_scale"], network, group)
+    add_scan_keys(orc, sh, hoist=hoist, group=group)
     ev = ScanEvaluator(orc, sh, c, hoist=hoist)
     out = ev.run(*encrypt_inputs(orc, sh, c, x, a, B, C))
     return sh, ev, unpack_output(orc, sh, c, out), float_recurrence(x, a, B, C)
@@ -176,3 +176,43 @@ def test_other_prefix_networks(network):
     assert np.abs(m - ref).max() < 2.0**-22
     # deployed shape: depth log2 B instead of 2 log2 B - 1
     assert levels(24, 8, 8, network) == dict(l0=24, l1=22, lS=14, linj=8, lout=5)
+
+
+def test_grouped_leaf_build():
+    """Leaves built for groups of G tokens (one extraction, mask and fill per group, then a class mask and log2 G
+    signed steps per token): same contract output, same compositions, one level more, and exactly the rotations the
+    closed form predicts fewer."""
+    kw = dict(L=40, H=8, P=4, d_s=8, B_blk=16)
+    sh, ev0, m0, ref = _run("scan_small", **kw)
+    _, ev, m, _ = _run("scan_small", group=4, **kw)
+    assert np.abs(m - ref).max() < 2.0**-22 and np.abs(m - m0).max() < 2.0**-22
+    assert ev.c.lv == dict(l0=16, l1=13, lS=9, linj=6, lout=3) and ev0.c.lv["l1"] == 14
+    assert ev.count["compose"] == ev0.count["compose"] and ev.count["ctmul"] == ev0.count["ctmul"]
+    lg = lambda v: int(math.log2(v))
+    B, G, P, R, d_s = sh.B, 4, sh.P, sh.R, sh.d_s
+    plain = 2 * (B - 1) + B * (lg(d_s) + lg(R // P))
+    grouped = 2 * (B // G - 1) + (B // G) * (lg(d_s // G) + lg(R // (G * P))) + 2 * B * lg(G)
+    assert ev0.count["rot"] - ev.count["rot"] == sh.K_blk * sh.K_s * (plain - grouped) == 720
+    assert ev.count["ptmul"] - ev0.count["ptmul"] == sh.K_blk * sh.K_s * 2 * (B // G)
+    # the signed steps of class g reach every class exactly once
+    for G in (2, 4, 8):
+        for g in range(G):
+            reach = {0}
+            for d in sh.class_deltas(g, G, 1):
+                reach |= {r - d for r in reach}          # a LEFT shift by d moves a copy d slots down
+            assert sorted(g + r for r in reach) == list(range(G))
+    # deployed shape: 1 854 instead of 4 350 extraction and fill rotations per (block, chunk)
+    big = ScanShape(32768, L=2048, H=24, P=64, d_s=128, B_blk=256)
+    B, G, P, R, d_s = 256, 4, 64, big.R, 128
+    assert 2 * (B - 1) + B * (lg(d_s) + lg(R // P)) == 4350
+    assert 2 * (B // G - 1) + (B // G) * (lg(d_s // G) + lg(R // (G * P))) + 2 * B * lg(G) == 1854
+    assert levels(24, 8, 8, "bk", 4) == dict(l0=24, l1=21, lS=13, linj=6, lout=3)
+
+
+def test_grouped_leaf_build_other_shapes_and_hoisted_rotations():
+    sh, ev, m, ref = _run("scan_toy", group=2, L=4, H=2, P=4, d_s=2, B_blk=4)
+    assert np.abs(m - ref).max() < 2.0**-24
+    sh, ev, m, ref = _run("scan_small", hoist=True, group=4, L=64, H=3, P=4, d_s=4, B_blk=32)
+    assert (sh.K_s, sh.K_blk) == (3, 2) and np.abs(m - ref).max() < 2.0**-22
+    sh, ev, m, ref = _run("scan_small", network="sk", group=2, L=40, H=8, P=4, d_s=8, B_blk=16)
+    assert np.abs(m - ref).max() < 2.0**-22
