@@ -563,7 +563,7 @@ def run_ours(args):
 # ---------------------------------------------------------------------------------------------
 # optional second workload: the scan-contract of one Mamba-2-base layer (or a slice of it)
 # ---------------------------------------------------------------------------------------------
-def scan_rotation_amounts(n, P, d_s, B, stride, hoist=False):
+def scan_rotation_amounts(n, P, d_s, B, stride, hoist=False, group=0):
     """Slot rotations the scan-contract uses (see include/fesc.h), as left shifts modulo n."""
     import math
 
@@ -582,6 +582,20 @@ def scan_rotation_amounts(n, P, d_s, B, stride, hoist=False):
         lg = lambda v: int(math.log2(v))
         for unit, steps in ((-1, lg(P)), (-1, lg(d_s)), (-P, lg(R // P)), (-stride, lg(c_state)), (1, lg(d_s))):
             am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
+    if group:    # grouped leaf build: group offsets (two digits) and the signed class steps (and their pair sums)
+        cnt = B // group
+        dgg = min(16, cnt)
+        for unit in (group, group * P):
+            am |= {unit * t % n for t in range(1, dgg)} | {unit * dgg * t % n for t in range(1, cnt // dgg)}
+        if hoist:
+            for unit, steps in ((-group, int(math.log2(d_s // group))), (-group * P, int(math.log2(R // (group * P))))):
+                am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
+        for unit in (1, P):
+            for c in range(group):
+                d = [unit * (1 << b) if (c >> b) & 1 else -unit * (1 << b) for b in range(int(math.log2(group)))]
+                am |= {v % n for v in d}
+                if hoist:
+                    am |= {(d[b] + d[b + 1]) % n for b in range(0, len(d) - 1, 2)}
     am.discard(0)
     return sorted(am)
 
@@ -645,7 +659,8 @@ def run_scan(args):
     parts = scan_partition(K_s, world)
     first, mine = parts[rank]
     base = 100000
-    for r in scan_rotation_amounts(n, P, d_s, B, stride, bool(args.hoist)):
+    G = int(args.group)
+    for r in scan_rotation_amounts(n, P, d_s, B, stride, bool(args.hoist), G):
         ctx.add_galois_key(r, base + r)
     ctx.add_galois_key(fesc.CONJ, base + n)
     seed = S.config_seed(5)
@@ -664,15 +679,22 @@ def run_scan(args):
     masks = [S.hashed_residues(seed, 10 + i, q, N, device=dev).contiguous() for i in range(4)]
     net = {"bk": fesc.NET_BRENT_KUNG, "ks": fesc.NET_KOGGE_STONE, "sk": fesc.NET_SKLANSKY}[args.network]
     # injection level: 2 log2(B) - 1 network stages below the leaves (Brent-Kung), or log2(B) stages and the carries
-    linj = l0 - 2 - 2 * 8 + 1 if args.network == "bk" else l0 - 2 - 8 - max(K_blk - 2, 0)
+    l1 = l0 - 3 if G else l0 - 2                               # the grouped leaf build spends one more level
+    linj = l1 - 2 * 8 + 1 if args.network == "bk" else l1 - 8 - max(K_blk - 2, 0)
+    gm = None
+    if G:
+        gm = [S.hashed_residues(seed, 20, q, N, device=dev).contiguous(),
+              S.hashed_residues(seed, 21, q, N, device=dev).contiguous(),
+              S.hashed_residues(seed, 22, q[:l0 - 1], G * N, device=dev).view(l0 - 1, G, N).permute(1, 0, 2).contiguous(),
+              S.hashed_residues(seed, 23, q[:l0 - 1], G * N, device=dev).view(l0 - 1, G, N).permute(1, 0, 2).contiguous()]
     out = torch.empty((K_blk, max(mine, 1), 2, linj - 3, N), dtype=torch.int64, device=dev)
     adj = [(1 << 49) + 12345 * i for i in range((l0 + 1) ** 2)]
-    desc = fesc.ScanDesc(L, mine * hpc, P, d_s, B, 0, l0, base, int(args.hoist), net)
+    desc = fesc.ScanDesc(L, mine * hpc, P, d_s, B, 0, l0, base, int(args.hoist), net, G)
     torch.cuda.empty_cache()
 
     def step():
         if mine:
-            ctx.scan_contract(x, a, Bc, Cc, desc, masks[0], masks[1], masks[2], masks[3][:linj - 2], adj, adj, out)
+            ctx.scan_contract(x, a, Bc, Cc, desc, masks[0], masks[1], masks[2], masks[3][:linj - 2], adj, adj, out, gm)
         return gather_chunk_outputs(out[:, :mine], parts, rank, world, K_blk, K_s) if world > 1 else out
 
     breakdown = None
@@ -708,7 +730,8 @@ def run_scan(args):
                           "config": {"workload": "%s: L=%d, H=%d, P=64, d_s=128, B_blk=256, K_s=%d, N=2^16, 24 limbs, %s network, %s"
                                                  % (args.workload, L, H, K_s,
                                                     {"bk": "Brent-Kung", "ks": "Kogge-Stone", "sk": "Sklansky"}[args.network],
-                                                    "radix-4 hoisted rotate-and-add chains" if args.hoist else "plain rotations"),
+                                                    ("radix-4 hoisted rotate-and-add chains" if args.hoist else "plain rotations")
+                                                    + (", leaves built in groups of %d tokens" % G if G else "")),
                                      "parallelism": "state chunks in pairs over %d rank(s): %s; one all-gather of the outputs"
                                                     % (world, [c for _, c in parts])},
                           "key_switches": ks, "limb_transforms": c1[0] - c0[0], "gpu_launches": c1[4] - c0[4],
@@ -906,6 +929,8 @@ def main():
                     help="1: one division by P per output for the whole giant-step sum")
     ap.add_argument("--hoist", type=int, default=1, choices=[0, 1],
                     help="1: baby rotations share one decomposition per input ciphertext (fesc_rotate_hoisted)")
+    ap.add_argument("--group", type=int, default=4, choices=[0, 2, 4, 8, 16],
+                    help="scan workloads: tokens per group of the grouped leaf build (0: token by token)")
     ap.add_argument("--network", default="bk", choices=["bk", "ks", "sk"],
                     help="scan workloads: prefix network (Brent-Kung, Kogge-Stone, Sklansky)")
     ap.add_argument("--workload", default="in_proj", choices=["in_proj", "out_proj", "rotations", "scan_slice", "scan_layer", "conv", "norm"],

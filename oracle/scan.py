@@ -125,6 +125,9 @@ class ScanShape:
             dgg = min(16, cnt)
             for unit in (G, G * self.P):                                                   # extraction of the groups
                 am |= {unit * t % n for t in range(1, dgg)} | {unit * dgg * t % n for t in range(1, cnt // dgg)}
+            if hoist:                                                                      # radix-4 group fills
+                for unit, steps in ((-G, int(math.log2(self.d_s // G))), (-G * self.P, int(math.log2(self.R // (G * self.P))))):
+                    am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
             for unit in (1, self.P):
                 for g in range(G):
                     d = self.class_deltas(g, G, unit)

@@ -262,26 +262,59 @@ struct Exec {
         top = mark;
     }
     void fill_right(const Arr& a, uint32_t unit, uint32_t steps) { chain(a, -(int64_t)unit, steps); }
-    // out[t] = rot(src, unit * t) for t = 0..B-1, via t = t_lo + dg * t_hi (hoisted mode: the dg-1 low-digit
-    // rotations of one ciphertext share its decomposition)
-    void extract_all(const Arr& src, int64_t unit, const Arr& out) {
+    // a += rot(a, delta) for every delta in turn (signed LEFT shifts).  Hoisted mode takes two steps together:
+    // a + rot(a, d1) + rot(a, d2) + rot(a, d1 + d2).
+    void signed_chain(const Arr& a, const std::vector<int64_t>& deltas) {
         size_t mark = top;
-        const uint32_t nh = g.B / g.dg;
-        Arr gi = alloc(nh, src.level);
-        for (uint32_t th = 0; th < nh; th++) rot(src, unit * (int64_t)(g.dg * th), at(gi, th));
-        if (desc->hoist && g.dg > 1) {
-            copy(gi, strided(out, 0, g.dg, nh));
-            std::vector<uint32_t> ids;
-            for (uint32_t tl = 1; tl < g.dg && ok(); tl++)
-                if (key_ok(unit * (int64_t)tl)) ids.push_back(key_for(unit * (int64_t)tl));
-            if (ok() && !dry)
-                rc = rotate_hoisted_internal(ctx, gi.p, gi.stride, out.p + out.stride, out.stride * g.dg, out.stride, nh,
-                                             src.level, ids.data(), (uint32_t)ids.size(), ks, st);
-        } else {
-            for (uint32_t tl = 0; tl < g.dg; tl++) rot(gi, unit * (int64_t)tl, strided(out, tl, g.dg, nh));
+        Arr t = alloc(a.count, a.level);
+        size_t b = 0;
+        while (b < deltas.size() && ok()) {
+            if (desc->hoist && b + 1 < deltas.size()) {
+                const int64_t d1 = deltas[b], d2 = deltas[b + 1];
+                if (!key_ok(d1) || !key_ok(d2) || !key_ok(d1 + d2)) break;
+                if (!dry) {
+                    const uint32_t ids[3] = {key_for(d1), key_for(d2), key_for(d1 + d2)};
+                    rc = rotate_sum_hoisted_internal(ctx, a.p, a.stride, t.p, t.stride, a.count, a.level, ids, 3, ks, st);
+                    copy(t, a);
+                }
+                b += 2;
+            } else {
+                rot(a, deltas[b], t);
+                add(a, t, a);
+                b += 1;
+            }
         }
         top = mark;
     }
+    // steps that copy class cls of a period of G blocks of `unit` slots to every class: bit b of cls set -> the
+    // copies move to lower slots (+unit 2^b), else to higher slots (-unit 2^b)
+    static std::vector<int64_t> class_deltas(uint32_t cls, uint32_t G, uint32_t unit) {
+        std::vector<int64_t> d;
+        for (uint32_t b = 0; (1u << b) < G; b++)
+            d.push_back(((cls >> b) & 1) ? (int64_t)unit * (1 << b) : -(int64_t)unit * (1 << b));
+        return d;
+    }
+    // out[t] = rot(src, unit * t) for t = 0..count-1, via t = t_lo + dg * t_hi, dg = min(16, count) (hoisted mode:
+    // the dg-1 low-digit rotations of one ciphertext share its decomposition)
+    void extract_n(const Arr& src, int64_t unit, uint32_t count, const Arr& out) {
+        size_t mark = top;
+        const uint32_t dg = count < 16 ? count : 16, nh = count / dg;
+        Arr gi = alloc(nh, src.level);
+        for (uint32_t th = 0; th < nh; th++) rot(src, unit * (int64_t)(dg * th), at(gi, th));
+        if (desc->hoist && dg > 1) {
+            copy(gi, strided(out, 0, dg, nh));
+            std::vector<uint32_t> ids;
+            for (uint32_t tl = 1; tl < dg && ok(); tl++)
+                if (key_ok(unit * (int64_t)tl)) ids.push_back(key_for(unit * (int64_t)tl));
+            if (ok() && !dry)
+                rc = rotate_hoisted_internal(ctx, gi.p, gi.stride, out.p + out.stride, out.stride * dg, out.stride, nh,
+                                             src.level, ids.data(), (uint32_t)ids.size(), ks, st);
+        } else {
+            for (uint32_t tl = 0; tl < dg; tl++) rot(gi, unit * (int64_t)tl, strided(out, tl, dg, nh));
+        }
+        top = mark;
+    }
+    void extract_all(const Arr& src, int64_t unit, const Arr& out) { extract_n(src, unit, g.B, out); }
 };
 
 }  // namespace
@@ -300,15 +333,21 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
     std::vector<uint32_t> carry_level(g.K_s, 0);
     for (uint32_t j = 0; j < g.K_blk && X.ok(); j++) {
         const size_t block_mark = X.top;
-        // ---- br(B_t) at l0-1 and br(C_t) at linj-1, shared by every chunk ----
-        Arr brB = X.alloc(B, l0 - 1), brC = X.alloc(B, linj - 1);
+        // ---- br(B_t) at l0-1 (l0-2 with the grouped leaf build) and br(C_t) at linj-1, shared by every chunk ----
+        const uint32_t G = X.desc->group, lB = G ? l0 - 2 : l0 - 1;
+        Arr brB = X.alloc(B, lB), brC = X.alloc(B, linj - 1);
         for (int which = 0; which < 2; which++) {
             size_t m = X.top;
             Arr src{const_cast<u64*>((which ? d_C : d_B) + (size_t)j * in_ctw), 1, l0, in_ctw};
             Arr ex = X.alloc(B, l0);
             X.extract_all(src, g.d_s, ex);
-            if (which == 0) {
+            if (which == 0 && !G) {
                 X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_b, brB);
+                X.fill_right(brB, g.stride, ilog2(g.c_state));
+            } else if (which == 0) {
+                Arr full = X.alloc(B, l0 - 1);
+                X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_b, full);
+                X.adjust(full, lB, 1, brB);
                 X.fill_right(brB, g.stride, ilog2(g.c_state));
             } else {
                 // br(C) is only needed at the injection level: bring it down first, fill there (cheap rotations)
@@ -326,7 +365,34 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
             // position slots of the prefix network: capacity l1, current level tracked on the host
             Arr Ps = X.alloc(B, l1), Ss = X.alloc(B, l1);
             std::vector<uint32_t> lp(B, l1), ls(B, l1);
-            {   // ---- leaves ----
+            if (G) {   // ---- leaves, grouped build: groups of G tokens share extraction, mask and fill ----
+                size_t m = X.top;
+                const uint32_t ng = B / G;
+                const size_t mask_words = (size_t)(l0 - 1) * N;
+                Arr srcx{const_cast<u64*>(d_x + ((size_t)j * g.K_s + kap) * in_ctw), 1, l0, in_ctw};
+                Arr apre = X.alloc(1, l0);
+                X.copy(Arr{const_cast<u64*>(d_a + ((size_t)j * g.K_s + kap) * in_ctw), 1, l0, in_ctw}, apre);
+                X.fill_right(apre, 1, ilog2(g.P));
+                Arr ex = X.alloc(ng, l0), xg = X.alloc(ng, l0 - 1), ag = X.alloc(ng, l0 - 1);
+                X.extract_n(srcx, G, ng, ex);
+                X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_xg, xg);
+                X.fill_right(xg, G, ilog2(g.d_s / G));
+                X.extract_n(apre, (int64_t)G * g.P, ng, ex);
+                X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_ag, ag);
+                X.fill_right(ag, G * g.P, ilog2(g.R / (G * g.P)));
+                Arr xr = X.alloc(B, l0 - 2), cls2 = X.alloc(ng, l0 - 2), cls1 = X.alloc(ng, l1);
+                for (uint32_t c = 0; c < G && X.ok(); c++) {      // the tokens u*G + c of every group u
+                    X.ptmul_rescale(xg, (const u64*)X.cs->d_mask_x2 + c * mask_words, cls2);
+                    X.signed_chain(cls2, Exec::class_deltas(c, G, 1));
+                    X.copy(cls2, X.strided(xr, c, G, ng));
+                    X.ptmul_rescale(ag, (const u64*)X.cs->d_mask_a2 + c * mask_words, cls2);
+                    X.adjust(cls2, l1, 1, cls1);
+                    X.signed_chain(cls1, Exec::class_deltas(c, G, g.P));
+                    X.copy(cls1, X.strided(Ps, c, G, ng));
+                }
+                X.mul_rescale(xr, brB, Ss);      // s_t = br(x_t) (.) br(B_t), level l1 = l0-3
+                X.top = m;
+            } else {   // ---- leaves ----
                 size_t m = X.top;
                 Arr srcx{const_cast<u64*>(d_x + ((size_t)j * g.K_s + kap) * in_ctw), 1, l0, in_ctw};
                 Arr apre = X.alloc(1, l0);
@@ -534,8 +600,16 @@ extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint
     if (desc->network > FESC_NET_SKLANSKY) return fesc_fail(ctx, FESC_EINVAL, "scan_contract: unknown prefix network");
     const uint32_t below_summary =
         desc->network == FESC_NET_BRENT_KUNG ? g.logB - 1 : (g.K_blk > 2 ? g.K_blk - 2 : 0);   // lS - linj
-    if (g.l0 > ctx->n_q || g.l0 < g.logB + below_summary + 6) return fesc_fail(ctx, FESC_ELEVEL, "scan_contract: not enough levels");
-    g.l1 = g.l0 - 2;
+    const uint32_t G = desc->group;
+    if (G) {
+        if (G < 2 || (G & (G - 1)) || G > g.B || G > g.d_s)
+            return fesc_fail(ctx, FESC_EINVAL, "scan_contract: group must be a power of two, at most B_blk and d_s");
+        if (!consts->d_mask_xg || !consts->d_mask_ag || !consts->d_mask_x2 || !consts->d_mask_a2)
+            return fesc_fail(ctx, FESC_EINVAL, "scan_contract: the grouped leaf build needs its four mask arrays");
+    }
+    if (g.l0 > ctx->n_q || g.l0 < g.logB + below_summary + 6 + (G ? 1 : 0))
+        return fesc_fail(ctx, FESC_ELEVEL, "scan_contract: not enough levels");
+    g.l1 = g.l0 - (G ? 3 : 2);
     g.lS = g.l1 - g.logB;
     g.linj = g.lS - below_summary;
     g.lout = g.linj - 3;

@@ -114,3 +114,17 @@ def test_two_gloo_ranks_gather_their_chunk_outputs_once():
         assert p.returncode == 0, e
         res = json.loads(o.strip().splitlines()[-1])
         assert res["ok"] and res["parts"] == [[0, 2], [2, 3]]      # 5 chunks: pair (0,1) | pair (2,3) and the odd chunk 4
+
+
+def test_bench_scan_rotation_amounts_match_the_dataflow():
+    """bench.py registers Galois keys from its own list of rotation amounts (the product path does not import the
+    oracle); the list equals the one the scan dataflow uses, in every mode."""
+    import bench
+    from oracle.scan import ScanShape
+
+    for n, kw in ((128, dict(L=40, H=8, P=4, d_s=8, B_blk=16)), (32768, dict(L=2048, H=24, P=64, d_s=128, B_blk=256))):
+        sh = ScanShape(n, **kw)
+        for hoist in (False, True):
+            for group in (0, 2, 4, 8):
+                want = sh.rotation_amounts(hoist, group)
+                assert bench.scan_rotation_amounts(n, sh.P, sh.d_s, sh.B, sh.stride, hoist, group) == want

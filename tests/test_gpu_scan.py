@@ -13,7 +13,7 @@ from tests.gpu_util import ctx_pair, to_dev, to_host
 pytestmark = pytest.mark.gpu
 
 
-def _run(name, hoist=0, network="bk", **kw):
+def _run(name, hoist=0, network="bk", group=0, **kw):
     import torch
     import paper_2608_17442_b200 as fesc
 
@@ -21,9 +21,9 @@ def _run(name, hoist=0, network="bk", **kw):
     sh = ScanShape(orc.n, **kw)
     l0 = p["n_q"]
     x, a, B, C = S.scan_inputs(p["seed"] + sh.L, sh.L, sh.H, sh.P, 1, sh.d_s)
-    c = ScanConsts(orc, sh, l0, p["log_scale"], network)
-    add_scan_keys(orc, sh, hoist=bool(hoist))
-    for r in sh.rotation_amounts(bool(hoist)) + [CONJ]:
+    c = ScanConsts(orc, sh, l0, p["log_scale"], network, group)
+    add_scan_keys(orc, sh, hoist=bool(hoist), group=group)
+    for r in sh.rotation_amounts(bool(hoist), group) + [CONJ]:
         ctx.add_galois_key(r, key_id_for(sh, r))
     ctX, ctA, ctB, ctC = encrypt_inputs(orc, sh, c, x, a, B, C)
     want = ScanEvaluator(orc, sh, c, hoist=bool(hoist)).run(ctX, ctA, ctB, ctC)
@@ -31,9 +31,10 @@ def _run(name, hoist=0, network="bk", **kw):
     adj_p = [c.adj_p.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
     out = torch.empty((sh.K_blk, sh.K_s, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
     desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000, hoist,
-                         {"bk": fesc.NET_BRENT_KUNG, "ks": fesc.NET_KOGGE_STONE, "sk": fesc.NET_SKLANSKY}[network])
+                         {"bk": fesc.NET_BRENT_KUNG, "ks": fesc.NET_KOGGE_STONE, "sk": fesc.NET_SKLANSKY}[network], group)
+    gm = [to_dev(m) for m in (c.mask_xg, c.mask_ag, c.mask_x2, c.mask_a2)] if group else None
     ctx.scan_contract(to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
-                      to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out)
+                      to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out, gm)
     ctx.sync()
     got = to_host(out)
     assert np.array_equal(got, want)
@@ -65,6 +66,17 @@ def test_scan_other_prefix_networks(network):
     assert _run("scan_small", 1, network, L=64, H=3, P=4, d_s=4, B_blk=32) < 2.0**-22
 
 
+@pytest.mark.parametrize("hoist", [0, 1])
+def test_scan_grouped_leaf_build(hoist):
+    """Leaves built for groups of G tokens: bit-exact against the oracle's grouped mode (G = 2 on the toy shape, G = 4
+    with carries over three blocks and a partial last block, G = 4 with two-digit group offsets, G = 2 under Sklansky)."""
+    assert _run("scan_toy", hoist, group=2, L=4, H=2, P=4, d_s=2, B_blk=4) < 2.0**-24
+    assert _run("scan_small", hoist, group=4, L=40, H=8, P=4, d_s=8, B_blk=16) < 2.0**-22
+    assert _run("scan_small", hoist, group=4, L=64, H=3, P=4, d_s=4, B_blk=32) < 2.0**-22
+    if hoist:
+        assert _run("scan_small", hoist, "sk", 2, L=40, H=8, P=4, d_s=8, B_blk=16) < 2.0**-22
+
+
 def test_scan_unknown_network_is_refused():
     import torch
     import paper_2608_17442_b200 as fesc
@@ -74,6 +86,11 @@ def test_scan_unknown_network_is_refused():
     with pytest.raises(fesc.FescError) as e:
         ctx.scan_contract(z, z, z, z, desc, z, z, z, z, [0], [0], z)
     assert e.value.code == fesc.EINVAL
+    for group, masks in ((3, (z, z, z, z)), (8, (z, z, z, z)), (2, None)):      # not a power of two; above d_s; no masks
+        desc = fesc.ScanDesc(4, 2, 4, 2, 4, 0, p["n_q"], 100000, 0, 0, group)
+        with pytest.raises(fesc.FescError) as e:
+            ctx.scan_contract(z, z, z, z, desc, z, z, z, z, [0], [0], z, masks)
+        assert e.value.code == fesc.EINVAL
 
 
 def test_scan_missing_key_is_reported():
@@ -88,8 +105,8 @@ def test_scan_missing_key_is_reported():
     assert e.value.code == fesc.ENOKEY
 
 
-@pytest.mark.parametrize("hoist", [1])
-def test_scan_deployed_geometry_decrypts_to_recurrence(hoist):
+@pytest.mark.parametrize("hoist,group", [(1, 0), (1, 4)])
+def test_scan_deployed_geometry_decrypts_to_recurrence(hoist, group):
     """N = 2^16, 24 limbs, stride 256, B_blk = 256, d_s = 128, P = 64 (the Mamba-2-base geometry) on a slice of
     the model: 4 heads (one chunk pair) and 512 tokens (two blocks, so the carry and its injection run).
     The oracle cannot follow ~36 000 key switches at this ring size, so the check here is the property that
@@ -103,17 +120,18 @@ def test_scan_deployed_geometry_decrypts_to_recurrence(hoist):
     assert (sh.stride, sh.c_state, sh.hpc, sh.K_s, sh.K_blk) == (256, 128, 2, 2, 2)
     l0 = 24
     x, a, B, C = S.scan_inputs(S.config_seed(5), sh.L, sh.H, sh.P, 1, sh.d_s)
-    c = ScanConsts(orc, sh, l0, 40)
-    assert c.lv == dict(l0=24, l1=22, lS=14, linj=7, lout=4)
-    for r in sh.rotation_amounts(bool(hoist)) + [CONJ]:
+    c = ScanConsts(orc, sh, l0, 40, "bk", group)
+    assert c.lv == (dict(l0=24, l1=21, lS=13, linj=6, lout=3) if group else dict(l0=24, l1=22, lS=14, linj=7, lout=4))
+    for r in sh.rotation_amounts(bool(hoist), group) + [CONJ]:
         ctx.add_galois_key(r, key_id_for(sh, r))
     ctX, ctA, ctB, ctC = encrypt_inputs(orc, sh, c, x, a, B, C)
     adj_s = [c.adj_s.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
     adj_p = [c.adj_p.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
     out = torch.empty((sh.K_blk, sh.K_s, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
-    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000, hoist)
+    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000, hoist, 0, group)
+    gm = [to_dev(m) for m in (c.mask_xg, c.mask_ag, c.mask_x2, c.mask_a2)] if group else None
     args = (to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
-            to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out)
+            to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out, gm)
     ks0 = ctx.counters()[1]
     torch.cuda.synchronize()
     t0 = time.perf_counter()
