@@ -18,7 +18,11 @@ implements the same graph independently and must reproduce every residue.
 Geometry (all powers of two).  n slots = c_state * stride, stride >= max(d_s, B_blk); one state ciphertext of
 chunk kappa holds coordinate (e = kappa*c_state + e', i) at slot e'*stride + i (i < d_s; the rest idle).
 hpc = c_state / P heads per chunk, each owning a slot region of R = n / hpc = P*stride slots.
-Inputs per token block j (B = B_blk tokens, t = token within the block):
+A block of B tokens is cut into segs = max(1, B/stride) segments of Bt = B/segs tokens; x, a and the output have one
+ciphertext per segment (stride >= B, one segment, is the paper's deployed shape with half of the state slots idle;
+stride = d_s < B uses every slot: s_state = n, half as many chunks).
+Inputs per token block j (B = B_blk tokens, t = token within the block; for X, A and the output t is the offset inside
+the segment and the arrays carry a segment axis after the chunk axis):
     X[j][kappa]: slot e'*stride + t      = x_{jB+t}[kappa*c_state + e']          scale S_s[l0]
     A[j][kappa]: slot hh*R + t*P          = a_{jB+t}[kappa*hpc + hh], else 0       scale S_p[l0]
     Bc[j], Cc[j]: slot t*d_s + i          = B_{jB+t}[i], C_{jB+t}[i]               scale S_p[l0]
@@ -78,7 +82,10 @@ class ScanShape:
         self.stride = stride or max(d_s, B_blk)
         self.c_state = n // self.stride
         self.E = H * P
-        assert self.c_state * self.stride == n and self.stride >= max(d_s, B_blk)
+        assert self.c_state * self.stride == n and self.stride >= d_s
+        assert self.stride >= B_blk or B_blk % self.stride == 0
+        self.segs = max(1, B_blk // self.stride)      # token segments of a block: one x / a / output ciphertext each
+        self.Bt = B_blk // self.segs                   # tokens per segment
         assert self.c_state % P == 0 and self.E % self.c_state == 0
         self.hpc = self.c_state // P
         self.R = n // self.hpc
@@ -86,8 +93,9 @@ class ScanShape:
         self.K_blk = -(-L // B_blk)
         self.logB = int(math.log2(B_blk))
         assert 1 << self.logB == B_blk and B_blk >= 2
-        assert B_blk * d_s <= n and B_blk * P <= self.R
-        self.dg = min(16, B_blk)                      # base of the two-digit token offset t = t_lo + dg*t_hi
+        assert B_blk * d_s <= n and self.Bt * P <= self.R
+        self.dg = min(16, B_blk)                      # base of the two-digit token offset t = t_lo + dg*t_hi (B, C)
+        self.dgt = min(16, self.Bt)                   # ... of the offset inside a segment (x, a, output)
 
     # rotation amounts (slot LEFT shifts, modulo n) the dataflow uses
     def chains(self):
@@ -105,13 +113,12 @@ class ScanShape:
     def rotation_amounts(self, hoist: bool = False, group: int = 0):
         """hoist=True adds the amounts 3 * unit * 2^b of the radix-4 chains (b even, b + 1 < steps); group=G adds the
         group extraction amounts and the signed class steps (in hoisted mode also the sums of their pairs)."""
-        n, dg, B = self.n, self.dg, self.B
-        lo = range(1, dg)
-        hi = range(1, B // dg)
+        n, dg, B, dgt, Bt = self.n, self.dg, self.B, self.dgt, self.Bt
         am = set()
-        for unit in (1, self.P, self.d_s):            # extraction of x, a, (B and C)
-            am |= {unit * t % n for t in lo} | {unit * dg * t % n for t in hi}
-        am |= {(-t) % n for t in lo} | {(-dg * t) % n for t in hi}                       # output placement
+        for unit in (1, self.P):                      # extraction of x, a (offsets inside a segment)
+            am |= {unit * t % n for t in range(1, dgt)} | {unit * dgt * t % n for t in range(1, Bt // dgt)}
+        am |= {self.d_s * t % n for t in range(1, dg)} | {self.d_s * dg * t % n for t in range(1, B // dg)}   # B, C
+        am |= {(-t) % n for t in range(1, dgt)} | {(-dgt * t) % n for t in range(1, Bt // dgt)}   # output placement
         am |= {(-(1 << b)) % n for b in range(int(math.log2(max(self.d_s, self.P))))}    # x fill, a pre-fill
         am |= {(-self.P * (1 << b)) % n for b in range(int(math.log2(self.R // self.P)))}        # a fill
         am |= {(-self.stride * (1 << b)) % n for b in range(int(math.log2(self.c_state)))}       # B, C fill
@@ -121,7 +128,7 @@ class ScanShape:
                 am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
         if group:
             G = group
-            cnt = B // G
+            cnt = Bt // G
             dgg = min(16, cnt)
             for unit in (G, G * self.P):                                                   # extraction of the groups
                 am |= {unit * t % n for t in range(1, dgg)} | {unit * dgg * t % n for t in range(1, cnt // dgg)}
@@ -182,7 +189,7 @@ class ScanConsts:
         self.mask_a = orc.encode(ma, self.S_p[l0], l0)
         if group:
             G, P, R, d_s = group, shape.P, shape.R, shape.d_s
-            assert G >= 2 and G & (G - 1) == 0 and G <= min(shape.B, d_s) and G * P <= R
+            assert G >= 2 and G & (G - 1) == 0 and G <= min(shape.Bt, d_s) and G * P <= R
             slot = np.arange(n)
             in_stride, in_region = slot % st, slot % R
             self.mask_xg = orc.encode((in_stride < G).astype(float), self.S_p[l0], l0)
@@ -213,8 +220,8 @@ def add_scan_keys(orc: Oracle, shape: ScanShape, base: int = 100000, hoist: bool
 def pack_inputs(shape: ScanShape, x, a, B, C):
     """Slot vectors of the compact factors: dict name -> array [K_blk, (K_s,) n]."""
     sh = shape
-    X = np.zeros((sh.K_blk, sh.K_s, sh.n))
-    A = np.zeros((sh.K_blk, sh.K_s, sh.n))
+    X = np.zeros((sh.K_blk, sh.K_s, sh.segs, sh.n))
+    A = np.zeros((sh.K_blk, sh.K_s, sh.segs, sh.n))
     Bc = np.zeros((sh.K_blk, sh.n))
     Cc = np.zeros((sh.K_blk, sh.n))
     xf = x.reshape(sh.L, sh.E)
@@ -222,10 +229,11 @@ def pack_inputs(shape: ScanShape, x, a, B, C):
         j, t = divmod(k, sh.B)
         Bc[j, t * sh.d_s:(t + 1) * sh.d_s] = B[k, 0]
         Cc[j, t * sh.d_s:(t + 1) * sh.d_s] = C[k, 0]
+        seg, tt = divmod(t, sh.Bt)
         for kap in range(sh.K_s):
-            X[j, kap, np.arange(sh.c_state) * sh.stride + t] = xf[k, kap * sh.c_state:(kap + 1) * sh.c_state]
+            X[j, kap, seg, np.arange(sh.c_state) * sh.stride + tt] = xf[k, kap * sh.c_state:(kap + 1) * sh.c_state]
             for hh in range(sh.hpc):
-                A[j, kap, hh * sh.R + t * sh.P] = a[k, kap * sh.hpc + hh]
+                A[j, kap, seg, hh * sh.R + tt * sh.P] = a[k, kap * sh.hpc + hh]
     return X, A, Bc, Cc
 
 
@@ -238,22 +246,27 @@ def encrypt_inputs(orc: Oracle, shape: ScanShape, consts: ScanConsts, x, a, B, C
         nonce[0] += 1
         return orc.encrypt(orc.encode(v, scale, l0), nonce[0])
 
-    ctX = np.stack([np.stack([enc(X[j, k], consts.S_s[l0]) for k in range(shape.K_s)]) for j in range(shape.K_blk)])
-    ctA = np.stack([np.stack([enc(A[j, k], consts.S_p[l0]) for k in range(shape.K_s)]) for j in range(shape.K_blk)])
+    segs = range(shape.segs)
+    ctX = np.stack([np.stack([np.stack([enc(X[j, k, g], consts.S_s[l0]) for g in segs]) for k in range(shape.K_s)])
+                    for j in range(shape.K_blk)])
+    ctA = np.stack([np.stack([np.stack([enc(A[j, k, g], consts.S_p[l0]) for g in segs]) for k in range(shape.K_s)])
+                    for j in range(shape.K_blk)])
     ctB = np.stack([enc(Bc[j], consts.S_p[l0]) for j in range(shape.K_blk)])
     ctC = np.stack([enc(Cc[j], consts.S_p[l0]) for j in range(shape.K_blk)])
     return ctX, ctA, ctB, ctC
 
 
 def unpack_output(orc: Oracle, shape: ScanShape, consts: ScanConsts, out):
-    """out [K_blk, K_s, 2, l_out, N] -> m [L, H, P] (float64, decrypted)."""
+    """out [K_blk, K_s, segs, 2, l_out, N] -> m [L, H, P] (float64, decrypted)."""
     sh = shape
     m = np.zeros((sh.K_blk * sh.B, sh.E))
     for j in range(sh.K_blk):
         for kap in range(sh.K_s):
-            slots = orc.decrypt(out[j, kap], consts.out_scale, 2).real
-            for t in range(sh.B):
-                m[j * sh.B + t, kap * sh.c_state:(kap + 1) * sh.c_state] = slots[np.arange(sh.c_state) * sh.stride + t]
+            for seg in range(sh.segs):
+                slots = orc.decrypt(out[j, kap, seg], consts.out_scale, 2).real
+                for tt in range(sh.Bt):
+                    m[j * sh.B + seg * sh.Bt + tt, kap * sh.c_state:(kap + 1) * sh.c_state] = \
+                        slots[np.arange(sh.c_state) * sh.stride + tt]
     return m[:sh.L].reshape(sh.L, sh.H, sh.P)
 
 
@@ -388,18 +401,20 @@ class ScanEvaluator:
         return out
 
     def leaves(self, ctX, ctA, brB):
+        """ctX, ctA: the `segs` ciphertexts of one (block, chunk), segment g holding the tokens g*Bt .. (g+1)*Bt-1."""
         sh, c = self.sh, self.c
         l1 = c.lv["l1"]
-        apre = self.fill_right(ctA, 1, int(math.log2(sh.P)))
-        ex, ea = self.extract_all(ctX, 1), self.extract_all(apre, sh.P)
         T = []
-        for t in range(sh.B):
-            xr = self.ptmul_rescale(ex[t], c.mask_x)
-            xr = self.fill_right(xr, 1, int(math.log2(sh.d_s)))
-            ar = self.adjust(self.ptmul_rescale(ea[t], c.mask_a), l1, "p")        # to the leaf level, then fill
-            ar = self.fill_right(ar, sh.P, int(math.log2(sh.R // sh.P)))
-            s = self.mul_rescale(xr, brB[t])
-            T.append((ar, s))
+        for seg in range(sh.segs):
+            apre = self.fill_right(ctA[seg], 1, int(math.log2(sh.P)))
+            ex, ea = self.extract_all(ctX[seg], 1, sh.Bt), self.extract_all(apre, sh.P, sh.Bt)
+            for tt in range(sh.Bt):
+                xr = self.ptmul_rescale(ex[tt], c.mask_x)
+                xr = self.fill_right(xr, 1, int(math.log2(sh.d_s)))
+                ar = self.adjust(self.ptmul_rescale(ea[tt], c.mask_a), l1, "p")        # to the leaf level, then fill
+                ar = self.fill_right(ar, sh.P, int(math.log2(sh.R // sh.P)))
+                s = self.mul_rescale(xr, brB[seg * sh.Bt + tt])
+                T.append((ar, s))
         return T
 
     def leaves_grouped(self, ctX, ctA, brB):
@@ -407,17 +422,19 @@ class ScanEvaluator:
         are extracted, masked and filled once; a second mask and log2 G signed steps separate the tokens."""
         sh, c, G = self.sh, self.c, self.group
         l1, lg = c.lv["l1"], lambda v: int(math.log2(v))
-        apre = self.fill_right(ctA, 1, lg(sh.P))
-        gx, ga = self.extract_all(ctX, G, sh.B // G), self.extract_all(apre, G * sh.P, sh.B // G)
         T = []
-        for u in range(sh.B // G):
-            xg = self.fill_right(self.ptmul_rescale(gx[u], c.mask_xg), G, lg(sh.d_s // G))
-            ag = self.fill_right(self.ptmul_rescale(ga[u], c.mask_ag), G * sh.P, lg(sh.R // (G * sh.P)))
-            for g in range(G):
-                xr = self.signed_chain(self.ptmul_rescale(xg, c.mask_x2[g]), sh.class_deltas(g, G, 1))
-                ar = self.adjust(self.ptmul_rescale(ag, c.mask_a2[g]), l1, "p")
-                ar = self.signed_chain(ar, sh.class_deltas(g, G, sh.P))
-                T.append((ar, self.mul_rescale(xr, brB[u * G + g])))
+        for seg in range(sh.segs):
+            apre = self.fill_right(ctA[seg], 1, lg(sh.P))
+            gx = self.extract_all(ctX[seg], G, sh.Bt // G)
+            ga = self.extract_all(apre, G * sh.P, sh.Bt // G)
+            for u in range(sh.Bt // G):
+                xg = self.fill_right(self.ptmul_rescale(gx[u], c.mask_xg), G, lg(sh.d_s // G))
+                ag = self.fill_right(self.ptmul_rescale(ga[u], c.mask_ag), G * sh.P, lg(sh.R // (G * sh.P)))
+                for g in range(G):
+                    xr = self.signed_chain(self.ptmul_rescale(xg, c.mask_x2[g]), sh.class_deltas(g, G, 1))
+                    ar = self.adjust(self.ptmul_rescale(ag, c.mask_a2[g]), l1, "p")
+                    ar = self.signed_chain(ar, sh.class_deltas(g, G, sh.P))
+                    T.append((ar, self.mul_rescale(xr, brB[seg * sh.Bt + u * G + g])))
         return T
 
     def brent_kung(self, T, need_p_down):
@@ -470,11 +487,11 @@ class ScanEvaluator:
         return (self.kogge_stone if self.network == "ks" else self.sklansky)(T, later_block)
 
     def run(self, ctX, ctA, ctB, ctC):
-        """ctX, ctA [K_blk, K_s, 2, l0, N]; ctB, ctC [K_blk, 2, l0, N] -> out [K_blk, K_s, 2, l_out, N]."""
+        """ctX, ctA [K_blk, K_s, segs, 2, l0, N]; ctB, ctC [K_blk, 2, l0, N] -> out [K_blk, K_s, segs, 2, l_out, N]."""
         sh, c, o = self.sh, self.c, self.o
         lv = c.lv
         linj, lout = lv["linj"], lv["lout"]
-        out = np.zeros((sh.K_blk, sh.K_s, 2, lout, o.N), dtype=np.uint64)
+        out = np.zeros((sh.K_blk, sh.K_s, sh.segs, 2, lout, o.N), dtype=np.uint64)
         carry = [None] * sh.K_s                       # g_j per chunk: the state before block j
         for j in range(sh.K_blk):
             brB = self.broadcast_bc(ctB[j], lv["l0"] - 2 if self.group else None)
@@ -517,8 +534,9 @@ class ScanEvaluator:
                     parts = [self.add(chi, chi)]                                           # same factor 2
                 for off, part in enumerate(parts):
                     y = self.ptmul_rescale(part, c.mask_out)
-                    y = self.rot(self.rot(y, -(t % sh.dg)), -sh.dg * (t // sh.dg))
-                    out[j, kap + off] = self.add(out[j, kap + off], y)
+                    seg, tt = divmod(t, sh.Bt)                      # placement inside the token's segment
+                    y = self.rot(self.rot(y, -(tt % sh.dgt)), -sh.dgt * (tt // sh.dgt))
+                    out[j, kap + off, seg] = self.add(out[j, kap + off, seg], y)
 
     def neg_times_i(self, ct):
         """-i * ct  =  X^(N/2) applied three times (exact monomial products)."""

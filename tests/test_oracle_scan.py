@@ -216,3 +216,21 @@ def test_grouped_leaf_build_other_shapes_and_hoisted_rotations():
     assert (sh.K_s, sh.K_blk) == (3, 2) and np.abs(m - ref).max() < 2.0**-22
     sh, ev, m, ref = _run("scan_small", network="sk", group=2, L=40, H=8, P=4, d_s=8, B_blk=16)
     assert np.abs(m - ref).max() < 2.0**-22
+
+
+def test_full_slot_variant_with_token_segments():
+    """stride = d_s < B_blk: every slot of a state ciphertext carries a state coordinate (s_state = n), a block's tokens
+    come in B_blk/stride segments with one x / a / output ciphertext each, and half as many chunks do the same work."""
+    kw = dict(L=40, H=8, P=4, d_s=8, B_blk=16)
+    sh0, ev0, m0, ref = _run("scan_small", **kw)
+    sh, ev, m, _ = _run("scan_small", stride=8, **kw)
+    assert (sh0.K_s, sh0.segs, sh0.hpc) == (4, 1, 2) and (sh.K_s, sh.segs, sh.Bt, sh.hpc, sh.R) == (2, 2, 8, 4, 32)
+    assert np.abs(m - ref).max() < 2.0**-22 and np.abs(m - m0).max() < 2.0**-22
+    assert ev.count["compose"] == closed_form_counts(sh)["compose"] == ev0.count["compose"] // 2
+    assert ev.count["ctmul"] == ev0.count["ctmul"] // 2 and ev.count["conj"] == ev0.count["conj"] // 2
+    # with the grouped leaf build and hoisted rotations on top
+    _, _, m, _ = _run("scan_small", hoist=True, group=4, stride=8, **kw)
+    assert np.abs(m - ref).max() < 2.0**-22
+    # deployed ring: K_s = 6 chunks of 4 heads, two segments of 128 tokens
+    big = ScanShape(32768, L=2048, H=24, P=64, d_s=128, B_blk=256, stride=128)
+    assert (big.K_s, big.segs, big.Bt, big.c_state, big.hpc, big.R) == (6, 2, 128, 256, 4, 8192)
