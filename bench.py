@@ -568,12 +568,15 @@ def scan_rotation_amounts(n, P, d_s, B, stride, hoist=False, group=0):
     import math
 
     dg = min(16, B)
+    Bt = B // max(1, B // stride)                 # tokens per segment
+    dgt = min(16, Bt)
     c_state = n // stride
     R = P * stride
     am = set()
-    for unit in (1, P, d_s):
-        am |= {unit * t % n for t in range(1, dg)} | {unit * dg * t % n for t in range(1, B // dg)}
-    am |= {(-t) % n for t in range(1, dg)} | {(-dg * t) % n for t in range(1, B // dg)}
+    for unit in (1, P):                           # x, a: offsets inside a segment
+        am |= {unit * t % n for t in range(1, dgt)} | {unit * dgt * t % n for t in range(1, Bt // dgt)}
+    am |= {d_s * t % n for t in range(1, dg)} | {d_s * dg * t % n for t in range(1, B // dg)}      # B, C
+    am |= {(-t) % n for t in range(1, dgt)} | {(-dgt * t) % n for t in range(1, Bt // dgt)}        # output placement
     am |= {(-(1 << b)) % n for b in range(int(math.log2(max(d_s, P))))}
     am |= {(-P * (1 << b)) % n for b in range(int(math.log2(R // P)))}
     am |= {(-stride * (1 << b)) % n for b in range(int(math.log2(c_state)))}
@@ -583,7 +586,7 @@ def scan_rotation_amounts(n, P, d_s, B, stride, hoist=False, group=0):
         for unit, steps in ((-1, lg(P)), (-1, lg(d_s)), (-P, lg(R // P)), (-stride, lg(c_state)), (1, lg(d_s))):
             am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
     if group:    # grouped leaf build: group offsets (two digits) and the signed class steps (and their pair sums)
-        cnt = B // group
+        cnt = Bt // group
         dgg = min(16, cnt)
         for unit in (group, group * P):
             am |= {unit * t % n for t in range(1, dgg)} | {unit * dgg * t % n for t in range(1, cnt // dgg)}
@@ -653,8 +656,11 @@ def run_scan(args):
     ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
     n, N = ctx.N // 2, ctx.N
     H, L = (4, 512) if args.workload == "scan_slice" else (24, 2048)
-    P, d_s, B, stride, l0 = 64, 128, 256, 256, 24
+    P, d_s, B, stride, l0 = 64, 128, 256, int(args.stride), 24
+    if stride == 128 and args.workload == "scan_slice":
+        H = 8                                                  # one chunk pair of 4 heads per chunk
     K_s, K_blk = H * P // (n // stride), L // B
+    segs = max(1, B // stride)
     hpc = (n // stride) // P                                   # heads per chunk
     parts = scan_partition(K_s, world)
     first, mine = parts[rank]
@@ -670,8 +676,8 @@ def run_scan(args):
         r = S.hashed_residues(seed, stream, q, count * 2 * N, device=dev)
         return r.view(l0, count, 2, N).permute(1, 2, 0, 3).contiguous()
 
-    def chunk_cts(stream):                                     # [K_blk][mine] ciphertexts of this rank's chunks
-        full = cts(K_blk * K_s, stream).view(K_blk, K_s, 2, l0, N)
+    def chunk_cts(stream):                                     # [K_blk][mine][segs] ciphertexts of this rank's chunks
+        full = cts(K_blk * K_s * segs, stream).view(K_blk, K_s, segs, 2, l0, N)
         return full[:, first:first + mine].contiguous()
 
     x, a = chunk_cts(1), chunk_cts(2)
@@ -687,9 +693,9 @@ def run_scan(args):
               S.hashed_residues(seed, 21, q, N, device=dev).contiguous(),
               S.hashed_residues(seed, 22, q[:l0 - 1], G * N, device=dev).view(l0 - 1, G, N).permute(1, 0, 2).contiguous(),
               S.hashed_residues(seed, 23, q[:l0 - 1], G * N, device=dev).view(l0 - 1, G, N).permute(1, 0, 2).contiguous()]
-    out = torch.empty((K_blk, max(mine, 1), 2, linj - 3, N), dtype=torch.int64, device=dev)
+    out = torch.empty((K_blk, max(mine, 1), segs, 2, linj - 3, N), dtype=torch.int64, device=dev)
     adj = [(1 << 49) + 12345 * i for i in range((l0 + 1) ** 2)]
-    desc = fesc.ScanDesc(L, mine * hpc, P, d_s, B, 0, l0, base, int(args.hoist), net, G)
+    desc = fesc.ScanDesc(L, mine * hpc, P, d_s, B, stride, l0, base, int(args.hoist), net, G)
     torch.cuda.empty_cache()
 
     def step():
@@ -727,8 +733,8 @@ def run_scan(args):
                           "n_gpus": world, "steps": 1, "warmup": 1 if args.workload == "scan_slice" else 0,
                           "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "dtype": "u64",
                           "data": "synthetic",
-                          "config": {"workload": "%s: L=%d, H=%d, P=64, d_s=128, B_blk=256, K_s=%d, N=2^16, 24 limbs, %s network, %s"
-                                                 % (args.workload, L, H, K_s,
+                          "config": {"workload": "%s: L=%d, H=%d, P=64, d_s=128, B_blk=256, stride=%d, K_s=%d, N=2^16, 24 limbs, %s network, %s"
+                                                 % (args.workload, L, H, stride, K_s,
                                                     {"bk": "Brent-Kung", "ks": "Kogge-Stone", "sk": "Sklansky"}[args.network],
                                                     ("radix-4 hoisted rotate-and-add chains" if args.hoist else "plain rotations")
                                                     + (", leaves built in groups of %d tokens" % G if G else "")),
@@ -931,6 +937,9 @@ def main():
                     help="1: baby rotations share one decomposition per input ciphertext (fesc_rotate_hoisted)")
     ap.add_argument("--group", type=int, default=4, choices=[0, 2, 4, 8, 16],
                     help="scan workloads: tokens per group of the grouped leaf build (0: token by token)")
+    ap.add_argument("--stride", type=int, default=256, choices=[128, 256],
+                    help="scan workloads: slots per channel of a state ciphertext; 256 (the paper's deployed shape: half of "
+                         "the slots idle, 12 chunks) or 128 (every slot used, 6 chunks, two token segments per block)")
     ap.add_argument("--network", default="bk", choices=["bk", "ks", "sk"],
                     help="scan workloads: prefix network (Brent-Kung, Kogge-Stone, Sklansky)")
     ap.add_argument("--workload", default="in_proj", choices=["in_proj", "out_proj", "rotations", "scan_slice", "scan_layer", "conv", "norm"],

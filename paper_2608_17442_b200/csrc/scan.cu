@@ -96,6 +96,7 @@ struct Arr {          // `count` compact ciphertexts [2][level][N], `stride` wor
 
 struct Geometry {
     uint32_t n, L, H, P, d_s, B, stride, c_state, E, hpc, R, K_s, K_blk, logB, dg;
+    uint32_t segs, Bt, dgt;      // token segments of a block (one x / a / output ciphertext each), tokens per segment
     uint32_t l0, l1, lS, linj, lout;
 };
 
@@ -325,7 +326,7 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
     const uint32_t N = X.N;
     const size_t in_ctw = X.ctw(l0), out_ctw = X.ctw(lout);
     if (!X.dry) {
-        cudaError_t e = cudaMemsetAsync(d_out, 0, (size_t)g.K_blk * g.K_s * out_ctw * sizeof(u64), X.st);
+        cudaError_t e = cudaMemsetAsync(d_out, 0, (size_t)g.K_blk * g.K_s * g.segs * out_ctw * sizeof(u64), X.st);
         if (e != cudaSuccess) return fesc_fail(X.ctx, FESC_ECUDA, cudaGetErrorString(e));
     }
     // carries g_j per chunk (level lS - (j-1)), stored at capacity lS
@@ -367,17 +368,19 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
             std::vector<uint32_t> lp(B, l1), ls(B, l1);
             if (G) {   // ---- leaves, grouped build: groups of G tokens share extraction, mask and fill ----
                 size_t m = X.top;
-                const uint32_t ng = B / G;
+                const uint32_t ng = B / G, ngs = g.Bt / G;      // groups per block / per segment
                 const size_t mask_words = (size_t)(l0 - 1) * N;
-                Arr srcx{const_cast<u64*>(d_x + ((size_t)j * g.K_s + kap) * in_ctw), 1, l0, in_ctw};
-                Arr apre = X.alloc(1, l0);
-                X.copy(Arr{const_cast<u64*>(d_a + ((size_t)j * g.K_s + kap) * in_ctw), 1, l0, in_ctw}, apre);
+                const size_t seg0 = ((size_t)j * g.K_s + kap) * g.segs;
+                Arr srcx{const_cast<u64*>(d_x + seg0 * in_ctw), g.segs, l0, in_ctw};
+                Arr apre = X.alloc(g.segs, l0);
+                X.copy(Arr{const_cast<u64*>(d_a + seg0 * in_ctw), g.segs, l0, in_ctw}, apre);
                 X.fill_right(apre, 1, ilog2(g.P));
                 Arr ex = X.alloc(ng, l0), xg = X.alloc(ng, l0 - 1), ag = X.alloc(ng, l0 - 1);
-                X.extract_n(srcx, G, ng, ex);
+                for (uint32_t sg = 0; sg < g.segs; sg++) X.extract_n(X.at(srcx, sg), G, ngs, X.at(ex, sg * ngs, ngs));
                 X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_xg, xg);
                 X.fill_right(xg, G, ilog2(g.d_s / G));
-                X.extract_n(apre, (int64_t)G * g.P, ng, ex);
+                for (uint32_t sg = 0; sg < g.segs; sg++)
+                    X.extract_n(X.at(apre, sg), (int64_t)G * g.P, ngs, X.at(ex, sg * ngs, ngs));
                 X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_ag, ag);
                 X.fill_right(ag, G * g.P, ilog2(g.R / (G * g.P)));
                 Arr xr = X.alloc(B, l0 - 2), cls2 = X.alloc(ng, l0 - 2), cls1 = X.alloc(ng, l1);
@@ -394,15 +397,16 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
                 X.top = m;
             } else {   // ---- leaves ----
                 size_t m = X.top;
-                Arr srcx{const_cast<u64*>(d_x + ((size_t)j * g.K_s + kap) * in_ctw), 1, l0, in_ctw};
-                Arr apre = X.alloc(1, l0);
-                X.copy(Arr{const_cast<u64*>(d_a + ((size_t)j * g.K_s + kap) * in_ctw), 1, l0, in_ctw}, apre);
+                const size_t seg0 = ((size_t)j * g.K_s + kap) * g.segs;
+                Arr srcx{const_cast<u64*>(d_x + seg0 * in_ctw), g.segs, l0, in_ctw};
+                Arr apre = X.alloc(g.segs, l0);
+                X.copy(Arr{const_cast<u64*>(d_a + seg0 * in_ctw), g.segs, l0, in_ctw}, apre);
                 X.fill_right(apre, 1, ilog2(g.P));
                 Arr ex = X.alloc(B, l0), xr = X.alloc(B, l0 - 1), ar = X.alloc(B, l0 - 1);
-                X.extract_all(srcx, 1, ex);
+                for (uint32_t sg = 0; sg < g.segs; sg++) X.extract_n(X.at(srcx, sg), 1, g.Bt, X.at(ex, sg * g.Bt, g.Bt));
                 X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_x, xr);
                 X.fill_right(xr, 1, ilog2(g.d_s));
-                X.extract_all(apre, g.P, ex);
+                for (uint32_t sg = 0; sg < g.segs; sg++) X.extract_n(X.at(apre, sg), g.P, g.Bt, X.at(ex, sg * g.Bt, g.Bt));
                 X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_a, ar);
                 X.adjust(ar, l1, 1, Ps);         // p_t = br(a_t): to the leaf level first, then the fill
                 X.fill_right(Ps, g.P, ilog2(g.R / g.P));
@@ -549,16 +553,18 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
                         X.mul_i(part, part, 3);                // -i (Xi - conj Xi) = 2 Im
                     }
                     X.ptmul_rescale(part, (const u64*)X.cs->d_mask_out, y);
-                    // placement: rotate right by t = t_lo + dg * t_hi
-                    const uint32_t nh = B / g.dg;
-                    for (uint32_t tl = 0; tl < g.dg; tl++)
-                        X.rot(X.strided(y, tl, g.dg, nh), -(int64_t)tl, X.strided(y2, tl, g.dg, nh));
+                    // placement: rotate right by the offset inside the token's segment, t' = t_lo + dgt * t_hi
+                    // (t = seg*Bt + t' and dgt divides Bt, so t mod dgt = t_lo and the high digit is (t / dgt) mod (Bt / dgt))
+                    const uint32_t nh = B / g.dgt, nhs = g.Bt / g.dgt;
+                    for (uint32_t tl = 0; tl < g.dgt; tl++)
+                        X.rot(X.strided(y, tl, g.dgt, nh), -(int64_t)tl, X.strided(y2, tl, g.dgt, nh));
                     for (uint32_t th = 0; th < nh; th++)
-                        X.rot(X.at(y2, th * g.dg, g.dg), -(int64_t)(g.dg * th), X.at(y, th * g.dg, g.dg));
-                    if (X.ok() && !X.dry) {
-                        u64* dst = d_out + ((size_t)j * g.K_s + k0 + which) * out_ctw;
+                        X.rot(X.at(y2, th * g.dgt, g.dgt), -(int64_t)(g.dgt * (th % nhs)), X.at(y, th * g.dgt, g.dgt));
+                    for (uint32_t sg = 0; sg < g.segs && X.ok() && !X.dry; sg++) {
+                        u64* dst = d_out + (((size_t)j * g.K_s + k0 + which) * g.segs + sg) * out_ctw;
                         prof_begin(X.ctx, PF_POINTWISE, X.st);
-                        k_ct_sum_into<<<dim3((N + 255) / 256, 2 * lout), 256, 0, X.st>>>(y.p, y.stride, B, dst, X.ctx->d_pc, N, lout);
+                        k_ct_sum_into<<<dim3((N + 255) / 256, 2 * lout), 256, 0, X.st>>>(y.p + (size_t)sg * g.Bt * y.stride, y.stride,
+                                                                                         g.Bt, dst, X.ctx->d_pc, N, lout);
                         prof_end(X.ctx, PF_POINTWISE, X.st);
                     }
                 }
@@ -583,8 +589,11 @@ extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint
     if (!g.L || !g.H || !pow2(g.P) || !pow2(g.d_s) || !pow2(g.B) || g.B < 2)
         return fesc_fail(ctx, FESC_EINVAL, "scan_contract: P, d_s, B_blk must be powers of two, B_blk >= 2");
     g.stride = desc->stride ? desc->stride : (g.d_s > g.B ? g.d_s : g.B);
-    if (!pow2(g.stride) || g.stride < g.d_s || g.stride < g.B || g.stride > g.n)
+    if (!pow2(g.stride) || g.stride < g.d_s || g.stride > g.n)
         return fesc_fail(ctx, FESC_EINVAL, "scan_contract: bad stride");
+    g.segs = g.B > g.stride ? g.B / g.stride : 1;
+    g.Bt = g.B / g.segs;
+    g.dgt = g.Bt < 16 ? g.Bt : 16;
     g.c_state = g.n / g.stride;
     g.E = g.H * g.P;
     if (g.c_state % g.P || g.E % g.c_state) return fesc_fail(ctx, FESC_EINVAL, "scan_contract: channels do not tile the chunks");
@@ -594,7 +603,7 @@ extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint
     g.K_blk = (g.L + g.B - 1) / g.B;
     g.logB = ilog2(g.B);
     g.dg = g.B < 16 ? g.B : 16;
-    if ((uint64_t)g.B * g.d_s > g.n || (uint64_t)g.B * g.P > g.R)
+    if ((uint64_t)g.B * g.d_s > g.n || (uint64_t)g.Bt * g.P > g.R)
         return fesc_fail(ctx, FESC_EINVAL, "scan_contract: block does not fit the compact packings");
     g.l0 = desc->n_limbs;
     if (desc->network > FESC_NET_SKLANSKY) return fesc_fail(ctx, FESC_EINVAL, "scan_contract: unknown prefix network");
@@ -602,8 +611,8 @@ extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint
         desc->network == FESC_NET_BRENT_KUNG ? g.logB - 1 : (g.K_blk > 2 ? g.K_blk - 2 : 0);   // lS - linj
     const uint32_t G = desc->group;
     if (G) {
-        if (G < 2 || (G & (G - 1)) || G > g.B || G > g.d_s)
-            return fesc_fail(ctx, FESC_EINVAL, "scan_contract: group must be a power of two, at most B_blk and d_s");
+        if (G < 2 || (G & (G - 1)) || G > g.Bt || G > g.d_s)
+            return fesc_fail(ctx, FESC_EINVAL, "scan_contract: group must be a power of two, at most the tokens of a segment and d_s");
         if (!consts->d_mask_xg || !consts->d_mask_ag || !consts->d_mask_x2 || !consts->d_mask_a2)
             return fesc_fail(ctx, FESC_EINVAL, "scan_contract: the grouped leaf build needs its four mask arrays");
     }

@@ -122,7 +122,9 @@ def test_bench_scan_rotation_amounts_match_the_dataflow():
     import bench
     from oracle.scan import ScanShape
 
-    for n, kw in ((128, dict(L=40, H=8, P=4, d_s=8, B_blk=16)), (32768, dict(L=2048, H=24, P=64, d_s=128, B_blk=256))):
+    for n, kw in ((128, dict(L=40, H=8, P=4, d_s=8, B_blk=16)), (32768, dict(L=2048, H=24, P=64, d_s=128, B_blk=256)),
+                  (128, dict(L=40, H=8, P=4, d_s=8, B_blk=16, stride=8)),
+                  (32768, dict(L=2048, H=24, P=64, d_s=128, B_blk=256, stride=128))):
         sh = ScanShape(n, **kw)
         for hoist in (False, True):
             for group in (0, 2, 4, 8):

@@ -29,8 +29,8 @@ def _run(name, hoist=0, network="bk", group=0, **kw):
     want = ScanEvaluator(orc, sh, c, hoist=bool(hoist)).run(ctX, ctA, ctB, ctC)
     adj_s = [c.adj_s.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
     adj_p = [c.adj_p.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
-    out = torch.empty((sh.K_blk, sh.K_s, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
-    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000, hoist,
+    out = torch.empty((sh.K_blk, sh.K_s, sh.segs, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
+    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, kw.get("stride", 0), l0, 100000, hoist,
                          {"bk": fesc.NET_BRENT_KUNG, "ks": fesc.NET_KOGGE_STONE, "sk": fesc.NET_SKLANSKY}[network], group)
     gm = [to_dev(m) for m in (c.mask_xg, c.mask_ag, c.mask_x2, c.mask_a2)] if group else None
     ctx.scan_contract(to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
@@ -77,6 +77,12 @@ def test_scan_grouped_leaf_build(hoist):
         assert _run("scan_small", hoist, "sk", 2, L=40, H=8, P=4, d_s=8, B_blk=16) < 2.0**-22
 
 
+@pytest.mark.parametrize("hoist,group", [(0, 0), (1, 0), (0, 4), (1, 4)])
+def test_scan_full_slot_variant_with_token_segments(hoist, group):
+    """stride = d_s < B_blk: two token segments per block, every slot of the state ciphertexts in use."""
+    assert _run("scan_small", hoist, group=group, L=40, H=8, P=4, d_s=8, B_blk=16, stride=8) < 2.0**-22
+
+
 def test_scan_unknown_network_is_refused():
     import torch
     import paper_2608_17442_b200 as fesc
@@ -105,8 +111,8 @@ def test_scan_missing_key_is_reported():
     assert e.value.code == fesc.ENOKEY
 
 
-@pytest.mark.parametrize("hoist,group", [(1, 0), (1, 4)])
-def test_scan_deployed_geometry_decrypts_to_recurrence(hoist, group):
+@pytest.mark.parametrize("hoist,group,stride", [(1, 0, 256), (1, 4, 256), (1, 4, 128)])
+def test_scan_deployed_geometry_decrypts_to_recurrence(hoist, group, stride):
     """N = 2^16, 24 limbs, stride 256, B_blk = 256, d_s = 128, P = 64 (the Mamba-2-base geometry) on a slice of
     the model: 4 heads (one chunk pair) and 512 tokens (two blocks, so the carry and its injection run).
     The oracle cannot follow ~36 000 key switches at this ring size, so the check here is the property that
@@ -116,8 +122,9 @@ def test_scan_deployed_geometry_decrypts_to_recurrence(hoist, group):
     import paper_2608_17442_b200 as fesc
 
     ctx, orc, p = ctx_pair("full")
-    sh = ScanShape(orc.n, L=512, H=4, P=64, d_s=128, B_blk=256)
-    assert (sh.stride, sh.c_state, sh.hpc, sh.K_s, sh.K_blk) == (256, 128, 2, 2, 2)
+    sh = ScanShape(orc.n, L=512, H=4 if stride == 256 else 8, P=64, d_s=128, B_blk=256, stride=stride)
+    assert (sh.stride, sh.c_state, sh.hpc, sh.K_s, sh.K_blk, sh.segs) == ((256, 128, 2, 2, 2, 1) if stride == 256 else
+                                                                         (128, 256, 4, 2, 2, 2))
     l0 = 24
     x, a, B, C = S.scan_inputs(S.config_seed(5), sh.L, sh.H, sh.P, 1, sh.d_s)
     c = ScanConsts(orc, sh, l0, 40, "bk", group)
@@ -127,8 +134,8 @@ def test_scan_deployed_geometry_decrypts_to_recurrence(hoist, group):
     ctX, ctA, ctB, ctC = encrypt_inputs(orc, sh, c, x, a, B, C)
     adj_s = [c.adj_s.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
     adj_p = [c.adj_p.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
-    out = torch.empty((sh.K_blk, sh.K_s, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
-    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, 0, l0, 100000, hoist, 0, group)
+    out = torch.empty((sh.K_blk, sh.K_s, sh.segs, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
+    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, sh.stride, l0, 100000, hoist, 0, group)
     gm = [to_dev(m) for m in (c.mask_xg, c.mask_ag, c.mask_x2, c.mask_a2)] if group else None
     args = (to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
             to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out, gm)
