@@ -656,7 +656,7 @@ def run_scan(args):
     ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
     n, N = ctx.N // 2, ctx.N
     H, L = (4, 512) if args.workload == "scan_slice" else (24, 2048)
-    P, d_s, B, stride, l0 = 64, 128, 256, int(args.stride), 24
+    P, d_s, B, stride, l0 = 64, 128, 256, int(args.stride), int(args.scan_limbs)
     if stride == 128 and args.workload == "scan_slice":
         H = 8                                                  # one chunk pair of 4 heads per chunk
     K_s, K_blk = H * P // (n // stride), L // B
@@ -733,8 +733,8 @@ def run_scan(args):
                           "n_gpus": world, "steps": 1, "warmup": 1 if args.workload == "scan_slice" else 0,
                           "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "dtype": "u64",
                           "data": "synthetic",
-                          "config": {"workload": "%s: L=%d, H=%d, P=64, d_s=128, B_blk=256, stride=%d, K_s=%d, N=2^16, 24 limbs, %s network, %s"
-                                                 % (args.workload, L, H, stride, K_s,
+                          "config": {"workload": "%s: L=%d, H=%d, P=64, d_s=128, B_blk=256, stride=%d, K_s=%d, N=2^16, %d limbs, %s network, %s"
+                                                 % (args.workload, L, H, stride, K_s, l0,
                                                     {"bk": "Brent-Kung", "ks": "Kogge-Stone", "sk": "Sklansky"}[args.network],
                                                     ("radix-4 hoisted rotate-and-add chains" if args.hoist else "plain rotations")
                                                     + (", leaves built in groups of %d tokens" % G if G else "")),
@@ -937,6 +937,8 @@ def main():
                     help="1: baby rotations share one decomposition per input ciphertext (fesc_rotate_hoisted)")
     ap.add_argument("--group", type=int, default=4, choices=[0, 2, 4, 8, 16],
                     help="scan workloads: tokens per group of the grouped leaf build (0: token by token)")
+    ap.add_argument("--scan-limbs", dest="scan_limbs", type=int, default=24,
+                    help="scan workloads: limbs of the input ciphertexts (24 = fresh; the grouped Brent-Kung schedule needs 22)")
     ap.add_argument("--stride", type=int, default=256, choices=[128, 256],
                     help="scan workloads: slots per channel of a state ciphertext; 256 (the paper's deployed shape: half of "
                          "the slots idle, 12 chunks) or 128 (every slot used, 6 chunks, two token segments per block)")

@@ -111,8 +111,8 @@ def test_scan_missing_key_is_reported():
     assert e.value.code == fesc.ENOKEY
 
 
-@pytest.mark.parametrize("hoist,group,stride", [(1, 0, 256), (1, 4, 256), (1, 4, 128)])
-def test_scan_deployed_geometry_decrypts_to_recurrence(hoist, group, stride):
+@pytest.mark.parametrize("hoist,group,stride,l0", [(1, 0, 256, 24), (1, 4, 256, 24), (1, 4, 128, 24), (1, 4, 128, 22)])
+def test_scan_deployed_geometry_decrypts_to_recurrence(hoist, group, stride, l0):
     """N = 2^16, 24 limbs, stride 256, B_blk = 256, d_s = 128, P = 64 (the Mamba-2-base geometry) on a slice of
     the model: 4 heads (one chunk pair) and 512 tokens (two blocks, so the carry and its injection run).
     The oracle cannot follow ~36 000 key switches at this ring size, so the check here is the property that
@@ -125,10 +125,10 @@ def test_scan_deployed_geometry_decrypts_to_recurrence(hoist, group, stride):
     sh = ScanShape(orc.n, L=512, H=4 if stride == 256 else 8, P=64, d_s=128, B_blk=256, stride=stride)
     assert (sh.stride, sh.c_state, sh.hpc, sh.K_s, sh.K_blk, sh.segs) == ((256, 128, 2, 2, 2, 1) if stride == 256 else
                                                                          (128, 256, 4, 2, 2, 2))
-    l0 = 24
     x, a, B, C = S.scan_inputs(S.config_seed(5), sh.L, sh.H, sh.P, 1, sh.d_s)
-    c = ScanConsts(orc, sh, l0, 40, "bk", group)
-    assert c.lv == (dict(l0=24, l1=21, lS=13, linj=6, lout=3) if group else dict(l0=24, l1=22, lS=14, linj=7, lout=4))
+    c = ScanConsts(orc, sh, l0, 40, "bk", group)     # l0 = 22: inputs two limbs down, output at the last level
+    assert c.lv == (dict(l0=l0, l1=l0 - 3, lS=l0 - 11, linj=l0 - 18, lout=l0 - 21) if group else
+                    dict(l0=24, l1=22, lS=14, linj=7, lout=4))
     for r in sh.rotation_amounts(bool(hoist), group) + [CONJ]:
         ctx.add_galois_key(r, key_id_for(sh, r))
     ctX, ctA, ctB, ctC = encrypt_inputs(orc, sh, c, x, a, B, C)
