@@ -150,21 +150,21 @@ __device__ __forceinline__ void strided_body(u64* __restrict__ p, u64* __restric
     const uint32_t h2 = sub >> 2, l2 = sub & 3;
     u64 x[8];
     if (!INV) {
-        // round 1: hi = k*32 + sub, local stages 0,1,2
+        // first register round: hi = k*32 + sub, local stages 0,1,2
 #pragma unroll
         for (int k = 0; k < 8; k++) x[k] = p[(size_t)(k * 32 + sub) * 256 + col];
         fwd_round3<W>(x, tw, 1, 2, 4, q, q2);
 #pragma unroll
         for (int k = 0; k < 8; k++) sm[(k * 32 + sub) * NTT_COLS + col] = x[k];
         __syncthreads();
-        // round 2: hi = h2*32 + k*4 + l2, local stages 3,4,5
+        // second register round: hi = h2*32 + k*4 + l2, local stages 3,4,5
 #pragma unroll
         for (int k = 0; k < 8; k++) x[k] = sm[(h2 * 32 + k * 4 + l2) * NTT_COLS + col];
         fwd_round3<W>(x, tw, 8 + h2, 16 + 2 * h2, 32 + 4 * h2, q, q2);
 #pragma unroll
         for (int k = 0; k < 8; k++) sm[(h2 * 32 + k * 4 + l2) * NTT_COLS + col] = x[k];
         __syncthreads();
-        // round 3: hi = sub*8 + k, local stages 6,7
+        // third register round: hi = sub*8 + k, local stages 6,7
 #pragma unroll
         for (int k = 0; k < 8; k++) x[k] = sm[(sub * 8 + k) * NTT_COLS + col];
         fwd_round2<W>(x, tw, 64 + 2 * sub, 128 + 4 * sub, q, q2);
