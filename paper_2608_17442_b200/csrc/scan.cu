@@ -10,6 +10,7 @@
 #include <math.h>
 
 #include "ops.cuh"
+#include <map>
 
 // ---------------------------------------------------------------------------------------
 // pointwise kernels on batches of compact ciphertexts [2][level][N]
@@ -232,6 +233,44 @@ struct Exec {
         rescale(t, out);
         top = mark;
     }
+    // out[i] (level dst, contiguous) = slot pos[i] of `base` (capacity stride base.stride, current level lev[pos[i]])
+    // brought to dst.  Slots that sit at the same level go down in ONE batch: straight from the slots when their
+    // positions are equally spaced, through a gathered copy otherwise; the result lands in out directly when the
+    // group is a run of consecutive outputs.
+    void adjust_many(const Arr& base, const std::vector<uint32_t>& pos, const std::vector<uint32_t>& lev, uint32_t dst,
+                     int kind, const Arr& out) {
+        std::map<uint32_t, std::vector<uint32_t>> groups;      // source level -> output indices
+        for (uint32_t i = 0; i < pos.size(); i++) groups[lev[pos[i]]].push_back(i);
+        for (auto& kv : groups) {
+            const uint32_t src = kv.first;
+            const std::vector<uint32_t>& idx = kv.second;
+            const uint32_t cnt = (uint32_t)idx.size();
+            auto slot = [&](uint32_t i) { return Arr{base.p + (size_t)pos[i] * base.stride, 1, src, ctw(src)}; };
+            if (src == dst || cnt == 1) {
+                for (uint32_t i : idx) adjust(slot(i), dst, kind, at(out, i));
+                continue;
+            }
+            bool spaced = true, run = true;
+            const int64_t step = (int64_t)pos[idx[1]] - (int64_t)pos[idx[0]];
+            for (uint32_t k = 1; k < cnt; k++) {
+                spaced = spaced && step > 0 && (int64_t)pos[idx[k]] - (int64_t)pos[idx[k - 1]] == step;
+                run = run && idx[k] == idx[k - 1] + 1;
+            }
+            size_t mark = top;
+            Arr gin = spaced ? Arr{base.p + (size_t)pos[idx[0]] * base.stride, cnt, src, base.stride * (size_t)step}
+                             : alloc(cnt, src);
+            if (!spaced)
+                for (uint32_t k = 0; k < cnt; k++) copy(slot(idx[k]), at(gin, k));
+            if (run) {
+                adjust(gin, dst, kind, at(out, idx[0], cnt));
+            } else {
+                Arr gout = alloc(cnt, dst);
+                adjust(gin, dst, kind, gout);
+                for (uint32_t k = 0; k < cnt; k++) copy(at(gout, k), at(out, idx[k]));
+            }
+            top = mark;
+        }
+    }
     bool key_ok(int64_t amount) {
         uint32_t kid = key_for(amount);
         if (ctx->keys.count(kid)) return true;
@@ -421,13 +460,10 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
                 size_t m = X.top;
                 Arr pL = X.alloc(cnt, lvl), sL = X.alloc(cnt, lvl), pR = X.alloc(cnt, lvl), sR = X.alloc(cnt, lvl - 1);
                 Arr np_ = X.alloc(cnt, lvl - 1), ns = X.alloc(cnt, lvl - 1);
-                for (uint32_t i = 0; i < cnt; i++) {
-                    const uint32_t a = left[i], b = right[i];
-                    if (need_p) X.adjust(Arr{Ps.p + (size_t)a * Ps.stride, 1, lp[a], X.ctw(lp[a])}, lvl, 1, X.at(pL, i));
-                    X.adjust(Arr{Ss.p + (size_t)a * Ss.stride, 1, ls[a], X.ctw(ls[a])}, lvl, 0, X.at(sL, i));
-                    X.adjust(Arr{Ps.p + (size_t)b * Ps.stride, 1, lp[b], X.ctw(lp[b])}, lvl, 1, X.at(pR, i));
-                    X.adjust(Arr{Ss.p + (size_t)b * Ss.stride, 1, ls[b], X.ctw(ls[b])}, lvl - 1, 0, X.at(sR, i));
-                }
+                if (need_p) X.adjust_many(Ps, left, lp, lvl, 1, pL);
+                X.adjust_many(Ss, left, ls, lvl, 0, sL);
+                X.adjust_many(Ps, right, lp, lvl, 1, pR);
+                X.adjust_many(Ss, right, ls, lvl - 1, 0, sR);
                 if (need_p) X.mul_rescale(pR, pL, np_);
                 X.mul_rescale(pR, sL, ns);
                 X.add(ns, sR, ns);
@@ -488,12 +524,12 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
             {
                 size_t m = X.top;
                 Arr h = X.alloc(B, linj - 1);
-                for (uint32_t t = 0; t < B; t++)
-                    X.adjust(Arr{Ss.p + (size_t)t * Ss.stride, 1, ls[t], X.ctw(ls[t])}, linj - 1, 0, X.at(h, t));
+                std::vector<uint32_t> every(B);
+                for (uint32_t t = 0; t < B; t++) every[t] = t;
+                X.adjust_many(Ss, every, ls, linj - 1, 0, h);
                 if (j > 0) {
                     Arr pp = X.alloc(B, linj), gg = X.alloc(1, linj), pg = X.alloc(B, linj - 1);
-                    for (uint32_t t = 0; t < B; t++)
-                        X.adjust(Arr{Ps.p + (size_t)t * Ps.stride, 1, lp[t], X.ctw(lp[t])}, linj, 1, X.at(pp, t));
+                    X.adjust_many(Ps, every, lp, linj, 1, pp);
                     X.adjust(Arr{carry.p + (size_t)kap * carry.stride, 1, carry_level[kap], X.ctw(carry_level[kap])}, linj, 0, gg);
                     X.mul_rescale(pp, gg, pg);
                     X.add(h, pg, h);
