@@ -43,10 +43,15 @@ contraction -> linj-2;  reduction, conjugation, unpacking there;  output mask ->
 Grouped leaf build (`group` = G > 0, a separately defined mode: other residues, same values).  Building br(x_t) and
 br(a_t) token by token costs log2(d_s) and log2(R/P) rotate-and-add steps per token at the top levels.  With groups of
 G consecutive tokens the group is extracted, masked (slots [0,G) of every stride for x, [0,GP) of every head region for
-a) and filled ONCE for its G tokens (log2(d_s/G), log2(R/(GP)) steps: the pattern of G tokens repeats), a second mask
-keeps the copies of one token (slot class g modulo G, block class g modulo GP) one level lower, and log2 G signed steps
-(towards lower slots for the bits set in g, higher slots for the others) fill the classes in between.  The second mask
-costs one level: br(B_t) is brought to l0-2 before its fill and the leaves sit at l1 = l0-3.
+a) and filled ONCE for its G tokens (log2(d_s/G), log2(R/(GP)) steps: the pattern of G tokens repeats with period G
+slots resp. G blocks of P slots).  The copies of token g of the group sit in class g of every period; class j of its
+broadcast takes them from class g, i.e. from the group ciphertext rotated by (g - j) units, so
+
+    br(token g of the group) = rescale( sum_{j<G} classmask_j (.) rot(group, (g - j) unit) ),   unit = 1 (x), P (a):
+
+the 2(G-1) rotations by +-unit..+-(G-1) unit are taken ONCE per group (one decomposition in hoisted mode) and every
+token is G plaintext multiply-accumulates and one rescale (no copy leaves its period, so nothing crosses a channel or
+head boundary).  The class masks cost one level: br(B_t) is brought to l0-2 before its fill, leaves at l1 = l0-3.
 
 Other prefix networks (App. "Prefix-Network Selection"; `network` = "ks" Kogge-Stone, "sk" Sklansky; "bk" above is the
 default): stage s = 1..logB combines operands at l1-(s-1) into results at l1-s, every prefix is complete at lS and there
@@ -105,14 +110,15 @@ class ScanShape:
                 (-self.stride, lg(self.c_state)), (1, lg(self.d_s))]
 
     @staticmethod
-    def class_deltas(g: int, G: int, unit: int):
-        """Signed slot shifts (LEFT positive) of the steps that copy class g of a period of G blocks of `unit` slots to
-        every class: bit b of g set -> the copies move to lower slots (+unit 2^b), else to higher slots (-unit 2^b)."""
-        return [unit * (1 << b) if (g >> b) & 1 else -unit * (1 << b) for b in range(int(math.log2(G)))]
+    def class_shifts(G: int, unit: int):
+        """Rotation amounts (LEFT positive) of the grouped leaf build, in the order the rotated copies are kept:
+        +unit, .., +(G-1) unit, -unit, .., -(G-1) unit.  The copy for class difference g - j = k sits at index k - 1
+        (k > 0) or G - 2 - k (k < 0)."""
+        return [k * unit for k in range(1, G)] + [-k * unit for k in range(1, G)]
 
     def rotation_amounts(self, hoist: bool = False, group: int = 0):
         """hoist=True adds the amounts 3 * unit * 2^b of the radix-4 chains (b even, b + 1 < steps); group=G adds the
-        group extraction amounts and the signed class steps (in hoisted mode also the sums of their pairs)."""
+        group extraction amounts and the class shifts +-unit .. +-(G-1) unit."""
         n, dg, B, dgt, Bt = self.n, self.dg, self.B, self.dgt, self.Bt
         am = set()
         for unit in (1, self.P):                      # extraction of x, a (offsets inside a segment)
@@ -136,11 +142,7 @@ class ScanShape:
                 for unit, steps in ((-G, int(math.log2(self.d_s // G))), (-G * self.P, int(math.log2(self.R // (G * self.P))))):
                     am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
             for unit in (1, self.P):
-                for g in range(G):
-                    d = self.class_deltas(g, G, unit)
-                    am |= {v % n for v in d}
-                    if hoist:
-                        am |= {(d[b] + d[b + 1]) % n for b in range(0, len(d) - 1, 2)}
+                am |= {v % n for v in self.class_shifts(G, unit)}
         am.discard(0)
         return sorted(am)
 
@@ -335,20 +337,26 @@ class ScanEvaluator:
                 b += 1
         return ct
 
-    def signed_chain(self, ct, deltas):
-        """ct += rot(ct, delta) for every delta in turn (LEFT shifts, signed).  Hoisted mode: two steps together as
-        ct + rot(ct, d1) + rot(ct, d2) + rot(ct, d1 + d2), one decomposition and one division by P."""
-        b = 0
-        while b < len(deltas):
-            if self.hoist and b + 1 < len(deltas):
-                d1, d2 = deltas[b], deltas[b + 1]
-                self.count["rot"] += 3
-                ct = self.o.rotate_sum_hoisted(ct, [key_id_for(self.sh, d, self.kb) for d in (d1, d2, d1 + d2)])
-                b += 2
-            else:
-                ct = self.add(ct, self.rot(ct, deltas[b]))
-                b += 1
-        return ct
+    def class_broadcasts(self, group_ct, masks, unit):
+        """[rescale(sum_j masks[j] (.) rot(group_ct, (g - j) unit)) for g < G]: the broadcasts of the G tokens of one
+        filled group ciphertext.  The 2(G-1) rotations are taken once (hoisted mode: one decomposition)."""
+        G = self.group
+        shifts = self.sh.class_shifts(G, unit)
+        if self.hoist:
+            self.count["rot"] += len(shifts)
+            rots = self.o.rotate_hoisted(group_ct, [key_id_for(self.sh, d, self.kb) for d in shifts])
+        else:
+            rots = [self.rot(group_ct, d) for d in shifts]
+        out = []
+        for g in range(G):
+            acc = np.zeros_like(group_ct)
+            for j in range(G):
+                k = g - j
+                src = group_ct if k == 0 else rots[k - 1 if k > 0 else G - 2 - k]
+                acc = self.o.ct_pt_mac(src, masks[j], acc)
+            self.count["ptmul"] += G
+            out.append(self.o.rescale(acc))
+        return out
 
     def fill_right(self, ct, unit, steps):
         """ct += rot(ct, -unit*2^b) for b = 0..steps-1 (copies a block to 2^steps consecutive blocks)."""
@@ -419,7 +427,7 @@ class ScanEvaluator:
 
     def leaves_grouped(self, ctX, ctA, brB):
         """Leaves (br a_t, br x_t (.) br B_t) at l1 = l0-3 with the grouped build (module header): groups of G tokens
-        are extracted, masked and filled once; a second mask and log2 G signed steps separate the tokens."""
+        are extracted, masked and filled once; masked sums of the group's 2(G-1) rotations separate the tokens."""
         sh, c, G = self.sh, self.c, self.group
         l1, lg = c.lv["l1"], lambda v: int(math.log2(v))
         T = []
@@ -430,11 +438,10 @@ class ScanEvaluator:
             for u in range(sh.Bt // G):
                 xg = self.fill_right(self.ptmul_rescale(gx[u], c.mask_xg), G, lg(sh.d_s // G))
                 ag = self.fill_right(self.ptmul_rescale(ga[u], c.mask_ag), G * sh.P, lg(sh.R // (G * sh.P)))
+                bx, ba = self.class_broadcasts(xg, c.mask_x2, 1), self.class_broadcasts(ag, c.mask_a2, sh.P)
                 for g in range(G):
-                    xr = self.signed_chain(self.ptmul_rescale(xg, c.mask_x2[g]), sh.class_deltas(g, G, 1))
-                    ar = self.adjust(self.ptmul_rescale(ag, c.mask_a2[g]), l1, "p")
-                    ar = self.signed_chain(ar, sh.class_deltas(g, G, sh.P))
-                    T.append((ar, self.mul_rescale(xr, brB[seg * sh.Bt + u * G + g])))
+                    ar = self.adjust(ba[g], l1, "p")
+                    T.append((ar, self.mul_rescale(bx[g], brB[seg * sh.Bt + u * G + g])))
         return T
 
     def brent_kung(self, T, need_p_down):

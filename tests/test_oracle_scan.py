@@ -179,9 +179,9 @@ def test_other_prefix_networks(network):
 
 
 def test_grouped_leaf_build():
-    """Leaves built for groups of G tokens (one extraction, mask and fill per group, then a class mask and log2 G
-    signed steps per token): same contract output, same compositions, one level more, and exactly the rotations the
-    closed form predicts fewer."""
+    """Leaves built for groups of G tokens (one extraction, mask and fill per group, then every token as a masked sum
+    of the group's 2(G-1) rotations): same contract output, same compositions, one level more, and exactly the
+    rotations the closed form predicts fewer."""
     kw = dict(L=40, H=8, P=4, d_s=8, B_blk=16)
     sh, ev0, m0, ref = _run("scan_small", **kw)
     _, ev, m, _ = _run("scan_small", group=4, **kw)
@@ -191,21 +191,21 @@ def test_grouped_leaf_build():
     lg = lambda v: int(math.log2(v))
     B, G, P, R, d_s = sh.B, 4, sh.P, sh.R, sh.d_s
     plain = 2 * (B - 1) + B * (lg(d_s) + lg(R // P))
-    grouped = 2 * (B // G - 1) + (B // G) * (lg(d_s // G) + lg(R // (G * P))) + 2 * B * lg(G)
-    assert ev0.count["rot"] - ev.count["rot"] == sh.K_blk * sh.K_s * (plain - grouped) == 720
-    assert ev.count["ptmul"] - ev0.count["ptmul"] == sh.K_blk * sh.K_s * 2 * (B // G)
-    # the signed steps of class g reach every class exactly once
+    grouped = 2 * (B // G - 1) + (B // G) * (lg(d_s // G) + lg(R // (G * P))) + 2 * (B // G) * 2 * (G - 1)
+    assert ev0.count["rot"] - ev.count["rot"] == sh.K_blk * sh.K_s * (plain - grouped) == 912
+    assert ev.count["ptmul"] - ev0.count["ptmul"] == sh.K_blk * sh.K_s * (2 * (B // G) + 2 * B * G - 2 * B)
+    # the rotated copy kept for the class difference k = g - j is the rotation by k units
     for G in (2, 4, 8):
-        for g in range(G):
-            reach = {0}
-            for d in sh.class_deltas(g, G, 1):
-                reach |= {r - d for r in reach}          # a LEFT shift by d moves a copy d slots down
-            assert sorted(g + r for r in reach) == list(range(G))
-    # deployed shape: 1 854 instead of 4 350 extraction and fill rotations per (block, chunk)
+        shifts = sh.class_shifts(G, 3)
+        assert len(set(shifts)) == 2 * (G - 1)
+        for k in range(-(G - 1), G):
+            if k:
+                assert shifts[k - 1 if k > 0 else G - 2 - k] == 3 * k
+    # deployed shape: 1 598 instead of 4 350 extraction and fill rotations per (block, chunk)
     big = ScanShape(32768, L=2048, H=24, P=64, d_s=128, B_blk=256)
     B, G, P, R, d_s = 256, 4, 64, big.R, 128
     assert 2 * (B - 1) + B * (lg(d_s) + lg(R // P)) == 4350
-    assert 2 * (B // G - 1) + (B // G) * (lg(d_s // G) + lg(R // (G * P))) + 2 * B * lg(G) == 1854
+    assert 2 * (B // G - 1) + (B // G) * (lg(d_s // G) + lg(R // (G * P))) + 2 * (B // G) * 2 * (G - 1) == 1598
     assert levels(24, 8, 8, "bk", 4) == dict(l0=24, l1=21, lS=13, linj=6, lout=3)
 
 
