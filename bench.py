@@ -585,7 +585,7 @@ def scan_rotation_amounts(n, P, d_s, B, stride, hoist=False, group=0):
         lg = lambda v: int(math.log2(v))
         for unit, steps in ((-1, lg(P)), (-1, lg(d_s)), (-P, lg(R // P)), (-stride, lg(c_state)), (1, lg(d_s))):
             am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
-    if group:    # grouped leaf build: group offsets (two digits) and the signed class steps (and their pair sums)
+    if group:    # grouped leaf build: group offsets (two digits) and the class shifts +-unit .. +-(G-1) unit
         cnt = Bt // group
         dgg = min(16, cnt)
         for unit in (group, group * P):
@@ -594,11 +594,7 @@ def scan_rotation_amounts(n, P, d_s, B, stride, hoist=False, group=0):
             for unit, steps in ((-group, int(math.log2(d_s // group))), (-group * P, int(math.log2(R // (group * P))))):
                 am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
         for unit in (1, P):
-            for c in range(group):
-                d = [unit * (1 << b) if (c >> b) & 1 else -unit * (1 << b) for b in range(int(math.log2(group)))]
-                am |= {v % n for v in d}
-                if hoist:
-                    am |= {(d[b] + d[b + 1]) % n for b in range(0, len(d) - 1, 2)}
+            am |= {(k * unit) % n for k in range(1, group)} | {(-k * unit) % n for k in range(1, group)}
     am.discard(0)
     return sorted(am)
 

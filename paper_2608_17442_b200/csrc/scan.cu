@@ -302,37 +302,47 @@ struct Exec {
         top = mark;
     }
     void fill_right(const Arr& a, uint32_t unit, uint32_t steps) { chain(a, -(int64_t)unit, steps); }
-    // a += rot(a, delta) for every delta in turn (signed LEFT shifts).  Hoisted mode takes two steps together:
-    // a + rot(a, d1) + rot(a, d2) + rot(a, d1 + d2).
-    void signed_chain(const Arr& a, const std::vector<int64_t>& deltas) {
+    // Broadcasts of the tokens of filled group ciphertexts (grouped leaf build): for class c < G
+    //   out_c[u] = rescale( sum_{j<G} masks[j] (.) rot(grp[u], (c - j) unit) ),
+    // with the 2(G-1) rotations by +unit..+(G-1)unit, -unit..-(G-1)unit taken once for the whole batch of groups
+    // (hoisted mode: one decomposition per group).  `deliver(c, res)` receives the batch of class c (level - 1,
+    // contiguous, valid until it returns).
+    template <class F>
+    void class_broadcasts(const Arr& grp, const u64* masks, uint32_t G, uint32_t unit, F deliver) {
         size_t mark = top;
-        Arr t = alloc(a.count, a.level);
-        size_t b = 0;
-        while (b < deltas.size() && ok()) {
-            if (desc->hoist && b + 1 < deltas.size()) {
-                const int64_t d1 = deltas[b], d2 = deltas[b + 1];
-                if (!key_ok(d1) || !key_ok(d2) || !key_ok(d1 + d2)) break;
-                if (!dry) {
-                    const uint32_t ids[3] = {key_for(d1), key_for(d2), key_for(d1 + d2)};
-                    rc = rotate_sum_hoisted_internal(ctx, a.p, a.stride, t.p, t.stride, a.count, a.level, ids, 3, ks, st);
-                    copy(t, a);
+        const uint32_t nk = 2 * (G - 1), cnt = grp.count, lvl = grp.level;
+        const size_t mask_words = (size_t)lvl * N;
+        Arr rots = alloc(nk * cnt, lvl);       // [shift][group]
+        std::vector<int64_t> shifts;
+        for (uint32_t k = 1; k < G; k++) shifts.push_back((int64_t)k * unit);
+        for (uint32_t k = 1; k < G; k++) shifts.push_back(-(int64_t)k * unit);
+        if (desc->hoist) {
+            std::vector<uint32_t> ids;
+            for (int64_t d : shifts)
+                if (key_ok(d)) ids.push_back(key_for(d));
+            if (ok() && !dry)
+                rc = rotate_hoisted_internal(ctx, grp.p, grp.stride, rots.p, rots.stride, (size_t)cnt * rots.stride, cnt, lvl,
+                                             ids.data(), nk, ks, st);
+        } else {
+            for (uint32_t i = 0; i < nk; i++) rot(grp, shifts[i], at(rots, i * cnt, cnt));
+        }
+        Arr acc = alloc(cnt, lvl), res = alloc(cnt, lvl - 1);
+        for (uint32_t c = 0; c < G && ok(); c++) {
+            if (!dry) {
+                cudaError_t e = cudaMemsetAsync(acc.p, 0, (size_t)cnt * ctw(lvl) * sizeof(u64), st);
+                if (e != cudaSuccess) rc = fesc_fail(ctx, FESC_ECUDA, cudaGetErrorString(e));
+                for (uint32_t j = 0; j < G && ok(); j++) {
+                    const int k = (int)c - (int)j;
+                    const Arr src = k == 0 ? grp : at(rots, (uint32_t)(k > 0 ? k - 1 : (int)G - 2 - k) * cnt, cnt);
+                    // the public multiply-accumulate takes a contiguous batch; group ciphertexts are contiguous
+                    rc = fesc_ct_pt_mac(ctx, (const uint64_t*)src.p, (const uint64_t*)(masks + j * mask_words), 0,
+                                        (uint64_t*)acc.p, cnt, lvl, (void*)st);
                 }
-                b += 2;
-            } else {
-                rot(a, deltas[b], t);
-                add(a, t, a);
-                b += 1;
             }
+            rescale(acc, res);
+            deliver(c, res);
         }
         top = mark;
-    }
-    // steps that copy class cls of a period of G blocks of `unit` slots to every class: bit b of cls set -> the
-    // copies move to lower slots (+unit 2^b), else to higher slots (-unit 2^b)
-    static std::vector<int64_t> class_deltas(uint32_t cls, uint32_t G, uint32_t unit) {
-        std::vector<int64_t> d;
-        for (uint32_t b = 0; (1u << b) < G; b++)
-            d.push_back(((cls >> b) & 1) ? (int64_t)unit * (1 << b) : -(int64_t)unit * (1 << b));
-        return d;
     }
     // out[t] = rot(src, unit * t) for t = 0..count-1, via t = t_lo + dg * t_hi, dg = min(16, count) (hoisted mode:
     // the dg-1 low-digit rotations of one ciphertext share its decomposition)
@@ -408,7 +418,6 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
             if (G) {   // ---- leaves, grouped build: groups of G tokens share extraction, mask and fill ----
                 size_t m = X.top;
                 const uint32_t ng = B / G, ngs = g.Bt / G;      // groups per block / per segment
-                const size_t mask_words = (size_t)(l0 - 1) * N;
                 const size_t seg0 = ((size_t)j * g.K_s + kap) * g.segs;
                 Arr srcx{const_cast<u64*>(d_x + seg0 * in_ctw), g.segs, l0, in_ctw};
                 Arr apre = X.alloc(g.segs, l0);
@@ -422,16 +431,14 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
                     X.extract_n(X.at(apre, sg), (int64_t)G * g.P, ngs, X.at(ex, sg * ngs, ngs));
                 X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_ag, ag);
                 X.fill_right(ag, G * g.P, ilog2(g.R / (G * g.P)));
-                Arr xr = X.alloc(B, l0 - 2), cls2 = X.alloc(ng, l0 - 2), cls1 = X.alloc(ng, l1);
-                for (uint32_t c = 0; c < G && X.ok(); c++) {      // the tokens u*G + c of every group u
-                    X.ptmul_rescale(xg, (const u64*)X.cs->d_mask_x2 + c * mask_words, cls2);
-                    X.signed_chain(cls2, Exec::class_deltas(c, G, 1));
-                    X.copy(cls2, X.strided(xr, c, G, ng));
-                    X.ptmul_rescale(ag, (const u64*)X.cs->d_mask_a2 + c * mask_words, cls2);
-                    X.adjust(cls2, l1, 1, cls1);
-                    X.signed_chain(cls1, Exec::class_deltas(c, G, g.P));
+                Arr xr = X.alloc(B, l0 - 2), cls1 = X.alloc(ng, l1);
+                // class c = the tokens u*G + c of every group u
+                X.class_broadcasts(xg, (const u64*)X.cs->d_mask_x2, G, 1,
+                                   [&](uint32_t c, const Arr& res) { X.copy(res, X.strided(xr, c, G, ng)); });
+                X.class_broadcasts(ag, (const u64*)X.cs->d_mask_a2, G, g.P, [&](uint32_t c, const Arr& res) {
+                    X.adjust(res, l1, 1, cls1);          // p_t = br(a_t) at the leaf level
                     X.copy(cls1, X.strided(Ps, c, G, ng));
-                }
+                });
                 X.mul_rescale(xr, brB, Ss);      // s_t = br(x_t) (.) br(B_t), level l1 = l0-3
                 X.top = m;
             } else {   // ---- leaves ----
