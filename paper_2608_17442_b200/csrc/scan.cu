@@ -1,7 +1,8 @@
 // Factorized scan-contract on packed ciphertexts:
 //   h_k = br(a_k) (.) h_{k-1} + x_k (x) B_k,  h_0 = 0,   m_k = Sigma_{d_s}(h_k (.) br(C_k))
 // evaluated as: per token block, broadcast of the compact factors to the state packing (rotations,
-// masks, rotate-and-add fills), leaves (p, s) = (br a, br x (.) br B), a Brent-Kung network of affine
+// masks, rotate-and-add fills; optionally for groups of tokens at once), leaves (p, s) = (br a, br x (.) br B),
+// a prefix network (Brent-Kung, Kogge-Stone or Sklansky) of affine
 // compositions (p_R p_L, p_R s_L + s_R), serialized block carries, carry injection, contraction with
 // br(C), a complex-paired rotate-add reduction over the state axis with one conjugation per chunk
 // pair, output mask and placement.  The host code below only sequences batched kernels (rotations
@@ -9,8 +10,9 @@
 // pointwise kernels here.  Levels follow a fixed schedule (see fesc.h).
 #include <math.h>
 
-#include "ops.cuh"
 #include <map>
+
+#include "ops.cuh"
 
 // ---------------------------------------------------------------------------------------
 // pointwise kernels on batches of compact ciphertexts [2][level][N]
