@@ -699,6 +699,13 @@ def run_scan(args):
             ctx.scan_contract(x, a, Bc, Cc, desc, masks[0], masks[1], masks[2], masks[3][:linj - 2], adj, adj, out, gm)
         return gather_chunk_outputs(out[:, :mine], parts, rank, world, K_blk, K_s) if world > 1 else out
 
+    if args.profile_step:           # one bare step for a profiler's launch list (no warm-up, no timing claims)
+        step()
+        ctx.sync()
+        if rank == 0:
+            print(json.dumps({"profile_run": True, "gpu_launches": ctx.counters()[4], "key_switches": ctx.counters()[1]}),
+                  flush=True)
+        return
     breakdown = None
     if args.workload == "scan_slice":
         step()                      # warm-up (sizes the scratch arena)
