@@ -305,14 +305,19 @@ __global__ void __launch_bounds__(256, (TT * PT > 16 ? 1 : 2)) k_bsgs_accumulate
 // congruent to the low part modulo 2^64 and within 2^63 of the approximation; one 128-bit reduction follows.
 // Per term that is 8 multiplier-pipe cycles and 2 FP64-pipe cycles per warp, on pipes that run concurrently,
 // instead of 6 FP64 operations and a rounding.
+// threads per CTA: two CTAs of 128 per SM (the registers allow 256 threads in all) overlap one CTA's reconstruction and
+// stores with the other's term loop
+#ifndef MIX_THREADS
+#define MIX_THREADS 128
+#endif
 template <int TT, int PT, int STAGES>
-__global__ void __launch_bounds__(256, (TT * PT >= 12 ? 1 : 2)) k_bsgs_accumulate_mixed(
+__global__ void __launch_bounds__(MIX_THREADS, (TT * PT >= 12 ? 256 / MIX_THREADS : 2 * 256 / MIX_THREADS)) k_bsgs_accumulate_mixed(
     const u64* __restrict__ rot, const u64* __restrict__ diags, u64* __restrict__ acc,
     const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level, uint32_t tbs, uint32_t terms, uint32_t bp_count) {
     constexpr int ROWS = 2 * TT + PT;
-    extern __shared__ __align__(16) u64 stage[];          // [STAGES][ROWS][256]
+    extern __shared__ __align__(16) u64 stage[];          // [STAGES][ROWS][MIX_THREADS]
     const uint32_t tid = threadIdx.x;
-    const uint32_t c = blockIdx.y * 256 + tid;
+    const uint32_t c = blockIdx.y * MIX_THREADS + tid;
     // blockIdx.x = (b,p) tile * token-block tiles + token-block tile: CTAs that read the same diagonal rows are
     // scheduled next to each other (the second read hits L2), and so are the (b,p) tiles that share ciphertext rows
     const uint32_t tb_tiles = (tbs + TT - 1) / TT;
@@ -332,14 +337,14 @@ __global__ void __launch_bounds__(256, (TT * PT >= 12 ? 1 : 2)) k_bsgs_accumulat
     uint32_t slot = 0;                                     // stage that the next issue fills
     const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(stage) + tid * 8;
     auto issue = [&]() {
-        const uint32_t dst = sbase + slot * (ROWS * 2048);
+        const uint32_t dst = sbase + slot * (ROWS * MIX_THREADS * 8);
 #pragma unroll
         for (int i = 0; i < TT; i++) {
-            cp_async8s(dst + (2 * i) * 2048, xrun + xoff[i]);
-            cp_async8s(dst + (2 * i + 1) * 2048, xrun + xoff[i] + poly);
+            cp_async8s(dst + (2 * i) * (MIX_THREADS * 8), xrun + xoff[i]);
+            cp_async8s(dst + (2 * i + 1) * (MIX_THREADS * 8), xrun + xoff[i] + poly);
         }
 #pragma unroll
-        for (int j = 0; j < PT; j++) cp_async8s(dst + (2 * TT + j) * 2048, drun + doff[j]);
+        for (int j = 0; j < PT; j++) cp_async8s(dst + (2 * TT + j) * (MIX_THREADS * 8), drun + doff[j]);
         xrun += ctw;
         drun += poly;
         slot = slot + 1 == STAGES ? 0 : slot + 1;
@@ -363,7 +368,7 @@ __global__ void __launch_bounds__(256, (TT * PT >= 12 ? 1 : 2)) k_bsgs_accumulat
         if (t + STAGES - 1 < terms) issue();
         cp_async_commit();
         cp_async_wait<STAGES - 1>();
-        const u64* sm = stage + (size_t)rslot * ROWS * 256 + tid;
+        const u64* sm = stage + (size_t)rslot * ROWS * MIX_THREADS + tid;
         rslot = rslot + 1 == STAGES ? 0 : rslot + 1;
         uint32_t x0[TT][2], x1[TT][2];
         double xd[TT][2];
@@ -371,14 +376,14 @@ __global__ void __launch_bounds__(256, (TT * PT >= 12 ? 1 : 2)) k_bsgs_accumulat
         for (int i = 0; i < TT; i++)
 #pragma unroll
             for (int p = 0; p < 2; p++) {
-                const u64 v = sm[(2 * i + p) * 256];
+                const u64 v = sm[(2 * i + p) * MIX_THREADS];
                 x0[i][p] = (uint32_t)v;
                 x1[i][p] = (uint32_t)(v >> 32);
                 xd[i][p] = __ull2double_rn(v);       // exact: v < 2^50
             }
 #pragma unroll
         for (int j = 0; j < PT; j++) {
-            const u64 v = sm[(2 * TT + j) * 256];
+            const u64 v = sm[(2 * TT + j) * MIX_THREADS];
             const uint32_t w0 = (uint32_t)v, w1 = (uint32_t)(v >> 32);
             const double wd = __ull2double_rn(v);
 #pragma unroll
@@ -522,11 +527,11 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
         // otherwise 128-bit integer accumulation.  FESC_BSGS_INT=1 forces the integer kernel (for comparisons).
 #define BSGS_MIX(TT, PT, ST)                                                                                  \
     do {                                                                                                      \
-        dim3 grid(((bp_count + PT - 1) / PT) * ((nt + TT - 1) / TT), N / 256, level);                         \
-        const size_t smem = (size_t)ST * (2 * TT + PT) * 2048;                                                \
+        dim3 grid(((bp_count + PT - 1) / PT) * ((nt + TT - 1) / TT), N / MIX_THREADS, level);                 \
+        const size_t smem = (size_t)ST * (2 * TT + PT) * MIX_THREADS * 8;                                     \
         auto kern = k_bsgs_accumulate_mixed<TT, PT, ST>;                                                      \
         FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        kern<<<grid, 256, smem, st>>>(rot, diags, acc, ctx->d_pc, N, level, nt, gin * n1, bp_count);          \
+        kern<<<grid, MIX_THREADS, smem, st>>>(rot, diags, acc, ctx->d_pc, N, level, nt, gin * n1, bp_count);  \
     } while (0)
         const bool fp_ok = qbits <= 50 && bsgs_kernel() != 2;
         if (fp_ok && bsgs_kernel() == 0 && N % 256 == 0 && nt >= 2 && gin * n1 <= 256) BSGS_MIX(2, 8, 3);
