@@ -51,7 +51,10 @@ broadcast takes them from class g, i.e. from the group ciphertext rotated by (g 
 
 the 2(G-1) rotations by +-unit..+-(G-1) unit are taken ONCE per group (one decomposition in hoisted mode) and every
 token is G plaintext multiply-accumulates and one rescale (no copy leaves its period, so nothing crosses a channel or
-head boundary).  The class masks cost one level: br(B_t) is brought to l0-2 before its fill, leaves at l1 = l0-3.
+head boundary).  The class masks cost one level: leaves at l1 = l0-3.  br(B_t) is built the same way (groups of G
+tokens = G d_s consecutive slots, mask [0, G d_s), log2(n/(G d_s)) steps, class shifts of d_s slots), which lands it
+at l0-2 where the leaves need it; br(C_t) keeps the token-by-token build (its fill runs at the injection level, where
+rotations are cheap).
 
 Other prefix networks (App. "Prefix-Network Selection"; `network` = "ks" Kogge-Stone, "sk" Sklansky; "bk" above is the
 default): stage s = 1..logB combines operands at l1-(s-1) into results at l1-s, every prefix is complete at lS and there
@@ -141,8 +144,15 @@ class ScanShape:
             if hoist:                                                                      # radix-4 group fills
                 for unit, steps in ((-G, int(math.log2(self.d_s // G))), (-G * self.P, int(math.log2(self.R // (G * self.P))))):
                     am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
-            for unit in (1, self.P):
+            for unit in (1, self.P, self.d_s):
                 am |= {v % n for v in self.class_shifts(G, unit)}
+            cntB = B // G                                                                  # groups of br(B)
+            dgB = min(16, cntB)
+            unit = G * self.d_s
+            am |= {unit * t % n for t in range(1, dgB)} | {unit * dgB * t % n for t in range(1, cntB // dgB)}
+            if hoist:
+                am |= {(-3 * unit * (1 << b)) % n for b in range(0, int(math.log2(n // unit)) - 1, 2)}
+            am |= {(-unit * (1 << b)) % n for b in range(int(math.log2(n // unit)))}
         am.discard(0)
         return sorted(am)
 
@@ -199,6 +209,9 @@ class ScanConsts:
             self.mask_x2 = np.stack([orc.encode(((in_stride < d_s) & (in_stride % G == g)).astype(float),
                                                 self.S_p[l0 - 1], l0 - 1) for g in range(G)])
             self.mask_a2 = np.stack([orc.encode(((in_region // P) % G == g).astype(float), self.S_p[l0 - 1], l0 - 1)
+                                     for g in range(G)])
+            self.mask_bg = orc.encode((slot < G * d_s).astype(float), self.S_p[l0], l0)
+            self.mask_b2 = np.stack([orc.encode(((slot // d_s) % G == g).astype(float), self.S_p[l0 - 1], l0 - 1)
                                      for g in range(G)])
         lred, lout = self.lv["linj"] - 2, self.lv["lout"]
         # the unpacked reduction carries a factor 2 (Re*2, Im*2); the output mask removes it and lands on S_s[lout]
@@ -408,6 +421,17 @@ class ScanEvaluator:
             out.append(self.fill_right(u, sh.stride, int(math.log2(sh.c_state))))
         return out
 
+    def broadcast_b_grouped(self, ct):
+        """br(B_t) for every token of the block at l0-2, built for groups of G tokens (module header)."""
+        sh, c, G = self.sh, self.c, self.group
+        unit = G * sh.d_s
+        ex = self.extract_all(ct, unit, sh.B // G)
+        out = []
+        for u in range(sh.B // G):
+            gb = self.fill_right(self.ptmul_rescale(ex[u], c.mask_bg), unit, int(math.log2(sh.n // unit)))
+            out += self.class_broadcasts(gb, c.mask_b2, sh.d_s)
+        return out
+
     def leaves(self, ctX, ctA, brB):
         """ctX, ctA: the `segs` ciphertexts of one (block, chunk), segment g holding the tokens g*Bt .. (g+1)*Bt-1."""
         sh, c = self.sh, self.c
@@ -501,7 +525,7 @@ class ScanEvaluator:
         out = np.zeros((sh.K_blk, sh.K_s, sh.segs, 2, lout, o.N), dtype=np.uint64)
         carry = [None] * sh.K_s                       # g_j per chunk: the state before block j
         for j in range(sh.K_blk):
-            brB = self.broadcast_bc(ctB[j], lv["l0"] - 2 if self.group else None)
+            brB = self.broadcast_b_grouped(ctB[j]) if self.group else self.broadcast_bc(ctB[j])
             brC = self.broadcast_bc(ctC[j], linj - 1)
             v = [[None] * sh.K_s for _ in range(sh.B)]
             for kap in range(sh.K_s):

@@ -192,8 +192,12 @@ def test_grouped_leaf_build():
     B, G, P, R, d_s = sh.B, 4, sh.P, sh.R, sh.d_s
     plain = 2 * (B - 1) + B * (lg(d_s) + lg(R // P))
     grouped = 2 * (B // G - 1) + (B // G) * (lg(d_s // G) + lg(R // (G * P))) + 2 * (B // G) * 2 * (G - 1)
-    assert ev0.count["rot"] - ev.count["rot"] == sh.K_blk * sh.K_s * (plain - grouped) == 912
-    assert ev.count["ptmul"] - ev0.count["ptmul"] == sh.K_blk * sh.K_s * (2 * (B // G) + 2 * B * G - 2 * B)
+    # br(B) of every block (shared by the chunks) is built in groups too
+    plain_b = (B - 1) + B * lg(sh.c_state)
+    grouped_b = (B // G - 1) + (B // G) * lg(sh.n // (G * d_s)) + (B // G) * 2 * (G - 1)
+    assert ev0.count["rot"] - ev.count["rot"] == sh.K_blk * (sh.K_s * (plain - grouped) + plain_b - grouped_b) == 996
+    assert ev.count["ptmul"] - ev0.count["ptmul"] == sh.K_blk * (sh.K_s * (2 * (B // G) + 2 * B * G - 2 * B)
+                                                                 + B // G + B * G - B)
     # the rotated copy kept for the class difference k = g - j is the rotation by k units
     for G in (2, 4, 8):
         shifts = sh.class_shifts(G, 3)
