@@ -593,8 +593,14 @@ def scan_rotation_amounts(n, P, d_s, B, stride, hoist=False, group=0):
         if hoist:
             for unit, steps in ((-group, int(math.log2(d_s // group))), (-group * P, int(math.log2(R // (group * P))))):
                 am |= {(3 * unit * (1 << b)) % n for b in range(0, steps - 1, 2)}
-        for unit in (1, P):
+        for unit in (1, P, d_s):
             am |= {(k * unit) % n for k in range(1, group)} | {(-k * unit) % n for k in range(1, group)}
+        cnt_b, unit = B // group, group * d_s                   # br(B): groups of `group` tokens = unit slots
+        dg_b = min(16, cnt_b)
+        am |= {unit * t % n for t in range(1, dg_b)} | {unit * dg_b * t % n for t in range(1, cnt_b // dg_b)}
+        am |= {(-unit * (1 << b)) % n for b in range(int(math.log2(n // unit)))}
+        if hoist:
+            am |= {(-3 * unit * (1 << b)) % n for b in range(0, int(math.log2(n // unit)) - 1, 2)}
     am.discard(0)
     return sorted(am)
 
@@ -688,7 +694,9 @@ def run_scan(args):
         gm = [S.hashed_residues(seed, 20, q, N, device=dev).contiguous(),
               S.hashed_residues(seed, 21, q, N, device=dev).contiguous(),
               S.hashed_residues(seed, 22, q[:l0 - 1], G * N, device=dev).view(l0 - 1, G, N).permute(1, 0, 2).contiguous(),
-              S.hashed_residues(seed, 23, q[:l0 - 1], G * N, device=dev).view(l0 - 1, G, N).permute(1, 0, 2).contiguous()]
+              S.hashed_residues(seed, 23, q[:l0 - 1], G * N, device=dev).view(l0 - 1, G, N).permute(1, 0, 2).contiguous(),
+              S.hashed_residues(seed, 24, q, N, device=dev).contiguous(),
+              S.hashed_residues(seed, 25, q[:l0 - 1], G * N, device=dev).view(l0 - 1, G, N).permute(1, 0, 2).contiguous()]
     out = torch.empty((K_blk, max(mine, 1), segs, 2, linj - 3, N), dtype=torch.int64, device=dev)
     adj = [(1 << 49) + 12345 * i for i in range((l0 + 1) ** 2)]
     desc = fesc.ScanDesc(L, mine * hpc, P, d_s, B, stride, l0, base, int(args.hoist), net, G)

@@ -49,7 +49,7 @@ class ScanDesc(ctypes.Structure):
 
 class ScanConsts(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("d_mask_x", "d_mask_b", "d_mask_a", "d_mask_out", "adj_s", "adj_p",
-                                               "d_mask_xg", "d_mask_ag", "d_mask_x2", "d_mask_a2")]
+                                               "d_mask_xg", "d_mask_ag", "d_mask_x2", "d_mask_a2", "d_mask_bg", "d_mask_b2")]
 
 
 def lib():
@@ -249,12 +249,12 @@ class Context:
     def scan_contract(self, x, a, B, C, desc: ScanDesc, mask_x, mask_b, mask_a, mask_out, adj_s, adj_p, m_out,
                       group_masks=None):
         """adj_s / adj_p: sequences of (n_limbs+1)^2 Python ints (host tables); masks: CUDA tensors;
-        group_masks = (mask_xg, mask_ag, mask_x2, mask_a2) for desc.group > 0."""
+        group_masks = (mask_xg, mask_ag, mask_x2, mask_a2, mask_bg, mask_b2) for desc.group > 0."""
         n = (desc.n_limbs + 1) ** 2
         hs = (ctypes.c_uint64 * n)(*[int(v) for v in adj_s])
         hp = (ctypes.c_uint64 * n)(*[int(v) for v in adj_p])
         cs = ScanConsts(mask_x.data_ptr(), mask_b.data_ptr(), mask_a.data_ptr(), mask_out.data_ptr(),
                         ctypes.cast(hs, ctypes.c_void_p).value, ctypes.cast(hp, ctypes.c_void_p).value,
-                        *([t.data_ptr() for t in group_masks] if group_masks else [None] * 4))
+                        *([t.data_ptr() for t in group_masks] if group_masks else [None] * 6))
         self._chk(lib().fesc_scan_contract(self.h, _ptr(x), _ptr(a), _ptr(B), _ptr(C), ctypes.byref(desc),
                                            ctypes.byref(cs), _ptr(m_out), _stream()))

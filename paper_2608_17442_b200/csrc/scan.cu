@@ -391,15 +391,23 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
         for (int which = 0; which < 2; which++) {
             size_t m = X.top;
             Arr src{const_cast<u64*>((which ? d_C : d_B) + (size_t)j * in_ctw), 1, l0, in_ctw};
+            if (which == 0 && G) {
+                // br(B_t) for groups of G tokens (G d_s consecutive slots): one extraction, mask and fill per group,
+                // then every token as a masked sum of the group's rotations by multiples of d_s; lands at l0-2
+                const uint32_t ng = B / G, unit = G * g.d_s;
+                Arr exg = X.alloc(ng, l0), gb = X.alloc(ng, l0 - 1);
+                X.extract_n(src, unit, ng, exg);
+                X.ptmul_rescale(exg, (const u64*)X.cs->d_mask_bg, gb);
+                X.fill_right(gb, unit, ilog2(g.n / unit));
+                X.class_broadcasts(gb, (const u64*)X.cs->d_mask_b2, G, g.d_s,
+                                   [&](uint32_t c, const Arr& res) { X.copy(res, X.strided(brB, c, G, ng)); });
+                X.top = m;
+                continue;
+            }
             Arr ex = X.alloc(B, l0);
             X.extract_all(src, g.d_s, ex);
-            if (which == 0 && !G) {
+            if (which == 0) {
                 X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_b, brB);
-                X.fill_right(brB, g.stride, ilog2(g.c_state));
-            } else if (which == 0) {
-                Arr full = X.alloc(B, l0 - 1);
-                X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_b, full);
-                X.adjust(full, lB, 1, brB);
                 X.fill_right(brB, g.stride, ilog2(g.c_state));
             } else {
                 // br(C) is only needed at the injection level: bring it down first, fill there (cheap rotations)
@@ -658,8 +666,9 @@ extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint
     if (G) {
         if (G < 2 || (G & (G - 1)) || G > g.Bt || G > g.d_s)
             return fesc_fail(ctx, FESC_EINVAL, "scan_contract: group must be a power of two, at most the tokens of a segment and d_s");
-        if (!consts->d_mask_xg || !consts->d_mask_ag || !consts->d_mask_x2 || !consts->d_mask_a2)
-            return fesc_fail(ctx, FESC_EINVAL, "scan_contract: the grouped leaf build needs its four mask arrays");
+        if (!consts->d_mask_xg || !consts->d_mask_ag || !consts->d_mask_x2 || !consts->d_mask_a2 || !consts->d_mask_bg ||
+            !consts->d_mask_b2)
+            return fesc_fail(ctx, FESC_EINVAL, "scan_contract: the grouped leaf build needs its six mask arrays");
     }
     if (g.l0 > ctx->n_q || g.l0 < g.logB + below_summary + 6 + (G ? 1 : 0))
         return fesc_fail(ctx, FESC_ELEVEL, "scan_contract: not enough levels");

@@ -32,7 +32,7 @@ def _run(name, hoist=0, network="bk", group=0, **kw):
     out = torch.empty((sh.K_blk, sh.K_s, sh.segs, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
     desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, kw.get("stride", 0), l0, 100000, hoist,
                          {"bk": fesc.NET_BRENT_KUNG, "ks": fesc.NET_KOGGE_STONE, "sk": fesc.NET_SKLANSKY}[network], group)
-    gm = [to_dev(m) for m in (c.mask_xg, c.mask_ag, c.mask_x2, c.mask_a2)] if group else None
+    gm = [to_dev(m) for m in (c.mask_xg, c.mask_ag, c.mask_x2, c.mask_a2, c.mask_bg, c.mask_b2)] if group else None
     ctx.scan_contract(to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
                       to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out, gm)
     ctx.sync()
@@ -92,7 +92,7 @@ def test_scan_unknown_network_is_refused():
     with pytest.raises(fesc.FescError) as e:
         ctx.scan_contract(z, z, z, z, desc, z, z, z, z, [0], [0], z)
     assert e.value.code == fesc.EINVAL
-    for group, masks in ((3, (z, z, z, z)), (8, (z, z, z, z)), (2, None)):      # not a power of two; above d_s; no masks
+    for group, masks in ((3, (z,) * 6), (8, (z,) * 6), (2, None)):      # not a power of two; above d_s; no masks
         desc = fesc.ScanDesc(4, 2, 4, 2, 4, 0, p["n_q"], 100000, 0, 0, group)
         with pytest.raises(fesc.FescError) as e:
             ctx.scan_contract(z, z, z, z, desc, z, z, z, z, [0], [0], z, masks)
@@ -136,7 +136,7 @@ def test_scan_deployed_geometry_decrypts_to_recurrence(hoist, group, stride, l0)
     adj_p = [c.adj_p.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
     out = torch.empty((sh.K_blk, sh.K_s, sh.segs, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
     desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, sh.stride, l0, 100000, hoist, 0, group)
-    gm = [to_dev(m) for m in (c.mask_xg, c.mask_ag, c.mask_x2, c.mask_a2)] if group else None
+    gm = [to_dev(m) for m in (c.mask_xg, c.mask_ag, c.mask_x2, c.mask_a2, c.mask_bg, c.mask_b2)] if group else None
     args = (to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
             to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out, gm)
     ks0 = ctx.counters()[1]
