@@ -86,6 +86,31 @@ __global__ void __launch_bounds__(256) k_ct_sum_into(const u64* __restrict__ a, 
     acc[o] = s;
 }
 
+// out[b] = sum_{j<terms} src_j[b] (.) mask_j on both polynomials (mask_j = masks + j*level*N, shared by the batch);
+// the products are summed in 128 bits and reduced once
+struct ClassSources {
+    const u64* src[16];
+};
+__global__ void __launch_bounds__(256) k_class_mac(ClassSources s, uint32_t terms, size_t src_stride,
+                                                   const u64* __restrict__ masks, u64* __restrict__ out,
+                                                   size_t out_stride, const PrimeConst* __restrict__ pcs, uint32_t N,
+                                                   uint32_t level) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t l = blockIdx.y, b = blockIdx.z;
+    if (c >= N) return;
+    const PrimeConst pc = pcs[l];
+    const size_t poly = (size_t)level * N, o = (size_t)l * N + c;
+    acc128 a0{0, 0}, a1{0, 0};
+    for (uint32_t j = 0; j < terms; j++) {
+        const u64 w = masks[(size_t)j * poly + o];
+        const u64* x = s.src[j] + (size_t)b * src_stride;
+        mac128(a0, x[o], w);
+        mac128(a1, x[poly + o], w);
+    }
+    out[(size_t)b * out_stride + o] = reduce128(a0.hi, a0.lo, pc);
+    out[(size_t)b * out_stride + poly + o] = reduce128(a1.hi, a1.lo, pc);
+}
+
 // ---------------------------------------------------------------------------------------
 // host-side sequencing
 // ---------------------------------------------------------------------------------------
@@ -313,7 +338,6 @@ struct Exec {
     void class_broadcasts(const Arr& grp, const u64* masks, uint32_t G, uint32_t unit, F deliver) {
         size_t mark = top;
         const uint32_t nk = 2 * (G - 1), cnt = grp.count, lvl = grp.level;
-        const size_t mask_words = (size_t)lvl * N;
         Arr rots = alloc(nk * cnt, lvl);       // [shift][group]
         std::vector<int64_t> shifts;
         for (uint32_t k = 1; k < G; k++) shifts.push_back((int64_t)k * unit);
@@ -331,15 +355,15 @@ struct Exec {
         Arr acc = alloc(cnt, lvl), res = alloc(cnt, lvl - 1);
         for (uint32_t c = 0; c < G && ok(); c++) {
             if (!dry) {
-                cudaError_t e = cudaMemsetAsync(acc.p, 0, (size_t)cnt * ctw(lvl) * sizeof(u64), st);
-                if (e != cudaSuccess) rc = fesc_fail(ctx, FESC_ECUDA, cudaGetErrorString(e));
-                for (uint32_t j = 0; j < G && ok(); j++) {
+                ClassSources cs_;
+                for (uint32_t j = 0; j < G; j++) {
                     const int k = (int)c - (int)j;
-                    const Arr src = k == 0 ? grp : at(rots, (uint32_t)(k > 0 ? k - 1 : (int)G - 2 - k) * cnt, cnt);
-                    // the public multiply-accumulate takes a contiguous batch; group ciphertexts are contiguous
-                    rc = fesc_ct_pt_mac(ctx, (const uint64_t*)src.p, (const uint64_t*)(masks + j * mask_words), 0,
-                                        (uint64_t*)acc.p, cnt, lvl, (void*)st);
+                    cs_.src[j] = k == 0 ? grp.p : rots.p + (size_t)(k > 0 ? k - 1 : (int)G - 2 - k) * cnt * rots.stride;
                 }
+                prof_begin(ctx, PF_POINTWISE, st);
+                k_class_mac<<<grid(lvl, cnt), 256, 0, st>>>(cs_, G, grp.stride, masks, acc.p, acc.stride, ctx->d_pc, N, lvl);
+                prof_end(ctx, PF_POINTWISE, st);
+                ctx->counters[2] += (uint64_t)G * cnt;
             }
             rescale(acc, res);
             deliver(c, res);
@@ -664,8 +688,8 @@ extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint
         desc->network == FESC_NET_BRENT_KUNG ? g.logB - 1 : (g.K_blk > 2 ? g.K_blk - 2 : 0);   // lS - linj
     const uint32_t G = desc->group;
     if (G) {
-        if (G < 2 || (G & (G - 1)) || G > g.Bt || G > g.d_s)
-            return fesc_fail(ctx, FESC_EINVAL, "scan_contract: group must be a power of two, at most the tokens of a segment and d_s");
+        if (G < 2 || (G & (G - 1)) || G > 16 || G > g.Bt || G > g.d_s)
+            return fesc_fail(ctx, FESC_EINVAL, "scan_contract: group must be a power of two, at most 16, the tokens of a segment and d_s");
         if (!consts->d_mask_xg || !consts->d_mask_ag || !consts->d_mask_x2 || !consts->d_mask_a2 || !consts->d_mask_bg ||
             !consts->d_mask_b2)
             return fesc_fail(ctx, FESC_EINVAL, "scan_contract: the grouped leaf build needs its six mask arrays");
