@@ -46,3 +46,38 @@ def random_ct(orc, seed: int, stream: int, level: int, batch: int) -> np.ndarray
         for p in range(2):
             out[b, p] = S.uniform_residues_np(seed, stream * 4096 + b * 2 + p, orc.q[:level], orc.N)
     return out
+
+
+def run_scan_parity(name, hoist=0, network="bk", group=0, **kw):
+    """fesc_scan_contract against ScanEvaluator.run on the named parameter set and shape: asserts that every output
+    residue is equal and returns the largest deviation of the decrypted result from the float64 recurrence."""
+    import torch
+    import fesc_synth as S
+    import paper_2608_17442_b200 as fesc
+    from oracle.ckks import CONJ
+    from oracle.scan import (ScanConsts, ScanEvaluator, ScanShape, add_scan_keys, encrypt_inputs, float_recurrence,
+                             key_id_for, unpack_output)
+
+    ctx, orc, p = ctx_pair(name)
+    sh = ScanShape(orc.n, **kw)
+    l0 = p["n_q"]
+    x, a, B, C = S.scan_inputs(p["seed"] + sh.L, sh.L, sh.H, sh.P, 1, sh.d_s)
+    c = ScanConsts(orc, sh, l0, p["log_scale"], network, group)
+    add_scan_keys(orc, sh, hoist=bool(hoist), group=group)
+    for r in sh.rotation_amounts(bool(hoist), group) + [CONJ]:
+        ctx.add_galois_key(r, key_id_for(sh, r))
+    ctX, ctA, ctB, ctC = encrypt_inputs(orc, sh, c, x, a, B, C)
+    want = ScanEvaluator(orc, sh, c, hoist=bool(hoist)).run(ctX, ctA, ctB, ctC)
+    adj_s = [c.adj_s.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
+    adj_p = [c.adj_p.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
+    out = torch.empty((sh.K_blk, sh.K_s, sh.segs, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
+    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, kw.get("stride", 0), l0, 100000, hoist,
+                         {"bk": fesc.NET_BRENT_KUNG, "ks": fesc.NET_KOGGE_STONE, "sk": fesc.NET_SKLANSKY}[network], group)
+    gm = [to_dev(m) for m in (c.mask_xg, c.mask_ag, c.mask_x2, c.mask_a2, c.mask_bg, c.mask_b2)] if group else None
+    ctx.scan_contract(to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
+                      to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out, gm)
+    ctx.sync()
+    got = to_host(out)
+    assert np.array_equal(got, want)
+    m = unpack_output(orc, sh, c, got)
+    return np.abs(m - float_recurrence(x, a, B, C)).max()

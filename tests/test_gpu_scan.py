@@ -8,38 +8,9 @@ import fesc_synth as S
 from oracle.ckks import CONJ
 from oracle.scan import (ScanConsts, ScanEvaluator, ScanShape, add_scan_keys, encrypt_inputs, float_recurrence,
                          key_id_for, unpack_output)
-from tests.gpu_util import ctx_pair, to_dev, to_host
+from tests.gpu_util import ctx_pair, run_scan_parity as _run, to_dev, to_host
 
 pytestmark = pytest.mark.gpu
-
-
-def _run(name, hoist=0, network="bk", group=0, **kw):
-    import torch
-    import paper_2608_17442_b200 as fesc
-
-    ctx, orc, p = ctx_pair(name)
-    sh = ScanShape(orc.n, **kw)
-    l0 = p["n_q"]
-    x, a, B, C = S.scan_inputs(p["seed"] + sh.L, sh.L, sh.H, sh.P, 1, sh.d_s)
-    c = ScanConsts(orc, sh, l0, p["log_scale"], network, group)
-    add_scan_keys(orc, sh, hoist=bool(hoist), group=group)
-    for r in sh.rotation_amounts(bool(hoist), group) + [CONJ]:
-        ctx.add_galois_key(r, key_id_for(sh, r))
-    ctX, ctA, ctB, ctC = encrypt_inputs(orc, sh, c, x, a, B, C)
-    want = ScanEvaluator(orc, sh, c, hoist=bool(hoist)).run(ctX, ctA, ctB, ctC)
-    adj_s = [c.adj_s.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
-    adj_p = [c.adj_p.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
-    out = torch.empty((sh.K_blk, sh.K_s, sh.segs, 2, c.lv["lout"], orc.N), dtype=torch.int64, device="cuda")
-    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, kw.get("stride", 0), l0, 100000, hoist,
-                         {"bk": fesc.NET_BRENT_KUNG, "ks": fesc.NET_KOGGE_STONE, "sk": fesc.NET_SKLANSKY}[network], group)
-    gm = [to_dev(m) for m in (c.mask_xg, c.mask_ag, c.mask_x2, c.mask_a2, c.mask_bg, c.mask_b2)] if group else None
-    ctx.scan_contract(to_dev(ctX), to_dev(ctA), to_dev(ctB), to_dev(ctC), desc, to_dev(c.mask_x), to_dev(c.mask_b),
-                      to_dev(c.mask_a), to_dev(c.mask_out), adj_s, adj_p, out, gm)
-    ctx.sync()
-    got = to_host(out)
-    assert np.array_equal(got, want)
-    m = unpack_output(orc, sh, c, got)
-    return np.abs(m - float_recurrence(x, a, B, C)).max()
 
 
 @pytest.mark.parametrize("hoist", [0, 1])
@@ -116,7 +87,8 @@ def test_scan_deployed_geometry_decrypts_to_recurrence(hoist, group, stride, l0)
     """N = 2^16, 24 limbs, stride 256, B_blk = 256, d_s = 128, P = 64 (the Mamba-2-base geometry) on a slice of
     the model: 4 heads (one chunk pair) and 512 tokens (two blocks, so the carry and its injection run).
     The oracle cannot follow ~36 000 key switches at this ring size, so the check here is the property that
-    holds at any size: the decrypted output equals the float64 recurrence."""
+    holds at any size: the decrypted output equals the float64 recurrence within 2^-18 (|m| <= 1.5).  Residue-level
+    parity on this ring, with a block of 4 tokens, is in test_gpu_scan_full_ring.py."""
     import time
     import torch
     import paper_2608_17442_b200 as fesc
@@ -151,4 +123,4 @@ def test_scan_deployed_geometry_decrypts_to_recurrence(hoist, group, stride, l0)
     err = np.abs(m - ref).max()
     print("scan slice: %d key switches in %.2f s (%.0f /s), scratch %.1f GiB, max err 2^%.2f, max|m| %.2f"
           % (ks, dt, ks / dt, ctx.counters()[3] / 2**30, np.log2(err), np.abs(ref).max()))
-    assert err < 2.0**-16
+    assert err < 2.0**-18
