@@ -31,7 +31,15 @@ class FescError(RuntimeError):
 class BsgsDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint32) for n in
                 ("n1", "n2", "in_blocks", "out_blocks", "token_blocks", "n_limbs", "baby_key_base", "giant_key_base",
-                 "hoist", "defer")]
+                 "hoist", "defer", "packed")]
+
+
+class Info(ctypes.Structure):
+    _fields_ = ([(n, ctypes.c_uint32) for n in ("log_n", "n_q", "n_p", "dnum", "alpha", "digits", "flags", "reserved")]
+                + [("log2_P", ctypes.c_double), ("log2_Qmax", ctypes.c_double)])
+
+
+INFO_KEYSWITCH_NOISE = 1
 
 
 class ConvDesc(ctypes.Structure):
@@ -88,6 +96,10 @@ def lib():
             "fesc_rescale_static": [vp, vp, vp, u32, u32, vp],
             "fesc_ct_ct_mul": [vp, vp, vp, vp, u32, u32, vp],
             "fesc_linear": [vp, vp, vp, c.POINTER(BsgsDesc), vp, vp],
+            "fesc_linear_pack_diags": [vp, vp, c.POINTER(BsgsDesc), u32, u32, vp, vp],
+            "fesc_params_info": [u32, c.POINTER(u64), u32, u32, u32, c.POINTER(Info)],
+            "fesc_ctx_info": [vp, c.POINTER(Info)],
+            "fesc_ctx_test_fail_allocs": [vp, u32],
             "fesc_scan_contract": [vp, vp, vp, vp, vp, c.POINTER(ScanDesc), c.POINTER(ScanConsts), vp, vp],
         }
         for name, args in sig.items():
@@ -96,10 +108,22 @@ def lib():
             f.restype = c.c_int
         L.fesc_last_error.argtypes = [vp]
         L.fesc_last_error.restype = c.c_char_p
+        L.fesc_linear_packed_bytes.argtypes = [vp, c.POINTER(BsgsDesc)]
+        L.fesc_linear_packed_bytes.restype = sz
         L.fesc_ctx_num_digits.argtypes = [vp]
         L.fesc_ctx_num_digits.restype = u32
         _lib = L
     return _lib
+
+
+def params_info(log_n: int, primes, n_q: int, n_p: int, dnum: int) -> Info:
+    """fesc_params_info: derived parameters and flags of a parameter set; runs on the host alone (no GPU needed)."""
+    arr = (ctypes.c_uint64 * len(primes))(*[int(p) for p in primes])
+    out = Info()
+    rc = lib().fesc_params_info(log_n, arr, n_q, n_p, dnum, ctypes.byref(out))
+    if rc != OK:
+        raise FescError(rc, "bad parameter set")
+    return out
 
 
 def _stream():
@@ -244,7 +268,28 @@ class Context:
         self._chk(lib().fesc_ct_ct_mul(self.h, _ptr(a), _ptr(b), _ptr(out), batch, n_limbs, _stream()))
 
     def linear(self, ct_in, diags, desc: BsgsDesc, ct_out):
-        self._chk(lib().fesc_linear(self.h, _ptr(ct_in), _ptr(diags), ctypes.byref(desc), _ptr(ct_out), _stream()))
+        """diags: the residue tensor, or (desc.packed = 1) the uint8 image filled by linear_pack_diags."""
+        assert diags.is_cuda and diags.is_contiguous()
+        self._chk(lib().fesc_linear(self.h, _ptr(ct_in), ctypes.c_void_p(diags.data_ptr()), ctypes.byref(desc),
+                                    _ptr(ct_out), _stream()))
+
+    def linear_packed_bytes(self, desc: BsgsDesc) -> int:
+        return int(lib().fesc_linear_packed_bytes(self.h, ctypes.byref(desc)))
+
+    def linear_pack_diags(self, diags, desc: BsgsDesc, first: int, count: int, packed):
+        """Packs the (b,p) pairs [first, first+count) from `diags` ([count][in_blocks][n1][n_limbs][N] residues) into
+        their place inside the uint8 CUDA tensor `packed` (linear_packed_bytes(desc) bytes)."""
+        assert packed.is_cuda and packed.is_contiguous() and packed.element_size() == 1
+        self._chk(lib().fesc_linear_pack_diags(self.h, _ptr(diags), ctypes.byref(desc), first, count,
+                                               ctypes.c_void_p(packed.data_ptr()), _stream()))
+
+    def info(self) -> Info:
+        out = Info()
+        self._chk(lib().fesc_ctx_info(self.h, ctypes.byref(out)))
+        return out
+
+    def test_fail_allocs(self, count: int):
+        self._chk(lib().fesc_ctx_test_fail_allocs(self.h, count))
 
     def scan_contract(self, x, a, B, C, desc: ScanDesc, mask_x, mask_b, mask_a, mask_out, adj_s, adj_p, m_out,
                       group_masks=None):

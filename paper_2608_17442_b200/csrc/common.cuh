@@ -108,6 +108,39 @@ __device__ __forceinline__ u64 fp_store(double x, double q, double qinv) {
     return (u64)__double_as_longlong(x + 4503599627370496.0) & 0x000FFFFFFFFFFFFFull;
 }
 
+// ---------------------------------------------------------------------------------------
+// Shared-memory barriers and bulk asynchronous copies (every copy targets the issuing CTA only; no multicast).
+// Every wait on a barrier is bounded: it polls a fixed number of times and reports failure instead of spinning.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// returns 0 when the phase completed, 1 when the poll budget ran out
+__device__ __forceinline__ uint32_t mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < (1u << 20); it++) {
+        if (mbar_try_wait(bar, parity)) return 0;
+        if (it > 64) __nanosleep(64);
+    }
+    return 1;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
 // counter-based generator (same public recipe as the header documents)
 __host__ __device__ __forceinline__ u64 mix64(u64 z) {
     z += 0x9E3779B97F4A7C15ull;
@@ -195,6 +228,7 @@ struct fesc_ctx {
     // scratch
     u64* d_scratch;
     size_t scratch_bytes;
+    uint32_t fail_allocs = 0;     // test hook: this many scratch allocations report FESC_ENOMEM
     uint32_t* d_status;           // device word: non-zero after a bounded device-side wait gave up
     uint64_t counters[8];
     Profiler prof;

@@ -135,9 +135,13 @@ int ctx_scratch(fesc_ctx* ctx, size_t bytes, u64** out) {
             cudaFree(ctx->d_scratch);
             ctx->d_scratch = nullptr;
             ctx->scratch_bytes = 0;
+            ctx->counters[3] = 0;
         }
         size_t want = (bytes + (1u << 20) - 1) & ~(size_t)((1u << 20) - 1);
-        if (cudaMalloc(&ctx->d_scratch, want) != cudaSuccess) {
+        const bool injected = ctx->fail_allocs > 0;       // test hook: report the failure without calling the driver
+        if (injected) ctx->fail_allocs--;
+        if (injected || cudaMalloc(&ctx->d_scratch, want) != cudaSuccess) {
+            ctx->d_scratch = nullptr;
             cudaGetLastError();
             return fesc_fail(ctx, FESC_ENOMEM, "scratch allocation of " + std::to_string(want) + " bytes failed");
         }
@@ -423,6 +427,63 @@ extern "C" int fesc_ctx_trim(fesc_ctx* ctx) {
         ctx->scratch_bytes = 0;
         ctx->counters[3] = 0;
     }
+    return FESC_OK;
+}
+
+// product of a list of primes as little-endian 64-bit words (host; exact)
+static std::vector<u64> h_product(const uint64_t* p, uint32_t first, uint32_t count) {
+    std::vector<u64> v(1, 1);
+    for (uint32_t i = 0; i < count; i++) {
+        u64 carry = 0;
+        for (size_t w = 0; w < v.size(); w++) {
+            const u128 t = (u128)v[w] * p[first + i] + carry;
+            v[w] = (u64)t;
+            carry = (u64)(t >> 64);
+        }
+        if (carry) v.push_back(carry);
+    }
+    return v;
+}
+static bool h_less(const std::vector<u64>& a, const std::vector<u64>& b) {
+    if (a.size() != b.size()) return a.size() < b.size();
+    for (size_t w = a.size(); w-- > 0;)
+        if (a[w] != b[w]) return a[w] < b[w];
+    return false;
+}
+
+extern "C" int fesc_params_info(uint32_t log_n, const uint64_t* primes, uint32_t n_q, uint32_t n_p, uint32_t dnum,
+                                fesc_info* out) {
+    if (!out || !primes || n_q == 0 || n_p == 0 || dnum == 0 || n_q + n_p > FESC_MAX_PRIMES || n_p > FESC_MAX_SPECIAL)
+        return FESC_EINVAL;
+    memset(out, 0, sizeof(*out));
+    out->log_n = log_n;
+    out->n_q = n_q;
+    out->n_p = n_p;
+    out->dnum = dnum;
+    out->alpha = (n_q + dnum - 1) / dnum;
+    out->digits = (n_q + out->alpha - 1) / out->alpha;
+    const std::vector<u64> P = h_product(primes, n_q, n_p);
+    for (uint32_t i = 0; i < n_p; i++) out->log2_P += log2((double)primes[n_q + i]);
+    bool noisy = false;
+    for (uint32_t j = 0; j < out->digits; j++) {
+        const uint32_t first = j * out->alpha, cnt = n_q - first < out->alpha ? n_q - first : out->alpha;
+        double lg = 0;
+        for (uint32_t i = 0; i < cnt; i++) lg += log2((double)primes[first + i]);
+        if (lg > out->log2_Qmax) out->log2_Qmax = lg;
+        if (h_less(P, h_product(primes, first, cnt))) noisy = true;
+    }
+    if (noisy) out->flags |= FESC_INFO_KEYSWITCH_NOISE;
+    return FESC_OK;
+}
+
+extern "C" int fesc_ctx_info(const fesc_ctx* ctx, fesc_info* out) {
+    if (!ctx) return FESC_EINVAL;
+    return fesc_params_info(ctx->log_n, (const uint64_t*)ctx->q.data(), ctx->n_q, ctx->n_p, ctx->dnum, out);
+}
+
+extern "C" int fesc_ctx_test_fail_allocs(fesc_ctx* ctx, uint32_t count) {
+    if (!ctx) return FESC_EINVAL;
+    ctx->fail_allocs = count;
     return FESC_OK;
 }
 

@@ -415,28 +415,167 @@ __global__ void __launch_bounds__(MIX_THREADS, (TT * PT >= 12 ? 256 / MIX_THREAD
         }
 }
 
+// Tensor-core accumulate for primes below 2^56 (at most 256 terms).  For one coefficient of one limb the sums
+//   S[tb,p][bp] = sum_t x_t[tb,p] * w_t[bp]
+// are a small dense integer matrix product over the terms.  Every residue is cut into 7 bytes; the byte planes
+// form u8 matrices and  S = sum_{k,j} 256^(k+j) D[k][j],  D[k][j] = sum_t w_t.byte(k) * x_t.byte(j),  where each
+// D is an exact s32 accumulator of mma.sync m16n8k32 (u8 x u8): 256 terms of 255^2 stay below 2^24.
+// Mapping: a warp owns ONE coefficient; M side = 8 (b,p) outputs x 2 byte planes per 16-row tile (4 tiles, the
+// last one half empty), N side = 8 (token block, polynomial) columns x 1 byte plane per 8-column tile (7 tiles),
+// K = 32 terms per instruction.  With that mapping lane (g, tg) ends up holding all 49 byte-plane sums of output
+// bp = g for token block tg and both polynomials, so the recombination needs no exchange between lanes.
+// A CTA = 8 warps = 8 neighbouring coefficients of one limb, 4 token blocks and ALL (b,p) outputs: the rotated
+// inputs of its coefficients stay in shared memory for the whole CTA, the diagonals stream through an 8-stage
+// cp.async ring (4 stages when more than 128 terms leave less room) (32 terms x 8 outputs x 8 coefficients per stage), every operand word is read from HBM once per
+// launch.  Fragments are built in registers from the raw 64-bit words: four words of consecutive terms are
+// byte-transposed with 15 byte permutes into the seven 4-term registers the instruction expects.
+// Recombination: E_d = sum_{k+j=d} D[k][j] (13 values below 2^27), groups of four E_d are packed exactly into
+// doubles T_m < 2^52, and S mod q = T_0 + T_1 2^32 + T_2 2^64 + T_3 2^96 mod q with exact FP64 products (primes below
+// 2^50) or as a 128-bit integer followed by the usual reduction (primes of 50..55 bits).
+#define IM_CW 8
+#define IM_ROWP 9                      // words per (row, 8 coefficients): one word of padding
+#define IM_BPP (32 * IM_ROWP + 1)      // words between the (b,p) blocks of a stage (= 1 mod 16: conflict-free fragment loads)
+#define IM_STAGE_WORDS (8 * IM_BPP)
+
+__device__ __forceinline__ void cp_async8z(uint32_t smem_dst, const void* gmem_src, bool valid) {
+    const uint32_t n = valid ? 8u : 0u;      // 0 source bytes: the destination is filled with zeros
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(smem_dst), "l"(gmem_src), "r"(n) : "memory");
+}
+
+template <bool FP, int IM_STAGES>
+__global__ void __launch_bounds__(32 * IM_CW, 1) k_bsgs_accumulate_imma(
+    const u64* __restrict__ rot, const u64* __restrict__ diags, u64* __restrict__ acc,
+    const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level, uint32_t tbs, uint32_t terms, uint32_t bp_count,
+    uint32_t xs_pitch) {
+    extern __shared__ __align__(16) u64 stage[];      // x: [8 (tb,p)][xs_pitch], then IM_STAGES x [8 (b,p)][IM_BPP]
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tg = lane & 3;
+    const uint32_t c0 = blockIdx.x * IM_CW, l = blockIdx.y, tb0 = blockIdx.z * 4;
+    const PrimeConst pc = pcs[l];
+    const size_t poly = (size_t)level * N, ctw = 2 * poly;
+    const uint32_t ksteps = (terms + 31) >> 5, bp_tiles = (bp_count + 7) >> 3, total = ksteps * bp_tiles;
+    const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(stage);
+    const uint32_t cw = tid & 7, rw = tid >> 3;       // word of a row, row of a pass (32 rows per pass)
+    const size_t goff = (size_t)l * N + c0 + cw;
+    // rotated inputs of the CTA's coefficients: rows (tb,p) x terms, zero beyond `terms`
+    {
+        const uint32_t tp = ksteps << 5;
+#pragma unroll 1
+        for (uint32_t tbp = 0; tbp < 8; tbp++) {
+            const uint32_t tb = tb0 + (tbp >> 1) < tbs ? tb0 + (tbp >> 1) : tbs - 1;
+            const u64* src = rot + goff + (size_t)tb * terms * ctw + (tbp & 1) * poly + (size_t)rw * ctw;
+            uint32_t dst = sm_base + (tbp * xs_pitch + rw * IM_ROWP + cw) * 8;
+#pragma unroll 1
+            for (uint32_t t = rw; t < tp; t += 32) {
+                cp_async8z(dst, t < terms ? src : rot, t < terms);
+                src += 32 * ctw;
+                dst += 32 * IM_ROWP * 8;
+            }
+        }
+        cp_async_commit();
+    }
+    // diagonals: a ring of stages, one stage = 32 terms x 8 outputs; this thread copies word cw of term rw of each output
+    const size_t bp_stride = (size_t)terms * poly;
+    const u64* ld_src = diags + goff + (size_t)rw * poly;     // output 0 of the tile to request, term rw of its k-step
+    uint32_t ld_ks = 0, ld_left = bp_count;                   // outputs from the requested tile on
+    uint32_t ld_dst = sm_base + (8 * xs_pitch + rw * IM_ROWP + cw) * 8;
+    const uint32_t ring_end = sm_base + (8 * xs_pitch + IM_STAGES * IM_STAGE_WORDS) * 8;
+    auto issue = [&]() {
+        const bool valid = (ld_ks << 5) + rw < terms;
+        const u64* src = valid ? ld_src : diags;
+        const uint32_t last = ld_left < 8 ? ld_left - 1 : 7;   // a partial tile repeats its last output
+#pragma unroll
+        for (uint32_t i = 0; i < 8; i++) cp_async8z(ld_dst + i * (IM_BPP * 8), src + (i < last ? i : last) * bp_stride, valid);
+        ld_src += 32 * poly;
+        if (++ld_ks == ksteps) {
+            ld_ks = 0;
+            ld_src += 8 * bp_stride - (size_t)ksteps * 32 * poly;
+            ld_left -= 8;
+        }
+        ld_dst += IM_STAGE_WORDS * 8;
+        if (ld_dst >= ring_end) ld_dst -= IM_STAGES * IM_STAGE_WORDS * 8;
+    };
+    for (uint32_t s = 0; s < IM_STAGES - 1; s++) {
+        if (s < total) issue();
+        cp_async_commit();
+    }
+    // constants of the recombination
+    const double q = pc.qd, qinv = pc.qinvd;
+    double c32 = 0, c64 = 0, c96 = 0;
+    if (FP) {
+        c32 = fp_reduce(4294967296.0, q, qinv);
+        c64 = fp_modmul(c32, c32, q, qinv);
+        c96 = fp_modmul(c64, c32, q, qinv);
+    }
+    int d[4][7][4];
+    const u64* a_ring = stage + 8 * xs_pitch + g * IM_BPP + (4 * tg) * IM_ROWP + warp;
+    const u64* b_frag = stage + g * xs_pitch + (4 * tg) * IM_ROWP + warp;
+    uint32_t slot = 0, s = 0;
+#pragma unroll 1
+    for (uint32_t bt = 0; bt < bp_tiles; bt++) {
+#pragma unroll 1
+        for (uint32_t ks = 0; ks < ksteps; ks++, s++) {
+            cp_async_wait<IM_STAGES - 2>();
+            __syncthreads();                  // stage s has landed for everyone; the slot of stage s-1 is free
+            if (s + IM_STAGES - 1 < total) issue();
+            cp_async_commit();
+            uint32_t fa[2][7], fb[2][7];
+            const u64* A = a_ring + slot * IM_STAGE_WORDS;
+            const u64* X = b_frag + (ks << 5) * IM_ROWP;
+#pragma unroll
+            for (int h = 0; h < 2; h++) {
+                byte_planes4(A[(16 * h) * IM_ROWP], A[(16 * h + 1) * IM_ROWP], A[(16 * h + 2) * IM_ROWP],
+                             A[(16 * h + 3) * IM_ROWP], fa[h]);
+                byte_planes4(X[(16 * h) * IM_ROWP], X[(16 * h + 1) * IM_ROWP], X[(16 * h + 2) * IM_ROWP],
+                             X[(16 * h + 3) * IM_ROWP], fb[h]);
+            }
+            slot = slot + 1 == IM_STAGES ? 0 : slot + 1;
+            if (ks == 0) {                    // the first k-step of a tile starts from zero accumulators
+#pragma unroll
+                for (int m = 0; m < 4; m++)
+#pragma unroll
+                    for (int j = 0; j < 7; j++)
+                        imma_u8_zero(d[m][j], fa[0][2 * m], m < 3 ? fa[0][2 * m + 1] : 0u, fa[1][2 * m],
+                                     m < 3 ? fa[1][2 * m + 1] : 0u, fb[0][j], fb[1][j]);
+            } else {
+#pragma unroll
+                for (int m = 0; m < 4; m++)
+#pragma unroll
+                    for (int j = 0; j < 7; j++)
+                        imma_u8(d[m][j], fa[0][2 * m], m < 3 ? fa[0][2 * m + 1] : 0u, fa[1][2 * m],
+                                m < 3 ? fa[1][2 * m + 1] : 0u, fb[0][j], fb[1][j]);
+            }
+        }
+        // recombine: lane (g, tg) holds output bp = 8 bt + g of token block tb0 + tg, both polynomials
+        const uint32_t bp = bt * 8 + g, tb = tb0 + tg;
+        const bool live = bp < bp_count && tb < tbs;
+        u64* dst = acc + ((size_t)(live ? tb : 0) * bp_count + (live ? bp : 0)) * ctw + (size_t)l * N + c0 + warp;
+        if (live) {
+            dst[0] = imma_recombine<FP>(d, 0, pc, c32, c64, c96);
+            dst[poly] = imma_recombine<FP>(d, 1, pc, c32, c64, c96);
+        }
+    }
+    cp_async_wait<0>();
+}
+
 // Knobs for experiments.  FESC_BSGS_KERNEL picks the accumulate kernel: "int" the 128-bit integer one, "fp" the
-// exact-FP64 one, anything else the default (mixed-pipe where it applies).  FESC_BSGS_GROUP_GIB fixes the scratch
+// exact-FP64 one, "mixed" the mixed-pipe one, anything else the default (tensor-core byte planes where they apply).  FESC_BSGS_GROUP_GIB fixes the scratch
 // budget that decides how many token blocks are processed per group (default: from the free device memory).
 static int bsgs_kernel() {
     static int v = -1;
     if (v < 0) {
         const char* e = getenv("FESC_BSGS_KERNEL");
-        v = !e ? 0 : (!strcmp(e, "int") ? 2 : (!strcmp(e, "fp") ? 1 : 0));
+        v = !e ? 0 : (!strcmp(e, "int") ? 2 : (!strcmp(e, "fp") ? 1 : (!strcmp(e, "mixed") ? 3 : 0)));
     }
     return v;
 }
 // Larger groups re-read the diagonals less often and give the key-switch kernels larger batches; every token block
-// of a group needs its rotated inputs and its partial sums resident.  Budget: 60% of what is free (counting the
-// scratch arena the context already holds), between 2 and 24 GiB.
-static size_t bsgs_group_bytes(fesc_ctx* ctx) {
+// of a group needs its rotated inputs and its partial sums resident.  Budget: 24 GiB of scratch for them (28 GiB with packed operands; a fixed
+// figure, so the launch shape does not depend on what else holds memory); if the device cannot provide the scratch,
+// the group is halved until it fits.
+static size_t bsgs_group_bytes(bool packed) {
     const char* e = getenv("FESC_BSGS_GROUP_GIB");
     if (e && atoi(e) > 0) return (size_t)atoi(e) << 30;
-    size_t free_b = 0, total_b = 0;
-    if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) return (size_t)12 << 30;
-    size_t budget = (free_b + ctx->scratch_bytes) / 10 * 6;
-    const size_t lo = (size_t)2 << 30, hi = (size_t)24 << 30;
-    return budget < lo ? lo : (budget > hi ? hi : budget);
+    return (size_t)(packed ? 28 : 24) << 30;      // the packed inputs of a group are scratch as well
 }
 
 extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_t* d_diags, const fesc_bsgs_desc* desc,
@@ -454,21 +593,39 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
             return fesc_fail(ctx, FESC_ENOKEY, "linear: missing giant-step key " + std::to_string(desc->giant_key_base + p));
     cudaStream_t st = (cudaStream_t)stream;
     const size_t ctw = (size_t)2 * level * N;
-    // token blocks per group, from the scratch budget
-    const size_t per_tb = ((size_t)gin * n1 + (size_t)nout * n2) * ctw * sizeof(u64);
-    uint32_t tbg = (uint32_t)(bsgs_group_bytes(ctx) / per_tb);
+    const bool packed = desc->packed != 0;
+    if (packed && !bsgs_packed_supported(ctx, level, gin * n1))
+        return fesc_fail(ctx, FESC_EINVAL, "linear: packed diagonals need N a multiple of 8, primes below 2^56 and at most 512 terms");
+    // token blocks per group, from the scratch budget (groups of packed inputs are whole tiles of 4 token blocks)
+    const size_t xpk_tb = packed ? bsgs_packed_bytes(N, level, 8, gin * n1) / 4 : 0;
+    const size_t per_tb = ((size_t)gin * n1 + (size_t)nout * n2) * ctw * sizeof(u64) + xpk_tb;
+    uint32_t tbg = (uint32_t)(bsgs_group_bytes(packed) / per_tb);
     if (tbg < 1) tbg = 1;
+    if (packed && tbg > 4) tbg -= tbg % 4;
     if (tbg > tbs) tbg = tbs;
-    const uint32_t max_batch = tbg * (gin > nout ? gin : nout);
-    const size_t ks_words = ks_scratch_words(ctx, level, ks_chunk(ctx, max_batch));
-    const size_t rs_words = (size_t)(tbg * nout < 16384 ? tbg * nout : 16384) * 2 * N;
-    const size_t rot_words = (size_t)tbg * gin * n1 * ctw, acc_words = (size_t)tbg * nout * n2 * ctw;
-    u64* scratch;
-    int rc = ctx_scratch(ctx, (rot_words + acc_words + (ks_words > rs_words ? ks_words : rs_words)) * sizeof(u64), &scratch);
-    if (rc != FESC_OK) return rc;
-    u64* rot = scratch;
-    u64* acc = rot + rot_words;
-    u64* ks = acc + acc_words;
+    u64 *scratch = nullptr, *rot = nullptr, *acc = nullptr, *ks = nullptr;
+    uint8_t* xpk = nullptr;
+    int rc;
+    for (;;) {
+        const uint32_t max_batch = tbg * (gin > nout ? gin : nout);
+        const size_t ks_words = ks_scratch_words(ctx, level, ks_chunk(ctx, max_batch));
+        const size_t rs_words = (size_t)(tbg * nout < 16384 ? tbg * nout : 16384) * 2 * N;
+        const size_t rot_words = (size_t)tbg * gin * n1 * ctw, acc_words = (size_t)tbg * nout * n2 * ctw;
+        const size_t xpk_words = packed ? bsgs_packed_bytes(N, level, 2 * tbg, gin * n1) / 8 : 0;
+        rc = ctx_scratch(ctx, (rot_words + acc_words + xpk_words + (ks_words > rs_words ? ks_words : rs_words)) * sizeof(u64),
+                         &scratch);
+        if (rc == FESC_OK) {
+            rot = scratch;
+            acc = rot + rot_words;
+            xpk = (uint8_t*)(acc + acc_words);
+            ks = acc + acc_words + xpk_words;
+            break;
+        }
+        if (rc != FESC_ENOMEM || tbg == 1) return rc;
+        tbg = (tbg + 1) / 2;
+        if (packed && tbg > 4) tbg -= tbg % 4;
+    }
+    ctx->counters[5] = tbg;
     // lazy 128-bit sums: reduce before terms * q^2 could reach 2^128
     uint32_t qbits = 0;
     for (uint32_t i = 0; i < level; i++) {
@@ -499,7 +656,7 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
             }
         }
         const uint32_t bp_count = nout * n2;
-        prof_begin(ctx, PF_BSGS, st);
+        if (!packed) prof_begin(ctx, PF_BSGS, st);
 #define BSGS(TT, PT)                                                                                          \
     do {                                                                                                      \
         dim3 grid((bp_count + PT - 1) / PT, (N + 255) / 256, level * ((nt + TT - 1) / TT));                   \
@@ -533,15 +690,39 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
         FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
         kern<<<grid, MIX_THREADS, smem, st>>>(rot, diags, acc, ctx->d_pc, N, level, nt, gin * n1, bp_count);  \
     } while (0)
+#define BSGS_IMMA(FP, ST)                                                                                       \
+    do {                                                                                                      \
+        const uint32_t tp = ((gin * n1 + 31) / 32) * 32;                                                      \
+        uint32_t pitch = tp * IM_ROWP;                                                                        \
+        pitch += (17 - pitch % 16) % 16;          /* = 1 mod 16 */                                            \
+        dim3 grid(N / IM_CW, level, (nt + 3) / 4);                                                            \
+        const size_t smem = ((size_t)8 * pitch + (size_t)ST * IM_STAGE_WORDS) * 8;                            \
+        auto kern = k_bsgs_accumulate_imma<FP, ST>;                                                           \
+        FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        kern<<<grid, 32 * IM_CW, smem, st>>>(rot, diags, acc, ctx->d_pc, N, level, nt, gin * n1, bp_count, pitch); \
+    } while (0)
+        if (packed) {
+            rc = bsgs_pack_inputs(ctx, rot, xpk, level, nt, gin * n1, st);
+            if (rc == FESC_OK)
+                rc = bsgs_accumulate_packed(ctx, xpk, (const uint8_t*)d_diags, acc, level, nt, gin * n1, bp_count, qbits <= 50, st);
+            if (rc != FESC_OK) return rc;
+        }
         const bool fp_ok = qbits <= 50 && bsgs_kernel() != 2;
-        if (fp_ok && bsgs_kernel() == 0 && N % 256 == 0 && nt >= 2 && gin * n1 <= 256) BSGS_MIX(2, 8, 3);
+        const bool imma_ok = bsgs_kernel() == 0 && qbits <= 56 && N % IM_CW == 0 && gin * n1 <= 256 && level <= 65535;
+        const bool deep = gin * n1 <= 128;       // room for 8 stages beside the rotated inputs
+        if (packed) {
+        } else if (imma_ok && qbits <= 50 && deep) BSGS_IMMA(true, 8);
+        else if (imma_ok && qbits <= 50) BSGS_IMMA(true, 4);
+        else if (imma_ok && deep) BSGS_IMMA(false, 8);
+        else if (imma_ok) BSGS_IMMA(false, 4);
+        else if (fp_ok && bsgs_kernel() == 3 && N % 256 == 0 && nt >= 2 && gin * n1 <= 256) BSGS_MIX(2, 8, 3);
         else if (fp_ok && N % 256 == 0 && nt >= 2) BSGS_FPS(2, 8, 3);
         else if (fp_ok && nt >= 2) BSGS_FP(2, 8);
         else if (fp_ok) BSGS_FP(1, 8);
         else if (nt >= 2) BSGS(2, 8);
         else BSGS(1, 8);
 #undef BSGS
-        prof_end(ctx, PF_BSGS, st);
+        if (!packed) prof_end(ctx, PF_BSGS, st);
         FESC_CHECK_CUDA(ctx, cudaGetLastError());
         ctx->counters[2] += (uint64_t)nt * bp_count * gin * n1;
         if (desc->defer) {

@@ -354,31 +354,6 @@ __global__ void __launch_bounds__(256, INNER_MINB) k_inner(const u64* __restrict
 // blocks) and a thread picks its word inside the block.  Every wait is bounded: a wait that runs out sets the
 // status word and the CTA returns.
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok;
-}
-// returns 0 when the phase completed, 1 when the poll budget ran out
-__device__ __forceinline__ uint32_t mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    for (uint32_t it = 0; it < (1u << 20); it++) {
-        if (mbar_try_wait(bar, parity)) return 0;
-        if (it > 64) __nanosleep(64);
-    }
-    return 1;
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
 // Self-test of the bounded wait: one warp waits on a barrier phase that nothing completes, with a small poll budget;
 // the wait runs out, the status word is set and the kernel returns (no copy is in flight, nothing faults).
 __global__ void k_wait_limit_selftest(uint32_t* __restrict__ status) {

@@ -35,14 +35,26 @@ def _setup(pair, T, C, n1, n2, tokens, d_in, d_out, level, scale, wscale=1.0, ke
     return X, W, cts, diags, (gin, nout, tbs)
 
 
-def _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=1000, hoist=0, defer=0):
+def _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=1000, hoist=0, defer=0, packed=0):
+    """packed=1: the diagonals go through fesc_linear_pack_diags first (two ranges when there are more than 8 (b,p)
+    pairs, so that the placement of a later range is exercised) and fesc_linear runs on the byte-plane image."""
     import torch
     import paper_2608_17442_b200 as fesc
 
     gin, nout, tbs = dims
-    desc = fesc.BsgsDesc(n1, n2, gin, nout, tbs, level, key_base, key_base + 500, hoist, defer)
+    desc = fesc.BsgsDesc(n1, n2, gin, nout, tbs, level, key_base, key_base + 500, hoist, defer, packed)
     out = torch.empty((tbs, nout, 2, level - 1, cts.shape[-1]), dtype=torch.int64, device="cuda")
-    ctx.linear(to_dev(cts), to_dev(diags), desc, out)
+    d = to_dev(diags)
+    if packed:
+        image = torch.full((ctx.linear_packed_bytes(desc),), 0xA5, dtype=torch.uint8, device="cuda")
+        pairs = nout * n2
+        flat = d.reshape(pairs, gin, n1, level, cts.shape[-1])
+        cut = 8 if pairs > 8 else pairs
+        ctx.linear_pack_diags(flat[:cut], desc, 0, cut, image)
+        if cut < pairs:
+            ctx.linear_pack_diags(flat[cut:].contiguous(), desc, cut, pairs - cut, image)
+        d = image
+    ctx.linear(to_dev(cts), d, desc, out)
     return to_host(out)
 
 
@@ -59,6 +71,7 @@ def test_linear_small_ring(shape):
     want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)},
                       {g: kb + 500 + g for g in range(1, n2)})
     assert np.array_equal(got, want)
+    assert np.array_equal(_run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=kb, packed=1), want)
     # hoisted baby rotations: other residues (own oracle mode), same values
     got_h = _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=kb, hoist=1)
     want_h = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)},
@@ -71,6 +84,7 @@ def test_linear_small_ring(shape):
         want_d = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)},
                             {g: kb + 500 + g for g in range(1, n2)}, hoist=bool(hoist), defer=True)
         assert np.array_equal(got_d, want_d)
+        assert np.array_equal(_run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=kb, hoist=hoist, defer=1, packed=1), want_d)
     gin, nout, tbs = dims
     for tb in range(tbs):
         for b in range(nout):
@@ -105,6 +119,9 @@ def test_linear_accumulate_extreme_residues_256_terms():
     for hoist in (0, 1):
         got = _run_gpu(ctx, cts, diags, n1, n2, (gin, nout, tbs), level, key_base=kb, hoist=hoist)
         want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)}, {}, hoist=bool(hoist))
+        assert np.array_equal(got, want)
+        # the byte-plane products on the tensor cores: 256 terms of 255 x 255 per plane pair, 8 k-steps
+        got = _run_gpu(ctx, cts, diags, n1, n2, (gin, nout, tbs), level, key_base=kb, hoist=hoist, packed=1)
         assert np.array_equal(got, want)
 
 
@@ -213,7 +230,8 @@ def test_linear_on_complex_paired_input_blocks():
 
 
 def test_linear_integer_kernels_with_55_bit_primes():
-    """The 128-bit integer accumulate kernel (primes above 50 bits) against the oracle."""
+    """Primes above 50 bits (the integer recombination of the tensor-core accumulate; the 128-bit integer kernel where
+    that does not apply) against the oracle."""
     pair = ctx_pair("wide")
     ctx, orc, _ = pair
     T, C, n1, n2, level = 32, 16, 4, 4, 6
@@ -222,6 +240,9 @@ def test_linear_integer_kernels_with_55_bit_primes():
         got = _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=3000, hoist=hoist, defer=defer)
         want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: 3000 + q for q in range(1, n1)},
                           {g: 3500 + g for g in range(1, n2)}, hoist=bool(hoist), defer=bool(defer))
+        assert np.array_equal(got, want)
+        # packed diagonals with 55-bit primes: the 128-bit integer recombination
+        got = _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=3000, hoist=hoist, defer=defer, packed=1)
         assert np.array_equal(got, want)
 
 
@@ -246,6 +267,7 @@ def test_linear_full_ring_one_block():
     want_m = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: 2000 + q for q in range(1, n1)},
                         {g: 2500 + g for g in range(1, n2)}, hoist=True, defer=True)
     assert np.array_equal(got_m, want_m)
+    assert np.array_equal(_run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=2000, hoist=1, defer=1, packed=1), want_m)
     err_m = np.abs(orc.decrypt(got_m[0, 0], scale, 2).real.reshape(C, T).T - X @ W).max()
     print("hoisted + deferred: max |decrypt - X@W| = 2^%.2f" % np.log2(err_m))
     assert err_m < 2.0**-18
