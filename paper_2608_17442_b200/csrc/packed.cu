@@ -27,7 +27,7 @@
 #define PK_CW 8
 #define PK_FRAG 1792
 #define PK_STAGE (PK_CW * PK_FRAG)
-#define PK_STAGES 12
+#define PK_STAGES 7
 #define PK_ROWP 9
 #define PK_BLK (32 * PK_ROWP + 1)
 
@@ -87,27 +87,34 @@ int bsgs_pack_inputs(fesc_ctx* ctx, const u64* rot, uint8_t* xpk, uint32_t level
     return FESC_OK;
 }
 
-// Accumulate: CTA = (coefficient tile of 8, limb, tile of 4 token blocks) = 8 warps, one coefficient each.  Every warp
-// streams the diagonal images of ITS coefficient (1792 bytes per k-step, one bulk asynchronous copy each) through a
-// private ring of PK_STAGES slots, each slot with its own barrier: the warp that consumed a slot requests the copy
-// that refills it, so warps never wait for one another and one warp's recombination overlaps the other warps' tensor
-// work.  Every barrier wait is bounded; a wait that runs out sets the status word (3), the warp waits (bounded) for
-// its other copies in flight and leaves.
+// Accumulate: CTA = (half a coefficient tile, limb, tile of 4 token blocks) = 4 warps, one coefficient each; three
+// CTAs share an SM, so every scheduler holds three warps: while one recombines its finished tile (a latency-bound
+// chain of integer and FP64 operations) the other two keep the tensor pipe busy.  Every warp streams the diagonal
+// images of ITS coefficient (1792 bytes per k-step, one bulk asynchronous copy each) through a private ring of
+// PK_STAGES slots, each slot with its own barrier: the warp that consumed a slot requests the copy that refills it,
+// so warps never wait for one another.  The input fragments of the coefficient (at most 3 k-steps) are copied once
+// into shared memory the same way.  Every barrier wait is bounded; a wait that runs out sets the status word (3), the
+// warp waits (bounded) for its other copies in flight and leaves.
+#define PK_WARPS 4
 template <bool FP, int KSR>
-__global__ void __launch_bounds__(32 * PK_CW, 1) k_bsgs_accumulate_packed(
+__global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
     const uint8_t* __restrict__ xpk, const uint8_t* __restrict__ dpk, u64* __restrict__ acc,
     const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level, uint32_t tbs, uint32_t ksteps, uint32_t bp_count,
     uint32_t* __restrict__ status) {
-    extern __shared__ __align__(128) uint8_t ring[];      // [warp 8][PK_STAGES][PK_FRAG], then barriers [warp 8][PK_STAGES]
+    // per warp: PK_STAGES ring slots, KSR input images; then per warp PK_STAGES + 1 barriers
+    extern __shared__ __align__(128) uint8_t ring[];
+    constexpr uint32_t WARP_BYTES = (PK_STAGES + KSR) * PK_FRAG;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tg = lane & 3;
-    const uint32_t ct = blockIdx.x, l = blockIdx.y, tbt = blockIdx.z, tiles = gridDim.x;
+    const uint32_t ct = blockIdx.x >> 1, coef = (blockIdx.x & 1) * PK_WARPS + warp, l = blockIdx.y, tbt = blockIdx.z;
+    const uint32_t tiles = gridDim.x >> 1;
     const uint32_t bp_tiles = (bp_count + 7) >> 3, total = bp_tiles * ksteps;
-    const uint32_t my_ring = (uint32_t)__cvta_generic_to_shared(ring) + warp * (PK_STAGES * PK_FRAG);
-    const uint32_t my_bar = (uint32_t)__cvta_generic_to_shared(ring) + PK_CW * PK_STAGES * PK_FRAG + warp * (PK_STAGES * 8);
-    const uint8_t* my_img = ring + warp * (PK_STAGES * PK_FRAG);
+    const uint32_t my_ring = (uint32_t)__cvta_generic_to_shared(ring) + warp * WARP_BYTES;
+    const uint32_t my_bar = (uint32_t)__cvta_generic_to_shared(ring) + PK_WARPS * WARP_BYTES + warp * ((PK_STAGES + 1) * 8);
+    const uint8_t* my_img = ring + warp * WARP_BYTES;
     // images of this warp's coefficient: k-steps of one (b,p) tile are PK_STAGE apart, tiles tile_stride apart
-    const uint8_t* src = dpk + ((size_t)l * tiles + ct) * ksteps * PK_STAGE + warp * PK_FRAG;
+    const uint8_t* src = dpk + ((size_t)l * tiles + ct) * ksteps * PK_STAGE + coef * PK_FRAG;
     const size_t tile_stride = (size_t)level * tiles * ksteps * PK_STAGE;
+    const uint8_t* ximg = xpk + ((((size_t)tbt * level + l) * tiles + ct) * ksteps * PK_CW + coef) * PK_FRAG;
     uint32_t ld_ks = 0, ld_s = 0;                         // next stage to request (lane 0)
     auto request = [&](uint32_t slot) {
         mbar_expect_tx(my_bar + slot * 8, PK_FRAG);
@@ -116,8 +123,13 @@ __global__ void __launch_bounds__(32 * PK_CW, 1) k_bsgs_accumulate_packed(
         ld_s++;
     };
     if (lane == 0) {
-        for (uint32_t i = 0; i < PK_STAGES; i++) mbar_init(my_bar + i * 8, 1);
+        for (uint32_t i = 0; i <= PK_STAGES; i++) mbar_init(my_bar + i * 8, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (KSR > 0) {
+            mbar_expect_tx(my_bar + PK_STAGES * 8, KSR * PK_FRAG);
+            for (uint32_t k = 0; k < KSR; k++)
+                bulk_g2s(my_ring + (PK_STAGES + k) * PK_FRAG, ximg + (size_t)k * PK_STAGE, PK_FRAG, my_bar + PK_STAGES * 8);
+        }
         for (uint32_t i = 0; i < PK_STAGES && i < total; i++) request(i);
     }
     __syncwarp();
@@ -129,19 +141,17 @@ __global__ void __launch_bounds__(32 * PK_CW, 1) k_bsgs_accumulate_packed(
         c64 = fp_modmul(c32, c32, pc.qd, pc.qinvd);
         c96 = fp_modmul(c64, c32, pc.qd, pc.qinvd);
     }
-    // input fragments of this warp's coefficient
-    const uint8_t* ximg = xpk + ((((size_t)tbt * level + l) * tiles + ct) * ksteps * PK_CW + warp) * PK_FRAG + lane * 8;
-    uint2 fb[KSR > 0 ? KSR : 1][7];
-    if (KSR > 0) {
-#pragma unroll
-        for (int k = 0; k < KSR; k++)
-#pragma unroll
-            for (int j = 0; j < 7; j++) fb[k][j] = __ldg((const uint2*)(ximg + (size_t)k * PK_STAGE + j * 256));
+    const uint32_t out_bar = (uint32_t)__cvta_generic_to_shared(ring) + PK_WARPS * (WARP_BYTES + (PK_STAGES + 1) * 8) + 2 * 256 * 8;
+    if (tid == 0) {
+        mbar_init(out_bar, PK_WARPS);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    __syncthreads();
     int d[4][7][4];
     uint32_t slot = 0, phase = 0, s = 0;
-    bool ok = true;
-    auto mma_stage = [&](const uint2 (&b)[7], bool first) {
+    bool ok = KSR == 0 || !mbar_wait_bounded(my_bar + PK_STAGES * 8, 0);
+    const bool x_ok = ok;
+    auto mma_stage = [&](const uint8_t* xfrag, bool first) {
         if (mbar_wait_bounded(my_bar + slot * 8, phase)) {
             ok = false;
             return;
@@ -149,22 +159,24 @@ __global__ void __launch_bounds__(32 * PK_CW, 1) k_bsgs_accumulate_packed(
         const uint8_t* img = my_img + slot * PK_FRAG;
         const uint4 a0 = *(const uint4*)(img + lane * 16), a1 = *(const uint4*)(img + 512 + lane * 16);
         const uint4 a2 = *(const uint4*)(img + 1024 + lane * 16);
-        const uint2 a3 = *(const uint2*)(img + 1536 + lane * 8);
-        if (first) {
+        uint4 a3;                                              // plane 6 and an empty plane
+        a3.x = *(const uint32_t*)(img + 1536 + lane * 8);
+        a3.z = *(const uint32_t*)(img + 1540 + lane * 8);
+        a3.y = a3.w = 0u;
 #pragma unroll
-            for (int j = 0; j < 7; j++) {
-                imma_u8_zero(d[0][j], a0.x, a0.y, a0.z, a0.w, b[j].x, b[j].y);
-                imma_u8_zero(d[1][j], a1.x, a1.y, a1.z, a1.w, b[j].x, b[j].y);
-                imma_u8_zero(d[2][j], a2.x, a2.y, a2.z, a2.w, b[j].x, b[j].y);
-                imma_u8_zero(d[3][j], a3.x, 0u, a3.y, 0u, b[j].x, b[j].y);
-            }
-        } else {
-#pragma unroll
-            for (int j = 0; j < 7; j++) {
-                imma_u8(d[0][j], a0.x, a0.y, a0.z, a0.w, b[j].x, b[j].y);
-                imma_u8(d[1][j], a1.x, a1.y, a1.z, a1.w, b[j].x, b[j].y);
-                imma_u8(d[2][j], a2.x, a2.y, a2.z, a2.w, b[j].x, b[j].y);
-                imma_u8(d[3][j], a3.x, 0u, a3.y, 0u, b[j].x, b[j].y);
+        for (int j = 0; j < 7; j++) {
+            const uint2 b = KSR > 0 ? *(const uint2*)(xfrag + j * 256 + lane * 8)
+                                    : __ldg((const uint2*)(xfrag + j * 256 + lane * 8));
+            if (first) {
+                imma_u8_zero(d[0][j], a0.x, a0.y, a0.z, a0.w, b.x, b.y);
+                imma_u8_zero(d[1][j], a1.x, a1.y, a1.z, a1.w, b.x, b.y);
+                imma_u8_zero(d[2][j], a2.x, a2.y, a2.z, a2.w, b.x, b.y);
+                imma_u8_zero(d[3][j], a3.x, a3.y, a3.z, a3.w, b.x, b.y);
+            } else {
+                imma_u8(d[0][j], a0.x, a0.y, a0.z, a0.w, b.x, b.y);
+                imma_u8(d[1][j], a1.x, a1.y, a1.z, a1.w, b.x, b.y);
+                imma_u8(d[2][j], a2.x, a2.y, a2.z, a2.w, b.x, b.y);
+                imma_u8(d[3][j], a3.x, a3.y, a3.z, a3.w, b.x, b.y);
             }
         }
         // The products above consumed every loaded register of every lane, so all reads of the slot have returned and
@@ -180,30 +192,43 @@ __global__ void __launch_bounds__(32 * PK_CW, 1) k_bsgs_accumulate_packed(
         if (KSR > 0) {
 #pragma unroll
             for (int k = 0; k < (KSR > 0 ? KSR : 1); k++)
-                if (ok) mma_stage(fb[k], k == 0);
+                if (ok) mma_stage(my_img + (PK_STAGES + k) * PK_FRAG, k == 0);
         } else {
 #pragma unroll 1
-            for (uint32_t k = 0; k < ksteps && ok; k++) {
-#pragma unroll
-                for (int j = 0; j < 7; j++) fb[0][j] = __ldg((const uint2*)(ximg + (size_t)k * PK_STAGE + j * 256));
-                mma_stage(fb[0], k == 0);
-            }
+            for (uint32_t k = 0; k < ksteps && ok; k++) mma_stage(ximg + (size_t)k * PK_STAGE, k == 0);
         }
         if (!ok) break;
-        // lane (g, tg) holds output bp = 8 bt + g of token block 4 tbt + tg, both polynomials
-        const uint32_t bp = bt * 8 + g, tb = tbt * 4 + tg;
-        if (bp < bp_count && tb < tbs) {
-            u64* dst = acc + ((size_t)tb * bp_count + bp) * ctw + (size_t)l * N + ct * PK_CW + warp;
-            dst[0] = imma_recombine<FP>(d, 0, pc, c32, c64, c96);
-            dst[poly] = imma_recombine<FP>(d, 1, pc, c32, c64, c96);
+        // lane (g, tg) holds output bp = 8 bt + g of token block 4 tbt + tg, both polynomials.  The four warps of the
+        // CTA (four neighbouring coefficients) exchange their results through shared memory so that every output row
+        // receives one full 32-byte sector instead of four separate words.
+        u64* stage_out = (u64*)(ring + PK_WARPS * (WARP_BYTES + (PK_STAGES + 1) * 8)) + (bt & 1) * 256;
+        stage_out[(lane * 2) * PK_WARPS + warp] = imma_recombine<FP>(d, 0, pc, c32, c64, c96);
+        stage_out[(lane * 2 + 1) * PK_WARPS + warp] = imma_recombine<FP>(d, 1, pc, c32, c64, c96);
+        // CTA-wide hand-over on a shared-memory barrier (one arrival per warp) so that this wait is bounded too
+        __syncwarp();
+        if (lane == 0) mbar_arrive(out_bar);
+        if (mbar_wait_bounded(out_bar, bt & 1)) {
+            ok = false;
+            break;
+        }
+        {
+            const uint32_t row = tid >> 1, rl = row >> 1, rg = rl >> 2, rtg = rl & 3;     // row = (lane of the owner) * 2 + polynomial
+            const uint32_t bp = bt * 8 + rg, tb = tbt * 4 + rtg;
+            if (bp < bp_count && tb < tbs) {
+                const ulonglong2 v = *(const ulonglong2*)(stage_out + row * PK_WARPS + (tid & 1) * 2);
+                u64* dst = acc + ((size_t)tb * bp_count + bp) * ctw + (row & 1) * poly + (size_t)l * N + ct * PK_CW +
+                           (blockIdx.x & 1) * PK_WARPS + (tid & 1) * 2;
+                *(ulonglong2*)dst = v;
+            }
         }
     }
     if (!ok) {
-        // stage s never arrived.  The copies requested after it (stages s+1 .. ld_s-1) may still be in flight: give each
-        // a bounded wait before this CTA's shared memory can be handed on.
+        // A copy never arrived.  The copies requested after the missing stage may still be in flight: give each a
+        // bounded wait before this CTA's shared memory can be handed on.
         if (lane == 0) {
             atomicExch(status, 3u);
-            for (uint32_t sp = s + 1; sp < ld_s; sp++) mbar_wait_bounded(my_bar + (sp % PK_STAGES) * 8, (sp / PK_STAGES) & 1);
+            for (uint32_t sp = x_ok ? s + 1 : 0; sp < ld_s; sp++)
+                mbar_wait_bounded(my_bar + (sp % PK_STAGES) * 8, (sp / PK_STAGES) & 1);
         }
         __syncwarp();
     }
@@ -212,14 +237,14 @@ __global__ void __launch_bounds__(32 * PK_CW, 1) k_bsgs_accumulate_packed(
 int bsgs_accumulate_packed(fesc_ctx* ctx, const uint8_t* xpk, const uint8_t* dpk, u64* acc, uint32_t level, uint32_t tbs,
                            uint32_t terms, uint32_t bp_count, bool fp, cudaStream_t st) {
     const uint32_t N = ctx->N, ksteps = (terms + 31) / 32;
-    dim3 grid(N / PK_CW, level, (tbs + 3) / 4);
-    const size_t smem = (size_t)PK_STAGES * PK_STAGE + PK_CW * PK_STAGES * 8;
+    dim3 grid(2 * (N / PK_CW), level, (tbs + 3) / 4);
 #define PK_LAUNCH(FP, KSR)                                                                                        \
     do {                                                                                                          \
+        const size_t smem = (size_t)PK_WARPS * ((PK_STAGES + KSR) * PK_FRAG + (PK_STAGES + 1) * 8) + 2 * 256 * 8 + 8; \
         auto kern = k_bsgs_accumulate_packed<FP, KSR>;                                                            \
         FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        kern<<<grid, 32 * PK_CW, smem, st>>>(xpk, dpk, acc, ctx->d_pc, N, level, tbs, ksteps, bp_count,     \
-                                                   ctx->d_status);                                                \
+        kern<<<grid, 32 * PK_WARPS, smem, st>>>(xpk, dpk, acc, ctx->d_pc, N, level, tbs, ksteps, bp_count,        \
+                                                ctx->d_status);                                                   \
     } while (0)
     prof_begin(ctx, PF_BSGS, st);
     if (fp) {
