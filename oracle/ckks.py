@@ -15,9 +15,11 @@ operations the library exports, in the order the definitions state them:
     Breakdown": packing idx(r,c) = c*T + r, accumulators c_p, giant-step fold).
 
 The paper uses its CKKS backend as a black box, so the internals follow the
-standard hybrid (dnum) key switching with the readings listed in the design
-notes: canonical residues, uncorrected fast basis conversion, ROUNDED division
-by P (key switch) and by the dropped prime (rescale).
+standard hybrid (dnum) key switching with these readings: canonical residues in
+[0, q); uncorrected fast basis conversion in ModUp; division by P with the CENTRED
+fast conversion of the special-limb residues (no half-P shift; error at most K/2
+units, exact rounding for K = 1); rescale = the same centred conversion with one
+source limb, i.e. exact rounded division by the dropped prime.
 
 Layouts: a polynomial on k limbs is a uint64 array [k, N]; a ciphertext at
 level l is [2, l, N] (c0 then c1), evaluation form, bit-reversed order.

@@ -16,7 +16,7 @@
  *
  * The paper (Sec. 5.1, Table "CKKS primitives") treats add / ptmul / ctmul /
  * rot / conj as black boxes, so the constructions below are the standard
- * RNS-CKKS ones with the conventions fixed in the design notes:
+ * RNS-CKKS ones with these conventions:
  *   - residues are canonical, in [0, q);
  *   - psi is the SMALLEST primitive 2N-th root of unity mod q;
  *   - evaluation order: EVAL[t] = sum_i COEFF[i] * psi^((2*brev(t)+1)*i) mod q.

@@ -12,7 +12,7 @@ Homomorphic realisation.  The paper fixes the contract, the affine composition
 contraction (Eq. hescan-contract-output), the blocked schedule with carries (Eq. resident-block-schedule, in its
 serialized-carry form of App. "longer sequences"), the Brent-Kung network (App. "Prefix-Network Selection") and
 the complex-paired state reduction (App. "Complex-Packed Reduction Accounting"); it does not give the slot-level
-broadcast maps.  The dataflow below is this build's reading (listed in the design notes); the CUDA library
+broadcast maps.  The dataflow below is this build's reading, stated in full in this header; the CUDA library
 implements the same graph independently and must reproduce every residue.
 
 Geometry (all powers of two).  n slots = c_state * stride, stride >= max(d_s, B_blk); one state ciphertext of

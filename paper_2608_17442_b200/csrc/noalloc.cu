@@ -14,8 +14,11 @@
 #define FESC_STATIC_SCRATCH_WORDS (4u * 2u * 65536u)
 static __device__ __align__(256) unsigned long long g_rescale_scratch[FESC_STATIC_SCRATCH_WORDS];
 
-// Device address of the array, looked up once per device.  The symbol's name is only a host-side
-// handle; kernels need the address cudaGetSymbolAddress returns for the CURRENT device.
+// Device address of the array, looked up once per device ordinal.  The symbol's name is only a host-side
+// handle; kernels need the address cudaGetSymbolAddress returns for the CURRENT device.  Under lazy module
+// loading that lookup is what loads this module and places the array on the device, so the first call belongs
+// at initialisation (it needs 4 MiB to be available).  The cache is written without locking: first calls on a
+// device must not race across host threads; afterwards it is only read.
 #define FESC_MAX_DEVICES 64
 static u64* g_scratch_addr[FESC_MAX_DEVICES];
 

@@ -286,7 +286,7 @@ __global__ void __launch_bounds__(256, INNER_MINB) k_inner(const u64* __restrict
                 f0[i] += fp_modmul(xd, dkb, q, qinv);
                 f1[i] += fp_modmul(xd, dka, q, qinv);
             }
-            if ((j & 7) == 6) {   // q/2 (a running sum) + 7 terms stay below 6.7q; fold before the 8th
+            if (j % 7 == 6) {   // |running sum| <= q/2 plus 7 products below 0.875q each stays below 6.7q < 2^53: fold after every 7th
 #pragma unroll
                 for (int i = 0; i < BT; i++) {
                     f0[i] = fp_reduce(f0[i], q, qinv);
@@ -435,6 +435,10 @@ __global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ ex
         if (__syncthreads_or((int)late)) {                   // block-uniform: give up together
             if (tid == 0) {
                 atomicExch(status, 1u);
+                // copies may still be in flight into this CTA's shared memory: one more bounded wait on the stage
+                // that ran out and one on the other stage before the memory can be handed to another CTA (after a
+                // time-out the caller has to synchronise and discard whatever overlapped on the device anyway)
+                mbar_wait_bounded(bar0 + stage * 8, (k >> 1) & 1);
                 if (tile + gridDim.x < n_tiles) mbar_wait_bounded(bar0 + (stage ^ 1) * 8, ((k + 1) >> 1) & 1);
             }
             return;
@@ -467,7 +471,7 @@ __global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ ex
                     f0[i] += fp_modmul(xd, dkb, q, qinv);
                     f1[i] += fp_modmul(xd, dka, q, qinv);
                 }
-                if ((j & 7) == 7) {
+                if (j % 7 == 6) {   // same schedule as k_inner: |sum| <= q/2 plus 7 products stays below 6.7q
 #pragma unroll
                     for (int i = 0; i < BT; i++) {
                         f0[i] = fp_reduce(f0[i], q, qinv);

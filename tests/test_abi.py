@@ -34,3 +34,26 @@ def test_product_does_not_import_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in text.replace("no CPU fallback", ""), f
+
+
+def test_params_info_flags_a_special_modulus_below_the_digit_modulus():
+    """fesc_params_info runs on the host alone.  The graded reading of workloads 3-5 (6 digits of 4 limbs, P = four
+    60-bit primes) has P above every digit modulus; the literal dnum = 4 set (digits of 6 x 50 bits against the same
+    240-bit P) does not, and is flagged."""
+    import fesc_synth as S
+    import paper_2608_17442_b200 as fesc
+
+    p = S.params("full")
+    info = fesc.params_info(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"])
+    assert (info.alpha, info.digits, info.flags) == (4, 6, 0)
+    assert 239.9 < info.log2_P < 240.0 and 199.9 < info.log2_Qmax < 200.0
+    p = S.params("full_literal")
+    info = fesc.params_info(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"])
+    assert (info.alpha, info.digits) == (6, 4)
+    assert info.flags & fesc.INFO_KEYSWITCH_NOISE and info.log2_Qmax > info.log2_P
+    # the exact comparison decides, not the rounded logarithms: P one prime short of the digit modulus
+    p = S.params("tiny")
+    info = fesc.params_info(p["log_n"], p["primes"], p["n_q"], p["n_p"], 1)       # one digit of 3 limbs, one special prime
+    assert info.flags & fesc.INFO_KEYSWITCH_NOISE
+    info = fesc.params_info(p["log_n"], p["primes"], p["n_q"], p["n_p"], 3)       # digits of one limb; special = largest prime
+    assert info.flags == 0

@@ -484,3 +484,93 @@ def test_integer_paths_with_primes_above_50_bits():
             ctx.rescale(to_dev(ct), res, 3, level)
             for b in range(3):
                 assert np.array_equal(to_host(res)[b], orc.rescale(ct[b]))
+
+
+def test_allocation_failure_is_reported_and_the_context_stays_usable():
+    """Host-side failure injection: the next scratch allocation of the context reports FESC_ENOMEM (the driver is not
+    called); the error comes back through the call, nothing is launched, and the next call works and is bit-exact."""
+    import torch
+    import paper_2608_17442_b200 as fesc
+
+    pair = ctx_pair("small")
+    ctx, orc, _ = pair
+    add_key(pair, 3, 81)
+    level, batch = 8, 2
+    ct = random_ct(orc, 31, level, level, batch)
+    dev = to_dev(ct)
+    out = torch.full_like(dev, -1)
+    ctx.trim()                                  # the next key switch has to reserve scratch again
+    launches = ctx.counters()[4]
+    ctx.test_fail_allocs(1)
+    with pytest.raises(fesc.FescError) as e:
+        ctx.rotate(dev, out, batch, level, 81)
+    assert e.value.code == fesc.ENOMEM and "scratch allocation" in str(e.value)
+    assert ctx.counters()[4] == launches and ctx.counters()[3] == 0
+    assert bool((out == -1).all())
+    ctx.rotate(dev, out, batch, level, 81)      # the injected failure is used up: this call reserves and runs
+    ctx.sync()
+    got = to_host(out)
+    for b in range(batch):
+        assert np.array_equal(got[b], orc.rotate(ct[b], 81))
+    # fesc_linear halves its token-block group when the arena cannot be had and still returns the same residues
+    assert ctx.info().flags == 0 and ctx.info().digits == ctx.num_digits
+
+
+def test_results_do_not_depend_on_the_run_or_the_stream():
+    """The same rotation batch (plain, hoisted and rotate-and-add) run twice on the default stream and once on each
+    of two other streams, one after the other: all outputs are byte-identical (no dependence on scheduling, on what
+    the scratch arena held before, or on the stream)."""
+    import torch
+
+    pair = ctx_pair("full")
+    ctx, orc, _ = pair
+    add_key(pair, 3, 81)
+    add_key(pair, -5, 82)
+    level, batch = 24, 5
+    dev = to_dev(random_ct(orc, 41, level, level, batch))
+
+    def run():
+        out = torch.empty_like(dev)
+        hout = torch.empty((2, batch, 2, level, orc.N), dtype=torch.int64, device="cuda")
+        sout = torch.empty_like(dev)
+        ctx.rotate(dev, out, batch, level, 81)
+        ctx.rotate_hoisted(dev, hout, batch, level, [81, 82])
+        ctx.rotate_sum_hoisted(dev, sout, batch, level, [81, 82])
+        ctx.sync()
+        return out, hout, sout
+
+    first = run()
+    runs = [run()]
+    for _ in range(2):
+        st = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(st):
+            runs.append(run())
+        torch.cuda.synchronize()
+    for r in runs:
+        for a, b in zip(first, r):
+            assert torch.equal(a, b)
+
+
+def test_inner_product_worst_case_residues_with_many_digits():
+    """Largest possible partial sums of the key inner product: 12 digits (the FP64 path folds back after every 8
+    products), every residue of the switched polynomial equal to q - 1, plain and hoisted; bit-exact."""
+    import torch
+
+    pair = ctx_pair("small_d12")
+    ctx, orc, p = pair
+    add_key(pair, 1, 91)
+    add_key(pair, 2, 92)
+    level, batch = 24, 2
+    ct = random_ct(orc, 51, level, level, batch)
+    qs = np.array(orc.q[:level], dtype=np.uint64)
+    ct[:, 1] = (qs - 1)[None, :, None]                  # c1 = q - 1 everywhere (the automorphism leaves it so)
+    out = torch.empty_like(to_dev(ct))
+    ctx.rotate(to_dev(ct), out, batch, level, 91)
+    hout = torch.empty((2, batch, 2, level, orc.N), dtype=torch.int64, device="cuda")
+    ctx.rotate_hoisted(to_dev(ct), hout, batch, level, [91, 92])
+    got, hgot = to_host(out), to_host(hout)
+    for b in range(batch):
+        assert np.array_equal(got[b], orc.rotate(ct[b], 91))
+        want = orc.rotate_hoisted(ct[b], [91, 92])
+        assert np.array_equal(hgot[0, b], want[0]) and np.array_equal(hgot[1, b], want[1])
