@@ -195,9 +195,12 @@ BFLY_FP64 = 8.5                   # FP64 butterfly (primes < 2^50): 5 ops produc
 MAC_FP64 = 6                      # FP64 multiply-accumulate: 5 ops exact product + 1 add
 MAC_MIXED_CYCLES = 8              # mixed-pipe multiply-accumulate: multiplier-pipe cycles per warp (one 32x32+64 = 4,
                                   # two 32-bit multiply-adds = 2 each) on each of the 4 sub-partitions of an SM
-# DRAM bytes of ONE accumulate launch of the default workload (4 token blocks x 112 accumulators x 96 terms),
-# read + written, from the ncu capture summarised in profiles/bsgs_accumulate_mixed.md
-BSGS_TRAFFIC_4TB = 145058871040 + 11272472832
+# DRAM traffic of one accumulate launch is not captured at full size: a small-case capture of the same kernel
+# (a few GB, inputs larger than L2) gives measured DRAM bytes / algorithmic bytes, and because every operand byte is
+# read once per launch and every output byte written once, traffic grows in proportion to the algorithmic bytes.
+BSGS_TRAFFIC_RATIO = {"packed": 1.010, "residues": 1.001}     # measured DRAM bytes / algorithmic bytes (small case)
+PACKED_BYTES_PER_WORD = 7                                     # a residue below 2^56 as byte planes
+NTT_TRAFFIC_RATIO = 1.0           # the transforms read and write every word of both passes through DRAM once
 INT_LIMB_SHARE = 32.0 / 224.0     # transforms on the 60-bit special primes per key switch (integer path)
 
 
@@ -293,27 +296,235 @@ def oracle_sample(steps: int, warmup: int, hoist: bool = True, defer: bool = Tru
     return ks / dt, dt * 1e3, cores
 
 
+def workload_text(args):
+    """config.workload of both arms (the reference arm times a bounded sample of this workload)."""
+    return ("%s %d->%d, L=2048 tokens, N=2^16, 24x50-bit limbs + 4x60-bit special primes, "
+            "6 key-switch digits, C=256 T=128 n1=%d n2=%d, baby rotations %s"
+            % (PROJ, D_IN, D_OUT, N1, N2, "hoisted (one decomposition per input ciphertext)" if args.hoist else "by plain rotations")
+            + (", one division by P per output for the giant-step sum" if args.defer else ""))
+
+
 SAMPLE_TEXT = ("1 token block x 1 output block x 1 input block of the projection "
                "(31 baby + 7 giant rotations, 256 ct-pt MACs, 1 rescale; 1/672 of the step's MACs)")
+
+
+def oracle_rates():
+    """Per-operation rates of the oracle as it stands at N = 2^16 and 24 limbs (a few seconds of host time):
+    limb transforms, ct-pt multiply-accumulates and plain rotations per second."""
+    import numpy as np
+    import fesc_synth as S
+    from oracle.ckks import Oracle
+
+    p = S.params("full")
+    orc = Oracle(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+    orc.add_galois_key(1, 7)
+    seed = S.config_seed(3)
+    idx = list(range(LEVEL))
+    ct = np.stack([S.uniform_residues_np(seed, 50 + i, orc.q[:LEVEL], orc.N) for i in range(2)])
+    pt = S.uniform_residues_np(seed, 60, orc.q[:LEVEL], orc.N)
+
+    def rate(fn, units, min_s=1.5):
+        fn()
+        n, t0 = 0, time.perf_counter()
+        while time.perf_counter() - t0 < min_s:
+            fn()
+            n += 1
+        return units * n / (time.perf_counter() - t0)
+
+    return {"limb_transforms_per_s": rate(lambda: orc.intt(orc.ntt(ct[0], idx), idx), 2 * LEVEL),
+            "ct_pt_macs_per_s": rate(lambda: orc.ct_pt_mac(ct, pt, ct), 1),
+            "rotations_per_s": rate(lambda: orc.rotate(ct, 7), 1, 3.0),
+            "at": "N=2^16, 24 limbs (a ciphertext-level unit each; rotation = automorphism + hybrid key switch, 6 digits)"}
+
+
+def measure_projection(args, ctx, dev, rank, world, key_base):
+    """One projection workload (the module's D_IN, D_OUT, N1, N2) timed on `ctx`: keys, synthetic inputs, packed or
+    residue diagonals, 3 warm-up steps, one profiled step, `args.steps` timed steps with the clocks sampled."""
+    import torch
+    import fesc_synth as S
+    import paper_2608_17442_b200 as fesc
+
+    p = S.params("full")
+    n = ctx.N
+    bb, gb = key_base
+    for q in range(1, N1):
+        ctx.add_galois_key(q * T_SEG, bb + q)
+    for g in range(1, N2):
+        ctx.add_galois_key(g * N1 * T_SEG, gb + g)
+    gin, nout, tbs = workload_dims(1)
+    desc = fesc.BsgsDesc(N1, N2, gin, nout, tbs, LEVEL, bb, gb, int(args.hoist), int(args.defer), int(args.packed))
+    ct, diags = make_inputs(p["primes"], n, gin, nout, tbs, S.config_seed(5) + rank, dev, ctx, desc)
+    out = torch.empty((tbs, nout, 2, LEVEL - 1, n), dtype=torch.int64, device=dev)
+    torch.cuda.empty_cache()
+    for _ in range(3):
+        ctx.linear(ct, diags, desc, out)
+    ctx.profile_enable(fesc.Context.PROFILE_FAMILIES, 120000)
+    ctx.linear(ct, diags, desc, out)
+    fam = ctx.profile_read()
+    ctx.profile_enable([])
+    c0 = ctx.counters()
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        ctx.linear(ct, diags, desc, out)
+    e1.record()
+    ctx.sync()
+    clocks = sampler.stop()
+    c1 = ctx.counters()
+    ms = e0.elapsed_time(e1) / args.steps
+    ks = (c1[1] - c0[1]) // args.steps
+    res = {"ms": ms, "key_switches": ks, "key_switches_per_s": ks / (ms * 1e-3), "gpu_launches": (c1[4] - c0[4]) // args.steps,
+           "clocks": clocks, "kernel_breakdown": {k: {"ms": round(v[0], 2), "records": v[1]} for k, v in fam.items() if v[1]},
+           "workload": workload_text(args), "input_cts": tbs * gin, "output_cts": tbs * nout,
+           "diagonals_gib": diags.numel() * diags.element_size() / 2**30, "token_blocks_per_group": int(c1[5])}
+    del ct, diags, out
+    return res
 
 
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    value, ms, cores = oracle_sample(args.steps, min(args.warmup, 1), bool(args.hoist), bool(args.defer))
+    value, ms, cores = oracle_sample(args.steps, args.warmup, bool(args.hoist), bool(args.defer))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "key-switches/s",
-        "n_gpus": args.gpus, "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": ms,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
-        "config": {"workload": "in_proj 768->3352, L=2048, N=2^16, 24x50-bit limbs + 4x60-bit special, 6 digits "
-                               "(bounded sample per step: " + SAMPLE_TEXT + ")"},
+        "config": {"workload": workload_text(args), "sample_per_step": SAMPLE_TEXT},
         "cpu_baseline": {"value": value, "unit": "key-switches/s", "cores": cores, "kind": "oracle",
-                         "sample": SAMPLE_TEXT},
+                         "sample": SAMPLE_TEXT, "rates": oracle_rates()},
         "e2e": {"value": value, "unit": "key-switches/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+def measure_variants(args, ctx, ct, diags, out, gin, nout, tbs, n, dev):
+    """The same 2048 x 768 -> 3352 job with two real blocks in the real and imaginary channels of one ciphertext
+    (token blocks, or the paper's input blocks); reported beside the headline."""
+    import torch
+    import paper_2608_17442_b200 as fesc
+
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # the same 2048 x 768 -> 3352 job with token blocks (2u, 2u+1) paired in the real and imaginary channels:
+    # half the ciphertexts go through fesc_linear (real diagonals act on complex slots), then one conjugation
+    # per output separates the two results.  Reported beside the headline, which keeps one block per ciphertext.
+    conj_id = GIANT_BASE + 400
+    ctx.add_galois_key(fesc.CONJ, conj_id)
+    half = tbs // 2
+    desc2 = fesc.BsgsDesc(N1, N2, gin, nout, half, LEVEL, BABY_BASE, GIANT_BASE, int(args.hoist), int(args.defer),
+                          int(args.packed))
+    zc = torch.empty((half * nout, 2, LEVEL - 1, n), dtype=torch.int64, device=dev)
+    o2 = out.reshape(2, half * nout, 2, LEVEL - 1, n)
+
+    def paired():
+        ctx.linear(ct[:half], diags, desc2, zc)
+        ctx.split_complex(zc, o2[0], o2[1], half * nout, LEVEL - 1, conj_id)
+
+    paired()
+    c0 = ctx.counters()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        paired()
+    e1.record()
+    torch.cuda.synchronize()
+    c1 = ctx.counters()
+    v_ms = e0.elapsed_time(e1) / args.steps
+    variants = {"paired_token_blocks": {"latency_ms": v_ms, "key_switches_per_step": (c1[1] - c0[1]) // args.steps,
+                                        "input_cts": half * gin, "output_cts": 2 * half * nout,
+                                        "note": "token blocks 2u and 2u+1 in the real and imaginary channels; "
+                                                "fesc_linear on 8 complex token blocks + fesc_split_complex"}}
+    del zc
+    # the paper's own pairing (App. "Projection Kernel Breakdown"): input blocks 2u and 2u+1 in the real and
+    # imaginary channels with complex diagonals, real part of every output by one conjugation.  Timed on the same
+    # buffers reinterpreted as ceil(gin/2) input blocks (residues are random either way).
+    gp = -(-gin // 2)
+    if gp < gin:
+        desc3 = fesc.BsgsDesc(N1, N2, gp, nout, tbs, LEVEL, BABY_BASE, GIANT_BASE, int(args.hoist), int(args.defer),
+                              int(args.packed))
+        ct3 = ct.reshape(-1)[: tbs * gp * 2 * LEVEL * n].view(tbs, gp, 2, LEVEL, n)
+        if args.packed:      # any bytes are valid byte planes: the head of the image serves as the smaller image
+            dg3 = diags[: ctx.linear_packed_bytes(desc3)]
+        else:
+            dg3 = diags.reshape(-1)[: nout * N2 * gp * N1 * LEVEL * n].view(nout, N2, gp, N1, LEVEL, n)
+        z3 = torch.empty((tbs * nout, 2, LEVEL - 1, n), dtype=torch.int64, device=dev)
+        o3 = out.reshape(tbs * nout, 2, LEVEL - 1, n)
+
+        def paired_in():
+            ctx.linear(ct3, dg3, desc3, z3)
+            ctx.split_complex(z3, o3, None, tbs * nout, LEVEL - 1, conj_id)
+
+        paired_in()
+        c0 = ctx.counters()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.steps):
+            paired_in()
+        e1.record()
+        torch.cuda.synchronize()
+        c1 = ctx.counters()
+        variants["paired_input_blocks"] = {
+            "latency_ms": e0.elapsed_time(e1) / args.steps, "key_switches_per_step": (c1[1] - c0[1]) // args.steps,
+            "input_cts": tbs * gp, "output_cts": tbs * nout,
+            "note": "input blocks 2u and 2u+1 in the real and imaginary channels, complex diagonals; "
+                    "fesc_linear on %d input blocks + real part by fesc_split_complex" % gp}
+        del z3
+    return variants
+
+
+def bsgs_roofline(args, gin, nout, n, tb_per_launch, timed, hbm_peak, sm_mhz):
+    """Roofline of the accumulate family from (milliseconds, launches).  Packed operands: the kernel streams the
+    byte-plane image once per launch (7 bytes per diagonal word), the packed inputs of its token blocks and writes the
+    partial sums: HBM-bound; the tensor-core ceiling (u8 mma.sync m16n8k32 at 8 cycles per scheduler, measured) is
+    reported beside it.  Residue operands: the multiplier-pipe bound of the mixed-pipe kernel."""
+    ms, launches = timed
+    t = ms * 1e-3 / max(1, launches)
+    ctw = 2 * LEVEL * n * 8
+    terms, bp = gin * N1, nout * N2
+    macs = tb_per_launch * bp * terms * 2 * LEVEL * n
+    if args.packed:
+        ksteps = -(-terms // 32)
+        image = -(-bp // 8) * LEVEL * n * ksteps * 1792                      # bytes: 8 rows x 32 terms x 7 planes per image
+        xpk = -(-2 * tb_per_launch // 8) * LEVEL * n * ksteps * 1792
+        alg = image + xpk + tb_per_launch * bp * ctw
+        mma = -(-bp // 8) * ksteps * 28 * LEVEL * n * -(-tb_per_launch // 4)      # m16n8k32 instructions per launch
+        tensor_peak = SM_COUNT * 4 * sm_mhz * 1e6 / 8                            # instructions / s
+        return {"kernel": "bsgs", "variant": "k_bsgs_accumulate_packed (byte planes on the tensor cores)", "bound": "hbm",
+                "achieved": alg / t / 1e9, "peak": hbm_peak, "unit": "GB/s", "frac": alg / t / 1e9 / hbm_peak,
+                "traffic": alg * BSGS_TRAFFIC_RATIO["packed"], "algorithmic_bytes_per_launch": alg,
+                "avg_launch_ms": t * 1e3, "launches": launches, "token_blocks_per_launch": tb_per_launch,
+                "modular_macs_per_s": macs / t,
+                "tensor": {"achieved": mma / t, "peak": tensor_peak, "unit": "u8 m16n8k32 mma.sync / s", "frac": mma / t / tensor_peak}}
+    alg = tb_per_launch * terms * ctw + bp * terms * (ctw // 2) + tb_per_launch * bp * ctw
+    alu_peak = SM_COUNT * 4 * 32 * sm_mhz * 1e6 / MAC_MIXED_CYCLES / 1e12
+    return {"kernel": "bsgs", "variant": "residue operands", "bound": "alu", "achieved": macs / t / 1e12, "peak": alu_peak,
+            "unit": "T modular mac/s (integer multiplier pipe, 8 cycles per warp-mac)", "frac": macs / t / 1e12 / alu_peak,
+            "traffic": alg * BSGS_TRAFFIC_RATIO["residues"], "avg_launch_ms": t * 1e3, "launches": launches,
+            "token_blocks_per_launch": tb_per_launch,
+            "hbm": {"achieved": alg / t / 1e9, "peak": hbm_peak, "unit": "GB/s", "frac": alg / t / 1e9 / hbm_peak,
+                    "algorithmic_bytes_per_launch": alg}}
+
+
+def ntt_roofline(p, n, timed, limb_ntts, hbm_peak, sm_mhz):
+    """All transform launches of the measured steps: butterflies per second against the FP64 / integer issue ceiling,
+    and the bytes the two passes of a limb transform move against the HBM peak."""
+    ms, launches = timed
+    bfly = limb_ntts * (n // 2) * p["log_n"]
+    peak_fp = SM_COUNT * FP64_PER_CLK_PER_SM * sm_mhz * 1e6 / BFLY_FP64 / 1e12
+    peak_int = SM_COUNT * IMAD_PER_CLK_PER_SM * sm_mhz * 1e6 / BFLY_IMAD / 1e12
+    alu_peak = 1.0 / ((1.0 - INT_LIMB_SHARE) / peak_fp + INT_LIMB_SHARE / peak_int)
+    ach = bfly / (ms * 1e-3) / 1e12
+    moved = limb_ntts * 2 * 2 * n * 8           # two passes, each reads and writes the limb
+    return {"kernel": "ntt", "variant": "ntt16_strided + ntt16_contig (two passes per limb transform)", "bound": "alu",
+            "achieved": ach, "peak": alu_peak, "unit": "T butterflies/s (FP64 pipe for 50-bit primes, integer pipe for 60-bit)",
+            "peak_fp64_path": peak_fp, "peak_integer_path": peak_int, "frac": ach / alu_peak,
+            "traffic": moved / max(1, launches) * NTT_TRAFFIC_RATIO, "launches": launches, "limb_transforms": limb_ntts,
+            "us_per_limb_transform": ms * 1e3 / max(1, limb_ntts), "family_ms": ms,
+            "hbm": {"achieved": moved / (ms * 1e-3) / 1e9, "peak": hbm_peak, "unit": "GB/s",
+                    "frac": moved / (ms * 1e-3) / 1e9 / hbm_peak, "bytes_moved_per_limb_transform": 4 * n * 8}}
 
 
 # ---------------------------------------------------------------------------------------------
@@ -361,8 +572,10 @@ def run_ours(args):
     for _ in range(max(3, args.warmup) - 1):
         step()
     ctx.profile_enable(fesc.Context.PROFILE_FAMILIES, 120000)
+    limb_ntts_profiled = ctx.counters()[0]
     step()
     fam = ctx.profile_read()
+    limb_ntts_profiled = ctx.counters()[0] - limb_ntts_profiled
     ctx.profile_enable([])
     total_fam = sum(v[0] for v in fam.values()) or 1.0
     breakdown = {k: {"ms": round(v[0], 3), "records": v[1], "share": round(v[0] / total_fam, 4)} for k, v in fam.items()}
@@ -392,49 +605,24 @@ def run_ours(args):
     ms_per_step = ms_total / args.steps
     value = world * ks_per_step / (ms_per_step * 1e-3)
 
-    # roofline of the dominant kernel family
+    # rooflines of the two heavy kernel families; `roofline` is the dominant one
     hbm_peak, peak_kind = peaks()
-    word = 8
-    ctw = 2 * LEVEL * n * word
-    roof = {"kernel": dominant, "peak_source": peak_kind}
-    if dominant == "bsgs":
-        # one launch = one group of token blocks: every distinct input word read once, every output written once
-        groups = max(1, dom_records // args.steps)
-        tb_per_launch = tbs / groups
-        alg = tb_per_launch * gin * N1 * ctw + nout * N2 * gin * N1 * (ctw // 2) + tb_per_launch * nout * N2 * ctw
-        macs = tb_per_launch * nout * N2 * gin * N1 * 2 * LEVEL * n          # 64x64->128 multiply-adds
-        t = dom_ms * 1e-3 / max(1, dom_records)
-        sm_mhz = clocks.get("sm_mhz") or 1350.0
-        # the default kernel keeps the low 64 bits of every sum on the integer multiplier pipe
-        alu_peak = SM_COUNT * 4 * 32 * sm_mhz * 1e6 / MAC_MIXED_CYCLES / 1e12        # T modular mul-adds / s
-        fp64_peak = SM_COUNT * FP64_PER_CLK_PER_SM * sm_mhz * 1e6 / MAC_FP64 / 1e12
-        traffic = BSGS_TRAFFIC_4TB if (PROJ == "in_proj" and args.scale_down == 1 and abs(tb_per_launch - 4) < 1e-9) else None
-        roof.update({"bound": "alu", "achieved": macs / t / 1e12, "peak": alu_peak,
-                     "unit": "T modular mac/s (integer multiplier pipe, 8 cycles per warp-mac)",
-                     "peak_fp64_only_scheme": fp64_peak,
-                     "frac": macs / t / 1e12 / alu_peak, "traffic": traffic,
-                     "hbm": {"achieved": alg / t / 1e9, "peak": hbm_peak, "unit": "GB/s", "frac": alg / t / 1e9 / hbm_peak,
-                             "algorithmic_bytes_per_launch": alg}})
-    elif dominant == "ntt":
-        # all transform launches of the timed steps: butterflies per second against the multiply-add ceiling
-        bfly = limb_ntts * (n // 2) * p["log_n"]
-        sm_mhz = clocks.get("sm_mhz") or 1350.0
-        peak_fp = SM_COUNT * FP64_PER_CLK_PER_SM * sm_mhz * 1e6 / BFLY_FP64 / 1e12
-        peak_int = SM_COUNT * IMAD_PER_CLK_PER_SM * sm_mhz * 1e6 / BFLY_IMAD / 1e12
-        alu_peak = 1.0 / ((1.0 - INT_LIMB_SHARE) / peak_fp + INT_LIMB_SHARE / peak_int)
-        ach = bfly / (dom_ms * 1e-3) / 1e12
-        roof.update({"bound": "alu", "achieved": ach, "peak": alu_peak,
-                     "unit": "T butterflies/s (FP64 pipe for 50-bit primes, integer pipe for 60-bit)",
-                     "peak_fp64_path": peak_fp, "peak_integer_path": peak_int,
-                     "frac": ach / alu_peak, "traffic": None, "limb_transforms_per_step": limb_ntts // args.steps,
-                     "family_ms_per_step": dom_ms / args.steps,
-                     "hbm": {"achieved": limb_ntts * 2 * n * 8 / (dom_ms * 1e-3) / 1e9, "peak": hbm_peak, "unit": "GB/s",
-                             "frac": limb_ntts * 2 * n * 8 / (dom_ms * 1e-3) / 1e9 / hbm_peak,
-                             "algorithmic_bytes_per_limb_transform": 2 * n * 8}})
+    sm_mhz = clocks.get("sm_mhz") or 1350.0
+    tb_per_launch = int(ctx.counters()[5]) or tbs
+    fam_roofs = {"bsgs": bsgs_roofline(args, gin, nout, n, tb_per_launch, fam["bsgs"], hbm_peak, sm_mhz),
+                 "ntt": ntt_roofline(p, n, fam["ntt"], limb_ntts_profiled, hbm_peak, sm_mhz)}
+    if dominant in fam_roofs:
+        # the dominant family was event-timed over the whole timed region: use those launches
+        if dominant == "bsgs":
+            fam_roofs["bsgs"] = bsgs_roofline(args, gin, nout, n, tb_per_launch, (dom_ms, dom_records), hbm_peak, sm_mhz)
+        else:
+            fam_roofs["ntt"] = ntt_roofline(p, n, (dom_ms, dom_records), limb_ntts, hbm_peak, sm_mhz)
+        roof = dict(fam_roofs[dominant], timed="all launches of the timed steps")
     else:
-        t = dom_ms * 1e-3 / max(1, dom_records)
-        roof.update({"bound": "alu", "achieved": None, "peak": None, "unit": "ms/launch", "frac": None,
-                     "traffic": None, "avg_launch_ms": t * 1e3})
+        roof = {"kernel": dominant, "bound": "alu", "achieved": None, "peak": None, "unit": "ms/launch", "frac": None,
+                "traffic": None, "avg_launch_ms": dom_ms / max(1, dom_records)}
+    roof["peak_source"] = peak_kind
+    others = {k: dict(v, timed="one profiled step") for k, v in fam_roofs.items() if k != dominant}
 
     # end to end: pinned host inputs -> device, projection, result -> pinned host, every step, all inside the timed
     # region.  The copies run on their own streams with double-buffered device tensors, so the upload of step i+1
@@ -476,105 +664,63 @@ def run_ours(args):
     torch.cuda.synchronize()
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), dev) / e2e_steps
+    # one request on its own: upload, projection, download on ONE stream, nothing overlapped
+    torch.cuda.synchronize()
+    barrier()
+    e0.record()
+    cts[0].copy_(h_in, non_blocking=True)
+    ctx.linear(cts[0], diags, desc, outs[0])
+    h_out.copy_(outs[0], non_blocking=True)
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    single_ms = max_over_ranks(e0.elapsed_time(e1), dev)
     e2e = {"value": world * ks_per_step / (e2e_ms * 1e-3), "unit": "key-switches/s", "latency_ms": e2e_ms,
            "h2d_bytes_per_step": ct.numel() * 8, "d2h_bytes_per_step": out.numel() * 8,
-           "overlap": "copies on separate streams, double-buffered device tensors"}
+           "overlap": "copies on separate streams, double-buffered device tensors (throughput of a stream of requests)",
+           "single_shot_ms": single_ms,
+           "single_shot": "one upload -> projection -> download on one stream, nothing overlapped (latency of one request)"}
     del cts, outs
     torch.cuda.empty_cache()
 
     isolated = isolated_kernels(ctx, fesc, torch, ct, out, hbm_peak, n) if (rank == 0 and args.scale_down == 1) else None
     variants = None
     if rank == 0 and args.scale_down == 1 and tbs % 2 == 0:
-        # the same 2048 x 768 -> 3352 job with token blocks (2u, 2u+1) paired in the real and imaginary channels:
-        # half the ciphertexts go through fesc_linear (real diagonals act on complex slots), then one conjugation
-        # per output separates the two results.  Reported beside the headline, which keeps one block per ciphertext.
-        conj_id = GIANT_BASE + 400
-        ctx.add_galois_key(fesc.CONJ, conj_id)
-        half = tbs // 2
-        desc2 = fesc.BsgsDesc(N1, N2, gin, nout, half, LEVEL, BABY_BASE, GIANT_BASE, int(args.hoist), int(args.defer),
-                              int(args.packed))
-        zc = torch.empty((half * nout, 2, LEVEL - 1, n), dtype=torch.int64, device=dev)
-        o2 = out.reshape(2, half * nout, 2, LEVEL - 1, n)
-
-        def paired():
-            ctx.linear(ct[:half], diags, desc2, zc)
-            ctx.split_complex(zc, o2[0], o2[1], half * nout, LEVEL - 1, conj_id)
-
-        paired()
-        c0 = ctx.counters()
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(args.steps):
-            paired()
-        e1.record()
-        torch.cuda.synchronize()
-        c1 = ctx.counters()
-        v_ms = e0.elapsed_time(e1) / args.steps
-        variants = {"paired_token_blocks": {"latency_ms": v_ms, "key_switches_per_step": (c1[1] - c0[1]) // args.steps,
-                                            "input_cts": half * gin, "output_cts": 2 * half * nout,
-                                            "note": "token blocks 2u and 2u+1 in the real and imaginary channels; "
-                                                    "fesc_linear on 8 complex token blocks + fesc_split_complex"}}
-        del zc
-        # the paper's own pairing (App. "Projection Kernel Breakdown"): input blocks 2u and 2u+1 in the real and
-        # imaginary channels with complex diagonals, real part of every output by one conjugation.  Timed on the same
-        # buffers reinterpreted as ceil(gin/2) input blocks (residues are random either way).
-        gp = -(-gin // 2)
-        if gp < gin:
-            desc3 = fesc.BsgsDesc(N1, N2, gp, nout, tbs, LEVEL, BABY_BASE, GIANT_BASE, int(args.hoist), int(args.defer),
-                                  int(args.packed))
-            ct3 = ct.reshape(-1)[: tbs * gp * 2 * LEVEL * n].view(tbs, gp, 2, LEVEL, n)
-            if args.packed:      # any bytes are valid byte planes: the head of the image serves as the smaller image
-                dg3 = diags[: ctx.linear_packed_bytes(desc3)]
-            else:
-                dg3 = diags.reshape(-1)[: nout * N2 * gp * N1 * LEVEL * n].view(nout, N2, gp, N1, LEVEL, n)
-            z3 = torch.empty((tbs * nout, 2, LEVEL - 1, n), dtype=torch.int64, device=dev)
-            o3 = out.reshape(tbs * nout, 2, LEVEL - 1, n)
-
-            def paired_in():
-                ctx.linear(ct3, dg3, desc3, z3)
-                ctx.split_complex(z3, o3, None, tbs * nout, LEVEL - 1, conj_id)
-
-            paired_in()
-            c0 = ctx.counters()
-            torch.cuda.synchronize()
-            e0.record()
-            for _ in range(args.steps):
-                paired_in()
-            e1.record()
-            torch.cuda.synchronize()
-            c1 = ctx.counters()
-            variants["paired_input_blocks"] = {
-                "latency_ms": e0.elapsed_time(e1) / args.steps, "key_switches_per_step": (c1[1] - c0[1]) // args.steps,
-                "input_cts": tbs * gp, "output_cts": tbs * nout,
-                "note": "input blocks 2u and 2u+1 in the real and imaginary channels, complex diagonals; "
-                        "fesc_linear on %d input blocks + real part by fesc_split_complex" % gp}
-            del z3
-
+        variants = measure_variants(args, ctx, ct, diags, out, gin, nout, tbs, n, dev)
+    stages = None
+    config_extra = {"l2": "inputs larger than L2 (diagonals %.1f GiB stream every step)" % (diags.numel() * diags.element_size() / 2**30),
+                    "diagonals_as": ("byte-plane image, %.1f GiB, packed once outside the timed region" % (diags.numel() / 2**30)
+                                     if args.packed else "residues")}
+    if rank == 0 and world == 1 and args.scale_down == 1 and args.stages and PROJ == "in_proj":
+        del ct, diags, out, h_in, h_out
+        torch.cuda.empty_cache()
+        ctx.trim()
+        stages = run_stages(args, ctx, dev)
     line = {
         "metric": METRIC, "value": value, "unit": "key-switches/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "latency_ms": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
-        "config": {"workload": "%s %d->%d, L=2048 tokens, N=2^16, 24x50-bit limbs + 4x60-bit special primes, "
-                               "6 key-switch digits, C=256 T=128 n1=%d n2=%d, baby rotations %s"
-                               % (PROJ, D_IN, D_OUT, N1, N2, "hoisted (one decomposition per input ciphertext)" if args.hoist else "by plain rotations")
-                               + (", one division by P per output for the giant-step sum" if args.defer else ""),
+        "config": {"workload": workload_text(args),
                    "input_cts": tbs * gin, "diagonals": nout * N2 * gin * N1, "output_cts": tbs * nout,
                    "key_switches_per_step": ks_per_step, "macs_per_step": tbs * nout * N2 * gin * N1,
-                   "l2": "inputs larger than L2 (diagonals %.1f GiB stream every step)" % (diags.numel() * 8 / 2**30),
+                   "l2": config_extra["l2"], "diagonals_as": config_extra["diagonals_as"],
+                   "token_blocks_per_group": tb_per_launch,
                    "parallelism": "replicas x%d (independent 2048-token batches)" % world},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-        "roofline": roof, "kernel_breakdown": breakdown,
+        "roofline": roof, "roofline_other": others, "kernel_breakdown": breakdown,
     }
     if isolated:
         line["isolated"] = isolated
     if variants:
         line["variants"] = variants
+    if stages:
+        line["stages"] = stages
     if args.scale_down > 1:
         line["config"]["workload"] += " [DEBUG scale_down=%d: not a reportable number]" % args.scale_down
     if rank == 0 and world == 1 and not args.no_cpu:
         v, ms, cores = oracle_sample(1, 0, bool(args.hoist), bool(args.defer))
         line["cpu_baseline"] = {"value": v, "unit": "key-switches/s", "cores": cores, "kind": "oracle",
-                                "sample": SAMPLE_TEXT, "ms": ms}
+                                "sample": SAMPLE_TEXT, "ms": ms, "rates": oracle_rates()}
     if rank == 0:
         print(json.dumps(line), flush=True)
     del ctx
@@ -660,7 +806,7 @@ def gather_chunk_outputs(local, parts, rank, world, K_blk, K_s):
     return full
 
 
-def run_scan(args):
+def run_scan(args, ctx=None, quiet=False):
     """Times fesc_scan_contract on synthetic residues of the deployed geometry (N=2^16, 24 limbs, stride 256,
     B_blk=256, d_s=128, P=64).  --workload scan_slice: 4 heads x 512 tokens; scan_layer: 24 heads x 2048 tokens.
     With --gpus N (one process per GPU) the state chunks are dealt out to the ranks in pairs (Alg. 7: chunks are
@@ -675,7 +821,8 @@ def run_scan(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     p = S.params("full")
-    ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+    if ctx is None:
+        ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
     n, N = ctx.N // 2, ctx.N
     H, L = (4, 512) if args.workload == "scan_slice" else (24, 2048)
     P, d_s, B, stride, l0 = 64, 128, 256, int(args.stride), int(args.scan_limbs)
@@ -698,9 +845,14 @@ def run_scan(args):
         r = S.hashed_residues(seed, stream, q, count * 2 * N, device=dev)
         return r.view(l0, count, 2, N).permute(1, 2, 0, 3).contiguous()
 
-    def chunk_cts(stream):                                     # [K_blk][mine][segs] ciphertexts of this rank's chunks
-        full = cts(K_blk * K_s * segs, stream).view(K_blk, K_s, segs, 2, l0, N)
-        return full[:, first:first + mine].contiguous()
+    def chunk_cts(stream):                                     # [K_blk][mine][segs] ciphertexts of this rank's chunks only
+        out_c = torch.empty((K_blk, max(mine, 1), segs, 2, l0, N), dtype=torch.int64, device=dev)
+        for j in range(K_blk):                                 # ciphertext (block j, chunk k, segment g) = index (j*K_s + k)*segs + g
+            for k in range(mine):
+                lo = ((j * K_s + first + k) * segs) * 2 * N
+                r = S.hashed_residues(seed, stream, q, segs * 2 * N, device=dev, first=lo)
+                out_c[j, k] = r.view(l0, segs, 2, N).permute(1, 2, 0, 3)
+        return out_c
 
     x, a = chunk_cts(1), chunk_cts(2)
     Bc, Cc = cts(K_blk, 3), cts(K_blk, 4)
@@ -746,12 +898,15 @@ def run_scan(args):
     ctx.sync()
     barrier()
     c0 = ctx.counters()
+    sampler = ClockSampler(local)
+    sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     step()
     e1.record()
     ctx.sync()
     barrier()
+    clocks = sampler.stop()
     c1 = ctx.counters()
     ms = max_over_ranks(e0.elapsed_time(e1), dev)
     ks_local = torch.tensor([float(c1[1] - c0[1])], dtype=torch.float64, device=dev)
@@ -759,8 +914,9 @@ def run_scan(args):
         import torch.distributed as dist
         dist.all_reduce(ks_local)
     ks = int(ks_local.item())
+    res = None
     if rank == 0:
-        print(json.dumps({"metric": "scan-contract key-switches/s", "value": ks / (ms * 1e-3), "unit": "key-switches/s",
+        res = ({"metric": "scan-contract key-switches/s", "value": ks / (ms * 1e-3), "unit": "key-switches/s",
                           "n_gpus": world, "steps": 1, "warmup": 1 if args.workload == "scan_slice" else 0,
                           "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "dtype": "u64",
                           "data": "synthetic",
@@ -772,7 +928,10 @@ def run_scan(args):
                                      "parallelism": "state chunks in pairs over %d rank(s): %s; one all-gather of the outputs"
                                                     % (world, [c for _, c in parts])},
                           "key_switches": ks, "limb_transforms": c1[0] - c0[0], "gpu_launches": c1[4] - c0[4],
-                          "scratch_gib": c1[3] / 2**30, "kernel_breakdown": breakdown}), flush=True)
+                          "scratch_gib": c1[3] / 2**30, "clocks": clocks, "kernel_breakdown": breakdown})
+        if not quiet:
+            print(json.dumps(res), flush=True)
+    return res
 
 
 def run_rotations(args):
@@ -838,16 +997,17 @@ def run_rotations(args):
                       "layouts": res}), flush=True)
 
 
-def run_conv(args):
+def run_conv(args, ctx=None, quiet=False):
     """Times fesc_conv on synthetic residues of the Mamba-2-base shape: the xBC channels (1536 + 2*128 = 1792 = 7
     channel blocks of 256) x 2048 tokens (16 token blocks of 128), d_conv = 4, 24 limbs."""
     import torch
     import fesc_synth as S
     import paper_2608_17442_b200 as fesc
 
-    torch.cuda.set_device(0)
     p = S.params("full")
-    ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+    if ctx is None:
+        torch.cuda.set_device(0)
+        ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
     N = ctx.N
     d_conv, T, blocks, tbs, level, base = 4, T_SEG, 7, 16, LEVEL, 3000
     for r in range(1, d_conv):
@@ -871,26 +1031,31 @@ def run_conv(args):
     fam = ctx.profile_read()
     ctx.profile_enable([])
     c0 = ctx.counters()
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
         ctx.conv(ct, masks, bias, desc, out)
     e1.record()
     ctx.sync()
+    clocks = sampler.stop()
     c1 = ctx.counters()
     ms = e0.elapsed_time(e1) / args.steps
     ks = (c1[1] - c0[1]) // args.steps
-    print(json.dumps({"metric": "causal depthwise convolution latency; key-switches/s", "value": ks / (ms * 1e-3),
+    res = ({"metric": "causal depthwise convolution latency; key-switches/s", "value": ks / (ms * 1e-3),
                       "unit": "key-switches/s", "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup),
                       "ms_per_step": ms, "higher_is_better": True, "dtype": "u64", "data": "synthetic",
                       "config": {"workload": "conv: 1792 channels x 2048 tokens, d_conv=4, T=128, 7 channel blocks x 16 "
                                              "token blocks, N=2^16, 24 limbs, hoisted rotations"},
-                      "key_switches_per_step": ks, "gpu_launches": (c1[4] - c0[4]) // args.steps,
-                      "kernel_breakdown": {k: {"ms": round(v[0], 2), "records": v[1]} for k, v in fam.items() if v[1]}}),
-          flush=True)
+                      "key_switches_per_step": ks, "gpu_launches": (c1[4] - c0[4]) // args.steps, "clocks": clocks,
+                      "kernel_breakdown": {k: {"ms": round(v[0], 2), "records": v[1]} for k, v in fam.items() if v[1]}})
+    if not quiet:
+        print(json.dumps(res), flush=True)
+    return res
 
 
-def run_norm(args):
+def run_norm(args, ctx=None, quiet=False):
     """Times the CKKS steps around the NeRMS protocol on synthetic residues of the Mamba-2-base shape: 1536 channels
     (6 channel blocks of 256) x 2048 tokens (16 token blocks of 128), 24 limbs: fesc_norm_square on the 96
     ciphertexts, then fesc_norm_scale (8 rotate-and-add steps per token block, 96 ciphertext products, 96 plaintext
@@ -899,9 +1064,10 @@ def run_norm(args):
     import fesc_synth as S
     import paper_2608_17442_b200 as fesc
 
-    torch.cuda.set_device(0)
     p = S.params("full")
-    ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+    if ctx is None:
+        torch.cuda.set_device(0)
+        ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
     N = ctx.N
     T, blocks, tbs, level, base = T_SEG, 6, 16, LEVEL, 3500
     steps_fill = (N // 2 // T).bit_length() - 1
@@ -931,23 +1097,69 @@ def run_norm(args):
     fam = ctx.profile_read()
     ctx.profile_enable([])
     c0 = ctx.counters()
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
         step()
     e1.record()
     ctx.sync()
+    clocks = sampler.stop()
     c1 = ctx.counters()
     ms = e0.elapsed_time(e1) / args.steps
     ks = (c1[1] - c0[1]) // args.steps
-    print(json.dumps({"metric": "NeRMS-side CKKS steps latency; key-switches/s", "value": ks / (ms * 1e-3),
+    res = ({"metric": "NeRMS-side CKKS steps latency; key-switches/s", "value": ks / (ms * 1e-3),
                       "unit": "key-switches/s", "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup),
                       "ms_per_step": ms, "higher_is_better": True, "dtype": "u64", "data": "synthetic",
                       "config": {"workload": "norm: squares and gamma (.) (y (.) br(s)) for 1536 channels x 2048 tokens, "
                                              "T=128, 6 channel blocks x 16 token blocks, N=2^16, 24 limbs"},
-                      "key_switches_per_step": ks, "gpu_launches": (c1[4] - c0[4]) // args.steps,
-                      "kernel_breakdown": {k: {"ms": round(v[0], 2), "records": v[1]} for k, v in fam.items() if v[1]}}),
-          flush=True)
+                      "key_switches_per_step": ks, "gpu_launches": (c1[4] - c0[4]) // args.steps, "clocks": clocks,
+                      "kernel_breakdown": {k: {"ms": round(v[0], 2), "records": v[1]} for k, v in fam.items() if v[1]}})
+    if not quiet:
+        print(json.dumps(res), flush=True)
+    return res
+
+
+def run_stages(args, ctx, dev):
+    """The other CKKS stages of one Mamba-2-base layer at L = 2048 (workload 5), timed one after the other on the same
+    context after the headline's buffers have been released: out_proj 1536 -> 768 (its own packed diagonals), the causal
+    depthwise convolution, the products around the normalisation, and a slice of the scan-contract (4 heads x 512
+    tokens of the deployed geometry; the whole layer takes about a minute and runs with --workload scan_layer or
+    --scan-layer 1).  Each stage: CUDA-event time, key switches, clocks sampled during its timed region, family times."""
+    import argparse as _ap
+    import torch
+
+    global D_IN, D_OUT, PROJ, N1, N2
+    stages = {}
+    sub = _ap.Namespace(**vars(args))
+    sub.steps, sub.warmup = 3, 3
+
+    def keep(res, extra=None):
+        out = {"ms": res["ms_per_step"], "key_switches": res.get("key_switches_per_step", res.get("key_switches")),
+               "key_switches_per_s": res["value"], "gpu_launches": res.get("gpu_launches"), "clocks": res.get("clocks"),
+               "kernel_breakdown": res.get("kernel_breakdown"), "workload": res["config"]["workload"]}
+        out.update(extra or {})
+        return out
+
+    # out_proj: 6 input blocks x 3 output blocks, 16 x 16 baby / giant split
+    saved = (D_IN, D_OUT, PROJ, N1, N2)
+    D_IN, D_OUT, PROJ, N1, N2 = 1536, 768, "out_proj", 16, 16
+    try:
+        stages["out_proj"] = measure_projection(sub, ctx, dev, rank=0, world=1, key_base=(BABY_BASE + 2000, GIANT_BASE + 2000))
+    finally:
+        D_IN, D_OUT, PROJ, N1, N2 = saved
+    torch.cuda.empty_cache()
+    ctx.trim()
+    stages["conv"] = keep(run_conv(sub, ctx, quiet=True))
+    torch.cuda.empty_cache()
+    stages["norm"] = keep(run_norm(sub, ctx, quiet=True))
+    torch.cuda.empty_cache()
+    ctx.trim()
+    sub.workload = "scan_layer" if args.scan_layer else "scan_slice"
+    r = run_scan(sub, ctx, quiet=True)
+    stages[sub.workload] = keep(r, {"scratch_gib": r["scratch_gib"], "limb_transforms": r["limb_transforms"]})
+    return stages
 
 
 def main():
@@ -967,6 +1179,11 @@ def main():
     ap.add_argument("--packed", type=int, default=1, choices=[0, 1],
                     help="1: the diagonals are packed once into byte-plane operand tiles (fesc_linear_pack_diags) and the "
                          "accumulate runs on the tensor cores; 0: residues as encoded")
+    ap.add_argument("--stages", type=int, default=1, choices=[0, 1],
+                    help="1: after the headline, time the other CKKS stages of a layer (out_proj, conv, norm, scan slice) "
+                         "and report them under `stages`")
+    ap.add_argument("--scan-layer", dest="scan_layer", type=int, default=0, choices=[0, 1],
+                    help="1: the scan stage of `stages` is the whole layer (24 heads x 2048 tokens, about a minute) instead of the slice")
     ap.add_argument("--hoist", type=int, default=1, choices=[0, 1],
                     help="1: baby rotations share one decomposition per input ciphertext (fesc_rotate_hoisted)")
     ap.add_argument("--group", type=int, default=4, choices=[0, 2, 4, 8, 16],
