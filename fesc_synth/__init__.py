@@ -100,12 +100,12 @@ def params(name: str) -> dict:
         special = ntt_primes(60, 10, 4, seed)
         return dict(name=name, log_n=10, primes=data + special, n_q=24, n_p=4, dnum=6,
                     seed=seed, log_scale=40)
-    if name == "small_d12":
-        # the small ring with 12 key-switch digits of two limbs (more digits than one FP64 fold-back interval)
+    if name == "small_d9":
+        # the small ring with 9 key-switch digits of two limbs (more digits than one FP64 fold-back interval)
         seed = config_seed(0)
-        data = ntt_primes(50, 10, 24, seed)
+        data = ntt_primes(50, 10, 18, seed)
         special = ntt_primes(60, 10, 2, seed)
-        return dict(name=name, log_n=10, primes=data + special, n_q=24, n_p=2, dnum=12, seed=seed, log_scale=40)
+        return dict(name=name, log_n=10, primes=data + special, n_q=18, n_p=2, dnum=9, seed=seed, log_scale=40)
     if name in ("scan_toy", "scan_small"):
         # rings for the scan-contract tests: the paper's toy shape (16 slots) and a 128-slot analogue of
         # the Mamba-2-base geometry; 50-bit chain, two 60-bit special primes, two limbs per digit

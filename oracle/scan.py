@@ -56,6 +56,18 @@ tokens = G d_s consecutive slots, mask [0, G d_s), log2(n/(G d_s)) steps, class 
 at l0-2 where the leaves need it; br(C_t) keeps the token-by-token build (its fill runs at the injection level, where
 rotations are cheap).
 
+Invariant families (App. "Invariant Families", "Shared HEScan Kernel Backend"; `plain` = (abar, Bbar, Cbar); S4D / S5 /
+LRU rows of Table "cross_ssm_family").  The decay abar[i] (per state coordinate), the input factor Bbar[i] and the output
+factor Cbar[i] are server-held plaintexts that do not depend on the token; only x_k is encrypted:
+    h_k[e,i] = abar[i] h_{k-1}[e,i] + x_k[e] Bbar[i],     m_k[e] = sum_i h_k[e,i] Cbar[i].
+The affine packet loses its decay component: the decay over a span of m tokens is the plaintext abar^m, so a composition
+is  s <- abar^m (.) s_L + s_R  with ONE ct-pt product and no ciphertext product anywhere ("Affine relin." 0 in the
+paper's table).  Everything else (layouts, br(x_t), Brent-Kung schedule, levels, carries, reduction) is the dataflow
+above with plaintexts in place of br(a), br(B), br(C): leaf s_t = br(x_t) (.) Bbar; up-sweep stage s and the down-sweep
+stage over the same span use abar^(2^(s-1)); the carry uses abar^B; the injection of token t uses abar^(t+1); the
+contraction uses Cbar.  Every plaintext is a slot pattern e'*stride + i -> v[i] encoded at scale S_p of the level where
+it is used.
+
 Other prefix networks (App. "Prefix-Network Selection"; `network` = "ks" Kogge-Stone, "sk" Sklansky; "bk" above is the
 default): stage s = 1..logB combines operands at l1-(s-1) into results at l1-s, every prefix is complete at lS and there
 is no down-sweep, so linj = lS - max(K_blk-2, 0) (the carry before the last block still sits at or above linj).
@@ -81,6 +93,18 @@ def float_recurrence(x, a, B, C):
     for k in range(L):
         h = a[k][:, None, None] * h + x[k][:, :, None] * B[k, 0][None, None, :]
         m[k] = h @ C[k, 0]
+    return m
+
+
+def float_recurrence_invariant(x, abar, Bbar, Cbar):
+    """Invariant families (App. "Invariant Families"): m[k,h,p] = sum_i h_k[h,p,i] Cbar[i],
+    h_k[h,p,i] = abar[i] h_{k-1}[h,p,i] + x_k[h,p] Bbar[i]  (float64, sequential)."""
+    L, H, P = x.shape
+    h = np.zeros((H, P, len(abar)))
+    m = np.zeros((L, H, P))
+    for k in range(L):
+        h = abar[None, None, :] * h + x[k][:, :, None] * Bbar[None, None, :]
+        m[k] = h @ Cbar
     return m
 
 
@@ -174,9 +198,11 @@ def levels(l0: int, logB: int, K_blk: int, network: str = "bk", group: int = 0):
 class ScanConsts:
     """Harness-side constants: canonical scales, level-adjust integers, mask plaintexts."""
 
-    def __init__(self, orc: Oracle, shape: ScanShape, l0: int, log_scale: int, network: str = "bk", group: int = 0):
+    def __init__(self, orc: Oracle, shape: ScanShape, l0: int, log_scale: int, network: str = "bk", group: int = 0,
+                 plain=None):
+        """plain = (abar, Bbar, Cbar), three float vectors of length d_s: the invariant-family mode (module header)."""
         q = orc.q
-        self.network, self.group = network, group
+        self.network, self.group, self.plain = network, group, plain is not None
         self.lv = levels(l0, shape.logB, shape.K_blk, network, group)
         self.S_s = {l0: float(2**log_scale)}
         self.S_p = {l0: float(q[l0 - 1])}
@@ -213,6 +239,24 @@ class ScanConsts:
             self.mask_bg = orc.encode((slot < G * d_s).astype(float), self.S_p[l0], l0)
             self.mask_b2 = np.stack([orc.encode(((slot // d_s) % G == g).astype(float), self.S_p[l0 - 1], l0 - 1)
                                      for g in range(G)])
+        if plain is not None:
+            assert network == "bk", "the invariant-family mode uses the Brent-Kung schedule"
+            abar, Bbar, Cbar = (np.asarray(v, dtype=np.float64) for v in plain)
+            assert abar.shape == Bbar.shape == Cbar.shape == (shape.d_s,)
+            lv, B, logB = self.lv, shape.B, shape.logB
+
+            def pt(vec, level):     # slot e'*stride + i -> vec[i], encoded where it multiplies
+                slots = np.zeros((shape.c_state, st))
+                slots[:, :shape.d_s] = vec[None, :]
+                return orc.encode(slots.reshape(-1), self.S_p[level], level)
+
+            lx = l0 - 2 if group else l0 - 1                       # level of br(x_t)
+            self.pt_b = pt(Bbar, lx)
+            self.pt_c = pt(Cbar, lv["linj"] - 1)
+            self.pt_up = {s: pt(abar ** (1 << (s - 1)), lv["l1"] - (s - 1)) for s in range(1, logB + 1)}
+            self.pt_down = {d: pt(abar ** (1 << (logB - d - 1)), lv["lS"] - (d - 1)) for d in range(1, logB)}
+            self.pt_carry = {j: pt(abar ** B, lv["lS"] - (j - 1)) for j in range(1, shape.K_blk - 1)}
+            self.pt_inj = [pt(abar ** (t + 1), lv["linj"]) for t in range(B)] if shape.K_blk > 1 else []
         lred, lout = self.lv["linj"] - 2, self.lv["lout"]
         # the unpacked reduction carries a factor 2 (Re*2, Im*2); the output mask removes it and lands on S_s[lout]
         self.out_mask_scale = self.S_s[lout] * q[lout] / (2.0 * self.S_s[lred])
@@ -269,6 +313,21 @@ def encrypt_inputs(orc: Oracle, shape: ScanShape, consts: ScanConsts, x, a, B, C
     ctB = np.stack([enc(Bc[j], consts.S_p[l0]) for j in range(shape.K_blk)])
     ctC = np.stack([enc(Cc[j], consts.S_p[l0]) for j in range(shape.K_blk)])
     return ctX, ctA, ctB, ctC
+
+
+def encrypt_x(orc: Oracle, shape: ScanShape, consts: ScanConsts, x, nonce0: int = 50000):
+    """Invariant-family mode: only the scan input is encrypted.  [K_blk, K_s, segs, 2, l0, N], the layout of X above."""
+    l0 = consts.lv["l0"]
+    X, _, _, _ = pack_inputs(shape, x, np.zeros((shape.L, shape.H)), np.zeros((shape.L, 1, shape.d_s)),
+                             np.zeros((shape.L, 1, shape.d_s)))
+    nonce = nonce0
+    rows = []
+    for j in range(shape.K_blk):
+        for k in range(shape.K_s):
+            for g in range(shape.segs):
+                nonce += 1
+                rows.append(orc.encrypt(orc.encode(X[j, k, g], consts.S_s[l0], l0), nonce))
+    return np.stack(rows).reshape(shape.K_blk, shape.K_s, shape.segs, 2, l0, orc.N)
 
 
 def unpack_output(orc: Oracle, shape: ScanShape, consts: ScanConsts, out):
@@ -546,6 +605,74 @@ class ScanEvaluator:
                         lg = g.shape[1]
                         carry[kap] = self.add(self.mul_rescale(self.adjust(summary[0], lg, "p"), g),
                                               self.adjust(summary[1], lg - 1, "s"))
+            self.contract_block(j, v, out)
+        return out
+
+    # -- invariant families: plaintext decay, input factor and output factor -----------------------
+    def compose_plain(self, sL, sR, lvl, pt):
+        """s <- abar^span (.) s_L + s_R with operands brought to lvl (one ct-pt product); result at lvl-1."""
+        self.count["compose"] += 1
+        return self.add(self.ptmul_rescale(self.adjust(sL, lvl, "s"), pt), self.adjust(sR, lvl - 1, "s"))
+
+    def leaves_plain(self, ctX):
+        """s_t = br(x_t) (.) Bbar at l1 for the tokens of one (block, chunk); br(x_t) as in `leaves` / `leaves_grouped`."""
+        sh, c, G = self.sh, self.c, self.group
+        lg = lambda v: int(math.log2(v))
+        T = []
+        for seg in range(sh.segs):
+            if G:
+                gx = self.extract_all(ctX[seg], G, sh.Bt // G)
+                for u in range(sh.Bt // G):
+                    xg = self.fill_right(self.ptmul_rescale(gx[u], c.mask_xg), G, lg(sh.d_s // G))
+                    T += [self.ptmul_rescale(b, c.pt_b) for b in self.class_broadcasts(xg, c.mask_x2, 1)]
+            else:
+                ex = self.extract_all(ctX[seg], 1, sh.Bt)
+                for tt in range(sh.Bt):
+                    xr = self.fill_right(self.ptmul_rescale(ex[tt], c.mask_x), 1, lg(sh.d_s))
+                    T.append(self.ptmul_rescale(xr, c.pt_b))
+        return T
+
+    def brent_kung_plain(self, T):
+        """In-place inclusive prefixes of the state inputs T[0..B-1]; returns the block summary (level lS)."""
+        sh, c = self.sh, self.c
+        B, logB, l1, lS = sh.B, sh.logB, c.lv["l1"], c.lv["lS"]
+        for s in range(1, logB + 1):
+            for k in range(1 << s, B + 1, 1 << s):
+                T[k - 1] = self.compose_plain(T[k - (1 << (s - 1)) - 1], T[k - 1], l1 - (s - 1), c.pt_up[s])
+        summary = T[B - 1]
+        d = 0
+        for s in range(logB - 1, 0, -1):
+            d += 1
+            for k in range(1 << s, B, 1 << s):
+                r = k + (1 << (s - 1))
+                if r < B:
+                    T[r - 1] = self.compose_plain(T[k - 1], T[r - 1], lS - (d - 1), c.pt_down[d])
+        return summary
+
+    def run_plain(self, ctX):
+        """Invariant-family scan-contract (module header): ctX [K_blk, K_s, segs, 2, l0, N] -> out as in `run`."""
+        sh, c, o = self.sh, self.c, self.o
+        assert c.plain
+        linj, lout = c.lv["linj"], c.lv["lout"]
+        out = np.zeros((sh.K_blk, sh.K_s, sh.segs, 2, lout, o.N), dtype=np.uint64)
+        carry = [None] * sh.K_s
+        for j in range(sh.K_blk):
+            v = [[None] * sh.K_s for _ in range(sh.B)]
+            for kap in range(sh.K_s):
+                T = self.leaves_plain(ctX[j, kap])
+                summary = self.brent_kung_plain(T)
+                g = carry[kap]
+                for t in range(sh.B):
+                    h = self.adjust(T[t], linj - 1, "s")
+                    if g is not None:       # state = abar^(t+1) (.) g_j + s_t
+                        h = self.add(self.ptmul_rescale(self.adjust(g, linj, "s"), c.pt_inj[t]), h)
+                    v[t][kap] = self.ptmul_rescale(h, c.pt_c)              # level linj-2
+                if j + 1 < sh.K_blk:                                       # serialized carry g_{j+1} = abar^B g_j + s_S
+                    if g is None:
+                        carry[kap] = summary
+                    else:
+                        lg = g.shape[1]
+                        carry[kap] = self.add(self.ptmul_rescale(g, c.pt_carry[j]), self.adjust(summary, lg - 1, "s"))
             self.contract_block(j, v, out)
         return out
 

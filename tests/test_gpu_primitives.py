@@ -553,15 +553,16 @@ def test_results_do_not_depend_on_the_run_or_the_stream():
 
 
 def test_inner_product_worst_case_residues_with_many_digits():
-    """Largest possible partial sums of the key inner product: 12 digits (the FP64 path folds back after every 8
-    products), every residue of the switched polynomial equal to q - 1, plain and hoisted; bit-exact."""
+    """Largest possible partial sums of the key inner product: 9 digits (the FP64 path folds back after every 7
+    products, so a second interval starts), every residue of the switched polynomial equal to q - 1, plain and
+    hoisted; bit-exact."""
     import torch
 
-    pair = ctx_pair("small_d12")
+    pair = ctx_pair("small_d9")
     ctx, orc, p = pair
     add_key(pair, 1, 91)
     add_key(pair, 2, 92)
-    level, batch = 24, 2
+    level, batch = 18, 2
     ct = random_ct(orc, 51, level, level, batch)
     qs = np.array(orc.q[:level], dtype=np.uint64)
     ct[:, 1] = (qs - 1)[None, :, None]                  # c1 = q - 1 everywhere (the automorphism leaves it so)

@@ -8,8 +8,8 @@ import pytest
 
 import fesc_synth as S
 from oracle.ckks import Oracle
-from oracle.scan import (ScanConsts, ScanEvaluator, ScanShape, add_scan_keys, closed_form_counts, encrypt_inputs,
-                         float_recurrence, levels, unpack_output)
+from oracle.scan import (ScanConsts, ScanEvaluator, ScanShape, add_scan_keys, closed_form_counts, encrypt_inputs, encrypt_x,
+                         float_recurrence, float_recurrence_invariant, levels, unpack_output)
 
 
 def test_recurrence_matches_unrolled_closed_form():
@@ -238,3 +238,77 @@ def test_full_slot_variant_with_token_segments():
     # deployed ring: K_s = 6 chunks of 4 heads, two segments of 128 tokens
     big = ScanShape(32768, L=2048, H=24, P=64, d_s=128, B_blk=256, stride=128)
     assert (big.K_s, big.segs, big.Bt, big.c_state, big.hpc, big.R) == (6, 2, 128, 256, 4, 8192)
+
+
+# ---------------------------------------------------------------------------------------------------------------------
+# invariant families (App. "Invariant Families"): plaintext decay, input factor and output factor
+# ---------------------------------------------------------------------------------------------------------------------
+def _invariant_factors(seed, d_s):
+    g = S.rng(seed, 300)
+    return g.uniform(0.9, 1.0, d_s), g.standard_normal(d_s) * 0.5, g.standard_normal(d_s) * 0.5
+
+
+def test_invariant_recurrence_closed_form_and_reduction_to_the_selective_one():
+    x, _, _, _ = S.scan_inputs(5, 11, 2, 3, 1, 4)
+    abar, Bbar, Cbar = _invariant_factors(5, 4)
+    m = float_recurrence_invariant(x, abar, Bbar, Cbar)
+    # unrolled: m_k[e] = sum_i Cbar_i Bbar_i sum_{j<=k} abar_i^(k-j) x_j[e]
+    for k in (0, 3, 10):
+        want = sum((Cbar * Bbar * abar ** (k - j)).sum() * x[j] for j in range(k + 1))
+        assert np.allclose(m[k], want, rtol=1e-12, atol=1e-12)
+    # a decay that is the same for every state coordinate is the selective recurrence with constant factors
+    alpha = 0.93
+    a = np.full((11, 2), alpha)
+    Bk, Ck = np.tile(Bbar, (11, 1, 1)), np.tile(Cbar, (11, 1, 1))
+    assert np.allclose(float_recurrence_invariant(x, np.full(4, alpha), Bbar, Cbar), float_recurrence(x, a, Bk, Ck),
+                       rtol=1e-12, atol=1e-12)
+
+
+def _run_plain(name, hoist=False, group=0, **shape_kw):
+    p = S.params(name)
+    orc = Oracle(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+    sh = ScanShape(orc.n, **shape_kw)
+    x, _, _, _ = S.scan_inputs(p["seed"], sh.L, sh.H, sh.P, 1, sh.d_s)
+    fac = _invariant_factors(p["seed"], sh.d_s)
+    c = ScanConsts(orc, sh, p["n_q"], p["log_scale"], "bk", group, plain=fac)
+    add_scan_keys(orc, sh, hoist=hoist, group=group)
+    ev = ScanEvaluator(orc, sh, c, hoist=hoist)
+    out = ev.run_plain(encrypt_x(orc, sh, c, x))
+    return sh, ev, unpack_output(orc, sh, c, out), float_recurrence_invariant(x, *fac)
+
+
+def test_invariant_scan_matches_the_recurrence_without_any_ciphertext_product():
+    """Toy shape; three blocks with carries and a partial last block; grouped leaves with hoisted rotations; every slot
+    in use with token segments.  No relinearisation anywhere (the table's "Affine relin." 0), the Brent-Kung
+    composition count of the selective scan, and fewer rotations (no br(a), br(B), br(C))."""
+    sh, ev, m, ref = _run_plain("scan_toy", L=4, H=2, P=4, d_s=2, B_blk=4)
+    assert ev.count["ctmul"] == 0 and ev.count["compose"] == closed_form_counts(sh)["compose"] == 8
+    assert np.abs(m - ref).max() < 2.0**-24
+    kw = dict(L=40, H=8, P=4, d_s=8, B_blk=16)
+    sh, ev, m, ref = _run_plain("scan_small", **kw)
+    cf = closed_form_counts(sh)
+    assert ev.count["ctmul"] == 0 and ev.count["compose"] == cf["compose"] == 312
+    assert ev.count["conj"] == cf["reduce_conj"] == 96
+    lg = lambda v: int(math.log2(v))
+    # rotations: extraction and fill of br(x_t), state-axis reduction, output placement; nothing for a, B, C
+    extract_fill = sh.K_blk * sh.K_s * ((sh.B - 1) + sh.B * lg(sh.d_s))
+    assert ev.count["rot"] == extract_fill + cf["reduce_rot"] + sh.K_blk * sh.K_s * (sh.B - 1)
+    assert np.abs(m - ref).max() < 2.0**-22
+    _, ev_g, m_g, _ = _run_plain("scan_small", hoist=True, group=4, **kw)
+    assert ev_g.count["ctmul"] == 0 and np.abs(m_g - ref).max() < 2.0**-22
+    sh2, ev2, m2, _ = _run_plain("scan_small", hoist=True, group=4, stride=8, **kw)
+    assert (sh2.K_s, sh2.segs) == (2, 2) and ev2.count["ctmul"] == 0 and np.abs(m2 - ref).max() < 2.0**-22
+
+
+def test_invariant_rows_of_the_paper_table():
+    """Table "cross_ssm_family", S4D / S5 / LRU rows: d_s, K_s at E = 1536 channels, and 0 affine relinearisations."""
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "cross_ssm_family.txt")
+    rows = [[int(v) for v in line.split()[1:]] for line in open(path) if line.startswith("#inv")]
+    assert rows == [[64, 6, 0], [128, 12, 0], [128, 12, 0]]
+    # the paper's state chunks hold s_state = 16384 = n/2 slots: K_s = E d_s / s_state
+    for d_s, K_s, relin in rows:
+        assert 1536 * d_s // 16384 == K_s and relin == 0
+    # this build's layouts at L = 128: S4D (d_s = 64) with one block of 128 tokens, S5 / LRU (d_s = 128) with stride 256
+    assert ScanShape(32768, L=128, H=24, P=64, d_s=64, B_blk=128).K_s == 6
+    assert ScanShape(32768, L=128, H=24, P=64, d_s=128, B_blk=128, stride=256).K_s == 12
