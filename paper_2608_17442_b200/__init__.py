@@ -52,12 +52,13 @@ class NormDesc(ctypes.Structure):
 
 class ScanDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint32) for n in ("L", "H", "P", "d_s", "B_blk", "stride", "n_limbs", "key_base",
-                                                       "hoist", "network", "group")]
+                                                       "hoist", "network", "group", "plain")]
 
 
 class ScanConsts(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("d_mask_x", "d_mask_b", "d_mask_a", "d_mask_out", "adj_s", "adj_p",
-                                               "d_mask_xg", "d_mask_ag", "d_mask_x2", "d_mask_a2", "d_mask_bg", "d_mask_b2")]
+                                               "d_mask_xg", "d_mask_ag", "d_mask_x2", "d_mask_a2", "d_mask_bg", "d_mask_b2",
+                                               "d_pt_b", "d_pt_c", "d_pt_up", "d_pt_down", "d_pt_carry", "d_pt_inj")]
 
 
 def lib():
@@ -292,14 +293,18 @@ class Context:
         self._chk(lib().fesc_ctx_test_fail_allocs(self.h, count))
 
     def scan_contract(self, x, a, B, C, desc: ScanDesc, mask_x, mask_b, mask_a, mask_out, adj_s, adj_p, m_out,
-                      group_masks=None):
-        """adj_s / adj_p: sequences of (n_limbs+1)^2 Python ints (host tables); masks: CUDA tensors;
-        group_masks = (mask_xg, mask_ag, mask_x2, mask_a2, mask_bg, mask_b2) for desc.group > 0."""
+                      group_masks=None, plain_tables=None):
+        """adj_s / adj_p: sequences of (n_limbs+1)^2 Python ints (host tables); masks: CUDA tensors (None where the
+        mode does not use one); group_masks = (mask_xg, mask_ag, mask_x2, mask_a2, mask_bg, mask_b2) for desc.group > 0;
+        plain_tables = (pt_b, pt_c, pt_up, pt_down, pt_carry, pt_inj) for desc.plain = 1 (a, B, C may then be None)."""
         n = (desc.n_limbs + 1) ** 2
         hs = (ctypes.c_uint64 * n)(*[int(v) for v in adj_s])
-        hp = (ctypes.c_uint64 * n)(*[int(v) for v in adj_p])
-        cs = ScanConsts(mask_x.data_ptr(), mask_b.data_ptr(), mask_a.data_ptr(), mask_out.data_ptr(),
+        hp = (ctypes.c_uint64 * n)(*[int(v) for v in (adj_p if adj_p is not None else [0] * n)])
+        ptr = lambda t: t.data_ptr() if t is not None else None
+        cs = ScanConsts(ptr(mask_x), ptr(mask_b), ptr(mask_a), ptr(mask_out),
                         ctypes.cast(hs, ctypes.c_void_p).value, ctypes.cast(hp, ctypes.c_void_p).value,
-                        *([t.data_ptr() for t in group_masks] if group_masks else [None] * 6))
-        self._chk(lib().fesc_scan_contract(self.h, _ptr(x), _ptr(a), _ptr(B), _ptr(C), ctypes.byref(desc),
+                        *([ptr(t) for t in group_masks] if group_masks else [None] * 6),
+                        *([ptr(t) for t in plain_tables] if plain_tables else [None] * 6))
+        opt = lambda t: _ptr(t) if t is not None else None
+        self._chk(lib().fesc_scan_contract(self.h, _ptr(x), opt(a), opt(B), opt(C), ctypes.byref(desc),
                                            ctypes.byref(cs), _ptr(m_out), _stream()))

@@ -30,16 +30,16 @@ __global__ void __launch_bounds__(256) k_ct_addsub(const u64* __restrict__ a, si
     const u64 x = a[bi * a_stride + o], y = b[bi * b_stride + o];
     out[bi * out_stride + o] = sub ? submod(x, y, q) : addmod(x, y, q);
 }
-// out = ct (.) pt  (pt shared by the batch, [level][N])
+// out[b] = ct[b] (.) pt[b]  (pt [level][N]; pt_stride = 0: one plaintext for the batch; a_stride = 0: one ciphertext)
 __global__ void __launch_bounds__(256) k_ct_ptmul(const u64* __restrict__ a, size_t a_stride, const u64* __restrict__ pt,
-                                                  u64* __restrict__ out, size_t out_stride,
+                                                  size_t pt_stride, u64* __restrict__ out, size_t out_stride,
                                                   const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level) {
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t l = blockIdx.y, bi = blockIdx.z;
     if (c >= N) return;
     const PrimeConst pc = pcs[l];
     const size_t o = (size_t)l * N + c, poly = (size_t)level * N;
-    const u64 w = pt[o];
+    const u64 w = pt[bi * pt_stride + o];
     out[bi * out_stride + o] = mulmod(a[bi * a_stride + o], w, pc);
     out[bi * out_stride + poly + o] = mulmod(a[bi * a_stride + poly + o], w, pc);
 }
@@ -216,15 +216,18 @@ struct Exec {
         if (!ok() || dry) return;
         rc = rescale_internal(ctx, in.p, in.stride, out.p, in.count, in.level, rs, st);
     }
-    // out (level-1, contiguous) = rescale(in (.) pt)
-    void ptmul_rescale(const Arr& in, const u64* pt, const Arr& out) {
+    // out (level-1, contiguous) = rescale(in (.) pt); pt_stride != 0: plaintext i for element i; a single `in` with
+    // out.count plaintexts multiplies that one ciphertext by each of them
+    void ptmul_rescale(const Arr& in, const u64* pt, const Arr& out, size_t pt_stride = 0) {
         size_t mark = top;
-        Arr t = alloc(in.count, in.level);
+        const uint32_t cnt = out.count;
+        Arr t = alloc(cnt, in.level);
         if (ok() && !dry) {
             prof_begin(ctx, PF_POINTWISE, st);
-            k_ct_ptmul<<<grid(in.level, in.count), 256, 0, st>>>(in.p, in.stride, pt, t.p, t.stride, ctx->d_pc, N, in.level);
+            k_ct_ptmul<<<grid(in.level, cnt), 256, 0, st>>>(in.p, in.count == 1 && cnt > 1 ? 0 : in.stride, pt, pt_stride, t.p,
+                                                            t.stride, ctx->d_pc, N, in.level);
             prof_end(ctx, PF_POINTWISE, st);
-            ctx->counters[2] += in.count;
+            ctx->counters[2] += cnt;
         }
         rescale(t, out);
         top = mark;
@@ -411,8 +414,10 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
         const size_t block_mark = X.top;
         // ---- br(B_t) at l0-1 (l0-2 with the grouped leaf build) and br(C_t) at linj-1, shared by every chunk ----
         const uint32_t G = X.desc->group, lB = G ? l0 - 2 : l0 - 1;
-        Arr brB = X.alloc(B, lB), brC = X.alloc(B, linj - 1);
-        for (int which = 0; which < 2; which++) {
+        const bool plain = X.desc->plain != 0;      // invariant families: plaintext decay, B and C; nothing to broadcast
+        const size_t row0 = (size_t)l0 * N;         // pitch of the plaintext tables that hold one level per row
+        Arr brB = X.alloc(plain ? 0 : B, lB), brC = X.alloc(plain ? 0 : B, linj - 1);
+        for (int which = 0; which < 2 && !plain; which++) {
             size_t m = X.top;
             Arr src{const_cast<u64*>((which ? d_C : d_B) + (size_t)j * in_ctw), 1, l0, in_ctw};
             if (which == 0 && G) {
@@ -447,9 +452,30 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
         for (uint32_t kap = 0; kap < g.K_s && X.ok(); kap++) {
             const size_t chunk_mark = X.top;
             // position slots of the prefix network: capacity l1, current level tracked on the host
-            Arr Ps = X.alloc(B, l1), Ss = X.alloc(B, l1);
+            Arr Ps = X.alloc(plain ? 0 : B, l1), Ss = X.alloc(B, l1);
             std::vector<uint32_t> lp(B, l1), ls(B, l1);
-            if (G) {   // ---- leaves, grouped build: groups of G tokens share extraction, mask and fill ----
+            if (plain) {   // ---- leaves of the invariant families: s_t = br(x_t) (.) Bbar, no decay component ----
+                size_t m = X.top;
+                const size_t seg0 = ((size_t)j * g.K_s + kap) * g.segs;
+                Arr srcx{const_cast<u64*>(d_x + seg0 * in_ctw), g.segs, l0, in_ctw};
+                Arr xr = X.alloc(B, lB);
+                if (G) {
+                    const uint32_t ng = B / G, ngs = g.Bt / G;
+                    Arr ex = X.alloc(ng, l0), xg = X.alloc(ng, l0 - 1);
+                    for (uint32_t sg = 0; sg < g.segs; sg++) X.extract_n(X.at(srcx, sg), G, ngs, X.at(ex, sg * ngs, ngs));
+                    X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_xg, xg);
+                    X.fill_right(xg, G, ilog2(g.d_s / G));
+                    X.class_broadcasts(xg, (const u64*)X.cs->d_mask_x2, G, 1,
+                                       [&](uint32_t c, const Arr& res) { X.copy(res, X.strided(xr, c, G, ng)); });
+                } else {
+                    Arr ex = X.alloc(B, l0);
+                    for (uint32_t sg = 0; sg < g.segs; sg++) X.extract_n(X.at(srcx, sg), 1, g.Bt, X.at(ex, sg * g.Bt, g.Bt));
+                    X.ptmul_rescale(ex, (const u64*)X.cs->d_mask_x, xr);
+                    X.fill_right(xr, 1, ilog2(g.d_s));
+                }
+                X.ptmul_rescale(xr, (const u64*)X.cs->d_pt_b, Ss);
+                X.top = m;
+            } else if (G) {   // ---- leaves, grouped build: groups of G tokens share extraction, mask and fill ----
                 size_t m = X.top;
                 const uint32_t ng = B / G, ngs = g.Bt / G;      // groups per block / per segment
                 const size_t seg0 = ((size_t)j * g.K_s + kap) * g.segs;
@@ -495,10 +521,25 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
             }
             // ---- Brent-Kung network ----
             // one stage: nodes (left position, right position), operands brought to `lvl`, results at lvl-1
+            const u64* stage_pt = nullptr;          // invariant families: abar^span at the stage's level
             auto stage = [&](const std::vector<uint32_t>& left, const std::vector<uint32_t>& right, uint32_t lvl, bool need_p) {
                 const uint32_t cnt = (uint32_t)left.size();
                 if (!cnt || !X.ok()) return;
                 size_t m = X.top;
+                if (plain) {        // s <- abar^span (.) s_L + s_R: one ct-pt product per node
+                    Arr sL = X.alloc(cnt, lvl), sR = X.alloc(cnt, lvl - 1), ns = X.alloc(cnt, lvl - 1);
+                    X.adjust_many(Ss, left, ls, lvl, 0, sL);
+                    X.adjust_many(Ss, right, ls, lvl - 1, 0, sR);
+                    X.ptmul_rescale(sL, stage_pt, ns);
+                    X.add(ns, sR, ns);
+                    for (uint32_t i = 0; i < cnt; i++) {
+                        const uint32_t b = right[i];
+                        X.copy(X.at(ns, i), Arr{Ss.p + (size_t)b * Ss.stride, 1, lvl - 1, X.ctw(lvl - 1)});
+                        ls[b] = lvl - 1;
+                    }
+                    X.top = m;
+                    return;
+                }
                 Arr pL = X.alloc(cnt, lvl), sL = X.alloc(cnt, lvl), pR = X.alloc(cnt, lvl), sR = X.alloc(cnt, lvl - 1);
                 Arr np_ = X.alloc(cnt, lvl - 1), ns = X.alloc(cnt, lvl - 1);
                 if (need_p) X.adjust_many(Ps, left, lp, lvl, 1, pL);
@@ -541,12 +582,13 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
                     }
                 }
                 // the last stage of a one-pass network forms decay products only for an incoming state
+                if (plain) stage_pt = (const u64*)X.cs->d_pt_up + (size_t)(s - 1) * row0;
                 stage(left, right, l1 - (s - 1), network == FESC_NET_BRENT_KUNG || s < g.logB || j > 0);
             }
             // summary of the block = last position after the up-sweep (after the last stage of a one-pass network);
             // keep a copy for the carry (the first block's decay product is not used)
             Arr sumP = X.alloc(1, lS), sumS = X.alloc(1, lS);
-            if (network == FESC_NET_BRENT_KUNG || j > 0) X.copy(Arr{Ps.p + (size_t)(B - 1) * Ps.stride, 1, lS, X.ctw(lS)}, sumP);
+            if (!plain && (network == FESC_NET_BRENT_KUNG || j > 0)) X.copy(Arr{Ps.p + (size_t)(B - 1) * Ps.stride, 1, lS, X.ctw(lS)}, sumP);
             X.copy(Arr{Ss.p + (size_t)(B - 1) * Ss.stride, 1, lS, X.ctw(lS)}, sumS);
             uint32_t d = 0;
             for (uint32_t s = g.logB - 1; s >= 1 && network == FESC_NET_BRENT_KUNG; s--) {
@@ -559,6 +601,7 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
                         right.push_back(r - 1);
                     }
                 }
+                if (plain) stage_pt = (const u64*)X.cs->d_pt_down + (size_t)(d - 1) * row0;
                 stage(left, right, lS - (d - 1), j > 0);
             }
             // ---- carry injection and contraction with br(C_t) ----
@@ -569,13 +612,18 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
                 for (uint32_t t = 0; t < B; t++) every[t] = t;
                 X.adjust_many(Ss, every, ls, linj - 1, 0, h);
                 if (j > 0) {
-                    Arr pp = X.alloc(B, linj), gg = X.alloc(1, linj), pg = X.alloc(B, linj - 1);
-                    X.adjust_many(Ps, every, lp, linj, 1, pp);
+                    Arr pp = X.alloc(plain ? 0 : B, linj), gg = X.alloc(1, linj), pg = X.alloc(B, linj - 1);
                     X.adjust(Arr{carry.p + (size_t)kap * carry.stride, 1, carry_level[kap], X.ctw(carry_level[kap])}, linj, 0, gg);
-                    X.mul_rescale(pp, gg, pg);
+                    if (plain) {    // state_t = abar^(t+1) (.) g_j + s_t
+                        X.ptmul_rescale(gg, (const u64*)X.cs->d_pt_inj, pg, (size_t)linj * N);
+                    } else {
+                        X.adjust_many(Ps, every, lp, linj, 1, pp);
+                        X.mul_rescale(pp, gg, pg);
+                    }
                     X.add(h, pg, h);
                 }
-                X.mul_rescale(h, brC, X.at(V, (kap & 1) * B, B));
+                if (plain) X.ptmul_rescale(h, (const u64*)X.cs->d_pt_c, X.at(V, (kap & 1) * B, B));
+                else X.mul_rescale(h, brC, X.at(V, (kap & 1) * B, B));
                 X.top = m;
             }
             // ---- serialized carry g_{j+1} = S_j(g_j) ----
@@ -591,9 +639,13 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
                     size_t m = X.top;
                     Arr gcur{slot.p, 1, lg, X.ctw(lg)};
                     Arr pa = X.alloc(1, lg), sa = X.alloc(1, lg - 1), ng = X.alloc(1, lg - 1);
-                    X.adjust(sumP, lg, 1, pa);
                     X.adjust(sumS, lg - 1, 0, sa);
-                    X.mul_rescale(pa, gcur, ng);
+                    if (plain) {    // g_{j+1} = abar^B (.) g_j + s_S
+                        X.ptmul_rescale(gcur, (const u64*)X.cs->d_pt_carry + (size_t)j * row0, ng);
+                    } else {
+                        X.adjust(sumP, lg, 1, pa);
+                        X.mul_rescale(pa, gcur, ng);
+                    }
                     X.add(ng, sa, ng);
                     X.copy(ng, Arr{slot.p, 1, lg - 1, X.ctw(lg - 1)});
                     carry_level[kap] = lg - 1;
@@ -656,9 +708,13 @@ static int scan_run(Exec& X, const u64* d_x, const u64* d_a, const u64* d_B, con
 extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint64_t* d_a, const uint64_t* d_B,
                                   const uint64_t* d_C, const fesc_scan_desc* desc, const fesc_scan_consts* consts,
                                   uint64_t* d_m_out, void* stream) {
-    if (!ctx || !d_x || !d_a || !d_B || !d_C || !desc || !consts || !d_m_out) return FESC_EINVAL;
-    if (!consts->d_mask_x || !consts->d_mask_a || !consts->d_mask_b || !consts->d_mask_out || !consts->adj_s || !consts->adj_p)
+    if (!ctx || !d_x || !desc || !consts || !d_m_out) return FESC_EINVAL;
+    const bool plain = desc->plain != 0;
+    if (!plain && (!d_a || !d_B || !d_C)) return FESC_EINVAL;
+    if (!consts->d_mask_x || !consts->d_mask_out || !consts->adj_s || (!plain && (!consts->d_mask_a || !consts->d_mask_b || !consts->adj_p)))
         return fesc_fail(ctx, FESC_EINVAL, "scan_contract: missing constants");
+    if (plain && desc->network != FESC_NET_BRENT_KUNG)
+        return fesc_fail(ctx, FESC_EINVAL, "scan_contract: the invariant-family mode uses the Brent-Kung schedule");
     Geometry g;
     g.n = ctx->N / 2;
     g.L = desc->L, g.H = desc->H, g.P = desc->P, g.d_s = desc->d_s, g.B = desc->B_blk;
@@ -690,9 +746,9 @@ extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint
     if (G) {
         if (G < 2 || (G & (G - 1)) || G > 16 || G > g.Bt || G > g.d_s)
             return fesc_fail(ctx, FESC_EINVAL, "scan_contract: group must be a power of two, at most 16, the tokens of a segment and d_s");
-        if (!consts->d_mask_xg || !consts->d_mask_ag || !consts->d_mask_x2 || !consts->d_mask_a2 || !consts->d_mask_bg ||
-            !consts->d_mask_b2)
-            return fesc_fail(ctx, FESC_EINVAL, "scan_contract: the grouped leaf build needs its six mask arrays");
+        if (!consts->d_mask_xg || !consts->d_mask_x2 ||
+            (!plain && (!consts->d_mask_ag || !consts->d_mask_a2 || !consts->d_mask_bg || !consts->d_mask_b2)))
+            return fesc_fail(ctx, FESC_EINVAL, "scan_contract: the grouped leaf build needs its mask arrays");
     }
     if (g.l0 > ctx->n_q || g.l0 < g.logB + below_summary + 6 + (G ? 1 : 0))
         return fesc_fail(ctx, FESC_ELEVEL, "scan_contract: not enough levels");
@@ -702,6 +758,9 @@ extern "C" int fesc_scan_contract(fesc_ctx* ctx, const uint64_t* d_x, const uint
     g.lout = g.linj - 3;
     if (g.K_blk > 1 && g.lS < g.linj + (g.K_blk - 2))
         return fesc_fail(ctx, FESC_ELEVEL, "scan_contract: carry chain runs below the injection level");
+    if (plain && (!consts->d_pt_b || !consts->d_pt_c || !consts->d_pt_up || (g.logB > 1 && !consts->d_pt_down) ||
+                  (g.K_blk > 1 && !consts->d_pt_inj) || (g.K_blk > 2 && !consts->d_pt_carry)))
+        return fesc_fail(ctx, FESC_EINVAL, "scan_contract: the invariant-family mode needs its plaintext tables");
     Exec X;
     X.ctx = ctx, X.st = (cudaStream_t)stream, X.g = g, X.desc = desc, X.cs = consts;
     X.N = ctx->N, X.rc = FESC_OK;

@@ -81,3 +81,55 @@ def run_scan_parity(name, hoist=0, network="bk", group=0, **kw):
     assert np.array_equal(got, want)
     m = unpack_output(orc, sh, c, got)
     return np.abs(m - float_recurrence(x, a, B, C)).max()
+
+
+def run_scan_parity_invariant(name, hoist=0, group=0, seed_stream=300, **kw):
+    """The invariant-family mode (plaintext decay, input and output factors): fesc_scan_contract with desc.plain = 1
+    against ScanEvaluator.run_plain; asserts equal residues, returns the largest deviation of the decrypted result
+    from the float64 recurrence and the library's key-switch count."""
+    import torch
+    import fesc_synth as S
+    import paper_2608_17442_b200 as fesc
+    from oracle.ckks import CONJ
+    from oracle.scan import (ScanConsts, ScanEvaluator, ScanShape, add_scan_keys, encrypt_x, float_recurrence_invariant,
+                             key_id_for, unpack_output)
+
+    ctx, orc, p = ctx_pair(name)
+    sh = ScanShape(orc.n, **kw)
+    l0 = p["n_q"]
+    x, _, _, _ = S.scan_inputs(p["seed"] + sh.L, sh.L, sh.H, sh.P, 1, sh.d_s)
+    g = S.rng(p["seed"], seed_stream)
+    fac = (g.uniform(0.9, 1.0, sh.d_s), g.standard_normal(sh.d_s) * 0.5, g.standard_normal(sh.d_s) * 0.5)
+    c = ScanConsts(orc, sh, l0, p["log_scale"], "bk", group, plain=fac)
+    add_scan_keys(orc, sh, hoist=bool(hoist), group=group)
+    for r in sh.rotation_amounts(bool(hoist), group) + [CONJ]:
+        ctx.add_galois_key(r, key_id_for(sh, r))
+    ctX = encrypt_x(orc, sh, c, x)
+    ev = ScanEvaluator(orc, sh, c, hoist=bool(hoist))
+    want = ev.run_plain(ctX)
+    assert ev.count["ctmul"] == 0
+
+    def table(rows, count):       # {index: [level, N]} -> [count][l0][N], zero beyond each row's level
+        out = np.zeros((max(count, 1), l0, orc.N), dtype=np.uint64)
+        for i, v in rows.items():
+            out[i, :v.shape[0]] = v
+        return to_dev(out)
+
+    lv = c.lv
+    tables = (to_dev(c.pt_b), to_dev(c.pt_c), table({s - 1: v for s, v in c.pt_up.items()}, sh.logB),
+              table({d - 1: v for d, v in c.pt_down.items()}, sh.logB - 1), table(dict(c.pt_carry), sh.K_blk),
+              to_dev(np.stack(c.pt_inj)) if c.pt_inj else None)
+    adj_s = [c.adj_s.get((s, d), 0) for s in range(l0 + 1) for d in range(l0 + 1)]
+    out = torch.empty((sh.K_blk, sh.K_s, sh.segs, 2, lv["lout"], orc.N), dtype=torch.int64, device="cuda")
+    desc = fesc.ScanDesc(sh.L, sh.H, sh.P, sh.d_s, sh.B, kw.get("stride", 0), l0, 100000, hoist, fesc.NET_BRENT_KUNG, group, 1)
+    gm = [to_dev(c.mask_xg), None, to_dev(c.mask_x2), None, None, None] if group else None
+    ks0 = ctx.counters()[1]
+    ctx.scan_contract(to_dev(ctX), None, None, None, desc, to_dev(c.mask_x), None, None, to_dev(c.mask_out), adj_s, None,
+                      out, gm, tables)
+    ctx.sync()
+    ks = ctx.counters()[1] - ks0
+    got = to_host(out)
+    assert np.array_equal(got, want)
+    assert ks == ev.count["rot"] + ev.count["conj"]          # rotations and conjugations only: no relinearisation
+    m = unpack_output(orc, sh, c, got)
+    return np.abs(m - float_recurrence_invariant(x, *fac)).max()

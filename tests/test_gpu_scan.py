@@ -8,7 +8,7 @@ import fesc_synth as S
 from oracle.ckks import CONJ
 from oracle.scan import (ScanConsts, ScanEvaluator, ScanShape, add_scan_keys, encrypt_inputs, float_recurrence,
                          key_id_for, unpack_output)
-from tests.gpu_util import ctx_pair, run_scan_parity as _run, to_dev, to_host
+from tests.gpu_util import ctx_pair, run_scan_parity as _run, run_scan_parity_invariant as _run_inv, to_dev, to_host
 
 pytestmark = pytest.mark.gpu
 
@@ -52,6 +52,31 @@ def test_scan_grouped_leaf_build(hoist):
 def test_scan_full_slot_variant_with_token_segments(hoist, group):
     """stride = d_s < B_blk: two token segments per block, every slot of the state ciphertexts in use."""
     assert _run("scan_small", hoist, group=group, L=40, H=8, P=4, d_s=8, B_blk=16, stride=8) < 2.0**-22
+
+
+@pytest.mark.parametrize("hoist", [0, 1])
+def test_scan_invariant_families_plaintext_decay(hoist):
+    """desc.plain = 1 (S4D / S5 / LRU packets: plaintext abar, Bbar, Cbar, encrypted x): bit-exact against the oracle's
+    invariant-family mode on the toy shape, with carries over three blocks and a partial last block, with grouped
+    leaves, and with every slot in use; the library's key-switch count equals the oracle's rotations + conjugations
+    (no relinearisation anywhere)."""
+    assert _run_inv("scan_toy", hoist, L=4, H=2, P=4, d_s=2, B_blk=4) < 2.0**-24
+    assert _run_inv("scan_small", hoist, L=40, H=8, P=4, d_s=8, B_blk=16) < 2.0**-22
+    assert _run_inv("scan_small", hoist, group=4, L=40, H=8, P=4, d_s=8, B_blk=16) < 2.0**-22
+    assert _run_inv("scan_small", hoist, group=4, L=40, H=8, P=4, d_s=8, B_blk=16, stride=8) < 2.0**-22
+    assert _run_inv("scan_small", hoist, L=64, H=3, P=4, d_s=4, B_blk=32) < 2.0**-22
+
+
+def test_scan_invariant_mode_refuses_other_networks_and_missing_tables():
+    import torch
+    import paper_2608_17442_b200 as fesc
+    ctx, orc, p = ctx_pair("scan_toy")
+    z = torch.zeros(8, dtype=torch.int64, device="cuda")
+    for net, tables in ((fesc.NET_SKLANSKY, (z,) * 6), (fesc.NET_BRENT_KUNG, None)):
+        desc = fesc.ScanDesc(4, 2, 4, 2, 4, 0, p["n_q"], 100000, 0, net, 0, 1)
+        with pytest.raises(fesc.FescError) as e:
+            ctx.scan_contract(z, None, None, None, desc, z, None, None, z, [0], None, z, None, tables)
+        assert e.value.code == fesc.EINVAL
 
 
 def test_scan_unknown_network_is_refused():
