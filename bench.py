@@ -871,12 +871,18 @@ def run_scan(args, ctx=None, quiet=False):
               S.hashed_residues(seed, 25, q[:l0 - 1], G * N, device=dev).view(l0 - 1, G, N).permute(1, 0, 2).contiguous()]
     out = torch.empty((K_blk, max(mine, 1), segs, 2, linj - 3, N), dtype=torch.int64, device=dev)
     adj = [(1 << 49) + 12345 * i for i in range((l0 + 1) ** 2)]
-    desc = fesc.ScanDesc(L, mine * hpc, P, d_s, B, stride, l0, base, int(args.hoist), net, G)
+    plain = int(getattr(args, "plain", 0))
+    pts = None
+    if plain:       # invariant families: plaintext tables (abar powers, Bbar, Cbar) in place of the a, B, C ciphertexts
+        rows = lambda stream, count, lim: S.hashed_residues(seed, stream, q[:lim], count * N, device=dev).view(lim, count, N).permute(1, 0, 2).contiguous()
+        pts = [rows(30, 1, l0 - 2 if G else l0 - 1)[0], rows(31, 1, linj - 1)[0], rows(32, 8, l0), rows(33, 7, l0),
+               rows(34, K_blk, l0), rows(35, B, linj)]
+    desc = fesc.ScanDesc(L, mine * hpc, P, d_s, B, stride, l0, base, int(args.hoist), net, G, plain)
     torch.cuda.empty_cache()
 
     def step():
         if mine:
-            ctx.scan_contract(x, a, Bc, Cc, desc, masks[0], masks[1], masks[2], masks[3][:linj - 2], adj, adj, out, gm)
+            ctx.scan_contract(x, a, Bc, Cc, desc, masks[0], masks[1], masks[2], masks[3][:linj - 2], adj, adj, out, gm, pts)
         return gather_chunk_outputs(out[:, :mine], parts, rank, world, K_blk, K_s) if world > 1 else out
 
     if args.profile_step:           # one bare step for a profiler's launch list (no warm-up, no timing claims)
@@ -924,7 +930,8 @@ def run_scan(args, ctx=None, quiet=False):
                                                  % (args.workload, L, H, stride, K_s, l0,
                                                     {"bk": "Brent-Kung", "ks": "Kogge-Stone", "sk": "Sklansky"}[args.network],
                                                     ("radix-4 hoisted rotate-and-add chains" if args.hoist else "plain rotations")
-                                                    + (", leaves built in groups of %d tokens" % G if G else "")),
+                                                    + (", leaves built in groups of %d tokens" % G if G else "")
+                                                    + (", invariant-family mode (plaintext decay, B, C)" if plain else "")),
                                      "parallelism": "state chunks in pairs over %d rank(s): %s; one all-gather of the outputs"
                                                     % (world, [c for _, c in parts])},
                           "key_switches": ks, "limb_transforms": c1[0] - c0[0], "gpu_launches": c1[4] - c0[4],
@@ -1193,6 +1200,8 @@ def main():
     ap.add_argument("--stride", type=int, default=256, choices=[128, 256],
                     help="scan workloads: slots per channel of a state ciphertext; 256 (the paper's deployed shape: half of "
                          "the slots idle, 12 chunks) or 128 (every slot used, 6 chunks, two token segments per block)")
+    ap.add_argument("--plain", type=int, default=0, choices=[0, 1],
+                    help="scan workloads: 1 = the invariant-family mode (plaintext decay, input and output factors; S4D / S5 / LRU)")
     ap.add_argument("--network", default="bk", choices=["bk", "ks", "sk"],
                     help="scan workloads: prefix network (Brent-Kung, Kogge-Stone, Sklansky)")
     ap.add_argument("--workload", default="in_proj", choices=["in_proj", "out_proj", "rotations", "scan_slice", "scan_layer", "conv", "norm"],
