@@ -158,19 +158,23 @@ def make_inputs(primes, n, gin, nout, tbs, seed, device, ctx=None, desc=None):
             r = S.hashed_residues(seed, tb * gin + g, q, 2 * n, device=device)      # [LEVEL, 2n]
             ct[tb, g] = r.view(LEVEL, 2, n).permute(1, 0, 2)
     packed = bool(desc is not None and desc.packed)
+    per = 1                         # output blocks per pack call: a range must start at a multiple of 8 (b,p) pairs
+    while (per * N2) % 8 and per < nout:
+        per += 1
     if packed:
-        assert N2 % 8 == 0 or nout == 1, "a pack range must start at a multiple of 8 (b,p) pairs"
+        assert (per * N2) % 8 == 0 or per == nout
         diags = torch.empty((ctx.linear_packed_bytes(desc),), dtype=torch.uint8, device=device)
-        one = torch.empty((N2, gin, N1, LEVEL, n), dtype=torch.int64, device=device)
+        one = torch.empty((per, N2, gin, N1, LEVEL, n), dtype=torch.int64, device=device)
     else:
         diags = torch.empty((nout, N2, gin, N1, LEVEL, n), dtype=torch.int64, device=device)
     for b in range(nout):
         for p in range(N2):
             r = S.hashed_residues(seed, 100000 + b * N2 + p, q, gin * N1 * n, device=device)
-            (one if packed else diags[b])[p] = r.view(LEVEL, gin, N1, n).permute(1, 2, 0, 3)
+            (one[b % per] if packed else diags[b])[p] = r.view(LEVEL, gin, N1, n).permute(1, 2, 0, 3)
             del r
-        if packed:
-            ctx.linear_pack_diags(one, desc, b * N2, N2, diags)
+        if packed and (b % per == per - 1 or b == nout - 1):
+            first, cnt = (b // per) * per, b % per + 1
+            ctx.linear_pack_diags(one[:cnt], desc, first * N2, cnt * N2, diags)
     if packed:
         ctx.sync()
         del one
@@ -543,13 +547,18 @@ def run_ours(args):
     p = S.params("full")
     ctx = fesc.Context(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
     n = ctx.N
+    gin, nout, tbs = workload_dims(args.scale_down)
+    if args.profile_case:
+        # small case for profiler captures, a few GB on the device, inputs larger than L2: the accumulate keeps its
+        # full-size structure (96 terms = 3 k-steps, 4 tiles of 8 (b,p) outputs, 4 token blocks) at 4 limbs, and the
+        # rotations run on batches of 48 and 32 ciphertexts; 10 Galois keys instead of 38
+        global N1, N2, LEVEL
+        N1, N2, LEVEL = 8, 4, 4
+        gin, nout, tbs = 12, 8, 4
     for q in range(1, N1):
         ctx.add_galois_key(q * T_SEG, BABY_BASE + q)
     for g in range(1, N2):
         ctx.add_galois_key(g * N1 * T_SEG, GIANT_BASE + g)
-    gin, nout, tbs = workload_dims(args.scale_down)
-    if args.profile_case:       # small case for profiler captures: a few GB on the device
-        gin, nout, tbs = 1, 1, 4
     ks_per_step = key_switches_per_step(gin, nout, tbs)
     desc = fesc.BsgsDesc(N1, N2, gin, nout, tbs, LEVEL, BABY_BASE, GIANT_BASE, int(args.hoist), int(args.defer),
                          int(args.packed))
@@ -1178,7 +1187,7 @@ def main():
     ap.add_argument("--scale-down", dest="scale_down", type=int, default=1, help=argparse.SUPPRESS)
     ap.add_argument("--no-cpu", dest="no_cpu", action="store_true", help="skip the CPU baseline leg")
     ap.add_argument("--profile-case", dest="profile_case", action="store_true",
-                    help="run ONE step of a small case (1 input block, 1 output block, 4 token blocks) and exit; for ncu")
+                    help="run ONE step of a small case (96 terms, 32 (b,p) outputs, 4 token blocks, 4 limbs) and exit; for ncu")
     ap.add_argument("--profile-step", dest="profile_step", action="store_true",
                     help="run ONE step of the full workload without warm-up and exit; for the ncu launch list")
     ap.add_argument("--defer", type=int, default=1, choices=[0, 1],

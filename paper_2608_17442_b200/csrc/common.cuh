@@ -263,13 +263,26 @@ static inline int fesc_fail(fesc_ctx* ctx, int code, const std::string& msg) {
     return code;
 }
 
+// Optional epilogue of the last pass of a forward N = 2^16 transform over rows r = bp * level + i (bp = ciphertext * 2 +
+// polynomial, i = data limb, all primes below 2^50): instead of storing the transformed row u, the pass stores the last
+// step of the division by P,  out[b][p][i] = (acc[bp][i] - u) * P^-1  (added to what out holds when bit p of add_mask
+// is set), which saves writing u, reading it back and a launch.
+struct NttFinish {
+    const u64* acc = nullptr;        // [batch * 2][acc_rows][N]; nullptr = no epilogue
+    u64* out = nullptr;              // ciphertext b at out + b * out_stride, [2][level][N]
+    size_t out_stride = 0;
+    const ModDownTab* tab = nullptr; // P^-1 mod q_i as doubles
+    uint32_t level = 0, acc_rows = 0;
+    int add_mask = 0;
+};
+
 // internal launchers (ntt.cu)
 // rows: number of N-word rows starting at d_data; map gives the prime per row.
 // in_double (forward, N = 2^16 only): rows on primes below 2^50 hold doubles with |x| <= q/2 (bit patterns) written by a
 // basis-conversion kernel instead of canonical words.
 // out_double (forward, N = 2^16 only): such rows are left as doubles with |x| <= q/2 for a consumer that computes in FP64.
 int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool inverse, cudaStream_t st,
-               bool in_double = false, bool out_double = false);
+               bool in_double = false, bool out_double = false, const NttFinish* finish = nullptr);
 // double with |x| <= q/2 as handed to the forward transform
 __device__ __forceinline__ u64 fp_handoff(double s, double q, double qinv) {
     return (u64)__double_as_longlong(fp_reduce(s, q, qinv));

@@ -507,6 +507,8 @@ __global__ void __launch_bounds__(32 * IM_CW, 1) k_bsgs_accumulate_imma(
         c96 = fp_modmul(c64, c32, q, qinv);
     }
     int d[4][7][4];
+    int z0 = 0, z1 = 0, z2 = 0, z3 = 0;       // a fixed quad of zero addends (see imma_u8_zero)
+    asm volatile("" : "+r"(z0), "+r"(z1), "+r"(z2), "+r"(z3));
     const u64* a_ring = stage + 8 * xs_pitch + g * IM_BPP + (4 * tg) * IM_ROWP + warp;
     const u64* b_frag = stage + g * xs_pitch + (4 * tg) * IM_ROWP + warp;
     uint32_t slot = 0, s = 0;
@@ -535,7 +537,7 @@ __global__ void __launch_bounds__(32 * IM_CW, 1) k_bsgs_accumulate_imma(
 #pragma unroll
                     for (int j = 0; j < 7; j++)
                         imma_u8_zero(d[m][j], fa[0][2 * m], m < 3 ? fa[0][2 * m + 1] : 0u, fa[1][2 * m],
-                                     m < 3 ? fa[1][2 * m + 1] : 0u, fb[0][j], fb[1][j]);
+                                     m < 3 ? fa[1][2 * m + 1] : 0u, fb[0][j], fb[1][j], z0, z1, z2, z3);
             } else {
 #pragma unroll
                 for (int m = 0; m < 4; m++)
@@ -575,7 +577,99 @@ static int bsgs_kernel() {
 static size_t bsgs_group_bytes(bool packed) {
     const char* e = getenv("FESC_BSGS_GROUP_GIB");
     if (e && atoi(e) > 0) return (size_t)atoi(e) << 30;
-    return (size_t)(packed ? 28 : 24) << 30;      // the packed inputs of a group are scratch as well
+    return (size_t)(packed ? 32 : 24) << 30;      // the packed inputs and the key-switch chunk of a group count as well (44 GiB allows groups of 8)
+}
+
+// Projection on packed diagonals.  Token blocks are processed in groups of up to 8 = two tiles of 4: the baby rotations
+// run on 4 token blocks at a time and their results are packed into the group's fragment images; the accumulate then
+// covers both tiles in one launch (the two CTAs that need the same diagonal images run side by side, so the images
+// cross HBM once per group), for one part of the output blocks at a time so that the partial sums of a part stay
+// small; giant steps and rescale follow per part.  With groups of 8 the image is streamed twice per 16 token blocks
+// instead of four times.
+static int linear_packed(fesc_ctx* ctx, const u64* in, const uint8_t* image, const fesc_bsgs_desc* desc, u64* out,
+                         cudaStream_t st, uint32_t qbits) {
+    const uint32_t n1 = desc->n1, n2 = desc->n2, gin = desc->in_blocks, nout = desc->out_blocks;
+    const uint32_t tbs = desc->token_blocks, level = desc->n_limbs, N = ctx->N, terms = gin * n1;
+    const size_t ctw = (size_t)2 * level * N, ctw_out = (size_t)2 * (level - 1) * N;
+    uint32_t bstep = 8;                    // a part starts at a (b,p) pair that is a multiple of 8
+    while (bstep > 1 && (bstep / 2) * n2 % 8 == 0) bstep /= 2;
+    if (n2 % 8 == 0) bstep = 1;
+    u64 *scratch = nullptr, *rot = nullptr, *acc = nullptr, *ks = nullptr;
+    uint8_t* xpk = nullptr;
+    uint32_t tbg = tbs >= 8 ? 8 : tbs, nb_part = nout;
+    int rc = FESC_ENOMEM;
+    for (;; tbg = tbg > 4 ? 4 : (tbg + 1) / 2) {
+        const uint32_t parts = (tbg + 3) / 4, sub = tbg < 4 ? tbg : 4;
+        nb_part = (nout + parts - 1) / parts;
+        nb_part = (nb_part + bstep - 1) / bstep * bstep;
+        if (nb_part > nout) nb_part = nout;
+        const uint32_t max_batch = sub * gin > tbg * nb_part ? sub * gin : tbg * nb_part;
+        const size_t ks_words = ks_scratch_words(ctx, level, ks_chunk(ctx, max_batch));
+        const size_t rs_words = (size_t)(nb_part < 16384 ? nb_part : 16384) * 2 * N;
+        const size_t rot_words = (size_t)sub * terms * ctw, acc_words = (size_t)tbg * nb_part * n2 * ctw;
+        const size_t xpk_words = bsgs_packed_bytes(N, level, 2 * tbg, terms) / 8;
+        const size_t total = (rot_words + acc_words + xpk_words + (ks_words > rs_words ? ks_words : rs_words)) * sizeof(u64);
+        if (total <= bsgs_group_bytes(true) || tbg == 1) {
+            rc = ctx_scratch(ctx, total, &scratch);
+            if (rc == FESC_OK) {
+                rot = scratch;
+                acc = rot + rot_words;
+                xpk = (uint8_t*)(acc + acc_words);
+                ks = acc + acc_words + xpk_words;
+                break;
+            }
+            if (rc != FESC_ENOMEM) return rc;
+        }
+        if (tbg == 1) return rc;
+    }
+    ctx->counters[5] = tbg;
+    const size_t tile_bytes = bsgs_packed_bytes(N, level, 8, terms);     // one tile of 8 rows, either side
+    for (uint32_t tb0 = 0; tb0 < tbs; tb0 += tbg) {
+        const uint32_t nt = tbs - tb0 < tbg ? tbs - tb0 : tbg;
+        for (uint32_t s0 = 0; s0 < nt; s0 += 4) {        // baby rotations of 4 token blocks, packed into their tile
+            const uint32_t ns = nt - s0 < 4 ? nt - s0 : 4;
+            const u64* gin_base = in + (size_t)(tb0 + s0) * gin * ctw;
+            FESC_CHECK_CUDA(ctx, cudaMemcpy2DAsync(rot, (size_t)n1 * ctw * sizeof(u64), gin_base, ctw * sizeof(u64),
+                                                   ctw * sizeof(u64), (size_t)ns * gin, cudaMemcpyDeviceToDevice, st));
+            if (desc->hoist && n1 > 1) {
+                std::vector<uint32_t> ids;
+                for (uint32_t q = 1; q < n1; q++) ids.push_back(desc->baby_key_base + q);
+                rc = rotate_hoisted_internal(ctx, gin_base, ctw, rot + ctw, (size_t)n1 * ctw, ctw, ns * gin, level, ids.data(),
+                                             n1 - 1, ks, st);
+                if (rc != FESC_OK) return rc;
+            } else {
+                for (uint32_t q = 1; q < n1; q++) {
+                    rc = rotate_internal(ctx, gin_base, ctw, rot + (size_t)q * ctw, (size_t)n1 * ctw, ns * gin, level,
+                                         desc->baby_key_base + q, ks, st, 0);
+                    if (rc != FESC_OK) return rc;
+                }
+            }
+            if ((rc = bsgs_pack_inputs(ctx, rot, xpk + (size_t)(s0 / 4) * tile_bytes, level, ns, terms, st)) != FESC_OK) return rc;
+        }
+        for (uint32_t b0 = 0; b0 < nout; b0 += nb_part) {
+            const uint32_t nb = nout - b0 < nb_part ? nout - b0 : nb_part;
+            rc = bsgs_accumulate_packed(ctx, xpk, image + (size_t)(b0 * n2 / 8) * tile_bytes, acc, level, nt, terms, nb * n2,
+                                        qbits <= 50, st);
+            if (rc != FESC_OK) return rc;
+            ctx->counters[2] += (uint64_t)nt * nb * n2 * terms;
+            if (desc->defer) {
+                rc = giant_sum_deferred_internal(ctx, acc, n2, ctw, nt * nb, level, desc->giant_key_base, ks, st);
+                if (rc != FESC_OK) return rc;
+            } else {
+                for (uint32_t p = 1; p < n2; p++) {
+                    rc = rotate_internal(ctx, acc + (size_t)p * ctw, (size_t)n2 * ctw, acc, (size_t)n2 * ctw, nt * nb, level,
+                                         desc->giant_key_base + p, ks, st, 1);
+                    if (rc != FESC_OK) return rc;
+                }
+            }
+            for (uint32_t tb = 0; tb < nt; tb++) {      // the outputs of a token block are contiguous, those of a part are not
+                rc = rescale_internal(ctx, acc + (size_t)tb * nb * n2 * ctw, (size_t)n2 * ctw,
+                                      out + ((size_t)(tb0 + tb) * nout + b0) * ctw_out, nb, level, ks, st);
+                if (rc != FESC_OK) return rc;
+            }
+        }
+    }
+    return FESC_OK;
 }
 
 extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_t* d_diags, const fesc_bsgs_desc* desc,
@@ -596,6 +690,14 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
     const bool packed = desc->packed != 0;
     if (packed && !bsgs_packed_supported(ctx, level, gin * n1))
         return fesc_fail(ctx, FESC_EINVAL, "linear: packed diagonals need N a multiple of 8, primes below 2^56 and at most 512 terms");
+    if (packed) {
+        uint32_t bits = 0;
+        for (uint32_t i = 0; i < level; i++) {
+            const uint32_t b = 64 - __builtin_clzll(ctx->q[i]);
+            if (b > bits) bits = b;
+        }
+        return linear_packed(ctx, (const u64*)d_ct_in, (const uint8_t*)d_diags, desc, (u64*)d_ct_out, st, bits);
+    }
     // token blocks per group, from the scratch budget (groups of packed inputs are whole tiles of 4 token blocks)
     const size_t xpk_tb = packed ? bsgs_packed_bytes(N, level, 8, gin * n1) / 4 : 0;
     const size_t per_tb = ((size_t)gin * n1 + (size_t)nout * n2) * ctw * sizeof(u64) + xpk_tb;

@@ -361,7 +361,9 @@ __device__ __forceinline__ void strided_body_fp(u64* __restrict__ p, double* __r
 
 template <bool INV>
 __device__ __forceinline__ void contig_body_fp(u64* __restrict__ p, double* __restrict__ sm, const double* __restrict__ tw,
-                                               const PrimeConst& pc, uint32_t pre, int out_double) {
+                                               const PrimeConst& pc, uint32_t pre, int out_double,
+                                               const u64* __restrict__ fin_acc = nullptr, u64* __restrict__ fin_out = nullptr,
+                                               double fin_pinv = 0.0, int fin_add = 0) {
     const double q = pc.qd, qinv = pc.qinvd;
     const uint32_t sub = threadIdx.x & 31;
     const uint32_t h2 = sub >> 2, l2 = sub & 3;
@@ -384,6 +386,25 @@ __device__ __forceinline__ void contig_body_fp(u64* __restrict__ p, double* __re
 #pragma unroll
         for (int k = 0; k < 8; k++) x[k] = sm[pad8(sub * 8 + k)];
         fp_fwd_round2(x, tw, 64 * pre + 2 * sub, 128 * pre + 4 * sub, q, qinv);
+        if (fin_acc) {
+            // last step of the division by P on the fly: (acc - u) * P^-1 (+ what the output holds); |acc - u| stays
+            // below 6q, the lazy product below 3q, so every sum is exact
+            const ulonglong2* a = reinterpret_cast<const ulonglong2*>(fin_acc + sub * 8);
+            ulonglong2* o = reinterpret_cast<ulonglong2*>(fin_out + sub * 8);
+#pragma unroll
+            for (int k = 0; k < 4; k++) {
+                const ulonglong2 av = a[k];
+                double s0 = fp_modmul(fp_load(av.x, q) - x[2 * k], fin_pinv, q, qinv);
+                double s1 = fp_modmul(fp_load(av.y, q) - x[2 * k + 1], fin_pinv, q, qinv);
+                if (fin_add) {
+                    const ulonglong2 ov = o[k];
+                    s0 += fp_load(ov.x, q);
+                    s1 += fp_load(ov.y, q);
+                }
+                o[k] = make_ulonglong2(fp_store(s0, q, qinv), fp_store(s1, q, qinv));
+            }
+            return;
+        }
         ulonglong2* o = reinterpret_cast<ulonglong2*>(p + sub * 8);
 #pragma unroll
         for (int k = 0; k < 4; k++)   // canonical words, or doubles with |x| <= q/2 for a consumer that computes in FP64
@@ -512,7 +533,7 @@ template <bool INV>
 __global__ void __launch_bounds__(NTT_WARPS * 32) ntt16_contig(u64* __restrict__ data, const ulonglong2* __restrict__ tw_all,
                                                     const double* __restrict__ twf_all,
                                                     const PrimeConst* __restrict__ pcs, RowMap map,
-                                                    uint32_t row_base, int out_double) {
+                                                    uint32_t row_base, int out_double, NttFinish fin, uint32_t row_first) {
     const uint32_t row = blockIdx.y;
     const uint32_t pi = map.prime[(row_base + row) % map.period];
     if (pi == 0xFF) return;
@@ -523,9 +544,17 @@ __global__ void __launch_bounds__(NTT_WARPS * 32) ntt16_contig(u64* __restrict__
     const uint32_t blk = blockIdx.x * NTT_WARPS + warp;   // 256-point block index within the limb
     u64* p = data + (size_t)row * N16 + (size_t)blk * 256;
     u64* sm = sm_all + warp * 288;
-    if (pc.q < FP_LIMIT)
-        contig_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, 256 + blk, out_double);
-    else if (pc.q < WIDE_LIMIT)
+    if (pc.q < FP_LIMIT) {
+        if (!INV && fin.acc) {      // rows of this launch: r = bp * level + i
+            const uint32_t r = row_first + row, bp = r / fin.level, i = r - bp * fin.level;
+            contig_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, 256 + blk, out_double,
+                                fin.acc + ((size_t)bp * fin.acc_rows + i) * N16 + (size_t)blk * 256,
+                                fin.out + (size_t)(bp >> 1) * fin.out_stride + ((size_t)(bp & 1) * fin.level + i) * N16 + (size_t)blk * 256,
+                                fin.tab->pinvd[i], (fin.add_mask >> (bp & 1)) & 1);
+        } else {
+            contig_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, 256 + blk, out_double);
+        }
+    } else if (pc.q < WIDE_LIMIT)
         contig_body<INV, true>(p, sm, tw, pc, 256 + blk);
     else
         contig_body<INV, false>(p, sm, tw, pc, 256 + blk);
@@ -587,7 +616,9 @@ __global__ void __launch_bounds__(256) ntt_small(u64* __restrict__ data, const u
 }
 
 int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool inverse, cudaStream_t st, bool in_double,
-               bool out_double) {
+               bool out_double, const NttFinish* finish) {
+    const NttFinish fin = finish ? *finish : NttFinish();
+    if (fin.acc && (inverse || ctx->log_n != 16)) return fesc_fail(ctx, FESC_EINVAL, "ntt: the fused epilogue belongs to a forward N = 2^16 transform");
     if (rows == 0) return FESC_OK;
     if (rows > 0x7fffffffu) return fesc_fail(ctx, FESC_EINVAL, "ntt: too many rows");
     const ulonglong2* tw = inverse ? ctx->d_itw : ctx->d_tw;
@@ -608,9 +639,9 @@ int ntt_launch(fesc_ctx* ctx, u64* d_data, size_t rows, const RowMap& map, bool 
             u64* base = d_data + r0 * (size_t)N16;
             if (!inverse) {
                 ntt16_strided<false><<<gs, NTT_COLS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb, in_double ? 1 : 0);
-                ntt16_contig<false><<<gc, NTT_WARPS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb, out_double ? 1 : 0);
+                ntt16_contig<false><<<gc, NTT_WARPS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb, out_double ? 1 : 0, fin, (uint32_t)r0);
             } else {
-                ntt16_contig<true><<<gc, NTT_WARPS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb, 0);
+                ntt16_contig<true><<<gc, NTT_WARPS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb, 0, NttFinish(), 0u);
                 ntt16_strided<true><<<gs, NTT_COLS * 32, 0, st>>>(base, tw, twf, ctx->d_pc, map, rb, 0);
             }
             launches += 2;

@@ -732,6 +732,14 @@ static int ks_moddown(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint32
     prof_end(ctx, PF_MODDOWN, st);
     m.period = level;
     for (uint32_t i = 0; i < level; i++) m.prime[i] = (uint8_t)i;
+    bool fuse = ctx->log_n == 16;          // the last pass of the transform finishes the division (FP64 rows only)
+    for (uint32_t i = 0; i < level; i++) fuse = fuse && ctx->q[i] < FESC_FP_LIMIT;
+    if (fuse) {
+        NttFinish fin;
+        fin.acc = ws.acc, fin.out = out, fin.out_stride = out_stride, fin.tab = ctx->tabs.d_moddown;
+        fin.level = level, fin.acc_rows = rows, fin.add_mask = add_mask;
+        return ntt_launch(ctx, ws.u, (size_t)batch * 2 * level, m, false, st, true, false, &fin);
+    }
     if ((rc = ntt_launch(ctx, ws.u, (size_t)batch * 2 * level, m, false, st, ctx->log_n == 16)) != FESC_OK) return rc;
     prof_begin(ctx, PF_MODDOWN, st);
     k_moddown_finish<<<dim3(gx, level, batch * 2), 256, 0, st>>>(ws.acc, ws.u, out, out_stride, ctx->tabs.d_moddown,

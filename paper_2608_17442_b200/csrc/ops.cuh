@@ -40,13 +40,13 @@ __device__ __forceinline__ void imma_u8(int (&d)[4], uint32_t a0, uint32_t a1, u
                  : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-// the same product with zero addends (first k-step of a tile)
+// the same product with zero addends (first k-step of a tile).  z0..z3 are four registers that hold zero and are kept
+// opaque to the optimiser, so that they stay one fixed operand quad instead of being rebuilt before every instruction.
 __device__ __forceinline__ void imma_u8_zero(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                             uint32_t b1) {
-    const int z = 0;
-    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+                                             uint32_t b1, int z0, int z1, int z2, int z3) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
                  : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(z));
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(z0), "r"(z1), "r"(z2), "r"(z3));
 }
 // d[k] = (byte k of w0) | (byte k of w1) << 8 | (byte k of w2) << 16 | (byte k of w3) << 24, k = 0..6
 __device__ __forceinline__ void byte_planes4(u64 w0, u64 w1, u64 w2, u64 w3, uint32_t (&d)[7]) {

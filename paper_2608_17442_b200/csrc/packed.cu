@@ -24,6 +24,9 @@
 // CTA needs for one (b,p) tile are contiguous.  Rows and terms beyond the valid ones are zero.
 #include "ops.cuh"
 
+#ifndef PK_VARIANT
+#define PK_VARIANT 0
+#endif
 #define PK_CW 8
 #define PK_FRAG 1792
 #define PK_STAGE (PK_CW * PK_FRAG)
@@ -105,8 +108,11 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
     extern __shared__ __align__(128) uint8_t ring[];
     constexpr uint32_t WARP_BYTES = (PK_STAGES + KSR) * PK_FRAG;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tg = lane & 3;
-    const uint32_t ct = blockIdx.x >> 1, coef = (blockIdx.x & 1) * PK_WARPS + warp, l = blockIdx.y, tbt = blockIdx.z;
-    const uint32_t tiles = gridDim.x >> 1;
+    // blockIdx.x = (coefficient half-tile) * token-block tiles + token-block tile: the CTAs that stream the same images
+    // for different token blocks start together, so only the first of them reads the images from HBM
+    const uint32_t tbts = (tbs + 3) >> 2, tbt = blockIdx.x % tbts, half_tile = blockIdx.x / tbts;
+    const uint32_t ct = half_tile >> 1, coef = (half_tile & 1) * PK_WARPS + warp, l = blockIdx.y;
+    const uint32_t tiles = gridDim.x / (2 * tbts);
     const uint32_t bp_tiles = (bp_count + 7) >> 3, total = bp_tiles * ksteps;
     const uint32_t my_ring = (uint32_t)__cvta_generic_to_shared(ring) + warp * WARP_BYTES;
     const uint32_t my_bar = (uint32_t)__cvta_generic_to_shared(ring) + PK_WARPS * WARP_BYTES + warp * ((PK_STAGES + 1) * 8);
@@ -148,6 +154,8 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
     }
     __syncthreads();
     int d[4][7][4];
+    int z0 = 0, z1 = 0, z2 = 0, z3 = 0;                   // a fixed quad of zero addends (see imma_u8_zero)
+    asm volatile("" : "+r"(z0), "+r"(z1), "+r"(z2), "+r"(z3));
     uint32_t slot = 0, phase = 0, s = 0;
     bool ok = KSR == 0 || !mbar_wait_bounded(my_bar + PK_STAGES * 8, 0);
     const bool x_ok = ok;
@@ -168,10 +176,10 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
             const uint2 b = KSR > 0 ? *(const uint2*)(xfrag + j * 256 + lane * 8)
                                     : __ldg((const uint2*)(xfrag + j * 256 + lane * 8));
             if (first) {
-                imma_u8_zero(d[0][j], a0.x, a0.y, a0.z, a0.w, b.x, b.y);
-                imma_u8_zero(d[1][j], a1.x, a1.y, a1.z, a1.w, b.x, b.y);
-                imma_u8_zero(d[2][j], a2.x, a2.y, a2.z, a2.w, b.x, b.y);
-                imma_u8_zero(d[3][j], a3.x, a3.y, a3.z, a3.w, b.x, b.y);
+                imma_u8_zero(d[0][j], a0.x, a0.y, a0.z, a0.w, b.x, b.y, z0, z1, z2, z3);
+                imma_u8_zero(d[1][j], a1.x, a1.y, a1.z, a1.w, b.x, b.y, z0, z1, z2, z3);
+                imma_u8_zero(d[2][j], a2.x, a2.y, a2.z, a2.w, b.x, b.y, z0, z1, z2, z3);
+                imma_u8_zero(d[3][j], a3.x, a3.y, a3.z, a3.w, b.x, b.y, z0, z1, z2, z3);
             } else {
                 imma_u8(d[0][j], a0.x, a0.y, a0.z, a0.w, b.x, b.y);
                 imma_u8(d[1][j], a1.x, a1.y, a1.z, a1.w, b.x, b.y);
@@ -202,8 +210,20 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
         // CTA (four neighbouring coefficients) exchange their results through shared memory so that every output row
         // receives one full 32-byte sector instead of four separate words.
         u64* stage_out = (u64*)(ring + PK_WARPS * (WARP_BYTES + (PK_STAGES + 1) * 8)) + (bt & 1) * 256;
+#if PK_VARIANT == 2
+        {
+            int x0 = 0, x1 = 0;
+#pragma unroll
+            for (int m = 0; m < 4; m++)
+#pragma unroll
+                for (int j = 0; j < 7; j++) x0 += d[m][j][0] + d[m][j][2], x1 += d[m][j][1] + d[m][j][3];
+            stage_out[(lane * 2) * PK_WARPS + warp] = (u64)(uint32_t)x0;
+            stage_out[(lane * 2 + 1) * PK_WARPS + warp] = (u64)(uint32_t)x1;
+        }
+#else
         stage_out[(lane * 2) * PK_WARPS + warp] = imma_recombine<FP>(d, 0, pc, c32, c64, c96);
         stage_out[(lane * 2 + 1) * PK_WARPS + warp] = imma_recombine<FP>(d, 1, pc, c32, c64, c96);
+#endif
         // CTA-wide hand-over on a shared-memory barrier (one arrival per warp) so that this wait is bounded too
         __syncwarp();
         if (lane == 0) mbar_arrive(out_bar);
@@ -217,7 +237,7 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
             if (bp < bp_count && tb < tbs) {
                 const ulonglong2 v = *(const ulonglong2*)(stage_out + row * PK_WARPS + (tid & 1) * 2);
                 u64* dst = acc + ((size_t)tb * bp_count + bp) * ctw + (row & 1) * poly + (size_t)l * N + ct * PK_CW +
-                           (blockIdx.x & 1) * PK_WARPS + (tid & 1) * 2;
+                           (half_tile & 1) * PK_WARPS + (tid & 1) * 2;
                 *(ulonglong2*)dst = v;
             }
         }
@@ -237,7 +257,7 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
 int bsgs_accumulate_packed(fesc_ctx* ctx, const uint8_t* xpk, const uint8_t* dpk, u64* acc, uint32_t level, uint32_t tbs,
                            uint32_t terms, uint32_t bp_count, bool fp, cudaStream_t st) {
     const uint32_t N = ctx->N, ksteps = (terms + 31) / 32;
-    dim3 grid(2 * (N / PK_CW), level, (tbs + 3) / 4);
+    dim3 grid(2 * (N / PK_CW) * ((tbs + 3) / 4), level);
 #define PK_LAUNCH(FP, KSR)                                                                                        \
     do {                                                                                                          \
         const size_t smem = (size_t)PK_WARPS * ((PK_STAGES + KSR) * PK_FRAG + (PK_STAGES + 1) * 8) + 2 * 256 * 8 + 8; \
