@@ -602,3 +602,62 @@ def conv_masks(w, b_conv, blk: int, T: int, C: int, n: int):
             if r >= 1:
                 M[d_conv - 1 + r, c * T:c * T + r] = w[ch, r]
     return M, bias
+
+
+# ---- token-major packing with periodic diagonals --------------------------------------------------------------
+# App. "Projection Kernel Breakdown" defines two slot shifts on the segment view idx(r, s) = s * l_seg + r: the
+# whole-segment shift Phi^delta (one rotation) and the intra-segment shift
+#   Psi^t(x) = M^stay_t (.) rho(x; t) + M^wrap_t (.) rho(x; t - l_seg)      (two rotations and public masks).
+# The projection of this build packs features as segments and tokens inside a segment, so a feature shift is a Phi and
+# needs one rotation.  The TRANSPOSED packing, slot r*C + c = X[r, gC + c] (one segment per token, l_seg = C features),
+# needs Psi for a feature shift, i.e. two rotations, but every plaintext diagonal then depends on the feature index
+# only: the slot vector has period C, the encoded polynomial lives in Z[X^(n/C)], and its evaluation form is constant on
+# aligned runs of N/(2C) indices, so a diagonal is N/(2C) times smaller (128 x at N = 2^16, C = 256).
+# With the masks folded into the diagonals the product is an ordinary baby-step / giant-step sum over the rotation sets
+#   baby  {0} + {q, q - C : 1 <= q < n1},      giant {0} + {p n1, p n1 - C : 1 <= p < n2}
+# (2 n1 - 1 and 2 n2 - 1 amounts), which is exactly what `Oracle.linear` evaluates when it is given those keys:
+#   y^(b) = sum_G rho( sum_{g, beta} D^(b)_{G,g,beta} (.) rho(x^(g); beta) ; G ).
+def token_major_amounts(C: int, n1: int, n2: int):
+    """(baby amounts, giant amounts) in slot order: index 0 is the identity, 2q-1 / 2q are q and q - C (baby),
+    2p-1 / 2p are p*n1 and p*n1 - C (giant)."""
+    baby = [0] + [a for q in range(1, n1) for a in (q, q - C)]
+    giant = [0] + [a for p in range(1, n2) for a in (p * n1, p * n1 - C)]
+    return baby, giant
+
+
+def pack_linear_input_token_major(x_block, T: int, C: int, n: int) -> np.ndarray:
+    """Slots r*C + c hold X[r, c] for one (token block, input block)."""
+    v = np.zeros((T, C))
+    rows, cols = x_block.shape
+    v[:rows, :cols] = x_block
+    return v.reshape(n)
+
+
+def linear_diagonal_token_major(W, b: int, g: int, gi: int, bi: int, T: int, C: int, n1: int) -> np.ndarray:
+    """Diagonal of giant slot gi and baby slot bi (see token_major_amounts) for output block b and input block g.
+    Output feature c' = c'' - P (stay) or c'' + C - P (wrap) is assembled at position c'' of the accumulator; it takes
+    input feature (c'' + q) mod C, which the baby rotation by q delivers where c'' + q < C and the one by q - C where
+    c'' + q >= C.  The vector depends on c'' only (period C)."""
+    d_in, d_out = W.shape
+    p, wrap_g = ((gi + 1) // 2, gi % 2 == 0) if gi else (0, False)
+    q, wrap_b = ((bi + 1) // 2, bi % 2 == 0) if bi else (0, False)
+    P = p * n1
+    cpp = np.arange(C)
+    support_g = (cpp < P) if wrap_g else (cpp >= P)              # positions this accumulator owns
+    c_out = cpp + C - P if wrap_g else cpp - P
+    support_b = (cpp + q >= C) if wrap_b else (cpp + q < C)      # positions this baby rotation serves
+    c_in = (cpp + q) % C
+    rows, cols = g * C + c_in, b * C + c_out
+    ok = support_g & support_b & (rows < d_in) & (cols < d_out) & (cols >= b * C)
+    vals = np.zeros(C)
+    vals[ok] = W[rows[ok], cols[ok]]
+    return np.tile(vals, T)
+
+
+def periodic_eval_runs(pt_eval: np.ndarray, run: int) -> np.ndarray:
+    """One word per aligned run of `run` evaluation indices of a plaintext whose slot vector is periodic (asserts that
+    the runs are constant): the compressed form of a token-major diagonal, [limbs, N / run]."""
+    k, N = pt_eval.shape
+    v = pt_eval.reshape(k, N // run, run)
+    assert np.all(v == v[:, :, :1]), "not constant on runs: the slot vector is not periodic"
+    return np.ascontiguousarray(v[:, :, 0])

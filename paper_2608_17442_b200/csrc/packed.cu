@@ -24,9 +24,6 @@
 // CTA needs for one (b,p) tile are contiguous.  Rows and terms beyond the valid ones are zero.
 #include "ops.cuh"
 
-#ifndef PK_VARIANT
-#define PK_VARIANT 0
-#endif
 #define PK_CW 8
 #define PK_FRAG 1792
 #define PK_STAGE (PK_CW * PK_FRAG)
@@ -210,20 +207,8 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
         // CTA (four neighbouring coefficients) exchange their results through shared memory so that every output row
         // receives one full 32-byte sector instead of four separate words.
         u64* stage_out = (u64*)(ring + PK_WARPS * (WARP_BYTES + (PK_STAGES + 1) * 8)) + (bt & 1) * 256;
-#if PK_VARIANT == 2
-        {
-            int x0 = 0, x1 = 0;
-#pragma unroll
-            for (int m = 0; m < 4; m++)
-#pragma unroll
-                for (int j = 0; j < 7; j++) x0 += d[m][j][0] + d[m][j][2], x1 += d[m][j][1] + d[m][j][3];
-            stage_out[(lane * 2) * PK_WARPS + warp] = (u64)(uint32_t)x0;
-            stage_out[(lane * 2 + 1) * PK_WARPS + warp] = (u64)(uint32_t)x1;
-        }
-#else
         stage_out[(lane * 2) * PK_WARPS + warp] = imma_recombine<FP>(d, 0, pc, c32, c64, c96);
         stage_out[(lane * 2 + 1) * PK_WARPS + warp] = imma_recombine<FP>(d, 1, pc, c32, c64, c96);
-#endif
         // CTA-wide hand-over on a shared-memory barrier (one arrival per warp) so that this wait is bounded too
         __syncwarp();
         if (lane == 0) mbar_arrive(out_bar);

@@ -127,3 +127,66 @@ def test_diagonal_formula_on_plain_slots():
                     acc += np.roll(x, -q * T) * linear_diagonal(W, b, g, p, q, T, C, n1)
             y += np.roll(acc, -p * n1 * T)
         assert np.allclose(y.reshape(C, T).T, (X @ W)[:, b * C:(b + 1) * C])
+
+
+def test_token_major_packing_with_periodic_diagonals():
+    """The transposed packing (slot r*C + c, one segment per token): a feature shift is the intra-segment shift Psi of
+    App. "Projection Kernel Breakdown" (two rotations, masks folded into the diagonals), the projection is a baby-step /
+    giant-step sum over 2 n1 - 1 and 2 n2 - 1 rotation amounts evaluated by the same `linear`, the result is X @ W, and
+    every diagonal has period C in the slots, i.e. is constant on aligned runs of N / (2C) evaluation indices."""
+    from oracle.ckks import (linear_diagonal_token_major, pack_linear_input_token_major, periodic_eval_runs,
+                             token_major_amounts)
+    p = S.params("small")
+    orc = Oracle(p["log_n"], p["primes"], p["n_q"], p["n_p"], p["dnum"], p["seed"])
+    n = orc.n
+    T, C, n1, n2, level, scale = 32, 16, 4, 4, 4, 2.0**40
+    tokens, d_in, d_out = 50, 24, 20                        # partial token block, partial input and output blocks
+    X, W = S.linear_inputs(p["seed"] + 4, tokens, d_in, d_out)
+    W = W * 10
+    gin, nout, tbs = -(-d_in // C), -(-d_out // C), -(-tokens // T)
+    baby, giant = token_major_amounts(C, n1, n2)
+    assert baby == [0, 1, 1 - C, 2, 2 - C, 3, 3 - C] and giant == [0, 4, 4 - C, 8, 8 - C, 12, 12 - C]
+    for i, a in enumerate(baby[1:], 1):
+        orc.add_galois_key(a, 100 + i)
+    for i, a in enumerate(giant[1:], 1):
+        orc.add_galois_key(a, 200 + i)
+    cts = np.empty((tbs, gin, 2, level, orc.N), dtype=np.uint64)
+    for tb in range(tbs):
+        for g in range(gin):
+            v = pack_linear_input_token_major(X[tb * T:(tb + 1) * T, g * C:(g + 1) * C], T, C, n)
+            cts[tb, g] = orc.encrypt(orc.encode(v, scale, level), 7000 + tb * gin + g)
+    nb, ng, run = len(baby), len(giant), orc.N // (2 * C)
+    diags = np.empty((nout, ng, gin, nb, level, orc.N), dtype=np.uint64)
+    for b in range(nout):
+        for gi in range(ng):
+            for g in range(gin):
+                for bi in range(nb):
+                    v = linear_diagonal_token_major(W, b, g, gi, bi, T, C, n1)
+                    assert np.array_equal(v.reshape(T, C), np.tile(v[:C], (T, 1)))        # period C in the slots
+                    diags[b, gi, g, bi] = orc.encode(v, float(orc.q[level - 1]), level)
+                    small = periodic_eval_runs(diags[b, gi, g, bi], run)                 # asserts constant runs
+                    assert small.shape == (level, 2 * C)
+                    assert np.array_equal(np.repeat(small, run, axis=1), diags[b, gi, g, bi])
+    # the stay / wrap split covers every (input feature, output feature) pair exactly once
+    cover = np.zeros((C, C), dtype=int)
+    for gi in range(ng):
+        for bi in range(nb):
+            v = linear_diagonal_token_major(np.ones((C, C)), 0, 0, gi, bi, T, C, n1)[:C]
+            pp, q = (gi + 1) // 2, (bi + 1) // 2
+            for cpp in np.nonzero(v)[0]:
+                c_out = cpp + C - pp * n1 if (gi and gi % 2 == 0) else cpp - pp * n1
+                cover[(cpp + q) % C, c_out] += 1
+    assert np.all(cover == 1)
+    for hoist, defer in ((False, False), (True, True)):
+        out = orc.linear(cts, diags, dict(n1=nb, n2=ng), {i: 100 + i for i in range(1, nb)},
+                         {i: 200 + i for i in range(1, ng)}, hoist=hoist, defer=defer)
+        Y = np.zeros((tbs * T, nout * C))
+        for tb in range(tbs):
+            for b in range(nout):
+                Y[tb * T:(tb + 1) * T, b * C:(b + 1) * C] = orc.decrypt(out[tb, b], scale, 2).real.reshape(T, C)
+        assert np.abs(Y[:tokens, :d_out] - X @ W).max() < 2.0**-18
+    # a vector that is not periodic is refused by the compression
+    with pytest.raises(AssertionError):
+        periodic_eval_runs(orc.encode(np.arange(n) / n, scale, level), run)
+    # deployed ring: period C = 256 at N = 2^16 leaves 512 of 65536 words per limb
+    assert 65536 // (2 * 256) == 128
