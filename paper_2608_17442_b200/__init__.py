@@ -31,7 +31,7 @@ class FescError(RuntimeError):
 class BsgsDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint32) for n in
                 ("n1", "n2", "in_blocks", "out_blocks", "token_blocks", "n_limbs", "baby_key_base", "giant_key_base",
-                 "hoist", "defer", "packed")]
+                 "hoist", "defer", "packed", "diag_run_log2")]
 
 
 class Info(ctypes.Structure):

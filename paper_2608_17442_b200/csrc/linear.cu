@@ -623,7 +623,9 @@ static int linear_packed(fesc_ctx* ctx, const u64* in, const uint8_t* image, con
         if (tbg == 1) return rc;
     }
     ctx->counters[5] = tbg;
-    const size_t tile_bytes = bsgs_packed_bytes(N, level, 8, terms);     // one tile of 8 rows, either side
+    const size_t tile_bytes = bsgs_packed_bytes(N, level, 8, terms);     // one tile of 8 rows of packed inputs
+    const uint32_t dshift = desc->diag_run_log2;
+    const size_t image_tile_bytes = bsgs_packed_bytes(N >> dshift, level, 8, terms);
     for (uint32_t tb0 = 0; tb0 < tbs; tb0 += tbg) {
         const uint32_t nt = tbs - tb0 < tbg ? tbs - tb0 : tbg;
         for (uint32_t s0 = 0; s0 < nt; s0 += 4) {        // baby rotations of 4 token blocks, packed into their tile
@@ -648,8 +650,8 @@ static int linear_packed(fesc_ctx* ctx, const u64* in, const uint8_t* image, con
         }
         for (uint32_t b0 = 0; b0 < nout; b0 += nb_part) {
             const uint32_t nb = nout - b0 < nb_part ? nout - b0 : nb_part;
-            rc = bsgs_accumulate_packed(ctx, xpk, image + (size_t)(b0 * n2 / 8) * tile_bytes, acc, level, nt, terms, nb * n2,
-                                        qbits <= 50, st);
+            rc = bsgs_accumulate_packed(ctx, xpk, image + (size_t)(b0 * n2 / 8) * image_tile_bytes, acc, level, nt, terms, nb * n2,
+                                        qbits <= 50, dshift, st);
             if (rc != FESC_OK) return rc;
             ctx->counters[2] += (uint64_t)nt * nb * n2 * terms;
             if (desc->defer) {
@@ -688,8 +690,10 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
     cudaStream_t st = (cudaStream_t)stream;
     const size_t ctw = (size_t)2 * level * N;
     const bool packed = desc->packed != 0;
-    if (packed && !bsgs_packed_supported(ctx, level, gin * n1))
-        return fesc_fail(ctx, FESC_EINVAL, "linear: packed diagonals need N a multiple of 8, primes below 2^56 and at most 512 terms");
+    if (!packed && desc->diag_run_log2)
+        return fesc_fail(ctx, FESC_EINVAL, "linear: periodic diagonals (diag_run_log2) are a property of the packed image");
+    if (packed && !bsgs_packed_supported(ctx, level, gin * n1, desc->diag_run_log2))
+        return fesc_fail(ctx, FESC_EINVAL, "linear: packed diagonals need N a multiple of 8, primes below 2^56, at most 512 terms and runs that leave 8 words per limb");
     if (packed) {
         uint32_t bits = 0;
         for (uint32_t i = 0; i < level; i++) {
@@ -803,12 +807,6 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
         FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
         kern<<<grid, 32 * IM_CW, smem, st>>>(rot, diags, acc, ctx->d_pc, N, level, nt, gin * n1, bp_count, pitch); \
     } while (0)
-        if (packed) {
-            rc = bsgs_pack_inputs(ctx, rot, xpk, level, nt, gin * n1, st);
-            if (rc == FESC_OK)
-                rc = bsgs_accumulate_packed(ctx, xpk, (const uint8_t*)d_diags, acc, level, nt, gin * n1, bp_count, qbits <= 50, st);
-            if (rc != FESC_OK) return rc;
-        }
         const bool fp_ok = qbits <= 50 && bsgs_kernel() != 2;
         const bool imma_ok = bsgs_kernel() == 0 && qbits <= 56 && N % IM_CW == 0 && gin * n1 <= 256 && level <= 65535;
         const bool deep = gin * n1 <= 128;       // room for 8 stages beside the rotated inputs

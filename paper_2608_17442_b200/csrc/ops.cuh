@@ -96,7 +96,7 @@ __device__ __forceinline__ u64 imma_recombine(const int (&d)[4][7][4], int sel, 
 
 // packed-operand BSGS accumulate (packed.cu)
 size_t bsgs_packed_bytes(uint32_t N, uint32_t level, uint32_t rows, uint32_t terms);
-bool bsgs_packed_supported(const fesc_ctx* ctx, uint32_t level, uint32_t terms);
+bool bsgs_packed_supported(const fesc_ctx* ctx, uint32_t level, uint32_t terms, uint32_t dshift);
 int bsgs_pack_inputs(fesc_ctx* ctx, const u64* rot, uint8_t* xpk, uint32_t level, uint32_t tbs, uint32_t terms, cudaStream_t st);
 int bsgs_accumulate_packed(fesc_ctx* ctx, const uint8_t* xpk, const uint8_t* dpk, u64* acc, uint32_t level, uint32_t tbs,
-                           uint32_t terms, uint32_t bp_count, bool fp, cudaStream_t st);
+                           uint32_t terms, uint32_t bp_count, bool fp, uint32_t dshift, cudaStream_t st);

@@ -100,7 +100,7 @@ template <bool FP, int KSR>
 __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
     const uint8_t* __restrict__ xpk, const uint8_t* __restrict__ dpk, u64* __restrict__ acc,
     const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level, uint32_t tbs, uint32_t ksteps, uint32_t bp_count,
-    uint32_t* __restrict__ status) {
+    uint32_t dshift, uint32_t* __restrict__ status) {
     // per warp: PK_STAGES ring slots, KSR input images; then per warp PK_STAGES + 1 barriers
     extern __shared__ __align__(128) uint8_t ring[];
     constexpr uint32_t WARP_BYTES = (PK_STAGES + KSR) * PK_FRAG;
@@ -114,9 +114,12 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
     const uint32_t my_ring = (uint32_t)__cvta_generic_to_shared(ring) + warp * WARP_BYTES;
     const uint32_t my_bar = (uint32_t)__cvta_generic_to_shared(ring) + PK_WARPS * WARP_BYTES + warp * ((PK_STAGES + 1) * 8);
     const uint8_t* my_img = ring + warp * WARP_BYTES;
-    // images of this warp's coefficient: k-steps of one (b,p) tile are PK_STAGE apart, tiles tile_stride apart
-    const uint8_t* src = dpk + ((size_t)l * tiles + ct) * ksteps * PK_STAGE + coef * PK_FRAG;
-    const size_t tile_stride = (size_t)level * tiles * ksteps * PK_STAGE;
+    // images of this warp's coefficient: k-steps of one (b,p) tile are PK_STAGE apart, tiles tile_stride apart.  Periodic
+    // diagonals (dshift > 0) hold one image per aligned run of 2^dshift coefficients: the image of a ring 2^dshift times
+    // smaller, shared by the coefficients of the run.
+    const uint32_t run = (ct * PK_CW + coef) >> dshift, tiles_d = tiles >> dshift;
+    const uint8_t* src = dpk + ((size_t)l * tiles_d + (run >> 3)) * ksteps * PK_STAGE + (run & 7) * PK_FRAG;
+    const size_t tile_stride = (size_t)level * tiles_d * ksteps * PK_STAGE;
     const uint8_t* ximg = xpk + ((((size_t)tbt * level + l) * tiles + ct) * ksteps * PK_CW + coef) * PK_FRAG;
     uint32_t ld_ks = 0, ld_s = 0;                         // next stage to request (lane 0)
     auto request = [&](uint32_t slot) {
@@ -240,7 +243,7 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
 }
 
 int bsgs_accumulate_packed(fesc_ctx* ctx, const uint8_t* xpk, const uint8_t* dpk, u64* acc, uint32_t level, uint32_t tbs,
-                           uint32_t terms, uint32_t bp_count, bool fp, cudaStream_t st) {
+                           uint32_t terms, uint32_t bp_count, bool fp, uint32_t dshift, cudaStream_t st) {
     const uint32_t N = ctx->N, ksteps = (terms + 31) / 32;
     dim3 grid(2 * (N / PK_CW) * ((tbs + 3) / 4), level);
 #define PK_LAUNCH(FP, KSR)                                                                                        \
@@ -248,7 +251,7 @@ int bsgs_accumulate_packed(fesc_ctx* ctx, const uint8_t* xpk, const uint8_t* dpk
         const size_t smem = (size_t)PK_WARPS * ((PK_STAGES + KSR) * PK_FRAG + (PK_STAGES + 1) * 8) + 2 * 256 * 8 + 8; \
         auto kern = k_bsgs_accumulate_packed<FP, KSR>;                                                            \
         FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        kern<<<grid, 32 * PK_WARPS, smem, st>>>(xpk, dpk, acc, ctx->d_pc, N, level, tbs, ksteps, bp_count,        \
+        kern<<<grid, 32 * PK_WARPS, smem, st>>>(xpk, dpk, acc, ctx->d_pc, N, level, tbs, ksteps, bp_count, dshift, \
                                                 ctx->d_status);                                                   \
     } while (0)
     prof_begin(ctx, PF_BSGS, st);
@@ -277,22 +280,24 @@ static uint32_t max_prime_bits(const fesc_ctx* ctx, uint32_t level) {
     }
     return qbits;
 }
-bool bsgs_packed_supported(const fesc_ctx* ctx, uint32_t level, uint32_t terms) {
+bool bsgs_packed_supported(const fesc_ctx* ctx, uint32_t level, uint32_t terms, uint32_t dshift) {
     return ctx->N % PK_CW == 0 && level >= 1 && level <= ctx->n_q && max_prime_bits(ctx, level) <= 56 && terms >= 1 &&
-           terms <= 512;
+           terms <= 512 && dshift < 32 && (ctx->N >> dshift) >= PK_CW;
 }
 
 extern "C" size_t fesc_linear_packed_bytes(const fesc_ctx* ctx, const fesc_bsgs_desc* desc) {
     if (!ctx || !desc) return 0;
-    return bsgs_packed_bytes(ctx->N, desc->n_limbs, desc->out_blocks * desc->n2, desc->in_blocks * desc->n1);
+    if (desc->diag_run_log2 >= 32) return 0;
+    return bsgs_packed_bytes(ctx->N >> desc->diag_run_log2, desc->n_limbs, desc->out_blocks * desc->n2, desc->in_blocks * desc->n1);
 }
 
 extern "C" int fesc_linear_pack_diags(fesc_ctx* ctx, const uint64_t* d_diags, const fesc_bsgs_desc* desc, uint32_t first,
                                       uint32_t count, void* d_packed, void* stream) {
     if (!ctx || !d_diags || !desc || !d_packed) return FESC_EINVAL;
-    const uint32_t N = ctx->N, level = desc->n_limbs, terms = desc->in_blocks * desc->n1, bp_count = desc->out_blocks * desc->n2;
-    if (!bsgs_packed_supported(ctx, level, terms))
-        return fesc_fail(ctx, FESC_EINVAL, "pack_diags: needs N a multiple of 8, primes below 2^56 and at most 512 terms");
+    const uint32_t level = desc->n_limbs, terms = desc->in_blocks * desc->n1, bp_count = desc->out_blocks * desc->n2;
+    if (!bsgs_packed_supported(ctx, level, terms, desc->diag_run_log2))
+        return fesc_fail(ctx, FESC_EINVAL, "pack_diags: needs N a multiple of 8, primes below 2^56, at most 512 terms and runs that leave 8 words per limb");
+    const uint32_t N = ctx->N >> desc->diag_run_log2;       // words per limb of the diagonals handed in
     if (first % 8 || first >= bp_count || !count || count > bp_count - first)
         return fesc_fail(ctx, FESC_EINVAL, "pack_diags: the range must start at a multiple of 8 and lie inside the (b,p) pairs");
     if ((first + count) % 8 && first + count != bp_count)

@@ -271,3 +271,67 @@ def test_linear_full_ring_one_block():
     err_m = np.abs(orc.decrypt(got_m[0, 0], scale, 2).real.reshape(C, T).T - X @ W).max()
     print("hoisted + deferred: max |decrypt - X@W| = 2^%.2f" % np.log2(err_m))
     assert err_m < 2.0**-18
+
+
+def test_linear_token_major_packing_with_periodic_diagonals():
+    """Token-major packing (slot r*C + c): the projection runs through the same fesc_linear with 2 n1 - 1 baby and
+    2 n2 - 1 giant rotation amounts, and its diagonals are periodic, so the packed image holds one operand per aligned
+    run of N/(2C) evaluation indices (desc.diag_run_log2 = 5 here: 32 times smaller).  Residues equal the oracle's
+    (which multiplies the full-size diagonals), values equal X @ W."""
+    import torch
+    import paper_2608_17442_b200 as fesc
+    from oracle.ckks import (linear_diagonal_token_major, pack_linear_input_token_major, periodic_eval_runs,
+                             token_major_amounts)
+
+    pair = ctx_pair("small")
+    ctx, orc, p = pair
+    n = orc.n
+    T, C, n1, n2, level, scale, kb = 32, 16, 4, 4, 5, 2.0**40, 9000
+    tokens, d_in, d_out = 150, 40, 20            # 5 token blocks (two groups), 3 input blocks, 2 output blocks
+    X, W = S.linear_inputs(p["seed"] + 14, tokens, d_in, d_out)
+    W = W * 10
+    gin, nout, tbs = -(-d_in // C), -(-d_out // C), -(-tokens // T)
+    baby, giant = token_major_amounts(C, n1, n2)
+    nb, ng, run = len(baby), len(giant), orc.N // (2 * C)
+    for i, a in enumerate(baby[1:], 1):
+        add_key(pair, a, kb + i)
+    for i, a in enumerate(giant[1:], 1):
+        add_key(pair, a, kb + 500 + i)
+    cts = np.empty((tbs, gin, 2, level, orc.N), dtype=np.uint64)
+    for tb in range(tbs):
+        for g in range(gin):
+            v = pack_linear_input_token_major(X[tb * T:(tb + 1) * T, g * C:(g + 1) * C], T, C, n)
+            cts[tb, g] = orc.encrypt(orc.encode(v, scale, level), 7900 + tb * gin + g)
+    diags = np.empty((nout, ng, gin, nb, level, orc.N), dtype=np.uint64)
+    small = np.empty((nout, ng, gin, nb, level, orc.N // run), dtype=np.uint64)
+    for b in range(nout):
+        for gi in range(ng):
+            for g in range(gin):
+                for bi in range(nb):
+                    diags[b, gi, g, bi] = orc.encode(linear_diagonal_token_major(W, b, g, gi, bi, T, C, n1),
+                                                     float(orc.q[level - 1]), level)
+                    small[b, gi, g, bi] = periodic_eval_runs(diags[b, gi, g, bi], run)
+    shift = run.bit_length() - 1
+    desc = fesc.BsgsDesc(nb, ng, gin, nout, tbs, level, kb, kb + 500, 1, 1, 1, shift)
+    image = torch.full((ctx.linear_packed_bytes(desc),), 0x5A, dtype=torch.uint8, device="cuda")
+    full_desc = fesc.BsgsDesc(nb, ng, gin, nout, tbs, level, kb, kb + 500, 1, 1, 1, 0)
+    assert ctx.linear_packed_bytes(desc) * run == ctx.linear_packed_bytes(full_desc)
+    pairs = nout * ng
+    flat = to_dev(small.reshape(pairs, gin, nb, level, orc.N // run))
+    ctx.linear_pack_diags(flat[:8], desc, 0, 8, image)
+    ctx.linear_pack_diags(flat[8:].contiguous(), desc, 8, pairs - 8, image)
+    out = torch.empty((tbs, nout, 2, level - 1, orc.N), dtype=torch.int64, device="cuda")
+    ctx.linear(to_dev(cts), image, desc, out)
+    got = to_host(out)
+    want = orc.linear(cts, diags, dict(n1=nb, n2=ng), {i: kb + i for i in range(1, nb)},
+                      {i: kb + 500 + i for i in range(1, ng)}, hoist=True, defer=True)
+    assert np.array_equal(got, want)
+    Y = np.zeros((tbs * T, nout * C))
+    for tb in range(tbs):
+        for b in range(nout):
+            Y[tb * T:(tb + 1) * T, b * C:(b + 1) * C] = orc.decrypt(got[tb, b], scale, 2).real.reshape(T, C)
+    assert np.abs(Y[:tokens, :d_out] - X @ W).max() < 2.0**-18
+    # periodic diagonals are a property of the packed image
+    with pytest.raises(fesc.FescError) as e:
+        ctx.linear(to_dev(cts), to_dev(diags), fesc.BsgsDesc(nb, ng, gin, nout, tbs, level, kb, kb + 500, 1, 1, 0, shift), out)
+    assert e.value.code == fesc.EINVAL
