@@ -39,6 +39,8 @@ D_IN, D_OUT, TOKENS = 768, 3352, 2048
 PROJ = "in_proj"            # "out_proj" (1536 -> 768) is selected by --workload out_proj
 LEVEL = 24
 BABY_BASE, GIANT_BASE = 1000, 1500
+DIAG_SHIFT = 0              # log2 of the run length of periodic diagonals (token-major packing): 7 at C = 256
+KEY_AMOUNTS = None          # (baby amounts, giant amounts) in slots when they are not q*T and p*n1*T
 
 
 def workload_dims(scale_down: int = 1):
@@ -158,19 +160,20 @@ def make_inputs(primes, n, gin, nout, tbs, seed, device, ctx=None, desc=None):
             r = S.hashed_residues(seed, tb * gin + g, q, 2 * n, device=device)      # [LEVEL, 2n]
             ct[tb, g] = r.view(LEVEL, 2, n).permute(1, 0, 2)
     packed = bool(desc is not None and desc.packed)
+    nd = n >> (desc.diag_run_log2 if desc is not None else 0)      # words per limb of a diagonal (periodic: one per run)
     per = 1                         # output blocks per pack call: a range must start at a multiple of 8 (b,p) pairs
     while (per * N2) % 8 and per < nout:
         per += 1
     if packed:
         assert (per * N2) % 8 == 0 or per == nout
         diags = torch.empty((ctx.linear_packed_bytes(desc),), dtype=torch.uint8, device=device)
-        one = torch.empty((per, N2, gin, N1, LEVEL, n), dtype=torch.int64, device=device)
+        one = torch.empty((per, N2, gin, N1, LEVEL, nd), dtype=torch.int64, device=device)
     else:
         diags = torch.empty((nout, N2, gin, N1, LEVEL, n), dtype=torch.int64, device=device)
     for b in range(nout):
         for p in range(N2):
-            r = S.hashed_residues(seed, 100000 + b * N2 + p, q, gin * N1 * n, device=device)
-            (one[b % per] if packed else diags[b])[p] = r.view(LEVEL, gin, N1, n).permute(1, 2, 0, 3)
+            r = S.hashed_residues(seed, 100000 + b * N2 + p, q, gin * N1 * nd, device=device)
+            (one[b % per] if packed else diags[b])[p] = r.view(LEVEL, gin, N1, nd).permute(1, 2, 0, 3)
             del r
         if packed and (b % per == per - 1 or b == nout - 1):
             first, cnt = (b // per) * per, b % per + 1
@@ -351,12 +354,16 @@ def measure_projection(args, ctx, dev, rank, world, key_base):
     p = S.params("full")
     n = ctx.N
     bb, gb = key_base
+    baby = KEY_AMOUNTS[0] if KEY_AMOUNTS else [q * T_SEG for q in range(N1)]
+    giant = KEY_AMOUNTS[1] if KEY_AMOUNTS else [g * N1 * T_SEG for g in range(N2)]
+    assert len(baby) == N1 and len(giant) == N2
     for q in range(1, N1):
-        ctx.add_galois_key(q * T_SEG, bb + q)
+        ctx.add_galois_key(baby[q], bb + q)
     for g in range(1, N2):
-        ctx.add_galois_key(g * N1 * T_SEG, gb + g)
+        ctx.add_galois_key(giant[g], gb + g)
     gin, nout, tbs = workload_dims(1)
-    desc = fesc.BsgsDesc(N1, N2, gin, nout, tbs, LEVEL, bb, gb, int(args.hoist), int(args.defer), int(args.packed))
+    desc = fesc.BsgsDesc(N1, N2, gin, nout, tbs, LEVEL, bb, gb, int(args.hoist), int(args.defer), int(args.packed),
+                         DIAG_SHIFT if args.packed else 0)
     ct, diags = make_inputs(p["primes"], n, gin, nout, tbs, S.config_seed(5) + rank, dev, ctx, desc)
     out = torch.empty((tbs, nout, 2, LEVEL - 1, n), dtype=torch.int64, device=dev)
     torch.cuda.empty_cache()
@@ -382,7 +389,8 @@ def measure_projection(args, ctx, dev, rank, world, key_base):
     res = {"ms": ms, "key_switches": ks, "key_switches_per_s": ks / (ms * 1e-3), "gpu_launches": (c1[4] - c0[4]) // args.steps,
            "clocks": clocks, "kernel_breakdown": {k: {"ms": round(v[0], 2), "records": v[1]} for k, v in fam.items() if v[1]},
            "workload": workload_text(args), "input_cts": tbs * gin, "output_cts": tbs * nout,
-           "diagonals_gib": diags.numel() * diags.element_size() / 2**30, "token_blocks_per_group": int(c1[5])}
+           "diagonals": nout * N2 * gin * N1, "diagonals_gib": diags.numel() * diags.element_size() / 2**30,
+           "token_blocks_per_group": int(c1[5])}
     del ct, diags, out
     return res
 
@@ -1165,6 +1173,27 @@ def run_stages(args, ctx, dev):
         stages["out_proj"] = measure_projection(sub, ctx, dev, rank=0, world=1, key_base=(BABY_BASE + 2000, GIANT_BASE + 2000))
     finally:
         D_IN, D_OUT, PROJ, N1, N2 = saved
+    torch.cuda.empty_cache()
+    ctx.trim()
+    # in_proj once more in the token-major packing (slot r*C + c): feature shifts are intra-segment shifts (two
+    # rotations each: 63 baby and 15 giant amounts), the diagonals are periodic and their packed image is 128 times
+    # smaller per diagonal, so that the weights of a whole model fit beside the activations
+    global DIAG_SHIFT, KEY_AMOUNTS
+    saved = (D_IN, D_OUT, PROJ, N1, N2)
+    n1t, n2t = 32, 8
+    KEY_AMOUNTS = ([0] + [a for q in range(1, n1t) for a in (q, q - C_SEG)],
+                   [0] + [a for pp in range(1, n2t) for a in (pp * n1t, pp * n1t - C_SEG)])
+    PROJ, N1, N2, DIAG_SHIFT = "in_proj (token-major packing, periodic diagonals)", 2 * n1t - 1, 2 * n2t - 1, 7
+    os.environ["FESC_BSGS_GROUP_GIB"] = "64"      # 189 terms x 210 accumulators per token block: groups of 4 need 55 GiB of scratch
+    try:
+        stages["in_proj_token_major"] = measure_projection(sub, ctx, dev, rank=0, world=1,
+                                                           key_base=(BABY_BASE + 4000, GIANT_BASE + 4000))
+        stages["in_proj_token_major"]["note"] = ("same 768 -> 3352 job; packed diagonals %.2f GiB instead of 110.25 GiB"
+                                                 % stages["in_proj_token_major"]["diagonals_gib"])
+    finally:
+        D_IN, D_OUT, PROJ, N1, N2 = saved
+        DIAG_SHIFT, KEY_AMOUNTS = 0, None
+        os.environ.pop("FESC_BSGS_GROUP_GIB", None)
     torch.cuda.empty_cache()
     ctx.trim()
     stages["conv"] = keep(run_conv(sub, ctx, quiet=True))
