@@ -14,12 +14,13 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("FESC_LIB", os.path.join(_HERE, "libfesc_b200.so"))
 
-OK, EINVAL, ENOMEM, ECUDA, ELEVEL, ENOKEY, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
+OK, EINVAL, ENOMEM, ECUDA, ELEVEL, ENOKEY, ETIMEOUT, EBOUNDS = 0, -1, -2, -3, -4, -5, -6, -7
 CONJ = -(1 << 31)
 NET_BRENT_KUNG, NET_KOGGE_STONE, NET_SKLANSKY = 0, 1, 2     # fesc_scan_desc.network
 RELIN_KEY_ID = 0
 
 _lib = None
+_debug_bounds = False      # the loaded library is the bounds-checking debug build
 
 
 class FescError(RuntimeError):
@@ -102,6 +103,9 @@ def lib():
             "fesc_ctx_info": [vp, c.POINTER(Info)],
             "fesc_ctx_test_fail_allocs": [vp, u32],
             "fesc_scan_contract": [vp, vp, vp, vp, vp, c.POINTER(ScanDesc), c.POINTER(ScanConsts), vp, vp],
+            "fesc_debug_bounds_register": [vp, sz],
+            "fesc_debug_bounds_clear": [],
+            "fesc_debug_bounds_report": [c.POINTER(u32), c.POINTER(u32), c.POINTER(u64), c.POINTER(u64)],
         }
         for name, args in sig.items():
             f = getattr(L, name)
@@ -115,6 +119,31 @@ def lib():
         L.fesc_ctx_num_digits.restype = u32
         _lib = L
     return _lib
+
+
+def debug_bounds() -> bool:
+    """True when the loaded library is the bounds-checking debug build (FESC_LIB pointing at libfesc_b200_dbg.so):
+    the binding then registers the extent of every tensor it passes, and Context.sync raises FescError(EBOUNDS) after
+    a kernel skipped a region outside every known extent.  The first call needs a GPU."""
+    global _debug_bounds
+    if not getattr(debug_bounds, "asked", False):
+        _debug_bounds = lib().fesc_debug_bounds_clear() == OK
+        debug_bounds.asked = True
+    return _debug_bounds
+
+
+def debug_bounds_clear():
+    if lib().fesc_debug_bounds_clear() != OK:
+        raise FescError(EINVAL, "not a debug build")
+
+
+def debug_bounds_report():
+    """(skipped regions since the last report, first site = file id << 16 | line, first address, its size in bytes)."""
+    c = ctypes
+    h, s, a, b = c.c_uint32(), c.c_uint32(), c.c_uint64(), c.c_uint64()
+    if lib().fesc_debug_bounds_report(c.byref(h), c.byref(s), c.byref(a), c.byref(b)) != OK:
+        raise FescError(EINVAL, "not a debug build")
+    return h.value, s.value, a.value, b.value
 
 
 def params_info(log_n: int, primes, n_q: int, n_p: int, dnum: int) -> Info:
@@ -133,9 +162,19 @@ def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
+def _raw(t):
+    """Data pointer of a contiguous CUDA tensor (None passes through); a debug build learns the tensor's extent."""
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous()
+    if debug_bounds():
+        lib().fesc_debug_bounds_register(t.data_ptr(), t.numel() * t.element_size())
+    return t.data_ptr()
+
+
 def _ptr(t):
-    assert t.is_cuda and t.is_contiguous() and t.element_size() == 8
-    return ctypes.c_void_p(t.data_ptr())
+    assert t.element_size() == 8
+    return ctypes.c_void_p(_raw(t))
 
 
 class Context:
@@ -271,7 +310,7 @@ class Context:
     def linear(self, ct_in, diags, desc: BsgsDesc, ct_out):
         """diags: the residue tensor, or (desc.packed = 1) the uint8 image filled by linear_pack_diags."""
         assert diags.is_cuda and diags.is_contiguous()
-        self._chk(lib().fesc_linear(self.h, _ptr(ct_in), ctypes.c_void_p(diags.data_ptr()), ctypes.byref(desc),
+        self._chk(lib().fesc_linear(self.h, _ptr(ct_in), ctypes.c_void_p(_raw(diags)), ctypes.byref(desc),
                                     _ptr(ct_out), _stream()))
 
     def linear_packed_bytes(self, desc: BsgsDesc) -> int:
@@ -282,7 +321,7 @@ class Context:
         their place inside the uint8 CUDA tensor `packed` (linear_packed_bytes(desc) bytes)."""
         assert packed.is_cuda and packed.is_contiguous() and packed.element_size() == 1
         self._chk(lib().fesc_linear_pack_diags(self.h, _ptr(diags), ctypes.byref(desc), first, count,
-                                               ctypes.c_void_p(packed.data_ptr()), _stream()))
+                                               ctypes.c_void_p(_raw(packed)), _stream()))
 
     def info(self) -> Info:
         out = Info()
@@ -300,7 +339,7 @@ class Context:
         n = (desc.n_limbs + 1) ** 2
         hs = (ctypes.c_uint64 * n)(*[int(v) for v in adj_s])
         hp = (ctypes.c_uint64 * n)(*[int(v) for v in (adj_p if adj_p is not None else [0] * n)])
-        ptr = lambda t: t.data_ptr() if t is not None else None
+        ptr = _raw
         cs = ScanConsts(ptr(mask_x), ptr(mask_b), ptr(mask_a), ptr(mask_out),
                         ctypes.cast(hs, ctypes.c_void_p).value, ctypes.cast(hp, ctypes.c_void_p).value,
                         *([ptr(t) for t in group_masks] if group_masks else [None] * 6),

@@ -14,6 +14,34 @@
 typedef unsigned long long u64;
 typedef unsigned __int128 u128;
 
+// ---------------------------------------------------------------------------------------
+// Debug build (-DFESC_DEBUG_BOUNDS -rdc=true): every kernel checks the regions its CTA (or thread) is about to touch
+// against a table of known extents: the library's own allocations and the caller's buffers as registered through
+// fesc_debug_bounds_register.  A region outside every extent is recorded (count, first site = file id << 16 | line,
+// address, size) and the accesses to it are skipped, so that a wrong index never reaches memory; nothing traps.
+// Checks sit where the outcome is the same for every thread that later meets a barrier.
+// ---------------------------------------------------------------------------------------
+#ifndef FESC_DBG_FILE
+#define FESC_DBG_FILE 0
+#endif
+#ifdef FESC_DEBUG_BOUNDS
+#define FESC_DBG_MAX 4096
+struct DbgTable {
+    uint32_t n, hits, first_site, pad;
+    unsigned long long first_addr, first_bytes;
+    unsigned long long lo[FESC_DBG_MAX], hi[FESC_DBG_MAX];
+};
+extern __device__ DbgTable g_fesc_dbg;
+__device__ bool fesc_dbg_region(const void* p, size_t bytes, uint32_t site);
+#define DBG_REGION(p, bytes) fesc_dbg_region((const void*)(p), (size_t)(bytes), ((uint32_t)FESC_DBG_FILE << 16) | __LINE__)
+void dbg_note_alloc(const void* p, size_t bytes);
+void dbg_note_free(const void* p);
+#else
+#define DBG_REGION(p, bytes) true
+static inline void dbg_note_alloc(const void*, size_t) {}
+static inline void dbg_note_free(const void*) {}
+#endif
+
 #define FESC_MAX_PRIMES 64
 #define FESC_MAX_SPECIAL 8
 #define FESC_MAX_ALPHA 8

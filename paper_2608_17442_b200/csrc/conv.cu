@@ -5,6 +5,7 @@
 // Every ciphertext is decomposed once and rotated by its 2(d_conv-1) amounts (hoisted rotations); the rotations by
 // T - r are kept for the next token block.  The masked sums use the plain ct-pt multiply-accumulate, then the bias
 // plaintext is added to c0 and the block is rescaled.
+#define FESC_DBG_FILE 7   // file id in the sites a debug build reports
 #include "ops.cuh"
 
 // c0 of every ciphertext += its plaintext (pt_stride words between plaintexts)
@@ -14,6 +15,7 @@ __global__ void __launch_bounds__(256) k_ct_add_pt(u64* __restrict__ ct, size_t 
     const uint32_t l = blockIdx.y, b = blockIdx.z;
     if (c >= N) return;
     u64* o = ct + (size_t)b * ct_stride + (size_t)l * N + c;
+    if (!DBG_REGION(o - c, N * sizeof(u64)) || !DBG_REGION(pt + (size_t)b * pt_stride + (size_t)l * N, N * sizeof(u64))) return;
     *o = addmod(*o, pt[(size_t)b * pt_stride + (size_t)l * N + c], pcs[l].q);
 }
 

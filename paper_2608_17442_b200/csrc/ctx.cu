@@ -1,5 +1,121 @@
 // Context: parameter validation, twiddle / basis-conversion tables, seeded key generation.
+#define FESC_DBG_FILE 1   // file id in the sites a debug build reports
 #include "common.cuh"
+
+#include <algorithm>
+
+// Every device allocation of the library goes through these two, so that a debug build knows the extents.
+template <typename T>
+static cudaError_t dev_alloc(T** p, size_t bytes) {
+    const cudaError_t e = cudaMalloc((void**)p, bytes);
+    if (e == cudaSuccess) dbg_note_alloc(*p, bytes);
+    return e;
+}
+static void dev_free(void* p) {
+    if (p) dbg_note_free(p);
+    cudaFree(p);
+}
+
+#ifdef FESC_DEBUG_BOUNDS
+__device__ DbgTable g_fesc_dbg;
+__device__ bool fesc_dbg_region(const void* p, size_t bytes, uint32_t site) {
+    const unsigned long long lo = (unsigned long long)p, hi = lo + bytes;
+    // the table is sorted and its ranges are disjoint: the only candidate is the last range that starts at or below lo
+    uint32_t a = 0, b = g_fesc_dbg.n;
+    while (a < b) {
+        const uint32_t m = (a + b) >> 1;
+        if (g_fesc_dbg.lo[m] <= lo) a = m + 1;
+        else b = m;
+    }
+    if (a > 0 && hi <= g_fesc_dbg.hi[a - 1]) return true;
+    if (atomicAdd(&g_fesc_dbg.hits, 1u) == 0) {
+        g_fesc_dbg.first_site = site;
+        g_fesc_dbg.first_addr = lo;
+        g_fesc_dbg.first_bytes = bytes;
+    }
+    return false;
+}
+// Host mirror: the library's allocations and the caller's registered buffers (oldest replaced when full).
+#define FESC_DBG_CALLERS 192
+struct DbgHost {
+    std::vector<std::pair<unsigned long long, unsigned long long>> own, caller;
+    size_t next = 0;
+};
+static DbgHost& dbg_host() {
+    static DbgHost h;
+    return h;
+}
+static void dbg_upload() {
+    DbgHost& h = dbg_host();
+    std::vector<std::pair<unsigned long long, unsigned long long>> all(h.own);
+    all.insert(all.end(), h.caller.begin(), h.caller.end());
+    std::sort(all.begin(), all.end());
+    static DbgTable t;      // host staging copy; the counters are left as the device has them
+    uint32_t n = 0;
+    for (auto& r : all) {   // overlapping ranges (a view inside a registered tensor) are joined; touching ones are not
+        if (n && r.first < t.hi[n - 1]) {
+            if (r.second > t.hi[n - 1]) t.hi[n - 1] = r.second;
+        } else if (n < FESC_DBG_MAX) {
+            t.lo[n] = r.first, t.hi[n] = r.second, n++;
+        }
+    }
+    cudaDeviceSynchronize();
+    cudaMemcpyToSymbol(g_fesc_dbg, &n, sizeof(n), offsetof(DbgTable, n));
+    cudaMemcpyToSymbol(g_fesc_dbg, t.lo, sizeof(u64) * (n ? n : 1), offsetof(DbgTable, lo));
+    cudaMemcpyToSymbol(g_fesc_dbg, t.hi, sizeof(u64) * (n ? n : 1), offsetof(DbgTable, hi));
+}
+void dbg_note_alloc(const void* p, size_t bytes) {
+    dbg_host().own.push_back({(unsigned long long)p, (unsigned long long)p + bytes});
+    dbg_upload();
+}
+void dbg_note_free(const void* p) {
+    auto& v = dbg_host().own;
+    for (size_t i = 0; i < v.size(); i++)
+        if (v[i].first == (unsigned long long)p) {
+            v.erase(v.begin() + i);
+            break;
+        }
+    dbg_upload();
+}
+extern "C" int fesc_debug_bounds_register(const void* d_ptr, size_t bytes) {
+    if (!d_ptr || !bytes) return FESC_EINVAL;
+    DbgHost& h = dbg_host();
+    const unsigned long long lo = (unsigned long long)d_ptr, hi = lo + bytes;
+    for (auto& r : h.caller)
+        if (r.first == lo) {          // the same base address again: the newest extent counts
+            if (r.second == hi) return FESC_OK;
+            r.second = hi;
+            dbg_upload();
+            return FESC_OK;
+        }
+    if (h.caller.size() < FESC_DBG_CALLERS) h.caller.push_back({lo, hi});
+    else h.caller[h.next++ % FESC_DBG_CALLERS] = {lo, hi};
+    dbg_upload();
+    return FESC_OK;
+}
+extern "C" int fesc_debug_bounds_clear(void) {
+    dbg_host().caller.clear();
+    dbg_host().next = 0;
+    dbg_upload();
+    return FESC_OK;
+}
+extern "C" int fesc_debug_bounds_report(uint32_t* hits, uint32_t* first_site, uint64_t* first_addr, uint64_t* first_bytes) {
+    DbgTable t;
+    if (cudaDeviceSynchronize() != cudaSuccess) return FESC_ECUDA;
+    if (cudaMemcpyFromSymbol(&t, g_fesc_dbg, offsetof(DbgTable, lo)) != cudaSuccess) return FESC_ECUDA;
+    if (hits) *hits = t.hits;
+    if (first_site) *first_site = t.first_site;
+    if (first_addr) *first_addr = t.first_addr;
+    if (first_bytes) *first_bytes = t.first_bytes;
+    const uint32_t zero[4] = {0, 0, 0, 0};      // hits, first_site, pad: start a new record
+    cudaMemcpyToSymbol(g_fesc_dbg, zero, 12, offsetof(DbgTable, hits));
+    return FESC_OK;
+}
+#else
+extern "C" int fesc_debug_bounds_register(const void*, size_t) { return FESC_EINVAL; }
+extern "C" int fesc_debug_bounds_clear(void) { return FESC_EINVAL; }
+extern "C" int fesc_debug_bounds_report(uint32_t*, uint32_t*, uint64_t*, uint64_t*) { return FESC_EINVAL; }
+#endif
 
 // ---------------------------------------------------------------------------------------
 // host modular arithmetic (table construction only)
@@ -74,6 +190,7 @@ __global__ void k_sample_uniform(u64* __restrict__ out, const PrimeConst* __rest
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
     u64 w = draw(seed, tag_base | ((u64)limb << 48), i);
+    if (!DBG_REGION(out + (size_t)limb * N, N * sizeof(u64))) return;
     out[(size_t)limb * N + i] = mulhi(w, pcs[limb].q);
 }
 // kind 0: ternary, kind 1: centred binomial (eta 21); the same small integer reduced on every limb
@@ -82,6 +199,7 @@ __global__ void k_sample_small(u64* __restrict__ out, const PrimeConst* __restri
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
     u64 w = draw(seed, tag, i);
+    if (!DBG_REGION(out, (size_t)n_limbs * N * sizeof(u64))) return;
     long long v;
     if (kind == 0) {
         v = (long long)mulhi(w, 3) - 1;
@@ -103,6 +221,9 @@ __global__ void k_make_b(u64* __restrict__ b, const u64* __restrict__ a, const u
     if (i >= N) return;
     const PrimeConst pc = pcs[limb];
     const size_t o = (size_t)limb * N + i;
+    if (!DBG_REGION(b + o - i, N * sizeof(u64)) || !DBG_REGION(a + o - i, N * sizeof(u64)) || !DBG_REGION(s + o - i, N * sizeof(u64)) ||
+        !DBG_REGION(e + o - i, N * sizeof(u64)) || !DBG_REGION(sp + o - i, N * sizeof(u64)))
+        return;
     u64 v = submod(e[o], mulmod(a[o], s[o], pc), pc.q);
     if (limb >= dig_lo && limb < dig_hi) v = addmod(v, mulmod(Pmod[limb], sp[o], pc), pc.q);
     b[o] = v;
@@ -113,6 +234,7 @@ __global__ void k_square(u64* __restrict__ out, const u64* __restrict__ s, const
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
     const size_t o = (size_t)limb * N + i;
+    if (!DBG_REGION(out + o - i, N * sizeof(u64)) || !DBG_REGION(s + o - i, N * sizeof(u64))) return;
     out[o] = mulmod(s[o], s[o], pcs[limb]);
 }
 // out[t] = in[pi_g(t)]: the Galois map in bit-reversed evaluation order
@@ -124,6 +246,7 @@ __global__ void k_autom_rows(u64* __restrict__ out, const u64* __restrict__ in, 
     uint32_t u = __brev(t) >> (32 - log_n);
     uint32_t e = (uint32_t)(((2ull * u + 1) * g) & (2ull * N - 1));
     uint32_t src = __brev((e - 1) >> 1) >> (32 - log_n);
+    if (src >= N || !DBG_REGION(out + row * N, N * sizeof(u64)) || !DBG_REGION(in + row * N, N * sizeof(u64))) return;
     out[row * N + t] = in[row * N + src];
 }
 
@@ -132,7 +255,7 @@ int ctx_scratch(fesc_ctx* ctx, size_t bytes, u64** out) {
     if (bytes > ctx->scratch_bytes) {
         if (ctx->d_scratch) {
             FESC_CHECK_CUDA(ctx, cudaDeviceSynchronize());
-            cudaFree(ctx->d_scratch);
+            dev_free(ctx->d_scratch);
             ctx->d_scratch = nullptr;
             ctx->scratch_bytes = 0;
             ctx->counters[3] = 0;
@@ -140,7 +263,7 @@ int ctx_scratch(fesc_ctx* ctx, size_t bytes, u64** out) {
         size_t want = (bytes + (1u << 20) - 1) & ~(size_t)((1u << 20) - 1);
         const bool injected = ctx->fail_allocs > 0;       // test hook: report the failure without calling the driver
         if (injected) ctx->fail_allocs--;
-        if (injected || cudaMalloc(&ctx->d_scratch, want) != cudaSuccess) {
+        if (injected || dev_alloc(&ctx->d_scratch, want) != cudaSuccess) {
             ctx->d_scratch = nullptr;
             cudaGetLastError();
             return fesc_fail(ctx, FESC_ENOMEM, "scratch allocation of " + std::to_string(want) + " bytes failed");
@@ -154,7 +277,7 @@ int ctx_scratch(fesc_ctx* ctx, size_t bytes, u64** out) {
 
 template <typename T>
 static int upload(fesc_ctx* ctx, T** d, const std::vector<T>& h) {
-    if (cudaMalloc(d, h.size() * sizeof(T)) != cudaSuccess) {
+    if (dev_alloc(d, h.size() * sizeof(T)) != cudaSuccess) {
         cudaGetLastError();
         return fesc_fail(ctx, FESC_ENOMEM, "table allocation failed");
     }
@@ -249,10 +372,10 @@ static int build_tables(fesc_ctx* ctx) {
     return upload(ctx, &ctx->tabs.d_rescale, rs);
 }
 static void free_tables(fesc_ctx* ctx) {
-    cudaFree(ctx->tabs.d_modup);
-    cudaFree(ctx->tabs.d_moddown);
-    cudaFree(ctx->tabs.d_rescale);
-    cudaFree(ctx->tabs.d_Pmod_all);
+    dev_free(ctx->tabs.d_modup);
+    dev_free(ctx->tabs.d_moddown);
+    dev_free(ctx->tabs.d_rescale);
+    dev_free(ctx->tabs.d_Pmod_all);
 }
 
 // Generate the switching key from s' (EVAL on all limbs, device) to s.
@@ -260,14 +383,14 @@ static int gen_key(fesc_ctx* ctx, uint32_t key_id, const u64* d_sp, u64 g) {
     const uint32_t N = ctx->N, np = ctx->n_primes;
     const size_t limb_words = (size_t)np * N;
     u64* d_key = nullptr;
-    if (cudaMalloc(&d_key, (size_t)ctx->beta_max * 2 * limb_words * sizeof(u64)) != cudaSuccess) {
+    if (dev_alloc(&d_key, (size_t)ctx->beta_max * 2 * limb_words * sizeof(u64)) != cudaSuccess) {
         cudaGetLastError();
         return fesc_fail(ctx, FESC_ENOMEM, "key allocation failed");
     }
     u64* d_e = nullptr;
-    if (cudaMalloc(&d_e, limb_words * sizeof(u64)) != cudaSuccess) {
+    if (dev_alloc(&d_e, limb_words * sizeof(u64)) != cudaSuccess) {
         cudaGetLastError();
-        cudaFree(d_key);
+        dev_free(d_key);
         return fesc_fail(ctx, FESC_ENOMEM, "key allocation failed");
     }
     dim3 grid((N + 255) / 256, np);
@@ -284,17 +407,17 @@ static int gen_key(fesc_ctx* ctx, uint32_t key_id, const u64* d_sp, u64 g) {
         k_make_b<<<grid, 256>>>(b, a, ctx->d_s, d_e, d_sp, ctx->d_pc, ctx->tabs.d_Pmod_all, N, lo, hi);
     }
     cudaError_t e = cudaDeviceSynchronize();
-    cudaFree(d_e);
+    dev_free(d_e);
     if (rc == FESC_OK && e != cudaSuccess) {
         ctx->err = std::string("key generation: ") + cudaGetErrorString(e);
         rc = FESC_ECUDA;
     }
     if (rc != FESC_OK) {
-        cudaFree(d_key);
+        dev_free(d_key);
         return rc;
     }
     auto it = ctx->keys.find(key_id);
-    if (it != ctx->keys.end()) cudaFree(it->second.d_key);
+    if (it != ctx->keys.end()) dev_free(it->second.d_key);
     ctx->keys[key_id] = EvalKey{g, d_key};
     return FESC_OK;
 }
@@ -384,16 +507,16 @@ extern "C" int fesc_ctx_create(fesc_ctx** out, uint32_t log_n, const uint64_t* p
     if ((rc = upload(ctx, &ctx->d_itwf, itwf)) != FESC_OK) return bail(rc);
     if ((rc = build_tables(ctx)) != FESC_OK) return bail(rc);
     // ---- secret key and relinearisation key ----
-    if (cudaMalloc(&ctx->d_s, (size_t)np * N * sizeof(u64)) != cudaSuccess) return bail(FESC_ENOMEM);
-    if (cudaMalloc(&ctx->d_status, sizeof(uint32_t)) != cudaSuccess) return bail(FESC_ENOMEM);
+    if (dev_alloc(&ctx->d_s, (size_t)np * N * sizeof(u64)) != cudaSuccess) return bail(FESC_ENOMEM);
+    if (dev_alloc(&ctx->d_status, sizeof(uint32_t)) != cudaSuccess) return bail(FESC_ENOMEM);
     if (cudaMemset(ctx->d_status, 0, sizeof(uint32_t)) != cudaSuccess) return bail(FESC_ECUDA);
     k_sample_small<<<(N + 255) / 256, 256>>>(ctx->d_s, ctx->d_pc, N, np, seed, make_tag(1, 0, 0, 0), 0);
     if ((rc = ntt_launch(ctx, ctx->d_s, np, all_limbs_map(ctx), false, 0)) != FESC_OK) return bail(rc);
     u64* d_s2 = nullptr;
-    if (cudaMalloc(&d_s2, (size_t)np * N * sizeof(u64)) != cudaSuccess) return bail(FESC_ENOMEM);
+    if (dev_alloc(&d_s2, (size_t)np * N * sizeof(u64)) != cudaSuccess) return bail(FESC_ENOMEM);
     k_square<<<dim3((N + 255) / 256, np), 256>>>(d_s2, ctx->d_s, ctx->d_pc, N);
     rc = gen_key(ctx, FESC_RELIN_KEY_ID, d_s2, 0);
-    cudaFree(d_s2);
+    dev_free(d_s2);
     if (rc != FESC_OK) return bail(rc);
     memset(ctx->counters, 0, sizeof(ctx->counters));
     *out = ctx;
@@ -403,16 +526,16 @@ extern "C" int fesc_ctx_create(fesc_ctx** out, uint32_t log_n, const uint64_t* p
 extern "C" int fesc_ctx_destroy(fesc_ctx* ctx) {
     if (!ctx) return FESC_OK;
     cudaDeviceSynchronize();
-    for (auto& kv : ctx->keys) cudaFree(kv.second.d_key);
+    for (auto& kv : ctx->keys) dev_free(kv.second.d_key);
     for (cudaEvent_t e : ctx->prof.ev) cudaEventDestroy(e);
-    cudaFree(ctx->d_pc);
-    cudaFree(ctx->d_tw);
-    cudaFree(ctx->d_itw);
-    cudaFree(ctx->d_twf);
-    cudaFree(ctx->d_itwf);
-    cudaFree(ctx->d_s);
-    cudaFree(ctx->d_scratch);
-    cudaFree(ctx->d_status);
+    dev_free(ctx->d_pc);
+    dev_free(ctx->d_tw);
+    dev_free(ctx->d_itw);
+    dev_free(ctx->d_twf);
+    dev_free(ctx->d_itwf);
+    dev_free(ctx->d_s);
+    dev_free(ctx->d_scratch);
+    dev_free(ctx->d_status);
     free_tables(ctx);
     delete ctx;
     return FESC_OK;
@@ -422,7 +545,7 @@ extern "C" int fesc_ctx_trim(fesc_ctx* ctx) {
     if (!ctx) return FESC_EINVAL;
     if (ctx->d_scratch) {
         FESC_CHECK_CUDA(ctx, cudaDeviceSynchronize());
-        cudaFree(ctx->d_scratch);
+        dev_free(ctx->d_scratch);
         ctx->d_scratch = nullptr;
         ctx->scratch_bytes = 0;
         ctx->counters[3] = 0;
@@ -501,6 +624,15 @@ extern "C" int fesc_sync(fesc_ctx* ctx, void* stream) {
         return fesc_fail(ctx, FESC_ETIMEOUT, "a device-side wait on an asynchronous copy gave up (code " +
                                                  std::to_string(status) + "); results of that call are invalid");
     }
+#ifdef FESC_DEBUG_BOUNDS
+    uint32_t hits = 0, site = 0;
+    uint64_t addr = 0, bytes = 0;
+    if (fesc_debug_bounds_report(&hits, &site, &addr, &bytes) != FESC_OK) return fesc_fail(ctx, FESC_ECUDA, "reading the bounds record failed");
+    if (hits)
+        return fesc_fail(ctx, FESC_EBOUNDS, std::to_string(hits) + " region(s) outside every known extent were skipped; first: file " +
+                                                std::to_string(site >> 16) + " line " + std::to_string(site & 0xffff) + ", address " +
+                                                std::to_string(addr) + ", " + std::to_string(bytes) + " bytes");
+#endif
     return FESC_OK;
 }
 
@@ -522,13 +654,13 @@ extern "C" int fesc_ctx_add_galois_key(fesc_ctx* ctx, int32_t rot, uint32_t key_
         }
     }
     u64* d_sp = nullptr;
-    if (cudaMalloc(&d_sp, (size_t)ctx->n_primes * ctx->N * sizeof(u64)) != cudaSuccess) {
+    if (dev_alloc(&d_sp, (size_t)ctx->n_primes * ctx->N * sizeof(u64)) != cudaSuccess) {
         cudaGetLastError();
         return fesc_fail(ctx, FESC_ENOMEM, "key allocation failed");
     }
     k_autom_rows<<<dim3((ctx->N + 255) / 256, ctx->n_primes), 256>>>(d_sp, ctx->d_s, ctx->log_n, g);
     int rc = gen_key(ctx, key_id, d_sp, g);
-    cudaFree(d_sp);
+    dev_free(d_sp);
     return rc;
 }
 

@@ -11,7 +11,26 @@
 #include <stdlib.h>
 #include <string.h>
 
+#define FESC_DBG_FILE 4   // file id in the sites a debug build reports
 #include "ops.cuh"
+
+// Debug build: the spans an accumulate CTA reads and writes (token blocks [tb0, tb0 + tt), (b,p) pairs [bp0, bp0 + pt),
+// all terms, both polynomials, every limb), the same for all its threads.
+__device__ __forceinline__ bool dbg_accumulate_spans(const u64* rot, const u64* diags, const u64* acc, uint32_t N, uint32_t level,
+                                                     uint32_t tbs, uint32_t terms, uint32_t bp_count, uint32_t tb0,
+                                                     uint32_t bp0, uint32_t tt, uint32_t pt) {
+#ifdef FESC_DEBUG_BOUNDS
+    const size_t poly = (size_t)level * N, ctw = 2 * poly;
+    for (uint32_t i = 0; i < tt && tb0 + i < tbs; i++) {
+        if (!DBG_REGION(rot + (size_t)(tb0 + i) * terms * ctw, terms * ctw * sizeof(u64))) return false;
+        for (uint32_t j = 0; j < pt && bp0 + j < bp_count; j++)
+            if (!DBG_REGION(acc + ((size_t)(tb0 + i) * bp_count + bp0 + j) * ctw, ctw * sizeof(u64))) return false;
+    }
+    for (uint32_t j = 0; j < pt && bp0 + j < bp_count; j++)
+        if (!DBG_REGION(diags + (size_t)(bp0 + j) * terms * poly, terms * poly * sizeof(u64))) return false;
+#endif
+    return true;
+}
 
 template <int TT, int PT>
 __global__ void __launch_bounds__(256, (TT * PT >= 16 ? 1 : (TT * PT >= 4 ? 2 : 3))) k_bsgs_accumulate(
@@ -26,6 +45,7 @@ __global__ void __launch_bounds__(256, (TT * PT >= 16 ? 1 : (TT * PT >= 4 ? 2 : 
     const uint32_t l = blockIdx.z % level;
     const uint32_t tb0 = (blockIdx.z / level) * TT, bp0 = blockIdx.x * PT;
     if (c >= N) return;
+    if (!dbg_accumulate_spans(rot, diags, acc, N, level, tbs, terms, bp_count, tb0, bp0, TT, PT)) return;
     const PrimeConst pc = pcs[l];
     const size_t poly = (size_t)level * N, ctw = 2 * poly;
     const size_t o = (size_t)l * N + c;
@@ -118,6 +138,7 @@ __global__ void __launch_bounds__(256, 2) k_bsgs_accumulate_fp(
     const uint32_t l = blockIdx.z % level;
     const uint32_t tb0 = (blockIdx.z / level) * TT, bp0 = blockIdx.x * PT;
     if (c >= N) return;
+    if (!dbg_accumulate_spans(rot, diags, acc, N, level, tbs, terms, bp_count, tb0, bp0, TT, PT)) return;
     const double q = pcs[l].qd, qinv = pcs[l].qinvd;
     const size_t poly = (size_t)level * N, ctw = 2 * poly;
     const size_t o = (size_t)l * N + c;
@@ -220,6 +241,7 @@ __global__ void __launch_bounds__(256, (TT * PT > 16 ? 1 : 2)) k_bsgs_accumulate
     const uint32_t c = blockIdx.y * 256 + tid;            // N is a multiple of 256
     const uint32_t l = blockIdx.z % level;
     const uint32_t tb0 = (blockIdx.z / level) * TT, bp0 = blockIdx.x * PT;
+    if (!dbg_accumulate_spans(rot, diags, acc, N, level, tbs, terms, bp_count, tb0, bp0, TT, PT)) return;   // before any barrier
     const double q = pcs[l].qd, qinv = pcs[l].qinvd;
     const size_t poly = (size_t)level * N, ctw = 2 * poly;
     const size_t o = (size_t)l * N + c;
@@ -323,6 +345,7 @@ __global__ void __launch_bounds__(MIX_THREADS, (TT * PT >= 12 ? 256 / MIX_THREAD
     const uint32_t tb_tiles = (tbs + TT - 1) / TT;
     const uint32_t l = blockIdx.z;
     const uint32_t tb0 = (blockIdx.x % tb_tiles) * TT, bp0 = (blockIdx.x / tb_tiles) * PT;
+    if (!dbg_accumulate_spans(rot, diags, acc, N, level, tbs, terms, bp_count, tb0, bp0, TT, PT)) return;   // before any barrier
     const PrimeConst pc = pcs[l];
     const size_t poly = (size_t)level * N, ctw = 2 * poly;
     const size_t o = (size_t)l * N + c;
@@ -450,6 +473,7 @@ __global__ void __launch_bounds__(32 * IM_CW, 1) k_bsgs_accumulate_imma(
     extern __shared__ __align__(16) u64 stage[];      // x: [8 (tb,p)][xs_pitch], then IM_STAGES x [8 (b,p)][IM_BPP]
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tg = lane & 3;
     const uint32_t c0 = blockIdx.x * IM_CW, l = blockIdx.y, tb0 = blockIdx.z * 4;
+    if (!dbg_accumulate_spans(rot, diags, acc, N, level, tbs, terms, bp_count, tb0, 0, 4, bp_count)) return;   // before any barrier
     const PrimeConst pc = pcs[l];
     const size_t poly = (size_t)level * N, ctw = 2 * poly;
     const uint32_t ksteps = (terms + 31) >> 5, bp_tiles = (bp_count + 7) >> 3, total = ksteps * bp_tiles;

@@ -6,6 +6,7 @@
 // allocator calls on its threads.  fesc_rescale sizes its scratch from the context arena, which
 // may grow on first use.  The entry point below does the same arithmetic with its scratch in a
 // fixed device array that is part of the library image, so it never allocates.
+#define FESC_DBG_FILE 9   // file id in the sites a debug build reports
 #include "ops.cuh"
 
 // Scratch of the rescale: the last limb of every polynomial of the batch (batch * 2 rows of N words),
@@ -39,6 +40,7 @@ extern "C" int fesc_rescale_static(fesc_ctx* ctx, const uint64_t* d_in, uint64_t
         void* p = nullptr;
         FESC_CHECK_CUDA(ctx, cudaGetSymbolAddress(&p, g_rescale_scratch));
         g_scratch_addr[dev] = (u64*)p;
+        dbg_note_alloc(p, sizeof(g_rescale_scratch));      // a debug build checks the kernels' regions against known extents
     }
     return rescale_internal(ctx, (const u64*)d_in, (size_t)2 * n_limbs * ctx->N, (u64*)d_out, batch, n_limbs,
                             g_scratch_addr[dev], (cudaStream_t)stream);

@@ -4,6 +4,7 @@
 //   y^ = gamma_RMS (.) (y~ (.) br(s_RMS))            (the input of HEOutProj)
 // br(s): the token factors sit in slots k < T of one ciphertext per token block; log2(n/T) rotate-right-and-add
 // steps by T*2^b copy them to every channel of the block.  Products are relinearised and rescaled.
+#define FESC_DBG_FILE 8   // file id in the sites a debug build reports
 #include "ops.cuh"
 
 // out[b] = ct[b] (.) pt[b] on both polynomials (pt_stride words between plaintexts)
@@ -16,6 +17,11 @@ __global__ void __launch_bounds__(256) k_ct_mul_pt(const u64* ct, size_t ct_stri
     if (c >= N) return;
     const PrimeConst pc = pcs[l];
     const size_t poly = (size_t)level * N, o = (size_t)l * N + c;
+    if (!DBG_REGION(pt + (size_t)b * pt_stride + o - c, N * sizeof(u64))) return;
+    for (int p = 0; p < 2; p++)
+        if (!DBG_REGION(ct + (size_t)b * ct_stride + p * poly + o - c, N * sizeof(u64)) ||
+            !DBG_REGION(out + (size_t)b * out_stride + p * poly + o - c, N * sizeof(u64)))
+            return;
     const u64 w = pt[(size_t)b * pt_stride + o];
     out[(size_t)b * out_stride + o] = mulmod(ct[(size_t)b * ct_stride + o], w, pc);
     out[(size_t)b * out_stride + poly + o] = mulmod(ct[(size_t)b * ct_stride + poly + o], w, pc);

@@ -13,6 +13,7 @@
 //   * "contiguous" kernel: stages with distance < 256.  One WARP owns one 256-point block, so
 //     the exchanges need only __syncwarp.
 // N <= 2^12 runs as one shared-memory kernel per row (tests and the tiny workload).
+#define FESC_DBG_FILE 2   // file id in the sites a debug build reports
 #include "common.cuh"
 
 // CTA shapes of the N = 2^16 kernels: columns per CTA of the strided kernel (x 32 sub-threads) and
@@ -452,6 +453,7 @@ __global__ void __launch_bounds__(NTT_COLS * 32) ntt16_strided(u64* __restrict__
     const PrimeConst pc = pcs[pi];
     const ulonglong2* tw = tw_all + (size_t)pi * N16;
     u64* p = data + (size_t)row * N16 + blockIdx.x * NTT_COLS;
+    if (!DBG_REGION(data + (size_t)row * N16, N16 * sizeof(u64))) return;   // the CTA's columns span the whole row
     if (pc.q < FP_LIMIT)
         strided_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, in_double);
     else if (pc.q < WIDE_LIMIT)
@@ -544,9 +546,14 @@ __global__ void __launch_bounds__(NTT_WARPS * 32) ntt16_contig(u64* __restrict__
     const uint32_t blk = blockIdx.x * NTT_WARPS + warp;   // 256-point block index within the limb
     u64* p = data + (size_t)row * N16 + (size_t)blk * 256;
     u64* sm = sm_all + warp * 288;
+    if (!DBG_REGION(p, 256 * sizeof(u64))) return;      // one warp per 256-point block, warp barriers only
     if (pc.q < FP_LIMIT) {
         if (!INV && fin.acc) {      // rows of this launch: r = bp * level + i
             const uint32_t r = row_first + row, bp = r / fin.level, i = r - bp * fin.level;
+            if (!DBG_REGION(fin.acc + ((size_t)bp * fin.acc_rows + i) * N16 + (size_t)blk * 256, 256 * sizeof(u64)) ||
+                !DBG_REGION(fin.out + (size_t)(bp >> 1) * fin.out_stride + ((size_t)(bp & 1) * fin.level + i) * N16 + (size_t)blk * 256,
+                            256 * sizeof(u64)))
+                return;
             contig_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, 256 + blk, out_double,
                                 fin.acc + ((size_t)bp * fin.acc_rows + i) * N16 + (size_t)blk * 256,
                                 fin.out + (size_t)(bp >> 1) * fin.out_stride + ((size_t)(bp & 1) * fin.level + i) * N16 + (size_t)blk * 256,
@@ -575,6 +582,7 @@ __global__ void __launch_bounds__(256) ntt_small(u64* __restrict__ data, const u
     const u64 q = pc.q, q2 = 2 * pc.q;
     const ulonglong2* tw = tw_all + (size_t)pi * N;
     u64* p = data + (size_t)row * N;
+    if (!DBG_REGION(p, N * sizeof(u64)) || !DBG_REGION(tw, N * sizeof(ulonglong2))) return;
     for (uint32_t i = threadIdx.x; i < N; i += blockDim.x) smx[i] = p[i];
     __syncthreads();
     if (!INV) {

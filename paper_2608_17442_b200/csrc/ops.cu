@@ -1,6 +1,7 @@
 // Ciphertext operations: ct-pt MAC, Galois automorphism, hybrid key switch, rotation,
 // rescale, ct x ct.  Every kernel streams limb rows of N words with coalesced accesses;
 // products of two data words are accumulated lazily in 128 bits and reduced once.
+#define FESC_DBG_FILE 3   // file id in the sites a debug build reports
 #include "ops.cuh"
 
 // ---------------------------------------------------------------------------------------
@@ -15,6 +16,9 @@ __global__ void __launch_bounds__(256) k_ct_pt_mac(const u64* __restrict__ ct, c
     const PrimeConst pc = pcs[l];
     const size_t poly = (size_t)n_limbs * N;
     const size_t o = (size_t)b * 2 * poly + (size_t)l * N + c;
+    if (!DBG_REGION(pt + (size_t)b * pt_stride + (size_t)l * N, N * sizeof(u64))) return;
+    for (int p = 0; p < 2; p++)
+        if (!DBG_REGION(ct + o - c + p * poly, N * sizeof(u64)) || !DBG_REGION(acc + o - c + p * poly, N * sizeof(u64))) return;
     const u64 w = pt[(size_t)b * pt_stride + (size_t)l * N + c];
 #pragma unroll
     for (int p = 0; p < 2; p++) {
@@ -101,6 +105,10 @@ __global__ void __launch_bounds__(256) k_autom_ct(const u64* __restrict__ in, si
     const u64* ib = in + (size_t)b * in_stride;
     const size_t poly = (size_t)level * N;
     u64* o0 = out0 + (size_t)b * out_stride + (size_t)l * N + t;
+    if (src >= N || !DBG_REGION(ib + (size_t)l * N, N * sizeof(u64)) || !DBG_REGION(ib + poly + (size_t)l * N, N * sizeof(u64)) ||
+        !DBG_REGION(o0 - t, N * sizeof(u64)) || !DBG_REGION(d.ext + own_index(d, b, l, N), N * sizeof(u64)) ||
+        !DBG_REGION(dcoef + ((size_t)b * level + l) * N, N * sizeof(u64)))
+        return;
     u64 v0 = ib[(size_t)l * N + src];
     if (accumulate) v0 = addmod(v0, *o0, pcs[l].q);
     *o0 = v0;
@@ -151,6 +159,9 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
     if (c >= N) return;
     const ModUpDigit* dg = tab + j;
     const uint32_t first = dg->first, n_src = dg->n_src;
+    if (!DBG_REGION(dg, sizeof(ModUpDigit)) || !DBG_REGION(dcoef + ((size_t)b * level + first) * N, (size_t)n_src * N * sizeof(u64)) ||
+        !DBG_REGION(ext + ((size_t)b * beta + j) * (level + K) * N, (size_t)(level + K) * N * sizeof(u64)))
+        return;
     u64 y[ALPHA][VEC];
     bool src_small = true;
 #pragma unroll
@@ -249,6 +260,21 @@ __global__ void __launch_bounds__(256, INNER_MINB) k_inner(const u64* __restrict
         const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
         xp[i] = ext + ((size_t)b * beta * rows + t) * N + cs;
     }
+#ifdef FESC_DEBUG_BOUNDS
+    if (cs >= N) return;
+    for (uint32_t j = 0; j < beta; j++) {
+        if (!DBG_REGION(kp - c + (size_t)(2 * j) * kstride, N * sizeof(u64)) || !DBG_REGION(kp - c + (size_t)(2 * j + 1) * kstride, N * sizeof(u64)))
+            return;
+        for (int i = 0; i < BT; i++)
+            if (!DBG_REGION(xp[i] - cs + (size_t)j * xstride, N * sizeof(u64))) return;
+    }
+    for (int i = 0; i < BT; i++) {
+        const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
+        if (!DBG_REGION(acc + (((size_t)b * 2 + 0) * rows + t) * N, N * sizeof(u64)) ||
+            !DBG_REGION(acc + (((size_t)b * 2 + 1) * rows + t) * N, N * sizeof(u64)))
+            return;
+    }
+#endif
     auto load_digit = [&](uint32_t j, u64& kb, u64& ka, u64 (&x)[BT]) {
         kb = __ldg(kp + (size_t)(2 * j) * kstride);
         ka = __ldg(kp + (size_t)(2 * j + 1) * kstride);
@@ -411,6 +437,17 @@ __global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ ex
         const uint32_t sblk = g ? (galois_src(cblk << 8, log_n, g) >> 8) : cblk;
         const uint32_t bar = bar0 + stage * 8;
         uint32_t dst = sbase + stage * stage_words * 8;
+#ifdef FESC_DEBUG_BOUNDS
+        for (uint32_t j = 0; j < beta; j++) {      // a bad source: no copy is issued, the wait below runs out and the CTA returns
+            if (!DBG_REGION(key + ((size_t)(2 * j) * np + pt) * N + (cblk << 8), 2048) ||
+                !DBG_REGION(key + ((size_t)(2 * j + 1) * np + pt) * N + (cblk << 8), 2048))
+                return;
+            for (int i = 0; i < BT; i++) {
+                const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
+                if (!DBG_REGION(ext + (((size_t)b * beta + j) * rows + t) * N + (sblk << 8), 2048)) return;
+            }
+        }
+#endif
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier reads of this half precede the refill
         mbar_expect_tx(bar, stage_words * 8);
         for (uint32_t j = 0; j < beta; j++) {
@@ -446,6 +483,20 @@ __global__ void __launch_bounds__(256, 1) k_inner_tma(const u64* __restrict__ ex
         uint32_t t, cblk, b0;
         decode(tile, t, cblk, b0);
         const uint32_t c = (cblk << 8) + tid;
+#ifdef FESC_DEBUG_BOUNDS
+        {
+            bool ok = true;                                  // the same for every thread of the CTA
+            for (int i = 0; i < BT; i++) {
+                const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
+                ok = ok && DBG_REGION(acc + (((size_t)b * 2 + 0) * rows + t) * N + (cblk << 8), 2048) &&
+                     DBG_REGION(acc + (((size_t)b * 2 + 1) * rows + t) * N + (cblk << 8), 2048);
+            }
+            if (!ok) {
+                __syncthreads();
+                continue;
+            }
+        }
+#endif
         const uint32_t si = g ? (galois_src(c, log_n, g) & 255u) : tid;
         const uint32_t pt = t < level ? t : n_q + (t - level);
         const u64* sm = smem + (size_t)stage * stage_words;
@@ -534,6 +585,9 @@ __global__ void __launch_bounds__(256) k_moddown_conv(const u64* __restrict__ ac
     const uint32_t bp = blockIdx.y;   // b*2 + p
     if (c >= N) return;
     const uint32_t rows = level + K;
+    if (!DBG_REGION(acc + ((size_t)bp * rows + level) * N, (size_t)K * N * sizeof(u64)) ||
+        !DBG_REGION(u + (size_t)bp * level * N, (size_t)level * N * sizeof(u64)) || !DBG_REGION(tab, sizeof(ModDownTab)))
+        return;
     u64 y[FESC_MAX_SPECIAL][VEC];
     uint32_t cnt[VEC];
 #pragma unroll
@@ -610,6 +664,9 @@ __global__ void __launch_bounds__(256) k_moddown_finish(const u64* __restrict__ 
     const uint32_t b = bp >> 1, p = bp & 1;
     const u64 q = pcs[i].q;
     u64* o = out + (size_t)b * out_stride + ((size_t)p * level + i) * N + c;
+    if (!DBG_REGION(o - c, N * sizeof(u64)) || !DBG_REGION(acc + ((size_t)bp * (level + K) + i) * N, N * sizeof(u64)) ||
+        !DBG_REGION(u + ((size_t)bp * level + i) * N, N * sizeof(u64)))
+        return;
     const u64 av = acc[((size_t)bp * (level + K) + i) * N + c], uv = u[((size_t)bp * level + i) * N + c];
     if (q < FESC_FP_LIMIT) {
         const double qd = pcs[i].qd, qinv = pcs[i].qinvd;
@@ -827,8 +884,14 @@ __global__ void __launch_bounds__(256) k_hoist_prepare(const u64* __restrict__ i
     if (t >= N) return;
     const u64* ib = in + (size_t)b * in_stride;
     if (g) {
+        if (galois_src(t, log_n, g) >= N || !DBG_REGION(ib + (size_t)l * N, N * sizeof(u64)) ||
+            !DBG_REGION(out0 + (size_t)b * out_stride + (size_t)l * N, N * sizeof(u64)))
+            return;
         out0[(size_t)b * out_stride + (size_t)l * N + t] = ib[(size_t)l * N + galois_src(t, log_n, g)];
     } else {
+        if (!DBG_REGION(ib + ((size_t)level + l) * N, N * sizeof(u64)) || !DBG_REGION(d.ext + own_index(d, b, l, N), N * sizeof(u64)) ||
+            !DBG_REGION(dcoef + ((size_t)b * level + l) * N, N * sizeof(u64)))
+            return;
         const u64 v = ib[((size_t)level + l) * N + t];
         d.ext[own_index(d, b, l, N) + t] = own_word(d, v, pcs[l]);
         dcoef[((size_t)b * level + l) * N + t] = v;
@@ -915,6 +978,9 @@ __global__ void __launch_bounds__(256) k_rotsum_prepare(const u64* __restrict__ 
     const u64* ib = in + (size_t)b * in_stride;
     u64* ob = out + (size_t)b * out_stride;
     const u64 q = pcs[l].q;
+    for (int p = 0; p < 2; p++)
+        if (!DBG_REGION(ib + ((size_t)p * level + l) * N, N * sizeof(u64)) || !DBG_REGION(ob + ((size_t)p * level + l) * N, N * sizeof(u64)))
+            return;
     u64 v = ib[(size_t)l * N + t];
     for (uint32_t k = 0; k < gs.n; k++) v = addmod(v, ib[(size_t)l * N + galois_src(t, log_n, gs.g[k])], q);
     ob[(size_t)l * N + t] = v;
@@ -1002,6 +1068,9 @@ __global__ void __launch_bounds__(256) k_take_last(const u64* __restrict__ in, s
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t bp = blockIdx.y;
     if (c >= N) return;
+    if (!DBG_REGION(r + (size_t)bp * N, N * sizeof(u64)) ||
+        !DBG_REGION(in + (size_t)(bp >> 1) * in_stride + ((size_t)(bp & 1) * level + level - 1) * N, N * sizeof(u64)))
+        return;
     r[(size_t)bp * N + c] = in[(size_t)(bp >> 1) * in_stride + ((size_t)(bp & 1) * level + level - 1) * N + c];
 }
 // out[b][p][i] = centred(r) mod q_i  (COEFF)
@@ -1011,6 +1080,9 @@ __global__ void __launch_bounds__(256) k_rescale_conv(const u64* __restrict__ r,
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t i = blockIdx.y, bp = blockIdx.z;
     if (c >= N) return;
+    if (!DBG_REGION(r + (size_t)bp * N, N * sizeof(u64)) || !DBG_REGION(tab, sizeof(RescaleTab)) ||
+        !DBG_REGION(out + (size_t)(bp >> 1) * out_stride + ((size_t)(bp & 1) * (level - 1) + i) * N, N * sizeof(u64)))
+        return;
     const u64 v = r[(size_t)bp * N + c];
     const PrimeConst pc = pcs[i];
     u64 w = v - mulhi(v, pc.mu) * pc.q;   // v mod q_i in [0, 2q)
@@ -1028,6 +1100,9 @@ __global__ void __launch_bounds__(256) k_rescale_finish(const u64* __restrict__ 
     if (c >= N) return;
     const u64 q = pcs[i].q;
     u64* o = out + (size_t)(bp >> 1) * out_stride + ((size_t)(bp & 1) * (level - 1) + i) * N + c;
+    if (!DBG_REGION(o - c, N * sizeof(u64)) || !DBG_REGION(tab, sizeof(RescaleTab)) ||
+        !DBG_REGION(in + (size_t)(bp >> 1) * in_stride + ((size_t)(bp & 1) * level + i) * N, N * sizeof(u64)))
+        return;
     u64 x = in[(size_t)(bp >> 1) * in_stride + ((size_t)(bp & 1) * level + i) * N + c];
     *o = shoup(submod(x, *o, q), tab->qinv[i], tab->qinvs[i], q);
 }
@@ -1090,6 +1165,11 @@ __global__ void __launch_bounds__(256) k_tensor(const u64* __restrict__ a, size_
     if (c >= N) return;
     const PrimeConst pc = pcs[l];
     const size_t poly = (size_t)level * N, o = (size_t)l * N + c;
+    for (int p = 0; p < 2; p++)
+        if (!DBG_REGION(a + b * a_stride + p * poly + o - c, N * sizeof(u64)) || !DBG_REGION(bb + b * b_stride + p * poly + o - c, N * sizeof(u64)) ||
+            !DBG_REGION(out + b * out_stride + p * poly + o - c, N * sizeof(u64)))
+            return;
+    if (!DBG_REGION(d.ext + own_index(d, b, l, N), N * sizeof(u64)) || !DBG_REGION(dcoef + ((size_t)b * level + l) * N, N * sizeof(u64))) return;
     const u64 a0 = a[b * a_stride + o], a1 = a[b * a_stride + poly + o];
     const u64 b0 = bb[b * b_stride + o], b1 = bb[b * b_stride + poly + o];
     out[b * out_stride + o] = mulmod(a0, b0, pc);

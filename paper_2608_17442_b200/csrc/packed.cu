@@ -22,6 +22,7 @@
 //                  ((token block, polynomial) g of the tile), b0 = terms 4tg..4tg+3, b1 = terms 16+4tg..16+4tg+3.
 // Images are ordered [row tile][limb][coefficient tile of 8][k-step][coefficient 8], so the 8 x ksteps images one
 // CTA needs for one (b,p) tile are contiguous.  Rows and terms beyond the valid ones are zero.
+#define FESC_DBG_FILE 5   // file id in the sites a debug build reports
 #include "ops.cuh"
 
 #define PK_CW 8
@@ -46,6 +47,19 @@ __global__ void __launch_bounds__(256) k_pack_fragments(const u64* __restrict__ 
     const uint32_t tid = threadIdx.x, cw = tid & 7, rw = tid >> 3;
     const uint32_t ct = blockIdx.x, l = blockIdx.y, tile = blockIdx.z / ksteps, ks = blockIdx.z - tile * ksteps;
     const uint32_t t = (ks << 5) + rw;
+#ifdef FESC_DEBUG_BOUNDS
+    {   // the same outcome for every thread of the CTA (there is a barrier below): all 8 rows x 32 terms, one limb row each
+        bool ok = DBG_REGION(dst + ((((size_t)tile * level + l) * gridDim.x + ct) * ksteps + ks) * PK_STAGE, PK_STAGE);
+        for (uint32_t g = 0; g < 8 && ok; g++)
+            for (uint32_t tt = ks << 5; tt < (ks << 5) + 32 && tt < terms && ok; tt++) {
+                const uint32_t r = tile * 8 + g;
+                if (r >= rows) break;
+                const size_t off = A_SIDE ? (size_t)r * stride_hi : (size_t)(r >> 1) * stride_hi + (size_t)(r & 1) * stride_lo;
+                ok = DBG_REGION(src + off + (size_t)tt * term_stride + (size_t)l * N + ct * PK_CW, PK_CW * sizeof(u64));
+            }
+        if (!ok) return;
+    }
+#endif
 #pragma unroll
     for (uint32_t g = 0; g < 8; g++) {
         const uint32_t r = tile * 8 + g;
@@ -121,6 +135,22 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
     const uint8_t* src = dpk + ((size_t)l * tiles_d + (run >> 3)) * ksteps * PK_STAGE + (run & 7) * PK_FRAG;
     const size_t tile_stride = (size_t)level * tiles_d * ksteps * PK_STAGE;
     const uint8_t* ximg = xpk + ((((size_t)tbt * level + l) * tiles + ct) * ksteps * PK_CW + coef) * PK_FRAG;
+#ifdef FESC_DEBUG_BOUNDS
+    {   // the same outcome for every thread of the CTA (barriers follow): the streams of all four warps and the output rows
+        bool ok = true;
+        for (uint32_t w = 0; w < PK_WARPS && ok; w++) {
+            const uint32_t cf = (half_tile & 1) * PK_WARPS + w, rn = (ct * PK_CW + cf) >> dshift;
+            const uint8_t* sw = dpk + ((size_t)l * tiles_d + (rn >> 3)) * ksteps * PK_STAGE + (rn & 7) * PK_FRAG;
+            for (uint32_t bt = 0; bt < bp_tiles && ok; bt++)
+                ok = DBG_REGION(sw + bt * tile_stride, (size_t)(ksteps - 1) * PK_STAGE + PK_FRAG);
+            ok = ok && DBG_REGION(xpk + ((((size_t)tbt * level + l) * tiles + ct) * ksteps * PK_CW + cf) * PK_FRAG,
+                                  (size_t)(ksteps - 1) * PK_STAGE + PK_FRAG);
+        }
+        for (uint32_t tb = tbt * 4; tb < tbt * 4 + 4 && tb < tbs && ok; tb++)
+            ok = DBG_REGION(acc + (size_t)tb * bp_count * 2 * level * N, (size_t)bp_count * 2 * level * N * sizeof(u64));
+        if (!ok) return;
+    }
+#endif
     uint32_t ld_ks = 0, ld_s = 0;                         // next stage to request (lane 0)
     auto request = [&](uint32_t slot) {
         mbar_expect_tx(my_bar + slot * 8, PK_FRAG);

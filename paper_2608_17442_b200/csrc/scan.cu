@@ -12,6 +12,7 @@
 
 #include <map>
 
+#define FESC_DBG_FILE 6   // file id in the sites a debug build reports
 #include "ops.cuh"
 
 // ---------------------------------------------------------------------------------------
@@ -27,6 +28,9 @@ __global__ void __launch_bounds__(256) k_ct_addsub(const u64* __restrict__ a, si
     if (c >= N) return;
     const u64 q = pcs[pl % level].q;
     const size_t o = (size_t)pl * N + c;
+    if (!DBG_REGION(a + bi * a_stride + o - c, N * sizeof(u64)) || !DBG_REGION(b + bi * b_stride + o - c, N * sizeof(u64)) ||
+        !DBG_REGION(out + bi * out_stride + o - c, N * sizeof(u64)))
+        return;
     const u64 x = a[bi * a_stride + o], y = b[bi * b_stride + o];
     out[bi * out_stride + o] = sub ? submod(x, y, q) : addmod(x, y, q);
 }
@@ -39,6 +43,10 @@ __global__ void __launch_bounds__(256) k_ct_ptmul(const u64* __restrict__ a, siz
     if (c >= N) return;
     const PrimeConst pc = pcs[l];
     const size_t o = (size_t)l * N + c, poly = (size_t)level * N;
+    if (!DBG_REGION(pt + bi * pt_stride + o - c, N * sizeof(u64))) return;
+    for (int p = 0; p < 2; p++)
+        if (!DBG_REGION(a + bi * a_stride + p * poly + o - c, N * sizeof(u64)) || !DBG_REGION(out + bi * out_stride + p * poly + o - c, N * sizeof(u64)))
+            return;
     const u64 w = pt[bi * pt_stride + o];
     out[bi * out_stride + o] = mulmod(a[bi * a_stride + o], w, pc);
     out[bi * out_stride + poly + o] = mulmod(a[bi * a_stride + poly + o], w, pc);
@@ -52,6 +60,9 @@ __global__ void __launch_bounds__(256) k_ct_scale_drop(const u64* __restrict__ a
     if (c >= N) return;
     const PrimeConst pc = pcs[l];
     const u64 kk = k - mulhi(k, pc.mu) * pc.q;   // k mod q in [0, 2q)
+    if (!DBG_REGION(out + bi * out_stride + ((size_t)p * keep + l) * N, N * sizeof(u64)) ||
+        !DBG_REGION(a + bi * a_stride + ((size_t)p * src + l) * N, N * sizeof(u64)))
+        return;
     out[bi * out_stride + ((size_t)p * keep + l) * N + c] =
         mulmod(a[bi * a_stride + ((size_t)p * src + l) * N + c], csub(kk, pc.q), pc);
 }
@@ -66,8 +77,11 @@ __global__ void __launch_bounds__(256) k_ct_mul_i(const u64* __restrict__ a, siz
     if (c >= N) return;
     const uint32_t l = pl % level;
     const u64 q = pcs[l].q;
-    const ulonglong2 I = tw[(size_t)l * N + 1];
     const size_t o = (size_t)pl * N + c;
+    if (!DBG_REGION(tw + (size_t)l * N, N * sizeof(ulonglong2)) || !DBG_REGION(a + bi * a_stride + o - c, N * sizeof(u64)) ||
+        !DBG_REGION(out + bi * out_stride + o - c, N * sizeof(u64)))
+        return;
+    const ulonglong2 I = tw[(size_t)l * N + 1];
     u64 v = shoup(a[bi * a_stride + o], I.x, I.y, q);
     const bool neg = (c >= N / 2) != (times == 3);
     out[bi * out_stride + o] = (neg && v) ? q - v : v;
@@ -81,6 +95,9 @@ __global__ void __launch_bounds__(256) k_ct_sum_into(const u64* __restrict__ a, 
     if (c >= N) return;
     const u64 q = pcs[pl % level].q;
     const size_t o = (size_t)pl * N + c;
+    if (!DBG_REGION(acc + o - c, N * sizeof(u64))) return;
+    for (uint32_t i = 0; i < count; i++)
+        if (!DBG_REGION(a + i * a_stride + o - c, N * sizeof(u64))) return;
     u64 s = acc[o];
     for (uint32_t i = 0; i < count; i++) s = addmod(s, a[i * a_stride + o], q);
     acc[o] = s;
@@ -101,6 +118,12 @@ __global__ void __launch_bounds__(256) k_class_mac(ClassSources s, uint32_t term
     const PrimeConst pc = pcs[l];
     const size_t poly = (size_t)level * N, o = (size_t)l * N + c;
     acc128 a0{0, 0}, a1{0, 0};
+    for (int p = 0; p < 2; p++)
+        if (!DBG_REGION(out + (size_t)b * out_stride + p * poly + o - c, N * sizeof(u64))) return;
+    for (uint32_t j = 0; j < terms; j++)
+        if (!DBG_REGION(masks + (size_t)j * poly + o - c, N * sizeof(u64)) || !DBG_REGION(s.src[j] + (size_t)b * src_stride + o - c, N * sizeof(u64)) ||
+            !DBG_REGION(s.src[j] + (size_t)b * src_stride + poly + o - c, N * sizeof(u64)))
+            return;
     for (uint32_t j = 0; j < terms; j++) {
         const u64 w = masks[(size_t)j * poly + o];
         const u64* x = s.src[j] + (size_t)b * src_stride;
