@@ -205,7 +205,7 @@ MAC_MIXED_CYCLES = 8              # mixed-pipe multiply-accumulate: multiplier-p
 # DRAM traffic of one accumulate launch is not captured at full size: a small-case capture of the same kernel
 # (a few GB, inputs larger than L2) gives measured DRAM bytes / algorithmic bytes, and because every operand byte is
 # read once per launch and every output byte written once, traffic grows in proportion to the algorithmic bytes.
-BSGS_TRAFFIC_RATIO = {"packed": 1.010, "residues": 1.001}     # measured DRAM bytes / algorithmic bytes (small case)
+BSGS_TRAFFIC_RATIO = {"packed": 1.000, "residues": 1.001}     # measured DRAM bytes / algorithmic bytes (small case)
 PACKED_BYTES_PER_WORD = 7                                     # a residue below 2^56 as byte planes
 NTT_TRAFFIC_RATIO = 1.0           # the transforms read and write every word of both passes through DRAM once
 INT_LIMB_SHARE = 32.0 / 224.0     # transforms on the 60-bit special primes per key switch (integer path)

@@ -595,13 +595,13 @@ static int bsgs_kernel() {
     return v;
 }
 // Larger groups re-read the diagonals less often and give the key-switch kernels larger batches; every token block
-// of a group needs its rotated inputs and its partial sums resident.  Budget: 24 GiB of scratch for them (28 GiB with packed operands; a fixed
-// figure, so the launch shape does not depend on what else holds memory); if the device cannot provide the scratch,
+// of a group needs its rotated inputs and its partial sums resident.  Budget: 24 GiB of scratch for them (32 GiB with packed operands, whose packed inputs
+// and key-switch chunk count as well; 44 GiB allows groups of 8; a fixed figure, so the launch shape does not depend on what else holds memory); if the device cannot provide the scratch,
 // the group is halved until it fits.
 static size_t bsgs_group_bytes(bool packed) {
     const char* e = getenv("FESC_BSGS_GROUP_GIB");
     if (e && atoi(e) > 0) return (size_t)atoi(e) << 30;
-    return (size_t)(packed ? 32 : 24) << 30;      // the packed inputs and the key-switch chunk of a group count as well (44 GiB allows groups of 8)
+    return (size_t)(packed ? 32 : 24) << 30;
 }
 
 // Projection on packed diagonals.  Token blocks are processed in groups of up to 8 = two tiles of 4: the baby rotations
@@ -726,34 +726,27 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
         }
         return linear_packed(ctx, (const u64*)d_ct_in, (const uint8_t*)d_diags, desc, (u64*)d_ct_out, st, bits);
     }
-    // token blocks per group, from the scratch budget (groups of packed inputs are whole tiles of 4 token blocks)
-    const size_t xpk_tb = packed ? bsgs_packed_bytes(N, level, 8, gin * n1) / 4 : 0;
-    const size_t per_tb = ((size_t)gin * n1 + (size_t)nout * n2) * ctw * sizeof(u64) + xpk_tb;
-    uint32_t tbg = (uint32_t)(bsgs_group_bytes(packed) / per_tb);
+    // residue diagonals from here on; token blocks per group, from the scratch budget
+    const size_t per_tb = ((size_t)gin * n1 + (size_t)nout * n2) * ctw * sizeof(u64);
+    uint32_t tbg = (uint32_t)(bsgs_group_bytes(false) / per_tb);
     if (tbg < 1) tbg = 1;
-    if (packed && tbg > 4) tbg -= tbg % 4;
     if (tbg > tbs) tbg = tbs;
     u64 *scratch = nullptr, *rot = nullptr, *acc = nullptr, *ks = nullptr;
-    uint8_t* xpk = nullptr;
     int rc;
     for (;;) {
         const uint32_t max_batch = tbg * (gin > nout ? gin : nout);
         const size_t ks_words = ks_scratch_words(ctx, level, ks_chunk(ctx, max_batch));
         const size_t rs_words = (size_t)(tbg * nout < 16384 ? tbg * nout : 16384) * 2 * N;
         const size_t rot_words = (size_t)tbg * gin * n1 * ctw, acc_words = (size_t)tbg * nout * n2 * ctw;
-        const size_t xpk_words = packed ? bsgs_packed_bytes(N, level, 2 * tbg, gin * n1) / 8 : 0;
-        rc = ctx_scratch(ctx, (rot_words + acc_words + xpk_words + (ks_words > rs_words ? ks_words : rs_words)) * sizeof(u64),
-                         &scratch);
+        rc = ctx_scratch(ctx, (rot_words + acc_words + (ks_words > rs_words ? ks_words : rs_words)) * sizeof(u64), &scratch);
         if (rc == FESC_OK) {
             rot = scratch;
             acc = rot + rot_words;
-            xpk = (uint8_t*)(acc + acc_words);
-            ks = acc + acc_words + xpk_words;
+            ks = acc + acc_words;
             break;
         }
         if (rc != FESC_ENOMEM || tbg == 1) return rc;
         tbg = (tbg + 1) / 2;
-        if (packed && tbg > 4) tbg -= tbg % 4;
     }
     ctx->counters[5] = tbg;
     // lazy 128-bit sums: reduce before terms * q^2 could reach 2^128
@@ -786,7 +779,7 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
             }
         }
         const uint32_t bp_count = nout * n2;
-        if (!packed) prof_begin(ctx, PF_BSGS, st);
+        prof_begin(ctx, PF_BSGS, st);
 #define BSGS(TT, PT)                                                                                          \
     do {                                                                                                      \
         dim3 grid((bp_count + PT - 1) / PT, (N + 255) / 256, level * ((nt + TT - 1) / TT));                   \
@@ -834,8 +827,7 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
         const bool fp_ok = qbits <= 50 && bsgs_kernel() != 2;
         const bool imma_ok = bsgs_kernel() == 0 && qbits <= 56 && N % IM_CW == 0 && gin * n1 <= 256 && level <= 65535;
         const bool deep = gin * n1 <= 128;       // room for 8 stages beside the rotated inputs
-        if (packed) {
-        } else if (imma_ok && qbits <= 50 && deep) BSGS_IMMA(true, 8);
+        if (imma_ok && qbits <= 50 && deep) BSGS_IMMA(true, 8);
         else if (imma_ok && qbits <= 50) BSGS_IMMA(true, 4);
         else if (imma_ok && deep) BSGS_IMMA(false, 8);
         else if (imma_ok) BSGS_IMMA(false, 4);
@@ -846,7 +838,7 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
         else if (nt >= 2) BSGS(2, 8);
         else BSGS(1, 8);
 #undef BSGS
-        if (!packed) prof_end(ctx, PF_BSGS, st);
+        prof_end(ctx, PF_BSGS, st);
         FESC_CHECK_CUDA(ctx, cudaGetLastError());
         ctx->counters[2] += (uint64_t)nt * bp_count * gin * n1;
         if (desc->defer) {

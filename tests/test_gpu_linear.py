@@ -335,3 +335,33 @@ def test_linear_token_major_packing_with_periodic_diagonals():
     with pytest.raises(fesc.FescError) as e:
         ctx.linear(to_dev(cts), to_dev(diags), fesc.BsgsDesc(nb, ng, gin, nout, tbs, level, kb, kb + 500, 1, 1, 0, shift), out)
     assert e.value.code == fesc.EINVAL
+
+
+@pytest.mark.parametrize("packed", [0, 1])
+def test_linear_falls_back_to_smaller_groups_when_scratch_cannot_be_had(packed):
+    """The projection sizes its token-block group from a scratch budget; when the arena cannot be reserved (failure
+    injected on the host, no driver call) it halves the group and tries again.  Same residues, smaller group; a failure
+    on every attempt comes back as FESC_ENOMEM and the context computes correctly afterwards."""
+    import paper_2608_17442_b200 as fesc
+
+    T, C, n1, n2, tokens, d_in, d_out, level = 32, 16, 4, 4, 8 * 32, 16, 32, 4       # 8 token blocks
+    pair = ctx_pair("small")
+    ctx, orc, _ = pair
+    kb = 1000 + 37 * T
+    X, W, cts, diags, dims = _setup(pair, T, C, n1, n2, tokens, d_in, d_out, level, 2.0**40, wscale=10.0, key_base=kb)
+    want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)}, {g: kb + 500 + g for g in range(1, n2)})
+    ctx.trim()
+    assert np.array_equal(_run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=kb, packed=packed), want)
+    full_group = ctx.counters()[5]
+    assert full_group == 8
+    ctx.trim()
+    ctx.test_fail_allocs(1)                    # the first reservation fails: one halving
+    assert np.array_equal(_run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=kb, packed=packed), want)
+    assert ctx.counters()[5] == 4
+    ctx.trim()
+    ctx.test_fail_allocs(16)                   # every attempt fails, down to a group of one
+    with pytest.raises(fesc.FescError) as e:
+        _run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=kb, packed=packed)
+    assert e.value.code == fesc.ENOMEM
+    ctx.test_fail_allocs(0)
+    assert np.array_equal(_run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=kb, packed=packed), want)

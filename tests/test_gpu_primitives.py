@@ -512,7 +512,6 @@ def test_allocation_failure_is_reported_and_the_context_stays_usable():
     got = to_host(out)
     for b in range(batch):
         assert np.array_equal(got[b], orc.rotate(ct[b], 81))
-    # fesc_linear halves its token-block group when the arena cannot be had and still returns the same residues
     assert ctx.info().flags == 0 and ctx.info().digits == ctx.num_digits
 
 
