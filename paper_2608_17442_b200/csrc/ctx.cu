@@ -39,7 +39,6 @@ __device__ bool fesc_dbg_region(const void* p, size_t bytes, uint32_t site) {
 #define FESC_DBG_CALLERS 192
 struct DbgHost {
     std::vector<std::pair<unsigned long long, unsigned long long>> own, caller;
-    size_t next = 0;
 };
 static DbgHost& dbg_host() {
     static DbgHost h;
@@ -81,21 +80,26 @@ extern "C" int fesc_debug_bounds_register(const void* d_ptr, size_t bytes) {
     if (!d_ptr || !bytes) return FESC_EINVAL;
     DbgHost& h = dbg_host();
     const unsigned long long lo = (unsigned long long)d_ptr, hi = lo + bytes;
-    for (auto& r : h.caller)
-        if (r.first == lo) {          // the same base address again: the newest extent counts
-            if (r.second == hi) return FESC_OK;
-            r.second = hi;
-            dbg_upload();
-            return FESC_OK;
+    // kept in order of last registration: a buffer registered again moves to the back (with its new extent), and the
+    // front, the one registered longest ago, is dropped when the list is full: never a buffer of the call being set up
+    bool same = false;
+    for (size_t i = 0; i < h.caller.size(); i++)
+        if (h.caller[i].first == lo) {
+            same = h.caller[i].second == hi;
+            h.caller.erase(h.caller.begin() + i);
+            break;
         }
-    if (h.caller.size() < FESC_DBG_CALLERS) h.caller.push_back({lo, hi});
-    else h.caller[h.next++ % FESC_DBG_CALLERS] = {lo, hi};
-    dbg_upload();
+    bool dropped = false;
+    if (h.caller.size() >= FESC_DBG_CALLERS) {
+        h.caller.erase(h.caller.begin());
+        dropped = true;
+    }
+    h.caller.push_back({lo, hi});
+    if (!same || dropped) dbg_upload();
     return FESC_OK;
 }
 extern "C" int fesc_debug_bounds_clear(void) {
     dbg_host().caller.clear();
-    dbg_host().next = 0;
     dbg_upload();
     return FESC_OK;
 }
