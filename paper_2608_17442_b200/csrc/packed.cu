@@ -106,18 +106,18 @@ int bsgs_pack_inputs(fesc_ctx* ctx, const u64* rot, uint8_t* xpk, uint32_t level
 // chain of integer and FP64 operations) the other two keep the tensor pipe busy.  Every warp streams the diagonal
 // images of ITS coefficient (1792 bytes per k-step, one bulk asynchronous copy each) through a private ring of
 // PK_STAGES slots, each slot with its own barrier: the warp that consumed a slot requests the copy that refills it,
-// so warps never wait for one another.  The input fragments of the coefficient (at most 3 k-steps) are copied once
+// so warps never wait for one another.  The input fragments of the coefficient (at most 6 k-steps, ring and inputs together at most 10 slots) are copied once
 // into shared memory the same way.  Every barrier wait is bounded; a wait that runs out sets the status word (3), the
 // warp waits (bounded) for its other copies in flight and leaves.
 #define PK_WARPS 4
-template <bool FP, int KSR>
+template <bool FP, int KSR, int ST>
 __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
     const uint8_t* __restrict__ xpk, const uint8_t* __restrict__ dpk, u64* __restrict__ acc,
     const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level, uint32_t tbs, uint32_t ksteps, uint32_t bp_count,
     uint32_t dshift, uint32_t* __restrict__ status) {
-    // per warp: PK_STAGES ring slots, KSR input images; then per warp PK_STAGES + 1 barriers
+    // per warp: ST ring slots, KSR input images; then per warp ST + 1 barriers
     extern __shared__ __align__(128) uint8_t ring[];
-    constexpr uint32_t WARP_BYTES = (PK_STAGES + KSR) * PK_FRAG;
+    constexpr uint32_t WARP_BYTES = (ST + KSR) * PK_FRAG;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tg = lane & 3;
     // blockIdx.x = (coefficient half-tile) * token-block tiles + token-block tile: the CTAs that stream the same images
     // for different token blocks start together, so only the first of them reads the images from HBM
@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
     const uint32_t tiles = gridDim.x / (2 * tbts);
     const uint32_t bp_tiles = (bp_count + 7) >> 3, total = bp_tiles * ksteps;
     const uint32_t my_ring = (uint32_t)__cvta_generic_to_shared(ring) + warp * WARP_BYTES;
-    const uint32_t my_bar = (uint32_t)__cvta_generic_to_shared(ring) + PK_WARPS * WARP_BYTES + warp * ((PK_STAGES + 1) * 8);
+    const uint32_t my_bar = (uint32_t)__cvta_generic_to_shared(ring) + PK_WARPS * WARP_BYTES + warp * ((ST + 1) * 8);
     const uint8_t* my_img = ring + warp * WARP_BYTES;
     // images of this warp's coefficient: k-steps of one (b,p) tile are PK_STAGE apart, tiles tile_stride apart.  Periodic
     // diagonals (dshift > 0) hold one image per aligned run of 2^dshift coefficients: the image of a ring 2^dshift times
@@ -159,14 +159,14 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
         ld_s++;
     };
     if (lane == 0) {
-        for (uint32_t i = 0; i <= PK_STAGES; i++) mbar_init(my_bar + i * 8, 1);
+        for (uint32_t i = 0; i <= ST; i++) mbar_init(my_bar + i * 8, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         if (KSR > 0) {
-            mbar_expect_tx(my_bar + PK_STAGES * 8, KSR * PK_FRAG);
+            mbar_expect_tx(my_bar + ST * 8, KSR * PK_FRAG);
             for (uint32_t k = 0; k < KSR; k++)
-                bulk_g2s(my_ring + (PK_STAGES + k) * PK_FRAG, ximg + (size_t)k * PK_STAGE, PK_FRAG, my_bar + PK_STAGES * 8);
+                bulk_g2s(my_ring + (ST + k) * PK_FRAG, ximg + (size_t)k * PK_STAGE, PK_FRAG, my_bar + ST * 8);
         }
-        for (uint32_t i = 0; i < PK_STAGES && i < total; i++) request(i);
+        for (uint32_t i = 0; i < ST && i < total; i++) request(i);
     }
     __syncwarp();
     const PrimeConst pc = pcs[l];
@@ -177,7 +177,7 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
         c64 = fp_modmul(c32, c32, pc.qd, pc.qinvd);
         c96 = fp_modmul(c64, c32, pc.qd, pc.qinvd);
     }
-    const uint32_t out_bar = (uint32_t)__cvta_generic_to_shared(ring) + PK_WARPS * (WARP_BYTES + (PK_STAGES + 1) * 8) + 2 * 256 * 8;
+    const uint32_t out_bar = (uint32_t)__cvta_generic_to_shared(ring) + PK_WARPS * (WARP_BYTES + (ST + 1) * 8) + 2 * 256 * 8;
     if (tid == 0) {
         mbar_init(out_bar, PK_WARPS);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -187,7 +187,7 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
     int z0 = 0, z1 = 0, z2 = 0, z3 = 0;                   // a fixed quad of zero addends (see imma_u8_zero)
     asm volatile("" : "+r"(z0), "+r"(z1), "+r"(z2), "+r"(z3));
     uint32_t slot = 0, phase = 0, s = 0;
-    bool ok = KSR == 0 || !mbar_wait_bounded(my_bar + PK_STAGES * 8, 0);
+    bool ok = KSR == 0 || !mbar_wait_bounded(my_bar + ST * 8, 0);
     const bool x_ok = ok;
     auto mma_stage = [&](const uint8_t* xfrag, bool first) {
         if (mbar_wait_bounded(my_bar + slot * 8, phase)) {
@@ -223,14 +223,14 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
         __syncwarp();
         if (lane == 0 && ld_s < total) request(slot);
         s++;
-        if (++slot == PK_STAGES) slot = 0, phase ^= 1;
+        if (++slot == ST) slot = 0, phase ^= 1;
     };
 #pragma unroll 1
     for (uint32_t bt = 0; bt < bp_tiles && ok; bt++) {
         if (KSR > 0) {
 #pragma unroll
             for (int k = 0; k < (KSR > 0 ? KSR : 1); k++)
-                if (ok) mma_stage(my_img + (PK_STAGES + k) * PK_FRAG, k == 0);
+                if (ok) mma_stage(my_img + (ST + k) * PK_FRAG, k == 0);
         } else {
 #pragma unroll 1
             for (uint32_t k = 0; k < ksteps && ok; k++) mma_stage(ximg + (size_t)k * PK_STAGE, k == 0);
@@ -239,7 +239,7 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
         // lane (g, tg) holds output bp = 8 bt + g of token block 4 tbt + tg, both polynomials.  The four warps of the
         // CTA (four neighbouring coefficients) exchange their results through shared memory so that every output row
         // receives one full 32-byte sector instead of four separate words.
-        u64* stage_out = (u64*)(ring + PK_WARPS * (WARP_BYTES + (PK_STAGES + 1) * 8)) + (bt & 1) * 256;
+        u64* stage_out = (u64*)(ring + PK_WARPS * (WARP_BYTES + (ST + 1) * 8)) + (bt & 1) * 256;
         stage_out[(lane * 2) * PK_WARPS + warp] = imma_recombine<FP>(d, 0, pc, c32, c64, c96);
         stage_out[(lane * 2 + 1) * PK_WARPS + warp] = imma_recombine<FP>(d, 1, pc, c32, c64, c96);
         // CTA-wide hand-over on a shared-memory barrier (one arrival per warp) so that this wait is bounded too
@@ -266,7 +266,7 @@ __global__ void __launch_bounds__(32 * PK_WARPS, 3) k_bsgs_accumulate_packed(
         if (lane == 0) {
             atomicExch(status, 3u);
             for (uint32_t sp = x_ok ? s + 1 : 0; sp < ld_s; sp++)
-                mbar_wait_bounded(my_bar + (sp % PK_STAGES) * 8, (sp / PK_STAGES) & 1);
+                mbar_wait_bounded(my_bar + (sp % ST) * 8, (sp / ST) & 1);
         }
         __syncwarp();
     }
@@ -276,26 +276,30 @@ int bsgs_accumulate_packed(fesc_ctx* ctx, const uint8_t* xpk, const uint8_t* dpk
                            uint32_t terms, uint32_t bp_count, bool fp, uint32_t dshift, cudaStream_t st) {
     const uint32_t N = ctx->N, ksteps = (terms + 31) / 32;
     dim3 grid(2 * (N / PK_CW) * ((tbs + 3) / 4), level);
-#define PK_LAUNCH(FP, KSR)                                                                                        \
+#define PK_LAUNCH(FP, KSR, ST)                                                                                    \
     do {                                                                                                          \
-        const size_t smem = (size_t)PK_WARPS * ((PK_STAGES + KSR) * PK_FRAG + (PK_STAGES + 1) * 8) + 2 * 256 * 8 + 8; \
-        auto kern = k_bsgs_accumulate_packed<FP, KSR>;                                                            \
+        const size_t smem = (size_t)PK_WARPS * ((ST + KSR) * PK_FRAG + (ST + 1) * 8) + 2 * 256 * 8 + 8;           \
+        auto kern = k_bsgs_accumulate_packed<FP, KSR, ST>;                                                        \
         FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
         kern<<<grid, 32 * PK_WARPS, smem, st>>>(xpk, dpk, acc, ctx->d_pc, N, level, tbs, ksteps, bp_count, dshift, \
                                                 ctx->d_status);                                                   \
     } while (0)
+    // input fragments of up to 6 k-steps stay in shared memory (ring + inputs = 10 slots per warp, so that three CTAs
+    // still share an SM); longer sums read them through L1 / L2 at every step
+#define PK_PICK(FP)                                   \
+    do {                                              \
+        if (ksteps == 1) PK_LAUNCH(FP, 1, PK_STAGES); \
+        else if (ksteps == 2) PK_LAUNCH(FP, 2, PK_STAGES); \
+        else if (ksteps == 3) PK_LAUNCH(FP, 3, PK_STAGES); \
+        else if (ksteps == 4) PK_LAUNCH(FP, 4, 6);    \
+        else if (ksteps == 5) PK_LAUNCH(FP, 5, 5);    \
+        else if (ksteps == 6) PK_LAUNCH(FP, 6, 4);    \
+        else PK_LAUNCH(FP, 0, PK_STAGES);             \
+    } while (0)
     prof_begin(ctx, PF_BSGS, st);
-    if (fp) {
-        if (ksteps == 1) PK_LAUNCH(true, 1);
-        else if (ksteps == 2) PK_LAUNCH(true, 2);
-        else if (ksteps == 3) PK_LAUNCH(true, 3);
-        else PK_LAUNCH(true, 0);
-    } else {
-        if (ksteps == 1) PK_LAUNCH(false, 1);
-        else if (ksteps == 2) PK_LAUNCH(false, 2);
-        else if (ksteps == 3) PK_LAUNCH(false, 3);
-        else PK_LAUNCH(false, 0);
-    }
+    if (fp) PK_PICK(true);
+    else PK_PICK(false);
+#undef PK_PICK
 #undef PK_LAUNCH
     prof_end(ctx, PF_BSGS, st);
     FESC_CHECK_CUDA(ctx, cudaGetLastError());

@@ -365,3 +365,18 @@ def test_linear_falls_back_to_smaller_groups_when_scratch_cannot_be_had(packed):
     assert e.value.code == fesc.ENOMEM
     ctx.test_fail_allocs(0)
     assert np.array_equal(_run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=kb, packed=packed), want)
+
+
+@pytest.mark.parametrize("gin", [7, 9, 11])
+def test_linear_packed_input_fragments_of_4_to_6_ksteps(gin):
+    """Sums of 112, 144 and 176 terms: the packed accumulate keeps the input fragments of 4, 5 and 6 k-steps in shared
+    memory beside a shorter ring (the token-major in_proj has 189 terms); residues against the oracle, both operand forms."""
+    T, C, n1, n2, tokens, d_out, level = 16, 32, 16, 2, 40, 40, 3
+    pair = ctx_pair("small")
+    ctx, orc, _ = pair
+    kb = 1000 + 37 * T + 5000
+    X, W, cts, diags, dims = _setup(pair, T, C, n1, n2, tokens, gin * C - 3, d_out, level, 2.0**40, wscale=10.0, key_base=kb)
+    assert dims[0] == gin
+    want = orc.linear(cts, diags, dict(n1=n1, n2=n2), {q: kb + q for q in range(1, n1)}, {g: kb + 500 + g for g in range(1, n2)})
+    assert np.array_equal(_run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=kb, packed=1), want)
+    assert np.array_equal(_run_gpu(ctx, cts, diags, n1, n2, dims, level, key_base=kb, packed=0), want)
