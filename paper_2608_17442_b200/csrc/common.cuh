@@ -215,6 +215,7 @@ struct RescaleTab {
     u64 qinv[FESC_MAX_PRIMES], qinvs[FESC_MAX_PRIMES];   // q_{l-1}^-1 mod q_i
     u64 wrap[FESC_MAX_PRIMES];                           // q_{l-1} mod q_i
     u64 half;                                            // floor(q_{l-1} / 2)
+    double qinvd[FESC_MAX_PRIMES];                       // qinv as doubles (exact below 2^53)
 };
 struct Tables {
     ModUpDigit* d_modup;      // [(level-1) * beta_max + digit], level = 1..n_q
@@ -293,13 +294,15 @@ static inline int fesc_fail(fesc_ctx* ctx, int code, const std::string& msg) {
 
 // Optional epilogue of the last pass of a forward N = 2^16 transform over rows r = bp * level + i (bp = ciphertext * 2 +
 // polynomial, i = data limb, all primes below 2^50): instead of storing the transformed row u, the pass stores the last
-// step of the division by P,  out[b][p][i] = (acc[bp][i] - u) * P^-1  (added to what out holds when bit p of add_mask
-// is set), which saves writing u, reading it back and a launch.
+// step of an exact division,  out[b][p][i] = (acc[bp][i] - u) * c_i  (added to what out holds when bit p of add_mask
+// is set), which saves writing u, reading it back and a launch.  Division by P after a key switch: acc = the inner
+// products, c_i = P^-1 mod q_i.  Rescale: acc = the input ciphertexts, c_i = q_last^-1 mod q_i, out may be the buffer
+// that holds u.
 struct NttFinish {
     const u64* acc = nullptr;        // [batch * 2][acc_rows][N]; nullptr = no epilogue
     u64* out = nullptr;              // ciphertext b at out + b * out_stride, [2][level][N]
     size_t out_stride = 0;
-    const ModDownTab* tab = nullptr; // P^-1 mod q_i as doubles
+    const double* cinv = nullptr;    // device array: c_i as doubles
     uint32_t level = 0, acc_rows = 0;
     int add_mask = 0;
 };

@@ -371,6 +371,7 @@ static int build_tables(fesc_ctx* ctx) {
             rs[level].qinv[i] = h_inv(ql % q[i], q[i]);
             rs[level].qinvs[i] = h_shoup(rs[level].qinv[i], q[i]);
             rs[level].wrap[i] = ql % q[i];
+            rs[level].qinvd[i] = (double)rs[level].qinv[i];
         }
     }
     return upload(ctx, &ctx->tabs.d_rescale, rs);

@@ -557,7 +557,7 @@ __global__ void __launch_bounds__(NTT_WARPS * 32) ntt16_contig(u64* __restrict__
             contig_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, 256 + blk, out_double,
                                 fin.acc + ((size_t)bp * fin.acc_rows + i) * N16 + (size_t)blk * 256,
                                 fin.out + (size_t)(bp >> 1) * fin.out_stride + ((size_t)(bp & 1) * fin.level + i) * N16 + (size_t)blk * 256,
-                                fin.tab->pinvd[i], (fin.add_mask >> (bp & 1)) & 1);
+                                fin.cinv[i], (fin.add_mask >> (bp & 1)) & 1);
         } else {
             contig_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, 256 + blk, out_double);
         }
