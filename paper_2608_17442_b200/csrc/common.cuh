@@ -222,6 +222,8 @@ struct Tables {
     ModDownTab* d_moddown;
     RescaleTab* d_rescale;    // [level], level = 2..n_q (index 0,1 unused)
     u64* d_Pmod_all;          // P mod q_t for every prime index (0 on special primes)
+    uint4* d_md_frag;         // constant operand fragments of the tensor-core conversion of the division by P
+                              // (bconv.cu), 512 uint4; nullptr when the shapes are not covered
 };
 
 // ---------------------------------------------------------------------------------------

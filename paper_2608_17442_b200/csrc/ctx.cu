@@ -297,6 +297,25 @@ static RowMap all_limbs_map(const fesc_ctx* ctx) {
 }
 
 // Basis-conversion tables, computed with 128-bit host arithmetic.
+// Constant A-operand fragments of one basis conversion for mma.sync.m16n8k32 (u8): tile t of 16 target rows, byte plane a
+// of the constants C(row, k, b) = M[k][row] * 256^b mod q_row, K index = 8 k + b.  Lane (g, tg) holds, for rows 16 t + g
+// (x, z) and 16 t + g + 8 (y, w), the K bytes 4 tg .. 4 tg + 3 (x, y) and 16 + 4 tg .. (z, w).
+template <typename F>
+static void bconv_fragments(uint4* out, F C) {
+    for (uint32_t t = 0; t < 2; t++)
+        for (uint32_t a = 0; a < 8; a++)
+            for (uint32_t lane = 0; lane < 32; lane++) {
+                const uint32_t g = lane >> 2, tg = lane & 3;
+                auto pack = [&](uint32_t row, uint32_t k) {
+                    uint32_t w = 0;
+                    for (uint32_t jj = 0; jj < 4; jj++) w |= (uint32_t)((C(row, k, 4 * (tg & 1) + jj) >> (8 * a)) & 0xff) << (8 * jj);
+                    return w;
+                };
+                out[(t * 8 + a) * 32 + lane] = make_uint4(pack(16 * t + g, tg >> 1), pack(16 * t + g + 8, tg >> 1),
+                                                          pack(16 * t + g, 2 + (tg >> 1)), pack(16 * t + g + 8, 2 + (tg >> 1)));
+            }
+}
+
 static int build_tables(fesc_ctx* ctx) {
     const uint32_t nq = ctx->n_q, np = ctx->n_primes, K = ctx->n_p, alpha = ctx->alpha;
     const std::vector<u64>& q = ctx->q;
@@ -360,6 +379,16 @@ static int build_tables(fesc_ctx* ctx) {
         md.pinvd[i] = (double)md.pinv[i];
     }
     if ((rc = upload(ctx, &ctx->tabs.d_moddown, mdv)) != FESC_OK) return rc;
+    if (K <= 4) {
+        std::vector<uint4> df(512);
+        bconv_fragments(df.data(), [&](uint32_t row, uint32_t k, uint32_t b) -> u64 {
+            if (row >= nq || k >= K) return 0;
+            u64 s = 1;
+            for (uint32_t e = 0; e < b; e++) s = h_mul(s, 256, q[row]);
+            return h_mul(md.mat[k][row], s, q[row]);
+        });
+        if ((rc = upload(ctx, &ctx->tabs.d_md_frag, df)) != FESC_OK) return rc;
+    }
     if ((rc = upload(ctx, &ctx->tabs.d_Pmod_all, Pmod)) != FESC_OK) return rc;
     // Rescale
     std::vector<RescaleTab> rs(nq + 1);
@@ -381,6 +410,7 @@ static void free_tables(fesc_ctx* ctx) {
     dev_free(ctx->tabs.d_moddown);
     dev_free(ctx->tabs.d_rescale);
     dev_free(ctx->tabs.d_Pmod_all);
+    dev_free(ctx->tabs.d_md_frag);
 }
 
 // Generate the switching key from s' (EVAL on all limbs, device) to s.

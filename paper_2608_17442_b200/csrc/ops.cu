@@ -782,7 +782,9 @@ static int ks_moddown(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint32
     for (uint32_t t = 0; t < rows; t++) m.prime[t] = t < level ? 0xFF : (uint8_t)(nq + (t - level));
     if ((rc = ntt_launch(ctx, ws.acc, (size_t)batch * 2 * rows, m, true, st)) != FESC_OK) return rc;
     prof_begin(ctx, PF_MODDOWN, st);
-    if (N % (256 * KS_VEC) == 0)
+    if (bconv_supported(ctx, level))
+        moddown_conv_imma_launch(ctx, ws.acc, ws.u, level, batch, ctx->log_n == 16, st);
+    else if (N % (256 * KS_VEC) == 0)
         k_moddown_conv<KS_VEC><<<dim3(N / (256 * KS_VEC), batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K, ctx->log_n == 16);
     else
         k_moddown_conv<1><<<dim3(gx, batch * 2), 256, 0, st>>>(ws.acc, ws.u, ctx->tabs.d_moddown, ctx->d_pc, N, level, nq, K, ctx->log_n == 16);

@@ -94,6 +94,10 @@ __device__ __forceinline__ u64 imma_recombine(const int (&d)[4][7][4], int sel, 
 }
 #endif
 
+// basis conversions on the tensor cores (bconv.cu)
+bool bconv_supported(const fesc_ctx* ctx, uint32_t level);
+void moddown_conv_imma_launch(fesc_ctx* ctx, const u64* acc, u64* u, uint32_t level, uint32_t batch, int out_double, cudaStream_t st);
+
 // packed-operand BSGS accumulate (packed.cu)
 size_t bsgs_packed_bytes(uint32_t N, uint32_t level, uint32_t rows, uint32_t terms);
 bool bsgs_packed_supported(const fesc_ctx* ctx, uint32_t level, uint32_t terms, uint32_t dshift);
