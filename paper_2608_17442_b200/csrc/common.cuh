@@ -301,7 +301,8 @@ static inline int fesc_fail(fesc_ctx* ctx, int code, const std::string& msg) {
 // products, c_i = P^-1 mod q_i.  Rescale: acc = the input ciphertexts, c_i = q_last^-1 mod q_i, out may be the buffer
 // that holds u.
 struct NttFinish {
-    const u64* acc = nullptr;        // [batch * 2][acc_rows][N]; nullptr = no epilogue
+    const u64* acc = nullptr;        // ciphertext b at acc + b * acc_stride, [2][acc_rows][N]; nullptr = no epilogue
+    size_t acc_stride = 0;
     u64* out = nullptr;              // ciphertext b at out + b * out_stride, [2][level][N]
     size_t out_stride = 0;
     const double* cinv = nullptr;    // device array: c_i as doubles

@@ -550,12 +550,12 @@ __global__ void __launch_bounds__(NTT_WARPS * 32) ntt16_contig(u64* __restrict__
     if (pc.q < FP_LIMIT) {
         if (!INV && fin.acc) {      // rows of this launch: r = bp * level + i
             const uint32_t r = row_first + row, bp = r / fin.level, i = r - bp * fin.level;
-            if (!DBG_REGION(fin.acc + ((size_t)bp * fin.acc_rows + i) * N16 + (size_t)blk * 256, 256 * sizeof(u64)) ||
+            if (!DBG_REGION(fin.acc + (size_t)(bp >> 1) * fin.acc_stride + ((size_t)(bp & 1) * fin.acc_rows + i) * N16 + (size_t)blk * 256, 256 * sizeof(u64)) ||
                 !DBG_REGION(fin.out + (size_t)(bp >> 1) * fin.out_stride + ((size_t)(bp & 1) * fin.level + i) * N16 + (size_t)blk * 256,
                             256 * sizeof(u64)))
                 return;
             contig_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, 256 + blk, out_double,
-                                fin.acc + ((size_t)bp * fin.acc_rows + i) * N16 + (size_t)blk * 256,
+                                fin.acc + (size_t)(bp >> 1) * fin.acc_stride + ((size_t)(bp & 1) * fin.acc_rows + i) * N16 + (size_t)blk * 256,
                                 fin.out + (size_t)(bp >> 1) * fin.out_stride + ((size_t)(bp & 1) * fin.level + i) * N16 + (size_t)blk * 256,
                                 fin.cinv[i], (fin.add_mask >> (bp & 1)) & 1);
         } else {

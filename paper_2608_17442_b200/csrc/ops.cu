@@ -795,7 +795,7 @@ static int ks_moddown(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint32
     for (uint32_t i = 0; i < level; i++) fuse = fuse && ctx->q[i] < FESC_FP_LIMIT;
     if (fuse) {
         NttFinish fin;
-        fin.acc = ws.acc, fin.out = out, fin.out_stride = out_stride, fin.cinv = ctx->tabs.d_moddown->pinvd;
+        fin.acc = ws.acc, fin.acc_stride = (size_t)2 * rows * N, fin.out = out, fin.out_stride = out_stride, fin.cinv = ctx->tabs.d_moddown->pinvd;
         fin.level = level, fin.acc_rows = rows, fin.add_mask = add_mask;
         return ntt_launch(ctx, ws.u, (size_t)batch * 2 * level, m, false, st, true, false, &fin);
     }
@@ -1132,12 +1132,12 @@ int rescale_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, u
         prof_end(ctx, PF_RESCALE, st);
         m.period = level - 1;
         for (uint32_t i = 0; i + 1 < level; i++) m.prime[i] = (uint8_t)i;
-        // N = 2^16, FP64 rows, contiguous input: the last pass of the transform stores (in - u) * q_last^-1 itself
-        bool fuse = ctx->log_n == 16 && in_stride == (size_t)2 * level * N;
+        // N = 2^16, FP64 rows: the last pass of the transform stores (in - u) * q_last^-1 itself
+        bool fuse = ctx->log_n == 16;
         for (uint32_t i = 0; i + 1 < level; i++) fuse = fuse && ctx->q[i] < FESC_FP_LIMIT;
         if (fuse) {
             NttFinish fin;
-            fin.acc = ib, fin.out = ob, fin.out_stride = out_stride, fin.cinv = tab->qinvd;
+            fin.acc = ib, fin.acc_stride = in_stride, fin.out = ob, fin.out_stride = out_stride, fin.cinv = tab->qinvd;
             fin.level = level - 1, fin.acc_rows = level, fin.add_mask = 0;
             if ((rc = ntt_launch(ctx, ob, (size_t)nb * 2 * (level - 1), m, false, st, false, false, &fin)) != FESC_OK) return rc;
             continue;
