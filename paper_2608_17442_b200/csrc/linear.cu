@@ -595,13 +595,13 @@ static int bsgs_kernel() {
     return v;
 }
 // Larger groups re-read the diagonals less often and give the key-switch kernels larger batches; every token block
-// of a group needs its rotated inputs and its partial sums resident.  Budget: 24 GiB of scratch for them (32 GiB with packed operands, whose packed inputs
+// of a group needs its rotated inputs and its partial sums resident.  Budget: 28 GiB of scratch for them (37 GiB with packed operands, whose packed inputs
 // and key-switch chunk count as well; 44 GiB allows groups of 8; a fixed figure, so the launch shape does not depend on what else holds memory); if the device cannot provide the scratch,
 // the group is halved until it fits.
 static size_t bsgs_group_bytes(bool packed) {
     const char* e = getenv("FESC_BSGS_GROUP_GIB");
     if (e && atoi(e) > 0) return (size_t)atoi(e) << 30;
-    return (size_t)(packed ? 32 : 24) << 30;
+    return (size_t)(packed ? 37 : 28) << 30;
 }
 
 // Projection on packed diagonals.  Token blocks are processed in groups of up to 8 = two tiles of 4: the baby rotations
@@ -628,7 +628,7 @@ static int linear_packed(fesc_ctx* ctx, const u64* in, const uint8_t* image, con
         nb_part = (nb_part + bstep - 1) / bstep * bstep;
         if (nb_part > nout) nb_part = nout;
         const uint32_t max_batch = sub * gin > tbg * nb_part ? sub * gin : tbg * nb_part;
-        const size_t ks_words = ks_scratch_words(ctx, level, ks_chunk(ctx, max_batch));
+        const size_t ks_words = ks_scratch_words(ctx, level, ks_chunk(ctx, max_batch), desc->defer ? giant_ext_buffers(n2) : 1);
         const size_t rs_words = (size_t)(nb_part < 16384 ? nb_part : 16384) * 2 * N;
         const size_t rot_words = (size_t)sub * terms * ctw, acc_words = (size_t)tbg * nb_part * n2 * ctw;
         const size_t xpk_words = bsgs_packed_bytes(N, level, 2 * tbg, terms) / 8;
@@ -735,7 +735,7 @@ extern "C" int fesc_linear(fesc_ctx* ctx, const uint64_t* d_ct_in, const uint64_
     int rc;
     for (;;) {
         const uint32_t max_batch = tbg * (gin > nout ? gin : nout);
-        const size_t ks_words = ks_scratch_words(ctx, level, ks_chunk(ctx, max_batch));
+        const size_t ks_words = ks_scratch_words(ctx, level, ks_chunk(ctx, max_batch), desc->defer ? giant_ext_buffers(n2) : 1);
         const size_t rs_words = (size_t)(tbg * nout < 16384 ? tbg * nout : 16384) * 2 * N;
         const size_t rot_words = (size_t)tbg * gin * n1 * ctw, acc_words = (size_t)tbg * nout * n2 * ctw;
         rc = ctx_scratch(ctx, (rot_words + acc_words + (ks_words > rs_words ? ks_words : rs_words)) * sizeof(u64), &scratch);

@@ -234,39 +234,48 @@ __global__ void __launch_bounds__(256) k_modup(const u64* __restrict__ dcoef, u6
 #ifndef INNER_MINB
 #define INNER_MINB 4
 #endif
+// Several sources can be summed in one pass: source s contributes sum_j dt_j(ext_s)[pi_{g_s}(t)] * key_s[j].  The giant
+// steps of a projection (different converted polynomials, different keys, one sum) and the rotate-and-add chains (one
+// converted polynomial read through several Galois permutations, one key each) then read and write the accumulators
+// once instead of once per key, and the later reads of a shared source hit L2.
+#define INNER_MAX_SRC 8
+struct InnerSrc {
+    const u64* ext;   // [batch][beta][level+K][N]
+    const u64* key;   // [beta][2][n_q+K][N]
+    u64 g;            // Galois element the digits are read through (0: none)
+};
+struct InnerSrcs {
+    InnerSrc s[INNER_MAX_SRC];
+    uint32_t n;
+};
 // PATH 0: the row's prime decides at run time; 1: the caller guarantees primes below 2^50 on rows
 // [row0, row0 + gridDim.y) (exact FP64 products only); 2: the caller sends those rows to the 128-bit integer sums.
 template <int BT, int PATH>
-__global__ void __launch_bounds__(256, INNER_MINB) k_inner(const u64* __restrict__ ext,
-                                               const u64* __restrict__ key, u64* __restrict__ acc,
+__global__ void __launch_bounds__(256, INNER_MINB) k_inner(InnerSrcs S, u64* __restrict__ acc,
                                                const PrimeConst* __restrict__ pcs, uint32_t N, uint32_t level,
                                                uint32_t n_q, uint32_t K, uint32_t alpha, uint32_t beta,
-                                               uint32_t batch, uint32_t log_n, u64 g, int accumulate, uint32_t row0,
+                                               uint32_t batch, uint32_t log_n, int accumulate, uint32_t row0,
                                                int x_double) {
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t t = row0 + blockIdx.y, b0 = blockIdx.z * BT;
     if (c >= N) return;
-    // hoisted rotations: the automorphism acts on the extended digits, i.e. they are read at pi_g(c)
-    const uint32_t cs = g ? galois_src(c, log_n, g) : c;
     const uint32_t rows = level + K, np = n_q + K;
     const uint32_t pt = t < level ? t : n_q + (t - level);
     // operand words of one digit: key (b, a) and the BT ciphertext words; clamped indices keep loads valid.
     // All addresses are a per-thread base plus a multiple of one stride (no per-load index products).
     const size_t kstride = (size_t)np * N, xstride = (size_t)rows * N;
-    const u64* kp = key + (size_t)pt * N + c;
-    const u64* xp[BT];
-#pragma unroll
-    for (int i = 0; i < BT; i++) {
-        const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
-        xp[i] = ext + ((size_t)b * beta * rows + t) * N + cs;
-    }
 #ifdef FESC_DEBUG_BOUNDS
-    if (cs >= N) return;
-    for (uint32_t j = 0; j < beta; j++) {
-        if (!DBG_REGION(kp - c + (size_t)(2 * j) * kstride, N * sizeof(u64)) || !DBG_REGION(kp - c + (size_t)(2 * j + 1) * kstride, N * sizeof(u64)))
-            return;
-        for (int i = 0; i < BT; i++)
-            if (!DBG_REGION(xp[i] - cs + (size_t)j * xstride, N * sizeof(u64))) return;
+    for (uint32_t s = 0; s < S.n; s++) {
+        if (S.s[s].g && galois_src(c, log_n, S.s[s].g) >= N) return;
+        for (uint32_t j = 0; j < beta; j++) {
+            if (!DBG_REGION(S.s[s].key + ((size_t)(2 * j) * np + pt) * N, N * sizeof(u64)) ||
+                !DBG_REGION(S.s[s].key + ((size_t)(2 * j + 1) * np + pt) * N, N * sizeof(u64)))
+                return;
+            for (int i = 0; i < BT; i++) {
+                const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
+                if (!DBG_REGION(S.s[s].ext + (((size_t)b * beta + j) * rows + t) * N, N * sizeof(u64))) return;
+            }
+        }
     }
     for (int i = 0; i < BT; i++) {
         const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
@@ -275,15 +284,36 @@ __global__ void __launch_bounds__(256, INNER_MINB) k_inner(const u64* __restrict
             return;
     }
 #endif
-    auto load_digit = [&](uint32_t j, u64& kb, u64& ka, u64 (&x)[BT]) {
-        kb = __ldg(kp + (size_t)(2 * j) * kstride);
-        ka = __ldg(kp + (size_t)(2 * j + 1) * kstride);
+    // the (source, digit) whose words are requested next; hoisted rotations: the automorphism acts on the extended
+    // digits, i.e. they are read at pi_g(c)
+    uint32_t sn = 0, jn = 0;
+    const u64* kp;
+    const u64* xp[BT];
+    auto setup = [&](uint32_t s) {
+        const u64 g = S.s[s].g;
+        const uint32_t cs = g ? galois_src(c, log_n, g) : c;
+        kp = S.s[s].key + (size_t)pt * N + c;
 #pragma unroll
-        for (int i = 0; i < BT; i++) x[i] = xp[i][(size_t)j * xstride];
+        for (int i = 0; i < BT; i++) {
+            const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
+            xp[i] = S.s[s].ext + ((size_t)b * beta * rows + t) * N + cs;
+        }
     };
+    auto load_next = [&](u64& kb, u64& ka, u64 (&x)[BT]) {
+        kb = __ldg(kp + (size_t)(2 * jn) * kstride);
+        ka = __ldg(kp + (size_t)(2 * jn + 1) * kstride);
+#pragma unroll
+        for (int i = 0; i < BT; i++) x[i] = xp[i][(size_t)jn * xstride];
+        if (++jn == beta) {
+            jn = 0;
+            if (++sn < S.n) setup(sn);
+        }
+    };
+    const uint32_t total = S.n * beta;
+    setup(0);
     if (PATH == 1 || (PATH == 0 && pcs[pt].q < FESC_FP_LIMIT)) {
         // exact FP64 products of canonical words (both below q): every product is below 0.875q, so a running sum of
-        // at most q/2 plus 7 terms stays below 2^53 = 8q; longer sums are folded back after every 7th digit.  The next digit's words
+        // at most q/2 plus 7 terms stays below 2^53 = 8q; longer sums are folded back after every 7th term.  The next digit's words
         // are requested before this digit's products start: 2 + BT loads in flight per thread, few registers,
         // so that four CTAs per SM overlap their loads and products (measured: one digit ahead with 4 CTAs of 4
         // ciphertexts per thread moves 1.6x the bytes per second of all-digits-up-front with 2 CTAs; 8 ciphertexts
@@ -293,17 +323,19 @@ __global__ void __launch_bounds__(256, INNER_MINB) k_inner(const u64* __restrict
 #pragma unroll
         for (int i = 0; i < BT; i++) {
             f0[i] = f1[i] = 0.0;
-            if (accumulate) {   // running sum over several keys (division by P deferred)
+            if (accumulate) {   // running sum over several passes (division by P deferred)
                 const uint32_t b = b0 + i < batch ? b0 + i : batch - 1;
                 f0[i] = fp_load(acc[(((size_t)b * 2 + 0) * rows + t) * N + c], q);
                 f1[i] = fp_load(acc[(((size_t)b * 2 + 1) * rows + t) * N + c], q);
             }
         }
-        u64 kb, ka, x[BT], nkb, nka, nx[BT];
-        load_digit(0, kb, ka, x);
+        u64 kb, ka, x[BT], nkb = 0, nka = 0, nx[BT];
+#pragma unroll
+        for (int i = 0; i < BT; i++) nx[i] = 0;
+        load_next(kb, ka, x);
 #pragma unroll 1
-        for (uint32_t j = 0; j < beta; j++) {
-            load_digit(j + 1 < beta ? j + 1 : j, nkb, nka, nx);
+        for (uint32_t it = 0; it < total; it++) {
+            if (it + 1 < total) load_next(nkb, nka, nx);
             const double dkb = fp_from_u64(kb), dka = fp_from_u64(ka);
 #pragma unroll
             for (int i = 0; i < BT; i++) {
@@ -312,7 +344,7 @@ __global__ void __launch_bounds__(256, INNER_MINB) k_inner(const u64* __restrict
                 f0[i] += fp_modmul(xd, dkb, q, qinv);
                 f1[i] += fp_modmul(xd, dka, q, qinv);
             }
-            if (j % 7 == 6) {   // |running sum| <= q/2 plus 7 products below 0.875q each stays below 6.7q < 2^53: fold after every 7th
+            if (it % 7 == 6) {   // |running sum| <= q/2 plus 7 products below 0.875q each stays below 6.7q < 2^53: fold after every 7th
 #pragma unroll
                 for (int i = 0; i < BT; i++) {
                     f0[i] = fp_reduce(f0[i], q, qinv);
@@ -334,26 +366,36 @@ __global__ void __launch_bounds__(256, INNER_MINB) k_inner(const u64* __restrict
         return;
     }
     if (PATH != 1) {
+        const PrimeConst pc = pcs[pt];
         acc128 a0[BT], a1[BT];
-    #pragma unroll
+#pragma unroll
         for (int i = 0; i < BT; i++) a0[i] = a1[i] = acc128{0, 0};
         {
-            u64 kb, ka, x[BT], nkb, nka, nx[BT];
-            load_digit(0, kb, ka, x);
-            for (uint32_t j = 0; j < beta; j++) {
-                load_digit(j + 1 < beta ? j + 1 : j, nkb, nka, nx);
-    #pragma unroll
+            u64 kb, ka, x[BT], nkb = 0, nka = 0, nx[BT];
+#pragma unroll
+            for (int i = 0; i < BT; i++) nx[i] = 0;
+            load_next(kb, ka, x);
+#pragma unroll 1
+            for (uint32_t it = 0; it < total; it++) {
+                if (it + 1 < total) load_next(nkb, nka, nx);
+#pragma unroll
                 for (int i = 0; i < BT; i++) {
                     mac128(a0[i], x[i], kb);
                     mac128(a1[i], x[i], ka);
                 }
+                if ((it & 7) == 7 && it + 1 < total) {   // 8 products below 2^124 cannot wrap 128 bits: longer sums are reduced in between
+#pragma unroll
+                    for (int i = 0; i < BT; i++) {
+                        a0[i] = acc128{reduce128(a0[i].hi, a0[i].lo, pc), 0};
+                        a1[i] = acc128{reduce128(a1[i].hi, a1[i].lo, pc), 0};
+                    }
+                }
                 kb = nkb, ka = nka;
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < BT; i++) x[i] = nx[i];
             }
         }
-        const PrimeConst pc = pcs[pt];
-    #pragma unroll
+#pragma unroll
         for (int i = 0; i < BT; i++) {
             const uint32_t b = b0 + i;
             if (b < batch) {
@@ -724,20 +766,20 @@ static int ks_decompose(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint
     return FESC_OK;
 }
 
-// Step 4: inner product with `key` (digits read through the Galois permutation of g when g != 0) into ws.acc;
-// accumulate != 0 adds to what ws.acc holds (sums over several keys before one division by P).
-static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint32_t level, uint32_t batch,
-                    cudaStream_t st, u64 g, int accumulate) {
+// Step 4: inner products of the sources `S` (converted digits, key, Galois element each) summed into ws.acc;
+// accumulate != 0 adds to what ws.acc holds (sums over several passes before one division by P).
+static int ks_inner_multi(fesc_ctx* ctx, const KsScratch& ws, const InnerSrcs& S, uint32_t level, uint32_t batch,
+                          cudaStream_t st, int accumulate) {
     const uint32_t N = ctx->N, K = ctx->n_p, nq = ctx->n_q, alpha = ctx->alpha;
     const uint32_t beta = (level + alpha - 1) / alpha, rows = level + K;
     const uint32_t gx = (N + 255) / 256;
     prof_begin(ctx, PF_INNER, st);
-    const bool use_tma = getenv("FESC_INNER_TMA") != nullptr;   // read per call so a test can switch it
+    const bool use_tma = S.n == 1 && getenv("FESC_INNER_TMA") != nullptr;   // read per call so a test can switch it
 #define INNER(BT_, PATH_, ROW0_, NROWS_)                                                                        \
     do {                                                                                                        \
         dim3 gd(gx, NROWS_, (batch + BT_ - 1) / BT_);                                                           \
-        k_inner<BT_, PATH_><<<gd, 256, 0, st>>>(ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, \
-                                                beta, batch, ctx->log_n, g, accumulate, ROW0_, ctx->log_n == 16); \
+        k_inner<BT_, PATH_><<<gd, 256, 0, st>>>(S, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta, batch,     \
+                                                ctx->log_n, accumulate, ROW0_, ctx->log_n == 16);              \
     } while (0)
     // data rows on primes below 2^50 and special rows above: one launch per kind, each compiled for its arithmetic
     bool split = true;
@@ -751,8 +793,8 @@ static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         FESC_CHECK_CUDA(ctx, cudaFuncSetAttribute(k_inner_tma<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         const uint32_t grid = n_tiles < (uint32_t)sms ? n_tiles : (uint32_t)sms;
-        k_inner_tma<4><<<grid, 256, smem, st>>>(ws.ext, key.d_key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta,
-                                                 batch, ctx->log_n, g, accumulate, n_tiles, ctx->d_status, ctx->log_n == 16);
+        k_inner_tma<4><<<grid, 256, smem, st>>>(S.s[0].ext, S.s[0].key, ws.acc, ctx->d_pc, N, level, nq, K, alpha, beta,
+                                                 batch, ctx->log_n, S.s[0].g, accumulate, n_tiles, ctx->d_status, ctx->log_n == 16);
     } else if (split) {
         if (batch >= 3) INNER(4, 1, 0, level);
         else if (batch == 2) INNER(2, 1, 0, level);
@@ -766,8 +808,16 @@ static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint
 #undef INNER
     prof_end(ctx, PF_INNER, st);
     FESC_CHECK_CUDA(ctx, cudaGetLastError());
-    ctx->counters[1] += batch;
+    ctx->counters[1] += (uint64_t)batch * S.n;
     return FESC_OK;
+}
+// one source: ws.ext with `key`, digits read through the Galois permutation of g when g != 0
+static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint32_t level, uint32_t batch,
+                    cudaStream_t st, u64 g, int accumulate) {
+    InnerSrcs S;
+    S.n = 1;
+    S.s[0] = InnerSrc{ws.ext, key.d_key, g};
+    return ks_inner_multi(ctx, ws, S, level, batch, st, accumulate);
 }
 
 // Step 5: division of ws.acc by P; the result is ADDED to out[b][p] when bit p of add_mask is set, else stored.
@@ -829,17 +879,17 @@ static OwnRows own_rows(const fesc_ctx* ctx, const KsScratch& ws, uint32_t level
     return OwnRows{ws.ext, ctx->alpha, (level + ctx->alpha - 1) / ctx->alpha, level + ctx->n_p, ctx->log_n == 16};
 }
 
-size_t ks_scratch_words(const fesc_ctx* ctx, uint32_t level, uint32_t chunk) {
+size_t ks_scratch_words(const fesc_ctx* ctx, uint32_t level, uint32_t chunk, uint32_t n_ext) {
     const uint32_t beta = (level + ctx->alpha - 1) / ctx->alpha, rows = level + ctx->n_p;
-    return (size_t)chunk * ctx->N * ((size_t)level + (size_t)beta * rows + 2 * rows + 2 * level);
+    return (size_t)chunk * ctx->N * ((size_t)level + (size_t)n_ext * beta * rows + 2 * rows + 2 * level);
 }
-KsScratch ks_scratch_carve(const fesc_ctx* ctx, u64* base, uint32_t level, uint32_t chunk) {
+KsScratch ks_scratch_carve(const fesc_ctx* ctx, u64* base, uint32_t level, uint32_t chunk, uint32_t n_ext) {
     const uint32_t beta = (level + ctx->alpha - 1) / ctx->alpha, rows = level + ctx->n_p;
     const size_t N = ctx->N;
     KsScratch ws;
     ws.dcoef = base;
     ws.ext = ws.dcoef + (size_t)chunk * level * N;
-    ws.acc = ws.ext + (size_t)chunk * beta * rows * N;
+    ws.acc = ws.ext + (size_t)n_ext * chunk * beta * rows * N;
     ws.u = ws.acc + (size_t)chunk * 2 * rows * N;
     return ws;
 }
@@ -909,22 +959,34 @@ int giant_sum_deferred_internal(fesc_ctx* ctx, u64* acc, uint32_t n_terms, size_
     for (uint32_t p = 1; p < n_terms; p++)
         if (!ctx->keys.count(key_base + p) || key_base + p == FESC_RELIN_KEY_ID)
             return fesc_fail(ctx, FESC_ENOKEY, "giant steps: no Galois key " + std::to_string(key_base + p));
-    const uint32_t chunk = ks_chunk(ctx, batch);
-    KsScratch ws = ks_scratch_carve(ctx, scratch, level, chunk);
+    const uint32_t chunk = ks_chunk(ctx, batch), n_ext = giant_ext_buffers(n_terms);
+    KsScratch ws = ks_scratch_carve(ctx, scratch, level, chunk, n_ext);
     const size_t stride = (size_t)n_terms * ct_words;
+    const size_t ext_words = (size_t)chunk * ((level + ctx->alpha - 1) / ctx->alpha) * (level + ctx->n_p) * ctx->N;
     for (uint32_t b0 = 0; b0 < batch; b0 += chunk) {
         const uint32_t nb = batch - b0 < chunk ? batch - b0 : chunk;
         dim3 g((ctx->N + 255) / 256, level, nb);
         u64* base = acc + (size_t)b0 * stride;
-        for (uint32_t p = 1; p < n_terms; p++) {
-            const EvalKey& key = ctx->keys[key_base + p];
-            prof_begin(ctx, PF_AUTOM, st);
-            k_autom_ct<<<g, 256, 0, st>>>(base + (size_t)p * ct_words, stride, base, stride, own_rows(ctx, ws, level), ws.dcoef, ctx->log_n,
-                                          level, key.g, ctx->d_pc, 1);
-            prof_end(ctx, PF_AUTOM, st);
-            int rc = ks_decompose(ctx, ws, level, nb, st);
+        // up to n_ext terms are rotated and converted side by side, then one inner-product pass sums them: the
+        // accumulators on the extended basis are read and written once per pass instead of once per term
+        for (uint32_t p0 = 1; p0 < n_terms; p0 += n_ext) {
+            const uint32_t np = n_terms - p0 < n_ext ? n_terms - p0 : n_ext;
+            InnerSrcs S;
+            S.n = np;
+            for (uint32_t s = 0; s < np; s++) {
+                const EvalKey& key = ctx->keys[key_base + p0 + s];
+                KsScratch wss = ws;
+                wss.ext = ws.ext + (size_t)s * ext_words;
+                prof_begin(ctx, PF_AUTOM, st);
+                k_autom_ct<<<g, 256, 0, st>>>(base + (size_t)(p0 + s) * ct_words, stride, base, stride, own_rows(ctx, wss, level),
+                                              wss.dcoef, ctx->log_n, level, key.g, ctx->d_pc, 1);
+                prof_end(ctx, PF_AUTOM, st);
+                int rc = ks_decompose(ctx, wss, level, nb, st);
+                if (rc != FESC_OK) return rc;
+                S.s[s] = InnerSrc{wss.ext, key.d_key, 0};
+            }
+            int rc = ks_inner_multi(ctx, ws, S, level, nb, st, p0 > 1);
             if (rc != FESC_OK) return rc;
-            if ((rc = ks_inner(ctx, ws, key, level, nb, st, 0, p > 1)) != FESC_OK) return rc;
         }
         int rc = ks_moddown(ctx, ws, level, nb, base, stride, 3, st);
         if (rc != FESC_OK) return rc;
@@ -1015,8 +1077,10 @@ int rotate_sum_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, 
         prof_end(ctx, PF_AUTOM, st, 2);
         int rc = ks_decompose(ctx, ws, level, nb, st);
         if (rc != FESC_OK) return rc;
-        for (uint32_t k = 0; k < n_keys; k++)
-            if ((rc = ks_inner(ctx, ws, ctx->keys[key_ids[k]], level, nb, st, gs.g[k], k > 0)) != FESC_OK) return rc;
+        InnerSrcs S;                                   // one converted polynomial, read through every key's permutation
+        S.n = n_keys;
+        for (uint32_t k = 0; k < n_keys; k++) S.s[k] = InnerSrc{ws.ext, ctx->keys[key_ids[k]].d_key, gs.g[k]};
+        if ((rc = ks_inner_multi(ctx, ws, S, level, nb, st, 0)) != FESC_OK) return rc;
         if ((rc = ks_moddown(ctx, ws, level, nb, ob, out_stride, 3, st)) != FESC_OK) return rc;
     }
     return FESC_OK;

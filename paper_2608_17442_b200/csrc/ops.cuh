@@ -4,14 +4,17 @@
 
 // Scratch of one key-switch chunk (all [chunk][...][N] words):
 //   dcoef [level]            the polynomial being switched, transformed to COEFF in place
-//   ext   [beta][level+K]    converted digits; the rows of a digit's own limbs hold the polynomial itself (EVAL)
+//   ext   [beta][level+K]    converted digits; the rows of a digit's own limbs hold the polynomial itself (EVAL);
+//                            n_ext such buffers in a row when several polynomials are switched before one sum
 //   acc   [2][level+K]       inner-product accumulators
 //   u     [2][level]         converted special-limb part
 struct KsScratch {
     u64 *dcoef, *ext, *acc, *u;
 };
-size_t ks_scratch_words(const fesc_ctx* ctx, uint32_t level, uint32_t chunk);
-KsScratch ks_scratch_carve(const fesc_ctx* ctx, u64* base, uint32_t level, uint32_t chunk);
+size_t ks_scratch_words(const fesc_ctx* ctx, uint32_t level, uint32_t chunk, uint32_t n_ext = 1);
+KsScratch ks_scratch_carve(const fesc_ctx* ctx, u64* base, uint32_t level, uint32_t chunk, uint32_t n_ext = 1);
+// converted polynomials a deferred giant-step sum of n_terms keeps side by side (one inner-product pass over them)
+static inline uint32_t giant_ext_buffers(uint32_t n_terms) { return n_terms < 2 ? 1 : (n_terms - 1 < 4 ? n_terms - 1 : 4); }
 uint32_t ks_chunk(const fesc_ctx* ctx, uint32_t batch);
 
 int rotate_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, size_t out_stride, uint32_t batch,
@@ -22,6 +25,7 @@ int rotate_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64*
 int rotate_sum_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, size_t out_stride,
                                 uint32_t batch, uint32_t level, const uint32_t* key_ids, uint32_t n_keys, u64* scratch,
                                 cudaStream_t st);
+// scratch: ks_scratch_words(ctx, level, ks_chunk(ctx, batch), giant_ext_buffers(n_terms)) words
 int giant_sum_deferred_internal(fesc_ctx* ctx, u64* acc, uint32_t n_terms, size_t ct_words, uint32_t batch,
                                 uint32_t level, uint32_t key_base, u64* scratch, cudaStream_t st);
 int rescale_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, uint32_t batch, uint32_t level,
