@@ -207,6 +207,7 @@ MAC_MIXED_CYCLES = 8              # mixed-pipe multiply-accumulate: multiplier-p
 # read once per launch and every output byte written once, traffic grows in proportion to the algorithmic bytes.
 BSGS_TRAFFIC_RATIO = {"packed": 1.000, "residues": 1.001}     # measured DRAM bytes / algorithmic bytes (small case)
 PACKED_BYTES_PER_WORD = 7                                     # a residue below 2^56 as byte planes
+NTT_DISPATCH_CYCLES = 27.1        # dispatch-port cycles per warp-butterfly of the FP64 transforms: 9.5 x 2 + 8.1 (ncu opcode mix)
 NTT_TRAFFIC_RATIO = 1.0           # the transforms read and write every word of both passes through DRAM once
 INT_LIMB_SHARE = 32.0 / 224.0     # transforms on the 60-bit special primes per key switch (integer path)
 
@@ -530,11 +531,18 @@ def ntt_roofline(p, n, timed, limb_ntts, hbm_peak, sm_mhz):
     alu_peak = 1.0 / ((1.0 - INT_LIMB_SHARE) / peak_fp + INT_LIMB_SHARE / peak_int)
     ach = bfly / (ms * 1e-3) / 1e12
     moved = limb_ntts * 2 * 2 * n * 8           # two passes, each reads and writes the limb
+    # What the dispatch port allows with the measured instruction mix of the FP64 path (ncu opcode counts: 17.6 warp
+    # instructions per warp-butterfly, 9.5 of them FP64, which hold the port for two cycles): 27.1 cycles per
+    # warp-butterfly on each of the 4 schedulers of an SM.  The kernels also have to load, exchange and store, so this,
+    # not the FP64-pipe figure above, is the ceiling they can approach.
+    issue_peak = SM_COUNT * 4 * 32 * sm_mhz * 1e6 / NTT_DISPATCH_CYCLES / 1e12
     return {"kernel": "ntt", "variant": "ntt16_strided + ntt16_contig (two passes per limb transform)", "bound": "alu",
             "achieved": ach, "peak": alu_peak, "unit": "T butterflies/s (FP64 pipe for 50-bit primes, integer pipe for 60-bit)",
             "peak_fp64_path": peak_fp, "peak_integer_path": peak_int, "frac": ach / alu_peak,
             "traffic": moved / max(1, launches) * NTT_TRAFFIC_RATIO, "launches": launches, "limb_transforms": limb_ntts,
             "us_per_limb_transform": ms * 1e3 / max(1, limb_ntts), "family_ms": ms,
+            "dispatch": {"achieved": ach, "peak": issue_peak, "unit": "T butterflies/s", "frac": ach / issue_peak,
+                         "cycles_per_warp_butterfly": NTT_DISPATCH_CYCLES},
             "hbm": {"achieved": moved / (ms * 1e-3) / 1e9, "peak": hbm_peak, "unit": "GB/s",
                     "frac": moved / (ms * 1e-3) / 1e9 / hbm_peak, "bytes_moved_per_limb_transform": 4 * n * 8}}
 
