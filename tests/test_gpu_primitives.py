@@ -553,8 +553,8 @@ def test_results_do_not_depend_on_the_run_or_the_stream():
 
 def test_inner_product_worst_case_residues_with_many_digits():
     """Largest possible partial sums of the key inner product: 9 digits (the FP64 path folds back after every 7
-    products, so a second interval starts), every residue of the switched polynomial equal to q - 1, plain and
-    hoisted; bit-exact."""
+    products, so a second interval starts), every residue of the switched polynomial equal to q - 1, plain,
+    hoisted and summed over 8 keys in one pass; bit-exact."""
     import torch
 
     pair = ctx_pair("small_d9")
@@ -574,3 +574,14 @@ def test_inner_product_worst_case_residues_with_many_digits():
         assert np.array_equal(got[b], orc.rotate(ct[b], 91))
         want = orc.rotate_hoisted(ct[b], [91, 92])
         assert np.array_equal(hgot[0, b], want[0]) and np.array_equal(hgot[1, b], want[1])
+    # sums over several sources in one pass: rotate-and-add over 8 keys = 72 products per accumulator (the FP64 sums fold
+    # back after every 7th, the 128-bit sums on the special primes are reduced after every 8th)
+    kids = []
+    for i, r in enumerate([1, 2, 3, 4, -1, -2, -3, -4]):
+        add_key(pair, r, 93 + i) if r not in (1, 2) else None
+        kids.append({1: 91, 2: 92}.get(r, 93 + i))
+    sout = torch.empty_like(to_dev(ct))
+    ctx.rotate_sum_hoisted(to_dev(ct), sout, batch, level, kids)
+    sgot = to_host(sout)
+    for b in range(batch):
+        assert np.array_equal(sgot[b], orc.rotate_sum_hoisted(ct[b], kids))
