@@ -294,6 +294,13 @@ static inline int fesc_fail(fesc_ctx* ctx, int code, const std::string& msg) {
     return code;
 }
 
+// Galois automorphism X -> X^g in evaluation (bit-reversed) order: out[t] = in[galois_src(t)]
+__device__ __forceinline__ uint32_t galois_src(uint32_t t, uint32_t log_n, u64 g) {
+    uint32_t u = __brev(t) >> (32 - log_n);
+    uint32_t e = (uint32_t)(((2ull * u + 1) * g) & ((2ull << log_n) - 1));
+    return __brev((e - 1) >> 1) >> (32 - log_n);
+}
+
 // Optional epilogue of the last pass of a forward N = 2^16 transform over rows r = bp * level + i (bp = ciphertext * 2 +
 // polynomial, i = data limb, all primes below 2^50): instead of storing the transformed row u, the pass stores the last
 // step of an exact division,  out[b][p][i] = (acc[bp][i] - u) * c_i  (added to what out holds when bit p of add_mask
@@ -308,6 +315,11 @@ struct NttFinish {
     const double* cinv = nullptr;    // device array: c_i as doubles
     uint32_t level = 0, acc_rows = 0;
     int add_mask = 0;
+    // rotation: the first polynomial also receives sigma_g(c0) of the input ciphertext, read through the permutation here
+    // (instead of a kernel that writes the permuted c0 to `out` first and add_mask bit 0)
+    const u64* rot_src = nullptr;    // ciphertext b at rot_src + b * rot_stride, first polynomial [level][N]
+    size_t rot_stride = 0;
+    u64 rot_g = 0;
 };
 
 // internal launchers (ntt.cu)

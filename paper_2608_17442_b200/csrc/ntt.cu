@@ -364,7 +364,8 @@ template <bool INV>
 __device__ __forceinline__ void contig_body_fp(u64* __restrict__ p, double* __restrict__ sm, const double* __restrict__ tw,
                                                const PrimeConst& pc, uint32_t pre, int out_double,
                                                const u64* __restrict__ fin_acc = nullptr, u64* __restrict__ fin_out = nullptr,
-                                               double fin_pinv = 0.0, int fin_add = 0) {
+                                               double fin_pinv = 0.0, int fin_add = 0, const u64* __restrict__ fin_rot = nullptr,
+                                               u64 fin_g = 0, uint32_t fin_t0 = 0) {
     const double q = pc.qd, qinv = pc.qinvd;
     const uint32_t sub = threadIdx.x & 31;
     const uint32_t h2 = sub >> 2, l2 = sub & 3;
@@ -397,7 +398,10 @@ __device__ __forceinline__ void contig_body_fp(u64* __restrict__ p, double* __re
                 const ulonglong2 av = a[k];
                 double s0 = fp_modmul(fp_load(av.x, q) - x[2 * k], fin_pinv, q, qinv);
                 double s1 = fp_modmul(fp_load(av.y, q) - x[2 * k + 1], fin_pinv, q, qinv);
-                if (fin_add) {
+                if (fin_rot) {        // + sigma_g(c0): the row of the input read through the permutation
+                    s0 += fp_load(fin_rot[galois_src(fin_t0 + sub * 8 + 2 * k, 16, fin_g)], q);
+                    s1 += fp_load(fin_rot[galois_src(fin_t0 + sub * 8 + 2 * k + 1, 16, fin_g)], q);
+                } else if (fin_add) {
                     const ulonglong2 ov = o[k];
                     s0 += fp_load(ov.x, q);
                     s1 += fp_load(ov.y, q);
@@ -552,12 +556,15 @@ __global__ void __launch_bounds__(NTT_WARPS * 32) ntt16_contig(u64* __restrict__
             const uint32_t r = row_first + row, bp = r / fin.level, i = r - bp * fin.level;
             if (!DBG_REGION(fin.acc + (size_t)(bp >> 1) * fin.acc_stride + ((size_t)(bp & 1) * fin.acc_rows + i) * N16 + (size_t)blk * 256, 256 * sizeof(u64)) ||
                 !DBG_REGION(fin.out + (size_t)(bp >> 1) * fin.out_stride + ((size_t)(bp & 1) * fin.level + i) * N16 + (size_t)blk * 256,
-                            256 * sizeof(u64)))
+                            256 * sizeof(u64)) ||
+                (fin.rot_src && !DBG_REGION(fin.rot_src + (size_t)(bp >> 1) * fin.rot_stride + (size_t)i * N16, N16 * sizeof(u64))))
                 return;
             contig_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, 256 + blk, out_double,
                                 fin.acc + (size_t)(bp >> 1) * fin.acc_stride + ((size_t)(bp & 1) * fin.acc_rows + i) * N16 + (size_t)blk * 256,
                                 fin.out + (size_t)(bp >> 1) * fin.out_stride + ((size_t)(bp & 1) * fin.level + i) * N16 + (size_t)blk * 256,
-                                fin.cinv[i], (fin.add_mask >> (bp & 1)) & 1);
+                                fin.cinv[i], (fin.add_mask >> (bp & 1)) & 1,
+                                (fin.rot_src && !(bp & 1)) ? fin.rot_src + (size_t)(bp >> 1) * fin.rot_stride + (size_t)i * N16 : nullptr,
+                                fin.rot_g, blk * 256);
         } else {
             contig_body_fp<INV>(p, reinterpret_cast<double*>(sm), twf_all + (size_t)pi * N16, pc, 256 + blk, out_double);
         }

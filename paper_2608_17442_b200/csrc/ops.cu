@@ -73,11 +73,6 @@ extern "C" int fesc_intt(fesc_ctx* ctx, uint64_t* d_data, uint32_t batch, uint32
 // c0 goes to out0 (the result's first polynomial), c1 goes to BOTH d (kept in EVAL form for
 // the digit's own limbs) and dcoef (transformed in place afterwards).
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t galois_src(uint32_t t, uint32_t log_n, u64 g) {
-    uint32_t u = __brev(t) >> (32 - log_n);
-    uint32_t e = (uint32_t)(((2ull * u + 1) * g) & ((2ull << log_n) - 1));
-    return __brev((e - 1) >> 1) >> (32 - log_n);
-}
 // Where the EVAL-form polynomial being switched is kept: the rows of the extended-digit buffer that belong to a
 // digit's own limbs (row l of digit l / alpha), which the basis extension leaves untouched.  The inner product then
 // reads every (digit, row) from one array.
@@ -821,8 +816,16 @@ static int ks_inner(fesc_ctx* ctx, const KsScratch& ws, const EvalKey& key, uint
 }
 
 // Step 5: division of ws.acc by P; the result is ADDED to out[b][p] when bit p of add_mask is set, else stored.
+// whether the last pass of the forward transform finishes the division (N = 2^16, every data prime below 2^50)
+static bool moddown_fused(const fesc_ctx* ctx, uint32_t level) {
+    bool fuse = ctx->log_n == 16;
+    for (uint32_t i = 0; i < level; i++) fuse = fuse && ctx->q[i] < FESC_FP_LIMIT;
+    return fuse;
+}
+// rot_src != nullptr (only when moddown_fused): out[b][0] also receives sigma_g(c0) of the ciphertext at
+// rot_src + b * rot_stride, read through the permutation by the fused epilogue
 static int ks_moddown(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint32_t batch, u64* out, size_t out_stride,
-                      int add_mask, cudaStream_t st) {
+                      int add_mask, cudaStream_t st, const u64* rot_src = nullptr, size_t rot_stride = 0, u64 rot_g = 0) {
     const uint32_t N = ctx->N, K = ctx->n_p, nq = ctx->n_q;
     const uint32_t rows = level + K;
     const uint32_t gx = (N + 255) / 256;
@@ -841,12 +844,13 @@ static int ks_moddown(fesc_ctx* ctx, const KsScratch& ws, uint32_t level, uint32
     prof_end(ctx, PF_MODDOWN, st);
     m.period = level;
     for (uint32_t i = 0; i < level; i++) m.prime[i] = (uint8_t)i;
-    bool fuse = ctx->log_n == 16;          // the last pass of the transform finishes the division (FP64 rows only)
-    for (uint32_t i = 0; i < level; i++) fuse = fuse && ctx->q[i] < FESC_FP_LIMIT;
+    const bool fuse = moddown_fused(ctx, level);
+    if (rot_src && !fuse) return fesc_fail(ctx, FESC_EINVAL, "key switch: the permuted addend needs the fused division epilogue");
     if (fuse) {
         NttFinish fin;
         fin.acc = ws.acc, fin.acc_stride = (size_t)2 * rows * N, fin.out = out, fin.out_stride = out_stride, fin.cinv = ctx->tabs.d_moddown->pinvd;
         fin.level = level, fin.acc_rows = rows, fin.add_mask = add_mask;
+        fin.rot_src = rot_src, fin.rot_stride = rot_stride, fin.rot_g = rot_g;
         return ntt_launch(ctx, ws.u, (size_t)batch * 2 * level, m, false, st, true, false, &fin);
     }
     if ((rc = ntt_launch(ctx, ws.u, (size_t)batch * 2 * level, m, false, st, ctx->log_n == 16)) != FESC_OK) return rc;
@@ -1016,6 +1020,11 @@ int rotate_hoisted_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64*
         for (uint32_t k = 0; k < n_keys; k++) {
             const EvalKey& key = ctx->keys[key_ids[k]];
             u64* ob = out + (size_t)k * key_stride + (size_t)b0 * out_stride;
+            if (moddown_fused(ctx, level)) {     // sigma_g(c0) is added by the division's epilogue, straight from the input
+                if ((rc = ks_inner(ctx, ws, key, level, nb, st, key.g, 0)) != FESC_OK) return rc;
+                if ((rc = ks_moddown(ctx, ws, level, nb, ob, out_stride, 0, st, ib, in_stride, key.g)) != FESC_OK) return rc;
+                continue;
+            }
             prof_begin(ctx, PF_AUTOM, st);
             k_hoist_prepare<<<g, 256, 0, st>>>(ib, in_stride, ob, out_stride, OwnRows{nullptr, 1, 1, 1, 0}, nullptr, ctx->log_n, level, key.g, ctx->d_pc);
             prof_end(ctx, PF_AUTOM, st);
