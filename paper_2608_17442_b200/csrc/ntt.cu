@@ -401,7 +401,8 @@ __device__ __forceinline__ void contig_body_fp(u64* __restrict__ p, double* __re
                 if (fin_rot) {        // + sigma_g(c0): the row of the input read through the permutation
                     s0 += fp_load(fin_rot[galois_src(fin_t0 + sub * 8 + 2 * k, 16, fin_g)], q);
                     s1 += fp_load(fin_rot[galois_src(fin_t0 + sub * 8 + 2 * k + 1, 16, fin_g)], q);
-                } else if (fin_add) {
+                }
+                if (fin_add) {
                     const ulonglong2 ov = o[k];
                     s0 += fp_load(ov.x, q);
                     s1 += fp_load(ov.y, q);

@@ -99,14 +99,16 @@ __global__ void __launch_bounds__(256) k_autom_ct(const u64* __restrict__ in, si
     const uint32_t src = galois_src(t, log_n, g);
     const u64* ib = in + (size_t)b * in_stride;
     const size_t poly = (size_t)level * N;
-    u64* o0 = out0 + (size_t)b * out_stride + (size_t)l * N + t;
-    if (src >= N || !DBG_REGION(ib + (size_t)l * N, N * sizeof(u64)) || !DBG_REGION(ib + poly + (size_t)l * N, N * sizeof(u64)) ||
-        !DBG_REGION(o0 - t, N * sizeof(u64)) || !DBG_REGION(d.ext + own_index(d, b, l, N), N * sizeof(u64)) ||
-        !DBG_REGION(dcoef + ((size_t)b * level + l) * N, N * sizeof(u64)))
+    if (src >= N || !DBG_REGION(ib + poly + (size_t)l * N, N * sizeof(u64)) ||
+        !DBG_REGION(d.ext + own_index(d, b, l, N), N * sizeof(u64)) || !DBG_REGION(dcoef + ((size_t)b * level + l) * N, N * sizeof(u64)))
         return;
-    u64 v0 = ib[(size_t)l * N + src];
-    if (accumulate) v0 = addmod(v0, *o0, pcs[l].q);
-    *o0 = v0;
+    if (out0) {        // nullptr: sigma_g(c0) is added later by the division's epilogue
+        u64* o0 = out0 + (size_t)b * out_stride + (size_t)l * N + t;
+        if (!DBG_REGION(ib + (size_t)l * N, N * sizeof(u64)) || !DBG_REGION(o0 - t, N * sizeof(u64))) return;
+        u64 v0 = ib[(size_t)l * N + src];
+        if (accumulate) v0 = addmod(v0, *o0, pcs[l].q);
+        *o0 = v0;
+    }
     u64 v = ib[poly + (size_t)l * N + src];
     d.ext[own_index(d, b, l, N) + t] = own_word(d, v, pcs[l]);
     dcoef[((size_t)b * level + l) * N + t] = v;
@@ -918,12 +920,21 @@ int rotate_internal(fesc_ctx* ctx, const u64* in, size_t in_stride, u64* out, si
     for (uint32_t b0 = 0; b0 < batch; b0 += chunk) {
         uint32_t nb = batch - b0 < chunk ? batch - b0 : chunk;
         dim3 g((ctx->N + 255) / 256, level, nb);
+        const bool fused = moddown_fused(ctx, level);   // then the division's epilogue adds sigma_g(c0) straight from the input
         prof_begin(ctx, PF_AUTOM, st);
-        k_autom_ct<<<g, 256, 0, st>>>(in + (size_t)b0 * in_stride, in_stride, out + (size_t)b0 * out_stride, out_stride,
+        k_autom_ct<<<g, 256, 0, st>>>(in + (size_t)b0 * in_stride, in_stride, fused ? nullptr : out + (size_t)b0 * out_stride, out_stride,
                                       own_rows(ctx, ws, level), ws.dcoef, ctx->log_n, level, it->second.g, ctx->d_pc, accumulate);
         prof_end(ctx, PF_AUTOM, st);
-        int rc = key_switch_chunk(ctx, ws, it->second, level, nb, out + (size_t)b0 * out_stride, out_stride,
+        int rc;
+        if (fused) {
+            if ((rc = ks_decompose(ctx, ws, level, nb, st)) != FESC_OK) return rc;
+            if ((rc = ks_inner(ctx, ws, it->second, level, nb, st, 0, 0)) != FESC_OK) return rc;
+            rc = ks_moddown(ctx, ws, level, nb, out + (size_t)b0 * out_stride, out_stride, accumulate ? 3 : 0, st,
+                            in + (size_t)b0 * in_stride, in_stride, it->second.g);
+        } else {
+            rc = key_switch_chunk(ctx, ws, it->second, level, nb, out + (size_t)b0 * out_stride, out_stride,
                                   accumulate ? 3 : 1, st);
+        }
         if (rc != FESC_OK) return rc;
     }
     return FESC_OK;
