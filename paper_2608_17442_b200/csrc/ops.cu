@@ -102,6 +102,7 @@ __global__ void __launch_bounds__(256) k_autom_ct(const u64* __restrict__ in, si
     if (src >= N || !DBG_REGION(ib + poly + (size_t)l * N, N * sizeof(u64)) ||
         !DBG_REGION(d.ext + own_index(d, b, l, N), N * sizeof(u64)) || !DBG_REGION(dcoef + ((size_t)b * level + l) * N, N * sizeof(u64)))
         return;
+    const u64 v = ib[poly + (size_t)l * N + src];       // requested before the c0 part so that both gathers are in flight together
     if (out0) {        // nullptr: sigma_g(c0) is added later by the division's epilogue
         u64* o0 = out0 + (size_t)b * out_stride + (size_t)l * N + t;
         if (!DBG_REGION(ib + (size_t)l * N, N * sizeof(u64)) || !DBG_REGION(o0 - t, N * sizeof(u64))) return;
@@ -109,7 +110,6 @@ __global__ void __launch_bounds__(256) k_autom_ct(const u64* __restrict__ in, si
         if (accumulate) v0 = addmod(v0, *o0, pcs[l].q);
         *o0 = v0;
     }
-    u64 v = ib[poly + (size_t)l * N + src];
     d.ext[own_index(d, b, l, N) + t] = own_word(d, v, pcs[l]);
     dcoef[((size_t)b * level + l) * N + t] = v;
 }
