@@ -1121,7 +1121,7 @@ extern "C" int fesc_rotate_sum_hoisted(fesc_ctx* ctx, const uint64_t* d_in, uint
 
 extern "C" int fesc_rotate_hoisted(fesc_ctx* ctx, const uint64_t* d_in, uint64_t* d_out, uint32_t batch,
                                    uint32_t n_limbs, const uint32_t* key_ids, uint32_t n_keys, void* stream) {
-    if (!ctx || !d_in || !d_out || (!key_ids && n_keys)) return FESC_EINVAL;
+    if (!ctx || !d_in || !d_out || (!key_ids && n_keys) || d_in == d_out) return FESC_EINVAL;
     if (n_limbs == 0 || n_limbs > ctx->n_q) return fesc_fail(ctx, FESC_ELEVEL, "rotate_hoisted: level out of range");
     if (batch == 0 || n_keys == 0) return FESC_OK;
     u64* scratch;
@@ -1134,7 +1134,7 @@ extern "C" int fesc_rotate_hoisted(fesc_ctx* ctx, const uint64_t* d_in, uint64_t
 
 extern "C" int fesc_rotate(fesc_ctx* ctx, const uint64_t* d_in, uint64_t* d_out, uint32_t batch, uint32_t n_limbs,
                            uint32_t key_id, void* stream) {
-    if (!ctx || !d_in || !d_out) return FESC_EINVAL;
+    if (!ctx || !d_in || !d_out || d_in == d_out) return FESC_EINVAL;      // the input is read while the output is written
     if (n_limbs == 0 || n_limbs > ctx->n_q) return fesc_fail(ctx, FESC_ELEVEL, "rotate: level out of range");
     if (batch == 0) return FESC_OK;
     u64* scratch;
