@@ -585,3 +585,21 @@ def test_inner_product_worst_case_residues_with_many_digits():
     sgot = to_host(sout)
     for b in range(batch):
         assert np.array_equal(sgot[b], orc.rotate_sum_hoisted(ct[b], kids))
+
+
+def test_rotations_refuse_an_output_at_the_inputs_address():
+    """fesc_rotate and fesc_rotate_hoisted read the input while they write the output: the same buffer for both is
+    refused (FESC_EINVAL) before anything is launched."""
+    import torch
+    import paper_2608_17442_b200 as fesc
+
+    pair = ctx_pair("small")
+    ctx, orc, _ = pair
+    add_key(pair, 3, 81)
+    ct = to_dev(random_ct(orc, 77, 4, 4, 2))
+    launches = ctx.counters()[4]
+    for call in (lambda: ctx.rotate(ct, ct, 2, 4, 81), lambda: ctx.rotate_hoisted(ct, ct, 2, 4, [81])):
+        with pytest.raises(fesc.FescError) as e:
+            call()
+        assert e.value.code == fesc.EINVAL
+    assert ctx.counters()[4] == launches
